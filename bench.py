@@ -1,0 +1,486 @@
+#!/usr/bin/env python
+"""Benchmark of the KV-Direct hot path on one B200 (or N independent replicas).
+
+One *step* is one pass of the whole per-layer hot path over one batch of synthetic input, on a
+single decoder layer shaped like Gemma-3-4B (hidden 2560, 8 query / 4 KV heads, head_dim 256,
+key norm, RoPE base 1e6) with T = 4096 checkpointed tokens:
+
+    kvd_checkpoint_residual (T rows)           STORE_RESIDUAL of Algorithm 1
+    kvd_recompute_kv        (T rows from store) Eq. 13-14: RMSNorm -> [W_K|W_V] GEMM -> key norm -> RoPE
+    kvd_recompute_kv        (1 row)             K_t, V_t of the current token
+    kvd_decode_attention    (T + 1 keys)        Eq. 6-7, query at position T
+
+The JSON line printed by rank 0 follows the repository's bench contract; `value` is recomputed-KV
+tokens per second over whole steps with inputs resident in HBM, `e2e` the same with host buffers and
+the copies timed, `roofline` describes the recompute GEMM against the measured dense-bf16 peak,
+`roofline_attention` the decode attention against the measured HBM copy bandwidth, `cached_read`
+the thing KV-Direct replaces (attention over a stored cache, and a plain device copy of it), and
+`cpu_baseline` the fp64 oracle timed on the host cores on a bounded sample.
+
+`--impl reference` times the CPU oracle alone (there is no other reference implementation of the
+paper's method to run).  `--sweep` adds the recompute-vs-read table over T = 256 .. 32768.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "recomputed_kv_tokens_per_s"
+UNIT = "tokens/s"
+T_TOKENS = 4096
+N_SETS = 16  # rotating buffer sets: 16 x (21 MB residual rows + 21 MB store + 16.8 MB K/V) >> 126 MB of L2
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------- clocks sampler
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(0.005)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle timing
+class OracleTimer:
+    """Times the fp64 oracle (as it stands) on a bounded sample of one step's work."""
+
+    def __init__(self, shape, T):
+        import oracle
+        from kvd_synth import bf16_to_f64, make_kv, make_layer_weights, make_query, make_residuals
+        self.oracle, self.shape, self.T = oracle, shape, T
+        w = make_layer_weights(shape)
+        self.args = (bf16_to_f64(w.gamma_in), bf16_to_f64(w.w_kv), shape.n_kv_heads, shape.d_head, shape.rms_eps,
+                     shape.rope_theta, bf16_to_f64(w.gamma_k) if w.gamma_k is not None else None, shape.rms_eps)
+        self.cores = oracle.max_threads()
+        self.X = bf16_to_f64(make_residuals(shape, T, seed=99, outliers=True))
+        K, V = make_kv(shape, T + 1, seed=99)
+        self.Kf, self.Vf = bf16_to_f64(K), bf16_to_f64(V)
+        self.q = bf16_to_f64(make_query(shape, 1, seed=99))[0]
+        t0 = time.perf_counter()
+        self._recompute(16)
+        self.s_per_row = (time.perf_counter() - t0) / 16  # calibration only
+
+    def _recompute(self, rows):
+        self.oracle.recompute_kv(self.X[:rows], np.arange(rows, dtype=np.int32), *self.args)
+
+    def step(self, budget_s):
+        """One bounded sample: recompute_kv on as many rows as fit the budget (16..T), then the
+        attention over all T + 1 keys; the row part is scaled linearly to T rows (rows are independent)."""
+        T = self.T
+        rows = int(min(self.X.shape[0], max(16, budget_s * 0.8 / max(self.s_per_row, 1e-6)))) // 16 * 16
+        t0 = time.perf_counter()
+        self._recompute(rows)
+        t_rec = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        self.oracle.decode_attention(self.q, T, [(self.Kf, self.Vf, 0)], 1.0 / math.sqrt(self.shape.d_head), 0)
+        t_att = time.perf_counter() - t0
+        step_s = t_rec * T / rows + t_att
+        return {"value": T / step_s, "unit": UNIT, "cores": self.cores, "kind": "oracle",
+                "sample": f"recompute_kv on {rows} of {T} rows ({t_rec:.2f} s, scaled linearly to {T} rows) + "
+                          f"decode_attention over all {T + 1} keys ({t_att * 1e3:.1f} ms)"}
+
+
+def run_reference(args):
+    from kvd_synth import GEMMA3_4B_GLOBAL
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    timer = OracleTimer(GEMMA3_4B_GLOBAL, T_TOKENS)
+    budget = min(4.0, max(0.05, 150.0 / max(args.steps + args.warmup, 1)))
+    for _ in range(args.warmup):
+        timer.step(budget)
+    vals, base = [], None
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        base = timer.step(budget)
+        vals.append(base["value"])
+    wall = time.perf_counter() - t0
+    v = float(np.mean(vals))
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * wall / max(args.steps, 1), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "gemma3-4b layer (d=2560, 8q/4kv heads, d_head=256, key norm, theta=1e6), "
+                                   "T=4096 checkpointed tokens, batch 1 (config 2)",
+                       "note": "each step times the fp64 CPU oracle on a bounded sample and scales linearly to T rows"},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": base["cores"], "kind": "oracle", "sample": base["sample"]},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- GPU arm
+class Workload:
+    """Device buffers and the step function for the Gemma-3-4B-shaped layer."""
+
+    def __init__(self, shape, T, n_sets):
+        import torch
+        import paper_2603_19664_b200 as kvd
+        from kvd_synth import make_layer_weights, make_query, make_residuals
+        self.torch, self.kvd, self.shape, self.T, self.n_sets = torch, kvd, shape, T, n_sets
+        self.kdim = shape.n_kv_heads * shape.d_head
+
+        def dev(bits):
+            return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+        w = make_layer_weights(shape)
+        self.desc = kvd.make_desc(1, shape.d_hidden, shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.rms_eps,
+                                  shape.qk_norm, shape.rms_eps, shape.rope_style, n_sets, T + 8, 1)
+        self.ctx = kvd.Kvd(self.desc)
+        self.w_kv, self.g_in = dev(w.w_kv), dev(w.gamma_in)
+        self.g_k = dev(w.gamma_k) if w.gamma_k is not None else None
+        self.ctx.kvd_set_layer(0, self.w_kv, self.g_in, self.g_k, shape.rope_theta, shape.sliding_window)
+        self.ws = torch.empty(kvd.kvd_workspace_bytes(self.desc), dtype=torch.uint8, device="cuda")
+        self.ctx.kvd_attach_workspace(self.ws)
+        self.arena = torch.empty(kvd.kvd_store_bytes(self.desc, 1), dtype=torch.uint8, device="cuda")
+        self.ctx.kvd_attach_store(self.arena, 1)
+        x_bits = make_residuals(shape, T + 1, seed=2, outliers=True)
+        self.x_host_bits = x_bits
+        x0 = dev(x_bits)
+        # distinct memory per set, same distribution: rows rotated by a set-dependent offset
+        self.X = [x0 if i == 0 else torch.roll(x0, shifts=97 * i, dims=0).contiguous() for i in range(n_sets)]
+        self.pos = torch.arange(T + 1, dtype=torch.int32, device="cuda")
+        self.K = [torch.empty((T + 1, self.kdim), dtype=torch.bfloat16, device="cuda") for _ in range(n_sets)]
+        self.V = [torch.empty((T + 1, self.kdim), dtype=torch.bfloat16, device="cuda") for _ in range(n_sets)]
+        self.q = dev(make_query(shape, n_sets, seed=2))  # one query per set
+        self.out = torch.empty((n_sets, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda")
+        self.ev = None
+
+    def step(self, i, events=None):
+        """One pass of the hot path on buffer set i % n_sets.  `events` (optional): 4 CUDA events
+        recorded around checkpoint / recompute / attention."""
+        s, T, c = i % self.n_sets, self.T, self.ctx
+        X, K, V = self.X[s], self.K[s], self.V[s]
+        c.kvd_reset_sequence(s)
+        if events:
+            events[0].record()
+        c.kvd_checkpoint_residual(s, 0, X, self.pos, T)
+        if events:
+            events[1].record()
+        c.kvd_recompute_kv(0, None, None, T, K, V, self.kdim, seq=s, first_row=0)
+        if events:
+            events[2].record()
+        c.kvd_recompute_kv(0, X[T:], self.pos[T:], 1, K[T:], V[T:], self.kdim)
+        if events:
+            events[3].record()
+        c.kvd_decode_attention(0, 1, self.q[s:s + 1], [T],
+                               [[(K, V, self.kdim, 0, T), (K[T:], V[T:], self.kdim, T, 1)]], 0.0, self.out[s:s + 1])
+        if events:
+            events[4].record()
+
+    def cached_read_step(self, i):
+        """What KV-Direct replaces: attention over the stored cache of T + 1 keys in one segment."""
+        s, T = i % self.n_sets, self.T
+        self.ctx.kvd_decode_attention(0, 1, self.q[s:s + 1], [T], [[(self.K[s], self.V[s], self.kdim, 0, T + 1)]],
+                                      0.0, self.out[s:s + 1])
+
+
+def run_gpu(args):
+    import torch
+    from kvd_synth import GEMMA3_4B_GLOBAL
+    import paper_2603_19664_b200 as kvd
+    from paper_2603_19664_b200.build import build
+    build()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist = dist_mod
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    shape, T = GEMMA3_4B_GLOBAL, T_TOKENS
+    peaks = load_peaks()
+    wl = Workload(shape, T, N_SETS)
+    steps, warmup = args.steps, max(args.warmup, 3)
+
+    # ---- warm-up
+    for i in range(warmup):
+        wl.step(i)
+    barrier()
+    assert wl.ctx.kvd_poll_status() == kvd.KVD_OK
+
+    # ---- timed region: exactly `steps` steps, whole-region CUDA events + per-kernel events
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = wl.ctx.kvd_launch_count()
+    barrier()
+    with ClockSampler(local) as clocks:
+        start.record()
+        for i in range(steps):
+            wl.step(warmup + i, ev[i])
+        stop.record()
+        barrier()
+    launches = wl.ctx.kvd_launch_count() - launches0
+    total_ms = start.elapsed_time(stop)
+    status = wl.ctx.kvd_poll_status()
+    if status != kvd.KVD_OK:
+        raise RuntimeError(f"device status after the timed region: {kvd.status_string(status)}")
+    t_ckpt = np.array([e[0].elapsed_time(e[1]) for e in ev])
+    t_gemm = np.array([e[1].elapsed_time(e[2]) for e in ev])
+    t_kt = np.array([e[2].elapsed_time(e[3]) for e in ev])
+    t_attn = np.array([e[3].elapsed_time(e[4]) for e in ev])
+    if dist is not None:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / steps
+    value = world * T / (ms_per_step * 1e-3)
+
+    # ---- the read that recomputation replaces (separate loops, same rotation)
+    def timed(fn, n):
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(n):
+            fn(3 + i)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    n_aux = min(max(steps, 20), 200)
+    read_attn_ms = timed(wl.cached_read_step, n_aux)
+    kv_copy_dst = torch.empty((2, T + 1, wl.kdim), dtype=torch.bfloat16, device="cuda")
+
+    def copy_step(i):
+        s = i % wl.n_sets
+        kv_copy_dst[0].copy_(wl.K[s])
+        kv_copy_dst[1].copy_(wl.V[s])
+
+    read_copy_ms = timed(copy_step, n_aux)
+
+    # ---- end to end through the C ABI with host buffers
+    x_pin = torch.from_numpy(wl.x_host_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    pos_pin = torch.arange(T + 1, dtype=torch.int32).pin_memory()
+    q_pin = wl.q[:1].cpu().pin_memory()
+    out_pin = torch.empty((1, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16).pin_memory()
+    x_dev = [torch.empty_like(wl.X[0]) for _ in range(2)]
+    pos_dev = torch.empty_like(wl.pos)
+    q_dev = torch.empty_like(wl.q[:1])
+    out_dev = torch.empty_like(wl.out[:1])
+
+    def e2e_step(i):
+        s = i % wl.n_sets
+        xd = x_dev[i % 2]
+        xd.copy_(x_pin, non_blocking=True)
+        pos_dev.copy_(pos_pin, non_blocking=True)
+        q_dev.copy_(q_pin, non_blocking=True)
+        c = wl.ctx
+        c.kvd_reset_sequence(s)
+        c.kvd_checkpoint_residual(s, 0, xd, pos_dev, T)
+        c.kvd_recompute_kv(0, None, None, T, wl.K[s], wl.V[s], wl.kdim, seq=s, first_row=0)
+        c.kvd_recompute_kv(0, xd[T:], pos_dev[T:], 1, wl.K[s][T:], wl.V[s][T:], wl.kdim)
+        c.kvd_decode_attention(0, 1, q_dev, [T], [[(wl.K[s], wl.V[s], wl.kdim, 0, T), (wl.K[s][T:], wl.V[s][T:], wl.kdim, T, 1)]],
+                               0.0, out_dev)
+        out_pin.copy_(out_dev, non_blocking=True)
+        torch.cuda.current_stream().synchronize()  # the caller reads the result of every step
+
+    n_e2e = min(max(steps, 10), 100)
+    e2e_ms = timed(e2e_step, n_e2e)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = x_pin.numel() * 2 + pos_pin.numel() * 4 + q_pin.numel() * 2
+    d2h = out_pin.numel() * 2
+
+    sweep = run_sweep(wl, peaks) if args.sweep and rank == 0 else None
+
+    if rank == 0:
+        flops = 4.0 * T * shape.n_kv_heads * shape.d_hidden * shape.d_head  # Eq. 26
+        gemm_ms = float(np.mean(t_gemm))
+        attn_ms = float(np.mean(t_attn))
+        attn_bytes = (T + 1) * 4 * shape.n_kv_heads * shape.d_head  # Eq. 27 for T + 1 keys
+        cpu = OracleTimer(shape, T).step(12.0)
+        clk = clocks.summary()
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "gemma3-4b layer (d=2560, 8q/4kv heads, d_head=256, key norm, theta=1e6), "
+                                   "T=4096 checkpointed tokens, batch 1 (config 2)",
+                       "step": "checkpoint T rows -> recompute K/V of T rows from the store -> K_t,V_t -> "
+                               "decode attention over T+1 keys",
+                       "l2": f"inputs rotate over {N_SETS} buffer sets (~{N_SETS * 59} MB), larger than L2",
+                       "replicas": "independent replicas per GPU, no collective" if world > 1 else "single GPU"},
+            "clocks": clk,
+            "e2e": {"value": world * T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+            "gpu_launches": int(launches),
+            "roofline": {"kernel": "kvd_recompute_kernel<256,256>", "bound": "tensor",
+                         "achieved": flops / (gemm_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                         "frac": flops / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "traffic": None,
+                         "peak_source": peaks["source"] + " burst", "avg_launch_us": gemm_ms * 1e3,
+                         "min_launch_us": float(np.min(t_gemm)) * 1e3,
+                         "frac_of_sustained": flops / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]},
+            "roofline_attention": {"kernel": "kvd_attn_split_kernel<256,2> + merge", "bound": "hbm",
+                                   "achieved": attn_bytes / (attn_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                                   "unit": "GB/s", "frac": attn_bytes / (attn_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                   "traffic": None, "avg_us": attn_ms * 1e3, "min_us": float(np.min(t_attn)) * 1e3},
+            "decode_step_us": {"checkpoint": float(np.mean(t_ckpt)) * 1e3, "recompute": gemm_ms * 1e3,
+                               "current_token_kv": float(np.mean(t_kt)) * 1e3, "attention": attn_ms * 1e3,
+                               "total": ms_per_step * 1e3},
+            "cached_read": {"attention_over_stored_cache_us": read_attn_ms * 1e3,
+                            "attention_gbs": attn_bytes / (read_attn_ms * 1e-3) / 1e9,
+                            "device_copy_us": read_copy_ms * 1e3,
+                            "device_copy_gbs": 2 * attn_bytes / (read_copy_ms * 1e-3) / 1e9,
+                            "recompute_over_read_ratio": gemm_ms / read_copy_ms},
+            "cpu_baseline": {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        }
+        if sweep is not None:
+            line["sweep"] = sweep
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_sweep(wl, peaks):
+    """Recompute-vs-read over T (the paper's Section 5.8 measurement, on this hardware)."""
+    import torch
+    rows = []
+    shape, kdim = wl.shape, wl.kdim
+    big_T = 32768
+    from kvd_synth import make_layer_weights  # noqa: F401
+    import paper_2603_19664_b200 as kvd
+    desc = kvd.make_desc(1, shape.d_hidden, shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.rms_eps,
+                         shape.qk_norm, shape.rms_eps, shape.rope_style, 1, big_T + 8, 1)
+    ctx = kvd.Kvd(desc)
+    ctx.kvd_set_layer(0, wl.w_kv, wl.g_in, wl.g_k, shape.rope_theta, 0)
+    ws = torch.empty(kvd.kvd_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_workspace(ws)
+    n_sets = 5
+    X = [torch.randn((big_T, shape.d_hidden), device="cuda", dtype=torch.float32).to(torch.bfloat16) for _ in range(n_sets)]
+    K = [torch.randn((big_T + 1, kdim), device="cuda", dtype=torch.float32).to(torch.bfloat16) for _ in range(n_sets)]
+    V = [torch.randn((big_T + 1, kdim), device="cuda", dtype=torch.float32).to(torch.bfloat16) for _ in range(n_sets)]
+    Ko = torch.empty((big_T, kdim), device="cuda", dtype=torch.bfloat16)
+    Vo = torch.empty_like(Ko)
+    dst = torch.empty((2, big_T, kdim), device="cuda", dtype=torch.bfloat16)
+    pos = torch.arange(big_T, dtype=torch.int32, device="cuda")
+    q = wl.q[:1]
+    out = wl.out[:1]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def timed(fn, n=20):
+        ts = []
+        for i in range(n + 3):
+            flush.zero_()  # evict L2 between iterations (the small T cases fit in it)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn(i)
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b))
+        return float(np.median(ts))
+
+    for T in (1, 10, 50, 100, 256, 500, 512, 1024, 2048, 4096, 8192, 16384, 32768):
+        rec = timed(lambda i: ctx.kvd_recompute_kv(0, X[i % n_sets], pos, T, Ko, Vo, kdim))
+        att = timed(lambda i: ctx.kvd_decode_attention(0, 1, q, [T], [[(K[i % n_sets], V[i % n_sets], kdim, 0, T + 1)]], 0.0, out))
+
+        def cp(i):
+            dst[0, :T].copy_(K[i % n_sets][:T])
+            dst[1, :T].copy_(V[i % n_sets][:T])
+
+        cpy = timed(cp)
+        flops = 4.0 * T * shape.n_kv_heads * shape.d_hidden * shape.d_head
+        byts = T * 4 * shape.n_kv_heads * shape.d_head
+        rows.append({"T": T, "recompute_us": rec * 1e3, "recompute_tflops": flops / (rec * 1e-3) / 1e12,
+                     "attention_us": att * 1e3, "attention_gbs": byts / (att * 1e-3) / 1e9,
+                     "copy_us": cpy * 1e3, "ratio_recompute_over_copy": rec / cpy})
+    ctx.close()
+    return rows
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="kvd", choices=["kvd", "reference"])
+    ap.add_argument("--sweep", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

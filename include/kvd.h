@@ -1,0 +1,204 @@
+/*
+ * kvd.h -- C ABI of the KV-Direct hot path for NVIDIA B200 (sm_100a).
+ *
+ * KV-Direct keeps, for every token, the residual row that entered each decoder layer instead of
+ * the layer's key/value pair, and rebuilds keys and values when attention needs them
+ * (paper Section 3.4, Algorithm 1; reconstruction identities Eq. 13-14).  This library is the
+ * per-layer hot path of that scheme:
+ *
+ *   kvd_checkpoint_residual  STORE_RESIDUAL(C, l) of Algorithm 1: append residual rows to the store.
+ *   kvd_recompute_kv         RECOMPUTE_KV(C, l): RMSNorm (Eq. 1-2) -> fused [W_K | W_V] projection
+ *                            (Eq. 13-14) -> optional per-head key norm -> rotation of the keys at each
+ *                            row's stored position (Eq. 11-12).  The same call produces the current
+ *                            token's (K_t, V_t), so "first pass" and "recomputed" K/V are the output
+ *                            of one routine and are bit-identical for the same row and position.
+ *   kvd_decode_attention     ATTENTION(Q, K_all, V_all) for one query token per sequence (Eq. 6-7)
+ *                            over the CONCAT of up to four position-contiguous K/V segments
+ *                            (recomputed, live window, current token), grouped-query heads,
+ *                            optional sliding-window mask.
+ *
+ * General rules
+ *   - Plain C.  Every pointer documented as DEVICE points to memory on the context's GPU that the
+ *     caller allocated and keeps alive until the work enqueued on `stream` has finished; the
+ *     library never frees or reallocates it.  HOST pointers are read before the call returns.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All kernels
+ *     are enqueued asynchronously on it; no call synchronises the device except kvd_create,
+ *     kvd_set_layer (one-time preparation), kvd_poll_status and kvd_destroy.
+ *   - Every call returns a kvd_status and never throws, aborts or traps the device.  Argument
+ *     errors are detected on the host before anything is launched.  Conditions that only the
+ *     device can see (a position outside [0, max_tokens_per_seq), a pipeline wait that ran out)
+ *     are recorded in a device status word that kvd_poll_status reads.
+ *   - bf16 everywhere a tensor is stored; fp32 accumulation and fp32 epilogue arithmetic.
+ *   - There is no CPU fallback: without a CUDA device of compute capability 10.x kvd_create fails.
+ */
+#ifndef KVD_H_
+#define KVD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kvd_ctx kvd_ctx; /* opaque; one per model per device */
+
+typedef enum {
+  KVD_OK = 0,
+  KVD_ERR_INVALID_ARG = 1, /* NULL pointer, negative size, index out of range            */
+  KVD_ERR_SHAPE = 2,       /* dimensions the kernels do not cover                          */
+  KVD_ERR_ALIGNMENT = 3,   /* a pointer or stride is not 16-byte aligned                   */
+  KVD_ERR_CAPACITY = 4,    /* store, workspace or batch limit exceeded                     */
+  KVD_ERR_STATE = 5,       /* call made before its prerequisite (layer not set, ...)       */
+  KVD_ERR_UNSUPPORTED = 6, /* no usable device / driver entry point                        */
+  KVD_ERR_CUDA = 7,        /* a CUDA runtime call failed; see kvd_last_cuda_error          */
+  KVD_ERR_TIMEOUT = 8,     /* a bounded wait inside a kernel expired (from kvd_poll_status) */
+  KVD_ERR_POSITION = 9     /* a row's position was outside [0, max_tokens_per_seq)         */
+} kvd_status;
+
+/* Pairing of channels rotated together by Eq. 11-12. */
+typedef enum {
+  KVD_ROPE_INTERLEAVED = 0, /* (2i, 2i+1): the pairing Eq. 11-12 print            */
+  KVD_ROPE_HALF = 1         /* (i, i + d_head/2): the same rotation after a fixed
+                               channel permutation of q and k                      */
+} kvd_rope_style;
+
+/* Model-wide constants.  Supported: d_hidden % 64 == 0; d_head in {64, 128, 256};
+ * n_q_heads % n_kv_heads == 0 with a group size of 1..8; 2*n_kv_heads*d_head % 128 == 0. */
+typedef struct {
+  int32_t n_layers;
+  int32_t d_hidden;
+  int32_t n_q_heads;
+  int32_t n_kv_heads;
+  int32_t d_head;
+  float rms_eps;              /* added to mean(x^2) inside the root of Eq. 2 (the paper prints none) */
+  int32_t qk_norm;            /* 1: RMS-normalise every key head over d_head before the rotation      */
+  float qk_norm_eps;
+  int32_t rope_style;         /* kvd_rope_style                                                         */
+  int32_t max_seqs;           /* sequences the residual store can hold                                  */
+  int32_t max_tokens_per_seq; /* rows per (layer, sequence) in the store; also the position bound       */
+  int32_t max_batch;          /* largest `batch` of kvd_decode_attention (sizes the workspace)          */
+} kvd_model_desc;
+
+/* One layer's frozen parameters (all DEVICE, bf16, read during kvd_set_layer only). */
+typedef struct {
+  const void *w_kv;       /* [d_hidden, 2*n_kv*d_head] row-major: W_K columns (head-major) then W_V columns */
+  const void *gamma_in;   /* [d_hidden] effective RMSNorm scale gamma of Eq. 1                               */
+  const void *gamma_k;    /* [d_head] key-norm scale shared by all heads; NULL when qk_norm == 0             */
+  float rope_theta;       /* base b of Eq. 11-12                                                             */
+  int32_t sliding_window; /* 0: global layer.  w > 0: a key is visible iff 0 <= q_pos - key_pos < w          */
+} kvd_layer_desc;
+
+/* A run of keys/values at consecutive positions first_pos .. first_pos+len-1 (DEVICE, bf16).
+ * Element (j, h, c) of k is at k[j*row_stride + h*d_head + c]; likewise v.  row_stride is in
+ * elements and a multiple of 8; k and v are 16-byte aligned.  Segments of one sequence must not
+ * overlap in position. */
+typedef struct {
+  const void *k;
+  const void *v;
+  int64_t row_stride;
+  int32_t first_pos;
+  int32_t len;
+} kvd_kv_segment;
+
+#define KVD_MAX_SEGMENTS 4
+
+/* Byte counts reported by kvd_memory_stats.  The eq* fields are the paper's closed forms for the
+ * numbers of tokens currently stored; the others are what this context actually occupies. */
+typedef struct {
+  uint64_t checkpoint_bytes_used;     /* residual rows + positions currently held in the store           */
+  uint64_t checkpoint_bytes_capacity; /* size the attached arena must have                                */
+  uint64_t workspace_bytes;           /* attention scratch (split partials)                               */
+  uint64_t prepared_weight_bytes;     /* gamma-folded K-major copies of W_kv, rotation tables, key scales */
+  uint64_t tokens_stored;             /* max over layers of the rows stored, summed over sequences        */
+  uint64_t eq23_kv_bytes_per_token;   /* 2 L n_kv d_head b                                                */
+  uint64_t eq24_residual_bytes_per_token; /* d_hidden b (one vector per token, the paper's accounting)    */
+  uint64_t per_layer_residual_bytes_per_token; /* L d_hidden b (what per-layer recomputation stores)      */
+} kvd_mem_stats;
+
+/* Create a context on the current CUDA device.  HOST desc.  Fails with KVD_ERR_UNSUPPORTED when the
+ * device is not compute capability 10.x, KVD_ERR_SHAPE for dimensions outside the supported set. */
+kvd_status kvd_create(const kvd_model_desc *desc, kvd_ctx **out);
+
+/* Release everything the context allocated (prepared weights, tables).  Synchronises the device. */
+void kvd_destroy(kvd_ctx *ctx);
+
+/* Prepare layer `layer`: build W' = diag(gamma_in) * W_kv rounded to bf16 and stored K-major, the
+ * fp32 key-norm scale, and the rotation tables for rope_theta.  Folding gamma into W is Eq. 1
+ * composed with Eq. 13-14: (x / rms * gamma) W = (x W') / rms.  Enqueues on `stream` and waits for it. */
+kvd_status kvd_set_layer(kvd_ctx *ctx, int layer, const kvd_layer_desc *ldesc, void *stream);
+
+/* Bytes the residual store needs for `layers_stored` layers (rows + positions). */
+size_t kvd_store_bytes(const kvd_model_desc *desc, int layers_stored);
+
+/* Hand the context a caller-owned DEVICE arena (256-byte aligned, >= kvd_store_bytes) for the
+ * residual store C of Algorithm 1.  Resets all row counts to zero. */
+kvd_status kvd_attach_store(kvd_ctx *ctx, void *arena, size_t bytes, int layers_stored);
+
+/* Forget the rows of one sequence (all layers) so that its slot can be reused. */
+kvd_status kvd_reset_sequence(kvd_ctx *ctx, int seq);
+
+/* Rows currently stored for (layer, seq); negative on bad arguments. */
+int kvd_rows_stored(const kvd_ctx *ctx, int layer, int seq);
+
+/* Bytes of attention scratch for the context's max_batch / max_tokens_per_seq. */
+size_t kvd_workspace_bytes(const kvd_model_desc *desc);
+
+/* Hand the context a caller-owned DEVICE workspace (256-byte aligned, >= kvd_workspace_bytes). */
+kvd_status kvd_attach_workspace(kvd_ctx *ctx, void *workspace, size_t bytes);
+
+/* STORE_RESIDUAL(C, l): append n residual rows (DEVICE bf16 [n, d_hidden], 16-byte aligned) and
+ * their absolute positions (DEVICE int32 [n]) to the store of (layer, seq).
+ * KVD_ERR_CAPACITY when the rows do not fit; KVD_ERR_STATE without an attached store. */
+kvd_status kvd_checkpoint_residual(kvd_ctx *ctx, int seq, int layer, const void *rows, const int32_t *positions,
+                                   int n, void *stream);
+
+/* RECOMPUTE_KV(C, l), Eq. 13-14.
+ *   rows != NULL: DEVICE bf16 [n, d_hidden] (16-byte aligned) with DEVICE int32 positions[n];
+ *                 seq and first_row are ignored.  This is also how (K_t, V_t) of new tokens is made.
+ *   rows == NULL: rows first_row .. first_row+n-1 of the store of (layer, seq) with their stored
+ *                 positions; `positions` must be NULL.
+ *   k_out, v_out: DEVICE bf16; row m, head h, channel c at [m*out_row_stride + h*d_head + c]
+ *                 (out_row_stride in elements, multiple of 8, >= n_kv*d_head; bases 16-byte aligned).
+ * n == 0 is a no-op.  Output bits for a row depend only on that row, its position and the layer,
+ * never on n or on the row's index in the batch. */
+kvd_status kvd_recompute_kv(kvd_ctx *ctx, int layer, const void *rows, const int32_t *positions, int n, int seq,
+                            int first_row, void *k_out, void *v_out, int64_t out_row_stride, void *stream);
+
+/* ATTENTION(Q, K_all, V_all) of Algorithm 1 for one new token per sequence (Eq. 6-7).
+ *   q      DEVICE bf16 [batch, n_q_heads, d_head], already normalised and rotated to q_pos.
+ *   q_pos  HOST int32 [batch]: position of each sequence's query token.
+ *   segs   HOST [batch][n_segs] (n_segs <= KVD_MAX_SEGMENTS); len == 0 entries are skipped.
+ *   scale  multiplies q.k before the softmax; <= 0 selects 1/sqrt(d_head) (Eq. 6).
+ *   out    DEVICE bf16 [batch, n_q_heads, d_head].
+ * Key j of a sequence is attended iff key_pos <= q_pos and, on a sliding-window layer,
+ * q_pos - key_pos < window.  Query head h reads KV head h / (n_q_heads / n_kv_heads).  A sequence
+ * with no visible key yields zeros.  The split of the keys into work units and the order in which
+ * partial results are merged depend on key positions only, not on which segment holds a key, so a
+ * full cache in one segment and the same keys spread over several segments give identical bits.
+ * Needs an attached workspace. */
+kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, const void *q, const int32_t *q_pos,
+                                const kvd_kv_segment *segs, int n_segs, float scale, void *out, void *stream);
+
+/* Fill `out` with the byte counts described at kvd_mem_stats. */
+kvd_status kvd_memory_stats(const kvd_ctx *ctx, kvd_mem_stats *out);
+
+/* Wait for `stream`, read and clear the device status word.  KVD_OK, KVD_ERR_TIMEOUT or
+ * KVD_ERR_POSITION. */
+kvd_status kvd_poll_status(kvd_ctx *ctx, void *stream);
+
+/* Number of kernels this context has launched since creation (all entry points). */
+uint64_t kvd_launch_count(const kvd_ctx *ctx);
+
+/* Text of the last CUDA error a call on this context hit ("" if none).  Valid until the next call. */
+const char *kvd_last_cuda_error(const kvd_ctx *ctx);
+
+const char *kvd_status_string(kvd_status s);
+
+/* Library version, "major.minor". */
+const char *kvd_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVD_H_ */

@@ -1,0 +1,252 @@
+"""ctypes binding of ``libkvd.so`` -- argument marshalling only.
+
+Every function here has the name of the C entry point it calls (``include/kvd.h``) and does nothing
+but convert Python / torch objects to pointers and sizes.  K/V recomputation and attention run
+entirely inside the CUDA kernels of the library; there is no Python or CPU fallback: if the library
+is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libkvd.so")
+
+KVD_OK = 0
+KVD_ERR_INVALID_ARG = 1
+KVD_ERR_SHAPE = 2
+KVD_ERR_ALIGNMENT = 3
+KVD_ERR_CAPACITY = 4
+KVD_ERR_STATE = 5
+KVD_ERR_UNSUPPORTED = 6
+KVD_ERR_CUDA = 7
+KVD_ERR_TIMEOUT = 8
+KVD_ERR_POSITION = 9
+KVD_ROPE_INTERLEAVED = 0
+KVD_ROPE_HALF = 1
+KVD_MAX_SEGMENTS = 4
+
+# every symbol include/kvd.h declares
+EXPORTED_SYMBOLS = (
+    "kvd_create", "kvd_destroy", "kvd_set_layer", "kvd_store_bytes", "kvd_attach_store", "kvd_reset_sequence",
+    "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
+    "kvd_decode_attention", "kvd_memory_stats", "kvd_poll_status", "kvd_launch_count", "kvd_last_cuda_error",
+    "kvd_status_string", "kvd_version",
+)
+
+
+class kvd_model_desc(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("d_hidden", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
+                ("n_kv_heads", ctypes.c_int32), ("d_head", ctypes.c_int32), ("rms_eps", ctypes.c_float),
+                ("qk_norm", ctypes.c_int32), ("qk_norm_eps", ctypes.c_float), ("rope_style", ctypes.c_int32),
+                ("max_seqs", ctypes.c_int32), ("max_tokens_per_seq", ctypes.c_int32), ("max_batch", ctypes.c_int32)]
+
+
+class kvd_layer_desc(ctypes.Structure):
+    _fields_ = [("w_kv", ctypes.c_void_p), ("gamma_in", ctypes.c_void_p), ("gamma_k", ctypes.c_void_p),
+                ("rope_theta", ctypes.c_float), ("sliding_window", ctypes.c_int32)]
+
+
+class kvd_kv_segment(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("row_stride", ctypes.c_int64),
+                ("first_pos", ctypes.c_int32), ("len", ctypes.c_int32)]
+
+
+class kvd_mem_stats(ctypes.Structure):
+    _fields_ = [("checkpoint_bytes_used", ctypes.c_uint64), ("checkpoint_bytes_capacity", ctypes.c_uint64),
+                ("workspace_bytes", ctypes.c_uint64), ("prepared_weight_bytes", ctypes.c_uint64),
+                ("tokens_stored", ctypes.c_uint64), ("eq23_kv_bytes_per_token", ctypes.c_uint64),
+                ("eq24_residual_bytes_per_token", ctypes.c_uint64),
+                ("per_layer_residual_bytes_per_token", ctypes.c_uint64)]
+
+
+class KvdError(RuntimeError):
+    def __init__(self, status: int, what: str, detail: str = ""):
+        self.status = status
+        msg = f"{what}: {status_string(status)} (status {status})"
+        if detail:
+            msg += f" [{detail}]"
+        super().__init__(msg)
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def load() -> ctypes.CDLL:
+    """Load libkvd.so (built by ``paper_2603_19664_b200.build``); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2603_19664_b200.build` "
+                           "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t
+    lib.kvd_create.argtypes = [ctypes.POINTER(kvd_model_desc), ctypes.POINTER(vp)]
+    lib.kvd_create.restype = i32
+    lib.kvd_destroy.argtypes = [vp]
+    lib.kvd_destroy.restype = None
+    lib.kvd_set_layer.argtypes = [vp, i32, ctypes.POINTER(kvd_layer_desc), vp]
+    lib.kvd_set_layer.restype = i32
+    lib.kvd_store_bytes.argtypes = [ctypes.POINTER(kvd_model_desc), i32]
+    lib.kvd_store_bytes.restype = sz
+    lib.kvd_attach_store.argtypes = [vp, vp, sz, i32]
+    lib.kvd_attach_store.restype = i32
+    lib.kvd_reset_sequence.argtypes = [vp, i32]
+    lib.kvd_reset_sequence.restype = i32
+    lib.kvd_rows_stored.argtypes = [vp, i32, i32]
+    lib.kvd_rows_stored.restype = i32
+    lib.kvd_workspace_bytes.argtypes = [ctypes.POINTER(kvd_model_desc)]
+    lib.kvd_workspace_bytes.restype = sz
+    lib.kvd_attach_workspace.argtypes = [vp, vp, sz]
+    lib.kvd_attach_workspace.restype = i32
+    lib.kvd_checkpoint_residual.argtypes = [vp, i32, i32, vp, vp, i32, vp]
+    lib.kvd_checkpoint_residual.restype = i32
+    lib.kvd_recompute_kv.argtypes = [vp, i32, vp, vp, i32, i32, i32, vp, vp, i64, vp]
+    lib.kvd_recompute_kv.restype = i32
+    lib.kvd_decode_attention.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
+                                         ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
+    lib.kvd_decode_attention.restype = i32
+    lib.kvd_memory_stats.argtypes = [vp, ctypes.POINTER(kvd_mem_stats)]
+    lib.kvd_memory_stats.restype = i32
+    lib.kvd_poll_status.argtypes = [vp, vp]
+    lib.kvd_poll_status.restype = i32
+    lib.kvd_launch_count.argtypes = [vp]
+    lib.kvd_launch_count.restype = ctypes.c_uint64
+    lib.kvd_last_cuda_error.argtypes = [vp]
+    lib.kvd_last_cuda_error.restype = ctypes.c_char_p
+    lib.kvd_status_string.argtypes = [i32]
+    lib.kvd_status_string.restype = ctypes.c_char_p
+    lib.kvd_version.argtypes = []
+    lib.kvd_version.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load().kvd_status_string(int(status)).decode()
+
+
+def kvd_version() -> str:
+    return load().kvd_version().decode()
+
+
+def make_desc(n_layers: int, d_hidden: int, n_q_heads: int, n_kv_heads: int, d_head: int, rms_eps: float,
+              qk_norm: bool, qk_norm_eps: float, rope_style: int = KVD_ROPE_INTERLEAVED, max_seqs: int = 1,
+              max_tokens_per_seq: int = 4096, max_batch: int = 1) -> kvd_model_desc:
+    return kvd_model_desc(n_layers, d_hidden, n_q_heads, n_kv_heads, d_head, rms_eps, 1 if qk_norm else 0,
+                          qk_norm_eps, rope_style, max_seqs, max_tokens_per_seq, max_batch)
+
+
+def kvd_store_bytes(desc: kvd_model_desc, layers_stored: int) -> int:
+    return int(load().kvd_store_bytes(ctypes.byref(desc), layers_stored))
+
+
+def kvd_workspace_bytes(desc: kvd_model_desc) -> int:
+    return int(load().kvd_workspace_bytes(ctypes.byref(desc)))
+
+
+def _ptr(t) -> int:
+    """Device (or host) address of a torch tensor, or None."""
+    return None if t is None else int(t.data_ptr())
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return int(torch.cuda.current_stream().cuda_stream)
+    return int(stream)
+
+
+Segment = Tuple[object, object, int, int, int]  # (k tensor/ptr, v tensor/ptr, row_stride, first_pos, len)
+
+
+class Kvd:
+    """One library context.  Method names mirror the C entry points."""
+
+    def __init__(self, desc: kvd_model_desc):
+        self._lib = load()
+        self.desc = desc
+        h = ctypes.c_void_p()
+        st = self._lib.kvd_create(ctypes.byref(desc), ctypes.byref(h))
+        if st != KVD_OK:
+            raise KvdError(st, "kvd_create")
+        self._h = h
+        self._keep: List[object] = []  # tensors the context borrows (store arena, workspace)
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            self._lib.kvd_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st: int, what: str) -> None:
+        if st != KVD_OK:
+            raise KvdError(st, what, self._lib.kvd_last_cuda_error(self._h).decode())
+
+    def kvd_set_layer(self, layer: int, w_kv, gamma_in, gamma_k, rope_theta: float, sliding_window: int = 0,
+                      stream=None) -> None:
+        ld = kvd_layer_desc(_ptr(w_kv), _ptr(gamma_in), _ptr(gamma_k), rope_theta, sliding_window)
+        self._check(self._lib.kvd_set_layer(self._h, layer, ctypes.byref(ld), _stream(stream)), "kvd_set_layer")
+
+    def kvd_attach_store(self, arena, layers_stored: int) -> None:
+        self._keep.append(arena)
+        self._check(self._lib.kvd_attach_store(self._h, _ptr(arena), arena.numel() * arena.element_size(),
+                                               layers_stored), "kvd_attach_store")
+
+    def kvd_attach_workspace(self, ws) -> None:
+        self._keep.append(ws)
+        self._check(self._lib.kvd_attach_workspace(self._h, _ptr(ws), ws.numel() * ws.element_size()),
+                    "kvd_attach_workspace")
+
+    def kvd_reset_sequence(self, seq: int) -> None:
+        self._check(self._lib.kvd_reset_sequence(self._h, seq), "kvd_reset_sequence")
+
+    def kvd_rows_stored(self, layer: int, seq: int) -> int:
+        return int(self._lib.kvd_rows_stored(self._h, layer, seq))
+
+    def kvd_checkpoint_residual(self, seq: int, layer: int, rows, positions, n: int, stream=None) -> None:
+        self._check(self._lib.kvd_checkpoint_residual(self._h, seq, layer, _ptr(rows), _ptr(positions), n,
+                                                      _stream(stream)), "kvd_checkpoint_residual")
+
+    def kvd_recompute_kv(self, layer: int, rows, positions, n: int, k_out, v_out, out_row_stride: int, seq: int = 0,
+                         first_row: int = 0, stream=None) -> None:
+        self._check(self._lib.kvd_recompute_kv(self._h, layer, _ptr(rows), _ptr(positions), n, seq, first_row,
+                                               _ptr(k_out), _ptr(v_out), out_row_stride, _stream(stream)),
+                    "kvd_recompute_kv")
+
+    def kvd_decode_attention(self, layer: int, batch: int, q, q_pos: Sequence[int],
+                             segs: Sequence[Sequence[Segment]], scale: float, out, stream=None) -> None:
+        n_segs = max((len(s) for s in segs), default=0)
+        pos_arr = (ctypes.c_int32 * max(batch, 1))(*[int(p) for p in q_pos])
+        seg_arr = (kvd_kv_segment * max(batch * n_segs, 1))()
+        for b in range(batch):
+            for s in range(n_segs):
+                e = seg_arr[b * n_segs + s]
+                if s < len(segs[b]):
+                    k, v, stride, first, ln = segs[b][s]
+                    e.k = k if isinstance(k, int) else _ptr(k)
+                    e.v = v if isinstance(v, int) else _ptr(v)
+                    e.row_stride, e.first_pos, e.len = int(stride), int(first), int(ln)
+                else:
+                    e.k, e.v, e.row_stride, e.first_pos, e.len = None, None, 0, 0, 0
+        self._check(self._lib.kvd_decode_attention(self._h, layer, batch, _ptr(q), pos_arr, seg_arr, n_segs,
+                                                   float(scale), _ptr(out), _stream(stream)), "kvd_decode_attention")
+
+    def kvd_memory_stats(self) -> dict:
+        ms = kvd_mem_stats()
+        self._check(self._lib.kvd_memory_stats(self._h, ctypes.byref(ms)), "kvd_memory_stats")
+        return {name: int(getattr(ms, name)) for name, _ in kvd_mem_stats._fields_}
+
+    def kvd_poll_status(self, stream=None) -> int:
+        return int(self._lib.kvd_poll_status(self._h, _stream(stream)))
+
+    def kvd_launch_count(self) -> int:
+        return int(self._lib.kvd_launch_count(self._h))

@@ -1,0 +1,496 @@
+// C ABI of the KV-Direct hot path: context management, argument validation, launch set-up.
+// All arithmetic of the method lives in the kernels; nothing here computes K, V or attention.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "kvd_internal.h"
+
+using namespace kvd;
+
+namespace kvd {
+kvd_status cuda_fail(kvd_ctx *ctx, cudaError_t e, const char *where) {
+  if (ctx) {
+    ctx->last_error = std::string(where) + ": " + cudaGetErrorString(e);
+  }
+  return KVD_ERR_CUDA;
+}
+}  // namespace kvd
+
+static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static kvd_status check_desc(const kvd_model_desc *d) {
+  if (!d) return KVD_ERR_INVALID_ARG;
+  if (d->n_layers <= 0 || d->d_hidden <= 0 || d->n_q_heads <= 0 || d->n_kv_heads <= 0 || d->max_seqs <= 0 ||
+      d->max_tokens_per_seq <= 0 || d->max_batch <= 0)
+    return KVD_ERR_INVALID_ARG;
+  if (!(d->rms_eps >= 0.f) || !(d->qk_norm_eps >= 0.f)) return KVD_ERR_INVALID_ARG;
+  if (d->rope_style != KVD_ROPE_INTERLEAVED && d->rope_style != KVD_ROPE_HALF) return KVD_ERR_INVALID_ARG;
+  if (d->d_hidden % 64 != 0) return KVD_ERR_SHAPE;
+  if (d->d_head != 64 && d->d_head != 128 && d->d_head != 256) return KVD_ERR_SHAPE;
+  if (d->n_q_heads % d->n_kv_heads != 0) return KVD_ERR_SHAPE;
+  const int g = d->n_q_heads / d->n_kv_heads;
+  if (!(g == 1 || g == 2 || g == 3 || g == 4 || g == 8)) return KVD_ERR_SHAPE;
+  if ((2 * d->n_kv_heads * d->d_head) % 128 != 0) return KVD_ERR_SHAPE;
+  return KVD_OK;
+}
+
+static int pick_block_n(const kvd_model_desc *d) {
+  const int n = 2 * d->n_kv_heads * d->d_head;
+  if (n % 256 == 0) return 256;
+  return 128;  // n % 128 == 0 was checked; d_head <= 128 follows because 2*n_kv*256 is a multiple of 256
+}
+
+extern "C" const char *kvd_version(void) { return "0.1"; }
+
+extern "C" const char *kvd_status_string(kvd_status s) {
+  switch (s) {
+    case KVD_OK: return "ok";
+    case KVD_ERR_INVALID_ARG: return "invalid argument";
+    case KVD_ERR_SHAPE: return "unsupported shape";
+    case KVD_ERR_ALIGNMENT: return "misaligned pointer or stride";
+    case KVD_ERR_CAPACITY: return "capacity exceeded";
+    case KVD_ERR_STATE: return "call made in the wrong state";
+    case KVD_ERR_UNSUPPORTED: return "no usable sm_100 device";
+    case KVD_ERR_CUDA: return "CUDA error";
+    case KVD_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
+    case KVD_ERR_POSITION: return "row position out of range";
+  }
+  return "unknown status";
+}
+
+extern "C" size_t kvd_store_bytes(const kvd_model_desc *d, int layers_stored) {
+  if (check_desc(d) != KVD_OK || layers_stored <= 0) return 0;
+  const size_t slots = static_cast<size_t>(layers_stored) * d->max_seqs * d->max_tokens_per_seq;
+  return round_up(slots * d->d_hidden * 2, 256) + round_up(slots * 4, 256);
+}
+
+extern "C" size_t kvd_workspace_bytes(const kvd_model_desc *d) {
+  if (check_desc(d) != KVD_OK) return 0;
+  const size_t parts = static_cast<size_t>(d->max_batch) * attn_max_chunks(d->d_head, d->max_tokens_per_seq);
+  return round_up(parts * d->n_q_heads * d->d_head * 4, 256) + round_up(parts * d->n_q_heads * 2 * 4, 256);
+}
+
+extern "C" kvd_status kvd_create(const kvd_model_desc *desc, kvd_ctx **out) {
+  if (!out) return KVD_ERR_INVALID_ARG;
+  *out = nullptr;
+  kvd_status st = check_desc(desc);
+  if (st != KVD_OK) return st;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    cudaGetLastError();
+    return KVD_ERR_UNSUPPORTED;
+  }
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return KVD_ERR_UNSUPPORTED;
+  }
+  if (prop.major != 10) return KVD_ERR_UNSUPPORTED;
+  kvd_ctx *ctx = new (std::nothrow) kvd_ctx();
+  if (!ctx) return KVD_ERR_CUDA;
+  ctx->desc = *desc;
+  ctx->device = dev;
+  ctx->num_sms = prop.multiProcessorCount;
+  ctx->block_n = pick_block_n(desc);
+  ctx->layers.resize(desc->n_layers);
+  void *fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess) {
+    cudaGetLastError();
+    delete ctx;
+    return KVD_ERR_UNSUPPORTED;
+  }
+  ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  cudaError_t e = cudaMalloc(&ctx->d_status, sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int));
+  if (e != cudaSuccess) {
+    delete ctx;
+    return KVD_ERR_CUDA;
+  }
+  const char *env = getenv("KVD_SPIN_LIMIT_MS");
+  if (env) {
+    const long ms = atol(env);
+    if (ms > 0) ctx->timeout_ns = static_cast<unsigned long long>(ms) * 1000000ull;
+  }
+  *out = ctx;
+  return KVD_OK;
+}
+
+extern "C" void kvd_destroy(kvd_ctx *ctx) {
+  if (!ctx) return;
+  cudaSetDevice(ctx->device);
+  cudaDeviceSynchronize();
+  for (auto &l : ctx->layers) {
+    if (l.wt) cudaFree(l.wt);
+    if (l.gamma_k) cudaFree(l.gamma_k);
+  }
+  for (auto &kv : ctx->rope_cache) {
+    if (kv.second.hi) cudaFree(kv.second.hi);
+    if (kv.second.lo) cudaFree(kv.second.lo);
+  }
+  if (ctx->d_status) cudaFree(ctx->d_status);
+  cudaGetLastError();
+  delete ctx;
+}
+
+static kvd_status encode_2d(kvd_ctx *ctx, CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer,
+                            uint32_t box_inner, uint32_t box_outer) {
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {inner * 2};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    char buf[64];
+    snprintf(buf, sizeof buf, "cuTensorMapEncodeTiled failed: %d", static_cast<int>(r));
+    ctx->last_error = buf;
+    return KVD_ERR_CUDA;
+  }
+  return KVD_OK;
+}
+
+// (cos, sin) tables of Eq. 11-12 split as position = 256*hi + lo; built in double on the host.
+static kvd_status get_rope(kvd_ctx *ctx, float theta, RopeTable *out) {
+  uint32_t key;
+  memcpy(&key, &theta, 4);
+  auto it = ctx->rope_cache.find(key);
+  if (it != ctx->rope_cache.end()) {
+    *out = it->second;
+    return KVD_OK;
+  }
+  const int half = ctx->desc.d_head / 2;
+  const int n_hi = (ctx->desc.max_tokens_per_seq + ROPE_LO_SIZE - 1) / ROPE_LO_SIZE;
+  std::vector<float2> hi(static_cast<size_t>(n_hi) * half), lo(static_cast<size_t>(ROPE_LO_SIZE) * half);
+  for (int i = 0; i < half; ++i) {
+    const double freq = pow(static_cast<double>(theta), -2.0 * i / ctx->desc.d_head);
+    for (int h = 0; h < n_hi; ++h) {
+      const double a = static_cast<double>(h) * ROPE_LO_SIZE * freq;
+      hi[static_cast<size_t>(h) * half + i] = make_float2(static_cast<float>(cos(a)), static_cast<float>(sin(a)));
+    }
+    for (int l = 0; l < ROPE_LO_SIZE; ++l) {
+      const double a = static_cast<double>(l) * freq;
+      lo[static_cast<size_t>(l) * half + i] = make_float2(static_cast<float>(cos(a)), static_cast<float>(sin(a)));
+    }
+  }
+  RopeTable t;
+  t.n_hi = n_hi;
+  cudaError_t e = cudaMalloc(&t.hi, hi.size() * sizeof(float2));
+  if (e == cudaSuccess) e = cudaMalloc(&t.lo, lo.size() * sizeof(float2));
+  if (e == cudaSuccess) e = cudaMemcpy(t.hi, hi.data(), hi.size() * sizeof(float2), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMemcpy(t.lo, lo.data(), lo.size() * sizeof(float2), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "rope tables");
+  ctx->prepared_bytes += (hi.size() + lo.size()) * sizeof(float2);
+  ctx->rope_cache[key] = t;
+  *out = t;
+  return KVD_OK;
+}
+
+extern "C" kvd_status kvd_set_layer(kvd_ctx *ctx, int layer, const kvd_layer_desc *ld, void *stream_) {
+  if (!ctx || !ld) return KVD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  if (!ld->w_kv || !ld->gamma_in) return KVD_ERR_INVALID_ARG;
+  if (ctx->desc.qk_norm && !ld->gamma_k) return KVD_ERR_INVALID_ARG;
+  if (!(ld->rope_theta > 1.0f) || ld->sliding_window < 0) return KVD_ERR_INVALID_ARG;
+  if (!aligned16(ld->w_kv)) return KVD_ERR_ALIGNMENT;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const kvd_model_desc &d = ctx->desc;
+  const int n_cols = 2 * d.n_kv_heads * d.d_head;
+  LayerState &ls = ctx->layers[layer];
+  cudaError_t e;
+  if (!ls.wt) {
+    e = cudaMalloc(&ls.wt, static_cast<size_t>(n_cols) * d.d_hidden * 2);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMalloc(prepared weights)");
+    ctx->prepared_bytes += static_cast<size_t>(n_cols) * d.d_hidden * 2;
+  }
+  if (d.qk_norm && !ls.gamma_k) {
+    e = cudaMalloc(&ls.gamma_k, d.d_head * sizeof(float));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMalloc(gamma_k)");
+    ctx->prepared_bytes += d.d_head * sizeof(float);
+  }
+  kvd_status st = launch_prepare_weights(ctx, static_cast<const __nv_bfloat16 *>(ld->w_kv),
+                                         static_cast<const __nv_bfloat16 *>(ld->gamma_in), ls.wt, d.d_hidden, n_cols,
+                                         stream);
+  if (st != KVD_OK) return st;
+  if (d.qk_norm) {
+    st = launch_convert_gamma(ctx, static_cast<const __nv_bfloat16 *>(ld->gamma_k), ls.gamma_k, d.d_head, stream);
+    if (st != KVD_OK) return st;
+  }
+  st = get_rope(ctx, ld->rope_theta, &ls.rope);
+  if (st != KVD_OK) return st;
+  st = encode_2d(ctx, &ls.tmap_b, ls.wt, d.d_hidden, n_cols, RC_BLOCK_K, ctx->block_n);
+  if (st != KVD_OK) return st;
+  e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "kvd_set_layer sync");
+  ls.theta = ld->rope_theta;
+  ls.window = ld->sliding_window;
+  ls.set = true;
+  return KVD_OK;
+}
+
+extern "C" kvd_status kvd_attach_store(kvd_ctx *ctx, void *arena, size_t bytes, int layers_stored) {
+  if (!ctx || !arena || layers_stored <= 0 || layers_stored > ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(arena) & 255u) != 0) return KVD_ERR_ALIGNMENT;
+  const size_t need = kvd_store_bytes(&ctx->desc, layers_stored);
+  if (bytes < need) return KVD_ERR_CAPACITY;
+  const kvd_model_desc &d = ctx->desc;
+  const size_t slots = static_cast<size_t>(layers_stored) * d.max_seqs * d.max_tokens_per_seq;
+  ctx->store_rows = static_cast<__nv_bfloat16 *>(arena);
+  ctx->store_pos = reinterpret_cast<int32_t *>(static_cast<uint8_t *>(arena) + round_up(slots * d.d_hidden * 2, 256));
+  ctx->layers_stored = layers_stored;
+  ctx->rows_stored.assign(static_cast<size_t>(layers_stored) * d.max_seqs, 0);
+  return KVD_OK;
+}
+
+extern "C" kvd_status kvd_reset_sequence(kvd_ctx *ctx, int seq) {
+  if (!ctx || seq < 0 || seq >= ctx->desc.max_seqs) return KVD_ERR_INVALID_ARG;
+  if (!ctx->store_rows) return KVD_ERR_STATE;
+  for (int l = 0; l < ctx->layers_stored; ++l) ctx->rows_stored[static_cast<size_t>(l) * ctx->desc.max_seqs + seq] = 0;
+  return KVD_OK;
+}
+
+extern "C" int kvd_rows_stored(const kvd_ctx *ctx, int layer, int seq) {
+  if (!ctx || !ctx->store_rows || layer < 0 || layer >= ctx->layers_stored || seq < 0 || seq >= ctx->desc.max_seqs)
+    return -1;
+  return ctx->rows_stored[static_cast<size_t>(layer) * ctx->desc.max_seqs + seq];
+}
+
+extern "C" kvd_status kvd_attach_workspace(kvd_ctx *ctx, void *ws, size_t bytes) {
+  if (!ctx || !ws) return KVD_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return KVD_ERR_ALIGNMENT;
+  const size_t need = kvd_workspace_bytes(&ctx->desc);
+  if (bytes < need) return KVD_ERR_CAPACITY;
+  const kvd_model_desc &d = ctx->desc;
+  const size_t parts = static_cast<size_t>(d.max_batch) * attn_max_chunks(d.d_head, d.max_tokens_per_seq);
+  ctx->part_o = static_cast<float *>(ws);
+  ctx->part_ml = reinterpret_cast<float *>(static_cast<uint8_t *>(ws) + round_up(parts * d.n_q_heads * d.d_head * 4, 256));
+  ctx->max_parts = static_cast<int>(parts);
+  ctx->workspace_bytes = need;
+  return KVD_OK;
+}
+
+static inline size_t store_slot(const kvd_ctx *ctx, int layer, int seq) {
+  return (static_cast<size_t>(layer) * ctx->desc.max_seqs + seq) * ctx->desc.max_tokens_per_seq;
+}
+
+extern "C" kvd_status kvd_checkpoint_residual(kvd_ctx *ctx, int seq, int layer, const void *rows,
+                                              const int32_t *positions, int n, void *stream_) {
+  if (!ctx || n < 0) return KVD_ERR_INVALID_ARG;
+  if (!ctx->store_rows) return KVD_ERR_STATE;
+  if (seq < 0 || seq >= ctx->desc.max_seqs || layer < 0 || layer >= ctx->layers_stored) return KVD_ERR_INVALID_ARG;
+  if (n == 0) return KVD_OK;
+  if (!rows || !positions) return KVD_ERR_INVALID_ARG;
+  if (!aligned16(rows)) return KVD_ERR_ALIGNMENT;
+  int &count = ctx->rows_stored[static_cast<size_t>(layer) * ctx->desc.max_seqs + seq];
+  if (count + n > ctx->desc.max_tokens_per_seq) return KVD_ERR_CAPACITY;
+  const size_t slot = store_slot(ctx, layer, seq) + count;
+  kvd_status st = launch_checkpoint(ctx, static_cast<const __nv_bfloat16 *>(rows), positions,
+                                    ctx->store_rows + slot * ctx->desc.d_hidden, ctx->store_pos + slot, n,
+                                    ctx->desc.d_hidden, static_cast<cudaStream_t>(stream_));
+  if (st == KVD_OK) count += n;
+  return st;
+}
+
+extern "C" kvd_status kvd_recompute_kv(kvd_ctx *ctx, int layer, const void *rows, const int32_t *positions, int n,
+                                       int seq, int first_row, void *k_out, void *v_out, int64_t out_row_stride,
+                                       void *stream_) {
+  if (!ctx || n < 0) return KVD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  const LayerState &ls = ctx->layers[layer];
+  if (!ls.set) return KVD_ERR_STATE;
+  if (n == 0) return KVD_OK;
+  if (!k_out || !v_out) return KVD_ERR_INVALID_ARG;
+  const kvd_model_desc &d = ctx->desc;
+  const int kdim = d.n_kv_heads * d.d_head;
+  if (out_row_stride < kdim) return KVD_ERR_INVALID_ARG;
+  if (out_row_stride % 8 != 0 || !aligned16(k_out) || !aligned16(v_out)) return KVD_ERR_ALIGNMENT;
+  const __nv_bfloat16 *a_rows;
+  const int32_t *a_pos;
+  if (rows) {
+    if (!positions) return KVD_ERR_INVALID_ARG;
+    if (!aligned16(rows)) return KVD_ERR_ALIGNMENT;
+    a_rows = static_cast<const __nv_bfloat16 *>(rows);
+    a_pos = positions;
+  } else {
+    if (positions) return KVD_ERR_INVALID_ARG;
+    if (!ctx->store_rows) return KVD_ERR_STATE;
+    if (seq < 0 || seq >= d.max_seqs || layer >= ctx->layers_stored || first_row < 0) return KVD_ERR_INVALID_ARG;
+    const int have = ctx->rows_stored[static_cast<size_t>(layer) * d.max_seqs + seq];
+    if (first_row + n > have) return KVD_ERR_CAPACITY;
+    const size_t slot = store_slot(ctx, layer, seq) + first_row;
+    a_rows = ctx->store_rows + slot * d.d_hidden;
+    a_pos = ctx->store_pos + slot;
+  }
+  CUtensorMap tmap_a;
+  kvd_status st = encode_2d(ctx, &tmap_a, a_rows, d.d_hidden, static_cast<uint64_t>(n), RC_BLOCK_K, RC_BLOCK_M);
+  if (st != KVD_OK) return st;
+  RecomputeParams p;
+  p.M = n;
+  p.num_k_blocks = d.d_hidden / RC_BLOCK_K;
+  p.num_m_blocks = (n + RC_BLOCK_M - 1) / RC_BLOCK_M;
+  p.num_n_blocks = 2 * kdim / ctx->block_n;
+  p.k_cols = kdim;
+  p.positions = a_pos;
+  p.k_out = static_cast<__nv_bfloat16 *>(k_out);
+  p.v_out = static_cast<__nv_bfloat16 *>(v_out);
+  p.out_row_stride = out_row_stride;
+  p.inv_d_hidden = 1.0f / static_cast<float>(d.d_hidden);
+  p.rms_eps = d.rms_eps;
+  p.qk_norm = d.qk_norm;
+  p.qk_eps = d.qk_norm_eps;
+  p.rope_style = d.rope_style;
+  p.rope_hi = ls.rope.hi;
+  p.rope_lo = ls.rope.lo;
+  p.max_pos = ls.rope.n_hi * ROPE_LO_SIZE < d.max_tokens_per_seq ? ls.rope.n_hi * ROPE_LO_SIZE : d.max_tokens_per_seq;
+  p.gamma_k = d.qk_norm ? ls.gamma_k : nullptr;
+  p.status = ctx->d_status;
+  p.timeout_ns = ctx->timeout_ns;
+  return launch_recompute(ctx, ls, tmap_a, p, static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, const void *q, const int32_t *q_pos,
+                                           const kvd_kv_segment *segs, int n_segs, float scale, void *out,
+                                           void *stream_) {
+  if (!ctx || batch < 0 || n_segs < 0 || n_segs > KVD_MAX_SEGMENTS) return KVD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  const LayerState &ls = ctx->layers[layer];
+  if (!ls.set) return KVD_ERR_STATE;
+  if (!ctx->part_o) return KVD_ERR_STATE;
+  if (batch == 0) return KVD_OK;
+  if (!q || !q_pos || !out || (n_segs > 0 && !segs)) return KVD_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out)) return KVD_ERR_ALIGNMENT;
+  const kvd_model_desc &d = ctx->desc;
+  if (batch > d.max_batch) return KVD_ERR_CAPACITY;
+  const int kdim = d.n_kv_heads * d.d_head;
+  const int group = d.n_q_heads / d.n_kv_heads;
+  // ---- validate every segment before anything is launched
+  for (int b = 0; b < batch; ++b) {
+    if (q_pos[b] < 0) return KVD_ERR_INVALID_ARG;
+    for (int s = 0; s < n_segs; ++s) {
+      const kvd_kv_segment &sg = segs[static_cast<size_t>(b) * n_segs + s];
+      if (sg.len < 0 || sg.first_pos < 0) return KVD_ERR_INVALID_ARG;
+      if (sg.len == 0) continue;
+      if (!sg.k || !sg.v || sg.row_stride < kdim) return KVD_ERR_INVALID_ARG;
+      if (!aligned16(sg.k) || !aligned16(sg.v) || sg.row_stride % 8 != 0) return KVD_ERR_ALIGNMENT;
+      if (static_cast<int64_t>(sg.first_pos) + sg.len > INT32_MAX) return KVD_ERR_INVALID_ARG;
+      for (int s2 = 0; s2 < s; ++s2) {
+        const kvd_kv_segment &o = segs[static_cast<size_t>(b) * n_segs + s2];
+        if (o.len == 0) continue;
+        if (sg.first_pos < o.first_pos + o.len && o.first_pos < sg.first_pos + sg.len) return KVD_ERR_INVALID_ARG;
+      }
+    }
+  }
+  const float sc = scale > 0.f ? scale : 1.0f / sqrtf(static_cast<float>(d.d_head));
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  static thread_local AttnLaunch L;  // large: keep it off the stack
+  for (int b0 = 0; b0 < batch; b0 += AT_MAX_SEQS) {
+    const int nb = batch - b0 < AT_MAX_SEQS ? batch - b0 : AT_MAX_SEQS;
+    int parts = 0;
+    for (int i = 0; i < nb; ++i) {
+      const int b = b0 + i;
+      AttnSeq &S = L.seq[i];
+      int min_first = INT32_MAX, max_last = -1;
+      for (int s = 0; s < KVD_MAX_SEGMENTS; ++s) {
+        S.k[s] = S.v[s] = nullptr;
+        S.stride[s] = 0;
+        S.first[s] = 0;
+        S.len[s] = 0;
+        if (s < n_segs) {
+          const kvd_kv_segment &sg = segs[static_cast<size_t>(b) * n_segs + s];
+          if (sg.len > 0) {
+            S.k[s] = static_cast<const __nv_bfloat16 *>(sg.k);
+            S.v[s] = static_cast<const __nv_bfloat16 *>(sg.v);
+            S.stride[s] = sg.row_stride;
+            S.first[s] = sg.first_pos;
+            S.len[s] = sg.len;
+            if (sg.first_pos < min_first) min_first = sg.first_pos;
+            if (sg.first_pos + sg.len - 1 > max_last) max_last = sg.first_pos + sg.len - 1;
+          }
+        }
+      }
+      S.q_pos = q_pos[b];
+      int lo = ls.window > 0 ? S.q_pos - ls.window + 1 : 0;
+      if (lo < 0) lo = 0;
+      if (min_first > lo) lo = min_first;
+      int hi = S.q_pos < max_last ? S.q_pos : max_last;
+      S.lo_pos = lo;
+      S.hi_pos = hi;
+      S.part_base = parts;
+      S.pad = 0;
+      if (max_last < 0 || hi < lo) {
+        S.n_chunks = 0;
+        S.iters = 1;
+        S.chunk0_pos = 0;
+      } else {
+        // the split depends on the visible position range only
+        S.iters = attn_iters_for_span(hi - lo + 1);
+        const int ck = attn_chunk_keys(d.d_head, S.iters);
+        S.chunk0_pos = lo / ck * ck;
+        S.n_chunks = hi / ck - lo / ck + 1;
+      }
+      parts += S.n_chunks;
+    }
+    if (parts > ctx->max_parts) return KVD_ERR_CAPACITY;
+    L.n_seqs = nb;
+    L.total_chunks = parts;
+    L.n_q = d.n_q_heads;
+    L.n_kv = d.n_kv_heads;
+    L.q = static_cast<const __nv_bfloat16 *>(q) + static_cast<size_t>(b0) * d.n_q_heads * d.d_head;
+    L.out = static_cast<__nv_bfloat16 *>(out) + static_cast<size_t>(b0) * d.n_q_heads * d.d_head;
+    L.part_o = ctx->part_o;
+    L.part_ml = ctx->part_ml;
+    L.scale_log2e = sc * 1.4426950408889634f;
+    kvd_status st = launch_attention(ctx, L, d.d_head, group, stream);
+    if (st != KVD_OK) return st;
+  }
+  return KVD_OK;
+}
+
+extern "C" kvd_status kvd_memory_stats(const kvd_ctx *ctx, kvd_mem_stats *out) {
+  if (!ctx || !out) return KVD_ERR_INVALID_ARG;
+  const kvd_model_desc &d = ctx->desc;
+  memset(out, 0, sizeof(*out));
+  uint64_t rows_total = 0, tokens = 0;
+  for (int l = 0; l < ctx->layers_stored; ++l) {
+    uint64_t layer_rows = 0;
+    for (int s = 0; s < d.max_seqs; ++s) layer_rows += ctx->rows_stored[static_cast<size_t>(l) * d.max_seqs + s];
+    rows_total += layer_rows;
+    if (layer_rows > tokens) tokens = layer_rows;
+  }
+  out->checkpoint_bytes_used = rows_total * (static_cast<uint64_t>(d.d_hidden) * 2 + 4);
+  out->checkpoint_bytes_capacity = ctx->layers_stored > 0 ? kvd_store_bytes(&d, ctx->layers_stored) : 0;
+  out->workspace_bytes = ctx->workspace_bytes;
+  out->prepared_weight_bytes = ctx->prepared_bytes;
+  out->tokens_stored = tokens;
+  out->eq23_kv_bytes_per_token = 2ull * d.n_layers * d.n_kv_heads * d.d_head * 2;
+  out->eq24_residual_bytes_per_token = static_cast<uint64_t>(d.d_hidden) * 2;
+  out->per_layer_residual_bytes_per_token = static_cast<uint64_t>(d.n_layers) * d.d_hidden * 2;
+  return KVD_OK;
+}
+
+extern "C" kvd_status kvd_poll_status(kvd_ctx *ctx, void *stream_) {
+  if (!ctx) return KVD_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  cudaError_t e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "kvd_poll_status sync");
+  int word = 0;
+  e = cudaMemcpy(&word, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "kvd_poll_status read");
+  if (word != 0) {
+    e = cudaMemset(ctx->d_status, 0, sizeof(int));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "kvd_poll_status clear");
+  }
+  if (word & STATUS_TIMEOUT) return KVD_ERR_TIMEOUT;
+  if (word & STATUS_POSITION) return KVD_ERR_POSITION;
+  return KVD_OK;
+}
+
+extern "C" uint64_t kvd_launch_count(const kvd_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" const char *kvd_last_cuda_error(const kvd_ctx *ctx) { return ctx ? ctx->last_error.c_str() : ""; }

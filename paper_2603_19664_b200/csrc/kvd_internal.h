@@ -1,0 +1,161 @@
+// Host-side context and the parameter blocks passed to the kernels.  Internal to the library.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <map>
+#include <string>
+#include <vector>
+
+#include "../../include/kvd.h"
+
+namespace kvd {
+
+// device status word bits (written by kernels with atomicOr, read by kvd_poll_status)
+constexpr int STATUS_TIMEOUT = 1;
+constexpr int STATUS_POSITION = 2;
+
+constexpr int ROPE_LO_BITS = 8;  // position = hi * 256 + lo; one table per part
+constexpr int ROPE_LO_SIZE = 1 << ROPE_LO_BITS;
+
+// ------------------------------------------------------------------------------ recompute GEMM
+constexpr int RC_BLOCK_M = 128;
+constexpr int RC_BLOCK_K = 64;
+constexpr int RC_THREADS = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 row statistics, warps 6-9 epilogue
+
+struct RecomputeParams {
+  int M;          // rows
+  int num_k_blocks;  // d_hidden / 64
+  int num_m_blocks;
+  int num_n_blocks;
+  int k_cols;  // n_kv * d_head: fused columns below this index are keys, the rest values
+  const int32_t *positions;  // [M]
+  __nv_bfloat16 *k_out;
+  __nv_bfloat16 *v_out;
+  long long out_row_stride;
+  float inv_d_hidden;
+  float rms_eps;
+  int qk_norm;
+  float qk_eps;
+  int rope_style;
+  const float2 *rope_hi;  // [n_hi][d_head/2] (cos, sin) of (pos & ~255) * freq_i
+  const float2 *rope_lo;  // [256][d_head/2]  (cos, sin) of (pos & 255) * freq_i
+  int max_pos;            // positions must be in [0, max_pos)
+  const float *gamma_k;   // [d_head] fp32 or nullptr
+  int *status;
+  unsigned long long timeout_ns;
+};
+
+// ------------------------------------------------------------------------------ decode attention
+constexpr int AT_THREADS = 128;
+constexpr int AT_WARPS = 4;
+constexpr int AT_UNROLL = 8;          // keys per lane group per iteration
+constexpr int AT_MAX_SEQS = 64;       // sequences per launch (bounded by the kernel parameter space)
+
+struct AttnSeq {
+  const __nv_bfloat16 *k[KVD_MAX_SEGMENTS];
+  const __nv_bfloat16 *v[KVD_MAX_SEGMENTS];
+  long long stride[KVD_MAX_SEGMENTS];
+  int first[KVD_MAX_SEGMENTS];
+  int len[KVD_MAX_SEGMENTS];
+  int q_pos;
+  int lo_pos;       // first visible position
+  int hi_pos;       // last visible position (<= q_pos)
+  int chunk0_pos;   // position of the first key of chunk 0 (multiple of the chunk size)
+  int n_chunks;
+  int part_base;    // index of this sequence's first partial in the scratch
+  int iters;        // warp iterations per chunk
+  int pad;
+};
+
+struct AttnLaunch {
+  AttnSeq seq[AT_MAX_SEQS];
+  int n_seqs;
+  int total_chunks;
+  int n_q;
+  int n_kv;
+  const __nv_bfloat16 *q;  // [n_seqs, n_q, d_head] (already offset to the launch's first sequence)
+  __nv_bfloat16 *out;      // [n_seqs, n_q, d_head]
+  float *part_o;           // [parts][n_q][d_head]
+  float *part_ml;          // [parts][n_q][2]
+  float scale_log2e;
+};
+
+// keys per chunk for a head size and iteration count
+inline int attn_keys_per_warp_iter(int d_head) { return (32 / (d_head / 8)) * AT_UNROLL; }
+inline int attn_iters_for_span(int span) { return span <= 8192 ? 2 : (span <= 65536 ? 4 : 8); }
+inline int attn_chunk_keys(int d_head, int iters) { return attn_keys_per_warp_iter(d_head) * AT_WARPS * iters; }
+inline int attn_max_chunks(int d_head, int max_tokens) {
+  int best = 0;
+  const int spans[3] = {max_tokens < 8192 ? max_tokens : 8192, max_tokens < 65536 ? max_tokens : 65536, max_tokens};
+  for (int i = 0; i < 3; ++i) {
+    const int ck = attn_chunk_keys(d_head, attn_iters_for_span(spans[i]));
+    const int c = spans[i] / ck + 2;
+    if (c > best) best = c;
+  }
+  return best;
+}
+
+// ------------------------------------------------------------------------------ context
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct RopeTable {
+  float2 *hi = nullptr;
+  float2 *lo = nullptr;
+  int n_hi = 0;
+};
+
+struct LayerState {
+  bool set = false;
+  __nv_bfloat16 *wt = nullptr;  // [2*n_kv*d_head, d_hidden]: gamma-folded, K-major
+  float *gamma_k = nullptr;     // [d_head] fp32
+  float theta = 0.f;
+  int window = 0;
+  RopeTable rope;
+  CUtensorMap tmap_b;
+};
+
+}  // namespace kvd
+
+struct kvd_ctx {
+  kvd_model_desc desc;
+  int device = 0;
+  int num_sms = 0;
+  int block_n = 0;
+  std::vector<kvd::LayerState> layers;
+  std::map<uint32_t, kvd::RopeTable> rope_cache;  // keyed by the bits of theta
+  // residual store
+  __nv_bfloat16 *store_rows = nullptr;
+  int32_t *store_pos = nullptr;
+  int layers_stored = 0;
+  std::vector<int> rows_stored;  // [layers_stored * max_seqs]
+  // attention scratch
+  float *part_o = nullptr;
+  float *part_ml = nullptr;
+  size_t workspace_bytes = 0;
+  int max_parts = 0;
+  int *d_status = nullptr;
+  uint64_t launches = 0;
+  uint64_t prepared_bytes = 0;
+  unsigned long long timeout_ns = 2000000000ull;
+  std::string last_error;
+  kvd::EncodeTiledFn encode = nullptr;
+};
+
+namespace kvd {
+// launchers implemented next to their kernels
+kvd_status launch_recompute(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_a, const RecomputeParams &p,
+                            cudaStream_t stream);
+kvd_status launch_attention(kvd_ctx *ctx, const AttnLaunch &L, int d_head, int group, cudaStream_t stream);
+kvd_status launch_prepare_weights(kvd_ctx *ctx, const __nv_bfloat16 *w, const __nv_bfloat16 *gamma, __nv_bfloat16 *wt,
+                                  int d_hidden, int n_cols, cudaStream_t stream);
+kvd_status launch_convert_gamma(kvd_ctx *ctx, const __nv_bfloat16 *g, float *out, int n, cudaStream_t stream);
+kvd_status launch_checkpoint(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, __nv_bfloat16 *dst_rows,
+                             int32_t *dst_pos, int n, int d_hidden, cudaStream_t stream);
+kvd_status cuda_fail(kvd_ctx *ctx, cudaError_t e, const char *where);
+}  // namespace kvd

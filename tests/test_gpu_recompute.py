@@ -1,0 +1,213 @@
+"""GPU parity of kvd_recompute_kv / kvd_checkpoint_residual against the fp64 oracle (through the C ABI).
+
+Tolerances (bf16 outputs against the fp64 oracle, per K and per V):
+    max |gpu - oracle| <= 2e-2   and   ||gpu - oracle||_F / ||oracle||_F <= 1e-2.
+Bit-identity tests compare raw bf16 bit patterns.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2603_19664_b200 as kvd
+from kvd_synth import (GEMMA3_4B_GLOBAL, GEMMA3_4B_LOCAL, QWEN3_4B, ROPE_HALF, SMOLLM2_135M, TINY_GQA, TINY_MHA,
+                       make_residuals, with_style)
+from gpu_util import dev, host_bits, host_f64, kv_errors, open_layer, oracle_kv
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS = 2e-2
+REL_FRO = 1e-2
+
+
+def run_gpu(ctx, shape, X_bits, pos, stride=None, sentinel_rows=0):
+    n = X_bits.shape[0]
+    kdim = shape.n_kv_heads * shape.d_head
+    stride = stride or kdim
+    x = dev(X_bits)
+    p = torch.from_numpy(np.asarray(pos, np.int32)).cuda()
+    k = torch.full((n + sentinel_rows, stride), -7.0, dtype=torch.bfloat16, device="cuda")
+    v = torch.full((n + sentinel_rows, stride), -7.0, dtype=torch.bfloat16, device="cuda")
+    ctx.kvd_recompute_kv(0, x, p, n, k, v, stride)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    return k, v
+
+
+def check(shape, K, V, Kref, Vref, rows=None):
+    kdim = shape.n_kv_heads * shape.d_head
+    Kg = host_f64(K)[:, :kdim]
+    Vg = host_f64(V)[:, :kdim]
+    if rows is not None:
+        Kg, Vg = Kg[rows], Vg[rows]
+    Kr = Kref.reshape(Kref.shape[0], kdim)
+    Vr = Vref.reshape(Vref.shape[0], kdim)
+    for name, g, r in (("K", Kg, Kr), ("V", Vg, Vr)):
+        mx, rel = kv_errors(g, r)
+        assert mx <= MAX_ABS, f"{name}: max abs {mx}"
+        assert rel <= REL_FRO, f"{name}: rel {rel}"
+
+
+@pytest.mark.parametrize("shape", [TINY_GQA, TINY_MHA, SMOLLM2_135M], ids=lambda s: s.name)
+@pytest.mark.parametrize("n", [1, 7, 127, 128, 129, 300])
+def test_small_shapes_and_ragged_tiles(shape, n):
+    ctx, w = open_layer(shape)
+    X = make_residuals(shape, n, seed=n)
+    pos = (np.arange(n) * 3 + 1) % 4096
+    K, V = run_gpu(ctx, shape, X, pos)
+    Kr, Vr = oracle_kv(shape, w, X, pos)
+    check(shape, K, V, Kr, Vr)
+
+
+def test_config1_smollm2_layer_full():
+    # SmolLM2-135M layer, 512 checkpointed tokens at positions 0..511
+    shape = SMOLLM2_135M
+    ctx, w = open_layer(shape)
+    X = make_residuals(shape, 512, seed=1)
+    pos = np.arange(512)
+    K, V = run_gpu(ctx, shape, X, pos, sentinel_rows=4)
+    Kr, Vr = oracle_kv(shape, w, X, pos)
+    check(shape, K[:512], V[:512], Kr, Vr)
+    # guard rows behind the output stay untouched
+    assert torch.all(K[512:] == -7.0) and torch.all(V[512:] == -7.0)
+
+
+@pytest.mark.parametrize("shape", [GEMMA3_4B_GLOBAL, GEMMA3_4B_LOCAL], ids=lambda s: s.name)
+def test_config2_gemma_layer_t4096_sampled(shape):
+    # full-size launch (T = 4096, outlier channels); the oracle checks the first and last row of
+    # every 128-row tile class plus a random sample
+    T = 4096
+    ctx, w = open_layer(shape, max_tokens=32768)
+    X = make_residuals(shape, T, seed=2, outliers=True)
+    pos = np.arange(T)
+    K, V = run_gpu(ctx, shape, X, pos)
+    rng = np.random.default_rng(0)
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, 129, 2047, 2048, T - 129, T - 128, T - 1],
+                                     rng.choice(T, 150, replace=False)]))
+    Kr, Vr = oracle_kv(shape, w, X[rows], pos[rows])
+    check(shape, K, V, Kr, Vr, rows=rows)
+
+
+def test_qwen3_shape_two_heads_per_tile_and_large_positions():
+    shape = QWEN3_4B
+    ctx, w = open_layer(shape, max_tokens=32768)
+    n = 333
+    X = make_residuals(shape, n, seed=3)
+    pos = np.concatenate([np.arange(32768 - 200, 32768), np.arange(0, n - 200)])
+    K, V = run_gpu(ctx, shape, X, pos)
+    rows = np.arange(0, n, 3)
+    Kr, Vr = oracle_kv(shape, w, X[rows], pos[rows])
+    check(shape, K, V, Kr, Vr, rows=rows)
+
+
+@pytest.mark.parametrize("shape", [TINY_GQA, SMOLLM2_135M, GEMMA3_4B_GLOBAL], ids=lambda s: s.name)
+def test_half_rotation_style(shape):
+    shape = with_style(shape, ROPE_HALF)
+    ctx, w = open_layer(shape, max_tokens=8192)
+    n = 140
+    X = make_residuals(shape, n, seed=4)
+    pos = np.arange(n) * 37 % 8192
+    K, V = run_gpu(ctx, shape, X, pos)
+    rows = np.arange(0, n, 2)
+    Kr, Vr = oracle_kv(shape, w, X[rows], pos[rows])
+    check(shape, K, V, Kr, Vr, rows=rows)
+
+
+def test_fused_output_buffer_with_row_stride():
+    # K and V side by side in one [n, 2*kdim] buffer
+    shape = TINY_GQA
+    ctx, w = open_layer(shape)
+    n, kdim = 70, shape.n_kv_heads * shape.d_head
+    X = make_residuals(shape, n, seed=5)
+    pos = np.arange(n)
+    buf = torch.zeros((n, 2 * kdim), dtype=torch.bfloat16, device="cuda")
+    x, p = dev(X), torch.from_numpy(pos.astype(np.int32)).cuda()
+    ctx._check(ctx._lib.kvd_recompute_kv(ctx._h, 0, x.data_ptr(), p.data_ptr(), n, 0, 0, buf.data_ptr(),
+                                         buf.data_ptr() + kdim * 2, 2 * kdim, None), "kvd_recompute_kv")
+    torch.cuda.synchronize()
+    Kr, Vr = oracle_kv(shape, w, X, pos)
+    check(shape, buf[:, :kdim], buf[:, kdim:], Kr, Vr)
+
+
+@pytest.mark.parametrize("shape", [TINY_GQA, SMOLLM2_135M, GEMMA3_4B_GLOBAL], ids=lambda s: s.name)
+def test_recompute_is_bit_identical_to_first_pass(shape):
+    """Proposition 3.2 on the GPU: a row's K/V bits do not depend on the batch it is computed in."""
+    ctx, w = open_layer(shape, max_tokens=8192)
+    T = 4096 if shape is GEMMA3_4B_GLOBAL else 600
+    X = make_residuals(shape, T, seed=6, outliers=shape is GEMMA3_4B_GLOBAL)
+    pos = np.arange(T) + 11
+    K, V = run_gpu(ctx, shape, X, pos)
+    Kb, Vb = host_bits(K), host_bits(V)
+    # first pass: one token at a time (M = 1), as a decode step produces K_t, V_t
+    for m in (0, 1, 127, 128, T - 1):
+        k1, v1 = run_gpu(ctx, shape, X[m:m + 1], pos[m:m + 1])
+        assert np.array_equal(host_bits(k1)[0], Kb[m]) and np.array_equal(host_bits(v1)[0], Vb[m])
+    # the same rows at other batch positions and batch sizes
+    for start, n in ((5, 7), (100, 128), (77, 129), (T - 130, 130)):
+        k2, v2 = run_gpu(ctx, shape, X[start:start + n], pos[start:start + n])
+        assert np.array_equal(host_bits(k2), Kb[start:start + n])
+        assert np.array_equal(host_bits(v2), Vb[start:start + n])
+    perm = np.random.default_rng(1).permutation(T)[:257]
+    k3, v3 = run_gpu(ctx, shape, X[perm], pos[perm])
+    assert np.array_equal(host_bits(k3), Kb[perm]) and np.array_equal(host_bits(v3), Vb[perm])
+    # run-to-run determinism
+    K2, V2 = run_gpu(ctx, shape, X, pos)
+    assert np.array_equal(host_bits(K2), Kb) and np.array_equal(host_bits(V2), Vb)
+
+
+def test_checkpoint_store_roundtrip_and_recompute_from_store():
+    shape = SMOLLM2_135M
+    ctx, w = open_layer(shape, max_tokens=512, max_seqs=2, with_store=True)
+    kdim = shape.n_kv_heads * shape.d_head
+    X = make_residuals(shape, 300, seed=7)
+    pos = np.arange(300) + 5
+    x, p = dev(X), torch.from_numpy(pos.astype(np.int32)).cuda()
+    # append in two pieces to sequence 1, something else to sequence 0
+    ctx.kvd_checkpoint_residual(1, 0, x[:100], p[:100], 100)
+    ctx.kvd_checkpoint_residual(0, 0, x[200:], p[200:], 100)
+    ctx.kvd_checkpoint_residual(1, 0, x[100:], p[100:], 200)
+    assert ctx.kvd_rows_stored(0, 1) == 300 and ctx.kvd_rows_stored(0, 0) == 100
+    stats = ctx.kvd_memory_stats()
+    assert stats["checkpoint_bytes_used"] == 400 * (shape.d_hidden * 2 + 4)
+    assert stats["eq24_residual_bytes_per_token"] == shape.d_hidden * 2
+    K, V = run_gpu(ctx, shape, X, pos)
+    k = torch.zeros((250, kdim), dtype=torch.bfloat16, device="cuda")
+    v = torch.zeros_like(k)
+    ctx.kvd_recompute_kv(0, None, None, 250, k, v, kdim, seq=1, first_row=50)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    assert torch.equal(k, K[50:300]) and torch.equal(v, V[50:300])
+    Kr, Vr = oracle_kv(shape, w, X[50:300], pos[50:300])
+    check(shape, k, v, Kr, Vr)
+    # capacity and state errors are reported, nothing is launched
+    with pytest.raises(kvd.KvdError) as e:
+        ctx.kvd_recompute_kv(0, None, None, 10, k, v, kdim, seq=0, first_row=95)
+    assert e.value.status == 4
+    with pytest.raises(kvd.KvdError) as e:
+        ctx.kvd_checkpoint_residual(1, 0, x, p, 300)
+    assert e.value.status == 4
+    ctx.kvd_reset_sequence(1)
+    assert ctx.kvd_rows_stored(0, 1) == 0
+
+
+def test_argument_errors_and_position_flag():
+    shape = TINY_GQA
+    ctx, w = open_layer(shape, max_tokens=1024)
+    kdim = shape.n_kv_heads * shape.d_head
+    X = make_residuals(shape, 16, seed=8)
+    x = dev(X)
+    p = torch.arange(16, dtype=torch.int32, device="cuda")
+    k = torch.zeros((16, kdim), dtype=torch.bfloat16, device="cuda")
+    v = torch.zeros_like(k)
+    lib, h = ctx._lib, ctx._h
+    assert lib.kvd_recompute_kv(h, 0, x.data_ptr() + 2, p.data_ptr(), 4, 0, 0, k.data_ptr(), v.data_ptr(), kdim, None) == 3
+    assert lib.kvd_recompute_kv(h, 0, x.data_ptr(), p.data_ptr(), 4, 0, 0, k.data_ptr(), v.data_ptr(), kdim - 8, None) == 1
+    assert lib.kvd_recompute_kv(h, 0, x.data_ptr(), p.data_ptr(), 4, 0, 0, k.data_ptr(), v.data_ptr(), kdim + 4, None) == 3
+    assert lib.kvd_recompute_kv(h, 3, x.data_ptr(), p.data_ptr(), 4, 0, 0, k.data_ptr(), v.data_ptr(), kdim, None) == 1
+    assert lib.kvd_recompute_kv(h, 0, x.data_ptr(), None, 4, 0, 0, k.data_ptr(), v.data_ptr(), kdim, None) == 1
+    assert lib.kvd_recompute_kv(h, 0, x.data_ptr(), p.data_ptr(), 0, 0, 0, None, None, kdim, None) == 0  # n = 0: no-op
+    # a position outside [0, max_tokens) is flagged, clamped, and faults nothing
+    bad = p.clone()
+    bad[3] = 5000
+    bad[9] = -2
+    ctx.kvd_recompute_kv(0, x, bad, 16, k, v, kdim)
+    assert ctx.kvd_poll_status() == 9
+    assert ctx.kvd_poll_status() == kvd.KVD_OK  # the flag is cleared by the read
+    assert ctx.kvd_launch_count() >= 2
