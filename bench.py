@@ -176,6 +176,30 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------- GPU arm
+class GraphEvent:
+    """A CUDA event that can be recorded inside a captured graph (an event-record node) and timed
+    afterwards; torch's own events cannot be timed when recorded during capture."""
+
+    def __init__(self):
+        try:
+            from cuda.bindings import runtime as rt
+        except ImportError:  # older cuda-python layout
+            from cuda import cudart as rt
+        self.rt = rt
+        err, self.e = rt.cudaEventCreate()
+        assert int(err) == 0, err
+
+    def record(self):
+        import torch
+        (err,) = self.rt.cudaEventRecordWithFlags(self.e, torch.cuda.current_stream().cuda_stream, 1)  # external
+        assert int(err) == 0, err
+
+    def elapsed_ms(self, other):
+        err, ms = self.rt.cudaEventElapsedTime(self.e, other.e)
+        assert int(err) == 0, err
+        return ms
+
+
 class Workload:
     """Device buffers and the step function for the Gemma-3-4B-shaped layer."""
 
@@ -265,35 +289,70 @@ def run_gpu(args):
 
     shape, T = GEMMA3_4B_GLOBAL, T_TOKENS
     peaks = load_peaks()
-    wl = Workload(shape, T, N_SETS)
+    n_sets = args.sets
+    wl = Workload(shape, T, n_sets)
     steps, warmup = args.steps, max(args.warmup, 3)
 
-    # ---- warm-up
+    # ---- warm-up (eager launches)
     for i in range(warmup):
         wl.step(i)
     barrier()
     assert wl.ctx.kvd_poll_status() == kvd.KVD_OK
 
-    # ---- timed region: exactly `steps` steps, whole-region CUDA events + per-kernel events
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
+    if args.profile:
+        # plain eager launches for a profiler: no graphs, no auxiliary measurements
+        for i in range(steps):
+            wl.step(warmup + i)
+        barrier()
+        if rank == 0:
+            print(json.dumps({"profile_run": True, "steps": steps, "launches": wl.ctx.kvd_launch_count()}))
+        return
+
+    # ---- the step is a fixed launch sequence: capture it once per buffer set into CUDA graphs
+    side = torch.cuda.Stream()
+
+    def capture(n, events=None):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for i in range(n):
+                wl.step(i, events[i] if events else None)
+        return g
+
+    l0 = wl.ctx.kvd_launch_count()
+    g_full = capture(n_sets)
+    launches_per_step = (wl.ctx.kvd_launch_count() - l0) // n_sets
+    g_rem = capture(steps % n_sets) if steps % n_sets else None
+    kev = [[GraphEvent() for _ in range(5)] for _ in range(n_sets)]
+    g_ev = capture(n_sets, kev)
+    for _ in range(2):
+        g_full.replay()
+    barrier()
+
+    # ---- timed region: exactly `steps` steps
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches0 = wl.ctx.kvd_launch_count()
     barrier()
     with ClockSampler(local) as clocks:
         start.record()
-        for i in range(steps):
-            wl.step(warmup + i, ev[i])
+        for _ in range(steps // n_sets):
+            g_full.replay()
+        if g_rem is not None:
+            g_rem.replay()
         stop.record()
         barrier()
-    launches = wl.ctx.kvd_launch_count() - launches0
+        # per-kernel durations: the same steps with event-record nodes between the kernels
+        t_k = [[], [], [], []]
+        for _ in range(max(2, min(20, steps // n_sets))):
+            g_ev.replay()
+            torch.cuda.synchronize()
+            for e in kev:
+                for j in range(4):
+                    t_k[j].append(e[j].elapsed_ms(e[j + 1]))
+    launches = launches_per_step * steps
     total_ms = start.elapsed_time(stop)
     status = wl.ctx.kvd_poll_status()
     if status != kvd.KVD_OK:
         raise RuntimeError(f"device status after the timed region: {kvd.status_string(status)}")
-    t_ckpt = np.array([e[0].elapsed_time(e[1]) for e in ev])
-    t_gemm = np.array([e[1].elapsed_time(e[2]) for e in ev])
-    t_kt = np.array([e[2].elapsed_time(e[3]) for e in ev])
-    t_attn = np.array([e[3].elapsed_time(e[4]) for e in ev])
+    t_ckpt, t_gemm, t_kt, t_attn = (np.array(t) for t in t_k)
     if dist is not None:
         t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -301,7 +360,24 @@ def run_gpu(args):
     ms_per_step = total_ms / steps
     value = world * T / (ms_per_step * 1e-3)
 
-    # ---- the read that recomputation replaces (separate loops, same rotation)
+    # ---- the read that recomputation replaces (graphs of n_sets calls, same rotation)
+    def timed_graph(fn, reps):
+        for i in range(n_sets):
+            fn(i)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for i in range(n_sets):
+                fn(i)
+        g.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / (reps * n_sets)
+
     def timed(fn, n):
         for i in range(3):
             fn(i)
@@ -314,8 +390,7 @@ def run_gpu(args):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / n
 
-    n_aux = min(max(steps, 20), 200)
-    read_attn_ms = timed(wl.cached_read_step, n_aux)
+    read_attn_ms = timed_graph(wl.cached_read_step, 10)
     kv_copy_dst = torch.empty((2, T + 1, wl.kdim), dtype=torch.bfloat16, device="cuda")
 
     def copy_step(i):
@@ -323,7 +398,7 @@ def run_gpu(args):
         kv_copy_dst[0].copy_(wl.K[s])
         kv_copy_dst[1].copy_(wl.V[s])
 
-    read_copy_ms = timed(copy_step, n_aux)
+    read_copy_ms = timed_graph(copy_step, 10)
 
     # ---- end to end through the C ABI with host buffers
     x_pin = torch.from_numpy(wl.x_host_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
@@ -351,7 +426,7 @@ def run_gpu(args):
         out_pin.copy_(out_dev, non_blocking=True)
         torch.cuda.current_stream().synchronize()  # the caller reads the result of every step
 
-    n_e2e = min(max(steps, 10), 100)
+    n_e2e = min(max(steps, 10), 50)
     e2e_ms = timed(e2e_step, n_e2e)
     if dist is not None:
         t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
@@ -377,7 +452,8 @@ def run_gpu(args):
                                    "T=4096 checkpointed tokens, batch 1 (config 2)",
                        "step": "checkpoint T rows -> recompute K/V of T rows from the store -> K_t,V_t -> "
                                "decode attention over T+1 keys",
-                       "l2": f"inputs rotate over {N_SETS} buffer sets (~{N_SETS * 59} MB), larger than L2",
+                       "l2": f"inputs rotate over {n_sets} buffer sets (~{n_sets * 59} MB), larger than L2",
+                       "launch": "steps replayed from CUDA graphs of the captured launch sequence",
                        "replicas": "independent replicas per GPU, no collective" if world > 1 else "single GPU"},
             "clocks": clk,
             "e2e": {"value": world * T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -475,6 +551,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="kvd", choices=["kvd", "reference"])
     ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--sets", type=int, default=N_SETS, help="rotating buffer sets (each ~59 MB)")
+    ap.add_argument("--profile", action="store_true", help="eager launches only, for a run under a profiler")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

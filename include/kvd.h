@@ -187,6 +187,16 @@ kvd_status kvd_memory_stats(const kvd_ctx *ctx, kvd_mem_stats *out);
  * KVD_ERR_POSITION. */
 kvd_status kvd_poll_status(kvd_ctx *ctx, void *stream);
 
+/* Diagnostic hook: attach (buf != NULL) or detach (buf == NULL) a DEVICE buffer of int64 slots that
+ * kvd_recompute_kv fills with a per-tile timeline in SM clock cycles: for CTA b and its i-th tile
+ * (i < 8) the 16 slots at ((b*8 + i)*16) hold
+ *   0 cycles the TMA producer waited for free stages   1/2 producer first / last issue
+ *   3 cycles the MMA issuer waited for data            4/5 MMA issue start / end
+ *   6/7 epilogue start / end     8 cycles the row-statistics warp waited   9 its total cycles
+ *   10 tile index                11 (tile 0 only) kernel start
+ * A call whose grid does not fit `bytes` records nothing.  No effect on results. */
+kvd_status kvd_set_trace(kvd_ctx *ctx, void *buf, size_t bytes);
+
 /* Number of kernels this context has launched since creation (all entry points). */
 uint64_t kvd_launch_count(const kvd_ctx *ctx);
 

@@ -32,7 +32,7 @@ KVD_MAX_SEGMENTS = 4
 EXPORTED_SYMBOLS = (
     "kvd_create", "kvd_destroy", "kvd_set_layer", "kvd_store_bytes", "kvd_attach_store", "kvd_reset_sequence",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
-    "kvd_decode_attention", "kvd_memory_stats", "kvd_poll_status", "kvd_launch_count", "kvd_last_cuda_error",
+    "kvd_decode_attention", "kvd_memory_stats", "kvd_poll_status", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
     "kvd_status_string", "kvd_version",
 )
 
@@ -113,6 +113,8 @@ def load() -> ctypes.CDLL:
     lib.kvd_memory_stats.restype = i32
     lib.kvd_poll_status.argtypes = [vp, vp]
     lib.kvd_poll_status.restype = i32
+    lib.kvd_set_trace.argtypes = [vp, vp, sz]
+    lib.kvd_set_trace.restype = i32
     lib.kvd_launch_count.argtypes = [vp]
     lib.kvd_launch_count.restype = ctypes.c_uint64
     lib.kvd_last_cuda_error.argtypes = [vp]
@@ -247,6 +249,13 @@ class Kvd:
 
     def kvd_poll_status(self, stream=None) -> int:
         return int(self._lib.kvd_poll_status(self._h, _stream(stream)))
+
+    def kvd_set_trace(self, buf) -> None:
+        if buf is None:
+            self._check(self._lib.kvd_set_trace(self._h, None, 0), "kvd_set_trace")
+        else:
+            self._keep.append(buf)
+            self._check(self._lib.kvd_set_trace(self._h, _ptr(buf), buf.numel() * buf.element_size()), "kvd_set_trace")
 
     def kvd_launch_count(self) -> int:
         return int(self._lib.kvd_launch_count(self._h))

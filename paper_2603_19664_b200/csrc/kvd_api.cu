@@ -156,7 +156,9 @@ static kvd_status encode_2d(kvd_ctx *ctx, CUtensorMap *map, const void *base, ui
   return KVD_OK;
 }
 
-// (cos, sin) tables of Eq. 11-12 split as position = 256*hi + lo; built in double on the host.
+// (cos, sin) tables of Eq. 11-12 split as position = 16*hi + lo; built in double on the host.
+// hi is row-major [hi][pair]; lo is pair-major [pair][lo] so that neighbouring positions read
+// neighbouring shared-memory words.
 static kvd_status get_rope(kvd_ctx *ctx, float theta, RopeTable *out) {
   uint32_t key;
   memcpy(&key, &theta, 4);
@@ -176,7 +178,7 @@ static kvd_status get_rope(kvd_ctx *ctx, float theta, RopeTable *out) {
     }
     for (int l = 0; l < ROPE_LO_SIZE; ++l) {
       const double a = static_cast<double>(l) * freq;
-      lo[static_cast<size_t>(l) * half + i] = make_float2(static_cast<float>(cos(a)), static_cast<float>(sin(a)));
+      lo[static_cast<size_t>(i) * ROPE_LO_SIZE + l] = make_float2(static_cast<float>(cos(a)), static_cast<float>(sin(a)));
     }
   }
   RopeTable t;
@@ -351,6 +353,12 @@ extern "C" kvd_status kvd_recompute_kv(kvd_ctx *ctx, int layer, const void *rows
   p.gamma_k = d.qk_norm ? ls.gamma_k : nullptr;
   p.status = ctx->d_status;
   p.timeout_ns = ctx->timeout_ns;
+  p.trace = nullptr;
+  if (ctx->trace) {
+    const int tiles = p.num_m_blocks * p.num_n_blocks;
+    const size_t ctas = tiles < ctx->num_sms ? tiles : ctx->num_sms;
+    if (ctas * RC_TRACE_TILES * RC_TRACE_FIELDS * sizeof(long long) <= ctx->trace_bytes) p.trace = ctx->trace;
+  }
   return launch_recompute(ctx, ls, tmap_a, p, static_cast<cudaStream_t>(stream_));
 }
 
@@ -488,6 +496,14 @@ extern "C" kvd_status kvd_poll_status(kvd_ctx *ctx, void *stream_) {
   }
   if (word & STATUS_TIMEOUT) return KVD_ERR_TIMEOUT;
   if (word & STATUS_POSITION) return KVD_ERR_POSITION;
+  return KVD_OK;
+}
+
+extern "C" kvd_status kvd_set_trace(kvd_ctx *ctx, void *buf, size_t bytes) {
+  if (!ctx) return KVD_ERR_INVALID_ARG;
+  if (buf && (reinterpret_cast<uintptr_t>(buf) & 7u) != 0) return KVD_ERR_ALIGNMENT;
+  ctx->trace = static_cast<long long *>(buf);
+  ctx->trace_bytes = buf ? bytes : 0;
   return KVD_OK;
 }
 

@@ -18,12 +18,14 @@ namespace kvd {
 constexpr int STATUS_TIMEOUT = 1;
 constexpr int STATUS_POSITION = 2;
 
-constexpr int ROPE_LO_BITS = 8;  // position = hi * 256 + lo; one table per part
+constexpr int ROPE_LO_BITS = 4;  // position = hi * 16 + lo; one table per part
 constexpr int ROPE_LO_SIZE = 1 << ROPE_LO_BITS;
 
 // ------------------------------------------------------------------------------ recompute GEMM
 constexpr int RC_BLOCK_M = 128;
 constexpr int RC_BLOCK_K = 64;
+constexpr int RC_TRACE_TILES = 8;    // tiles per CTA recorded when a trace buffer is attached
+constexpr int RC_TRACE_FIELDS = 16;  // int64 slots per (CTA, tile); see kvd_set_trace
 constexpr int RC_THREADS = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 row statistics, warps 6-9 epilogue
 
 struct RecomputeParams {
@@ -41,12 +43,13 @@ struct RecomputeParams {
   int qk_norm;
   float qk_eps;
   int rope_style;
-  const float2 *rope_hi;  // [n_hi][d_head/2] (cos, sin) of (pos & ~255) * freq_i
-  const float2 *rope_lo;  // [256][d_head/2]  (cos, sin) of (pos & 255) * freq_i
+  const float2 *rope_hi;  // [n_hi][d_head/2] (cos, sin) of (pos & ~15) * freq_i
+  const float2 *rope_lo;  // [d_head/2][16]   (cos, sin) of (pos & 15) * freq_i, pair-major
   int max_pos;            // positions must be in [0, max_pos)
   const float *gamma_k;   // [d_head] fp32 or nullptr
   int *status;
   unsigned long long timeout_ns;
+  long long *trace;  // nullptr unless a trace buffer is attached
 };
 
 // ------------------------------------------------------------------------------ decode attention
@@ -143,6 +146,8 @@ struct kvd_ctx {
   uint64_t launches = 0;
   uint64_t prepared_bytes = 0;
   unsigned long long timeout_ns = 2000000000ull;
+  long long *trace = nullptr;
+  size_t trace_bytes = 0;
   std::string last_error;
   kvd::EncodeTiledFn encode = nullptr;
 };

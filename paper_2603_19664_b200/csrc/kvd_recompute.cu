@@ -22,7 +22,7 @@
 
 namespace kvd {
 
-template <int BLOCK_N>
+template <int BLOCK_N, int D_HEAD>
 struct RcCfg {
   static constexpr int STAGES = BLOCK_N == 256 ? 4 : 6;
   static constexpr int A_BYTES = RC_BLOCK_M * RC_BLOCK_K * 2;
@@ -31,9 +31,17 @@ struct RcCfg {
   static constexpr int TMEM_COLS = 2 * BLOCK_N;
   // barriers: full[S], empty[S], tmem_full[2], tmem_empty[2], stats_full[2]
   static constexpr int NUM_BARS = 2 * STAGES + 6;
-  static constexpr int TAIL_BYTES = NUM_BARS * 8 + 16 /*tmem ptr, abort*/ + 2 * RC_BLOCK_M * 4 /*rstd*/ + 256 * 4 /*gamma_k*/;
+  static constexpr int ROPE_LO_BYTES = (D_HEAD / 2) * ROPE_LO_SIZE * 8;  // [pair][position low bits] (cos, sin)
+  static constexpr int TAIL_BYTES =
+      NUM_BARS * 8 + 16 /*tmem ptr, abort*/ + 2 * RC_BLOCK_M * 4 /*rstd*/ + 256 * 4 /*gamma_k*/ + ROPE_LO_BYTES;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + TAIL_BYTES + 1024 /*alignment slack*/;
 };
+
+// Optional per-tile timeline (SM clock cycles) for performance analysis; see kvd_set_trace.
+__device__ __forceinline__ void trace_put(long long *trace, int tile_iter, int field, long long v) {
+  if (trace != nullptr && tile_iter < RC_TRACE_TILES)
+    trace[(static_cast<size_t>(blockIdx.x) * RC_TRACE_TILES + tile_iter) * RC_TRACE_FIELDS + field] = v;
+}
 
 __device__ __forceinline__ void raise(int *status, int bit, volatile int *abort_flag) {
   atomicOr(status, bit);
@@ -44,7 +52,7 @@ template <int BLOCK_N, int D_HEAD>
 __global__ void __launch_bounds__(RC_THREADS, 1)
 kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                      const RecomputeParams p) {
-  using Cfg = RcCfg<BLOCK_N>;
+  using Cfg = RcCfg<BLOCK_N, D_HEAD>;
   constexpr int STAGES = Cfg::STAGES;
   static_assert(BLOCK_N % D_HEAD == 0, "a tile must hold whole heads");
 
@@ -56,6 +64,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
   float *s_rstd = reinterpret_cast<float *>(tail + Cfg::NUM_BARS * 8 + 16);
   float *s_gamma_k = s_rstd + 2 * RC_BLOCK_M;
+  float2 *s_rope_lo = reinterpret_cast<float2 *>(s_gamma_k + 256);
 
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_base = smem_u32(bars);
@@ -68,6 +77,23 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int num_tiles = p.num_m_blocks * p.num_n_blocks;
+  // Tile order: all key tiles first, then all value tiles, so that the last tile of a CTA (whose
+  // epilogue nothing overlaps) is a cheap value tile.  Falls back to row-major order when a tile
+  // mixes key and value heads.
+  const int nk_tiles = (p.k_cols % BLOCK_N == 0) ? p.k_cols / BLOCK_N : 0;
+  auto tile_coords = [&](int t, int &m0, int &n0) {
+    if (nk_tiles == 0) {
+      m0 = (t / p.num_n_blocks) * RC_BLOCK_M;
+      n0 = (t % p.num_n_blocks) * BLOCK_N;
+    } else if (t < p.num_m_blocks * nk_tiles) {
+      m0 = (t / nk_tiles) * RC_BLOCK_M;
+      n0 = (t % nk_tiles) * BLOCK_N;
+    } else {
+      const int u = t - p.num_m_blocks * nk_tiles, nv = p.num_n_blocks - nk_tiles;
+      m0 = (u / nv) * RC_BLOCK_M;
+      n0 = (nk_tiles + u % nv) * BLOCK_N;
+    }
+  };
   const unsigned long long tmo = p.timeout_ns;
 
   if (threadIdx.x == 0) {
@@ -86,6 +112,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     prefetch_tensormap(&tmap_b);
   }
   if (threadIdx.x < D_HEAD) s_gamma_k[threadIdx.x] = p.gamma_k ? p.gamma_k[threadIdx.x] : 1.0f;
+  for (int i = threadIdx.x; i < Cfg::ROPE_LO_BYTES / 16; i += RC_THREADS)
+    reinterpret_cast<float4 *>(s_rope_lo)[i] = reinterpret_cast<const float4 *>(p.rope_lo)[i];
   if (warp == 1) {
     tmem_alloc(smem_u32(s_tmem), Cfg::TMEM_COLS);
     tmem_relinquish();
@@ -94,6 +122,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
+  if (threadIdx.x == 0) trace_put(p.trace, 0, 11, clock64());
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -102,15 +131,20 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       uint32_t ph = 0;
       uint32_t issued = 0, issued_parity = 0;  // per-stage: a load is in flight with this parity
       bool ok = true;
-      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-        const int m0 = (t / p.num_n_blocks) * RC_BLOCK_M;
-        const int n0 = (t % p.num_n_blocks) * BLOCK_N;
+      int ti = 0;
+      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++ti) {
+        int m0, n0;
+        tile_coords(t, m0, n0);
+        long long waited = 0;
+        trace_put(p.trace, ti, 1, clock64());
         for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+          const long long w0 = p.trace ? clock64() : 0;
           if (!mbar_wait(bar_empty(s), ph ^ 1u, s_abort, tmo)) {
             raise(p.status, STATUS_TIMEOUT, s_abort);
             ok = false;
             break;
           }
+          if (p.trace) waited += clock64() - w0;
           mbar_arrive_expect_tx(bar_full(s), Cfg::STAGE_BYTES);
           const uint32_t a_dst = smem_base + s * Cfg::STAGE_BYTES;
           tma_load_2d(a_dst, &tmap_a, bar_full(s), kb * RC_BLOCK_K, m0);
@@ -122,6 +156,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
             ph ^= 1u;
           }
         }
+        trace_put(p.trace, ti, 0, waited);
+        trace_put(p.trace, ti, 2, clock64());
       }
       if (!ok) {
         // leave no bulk copy in flight behind us: wait (bounded) for every load already issued
@@ -142,19 +178,25 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       int s = 0, a = 0;
       uint32_t ph = 0, aph = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+      int ti = 0;
+      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++ti) {
         if (!mbar_wait(bar_tmem_empty(a), aph ^ 1u, s_abort, tmo)) {
           raise(p.status, STATUS_TIMEOUT, s_abort);
           break;
         }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + a * BLOCK_N;
+        long long waited = 0;
+        trace_put(p.trace, ti, 4, clock64());
+        trace_put(p.trace, ti, 10, t);
         for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+          const long long w0 = p.trace ? clock64() : 0;
           if (!mbar_wait(bar_full(s), ph, s_abort, tmo)) {
             raise(p.status, STATUS_TIMEOUT, s_abort);
             ok = false;
             break;
           }
+          if (p.trace) waited += clock64() - w0;
           tc_fence_after();
           const uint32_t a_addr = smem_base + s * Cfg::STAGE_BYTES;
           const uint64_t a_desc = umma_smem_desc_sw128(a_addr);
@@ -172,6 +214,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         }
         if (!ok) break;
         umma_commit(bar_tmem_full(a));
+        trace_put(p.trace, ti, 3, waited);
+        trace_put(p.trace, ti, 5, clock64());
         if (++a == 2) {
           a = 0;
           aph ^= 1u;
@@ -186,20 +230,27 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     int s = 0, a = 0;
     uint32_t ph = 0, aph = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+    int ti = 0;
+    for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++ti) {
+      long long waited = 0;
+      const long long st0 = p.trace ? clock64() : 0;
       // s_rstd[a] is free once the epilogue that read it released accumulator a
       // the whole warp takes the same branch: aligned instructions follow
       if (!__all_sync(0xffffffffu, mbar_wait(bar_tmem_empty(a), aph ^ 1u, s_abort, tmo))) {
         raise(p.status, STATUS_TIMEOUT, s_abort);
         break;
       }
-      float sum = 0.f;
+      // eight partial sums (one per element slot of a 16-byte chunk) keep the FMA chains short; they
+      // are combined in a fixed order below, the same for every row
+      float ps[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+        const long long w0 = p.trace ? clock64() : 0;
         if (!__all_sync(0xffffffffu, mbar_wait(bar_full(s), ph, s_abort, tmo))) {
           raise(p.status, STATUS_TIMEOUT, s_abort);
           ok = false;
           break;
         }
+        if (p.trace) waited += clock64() - w0;
         const uint32_t a_addr = smem_base + s * Cfg::STAGE_BYTES + row_off;
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
@@ -209,14 +260,14 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                        : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
                        : "r"(a_addr + ((static_cast<uint32_t>(c) << 4) ^ sw)));
           float x;
-          x = bf16_lo(w0); sum = fmaf(x, x, sum);
-          x = bf16_hi(w0); sum = fmaf(x, x, sum);
-          x = bf16_lo(w1); sum = fmaf(x, x, sum);
-          x = bf16_hi(w1); sum = fmaf(x, x, sum);
-          x = bf16_lo(w2); sum = fmaf(x, x, sum);
-          x = bf16_hi(w2); sum = fmaf(x, x, sum);
-          x = bf16_lo(w3); sum = fmaf(x, x, sum);
-          x = bf16_hi(w3); sum = fmaf(x, x, sum);
+          x = bf16_lo(w0); ps[0] = fmaf(x, x, ps[0]);
+          x = bf16_hi(w0); ps[1] = fmaf(x, x, ps[1]);
+          x = bf16_lo(w1); ps[2] = fmaf(x, x, ps[2]);
+          x = bf16_hi(w1); ps[3] = fmaf(x, x, ps[3]);
+          x = bf16_lo(w2); ps[4] = fmaf(x, x, ps[4]);
+          x = bf16_hi(w2); ps[5] = fmaf(x, x, ps[5]);
+          x = bf16_lo(w3); ps[6] = fmaf(x, x, ps[6]);
+          x = bf16_hi(w3); ps[7] = fmaf(x, x, ps[7]);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_empty(s));
@@ -226,8 +277,13 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         }
       }
       if (!ok) break;
+      const float sum = ((ps[0] + ps[1]) + (ps[2] + ps[3])) + ((ps[4] + ps[5]) + (ps[6] + ps[7]));
       s_rstd[a * RC_BLOCK_M + row] = 1.0f / sqrtf(sum * p.inv_d_hidden + p.rms_eps);
       mbar_arrive(bar_stats_full(a));
+      if (threadIdx.x == 64) {
+        trace_put(p.trace, ti, 8, waited);
+        trace_put(p.trace, ti, 9, clock64() - st0);
+      }
       if (++a == 2) {
         a = 0;
         aph ^= 1u;
@@ -241,15 +297,17 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     constexpr int HALF = D_HEAD / 2;
     int a = 0;
     uint32_t aph = 0;
-    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
-      const int m0 = (t / p.num_n_blocks) * RC_BLOCK_M;
-      const int n0 = (t % p.num_n_blocks) * BLOCK_N;
+    int ti = 0;
+    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++ti) {
+      int m0, n0;
+      tile_coords(t, m0, n0);
       const bool ready = mbar_wait(bar_tmem_full(a), aph, s_abort, tmo) && mbar_wait(bar_stats_full(a), aph, s_abort, tmo);
       if (!__all_sync(0xffffffffu, ready)) {  // warp-uniform: tcgen05.ld below is an aligned instruction
         raise(p.status, STATUS_TIMEOUT, s_abort);
         break;
       }
       tc_fence_after();
+      if (threadIdx.x == 6 * 32) trace_put(p.trace, ti, 6, clock64());
       const int m = m0 + row;
       const bool valid = m < p.M;
       const float rstd = s_rstd[a * RC_BLOCK_M + row];
@@ -258,8 +316,10 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         atomicOr(p.status, STATUS_POSITION);
         pos = pos < 0 ? 0 : p.max_pos - 1;
       }
-      const float2 *t_hi = p.rope_hi + static_cast<size_t>(pos >> ROPE_LO_BITS) * HALF;
-      const float2 *t_lo = p.rope_lo + static_cast<size_t>(pos & (ROPE_LO_SIZE - 1)) * HALF;
+      // (cos, sin) of pos * f_i = angle sum of the entries for (pos & ~15) [global, shared by 16
+      // neighbouring positions] and (pos & 15) [shared memory, laid out [pair][low bits]]
+      const float4 *t_hi = reinterpret_cast<const float4 *>(p.rope_hi + static_cast<size_t>(pos >> ROPE_LO_BITS) * HALF);
+      const float2 *t_lo = s_rope_lo + (pos & (ROPE_LO_SIZE - 1));
       const uint32_t acc = tmem_base + lane_field + a * BLOCK_N;
 
 #pragma unroll 1
@@ -304,20 +364,29 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
             kscale = rstd * (1.0f / sqrtf(ss * (1.0f / D_HEAD) + p.qk_eps));
           }
           if (p.rope_style == KVD_ROPE_INTERLEAVED) {
+            constexpr int NC = D_HEAD / 16;  // 16 columns = 8 rotation pairs per step
+            float4 hn[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) hn[j] = t_hi[j];
 #pragma unroll 1
-            for (int c = 0; c < D_HEAD / 16; ++c) {
+            for (int c = 0; c < NC; ++c) {
+              float4 h[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) h[j] = hn[j];
+              const int cn = c + 1 < NC ? c + 1 : c;  // prefetch the next step's table entries
+#pragma unroll
+              for (int j = 0; j < 4; ++j) hn[j] = t_hi[cn * 4 + j];
               uint32_t r[16];
               tmem_ld_x16(tcol + c * 16, r);
               tmem_wait_ld();
               uint32_t o[8];
 #pragma unroll
               for (int j = 0; j < 8; j += 2) {
-                // pairs i = c*8 + j, c*8 + j + 1: two (cos, sin) entries per 16-byte table load
-                const int i = c * 8 + j;
-                const float4 h = *reinterpret_cast<const float4 *>(t_hi + i);
-                const float4 l = *reinterpret_cast<const float4 *>(t_lo + i);
-                const float c0 = fmaf(h.x, l.x, -h.y * l.y), s0 = fmaf(h.y, l.x, h.x * l.y);
-                const float c1 = fmaf(h.z, l.z, -h.w * l.w), s1 = fmaf(h.w, l.z, h.z * l.w);
+                const int i = c * 8 + j;  // pairs i and i + 1
+                const float2 l0 = t_lo[i * ROPE_LO_SIZE], l1 = t_lo[(i + 1) * ROPE_LO_SIZE];
+                const float4 hh4 = h[j >> 1];
+                const float c0 = fmaf(hh4.x, l0.x, -hh4.y * l0.y), s0 = fmaf(hh4.y, l0.x, hh4.x * l0.y);
+                const float c1 = fmaf(hh4.z, l1.x, -hh4.w * l1.y), s1 = fmaf(hh4.w, l1.x, hh4.z * l1.y);
                 const float a0 = __uint_as_float(r[2 * j]) * kscale * s_gamma_k[c * 16 + 2 * j];
                 const float b0 = __uint_as_float(r[2 * j + 1]) * kscale * s_gamma_k[c * 16 + 2 * j + 1];
                 const float a1 = __uint_as_float(r[2 * j + 2]) * kscale * s_gamma_k[c * 16 + 2 * j + 2];
@@ -332,8 +401,18 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
               }
             }
           } else {
+            constexpr int NC = HALF / 16;  // 16 pairs (i, i + HALF) per step
+            float4 hn[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) hn[j] = t_hi[j];
 #pragma unroll 1
-            for (int c = 0; c < HALF / 16; ++c) {
+            for (int c = 0; c < NC; ++c) {
+              float4 h[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) h[j] = hn[j];
+              const int cn = c + 1 < NC ? c + 1 : c;
+#pragma unroll
+              for (int j = 0; j < 8; ++j) hn[j] = t_hi[cn * 8 + j];
               uint32_t ra[16], rb[16];
               tmem_ld_x16(tcol + c * 16, ra);
               tmem_ld_x16(tcol + HALF + c * 16, rb);
@@ -341,11 +420,11 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
               uint32_t oa[8], ob[8];
 #pragma unroll
               for (int j = 0; j < 16; j += 2) {
-                const int i = c * 16 + j;  // pair (i, i + HALF)
-                const float4 h = *reinterpret_cast<const float4 *>(t_hi + i);
-                const float4 l = *reinterpret_cast<const float4 *>(t_lo + i);
-                const float c0 = fmaf(h.x, l.x, -h.y * l.y), s0 = fmaf(h.y, l.x, h.x * l.y);
-                const float c1 = fmaf(h.z, l.z, -h.w * l.w), s1 = fmaf(h.w, l.z, h.z * l.w);
+                const int i = c * 16 + j;  // pairs (i, i + HALF) and (i + 1, i + 1 + HALF)
+                const float2 l0 = t_lo[i * ROPE_LO_SIZE], l1 = t_lo[(i + 1) * ROPE_LO_SIZE];
+                const float4 hh4 = h[j >> 1];
+                const float c0 = fmaf(hh4.x, l0.x, -hh4.y * l0.y), s0 = fmaf(hh4.y, l0.x, hh4.x * l0.y);
+                const float c1 = fmaf(hh4.z, l1.x, -hh4.w * l1.y), s1 = fmaf(hh4.w, l1.x, hh4.z * l1.y);
                 const float a0 = __uint_as_float(ra[j]) * kscale * s_gamma_k[i];
                 const float b0 = __uint_as_float(rb[j]) * kscale * s_gamma_k[i + HALF];
                 const float a1 = __uint_as_float(ra[j + 1]) * kscale * s_gamma_k[i + 1];
@@ -369,6 +448,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tmem_empty(a));
+      if (threadIdx.x == 6 * 32) trace_put(p.trace, ti, 7, clock64());
       if (++a == 2) {
         a = 0;
         aph ^= 1u;
@@ -388,7 +468,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
 template <int BLOCK_N, int D_HEAD>
 static kvd_status launch_impl(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_a, const RecomputeParams &p,
                               cudaStream_t stream) {
-  using Cfg = RcCfg<BLOCK_N>;
+  using Cfg = RcCfg<BLOCK_N, D_HEAD>;
   auto kern = kvd_recompute_kernel<BLOCK_N, D_HEAD>;
   static bool configured[64] = {};
   if (!configured[ctx->device & 63]) {
