@@ -226,7 +226,7 @@ extern "C" kvd_status kvd_set_layer(kvd_ctx *ctx, int layer, const kvd_layer_des
   }
   st = get_rope(ctx, ld->rope_theta, &ls.rope);
   if (st != KVD_OK) return st;
-  st = encode_2d(ctx, &ls.tmap_b, ls.wt, d.d_hidden, n_cols, RC_BLOCK_K, ctx->block_n);
+  st = encode_2d(ctx, &ls.tmap_b, ls.wt, d.d_hidden, n_cols, RC_BLOCK_K, ctx->block_n / 2);  // half tile per CTA
   if (st != KVD_OK) return st;
   e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "kvd_set_layer sync");
@@ -335,7 +335,7 @@ extern "C" kvd_status kvd_recompute_kv(kvd_ctx *ctx, int layer, const void *rows
   RecomputeParams p;
   p.M = n;
   p.num_k_blocks = d.d_hidden / RC_BLOCK_K;
-  p.num_m_blocks = (n + RC_BLOCK_M - 1) / RC_BLOCK_M;
+  p.num_m_blocks = (n + 2 * RC_BLOCK_M - 1) / (2 * RC_BLOCK_M);  // 256-row tiles, 128 rows per CTA of a pair
   p.num_n_blocks = 2 * kdim / ctx->block_n;
   p.k_cols = kdim;
   p.positions = a_pos;
@@ -356,7 +356,7 @@ extern "C" kvd_status kvd_recompute_kv(kvd_ctx *ctx, int layer, const void *rows
   p.trace = nullptr;
   if (ctx->trace) {
     const int tiles = p.num_m_blocks * p.num_n_blocks;
-    const size_t ctas = tiles < ctx->num_sms ? tiles : ctx->num_sms;
+    const size_t ctas = 2 * static_cast<size_t>(tiles < ctx->num_sms / 2 ? tiles : ctx->num_sms / 2);
     if (ctas * RC_TRACE_TILES * RC_TRACE_FIELDS * sizeof(long long) <= ctx->trace_bytes) p.trace = ctx->trace;
   }
   return launch_recompute(ctx, ls, tmap_a, p, static_cast<cudaStream_t>(stream_));

@@ -26,7 +26,7 @@ constexpr int RC_BLOCK_M = 128;
 constexpr int RC_BLOCK_K = 64;
 constexpr int RC_TRACE_TILES = 8;    // tiles per CTA recorded when a trace buffer is attached
 constexpr int RC_TRACE_FIELDS = 16;  // int64 slots per (CTA, tile); see kvd_set_trace
-constexpr int RC_THREADS = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 row statistics, warps 6-9 epilogue
+constexpr int RC_THREADS = 320;  // warp 2 TMA, warp 3 MMA, warps 0,1,8,9 row statistics, warps 4-7 epilogue
 
 struct RecomputeParams {
   int M;          // rows

@@ -56,10 +56,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 
 // Bounded wait: returns false when `timeout_ns` elapsed or another thread of the CTA raised the
-// abort flag.  Never spins forever.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag,
-                                          unsigned long long timeout_ns) {
-  if (mbar_try_wait(bar, parity)) return true;
+// abort flag.  Never spins forever.  The slow path (timer, abort flag) is kept out of line so that
+// a wait on a barrier that has already completed costs one try_wait.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const volatile int *abort_flag,
+                                            unsigned long long timeout_ns) {
   const unsigned long long t0 = globaltimer_ns();
   uint32_t it = 0;
   while (true) {
@@ -69,6 +69,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const v
       if (globaltimer_ns() - t0 > timeout_ns) return false;
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag,
+                                          unsigned long long timeout_ns) {
+  if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, timeout_ns);
 }
 
 // ------------------------------------------------------------------------------ TMA
@@ -135,6 +141,64 @@ __device__ __forceinline__ void tmem_ld_x16(uint32_t taddr, uint32_t (&r)[16]) {
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr)
       : "memory");
+}
+
+// ------------------------------------------------------------------------------ CTA pairs (cluster of 2)
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Barrier over all threads of the cluster; orders shared-memory initialisation before remote use.
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+// Arrive on an mbarrier that lives in another CTA of the cluster (address from map_to_cta).
+// Relaxed on purpose: a cluster-scope release makes the issuing thread wait for every outstanding
+// memory operation of a busy SM (measured: 700-1300 clocks inside the GEMM main loop against ~130
+// relaxed).  The callers use it only as a "you may now look" token for data that the async proxy
+// (TMA, tcgen05) wrote to shared memory / TMEM and whose completion the caller itself observed on
+// a local mbarrier; the signalling thread has no writes of its own to publish.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMEM management and MMA for a pair of CTAs (cta_group::2).  alloc / dealloc / relinquish are
+// executed by the same warp index in both CTAs; the MMA and its commits by one thread of the
+// even-ranked CTA only.
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_result, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B with M = 256 split over the pair (128 rows per CTA) and the
+// N columns of B split over the pair's shared memories (N/2 rows of the K-major tile per CTA).
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrive on the barrier at the same shared-memory offset in every CTA named by `cta_mask`, once all
+// MMAs this thread issued so far have finished.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t cta_mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(cta_mask)
+               : "memory");
 }
 
 // Shared-memory matrix descriptor for a K-major bf16 operand tile whose rows are 128 bytes

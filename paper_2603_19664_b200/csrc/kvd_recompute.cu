@@ -5,18 +5,30 @@
 //   K heads: optional RMS norm over d_head, scale gamma_k, rotation by the row's position
 //   K, V stored as bf16
 //
-// One persistent CTA per SM walks over 128 x BLOCK_N output tiles.  Warp roles:
-//   warp 0      TMA producer: 128x64 tile of X and BLOCK_Nx64 tile of W' per pipeline stage
-//   warp 1      owns TMEM; one lane issues tcgen05.mma (128 x BLOCK_N x 16 per instruction)
-//   warps 2-5   row statistics: each thread sums x^2 of one row from the X tiles as they land
-//   warps 6-9   epilogue: tcgen05.ld the fp32 accumulator, normalise, rotate, convert, store
+// Persistent CTA pairs (clusters of two, one CTA per SM) walk over 256 x BLOCK_N output tiles with
+// tcgen05.mma.cta_group::2: each CTA owns 128 rows of the tile and stages, per 64-wide k block, its
+// own 128x64 tile of X plus HALF of the BLOCK_Nx64 tile of W'; the tensor cores of the pair read
+// both halves, so a k block costs each SM 32 KB of L2 traffic instead of 48 KB.  Warp roles:
+//   warp 2         TMA producer (one lane; local tiles, local barrier)
+//   warp 3         even CTA: one lane issues the MMAs for the pair and commits to both CTAs' barriers
+//                  odd CTA:  one lane relays "my stage has landed" to the even CTA; owns TMEM alloc
+//   warps 0,1,8,9  row statistics: each thread sums x^2 of one row from the X tiles as they land
+//   warps 4-7      epilogue: tcgen05.ld the fp32 accumulator, normalise, rotate, convert, store
+// Warp w runs on scheduler w % 4, so the two single-thread roles (warps 2, 3) share their scheduler
+// with one epilogue warp only; the statistics warps sit on the other two schedulers.
 // The accumulator is double-buffered in TMEM (2 x BLOCK_N columns) so the epilogue of tile i
 // overlaps the main loop of tile i+1.
 //
+// The producer and the MMA issuer are single threads whose loop must finish well inside the 512
+// clocks a k block of MMAs takes; their loops are therefore kept to a few dozen instructions
+// (incremental addresses, one asm block per k block).  Every wait is bounded; on expiry the kernel records STATUS_TIMEOUT and drains.
+//
 // Bit-reproducibility: the k loop always runs over all of d_hidden in ascending order with one MMA
-// shape, row sums are taken thread-locally in ascending channel order, the key norm is reduced by
-// the single thread that owns the row, and cos/sin depend on (position, channel) only.  A row's
-// output bits are therefore independent of M and of the row's index.
+// shape, row sums are taken thread-locally in a fixed order, the key norm is reduced by the single
+// thread that owns the row, and cos/sin depend on (position, channel) only.  A row's output bits
+// are therefore independent of M and of the row's index.
+#include <string.h>
+
 #include "kvd_internal.h"
 #include "kvd_ptx.cuh"
 
@@ -24,13 +36,14 @@ namespace kvd {
 
 template <int BLOCK_N, int D_HEAD>
 struct RcCfg {
-  static constexpr int STAGES = BLOCK_N == 256 ? 4 : 6;
+  static constexpr int STAGES = BLOCK_N == 256 ? 6 : 8;
   static constexpr int A_BYTES = RC_BLOCK_M * RC_BLOCK_K * 2;
-  static constexpr int B_BYTES = BLOCK_N * RC_BLOCK_K * 2;
+  static constexpr int B_ROWS = BLOCK_N / 2;  // this CTA's half of the W' tile
+  static constexpr int B_BYTES = B_ROWS * RC_BLOCK_K * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = 2 * BLOCK_N;
-  // barriers: full[S], empty[S], tmem_full[2], tmem_empty[2], stats_full[2]
-  static constexpr int NUM_BARS = 2 * STAGES + 6;
+  // barriers: full[S], empty[S], peer_full[S], tmem_full[2], tmem_empty[2], stats_full[2], rstd_free[2]
+  static constexpr int NUM_BARS = 3 * STAGES + 8;
   static constexpr int ROPE_LO_BYTES = (D_HEAD / 2) * ROPE_LO_SIZE * 8;  // [pair][position low bits] (cos, sin)
   static constexpr int TAIL_BYTES =
       NUM_BARS * 8 + 16 /*tmem ptr, abort*/ + 2 * RC_BLOCK_M * 4 /*rstd*/ + 256 * 4 /*gamma_k*/ + ROPE_LO_BYTES;
@@ -38,9 +51,24 @@ struct RcCfg {
 };
 
 // Optional per-tile timeline (SM clock cycles) for performance analysis; see kvd_set_trace.
+template <bool TRACE>
 __device__ __forceinline__ void trace_put(long long *trace, int tile_iter, int field, long long v) {
-  if (trace != nullptr && tile_iter < RC_TRACE_TILES)
+  if (TRACE && tile_iter < RC_TRACE_TILES)
     trace[(static_cast<size_t>(blockIdx.x) * RC_TRACE_TILES + tile_iter) * RC_TRACE_FIELDS + field] = v;
+}
+template <bool TRACE>
+__device__ __forceinline__ void trace_put(long long *trace, int tile_iter, int field) {
+  if (TRACE) trace_put<TRACE>(trace, tile_iter, field, clock64());
+}
+
+// One lane waits on the barrier, the result is broadcast: the other 31 lanes do not poll shared
+// memory.  The shuffle also orders the lanes' later reads after lane 0's acquire.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag,
+                                          unsigned long long timeout_ns, int lane) {
+  int ok = 1;
+  if (lane == 0) ok = mbar_wait(bar, parity, abort_flag, timeout_ns) ? 1 : 0;
+  ok = __shfl_sync(0xffffffffu, ok, 0);
+  return ok != 0;
 }
 
 __device__ __forceinline__ void raise(int *status, int bit, volatile int *abort_flag) {
@@ -48,7 +76,45 @@ __device__ __forceinline__ void raise(int *status, int bit, volatile int *abort_
   *abort_flag = 1;
 }
 
-template <int BLOCK_N, int D_HEAD>
+// One k block (64 channels = four K=16 steps) of the pair MMA followed by the commit that frees the
+// stage in both CTAs.  a_lo / b_lo are the low words of the shared-memory descriptors of the stage
+// (the K step advances the start-address field by 32 bytes = 2 units); desc_hi is their common
+// high word.  `acc_first` = 0 makes the first step overwrite the accumulator.
+__device__ __forceinline__ void umma_kblock_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                                 uint32_t idesc, uint32_t acc_first, uint32_t bar_empty) {
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p, t;\n\t"
+      ".reg .b64 da, db;\n\t"
+      ".reg .b32 la, lb;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "setp.eq.b32 t, 0, 0;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t"
+      "add.u32 la, %1, 2;\n\t"
+      "add.u32 lb, %2, 2;\n\t"
+      "mov.b64 da, {la, %3};\n\t"
+      "mov.b64 db, {lb, %3};\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, t;\n\t"
+      "add.u32 la, %1, 4;\n\t"
+      "add.u32 lb, %2, 4;\n\t"
+      "mov.b64 da, {la, %3};\n\t"
+      "mov.b64 db, {lb, %3};\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, t;\n\t"
+      "add.u32 la, %1, 6;\n\t"
+      "add.u32 lb, %2, 6;\n\t"
+      "mov.b64 da, {la, %3};\n\t"
+      "mov.b64 db, {lb, %3};\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, t;\n\t"
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%6], %7;\n\t"
+      "}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc_first), "r"(bar_empty),
+        "h"(static_cast<uint16_t>(3))
+      : "memory");
+}
+
+template <int BLOCK_N, int D_HEAD, bool TRACE>
 __global__ void __launch_bounds__(RC_THREADS, 1)
 kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                      const RecomputeParams p) {
@@ -70,9 +136,14 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   const uint32_t bar_base = smem_u32(bars);
   auto bar_full = [&](int s) { return bar_base + 8u * s; };
   auto bar_empty = [&](int s) { return bar_base + 8u * (STAGES + s); };
-  auto bar_tmem_full = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
-  auto bar_tmem_empty = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
-  auto bar_stats_full = [&](int a) { return bar_base + 8u * (2 * STAGES + 4 + a); };
+  auto bar_peer_full = [&](int s) { return bar_base + 8u * (2 * STAGES + s); };  // even CTA only
+  auto bar_tmem_full = [&](int a) { return bar_base + 8u * (3 * STAGES + a); };
+  auto bar_tmem_empty = [&](int a) { return bar_base + 8u * (3 * STAGES + 2 + a); };  // even CTA only
+  auto bar_stats_full = [&](int a) { return bar_base + 8u * (3 * STAGES + 4 + a); };
+  auto bar_rstd_free = [&](int a) { return bar_base + 8u * (3 * STAGES + 6 + a); };
+  const uint32_t cta_rank = cluster_ctarank();  // 0: issues the MMAs, 1: its partner
+  const int cluster_id = static_cast<int>(blockIdx.x >> 1);
+  const int num_clusters = static_cast<int>(gridDim.x >> 1);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -83,16 +154,17 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   const int nk_tiles = (p.k_cols % BLOCK_N == 0) ? p.k_cols / BLOCK_N : 0;
   auto tile_coords = [&](int t, int &m0, int &n0) {
     if (nk_tiles == 0) {
-      m0 = (t / p.num_n_blocks) * RC_BLOCK_M;
+      m0 = (t / p.num_n_blocks) * (2 * RC_BLOCK_M);
       n0 = (t % p.num_n_blocks) * BLOCK_N;
     } else if (t < p.num_m_blocks * nk_tiles) {
-      m0 = (t / nk_tiles) * RC_BLOCK_M;
+      m0 = (t / nk_tiles) * (2 * RC_BLOCK_M);
       n0 = (t % nk_tiles) * BLOCK_N;
     } else {
       const int u = t - p.num_m_blocks * nk_tiles, nv = p.num_n_blocks - nk_tiles;
-      m0 = (u / nv) * RC_BLOCK_M;
+      m0 = (u / nv) * (2 * RC_BLOCK_M);
       n0 = (nk_tiles + u % nv) * BLOCK_N;
     }
+    m0 += static_cast<int>(cta_rank) * RC_BLOCK_M;  // this CTA's 128 rows of the 256-row tile
   };
   const unsigned long long tmo = p.timeout_ns;
 
@@ -100,11 +172,13 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(bar_full(s), 1);
       mbar_init(bar_empty(s), 1 + 4);  // MMA commit + one arrival per statistics warp
+      mbar_init(bar_peer_full(s), 1);  // the partner's relay
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tmem_full(a), 1);
-      mbar_init(bar_tmem_empty(a), 4);          // one arrival per epilogue warp
+      mbar_init(bar_tmem_empty(a), 8);           // one arrival per epilogue warp of both CTAs
       mbar_init(bar_stats_full(a), RC_BLOCK_M);  // one arrival per statistics thread
+      mbar_init(bar_rstd_free(a), 4);            // one arrival per local epilogue warp
     }
     *s_abort = 0;
     fence_mbar_init();
@@ -114,72 +188,88 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   if (threadIdx.x < D_HEAD) s_gamma_k[threadIdx.x] = p.gamma_k ? p.gamma_k[threadIdx.x] : 1.0f;
   for (int i = threadIdx.x; i < Cfg::ROPE_LO_BYTES / 16; i += RC_THREADS)
     reinterpret_cast<float4 *>(s_rope_lo)[i] = reinterpret_cast<const float4 *>(p.rope_lo)[i];
-  if (warp == 1) {
-    tmem_alloc(smem_u32(s_tmem), Cfg::TMEM_COLS);
-    tmem_relinquish();
+  if (warp == 3) {
+    tmem_alloc_pair(smem_u32(s_tmem), Cfg::TMEM_COLS);
+    tmem_relinquish_pair();
   }
   tc_fence_before();
-  __syncthreads();
+  cluster_sync_all();  // barriers of both CTAs are initialised before anyone signals across the pair
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
-  if (threadIdx.x == 0) trace_put(p.trace, 0, 11, clock64());
+  if (threadIdx.x == 0) trace_put<TRACE>(p.trace, 0, 11);
 
-  if (warp == 0) {
+  if (warp == 2) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int s = 0;
+      int s = 0, n_issued = 0;
       uint32_t ph = 0;
-      uint32_t issued = 0, issued_parity = 0;  // per-stage: a load is in flight with this parity
+      uint32_t full = bar_full(0), empty = bar_empty(0), dst = smem_base;
+      const int b_row_off = static_cast<int>(cta_rank) * Cfg::B_ROWS;
       bool ok = true;
       int ti = 0;
-      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++ti) {
+      for (int t = cluster_id; t < num_tiles && ok; t += num_clusters, ++ti) {
         int m0, n0;
         tile_coords(t, m0, n0);
+        n0 += b_row_off;
         long long waited = 0;
-        trace_put(p.trace, ti, 1, clock64());
-        for (int kb = 0; kb < p.num_k_blocks; ++kb) {
-          const long long w0 = p.trace ? clock64() : 0;
-          if (!mbar_wait(bar_empty(s), ph ^ 1u, s_abort, tmo)) {
+        trace_put<TRACE>(p.trace, ti, 1);
+        for (int k0 = 0; k0 < p.num_k_blocks * RC_BLOCK_K; k0 += RC_BLOCK_K) {
+          const long long w0 = TRACE ? clock64() : 0;
+          if (!mbar_wait(empty, ph ^ 1u, s_abort, tmo)) {
             raise(p.status, STATUS_TIMEOUT, s_abort);
             ok = false;
             break;
           }
-          if (p.trace) waited += clock64() - w0;
-          mbar_arrive_expect_tx(bar_full(s), Cfg::STAGE_BYTES);
-          const uint32_t a_dst = smem_base + s * Cfg::STAGE_BYTES;
-          tma_load_2d(a_dst, &tmap_a, bar_full(s), kb * RC_BLOCK_K, m0);
-          tma_load_2d(a_dst + Cfg::A_BYTES, &tmap_b, bar_full(s), kb * RC_BLOCK_K, n0);
-          issued |= 1u << s;
-          issued_parity = (issued_parity & ~(1u << s)) | (ph << s);
+          if (TRACE) waited += clock64() - w0;
+          mbar_arrive_expect_tx(full, Cfg::STAGE_BYTES);
+          tma_load_2d(dst, &tmap_a, full, k0, m0);
+          tma_load_2d(dst + Cfg::A_BYTES, &tmap_b, full, k0, n0);
+          ++n_issued;
+          full += 8u;
+          empty += 8u;
+          dst += Cfg::STAGE_BYTES;
           if (++s == STAGES) {
             s = 0;
             ph ^= 1u;
+            full = bar_full(0);
+            empty = bar_empty(0);
+            dst = smem_base;
           }
         }
-        trace_put(p.trace, ti, 0, waited);
-        trace_put(p.trace, ti, 2, clock64());
+        trace_put<TRACE>(p.trace, ti, 0, waited);
+        trace_put<TRACE>(p.trace, ti, 2);
       }
       if (!ok) {
-        // leave no bulk copy in flight behind us: wait (bounded) for every load already issued
+        // leave no bulk copy in flight behind us: wait (bounded) for every load already issued.
+        // Stages below s were last filled in the current round (parity ph), the others in the
+        // previous round.
         for (int i = 0; i < STAGES; ++i) {
-          if (issued & (1u << i)) {
+          if (n_issued > i) {
+            const uint32_t par = i < s ? ph : ph ^ 1u;
             const unsigned long long t0 = globaltimer_ns();
-            while (!mbar_try_wait(bar_full(i), (issued_parity >> i) & 1u)) {
+            while (!mbar_try_wait(bar_full(i), par)) {
               if (globaltimer_ns() - t0 > 100000000ull) break;
             }
           }
         }
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16_f32(RC_BLOCK_M, BLOCK_N);
+  } else if (warp == 3) {
+    if (lane == 0 && cta_rank == 0) {
+      // ---------------------------------------------------------------- MMA issuer (even CTA)
+      constexpr uint32_t idesc = umma_idesc_bf16_f32(2 * RC_BLOCK_M, BLOCK_N);
+      // descriptor words for 128-byte-swizzled K-major tiles: low = start address >> 4 | LBO field (1),
+      // high = SBO (1024 B >> 4) | version 1 (bit 46) | swizzle mode 2 (bits 61-63)
+      constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+      const uint32_t a_lo0 = ((smem_base & 0x3FFFFu) >> 4) | (1u << 16);
+      constexpr uint32_t stage_units = Cfg::STAGE_BYTES >> 4, b_off_units = Cfg::A_BYTES >> 4;
       int s = 0, a = 0;
       uint32_t ph = 0, aph = 0;
+      uint32_t full = bar_full(0), peer = bar_peer_full(0), empty = bar_empty(0), a_lo = a_lo0;
       bool ok = true;
       int ti = 0;
-      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++ti) {
+      for (int t = cluster_id; t < num_tiles && ok; t += num_clusters, ++ti) {
+        // both CTAs' epilogues have drained accumulator a
         if (!mbar_wait(bar_tmem_empty(a), aph ^ 1u, s_abort, tmo)) {
           raise(p.status, STATUS_TIMEOUT, s_abort);
           break;
@@ -187,56 +277,84 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + a * BLOCK_N;
         long long waited = 0;
-        trace_put(p.trace, ti, 4, clock64());
-        trace_put(p.trace, ti, 10, t);
+        trace_put<TRACE>(p.trace, ti, 4);
+        trace_put<TRACE>(p.trace, ti, 10, t);
         for (int kb = 0; kb < p.num_k_blocks; ++kb) {
-          const long long w0 = p.trace ? clock64() : 0;
-          if (!mbar_wait(bar_full(s), ph, s_abort, tmo)) {
+          const long long w0 = TRACE ? clock64() : 0;
+          // stage s has landed here and (relayed) in the partner CTA
+          if (!mbar_wait(full, ph, s_abort, tmo) || !mbar_wait(peer, ph, s_abort, tmo)) {
             raise(p.status, STATUS_TIMEOUT, s_abort);
             ok = false;
             break;
           }
-          if (p.trace) waited += clock64() - w0;
+          if (TRACE) waited += clock64() - w0;
           tc_fence_after();
-          const uint32_t a_addr = smem_base + s * Cfg::STAGE_BYTES;
-          const uint64_t a_desc = umma_smem_desc_sw128(a_addr);
-          const uint64_t b_desc = umma_smem_desc_sw128(a_addr + Cfg::A_BYTES);
-#pragma unroll
-          for (int k = 0; k < RC_BLOCK_K / 16; ++k) {
-            // 16 bf16 = 32 bytes along K inside the 128-byte swizzle row: +2 in the address field
-            umma_bf16(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-          }
-          umma_commit(bar_empty(s));
+          umma_kblock_pair(d_tmem, a_lo, a_lo + b_off_units, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
+          full += 8u;
+          peer += 8u;
+          empty += 8u;
+          a_lo += stage_units;
           if (++s == STAGES) {
             s = 0;
             ph ^= 1u;
+            full = bar_full(0);
+            peer = bar_peer_full(0);
+            empty = bar_empty(0);
+            a_lo = a_lo0;
           }
         }
         if (!ok) break;
-        umma_commit(bar_tmem_full(a));
-        trace_put(p.trace, ti, 3, waited);
-        trace_put(p.trace, ti, 5, clock64());
+        umma_commit_pair(bar_tmem_full(a), 3);  // accumulator a is complete in both CTAs
+        trace_put<TRACE>(p.trace, ti, 3, waited);
+        trace_put<TRACE>(p.trace, ti, 5);
         if (++a == 2) {
           a = 0;
           aph ^= 1u;
         }
       }
+    } else if (lane == 0) {
+      // ---------------------------------------------------------------- relay (odd CTA)
+      // tells the MMA issuer that this CTA's copy of stage s has landed
+      int s = 0;
+      uint32_t ph = 0;
+      uint32_t full = bar_full(0);
+      const uint32_t peer0 = map_to_cta(bar_peer_full(0), 0);
+      uint32_t peer = peer0;
+      bool ok = true;
+      for (int t = cluster_id; t < num_tiles && ok; t += num_clusters) {
+        for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+          if (!mbar_wait(full, ph, s_abort, tmo)) {
+            raise(p.status, STATUS_TIMEOUT, s_abort);
+            ok = false;
+            break;
+          }
+          mbar_arrive_cluster(peer);
+          full += 8u;
+          peer += 8u;
+          if (++s == STAGES) {
+            s = 0;
+            ph ^= 1u;
+            full = bar_full(0);
+            peer = peer0;
+          }
+        }
+      }
     }
-  } else if (warp < 6) {
+  } else if (warp < 2 || warp >= 8) {
     // ------------------------------------------------------------------ row statistics (Eq. 2)
-    const int row = (warp - 2) * 32 + lane;
+    const int row = (warp < 2 ? warp : warp - 6) * 32 + lane;  // warps 0, 1, 8, 9 -> rows 0..127
     const uint32_t row_off = row * 128u;
     const uint32_t sw = (row & 7u) << 4;
     int s = 0, a = 0;
     uint32_t ph = 0, aph = 0;
     bool ok = true;
     int ti = 0;
-    for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++ti) {
+    for (int t = cluster_id; t < num_tiles && ok; t += num_clusters, ++ti) {
       long long waited = 0;
-      const long long st0 = p.trace ? clock64() : 0;
-      // s_rstd[a] is free once the epilogue that read it released accumulator a
+      const long long st0 = TRACE ? clock64() : 0;
+      // s_rstd[a] is free once the local epilogue that read it has finished with accumulator a
       // the whole warp takes the same branch: aligned instructions follow
-      if (!__all_sync(0xffffffffu, mbar_wait(bar_tmem_empty(a), aph ^ 1u, s_abort, tmo))) {
+      if (!warp_wait(bar_rstd_free(a), aph ^ 1u, s_abort, tmo, lane)) {
         raise(p.status, STATUS_TIMEOUT, s_abort);
         break;
       }
@@ -244,13 +362,13 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       // are combined in a fixed order below, the same for every row
       float ps[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       for (int kb = 0; kb < p.num_k_blocks; ++kb) {
-        const long long w0 = p.trace ? clock64() : 0;
-        if (!__all_sync(0xffffffffu, mbar_wait(bar_full(s), ph, s_abort, tmo))) {
+        const long long w0 = TRACE ? clock64() : 0;
+        if (!warp_wait(bar_full(s), ph, s_abort, tmo, lane)) {
           raise(p.status, STATUS_TIMEOUT, s_abort);
           ok = false;
           break;
         }
-        if (p.trace) waited += clock64() - w0;
+        if (TRACE) waited += clock64() - w0;
         const uint32_t a_addr = smem_base + s * Cfg::STAGE_BYTES + row_off;
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
@@ -280,16 +398,16 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       const float sum = ((ps[0] + ps[1]) + (ps[2] + ps[3])) + ((ps[4] + ps[5]) + (ps[6] + ps[7]));
       s_rstd[a * RC_BLOCK_M + row] = 1.0f / sqrtf(sum * p.inv_d_hidden + p.rms_eps);
       mbar_arrive(bar_stats_full(a));
-      if (threadIdx.x == 64) {
-        trace_put(p.trace, ti, 8, waited);
-        trace_put(p.trace, ti, 9, clock64() - st0);
+      if (TRACE && threadIdx.x == 0) {
+        trace_put<TRACE>(p.trace, ti, 8, waited);
+        trace_put<TRACE>(p.trace, ti, 9, clock64() - st0);
       }
       if (++a == 2) {
         a = 0;
         aph ^= 1u;
       }
     }
-  } else {
+  } else if (warp >= 4 && warp < 8) {
     // ------------------------------------------------------------------ epilogue
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
     const int row = quarter * 32 + lane;
@@ -298,16 +416,16 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     int a = 0;
     uint32_t aph = 0;
     int ti = 0;
-    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++ti) {
+    for (int t = cluster_id; t < num_tiles; t += num_clusters, ++ti) {
       int m0, n0;
       tile_coords(t, m0, n0);
-      const bool ready = mbar_wait(bar_tmem_full(a), aph, s_abort, tmo) && mbar_wait(bar_stats_full(a), aph, s_abort, tmo);
-      if (!__all_sync(0xffffffffu, ready)) {  // warp-uniform: tcgen05.ld below is an aligned instruction
+      // warp-uniform outcome: tcgen05.ld below is an aligned instruction
+      if (!warp_wait(bar_tmem_full(a), aph, s_abort, tmo, lane) || !warp_wait(bar_stats_full(a), aph, s_abort, tmo, lane)) {
         raise(p.status, STATUS_TIMEOUT, s_abort);
         break;
       }
       tc_fence_after();
-      if (threadIdx.x == 6 * 32) trace_put(p.trace, ti, 6, clock64());
+      if (TRACE && threadIdx.x == 4 * 32) trace_put<TRACE>(p.trace, ti, 6);
       const int m = m0 + row;
       const bool valid = m < p.M;
       const float rstd = s_rstd[a * RC_BLOCK_M + row];
@@ -447,8 +565,12 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       // accumulator a (and s_rstd[a]) may be overwritten now
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_tmem_empty(a));
-      if (threadIdx.x == 6 * 32) trace_put(p.trace, ti, 7, clock64());
+      if (lane == 0) {
+        mbar_arrive(bar_rstd_free(a));
+        if (cta_rank == 0) mbar_arrive(bar_tmem_empty(a));
+        else mbar_arrive_cluster(map_to_cta(bar_tmem_empty(a), 0));
+      }
+      if (TRACE && threadIdx.x == 4 * 32) trace_put<TRACE>(p.trace, ti, 7);
       if (++a == 2) {
         a = 0;
         aph ^= 1u;
@@ -456,20 +578,21 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     }
   }
 
+  // nobody may leave while the partner can still signal into this CTA's shared memory
   tc_fence_before();
-  __syncthreads();
-  if (warp == 1) {
+  cluster_sync_all();
+  if (warp == 3) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+    tmem_dealloc_pair(tmem_base, Cfg::TMEM_COLS);
   }
 }
 
 // ------------------------------------------------------------------------------ host launcher
-template <int BLOCK_N, int D_HEAD>
+template <int BLOCK_N, int D_HEAD, bool TRACE>
 static kvd_status launch_impl(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_a, const RecomputeParams &p,
                               cudaStream_t stream) {
   using Cfg = RcCfg<BLOCK_N, D_HEAD>;
-  auto kern = kvd_recompute_kernel<BLOCK_N, D_HEAD>;
+  auto kern = kvd_recompute_kernel<BLOCK_N, D_HEAD, TRACE>;
   static bool configured[64] = {};
   if (!configured[ctx->device & 63]) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
@@ -477,24 +600,44 @@ static kvd_status launch_impl(kvd_ctx *ctx, const LayerState &ls, const CUtensor
     configured[ctx->device & 63] = true;
   }
   const int tiles = p.num_m_blocks * p.num_n_blocks;
-  const int grid = tiles < ctx->num_sms ? tiles : ctx->num_sms;
-  kern<<<grid, RC_THREADS, Cfg::SMEM_BYTES, stream>>>(tmap_a, ls.tmap_b, p);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return cuda_fail(ctx, e, "launch recompute");
+  const int max_clusters = ctx->num_sms / 2;
+  const int clusters = tiles < max_clusters ? tiles : max_clusters;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(2 * clusters, 1, 1);
+  cfg.blockDim = dim3(RC_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t le = cudaLaunchKernelEx(&cfg, kern, tmap_a, ls.tmap_b, p);
+  if (le != cudaSuccess) return cuda_fail(ctx, le, "launch recompute");
   ctx->launches += 1;
   return KVD_OK;
+}
+
+template <int BLOCK_N, int D_HEAD>
+static kvd_status launch_sel(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_a, const RecomputeParams &p,
+                             cudaStream_t stream) {
+  if (p.trace != nullptr) return launch_impl<BLOCK_N, D_HEAD, true>(ctx, ls, tmap_a, p, stream);
+  return launch_impl<BLOCK_N, D_HEAD, false>(ctx, ls, tmap_a, p, stream);
 }
 
 kvd_status launch_recompute(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_a, const RecomputeParams &p,
                             cudaStream_t stream) {
   const int dh = ctx->desc.d_head;
   if (ctx->block_n == 256) {
-    if (dh == 256) return launch_impl<256, 256>(ctx, ls, tmap_a, p, stream);
-    if (dh == 128) return launch_impl<256, 128>(ctx, ls, tmap_a, p, stream);
-    if (dh == 64) return launch_impl<256, 64>(ctx, ls, tmap_a, p, stream);
+    if (dh == 256) return launch_sel<256, 256>(ctx, ls, tmap_a, p, stream);
+    if (dh == 128) return launch_sel<256, 128>(ctx, ls, tmap_a, p, stream);
+    if (dh == 64) return launch_sel<256, 64>(ctx, ls, tmap_a, p, stream);
   } else if (ctx->block_n == 128) {
-    if (dh == 128) return launch_impl<128, 128>(ctx, ls, tmap_a, p, stream);
-    if (dh == 64) return launch_impl<128, 64>(ctx, ls, tmap_a, p, stream);
+    if (dh == 128) return launch_sel<128, 128>(ctx, ls, tmap_a, p, stream);
+    if (dh == 64) return launch_sel<128, 64>(ctx, ls, tmap_a, p, stream);
   }
   return KVD_ERR_SHAPE;
 }
