@@ -70,8 +70,9 @@ extern "C" size_t kvd_store_bytes(const kvd_model_desc *d, int layers_stored) {
 
 extern "C" size_t kvd_workspace_bytes(const kvd_model_desc *d) {
   if (check_desc(d) != KVD_OK) return 0;
-  const size_t parts = static_cast<size_t>(d->max_batch) * attn_max_chunks(d->d_head, d->max_tokens_per_seq);
-  return round_up(parts * d->n_q_heads * d->d_head * 4, 256) + round_up(parts * d->n_q_heads * 2 * 4, 256);
+  const size_t parts = static_cast<size_t>(d->max_batch) * attn_max_chunks(d->d_head, d->n_kv_heads, d->max_tokens_per_seq);
+  return round_up(parts * d->n_q_heads * d->d_head * 4, 256) + round_up(parts * d->n_q_heads * 2 * 4, 256) +
+         round_up(static_cast<size_t>(d->max_batch) * d->n_kv_heads * 4, 256);
 }
 
 extern "C" kvd_status kvd_create(const kvd_model_desc *desc, kvd_ctx **out) {
@@ -269,9 +270,15 @@ extern "C" kvd_status kvd_attach_workspace(kvd_ctx *ctx, void *ws, size_t bytes)
   const size_t need = kvd_workspace_bytes(&ctx->desc);
   if (bytes < need) return KVD_ERR_CAPACITY;
   const kvd_model_desc &d = ctx->desc;
-  const size_t parts = static_cast<size_t>(d.max_batch) * attn_max_chunks(d.d_head, d.max_tokens_per_seq);
+  const size_t parts = static_cast<size_t>(d.max_batch) * attn_max_chunks(d.d_head, d.n_kv_heads, d.max_tokens_per_seq);
   ctx->part_o = static_cast<float *>(ws);
-  ctx->part_ml = reinterpret_cast<float *>(static_cast<uint8_t *>(ws) + round_up(parts * d.n_q_heads * d.d_head * 4, 256));
+  uint8_t *base = static_cast<uint8_t *>(ws);
+  ctx->part_ml = reinterpret_cast<float *>(base + round_up(parts * d.n_q_heads * d.d_head * 4, 256));
+  ctx->counters = reinterpret_cast<int *>(base + round_up(parts * d.n_q_heads * d.d_head * 4, 256) +
+                                          round_up(parts * d.n_q_heads * 2 * 4, 256));
+  // the per-(sequence, head) arrival counters must start at zero; kernels leave them at zero
+  cudaError_t e = cudaMemset(ctx->counters, 0, static_cast<size_t>(d.max_batch) * d.n_kv_heads * 4);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "kvd_attach_workspace memset");
   ctx->max_parts = static_cast<int>(parts);
   ctx->workspace_bytes = need;
   return KVD_OK;
@@ -437,7 +444,7 @@ extern "C" kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, c
         S.chunk0_pos = 0;
       } else {
         // the split depends on the visible position range only
-        S.iters = attn_iters_for_span(hi - lo + 1);
+        S.iters = attn_iters_for_span(d.d_head, d.n_kv_heads, hi - lo + 1);
         const int ck = attn_chunk_keys(d.d_head, S.iters);
         S.chunk0_pos = lo / ck * ck;
         S.n_chunks = hi / ck - lo / ck + 1;
@@ -453,7 +460,17 @@ extern "C" kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, c
     L.out = static_cast<__nv_bfloat16 *>(out) + static_cast<size_t>(b0) * d.n_q_heads * d.d_head;
     L.part_o = ctx->part_o;
     L.part_ml = ctx->part_ml;
+    L.counters = ctx->counters;
+    L.seq0 = b0;
     L.scale_log2e = sc * 1.4426950408889634f;
+    // sequences without a visible key launch no work: their output is all zeros
+    for (int i = 0; i < nb; ++i) {
+      if (L.seq[i].n_chunks == 0) {
+        cudaError_t me = cudaMemsetAsync(L.out + static_cast<size_t>(i) * d.n_q_heads * d.d_head, 0,
+                                         static_cast<size_t>(d.n_q_heads) * d.d_head * 2, stream);
+        if (me != cudaSuccess) return cuda_fail(ctx, me, "zero output");
+      }
+    }
     kvd_status st = launch_attention(ctx, L, d.d_head, group, stream);
     if (st != KVD_OK) return st;
   }

@@ -6,8 +6,9 @@
 // coalesced 16-byte loads, every lane owning 8 channels, and serves all query heads of the group
 // from the same loads.  Scores of 8 keys at a time are reduced across the lanes of a key with a
 // transposing shuffle butterfly, the softmax runs online in base 2, and each CTA writes one partial
-// (max, sum, unnormalised output) per query head.  A second kernel merges the partials in chunk
-// order.
+// (max, sum, unnormalised output) per query head.  The CTA that finishes last for a (sequence, KV
+// head) -- found with one atomic counter, no waiting -- merges that head group's partials in chunk
+// order and writes the output, so a decode step is a single launch.
 //
 // Which chunk, warp, lane group and slot a key lands in is a function of its position only, and the
 // merge runs in chunk order, so the output bits do not depend on how the keys are spread over
@@ -61,8 +62,8 @@ __device__ __forceinline__ float reduce8_transposed(const float (&v)[8], int lig
   return w1;
 }
 
-template <int D_HEAD, int G>
-__global__ void __launch_bounds__(AT_THREADS) kvd_attn_split_kernel(const __grid_constant__ AttnLaunch P) {
+template <int D_HEAD, int G, int NSEQ>
+__global__ void __launch_bounds__(AT_THREADS, 4) kvd_attn_split_kernel(const __grid_constant__ AttnLaunchT<NSEQ> P) {
   constexpr int LPK = D_HEAD / 8;         // lanes per key
   constexpr int KPL = 32 / LPK;           // keys per warp-wide load
   constexpr int U = AT_UNROLL;            // keys per lane group per iteration
@@ -70,12 +71,13 @@ __global__ void __launch_bounds__(AT_THREADS) kvd_attn_split_kernel(const __grid
   __shared__ float s_o[NPART][G][D_HEAD];
   __shared__ float s_m[NPART][G];
   __shared__ float s_l[NPART][G];
+  __shared__ int s_last;
 
   // ---- which (sequence, chunk) is this CTA's?
   int si = 0;
   {
     int lo = 0, hi = P.n_seqs - 1;
-    const int b = blockIdx.x;
+    const int b = blockIdx.x / P.n_kv;
     while (lo < hi) {  // last sequence whose first partial index is <= b
       const int mid = (lo + hi + 1) >> 1;
       if (P.seq[mid].part_base - P.seq[0].part_base <= b) lo = mid; else hi = mid - 1;
@@ -83,8 +85,8 @@ __global__ void __launch_bounds__(AT_THREADS) kvd_attn_split_kernel(const __grid
     si = lo;
   }
   const AttnSeq &S = P.seq[si];
-  const int chunk = blockIdx.x - (S.part_base - P.seq[0].part_base);
-  const int kvh = blockIdx.y;
+  const int chunk = blockIdx.x / P.n_kv - (S.part_base - P.seq[0].part_base);
+  const int kvh = blockIdx.x % P.n_kv;  // the KV heads of one chunk are neighbours in the grid and in memory
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int grp = lane / LPK;   // lane group inside the warp
@@ -116,59 +118,89 @@ __global__ void __launch_bounds__(AT_THREADS) kvd_attn_split_kernel(const __grid
 
   const size_t head_off = static_cast<size_t>(kvh) * D_HEAD + lig * 8;
 
-  for (int it = 0; it < S.iters; ++it) {
-    const int pos0 = chunk_pos0 + ((it * AT_WARPS + warp) * KPL + grp) * U;  // this group's 8 positions
-    // ---- resolve the 8 keys to addresses (masked keys read a valid dummy row and score -inf)
-    const __nv_bfloat16 *kp[U];
-    const __nv_bfloat16 *vp[U];
-    uint32_t vmask = 0;
+  // Whole chunk inside one segment and inside the visible range (the common case): addresses are
+  // linear in the position.  Otherwise every key is looked up in the segment list.  The choice is
+  // uniform over the CTA and does not change which keys are read or in which order.
+  int fast_seg = -1;
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int pos = pos0 + u;
-      kp[u] = P.q;  // any mapped, 16-byte aligned address
-      vp[u] = P.q;
-      if (pos >= S.lo_pos && pos <= S.hi_pos) {
+  for (int sg = 0; sg < KVD_MAX_SEGMENTS; ++sg)
+    if (chunk_pos0 >= S.first[sg] && chunk_pos0 + chunk_keys <= S.first[sg] + S.len[sg]) fast_seg = sg;
+  const bool fast = fast_seg >= 0 && chunk_pos0 >= S.lo_pos && chunk_pos0 + chunk_keys - 1 <= S.hi_pos;
+  const __nv_bfloat16 *fk = P.q, *fv = P.q;
+  long long fstride = 0;
+  if (fast) {
+    fstride = S.stride[fast_seg];
+    const size_t off = static_cast<size_t>(chunk_pos0 - S.first[fast_seg]) * fstride + head_off;
+    fk = S.k[fast_seg] + off;
+    fv = S.v[fast_seg] + off;
+  }
+
+  // issue the 16 loads of one iteration (8 keys, 8 values) for this lane group
+  auto issue = [&](int it, uint4 (&kr)[U], uint4 (&vr)[U], uint32_t &vmask) {
+    const int rel0 = ((it * AT_WARPS + warp) * KPL + grp) * U;  // first of this group's 8 positions
+    if (fast) {
+      const __nv_bfloat16 *kp = fk + static_cast<size_t>(rel0) * fstride;
+      const __nv_bfloat16 *vp = fv + static_cast<size_t>(rel0) * fstride;
 #pragma unroll
-        for (int sg = 0; sg < KVD_MAX_SEGMENTS; ++sg) {
-          const int r = pos - S.first[sg];
-          if (r >= 0 && r < S.len[sg]) {
-            const size_t off = static_cast<size_t>(r) * S.stride[sg] + head_off;
-            kp[u] = S.k[sg] + off;
-            vp[u] = S.v[sg] + off;
-            vmask |= 1u << u;
+      for (int u = 0; u < U; ++u) kr[u] = ldg_stream(kp + u * fstride);
+#pragma unroll
+      for (int u = 0; u < U; ++u) vr[u] = ldg_stream(vp + u * fstride);
+      vmask = 0xFFu;
+    } else {
+      // masked keys are not loaded: they read as zeros and score -inf
+      vmask = 0;
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int pos = chunk_pos0 + rel0 + u;
+        const __nv_bfloat16 *kp = nullptr, *vp = nullptr;
+        if (pos >= S.lo_pos && pos <= S.hi_pos) {
+#pragma unroll
+          for (int sg = 0; sg < KVD_MAX_SEGMENTS; ++sg) {
+            const int r = pos - S.first[sg];
+            if (r >= 0 && r < S.len[sg]) {
+              const size_t off = static_cast<size_t>(r) * S.stride[sg] + head_off;
+              kp = S.k[sg] + off;
+              vp = S.v[sg] + off;
+              vmask |= 1u << u;
+            }
           }
+        }
+        kr[u] = make_uint4(0u, 0u, 0u, 0u);
+        vr[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (kp != nullptr) {
+          kr[u] = ldg_stream(kp);
+          vr[u] = ldg_stream(vp);
         }
       }
     }
-    uint4 kr[U], vr[U];
-#pragma unroll
-    for (int u = 0; u < U; ++u) kr[u] = ldg_stream(kp[u]);
-#pragma unroll
-    for (int u = 0; u < U; ++u) vr[u] = ldg_stream(vp[u]);
+  };
 
-    // ---- scores: per-lane partial dot products, then the transposing reduction
-    float kf[U][8];
+  // scores, online softmax and weighted values for the 8 keys of one iteration
+  auto compute = [&](const uint4 (&kr)[U], const uint4 (&vr)[U], uint32_t vmask) {
+    // ---- scores: per-lane partial dot products (one key unpacked at a time), then the transposing
+    // reduction
+    float part[G][U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      kf[u][0] = bf16_lo(kr[u].x); kf[u][1] = bf16_hi(kr[u].x);
-      kf[u][2] = bf16_lo(kr[u].y); kf[u][3] = bf16_hi(kr[u].y);
-      kf[u][4] = bf16_lo(kr[u].z); kf[u][5] = bf16_hi(kr[u].z);
-      kf[u][6] = bf16_lo(kr[u].w); kf[u][7] = bf16_hi(kr[u].w);
+      float kf[8];
+      kf[0] = bf16_lo(kr[u].x); kf[1] = bf16_hi(kr[u].x);
+      kf[2] = bf16_lo(kr[u].y); kf[3] = bf16_hi(kr[u].y);
+      kf[4] = bf16_lo(kr[u].z); kf[5] = bf16_hi(kr[u].z);
+      kf[6] = bf16_lo(kr[u].w); kf[7] = bf16_hi(kr[u].w);
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        float d = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) d = fmaf(qf[g][e], kf[e], d);
+        part[g][u] = d;
+      }
     }
     float pb[G][U];  // softmax numerators of the 8 keys, broadcast to every lane of the group
     float corr[G];
     const bool my_valid = (vmask >> my_slot) & 1u;
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      float part[U];
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        float d = 0.f;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) d = fmaf(qf[g][e], kf[u][e], d);
-        part[u] = d;
-      }
-      float sc = reduce8_transposed<LPK>(part, lig);
+      float sc = reduce8_transposed<LPK>(part[g], lig);
       sc = my_valid ? sc : -CUDART_INF_F;
       float bmax = sc;
       bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, LPK / 2));
@@ -185,8 +217,8 @@ __global__ void __launch_bounds__(AT_THREADS) kvd_attn_split_kernel(const __grid
       l_run[g] = l_run[g] * corr[g] + (counts ? pmine : 0.f);
 #pragma unroll
       for (int u = 0; u < U; ++u) {
-        const int src = grp * LPK + ((u & 4) ? LPK / 2 : 0) + ((u & 2) ? LPK / 4 : 0) + ((u & 1) ? LPK / 8 : 0);
-        pb[g][u] = __shfl_sync(0xffffffffu, pmine, src);
+        const int srcl = grp * LPK + ((u & 4) ? LPK / 2 : 0) + ((u & 2) ? LPK / 4 : 0) + ((u & 1) ? LPK / 8 : 0);
+        pb[g][u] = __shfl_sync(0xffffffffu, pmine, srcl);
       }
     }
     // ---- weighted values
@@ -205,6 +237,23 @@ __global__ void __launch_bounds__(AT_THREADS) kvd_attn_split_kernel(const __grid
       for (int g = 0; g < G; ++g)
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[g][e] = fmaf(pb[g][u], vf[e], acc[g][e]);
+    }
+  };
+  // a warp none of whose keys is visible has nothing to add (warp-uniform test: the reductions
+  // inside compute() use the whole warp)
+  auto step = [&](const uint4 (&kr)[U], const uint4 (&vr)[U], uint32_t vmask) {
+    if (__any_sync(0xffffffffu, vmask != 0u)) compute(kr, vr, vmask);
+  };
+
+  // One buffer of loads per iteration; latency is hidden by the other CTAs resident on the SM (the
+  // kernel is capped at 128 registers so that four fit), which measured faster than register double
+  // buffering or a shared-memory ring at half the occupancy.
+  {
+    uint4 ka[U], va[U];
+    uint32_t ma = 0;
+    for (int it = 0; it < S.iters; ++it) {
+      issue(it, ka, va, ma);
+      step(ka, va, ma);
     }
   }
 
@@ -245,55 +294,129 @@ __global__ void __launch_bounds__(AT_THREADS) kvd_attn_split_kernel(const __grid
       P.part_ml[hq * 2 + 1] = l;
     }
   }
+
+  // ---- the CTA that finishes last for this (sequence, KV head) merges all chunks, in chunk order
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int *cnt = P.counters + (P.seq0 + si) * P.n_kv + kvh;
+    const int old = atomicAdd(cnt, 1);
+    s_last = (old == S.n_chunks - 1) ? 1 : 0;
+    if (s_last) *cnt = 0;  // ready for the next call
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+
+  // Merge.  Pass 1: the global maximum of each head over all chunks.  Pass 2: every warp sums a
+  // contiguous quarter of the chunks with the common maximum (so no rescaling is needed), each lane
+  // owning D_HEAD/32 channels of every head; the four warp results are added in warp order.
+  constexpr int CPL = D_HEAD / 32;  // channels per lane
+  float *s_M = &s_m[0][0];          // [G] (the per-group scratch is free again)
+  const float *ml0 = P.part_ml + (static_cast<size_t>(S.part_base) * P.n_q + kvh * G) * 2;
+  const float *po0 = P.part_o + (static_cast<size_t>(S.part_base) * P.n_q + kvh * G) * D_HEAD;
+  const size_t ml_stride = static_cast<size_t>(P.n_q) * 2, po_stride = static_cast<size_t>(P.n_q) * D_HEAD;
+  __syncthreads();
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    float mx = -CUDART_INF_F;
+    for (int ch = threadIdx.x; ch < S.n_chunks; ch += AT_THREADS) mx = fmaxf(mx, __ldcg(ml0 + ch * ml_stride + g * 2));
+#pragma unroll
+    for (int msk = 16; msk >= 1; msk >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, msk));
+    if (lane == 0) s_l[warp][g] = mx;
+  }
+  __syncthreads();
+  if (threadIdx.x < G) {
+    float mx = s_l[0][threadIdx.x];
+#pragma unroll
+    for (int w = 1; w < AT_WARPS; ++w) mx = fmaxf(mx, s_l[w][threadIdx.x]);
+    s_M[threadIdx.x] = (mx == -CUDART_INF_F) ? 0.f : mx;
+  }
+  __syncthreads();
+  {
+    float o[G][CPL], l[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      l[g] = 0.f;
+#pragma unroll
+      for (int e = 0; e < CPL; ++e) o[g][e] = 0.f;
+    }
+    const int per_warp = (S.n_chunks + AT_WARPS - 1) / AT_WARPS;
+    const int c_begin = warp * per_warp;
+    const int c_end = c_begin + per_warp < S.n_chunks ? c_begin + per_warp : S.n_chunks;
+#pragma unroll 8
+    for (int ch = c_begin; ch < c_end; ++ch) {
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const float2 mlv = __ldcg(reinterpret_cast<const float2 *>(ml0 + ch * ml_stride + g * 2));
+        const float w = exp2f(mlv.x - s_M[g]);
+        l[g] = fmaf(w, mlv.y, l[g]);
+        const float *src = po0 + ch * po_stride + g * D_HEAD + lane * CPL;
+        if constexpr (CPL == 2) {
+          const float2 v = __ldcg(reinterpret_cast<const float2 *>(src));
+          o[g][0] = fmaf(w, v.x, o[g][0]);
+          o[g][1] = fmaf(w, v.y, o[g][1]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < CPL; e += 4) {
+            const float4 v = __ldcg(reinterpret_cast<const float4 *>(src + e));
+            o[g][e] = fmaf(w, v.x, o[g][e]);
+            o[g][e + 1] = fmaf(w, v.y, o[g][e + 1]);
+            o[g][e + 2] = fmaf(w, v.z, o[g][e + 2]);
+            o[g][e + 3] = fmaf(w, v.w, o[g][e + 3]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      if (lane == 0) s_l[warp][g] = l[g];
+#pragma unroll
+      for (int e = 0; e < CPL; ++e) s_o[warp][g][lane * CPL + e] = o[g][e];
+    }
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < G * D_HEAD; idx += AT_THREADS) {
+    const int g = idx / D_HEAD, c = idx % D_HEAD;
+    float o = s_o[0][g][c], l = s_l[0][g];
+#pragma unroll
+    for (int w = 1; w < AT_WARPS; ++w) {
+      o += s_o[w][g][c];
+      l += s_l[w][g];
+    }
+    const float r = l > 0.f ? o / l : 0.f;
+    P.out[(static_cast<size_t>(si) * P.n_q + kvh * G + g) * D_HEAD + c] = __float2bfloat16_rn(r);
+  }
 }
 
-// Merge the chunk partials of one (sequence, query head) in chunk order and normalise.
-template <int D_HEAD>
-__global__ void __launch_bounds__(D_HEAD) kvd_attn_merge_kernel(const __grid_constant__ AttnLaunch P) {
-  const int h = blockIdx.x;
-  const int si = blockIdx.y;
-  const AttnSeq &S = P.seq[si];
-  const int c = threadIdx.x;
-  float M = -CUDART_INF_F;
-  for (int ch = 0; ch < S.n_chunks; ++ch)
-    M = fmaxf(M, P.part_ml[(static_cast<size_t>(S.part_base + ch) * P.n_q + h) * 2]);
-  const float Mu = (M == -CUDART_INF_F) ? 0.f : M;
-  float o = 0.f, l = 0.f;
-  for (int ch = 0; ch < S.n_chunks; ++ch) {
-    const size_t hq = static_cast<size_t>(S.part_base + ch) * P.n_q + h;
-    const float w = exp2f(P.part_ml[hq * 2] - Mu);
-    o = fmaf(w, P.part_o[hq * D_HEAD + c], o);
-    l = fmaf(w, P.part_ml[hq * 2 + 1], l);
+template <int D_HEAD, int G, int NSEQ>
+static kvd_status launch_attn_impl(kvd_ctx *ctx, const AttnLaunch &L, cudaStream_t stream) {
+  if (L.total_chunks > 0) {
+    static thread_local AttnLaunchT<NSEQ> S;
+    static_cast<AttnLaunchHead &>(S) = static_cast<const AttnLaunchHead &>(L);
+    for (int i = 0; i < L.n_seqs; ++i) S.seq[i] = L.seq[i];
+    kvd_attn_split_kernel<D_HEAD, G, NSEQ><<<L.total_chunks * L.n_kv, AT_THREADS, 0, stream>>>(S);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "launch attention");
+    ctx->launches += 1;
   }
-  const float r = l > 0.f ? o / l : 0.f;
-  P.out[(static_cast<size_t>(si) * P.n_q + h) * D_HEAD + c] = __float2bfloat16_rn(r);
+  return KVD_OK;
 }
 
 template <int D_HEAD, int G>
-static kvd_status launch_attn_impl(kvd_ctx *ctx, const AttnLaunch &L, cudaStream_t stream) {
-  if (L.total_chunks > 0) {
-    dim3 grid(L.total_chunks, L.n_kv);
-    kvd_attn_split_kernel<D_HEAD, G><<<grid, AT_THREADS, 0, stream>>>(L);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return cuda_fail(ctx, e, "launch attention split");
-    ctx->launches += 1;
-  }
-  dim3 mgrid(L.n_q, L.n_seqs);
-  kvd_attn_merge_kernel<D_HEAD><<<mgrid, D_HEAD, 0, stream>>>(L);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return cuda_fail(ctx, e, "launch attention merge");
-  ctx->launches += 1;
-  return KVD_OK;
+static kvd_status launch_attn_nseq(kvd_ctx *ctx, const AttnLaunch &L, cudaStream_t stream) {
+  if (L.n_seqs <= 4) return launch_attn_impl<D_HEAD, G, 4>(ctx, L, stream);
+  return launch_attn_impl<D_HEAD, G, AT_MAX_SEQS>(ctx, L, stream);
 }
 
 template <int D_HEAD>
 static kvd_status launch_attn_group(kvd_ctx *ctx, const AttnLaunch &L, int group, cudaStream_t stream) {
   switch (group) {
-    case 1: return launch_attn_impl<D_HEAD, 1>(ctx, L, stream);
-    case 2: return launch_attn_impl<D_HEAD, 2>(ctx, L, stream);
-    case 3: return launch_attn_impl<D_HEAD, 3>(ctx, L, stream);
-    case 4: return launch_attn_impl<D_HEAD, 4>(ctx, L, stream);
-    case 8: return launch_attn_impl<D_HEAD, 8>(ctx, L, stream);
+    case 1: return launch_attn_nseq<D_HEAD, 1>(ctx, L, stream);
+    case 2: return launch_attn_nseq<D_HEAD, 2>(ctx, L, stream);
+    case 3: return launch_attn_nseq<D_HEAD, 3>(ctx, L, stream);
+    case 4: return launch_attn_nseq<D_HEAD, 4>(ctx, L, stream);
+    case 8: return launch_attn_nseq<D_HEAD, 8>(ctx, L, stream);
     default: return KVD_ERR_SHAPE;
   }
 }

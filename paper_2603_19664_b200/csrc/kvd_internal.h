@@ -74,32 +74,54 @@ struct AttnSeq {
   int pad;
 };
 
-struct AttnLaunch {
-  AttnSeq seq[AT_MAX_SEQS];
+// Launch-wide fields, followed by the per-sequence descriptors.  The kernel takes the variant whose
+// array is just large enough (AttnLaunchT<4> for small batches: a 10 KB parameter block costs
+// microseconds to launch).
+struct AttnLaunchHead {
   int n_seqs;
   int total_chunks;
   int n_q;
   int n_kv;
+  int seq0;                // index of the launch's first sequence in the batch (counter addressing)
+  float scale_log2e;
   const __nv_bfloat16 *q;  // [n_seqs, n_q, d_head] (already offset to the launch's first sequence)
   __nv_bfloat16 *out;      // [n_seqs, n_q, d_head]
   float *part_o;           // [parts][n_q][d_head]
   float *part_ml;          // [parts][n_q][2]
-  float scale_log2e;
+  int *counters;           // [max_batch][n_kv], zero between calls
 };
+template <int NSEQ>
+struct AttnLaunchT : AttnLaunchHead {
+  AttnSeq seq[NSEQ];
+};
+typedef AttnLaunchT<AT_MAX_SEQS> AttnLaunch;
 
 // keys per chunk for a head size and iteration count
 inline int attn_keys_per_warp_iter(int d_head) { return (32 / (d_head / 8)) * AT_UNROLL; }
-inline int attn_iters_for_span(int span) { return span <= 8192 ? 2 : (span <= 65536 ? 4 : 8); }
+// Iterations per chunk: the smallest power of two for which a (sequence, KV head) is cut into at
+// most `target` chunks -- 128 for spans up to 8192 keys, beyond that enough for roughly a thousand
+// work units per sequence.  Fat chunks matter (a CTA's prologue, combine and merge bookkeeping cost
+// as much as streaming a few dozen keys), and so does filling the ~600 CTA slots of the GPU when the
+// batch is 1.  A function of the model and of the visible span only, so a full cache and a
+// recomputed + window + current layout of the same positions are split identically.
+inline int attn_target_chunks(int n_kv, int span) {
+  if (span <= 8192) return 128;
+  const int t = 1024 / n_kv;
+  return t > 128 ? t : 128;
+}
+inline int attn_iters_for_span(int d_head, int n_kv, int span) {
+  const int per_iter = attn_keys_per_warp_iter(d_head) * AT_WARPS;
+  const int target = attn_target_chunks(n_kv, span);
+  int iters = 1;
+  while (iters < 64 && static_cast<long long>(per_iter) * iters * target < span) iters *= 2;
+  return iters;
+}
 inline int attn_chunk_keys(int d_head, int iters) { return attn_keys_per_warp_iter(d_head) * AT_WARPS * iters; }
-inline int attn_max_chunks(int d_head, int max_tokens) {
-  int best = 0;
-  const int spans[3] = {max_tokens < 8192 ? max_tokens : 8192, max_tokens < 65536 ? max_tokens : 65536, max_tokens};
-  for (int i = 0; i < 3; ++i) {
-    const int ck = attn_chunk_keys(d_head, attn_iters_for_span(spans[i]));
-    const int c = spans[i] / ck + 2;
-    if (c > best) best = c;
-  }
-  return best;
+inline int attn_max_chunks(int d_head, int n_kv, int max_tokens) {
+  const int per_iter = attn_keys_per_warp_iter(d_head) * AT_WARPS;
+  const int capped = max_tokens / (per_iter * 64) + 2;  // once the iteration count is capped
+  const int target = attn_target_chunks(n_kv, max_tokens) + 2;
+  return capped > target ? capped : target;
 }
 
 // ------------------------------------------------------------------------------ context
@@ -140,6 +162,7 @@ struct kvd_ctx {
   // attention scratch
   float *part_o = nullptr;
   float *part_ml = nullptr;
+  int *counters = nullptr;
   size_t workspace_bytes = 0;
   int max_parts = 0;
   int *d_status = nullptr;
