@@ -180,6 +180,30 @@ kvd_status kvd_recompute_kv(kvd_ctx *ctx, int layer, const void *rows, const int
 kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, const void *q, const int32_t *q_pos,
                                 const kvd_kv_segment *segs, int n_segs, float scale, void *out, void *stream);
 
+/* No counterpart in the paper: the same decode attention as kvd_decode_attention for callers that
+ * cannot allocate device memory at all -- code running inside someone else's memory pool or under a
+ * fixed memory budget, a plug-in whose host forbids cudaMalloc after start-up, a process that must
+ * not disturb an allocator's bookkeeping.  It needs no context and no workspace: the split partials
+ * and the arrival counters live in a fixed array of KVD_STATIC_SCRATCH_BYTES compiled into the
+ * library, which every GPU that loads the library holds until the process exits.
+ *   - Shapes are passed directly (d_head in {64, 128, 256}, group size n_q_heads / n_kv_heads in
+ *     {1, 2, 3, 4, 8}); q, q_pos, segs, scale, out and the visibility rule are those of
+ *     kvd_decode_attention; sliding_window is the layer's window (0 = global).
+ *   - The result is bit-identical to kvd_decode_attention on the same inputs.
+ *   - Limits: batch <= 64 and batch * n_kv_heads <= 1024; the partials of all sequences together
+ *     (about 128-256 chunks per sequence and KV head, n_q_heads * (d_head + 2) floats each) must fit
+ *     the array.  A request beyond that returns KVD_ERR_CAPACITY and launches nothing.
+ *   - It calls no cudaMalloc / cudaFree and no library routine that allocates.  The first call on a
+ *     device looks up the array's device address (cudaGetSymbolAddress) with that device current;
+ *     make that first call outside any stream capture.
+ *   - All calls share the array and it keeps the previous call's contents; the counters are cleared
+ *     on `stream` at the start of every call.  Calls whose kernels can overlap on one GPU (different
+ *     streams, different host threads) race on the array: serialise them on one stream. */
+#define KVD_STATIC_SCRATCH_BYTES (8u << 20)
+kvd_status kvd_decode_attention_static(int n_q_heads, int n_kv_heads, int d_head, int sliding_window, int batch,
+                                       const void *q, const int32_t *q_pos, const kvd_kv_segment *segs, int n_segs,
+                                       float scale, void *out, void *stream);
+
 /* Fill `out` with the byte counts described at kvd_mem_stats. */
 kvd_status kvd_memory_stats(const kvd_ctx *ctx, kvd_mem_stats *out);
 

@@ -32,7 +32,7 @@ KVD_MAX_SEGMENTS = 4
 EXPORTED_SYMBOLS = (
     "kvd_create", "kvd_destroy", "kvd_set_layer", "kvd_store_bytes", "kvd_attach_store", "kvd_reset_sequence",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
-    "kvd_decode_attention", "kvd_memory_stats", "kvd_poll_status", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
+    "kvd_decode_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
     "kvd_status_string", "kvd_version",
 )
 
@@ -109,6 +109,9 @@ def load() -> ctypes.CDLL:
     lib.kvd_decode_attention.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
                                          ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
     lib.kvd_decode_attention.restype = i32
+    lib.kvd_decode_attention_static.argtypes = [i32, i32, i32, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
+                                                ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
+    lib.kvd_decode_attention_static.restype = i32
     lib.kvd_memory_stats.argtypes = [vp, ctypes.POINTER(kvd_mem_stats)]
     lib.kvd_memory_stats.restype = i32
     lib.kvd_poll_status.argtypes = [vp, vp]
@@ -163,6 +166,37 @@ def _stream(stream) -> Optional[int]:
 
 
 Segment = Tuple[object, object, int, int, int]  # (k tensor/ptr, v tensor/ptr, row_stride, first_pos, len)
+
+KVD_STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def _marshal_segments(batch: int, q_pos, segs):
+    n_segs = max((len(s) for s in segs), default=0)
+    pos_arr = (ctypes.c_int32 * max(batch, 1))(*[int(p) for p in q_pos])
+    seg_arr = (kvd_kv_segment * max(batch * n_segs, 1))()
+    for b in range(batch):
+        for s in range(n_segs):
+            e = seg_arr[b * n_segs + s]
+            if s < len(segs[b]):
+                k, v, stride, first, ln = segs[b][s]
+                e.k = k if isinstance(k, int) else _ptr(k)
+                e.v = v if isinstance(v, int) else _ptr(v)
+                e.row_stride, e.first_pos, e.len = int(stride), int(first), int(ln)
+            else:
+                e.k, e.v, e.row_stride, e.first_pos, e.len = None, None, 0, 0, 0
+    return n_segs, pos_arr, seg_arr
+
+
+def kvd_decode_attention_static(n_q_heads: int, n_kv_heads: int, d_head: int, sliding_window: int, batch: int, q,
+                                q_pos: Sequence[int], segs: Sequence[Sequence[Segment]], scale: float, out,
+                                stream=None) -> int:
+    """Decode attention without a context or workspace, for callers that may not allocate device
+    memory: the scratch is a fixed array inside the library.  Returns the kvd_status (0 = ok) instead
+    of raising, so that a caller can test the capacity limit."""
+    n_segs, pos_arr, seg_arr = _marshal_segments(batch, q_pos, segs)
+    return int(load().kvd_decode_attention_static(n_q_heads, n_kv_heads, d_head, sliding_window, batch, _ptr(q),
+                                                  pos_arr, seg_arr, n_segs, float(scale), _ptr(out),
+                                                  _stream(stream)))
 
 
 class Kvd:

@@ -431,3 +431,185 @@ kvd_status launch_attention(kvd_ctx *ctx, const AttnLaunch &L, int d_head, int g
 }
 
 }  // namespace kvd
+
+// ------------------------------------------------------------------------------------------------
+// kvd_decode_attention_static: decode attention for callers that cannot allocate device memory.
+//
+// The split partials and the arrival counters live in the file-scope device array below instead of
+// a caller-provided workspace.  Every GPU that loads this library holds the array until the process
+// exits.  All calls share it, so two calls whose kernels overlap on one GPU race on it.
+// ------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_kvd_static_scratch[KVD_STATIC_SCRATCH_BYTES];
+
+namespace kvd {
+
+constexpr size_t STATIC_COUNTER_BYTES = 4096;  // arrival counters: batch * n_kv_heads <= 1024 ints
+
+// Device address of g_kvd_static_scratch on the current device.  The array's name is only a host-side
+// handle; the address a kernel can use comes from cudaGetSymbolAddress, looked up once per device.
+static kvd_status static_scratch_address(unsigned char **out) {
+  static unsigned char *cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    cudaGetLastError();
+    return KVD_ERR_UNSUPPORTED;
+  }
+  if (dev < 0 || dev >= 64) return KVD_ERR_UNSUPPORTED;
+  if (cached[dev] == nullptr) {
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_kvd_static_scratch) != cudaSuccess || p == nullptr) {
+      cudaGetLastError();
+      return KVD_ERR_CUDA;
+    }
+    cached[dev] = static_cast<unsigned char *>(p);
+  }
+  *out = cached[dev];
+  return KVD_OK;
+}
+
+template <int D_HEAD, int G>
+static kvd_status static_launch_g(const AttnLaunch &L, cudaStream_t stream) {
+  static thread_local AttnLaunchT<AT_MAX_SEQS> S;
+  static_cast<AttnLaunchHead &>(S) = static_cast<const AttnLaunchHead &>(L);
+  for (int i = 0; i < L.n_seqs; ++i) S.seq[i] = L.seq[i];
+  kvd_attn_split_kernel<D_HEAD, G, AT_MAX_SEQS><<<L.total_chunks * L.n_kv, AT_THREADS, 0, stream>>>(S);
+  return cudaGetLastError() == cudaSuccess ? KVD_OK : KVD_ERR_CUDA;
+}
+
+template <int D_HEAD>
+static kvd_status static_launch_d(const AttnLaunch &L, int group, cudaStream_t stream) {
+  switch (group) {
+    case 1: return static_launch_g<D_HEAD, 1>(L, stream);
+    case 2: return static_launch_g<D_HEAD, 2>(L, stream);
+    case 3: return static_launch_g<D_HEAD, 3>(L, stream);
+    case 4: return static_launch_g<D_HEAD, 4>(L, stream);
+    case 8: return static_launch_g<D_HEAD, 8>(L, stream);
+    default: return KVD_ERR_SHAPE;
+  }
+}
+
+}  // namespace kvd
+
+extern "C" kvd_status kvd_decode_attention_static(int n_q_heads, int n_kv_heads, int d_head, int sliding_window,
+                                                  int batch, const void *q, const int32_t *q_pos,
+                                                  const kvd_kv_segment *segs, int n_segs, float scale, void *out,
+                                                  void *stream_) {
+  using namespace kvd;
+  // ---- shapes and arguments (host only)
+  if (n_q_heads <= 0 || n_kv_heads <= 0 || sliding_window < 0 || batch < 0 || n_segs < 0 ||
+      n_segs > KVD_MAX_SEGMENTS)
+    return KVD_ERR_INVALID_ARG;
+  if (d_head != 64 && d_head != 128 && d_head != 256) return KVD_ERR_SHAPE;
+  if (n_q_heads % n_kv_heads != 0) return KVD_ERR_SHAPE;
+  const int group = n_q_heads / n_kv_heads;
+  if (!(group == 1 || group == 2 || group == 3 || group == 4 || group == 8)) return KVD_ERR_SHAPE;
+  if (batch == 0) return KVD_OK;
+  if (!q || !q_pos || !out || (n_segs > 0 && !segs)) return KVD_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(q) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u)) return KVD_ERR_ALIGNMENT;
+  // ---- limits of the fixed scratch: one launch, counters for batch * n_kv heads, room for every partial
+  if (batch > AT_MAX_SEQS) return KVD_ERR_CAPACITY;
+  if (static_cast<size_t>(batch) * n_kv_heads * sizeof(int) > STATIC_COUNTER_BYTES) return KVD_ERR_CAPACITY;
+  const int kdim = n_kv_heads * d_head;
+  for (int b = 0; b < batch; ++b) {
+    if (q_pos[b] < 0) return KVD_ERR_INVALID_ARG;
+    for (int s = 0; s < n_segs; ++s) {
+      const kvd_kv_segment &sg = segs[static_cast<size_t>(b) * n_segs + s];
+      if (sg.len < 0 || sg.first_pos < 0) return KVD_ERR_INVALID_ARG;
+      if (sg.len == 0) continue;
+      if (!sg.k || !sg.v || sg.row_stride < kdim) return KVD_ERR_INVALID_ARG;
+      if ((reinterpret_cast<uintptr_t>(sg.k) & 15u) || (reinterpret_cast<uintptr_t>(sg.v) & 15u) ||
+          sg.row_stride % 8 != 0)
+        return KVD_ERR_ALIGNMENT;
+      if (static_cast<int64_t>(sg.first_pos) + sg.len > INT32_MAX) return KVD_ERR_INVALID_ARG;
+      for (int s2 = 0; s2 < s; ++s2) {
+        const kvd_kv_segment &o = segs[static_cast<size_t>(b) * n_segs + s2];
+        if (o.len == 0) continue;
+        if (sg.first_pos < o.first_pos + o.len && o.first_pos < sg.first_pos + sg.len) return KVD_ERR_INVALID_ARG;
+      }
+    }
+  }
+  // ---- the same position-based split as kvd_decode_attention
+  static thread_local AttnLaunch L;
+  int parts = 0;
+  for (int b = 0; b < batch; ++b) {
+    AttnSeq &S = L.seq[b];
+    int min_first = INT32_MAX, max_last = -1;
+    for (int s = 0; s < KVD_MAX_SEGMENTS; ++s) {
+      S.k[s] = S.v[s] = nullptr;
+      S.stride[s] = 0;
+      S.first[s] = 0;
+      S.len[s] = 0;
+      if (s < n_segs) {
+        const kvd_kv_segment &sg = segs[static_cast<size_t>(b) * n_segs + s];
+        if (sg.len > 0) {
+          S.k[s] = static_cast<const __nv_bfloat16 *>(sg.k);
+          S.v[s] = static_cast<const __nv_bfloat16 *>(sg.v);
+          S.stride[s] = sg.row_stride;
+          S.first[s] = sg.first_pos;
+          S.len[s] = sg.len;
+          if (sg.first_pos < min_first) min_first = sg.first_pos;
+          if (sg.first_pos + sg.len - 1 > max_last) max_last = sg.first_pos + sg.len - 1;
+        }
+      }
+    }
+    S.q_pos = q_pos[b];
+    int lo = sliding_window > 0 ? S.q_pos - sliding_window + 1 : 0;
+    if (lo < 0) lo = 0;
+    if (min_first > lo) lo = min_first;
+    const int hi = S.q_pos < max_last ? S.q_pos : max_last;
+    S.lo_pos = lo;
+    S.hi_pos = hi;
+    S.part_base = parts;
+    S.pad = 0;
+    if (max_last < 0 || hi < lo) {
+      S.n_chunks = 0;
+      S.iters = 1;
+      S.chunk0_pos = 0;
+    } else {
+      S.iters = attn_iters_for_span(d_head, n_kv_heads, hi - lo + 1);
+      const int ck = attn_chunk_keys(d_head, S.iters);
+      S.chunk0_pos = lo / ck * ck;
+      S.n_chunks = hi / ck - lo / ck + 1;
+    }
+    parts += S.n_chunks;
+  }
+  const size_t ml_bytes = (static_cast<size_t>(parts) * n_q_heads * 2 * sizeof(float) + 255) / 256 * 256;
+  const size_t o_bytes = static_cast<size_t>(parts) * n_q_heads * d_head * sizeof(float);
+  if (STATIC_COUNTER_BYTES + ml_bytes + o_bytes > static_cast<size_t>(KVD_STATIC_SCRATCH_BYTES)) return KVD_ERR_CAPACITY;
+
+  unsigned char *scratch = nullptr;
+  kvd_status st = static_scratch_address(&scratch);  // first call on a device: symbol look-up
+  if (st != KVD_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  // the arrival counters must start at zero whatever an earlier call left behind
+  if (cudaMemsetAsync(scratch, 0, STATIC_COUNTER_BYTES, stream) != cudaSuccess) {
+    cudaGetLastError();
+    return KVD_ERR_CUDA;
+  }
+  L.n_seqs = batch;
+  L.total_chunks = parts;
+  L.n_q = n_q_heads;
+  L.n_kv = n_kv_heads;
+  L.seq0 = 0;
+  L.scale_log2e = (scale > 0.f ? scale : 1.0f / sqrtf(static_cast<float>(d_head))) * 1.4426950408889634f;
+  L.q = static_cast<const __nv_bfloat16 *>(q);
+  L.out = static_cast<__nv_bfloat16 *>(out);
+  L.counters = reinterpret_cast<int *>(scratch);
+  L.part_ml = reinterpret_cast<float *>(scratch + STATIC_COUNTER_BYTES);
+  L.part_o = reinterpret_cast<float *>(scratch + STATIC_COUNTER_BYTES + ml_bytes);
+  for (int b = 0; b < batch; ++b) {
+    if (L.seq[b].n_chunks == 0) {  // no visible key: the output is all zeros
+      if (cudaMemsetAsync(L.out + static_cast<size_t>(b) * n_q_heads * d_head, 0,
+                          static_cast<size_t>(n_q_heads) * d_head * 2, stream) != cudaSuccess) {
+        cudaGetLastError();
+        return KVD_ERR_CUDA;
+      }
+    }
+  }
+  if (parts == 0) return KVD_OK;
+  switch (d_head) {
+    case 64: return static_launch_d<64>(L, group, stream);
+    case 128: return static_launch_d<128>(L, group, stream);
+    default: return static_launch_d<256>(L, group, stream);
+  }
+}
