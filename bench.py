@@ -258,6 +258,28 @@ class Workload:
         if events:
             events[4].record()
 
+    # the four launches of a step, individually (for per-kernel timing)
+    def k_checkpoint(self, i):
+        s = i % self.n_sets
+        self.ctx.kvd_reset_sequence(s)
+        self.ctx.kvd_checkpoint_residual(s, 0, self.X[s], self.pos, self.T)
+
+    def k_recompute(self, i):
+        # rows come straight from the rotating residual buffers (same bytes as the stored copy)
+        s = i % self.n_sets
+        self.ctx.kvd_recompute_kv(0, self.X[s], self.pos, self.T, self.K[s], self.V[s], self.kdim)
+
+    def k_current(self, i):
+        s, T = i % self.n_sets, self.T
+        self.ctx.kvd_recompute_kv(0, self.X[s][T:], self.pos[T:], 1, self.K[s][T:], self.V[s][T:], self.kdim)
+
+    def k_attention(self, i):
+        s, T = i % self.n_sets, self.T
+        K, V = self.K[s], self.V[s]
+        self.ctx.kvd_decode_attention(0, 1, self.q[s:s + 1], [T],
+                                      [[(K, V, self.kdim, 0, T), (K[T:], V[T:], self.kdim, T, 1)]], 0.0,
+                                      self.out[s:s + 1])
+
     def cached_read_step(self, i):
         """What KV-Direct replaces: attention over the stored cache of T + 1 keys in one segment."""
         s, T = i % self.n_sets, self.T
@@ -304,6 +326,14 @@ def run_gpu(args):
         for i in range(steps):
             wl.step(warmup + i)
         barrier()
+        if args.profile_long_attn:
+            # a few eager decode-attention calls over 32769 keys (134 MB each, larger than L2)
+            def eager(fn, reps):
+                for i in range(3):
+                    fn(i)
+                torch.cuda.synchronize()
+                return 0.0
+            measure_long_attention(wl, peaks, eager)
         if rank == 0:
             print(json.dumps({"profile_run": True, "steps": steps, "launches": wl.ctx.kvd_launch_count()}))
         return
@@ -390,6 +420,10 @@ def run_gpu(args):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / n
 
+    # each kernel of the step on its own: a graph of n_sets back-to-back launches on rotating buffer
+    # sets between two CUDA events (launch gaps included), averaged per launch
+    iso_ms = {"checkpoint": timed_graph(wl.k_checkpoint, 10), "recompute": timed_graph(wl.k_recompute, 10),
+              "current_token_kv": timed_graph(wl.k_current, 10), "attention": timed_graph(wl.k_attention, 10)}
     read_attn_ms = timed_graph(wl.cached_read_step, 10)
     kv_copy_dst = torch.empty((2, T + 1, wl.kdim), dtype=torch.bfloat16, device="cuda")
 
@@ -435,12 +469,13 @@ def run_gpu(args):
     h2d = x_pin.numel() * 2 + pos_pin.numel() * 4 + q_pin.numel() * 2
     d2h = out_pin.numel() * 2
 
+    long_attn = measure_long_attention(wl, peaks, timed_graph) if rank == 0 else None
     sweep = run_sweep(wl, peaks) if args.sweep and rank == 0 else None
 
     if rank == 0:
         flops = 4.0 * T * shape.n_kv_heads * shape.d_hidden * shape.d_head  # Eq. 26
-        gemm_ms = float(np.mean(t_gemm))
-        attn_ms = float(np.mean(t_attn))
+        gemm_ms = iso_ms["recompute"]
+        attn_ms = iso_ms["attention"]
         attn_bytes = (T + 1) * 4 * shape.n_kv_heads * shape.d_head  # Eq. 27 for T + 1 keys
         cpu = OracleTimer(shape, T).step(12.0)
         clk = clocks.summary()
@@ -463,20 +498,27 @@ def run_gpu(args):
                          "achieved": flops / (gemm_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                          "frac": flops / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "traffic": None,
                          "peak_source": peaks["source"] + " burst", "avg_launch_us": gemm_ms * 1e3,
-                         "min_launch_us": float(np.min(t_gemm)) * 1e3,
+                         "in_step_us": float(np.mean(t_gemm)) * 1e3,
+                         "timing": "graph of back-to-back launches on rotating inputs, CUDA events, per launch",
                          "frac_of_sustained": flops / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]},
             "roofline_attention": {"kernel": "kvd_attn_split_kernel<256,2> + merge", "bound": "hbm",
                                    "achieved": attn_bytes / (attn_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                                    "unit": "GB/s", "frac": attn_bytes / (attn_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                                   "traffic": None, "avg_us": attn_ms * 1e3, "min_us": float(np.min(t_attn)) * 1e3},
-            "decode_step_us": {"checkpoint": float(np.mean(t_ckpt)) * 1e3, "recompute": gemm_ms * 1e3,
-                               "current_token_kv": float(np.mean(t_kt)) * 1e3, "attention": attn_ms * 1e3,
-                               "total": ms_per_step * 1e3},
+                                   "traffic": None, "avg_us": attn_ms * 1e3, "in_step_us": float(np.mean(t_attn)) * 1e3,
+                                   "note": "16.8 MB per call: launch-latency bound; see attention_long"},
+            "attention_long": long_attn,
+            "decode_step_us": {"total": ms_per_step * 1e3,
+                               "isolated": {k: v * 1e3 for k, v in iso_ms.items()},
+                               "in_step_with_event_nodes": {"checkpoint": float(np.mean(t_ckpt)) * 1e3,
+                                                            "recompute": float(np.mean(t_gemm)) * 1e3,
+                                                            "current_token_kv": float(np.mean(t_kt)) * 1e3,
+                                                            "attention": float(np.mean(t_attn)) * 1e3}},
             "cached_read": {"attention_over_stored_cache_us": read_attn_ms * 1e3,
                             "attention_gbs": attn_bytes / (read_attn_ms * 1e-3) / 1e9,
                             "device_copy_us": read_copy_ms * 1e3,
                             "device_copy_gbs": 2 * attn_bytes / (read_copy_ms * 1e-3) / 1e9,
-                            "recompute_over_read_ratio": gemm_ms / read_copy_ms},
+                            "recompute_over_read_ratio": gemm_ms / read_copy_ms,
+                            "paper_ratio_context": "0.17-0.3x at N=500 on Apple M3 Max / MLX (paper Section 5.8)"},
             "cpu_baseline": {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")},
         }
         if sweep is not None:
@@ -485,6 +527,34 @@ def run_gpu(args):
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def measure_long_attention(wl, peaks, timed_graph, T=32768):
+    """Decode attention over T + 1 keys of the same layer shape (134 MB per call): the size at which
+    the HBM roofline, not launch latency, is the bound."""
+    import torch
+    import paper_2603_19664_b200 as kvd
+    shape, kdim = wl.shape, wl.kdim
+    desc = kvd.make_desc(1, shape.d_hidden, shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.rms_eps,
+                         shape.qk_norm, shape.rms_eps, shape.rope_style, 1, T + 8, 1)
+    ctx = kvd.Kvd(desc)
+    ctx.kvd_set_layer(0, wl.w_kv, wl.g_in, wl.g_k, shape.rope_theta, 0)
+    ws = torch.empty(kvd.kvd_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_workspace(ws)
+    n = min(wl.n_sets, 5)
+    K = [torch.randn((T + 1, kdim), device="cuda", dtype=torch.float32).to(torch.bfloat16) for _ in range(n)]
+    V = [torch.randn((T + 1, kdim), device="cuda", dtype=torch.float32).to(torch.bfloat16) for _ in range(n)]
+
+    def call(i):
+        j = i % n
+        ctx.kvd_decode_attention(0, 1, wl.q[:1], [T], [[(K[j], V[j], kdim, 0, T + 1)]], 0.0, wl.out[:1])
+
+    ms = timed_graph(call, 5)
+    byts = (T + 1) * 4 * shape.n_kv_heads * shape.d_head
+    ctx.close()
+    return {"keys": T + 1, "bytes": byts, "avg_us": ms * 1e3, "achieved": byts / (ms * 1e-3) / 1e9,
+            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": byts / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "bound": "hbm"}
 
 
 def run_sweep(wl, peaks):
@@ -553,6 +623,8 @@ def main():
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--sets", type=int, default=N_SETS, help="rotating buffer sets (each ~59 MB)")
     ap.add_argument("--profile", action="store_true", help="eager launches only, for a run under a profiler")
+    ap.add_argument("--profile-long-attn", action="store_true",
+                    help="with --profile: also run decode attention over 32769 keys a few times")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
