@@ -39,6 +39,9 @@ if ROOT not in sys.path:
 METRIC = "recomputed_kv_tokens_per_s"
 UNIT = "tokens/s"
 T_TOKENS = 4096
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures under profiles/
+NCU_TRAFFIC_RECOMPUTE_T4096 = 31.79e6 + 0.17e6
+NCU_TRAFFIC_ATTENTION_T32768 = 134.28e6 + 3.49e6
 N_SETS = 16  # rotating buffer sets: 16 x (21 MB residual rows + 21 MB store + 16.8 MB K/V) >> 126 MB of L2
 
 
@@ -496,7 +499,11 @@ def run_gpu(args):
             "gpu_launches": int(launches),
             "roofline": {"kernel": "kvd_recompute_kernel<256,256>", "bound": "tensor",
                          "achieved": flops / (gemm_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                         "frac": flops / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "traffic": None,
+                         "frac": flops / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                         # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture
+                         # summarised in profiles/recompute_kernel_gemma3_4b_t4096.txt
+                         "traffic": NCU_TRAFFIC_RECOMPUTE_T4096, "algorithmic_bytes": 2 * (T * shape.d_hidden +
+                         shape.d_hidden * shape.n_kv_cols + T * shape.n_kv_cols),
                          "peak_source": peaks["source"] + " burst", "avg_launch_us": gemm_ms * 1e3,
                          "in_step_us": float(np.mean(t_gemm)) * 1e3,
                          "timing": "graph of back-to-back launches on rotating inputs, CUDA events, per launch",
@@ -554,7 +561,9 @@ def measure_long_attention(wl, peaks, timed_graph, T=32768):
     ctx.close()
     return {"keys": T + 1, "bytes": byts, "avg_us": ms * 1e3, "achieved": byts / (ms * 1e-3) / 1e9,
             "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": byts / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-            "bound": "hbm"}
+            "bound": "hbm", "kernel": "kvd_attn_split_kernel<256,2,4>",
+            # from profiles/attention_kernel_gemma3_4b_t32768.txt
+            "traffic": NCU_TRAFFIC_ATTENTION_T32768 if T == 32768 else None}
 
 
 def run_sweep(wl, peaks):
