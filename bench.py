@@ -178,6 +178,22 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------- replicas
+def aggregate_replicas(local_ms: float, units_per_rank: int, steps: int, dist=None, device="cpu"):
+    """Whole-job throughput of independent replicas: every rank processed `units_per_rank` units per
+    step; the job's time is the slowest rank's.  Returns (ms_per_step, units_per_second).  With
+    `dist` = None this is the single-process case."""
+    import torch
+    world = 1
+    if dist is not None:
+        t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        local_ms = float(t.item())
+        world = dist.get_world_size()
+    ms_per_step = local_ms / steps
+    return ms_per_step, world * units_per_rank / (ms_per_step * 1e-3)
+
+
 # ----------------------------------------------------------------------------- GPU arm
 class GraphEvent:
     """A CUDA event that can be recorded inside a captured graph (an event-record node) and timed
@@ -386,12 +402,7 @@ def run_gpu(args):
     if status != kvd.KVD_OK:
         raise RuntimeError(f"device status after the timed region: {kvd.status_string(status)}")
     t_ckpt, t_gemm, t_kt, t_attn = (np.array(t) for t in t_k)
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    ms_per_step = total_ms / steps
-    value = world * T / (ms_per_step * 1e-3)
+    ms_per_step, value = aggregate_replicas(total_ms, T, steps, dist, "cuda")
 
     # ---- the read that recomputation replaces (graphs of n_sets calls, same rotation)
     def timed_graph(fn, reps):
@@ -465,10 +476,7 @@ def run_gpu(args):
 
     n_e2e = min(max(steps, 10), 50)
     e2e_ms = timed(e2e_step, n_e2e)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms, _ = aggregate_replicas(e2e_ms, T, 1, dist, "cuda")
     h2d = x_pin.numel() * 2 + pos_pin.numel() * 4 + q_pin.numel() * 2
     d2h = out_pin.numel() * 2
 
