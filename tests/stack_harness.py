@@ -1,0 +1,152 @@
+"""Test scaffold: a whole decoder stack driven one token at a time on the GPU (Algorithm 1).
+
+The hot path -- checkpointing residual rows, K/V (re)computation and decode attention -- goes through
+the C ABI of the library.  Everything around it (embedding lookup, Q projection with q-norm and
+rotation, W_o, the gated MLP, the final norm, the vocabulary projection and the argmax) is plain
+torch arithmetic: it is scaffolding that both cache policies share line for line, needed only to
+produce realistic residual streams and to turn attention outputs into tokens.
+
+Two cache policies, as in the oracle's stack:
+  * "full"      every token's K/V is kept; attention reads one stored segment;
+  * "kvdirect"  at most B live K/V entries per layer; the K/V of evicted tokens are rebuilt every
+                step from the checkpointed residual rows (kvd_recompute_kv from the store) and
+                attention reads [rebuilt, live window incl. current].
+"""
+import math
+
+import numpy as np
+import torch
+
+import paper_2603_19664_b200 as kvd
+from kvd_synth import ROPE_HALF
+
+
+def _dev(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+class GpuStack:
+    def __init__(self, stack, weights, policy="full", budget=0, max_tokens=512):
+        assert policy in ("full", "kvdirect")
+        self.s, self.policy, self.budget, self.max_tokens = stack, policy, int(budget), max_tokens
+        s = stack
+        self.kdim = s.n_kv_heads * s.d_head
+        self.embed = _dev(weights.embed)
+        self.lm_head = _dev(weights.lm_head)
+        self.g_final = _dev(weights.gamma_final).float()
+        self.lw = []
+        for lw in weights.layers:
+            d = {k: _dev(v) for k, v in lw.items()}
+            self.lw.append(d)
+        desc = kvd.make_desc(s.n_layers, s.d_hidden, s.n_q_heads, s.n_kv_heads, s.d_head, s.rms_eps, s.qk_norm,
+                             s.rms_eps, s.rope_style, 1, max_tokens, 1)
+        self.ctx = kvd.Kvd(desc)
+        for l in range(s.n_layers):
+            ls = s.layer_shape(l)
+            self.ctx.kvd_set_layer(l, self.lw[l]["w_kv"], self.lw[l]["gamma_in"],
+                                   self.lw[l].get("gamma_k") if s.qk_norm else None, ls.rope_theta, ls.sliding_window)
+        self.ws = torch.empty(kvd.kvd_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+        self.ctx.kvd_attach_workspace(self.ws)
+        self.arena = torch.empty(kvd.kvd_store_bytes(desc, s.n_layers), dtype=torch.uint8, device="cuda")
+        self.ctx.kvd_attach_store(self.arena, s.n_layers)
+        # K/V storage indexed by position: the full cache, or the live window of the bounded policy
+        self.k_live = [torch.zeros((max_tokens, self.kdim), dtype=torch.bfloat16, device="cuda") for _ in range(s.n_layers)]
+        self.v_live = [torch.zeros((max_tokens, self.kdim), dtype=torch.bfloat16, device="cuda") for _ in range(s.n_layers)]
+        self.k_old = torch.zeros((max_tokens, self.kdim), dtype=torch.bfloat16, device="cuda")
+        self.v_old = torch.zeros((max_tokens, self.kdim), dtype=torch.bfloat16, device="cuda")
+        self.win_first = [0] * s.n_layers
+        self.t = 0
+        self.recomputed_rows = 0
+        # rotation angles for q (scaffold side), fp64 on the host like the library's tables
+        self.inv_freq = {}
+
+    def _rms(self, x, gamma):
+        xf = x.float()
+        return xf * torch.rsqrt(xf.pow(2).mean(-1, keepdim=True) + self.s.rms_eps) * gamma.float()
+
+    def _rope_q(self, q, pos, theta):
+        s = self.s
+        half = s.d_head // 2
+        key = float(theta)
+        if key not in self.inv_freq:
+            self.inv_freq[key] = torch.tensor([theta ** (-2.0 * i / s.d_head) for i in range(half)], dtype=torch.float64)
+        ang = (self.inv_freq[key] * pos)
+        c, sn = torch.cos(ang).float().cuda(), torch.sin(ang).float().cuda()
+        if s.rope_style == ROPE_HALF:
+            a, b = q[..., :half], q[..., half:]
+            return torch.cat([a * c - b * sn, a * sn + b * c], dim=-1)
+        a, b = q[..., 0::2], q[..., 1::2]
+        out = torch.empty_like(q)
+        out[..., 0::2] = a * c - b * sn
+        out[..., 1::2] = a * sn + b * c
+        return out
+
+    def _act(self, x):
+        if self.s.activation == "silu":
+            return torch.nn.functional.silu(x)
+        return torch.nn.functional.gelu(x, approximate="tanh")
+
+    def step(self, token):
+        s, ctx, pos = self.s, self.ctx, self.t
+        assert pos < self.max_tokens
+        h = self.embed[token].clone().view(1, -1)  # bf16 residual stream
+        pos_t = torch.tensor([pos], dtype=torch.int32, device="cuda")
+        for l in range(s.n_layers):
+            lw, ls = self.lw[l], s.layer_shape(l)
+            ctx.kvd_checkpoint_residual(0, l, h, pos_t, 1)  # STORE_RESIDUAL: the row entering layer l
+            # scaffold: query
+            xb = self._rms(h, lw["gamma_in"]).to(torch.bfloat16)
+            q = (xb @ lw["w_q"]).float().view(s.n_q_heads, s.d_head)
+            if s.qk_norm:
+                q = q * torch.rsqrt(q.pow(2).mean(-1, keepdim=True) + s.rms_eps) * lw["gamma_q"].float()
+            q = self._rope_q(q, pos, ls.rope_theta).to(torch.bfloat16).view(1, s.n_q_heads, s.d_head).contiguous()
+            # hot path: K_t, V_t of the current token, written at its position in the live storage
+            kl, vl = self.k_live[l], self.v_live[l]
+            ctx.kvd_recompute_kv(l, h, pos_t, 1, kl[pos:], vl[pos:], self.kdim)
+            lo = 0 if ls.sliding_window == 0 else max(0, pos - ls.sliding_window + 1)
+            wf = self.win_first[l] if self.policy == "kvdirect" else 0
+            wf = min(wf, pos)
+            segs = []
+            if self.policy == "kvdirect" and lo < wf:
+                n = wf - lo  # evicted tokens this layer still attends to: RECOMPUTE_KV(C, l)
+                ctx.kvd_recompute_kv(l, None, None, n, self.k_old, self.v_old, self.kdim, seq=0, first_row=lo)
+                self.recomputed_rows += n
+                segs.append((self.k_old, self.v_old, self.kdim, lo, n))
+            first_live = max(wf, lo) if self.policy == "kvdirect" else 0
+            segs.append((kl[first_live:], vl[first_live:], self.kdim, first_live, pos + 1 - first_live))
+            out = torch.empty((1, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
+            ctx.kvd_decode_attention(l, 1, q, [pos], [segs], 0.0, out)
+            # scaffold: W_o, MLP
+            h = (h.float() + (out.view(1, -1) @ lw["w_o"]).float()).to(torch.bfloat16)
+            xm = self._rms(h, lw["gamma_mlp"]).to(torch.bfloat16)
+            mlp = (self._act((xm @ lw["w_gate"]).float()) * (xm @ lw["w_up"]).float()).to(torch.bfloat16) @ lw["w_down"]
+            h = (h.float() + mlp.float()).to(torch.bfloat16)
+            if self.policy == "kvdirect":
+                self.win_first[l] = max(self.win_first[l], pos + 1 - self.budget)  # evict the oldest
+        self.t += 1
+        hf = self._rms(h, self.g_final).to(torch.bfloat16)
+        return (hf @ self.lm_head).float().view(-1)
+
+    def generate(self, prompt, n_new, forced=None):
+        logits = None
+        for tok in prompt:
+            logits = self.step(int(tok))
+        toks, lgs = [], []
+        for i in range(n_new):
+            nxt = int(torch.argmax(logits).item())
+            toks.append(nxt)
+            lgs.append(logits.clone())
+            if i + 1 < n_new:
+                logits = self.step(nxt if forced is None else int(forced[i]))
+        assert self.ctx.kvd_poll_status() == kvd.KVD_OK
+        return toks, lgs
+
+    def memory_report(self):
+        """Bytes the policy needs (Eq. 28 accounting next to what per-layer checkpoints cost)."""
+        s, T, B = self.s, self.t, self.budget
+        kv_tok = 2 * s.n_kv_heads * s.d_head * 2
+        live = T if self.policy == "full" else min(B, T)
+        return {"tokens": T, "live_kv_bytes": s.n_layers * live * kv_tok,
+                "checkpoint_bytes_per_layer_rows": self.ctx.kvd_memory_stats()["checkpoint_bytes_used"],
+                "eq28_bytes": 2 * min(B, T) * s.n_layers * s.n_kv_heads * s.d_head * 2 + max(T - B, 0) * s.d_hidden * 2,
+                "full_cache_bytes": s.n_layers * T * kv_tok}
