@@ -631,6 +631,102 @@ def run_sweep(wl, peaks):
     return rows
 
 
+def run_stack_configs(args):
+    """Hot-path timing of the stack-shaped configurations: the 34-layer Gemma-3-4B-shaped stack
+    (context 2048, 256 live K/V, batch 1..64: KV-Direct decode step against a full-cache step) and the
+    Qwen3-4B-shaped long-context case (36 layers, context 32768, batch 8, 512 live K/V).  Only the
+    library's kernels are timed; one layer of each kind is measured and multiplied by the layer count."""
+    import torch
+    import paper_2603_19664_b200 as kvd
+    from kvd_synth import GEMMA3_4B_GLOBAL, GEMMA3_4B_LOCAL, QWEN3_4B, make_layer_weights
+    from paper_2603_19664_b200.build import build
+    build()
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    peaks = load_peaks()
+
+    def dev(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+    def timed(fn, reps=5):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps * 1e3  # us
+
+    def layer_case(shape, ctx_len, budget, batch):
+        """(kvdirect_us, fullcache_us, detail) for one layer: decode step of `batch` sequences at position ctx_len."""
+        kdim = shape.n_kv_heads * shape.d_head
+        lo = 0 if shape.sliding_window == 0 else max(0, ctx_len - shape.sliding_window + 1)
+        n_old = max(0, ctx_len - budget - lo)  # evicted positions [lo, ctx_len - budget) this layer attends to
+        w = make_layer_weights(shape)
+        desc = kvd.make_desc(1, shape.d_hidden, shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.rms_eps,
+                             shape.qk_norm, shape.rms_eps, shape.rope_style, 1, ctx_len + 8, batch)
+        c = kvd.Kvd(desc)
+        tw, tg = dev(w.w_kv), dev(w.gamma_in)
+        tk = dev(w.gamma_k) if w.gamma_k is not None else None
+        c.kvd_set_layer(0, tw, tg, tk, shape.rope_theta, shape.sliding_window)
+        ws = torch.empty(kvd.kvd_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+        c.kvd_attach_workspace(ws)
+        M = batch * n_old
+        X = torch.randn((max(M, 1), shape.d_hidden), device="cuda").to(torch.bfloat16)
+        pos = (torch.arange(max(M, 1), device="cuda", dtype=torch.int32) % max(n_old, 1)) + lo
+        Ko = torch.empty((max(M, 1), kdim), device="cuda", dtype=torch.bfloat16)
+        Vo = torch.empty_like(Ko)
+        Kf = torch.randn((batch, ctx_len + 1, kdim), device="cuda").to(torch.bfloat16)  # stored cache / window / current
+        Vf = torch.randn((batch, ctx_len + 1, kdim), device="cuda").to(torch.bfloat16)
+        xc = torch.randn((batch, shape.d_hidden), device="cuda").to(torch.bfloat16)
+        pc = torch.full((batch,), ctx_len, device="cuda", dtype=torch.int32)
+        kc = torch.empty((batch, kdim), device="cuda", dtype=torch.bfloat16)
+        vc = torch.empty_like(kc)
+        q = torch.randn((batch, shape.n_q_heads, shape.d_head), device="cuda").to(torch.bfloat16)
+        out = torch.empty_like(q)
+        wf = ctx_len - budget
+        segs_kvd = [[(Ko[b * n_old:], Vo[b * n_old:], kdim, lo, n_old), (Kf[b, wf:], Vf[b, wf:], kdim, wf, budget),
+                     (kc[b:], vc[b:], kdim, ctx_len, 1)] for b in range(batch)]
+        first_full = lo
+        segs_full = [[(Kf[b, first_full:], Vf[b, first_full:], kdim, first_full, ctx_len + 1 - first_full)]
+                     for b in range(batch)]
+        qpos = [ctx_len] * batch
+        t_rec = timed(lambda: c.kvd_recompute_kv(0, X, pos, M, Ko, Vo, kdim)) if M > 0 else 0.0
+        t_cur = timed(lambda: c.kvd_recompute_kv(0, xc, pc, batch, kc, vc, kdim))
+        t_att = timed(lambda: c.kvd_decode_attention(0, batch, q, qpos, segs_kvd, 0.0, out))
+        t_full = timed(lambda: c.kvd_decode_attention(0, batch, q, qpos, segs_full, 0.0, out))
+        assert c.kvd_poll_status() == kvd.KVD_OK
+        flops = 4.0 * M * shape.n_kv_heads * shape.d_hidden * shape.d_head
+        keys = batch * (ctx_len + 1 - lo)
+        byts = keys * 4 * shape.n_kv_heads * shape.d_head
+        c.close()
+        return {"rows_recomputed": M, "recompute_us": t_rec, "recompute_tflops": flops / t_rec / 1e6 if M else None,
+                "current_kv_us": t_cur, "attention_us": t_att, "attention_gbs": byts / t_att / 1e3,
+                "fullcache_attention_us": t_full, "fullcache_attention_gbs": byts / t_full / 1e3}
+
+    result = {"peaks": peaks, "gemma3_4b_stack_ctx2048_window256": [], "qwen3_4b_ctx32768_batch8_window512": None}
+    for batch in (1, 4, 16, 64):
+        g = layer_case(GEMMA3_4B_GLOBAL, 2048, 256, batch)
+        l = layer_case(GEMMA3_4B_LOCAL, 2048, 256, batch)
+        kvd_step = 5 * (g["recompute_us"] + g["current_kv_us"] + g["attention_us"]) + \
+            29 * (l["recompute_us"] + l["current_kv_us"] + l["attention_us"])
+        full_step = 5 * (g["current_kv_us"] + g["fullcache_attention_us"]) + \
+            29 * (l["current_kv_us"] + l["fullcache_attention_us"])
+        result["gemma3_4b_stack_ctx2048_window256"].append(
+            {"batch": batch, "kvdirect_decode_step_us": kvd_step, "fullcache_decode_step_us": full_step,
+             "ratio": kvd_step / full_step, "recomputed_tokens_per_s": batch * (5 * g["rows_recomputed"] // batch +
+             29 * l["rows_recomputed"] // batch) / (kvd_step * 1e-6), "global_layer": g, "local_layer": l})
+    qw = layer_case(QWEN3_4B, 32768, 512, 8)
+    qw["step_us_36_layers"] = 36 * (qw["recompute_us"] + qw["current_kv_us"] + qw["attention_us"])
+    qw["recompute_frac_of_sustained_peak"] = qw["recompute_tflops"] / peaks["bf16_tflops_sustained"]
+    qw["recompute_frac_of_burst_peak"] = qw["recompute_tflops"] / peaks["bf16_tflops"]
+    qw["attention_frac_of_hbm_peak"] = qw["attention_gbs"] / peaks["hbm_gbs"]
+    result["qwen3_4b_ctx32768_batch8_window512"] = qw
+    print(json.dumps({"stack_configs": result}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -642,9 +738,13 @@ def main():
     ap.add_argument("--profile", action="store_true", help="eager launches only, for a run under a profiler")
     ap.add_argument("--profile-long-attn", action="store_true",
                     help="with --profile: also run decode attention over 32769 keys a few times")
+    ap.add_argument("--stack-configs", action="store_true",
+                    help="time the hot path of the stack-shaped configurations instead of the contract line")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.stack_configs:
+        run_stack_configs(args)
     else:
         run_gpu(args)
 

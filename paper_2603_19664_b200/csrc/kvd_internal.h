@@ -98,30 +98,33 @@ typedef AttnLaunchT<AT_MAX_SEQS> AttnLaunch;
 
 // keys per chunk for a head size and iteration count
 inline int attn_keys_per_warp_iter(int d_head) { return (32 / (d_head / 8)) * AT_UNROLL; }
-// Iterations per chunk: the smallest power of two for which a (sequence, KV head) is cut into at
-// most `target` chunks -- 128 for spans up to 8192 keys, beyond that enough for roughly a thousand
-// work units per sequence.  Fat chunks matter (a CTA's prologue, combine and merge bookkeeping cost
-// as much as streaming a few dozen keys), and so does filling the ~600 CTA slots of the GPU when the
-// batch is 1.  A function of the model and of the visible span only, so a full cache and a
-// recomputed + window + current layout of the same positions are split identically.
+// Iterations per chunk.  Short spans (<= 8192 keys) are cut into at most 64 chunks per (sequence, KV
+// head): there a CTA's prologue, combine and merge bookkeeping cost as much as streaming a few dozen
+// keys, so fat chunks win.  Longer spans are cut so that one sequence yields about 592 work units
+// (chunks x KV heads) -- four CTAs on each of a B200's 148 SMs -- which keeps every SM equally
+// loaded when the batch is 1.  A function of the model and of the visible span only, so a full
+// cache and a recomputed + window + current layout of the same positions are split identically,
+// and a sequence's result does not depend on what else is in the batch.
 inline int attn_target_chunks(int n_kv, int span) {
-  if (span <= 8192) return 128;
-  const int t = 1024 / n_kv;
-  return t > 128 ? t : 128;
+  if (span <= 8192) return 64;
+  const int t = 592 / n_kv;
+  return t > 16 ? t : 16;
 }
 inline int attn_iters_for_span(int d_head, int n_kv, int span) {
   const int per_iter = attn_keys_per_warp_iter(d_head) * AT_WARPS;
-  const int target = attn_target_chunks(n_kv, span);
-  int iters = 1;
-  while (iters < 64 && static_cast<long long>(per_iter) * iters * target < span) iters *= 2;
-  return iters;
+  const long long per_chunk_min = static_cast<long long>(per_iter) * attn_target_chunks(n_kv, span);
+  long long iters = (span + per_chunk_min - 1) / per_chunk_min;
+  if (iters < 1) iters = 1;
+  if (iters > 64) iters = 64;
+  return static_cast<int>(iters);
 }
 inline int attn_chunk_keys(int d_head, int iters) { return attn_keys_per_warp_iter(d_head) * AT_WARPS * iters; }
 inline int attn_max_chunks(int d_head, int n_kv, int max_tokens) {
   const int per_iter = attn_keys_per_warp_iter(d_head) * AT_WARPS;
   const int capped = max_tokens / (per_iter * 64) + 2;  // once the iteration count is capped
-  const int target = attn_target_chunks(n_kv, max_tokens) + 2;
-  return capped > target ? capped : target;
+  int target = attn_target_chunks(n_kv, max_tokens);
+  if (target < 64) target = 64;
+  return (capped > target ? capped : target) + 2;
 }
 
 // ------------------------------------------------------------------------------ context
