@@ -295,98 +295,138 @@ __global__ void __launch_bounds__(AT_THREADS, 4) kvd_attn_split_kernel(const __g
     }
   }
 
-  // ---- the CTA that finishes last for this (sequence, KV head) merges all chunks, in chunk order
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    int *cnt = P.counters + (P.seq0 + si) * P.n_kv + kvh;
-    const int old = atomicAdd(cnt, 1);
-    s_last = (old == S.n_chunks - 1) ? 1 : 0;
-    if (s_last) *cnt = 0;  // ready for the next call
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-
-  // Merge.  Pass 1: the global maximum of each head over all chunks.  Pass 2: every warp sums a
-  // contiguous quarter of the chunks with the common maximum (so no rescaling is needed), each lane
-  // owning D_HEAD/32 channels of every head; the four warp results are added in warp order.
+  // ---- two-level merge without waiting.  Chunks are grouped 16 at a time by chunk index (one group
+  // of everything when there are at most 64); the CTA
+  // that arrives last on a group's counter merges that group's partials into one group partial (this
+  // happens while other groups are still streaming), and the CTA that completes the last group merges
+  // the group partials and writes the output.  Grouping and order depend on chunk indices only.
   constexpr int CPL = D_HEAD / 32;  // channels per lane
-  float *s_M = &s_m[0][0];          // [G] (the per-group scratch is free again)
-  const float *ml0 = P.part_ml + (static_cast<size_t>(S.part_base) * P.n_q + kvh * G) * 2;
-  const float *po0 = P.part_o + (static_cast<size_t>(S.part_base) * P.n_q + kvh * G) * D_HEAD;
+  float *s_M = &s_m[0][0];          // [G] maximum used for scaling (0 when nothing is visible)
+  float *s_Mraw = &s_m[1][0];       // [G] the maximum itself (NPART >= 4 rows are available)
   const size_t ml_stride = static_cast<size_t>(P.n_q) * 2, po_stride = static_cast<size_t>(P.n_q) * D_HEAD;
-  __syncthreads();
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    float mx = -CUDART_INF_F;
-    for (int ch = threadIdx.x; ch < S.n_chunks; ch += AT_THREADS) mx = fmaxf(mx, __ldcg(ml0 + ch * ml_stride + g * 2));
-#pragma unroll
-    for (int msk = 16; msk >= 1; msk >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, msk));
-    if (lane == 0) s_l[warp][g] = mx;
-  }
-  __syncthreads();
-  if (threadIdx.x < G) {
-    float mx = s_l[0][threadIdx.x];
-#pragma unroll
-    for (int w = 1; w < AT_WARPS; ++w) mx = fmaxf(mx, s_l[w][threadIdx.x]);
-    s_M[threadIdx.x] = (mx == -CUDART_INF_F) ? 0.f : mx;
-  }
-  __syncthreads();
-  {
-    float o[G][CPL], l[G];
+
+  // Merge `count` consecutive partials starting at part index `first` for this CTA's head group.
+  // Pass 1: the maximum of each head.  Pass 2: every warp sums a contiguous quarter of the partials
+  // scaled to the common maximum, each lane owning CPL channels of every head; the four warp results
+  // are added in warp order.  The result becomes the partial `dst` or, normalised, the output.
+  auto merge = [&](size_t first, int count, bool final, size_t dst) {
+    const float *ml0 = P.part_ml + (first * P.n_q + kvh * G) * 2;
+    const float *po0 = P.part_o + (first * P.n_q + kvh * G) * D_HEAD;
+    __syncthreads();
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      l[g] = 0.f;
+      float mx = -CUDART_INF_F;
+      for (int ch = threadIdx.x; ch < count; ch += AT_THREADS) mx = fmaxf(mx, __ldcg(ml0 + ch * ml_stride + g * 2));
 #pragma unroll
-      for (int e = 0; e < CPL; ++e) o[g][e] = 0.f;
+      for (int msk = 16; msk >= 1; msk >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, msk));
+      if (lane == 0) s_l[warp][g] = mx;
     }
-    const int per_warp = (S.n_chunks + AT_WARPS - 1) / AT_WARPS;
-    const int c_begin = warp * per_warp;
-    const int c_end = c_begin + per_warp < S.n_chunks ? c_begin + per_warp : S.n_chunks;
-#pragma unroll 8
-    for (int ch = c_begin; ch < c_end; ++ch) {
+    __syncthreads();
+    if (threadIdx.x < G) {
+      float mx = s_l[0][threadIdx.x];
+#pragma unroll
+      for (int w = 1; w < AT_WARPS; ++w) mx = fmaxf(mx, s_l[w][threadIdx.x]);
+      s_Mraw[threadIdx.x] = mx;
+      s_M[threadIdx.x] = (mx == -CUDART_INF_F) ? 0.f : mx;
+    }
+    __syncthreads();
+    {
+      float o[G][CPL], l[G];
 #pragma unroll
       for (int g = 0; g < G; ++g) {
-        const float2 mlv = __ldcg(reinterpret_cast<const float2 *>(ml0 + ch * ml_stride + g * 2));
-        const float w = exp2f(mlv.x - s_M[g]);
-        l[g] = fmaf(w, mlv.y, l[g]);
-        const float *src = po0 + ch * po_stride + g * D_HEAD + lane * CPL;
-        if constexpr (CPL == 2) {
-          const float2 v = __ldcg(reinterpret_cast<const float2 *>(src));
-          o[g][0] = fmaf(w, v.x, o[g][0]);
-          o[g][1] = fmaf(w, v.y, o[g][1]);
-        } else {
+        l[g] = 0.f;
 #pragma unroll
-          for (int e = 0; e < CPL; e += 4) {
-            const float4 v = __ldcg(reinterpret_cast<const float4 *>(src + e));
-            o[g][e] = fmaf(w, v.x, o[g][e]);
-            o[g][e + 1] = fmaf(w, v.y, o[g][e + 1]);
-            o[g][e + 2] = fmaf(w, v.z, o[g][e + 2]);
-            o[g][e + 3] = fmaf(w, v.w, o[g][e + 3]);
+        for (int e = 0; e < CPL; ++e) o[g][e] = 0.f;
+      }
+      const int per_warp = (count + AT_WARPS - 1) / AT_WARPS;
+      const int c_begin = warp * per_warp;
+      const int c_end = c_begin + per_warp < count ? c_begin + per_warp : count;
+#pragma unroll 4
+      for (int ch = c_begin; ch < c_end; ++ch) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          const float2 mlv = __ldcg(reinterpret_cast<const float2 *>(ml0 + ch * ml_stride + g * 2));
+          const float w = exp2f(mlv.x - s_M[g]);
+          l[g] = fmaf(w, mlv.y, l[g]);
+          const float *src = po0 + ch * po_stride + g * D_HEAD + lane * CPL;
+          if constexpr (CPL == 2) {
+            const float2 v = __ldcg(reinterpret_cast<const float2 *>(src));
+            o[g][0] = fmaf(w, v.x, o[g][0]);
+            o[g][1] = fmaf(w, v.y, o[g][1]);
+          } else {
+#pragma unroll
+            for (int e = 0; e < CPL; e += 4) {
+              const float4 v = __ldcg(reinterpret_cast<const float4 *>(src + e));
+              o[g][e] = fmaf(w, v.x, o[g][e]);
+              o[g][e + 1] = fmaf(w, v.y, o[g][e + 1]);
+              o[g][e + 2] = fmaf(w, v.z, o[g][e + 2]);
+              o[g][e + 3] = fmaf(w, v.w, o[g][e + 3]);
+            }
           }
         }
       }
-    }
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-      if (lane == 0) s_l[warp][g] = l[g];
+      for (int g = 0; g < G; ++g) {
+        if (lane == 0) s_l[warp][g] = l[g];
 #pragma unroll
-      for (int e = 0; e < CPL; ++e) s_o[warp][g][lane * CPL + e] = o[g][e];
+        for (int e = 0; e < CPL; ++e) s_o[warp][g][lane * CPL + e] = o[g][e];
+      }
     }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < G * D_HEAD; idx += AT_THREADS) {
+      const int g = idx / D_HEAD, c = idx % D_HEAD;
+      float o = s_o[0][g][c], l = s_l[0][g];
+#pragma unroll
+      for (int w = 1; w < AT_WARPS; ++w) {
+        o += s_o[w][g][c];
+        l += s_l[w][g];
+      }
+      if (final) {
+        const float r = l > 0.f ? o / l : 0.f;
+        P.out[(static_cast<size_t>(si) * P.n_q + kvh * G + g) * D_HEAD + c] = __float2bfloat16_rn(r);
+      } else {
+        const size_t hq = dst * P.n_q + kvh * G + g;
+        P.part_o[hq * D_HEAD + c] = o;
+        if (c == 0) {
+          P.part_ml[hq * 2] = s_Mraw[g];
+          P.part_ml[hq * 2 + 1] = l;
+        }
+      }
+    }
+  };
+
+  // arrive on `cnt`; true for the CTA that is the `expected`-th (last) arrival, which also resets it
+  auto arrive_last = [&](int *cnt, int expected) -> bool {
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      const int old = atomicAdd(cnt, 1);
+      s_last = (old == expected - 1) ? 1 : 0;
+      if (s_last) *cnt = 0;  // ready for the next call
+    }
+    __syncthreads();
+    const bool last = s_last != 0;
+    if (last) __threadfence();
+    return last;
+  };
+
+  // up to 64 chunks are merged in one go (a second level would only add latency)
+  const int gsz = S.n_chunks <= 64 ? 64 : AT_MERGE_GROUP;
+  const int n_groups = (S.n_chunks + gsz - 1) / gsz;
+  const int grp_idx = chunk / gsz;
+  const int grp_size = S.n_chunks - grp_idx * gsz < gsz ? S.n_chunks - grp_idx * gsz : gsz;
+  const int head_slot = (P.seq0 + si) * P.n_kv + kvh;
+  int *cnt1 = P.counters + P.cnt1_off + static_cast<size_t>(head_slot) * P.max_groups + grp_idx;
+  int *cnt2 = P.counters + head_slot;
+  if (!arrive_last(cnt1, grp_size)) return;
+  const size_t first = static_cast<size_t>(S.part_base) + static_cast<size_t>(grp_idx) * gsz;
+  if (n_groups == 1) {
+    merge(first, grp_size, true, 0);
+    return;
   }
-  __syncthreads();
-  for (int idx = threadIdx.x; idx < G * D_HEAD; idx += AT_THREADS) {
-    const int g = idx / D_HEAD, c = idx % D_HEAD;
-    float o = s_o[0][g][c], l = s_l[0][g];
-#pragma unroll
-    for (int w = 1; w < AT_WARPS; ++w) {
-      o += s_o[w][g][c];
-      l += s_l[w][g];
-    }
-    const float r = l > 0.f ? o / l : 0.f;
-    P.out[(static_cast<size_t>(si) * P.n_q + kvh * G + g) * D_HEAD + c] = __float2bfloat16_rn(r);
-  }
+  merge(first, grp_size, false, static_cast<size_t>(S.group_base) + grp_idx);
+  if (!arrive_last(cnt2, n_groups)) return;
+  merge(static_cast<size_t>(S.group_base), n_groups, true, 0);
 }
 
 template <int D_HEAD, int G, int NSEQ>
@@ -443,7 +483,6 @@ static __device__ __align__(256) unsigned char g_kvd_static_scratch[KVD_STATIC_S
 
 namespace kvd {
 
-constexpr size_t STATIC_COUNTER_BYTES = 4096;  // arrival counters: batch * n_kv_heads <= 1024 ints
 
 // Device address of g_kvd_static_scratch on the current device.  The array's name is only a host-side
 // handle; the address a kernel can use comes from cudaGetSymbolAddress, looked up once per device.
@@ -508,7 +547,7 @@ extern "C" kvd_status kvd_decode_attention_static(int n_q_heads, int n_kv_heads,
   if ((reinterpret_cast<uintptr_t>(q) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u)) return KVD_ERR_ALIGNMENT;
   // ---- limits of the fixed scratch: one launch, counters for batch * n_kv heads, room for every partial
   if (batch > AT_MAX_SEQS) return KVD_ERR_CAPACITY;
-  if (static_cast<size_t>(batch) * n_kv_heads * sizeof(int) > STATIC_COUNTER_BYTES) return KVD_ERR_CAPACITY;
+  if (static_cast<size_t>(batch) * n_kv_heads > 1024) return KVD_ERR_CAPACITY;
   const int kdim = n_kv_heads * d_head;
   for (int b = 0; b < batch; ++b) {
     if (q_pos[b] < 0) return KVD_ERR_INVALID_ARG;
@@ -560,7 +599,7 @@ extern "C" kvd_status kvd_decode_attention_static(int n_q_heads, int n_kv_heads,
     S.lo_pos = lo;
     S.hi_pos = hi;
     S.part_base = parts;
-    S.pad = 0;
+    S.group_base = 0;
     if (max_last < 0 || hi < lo) {
       S.n_chunks = 0;
       S.iters = 1;
@@ -573,16 +612,28 @@ extern "C" kvd_status kvd_decode_attention_static(int n_q_heads, int n_kv_heads,
     }
     parts += S.n_chunks;
   }
-  const size_t ml_bytes = (static_cast<size_t>(parts) * n_q_heads * 2 * sizeof(float) + 255) / 256 * 256;
-  const size_t o_bytes = static_cast<size_t>(parts) * n_q_heads * d_head * sizeof(float);
-  if (STATIC_COUNTER_BYTES + ml_bytes + o_bytes > static_cast<size_t>(KVD_STATIC_SCRATCH_BYTES)) return KVD_ERR_CAPACITY;
+  // first-level group partials live behind the chunk partials; one counter per (sequence, KV head)
+  // and one per (sequence, KV head, group)
+  int groups = 0, max_groups = 1;
+  for (int b = 0; b < batch; ++b) {
+    const int g = (L.seq[b].n_chunks + AT_MERGE_GROUP - 1) / AT_MERGE_GROUP;
+    L.seq[b].group_base = parts + groups;
+    groups += g;
+    if (g > max_groups) max_groups = g;
+  }
+  const size_t all_parts = static_cast<size_t>(parts) + groups;
+  const size_t counter_bytes =
+      (static_cast<size_t>(batch) * n_kv_heads * (1 + max_groups) * sizeof(int) + 255) / 256 * 256;
+  const size_t ml_bytes = (all_parts * n_q_heads * 2 * sizeof(float) + 255) / 256 * 256;
+  const size_t o_bytes = all_parts * n_q_heads * d_head * sizeof(float);
+  if (counter_bytes + ml_bytes + o_bytes > static_cast<size_t>(KVD_STATIC_SCRATCH_BYTES)) return KVD_ERR_CAPACITY;
 
   unsigned char *scratch = nullptr;
   kvd_status st = static_scratch_address(&scratch);  // first call on a device: symbol look-up
   if (st != KVD_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   // the arrival counters must start at zero whatever an earlier call left behind
-  if (cudaMemsetAsync(scratch, 0, STATIC_COUNTER_BYTES, stream) != cudaSuccess) {
+  if (cudaMemsetAsync(scratch, 0, counter_bytes, stream) != cudaSuccess) {
     cudaGetLastError();
     return KVD_ERR_CUDA;
   }
@@ -591,12 +642,14 @@ extern "C" kvd_status kvd_decode_attention_static(int n_q_heads, int n_kv_heads,
   L.n_q = n_q_heads;
   L.n_kv = n_kv_heads;
   L.seq0 = 0;
+  L.max_groups = max_groups;
+  L.cnt1_off = batch * n_kv_heads;
   L.scale_log2e = (scale > 0.f ? scale : 1.0f / sqrtf(static_cast<float>(d_head))) * 1.4426950408889634f;
   L.q = static_cast<const __nv_bfloat16 *>(q);
   L.out = static_cast<__nv_bfloat16 *>(out);
   L.counters = reinterpret_cast<int *>(scratch);
-  L.part_ml = reinterpret_cast<float *>(scratch + STATIC_COUNTER_BYTES);
-  L.part_o = reinterpret_cast<float *>(scratch + STATIC_COUNTER_BYTES + ml_bytes);
+  L.part_ml = reinterpret_cast<float *>(scratch + counter_bytes);
+  L.part_o = reinterpret_cast<float *>(scratch + counter_bytes + ml_bytes);
   for (int b = 0; b < batch; ++b) {
     if (L.seq[b].n_chunks == 0) {  // no visible key: the output is all zeros
       if (cudaMemsetAsync(L.out + static_cast<size_t>(b) * n_q_heads * d_head, 0,

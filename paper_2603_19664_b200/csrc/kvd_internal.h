@@ -56,6 +56,7 @@ struct RecomputeParams {
 constexpr int AT_THREADS = 128;
 constexpr int AT_WARPS = 4;
 constexpr int AT_UNROLL = 8;          // keys per lane group per iteration
+constexpr int AT_MERGE_GROUP = 16;    // chunk partials merged per first-level group
 constexpr int AT_MAX_SEQS = 64;       // sequences per launch (bounded by the kernel parameter space)
 
 struct AttnSeq {
@@ -71,7 +72,7 @@ struct AttnSeq {
   int n_chunks;
   int part_base;    // index of this sequence's first partial in the scratch
   int iters;        // warp iterations per chunk
-  int pad;
+  int group_base;   // index of this sequence's first group partial in the scratch
 };
 
 // Launch-wide fields, followed by the per-sequence descriptors.  The kernel takes the variant whose
@@ -83,12 +84,14 @@ struct AttnLaunchHead {
   int n_q;
   int n_kv;
   int seq0;                // index of the launch's first sequence in the batch (counter addressing)
+  int max_groups;          // stride of the per-group counters
+  int cnt1_off;            // offset (ints) of the per-group counters inside `counters`
   float scale_log2e;
   const __nv_bfloat16 *q;  // [n_seqs, n_q, d_head] (already offset to the launch's first sequence)
   __nv_bfloat16 *out;      // [n_seqs, n_q, d_head]
   float *part_o;           // [parts][n_q][d_head]
   float *part_ml;          // [parts][n_q][2]
-  int *counters;           // [max_batch][n_kv], zero between calls
+  int *counters;           // [max_batch][n_kv] then [max_batch][n_kv][max_groups], zero between calls
 };
 template <int NSEQ>
 struct AttnLaunchT : AttnLaunchHead {
@@ -168,6 +171,7 @@ struct kvd_ctx {
   int *counters = nullptr;
   size_t workspace_bytes = 0;
   int max_parts = 0;
+  int max_groups = 0;
   int *d_status = nullptr;
   uint64_t launches = 0;
   uint64_t prepared_bytes = 0;
