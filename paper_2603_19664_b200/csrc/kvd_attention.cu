@@ -28,6 +28,29 @@ __device__ __forceinline__ uint4 ldg_stream(const void *p) {
   return r;
 }
 
+// Packed pairs of fp32 (sm_100 has two-wide fp32 FMA): halves the FMA count of the dot products and
+// of the weighted sum.
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &a, float &b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// the two bf16 halves of a 32-bit word as a packed pair of fp32
+__device__ __forceinline__ uint64_t bf16x2_to_f32x2(uint32_t w) { return pack2(bf16_lo(w), bf16_hi(w)); }
+
 // Sum each of the 8 values over the LPK lanes of a group; afterwards the lane whose index bits
 // (LPK/2, LPK/4, LPK/8) spell slot u holds the total of v[u].
 template <int LPK>
@@ -96,24 +119,25 @@ __global__ void __launch_bounds__(AT_THREADS, 4) kvd_attn_split_kernel(const __g
   const int chunk_pos0 = S.chunk0_pos + chunk * chunk_keys;
 
   // ---- query of every head of the group, pre-multiplied by scale * log2(e)
-  float qf[G][8];
+  uint64_t qf[G][4];  // channel pairs (2j, 2j+1)
 #pragma unroll
   for (int g = 0; g < G; ++g) {
     const __nv_bfloat16 *qp = P.q + (static_cast<size_t>(si) * P.n_q + kvh * G + g) * D_HEAD + lig * 8;
     const uint4 w = *reinterpret_cast<const uint4 *>(qp);
-    qf[g][0] = bf16_lo(w.x) * P.scale_log2e; qf[g][1] = bf16_hi(w.x) * P.scale_log2e;
-    qf[g][2] = bf16_lo(w.y) * P.scale_log2e; qf[g][3] = bf16_hi(w.y) * P.scale_log2e;
-    qf[g][4] = bf16_lo(w.z) * P.scale_log2e; qf[g][5] = bf16_hi(w.z) * P.scale_log2e;
-    qf[g][6] = bf16_lo(w.w) * P.scale_log2e; qf[g][7] = bf16_hi(w.w) * P.scale_log2e;
+    qf[g][0] = pack2(bf16_lo(w.x) * P.scale_log2e, bf16_hi(w.x) * P.scale_log2e);
+    qf[g][1] = pack2(bf16_lo(w.y) * P.scale_log2e, bf16_hi(w.y) * P.scale_log2e);
+    qf[g][2] = pack2(bf16_lo(w.z) * P.scale_log2e, bf16_hi(w.z) * P.scale_log2e);
+    qf[g][3] = pack2(bf16_lo(w.w) * P.scale_log2e, bf16_hi(w.w) * P.scale_log2e);
   }
 
-  float m_run[G], l_run[G], acc[G][8];
+  float m_run[G], l_run[G];
+  uint64_t acc[G][4];  // channel pairs
 #pragma unroll
   for (int g = 0; g < G; ++g) {
     m_run[g] = -CUDART_INF_F;
     l_run[g] = 0.f;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) acc[g][e] = 0.f;
+    for (int e = 0; e < 4; ++e) acc[g][e] = 0ull;
   }
 
   const size_t head_off = static_cast<size_t>(kvh) * D_HEAD + lig * 8;
@@ -182,17 +206,18 @@ __global__ void __launch_bounds__(AT_THREADS, 4) kvd_attn_split_kernel(const __g
     float part[G][U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      float kf[8];
-      kf[0] = bf16_lo(kr[u].x); kf[1] = bf16_hi(kr[u].x);
-      kf[2] = bf16_lo(kr[u].y); kf[3] = bf16_hi(kr[u].y);
-      kf[4] = bf16_lo(kr[u].z); kf[5] = bf16_hi(kr[u].z);
-      kf[6] = bf16_lo(kr[u].w); kf[7] = bf16_hi(kr[u].w);
+      const uint64_t k0 = bf16x2_to_f32x2(kr[u].x), k1 = bf16x2_to_f32x2(kr[u].y);
+      const uint64_t k2 = bf16x2_to_f32x2(kr[u].z), k3 = bf16x2_to_f32x2(kr[u].w);
 #pragma unroll
       for (int g = 0; g < G; ++g) {
-        float d = 0.f;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) d = fmaf(qf[g][e], kf[e], d);
-        part[g][u] = d;
+        // even and odd channels accumulate side by side, then are added
+        uint64_t d = fmul2(qf[g][0], k0);
+        d = ffma2(qf[g][1], k1, d);
+        d = ffma2(qf[g][2], k2, d);
+        d = ffma2(qf[g][3], k3, d);
+        float de, dodd;
+        unpack2(d, de, dodd);
+        part[g][u] = de + dodd;
       }
     }
     float pb[G][U];  // softmax numerators of the 8 keys, broadcast to every lane of the group
@@ -223,20 +248,23 @@ __global__ void __launch_bounds__(AT_THREADS, 4) kvd_attn_split_kernel(const __g
     }
     // ---- weighted values
 #pragma unroll
-    for (int g = 0; g < G; ++g)
+    for (int g = 0; g < G; ++g) {
+      const uint64_t c2 = pack2(corr[g], corr[g]);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) acc[g][e] *= corr[g];
+      for (int e = 0; e < 4; ++e) acc[g][e] = fmul2(acc[g][e], c2);
+    }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      float vf[8];
-      vf[0] = bf16_lo(vr[u].x); vf[1] = bf16_hi(vr[u].x);
-      vf[2] = bf16_lo(vr[u].y); vf[3] = bf16_hi(vr[u].y);
-      vf[4] = bf16_lo(vr[u].z); vf[5] = bf16_hi(vr[u].z);
-      vf[6] = bf16_lo(vr[u].w); vf[7] = bf16_hi(vr[u].w);
+      const uint64_t v0 = bf16x2_to_f32x2(vr[u].x), v1 = bf16x2_to_f32x2(vr[u].y);
+      const uint64_t v2 = bf16x2_to_f32x2(vr[u].z), v3 = bf16x2_to_f32x2(vr[u].w);
 #pragma unroll
-      for (int g = 0; g < G; ++g)
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc[g][e] = fmaf(pb[g][u], vf[e], acc[g][e]);
+      for (int g = 0; g < G; ++g) {
+        const uint64_t p2 = pack2(pb[g][u], pb[g][u]);
+        acc[g][0] = ffma2(p2, v0, acc[g][0]);
+        acc[g][1] = ffma2(p2, v1, acc[g][1]);
+        acc[g][2] = ffma2(p2, v2, acc[g][2]);
+        acc[g][3] = ffma2(p2, v3, acc[g][3]);
+      }
     }
   };
   // a warp none of whose keys is visible has nothing to add (warp-uniform test: the reductions
@@ -270,7 +298,12 @@ __global__ void __launch_bounds__(AT_THREADS, 4) kvd_attn_split_kernel(const __g
       s_l[part][g] = l;
     }
 #pragma unroll
-    for (int e = 0; e < 8; ++e) s_o[part][g][lig * 8 + e] = acc[g][e];
+    for (int e = 0; e < 4; ++e) {
+      float a0, a1;
+      unpack2(acc[g][e], a0, a1);
+      s_o[part][g][lig * 8 + 2 * e] = a0;
+      s_o[part][g][lig * 8 + 2 * e + 1] = a1;
+    }
   }
   __syncthreads();
   const size_t pidx = static_cast<size_t>(S.part_base + chunk);
