@@ -211,6 +211,13 @@ kvd_status kvd_memory_stats(const kvd_ctx *ctx, kvd_mem_stats *out);
  * KVD_ERR_POSITION. */
 kvd_status kvd_poll_status(kvd_ctx *ctx, void *stream);
 
+/* Self-test of the failure path: enqueue a one-thread kernel that waits (at most limit_ms, 1..1000)
+ * on a barrier nothing ever signals.  The wait expires, the kernel returns normally and the next
+ * kvd_poll_status reports KVD_ERR_TIMEOUT -- the same mechanism every pipeline wait of the recompute
+ * kernel uses (its limit is 2 s, or KVD_SPIN_LIMIT_MS from the environment at kvd_create).  The device
+ * stays usable. */
+kvd_status kvd_selftest_wait_timeout(kvd_ctx *ctx, int limit_ms, void *stream);
+
 /* Diagnostic hook: attach (buf != NULL) or detach (buf == NULL) a DEVICE buffer of int64 slots that
  * kvd_recompute_kv fills with a per-tile timeline in SM clock cycles: for CTA b and its i-th tile
  * (i < 8) the 16 slots at ((b*8 + i)*16) hold

@@ -32,7 +32,7 @@ KVD_MAX_SEGMENTS = 4
 EXPORTED_SYMBOLS = (
     "kvd_create", "kvd_destroy", "kvd_set_layer", "kvd_store_bytes", "kvd_attach_store", "kvd_reset_sequence",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
-    "kvd_decode_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
+    "kvd_decode_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
     "kvd_status_string", "kvd_version",
 )
 
@@ -116,6 +116,8 @@ def load() -> ctypes.CDLL:
     lib.kvd_memory_stats.restype = i32
     lib.kvd_poll_status.argtypes = [vp, vp]
     lib.kvd_poll_status.restype = i32
+    lib.kvd_selftest_wait_timeout.argtypes = [vp, i32, vp]
+    lib.kvd_selftest_wait_timeout.restype = i32
     lib.kvd_set_trace.argtypes = [vp, vp, sz]
     lib.kvd_set_trace.restype = i32
     lib.kvd_launch_count.argtypes = [vp]
@@ -283,6 +285,10 @@ class Kvd:
 
     def kvd_poll_status(self, stream=None) -> int:
         return int(self._lib.kvd_poll_status(self._h, _stream(stream)))
+
+    def kvd_selftest_wait_timeout(self, limit_ms: int, stream=None) -> None:
+        self._check(self._lib.kvd_selftest_wait_timeout(self._h, limit_ms, _stream(stream)),
+                    "kvd_selftest_wait_timeout")
 
     def kvd_set_trace(self, buf) -> None:
         if buf is None:

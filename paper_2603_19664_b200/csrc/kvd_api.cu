@@ -536,6 +536,12 @@ extern "C" kvd_status kvd_poll_status(kvd_ctx *ctx, void *stream_) {
   return KVD_OK;
 }
 
+extern "C" kvd_status kvd_selftest_wait_timeout(kvd_ctx *ctx, int limit_ms, void *stream_) {
+  if (!ctx || limit_ms <= 0 || limit_ms > 1000) return KVD_ERR_INVALID_ARG;
+  return launch_selftest_timeout(ctx, static_cast<unsigned long long>(limit_ms) * 1000000ull,
+                                 static_cast<cudaStream_t>(stream_));
+}
+
 extern "C" kvd_status kvd_set_trace(kvd_ctx *ctx, void *buf, size_t bytes) {
   if (!ctx) return KVD_ERR_INVALID_ARG;
   if (buf && (reinterpret_cast<uintptr_t>(buf) & 7u) != 0) return KVD_ERR_ALIGNMENT;

@@ -192,5 +192,6 @@ kvd_status launch_prepare_weights(kvd_ctx *ctx, const __nv_bfloat16 *w, const __
 kvd_status launch_convert_gamma(kvd_ctx *ctx, const __nv_bfloat16 *g, float *out, int n, cudaStream_t stream);
 kvd_status launch_checkpoint(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, __nv_bfloat16 *dst_rows,
                              int32_t *dst_pos, int n, int d_hidden, cudaStream_t stream);
+kvd_status launch_selftest_timeout(kvd_ctx *ctx, unsigned long long timeout_ns, cudaStream_t stream);
 kvd_status cuda_fail(kvd_ctx *ctx, cudaError_t e, const char *where);
 }  // namespace kvd

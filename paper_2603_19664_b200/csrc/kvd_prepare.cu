@@ -43,6 +43,27 @@ __global__ void __launch_bounds__(256) kvd_checkpoint_kernel(const uint4 *__rest
   for (long long i = tid; i < n; i += stride) dst_pos[i] = pos[i];
 }
 
+// Self-test of the bounded wait: one thread waits on an mbarrier that nothing ever arrives on.  The
+// wait gives up after `timeout_ns`, records STATUS_TIMEOUT and the kernel returns normally.
+__global__ void kvd_selftest_timeout_kernel(int *status, unsigned long long timeout_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    fence_mbar_init();
+    if (!mbar_wait(smem_u32(&bar), 0, &abort_flag, timeout_ns)) atomicOr(status, STATUS_TIMEOUT);
+  }
+}
+
+kvd_status launch_selftest_timeout(kvd_ctx *ctx, unsigned long long timeout_ns, cudaStream_t stream) {
+  kvd_selftest_timeout_kernel<<<1, 32, 0, stream>>>(ctx->d_status, timeout_ns);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "launch selftest");
+  ctx->launches += 1;
+  return KVD_OK;
+}
+
 kvd_status launch_prepare_weights(kvd_ctx *ctx, const __nv_bfloat16 *w, const __nv_bfloat16 *gamma, __nv_bfloat16 *wt,
                                   int d_hidden, int n_cols, cudaStream_t stream) {
   dim3 grid((n_cols + 31) / 32, (d_hidden + 31) / 32);

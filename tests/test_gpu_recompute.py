@@ -211,3 +211,26 @@ def test_argument_errors_and_position_flag():
     assert ctx.kvd_poll_status() == 9
     assert ctx.kvd_poll_status() == kvd.KVD_OK  # the flag is cleared by the read
     assert ctx.kvd_launch_count() >= 2
+
+
+def test_bounded_wait_expires_and_is_reported_without_harming_the_device():
+    """Failure detection: a wait that nothing satisfies gives up after its limit, the kernel returns,
+    kvd_poll_status says KVD_ERR_TIMEOUT, and the context keeps working."""
+    shape = TINY_GQA
+    ctx, w = open_layer(shape)
+    ctx.kvd_selftest_wait_timeout(5)
+    assert ctx.kvd_poll_status() == 8  # KVD_ERR_TIMEOUT
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    X = make_residuals(shape, 40, seed=9)
+    pos = np.arange(40)
+    K, V = run_gpu(ctx, shape, X, pos)
+    Kr, Vr = oracle_kv(shape, w, X, pos)
+    check(shape, K, V, Kr, Vr)
+    # the trace hook records a timeline and does not change results
+    tr = torch.zeros((148, 8, 16), dtype=torch.int64, device="cuda")
+    ctx.kvd_set_trace(tr)
+    K2, V2 = run_gpu(ctx, shape, X, pos)
+    ctx.kvd_set_trace(None)
+    assert torch.equal(K, K2) and torch.equal(V, V2)
+    t = tr.cpu().numpy()
+    assert t[0, 0, 5] > t[0, 0, 4] > 0 and t[0, 0, 7] > t[0, 0, 6] > 0  # MMA and epilogue intervals of tile 0
