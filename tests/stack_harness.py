@@ -25,21 +25,51 @@ def _dev(bits):
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
 
 
+def torch_stack_weights(stack, seed=0):
+    """Random-init weights of a (possibly full-size) stack drawn on the GPU with torch: N(0, 0.02)
+    matrices, N(0, 1) embeddings, norm scales 1 + N(0, 0.02).  Returns device tensors in the layout
+    GpuStack expects (use with `device_weights=True`)."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1000 + seed)
+
+    def rn(shape, std, mean=0.0):
+        return (torch.randn(shape, generator=g, device="cuda", dtype=torch.float32) * std + mean).to(torch.bfloat16)
+
+    s = stack
+    nq, nkv, dh, d = s.n_q_heads, s.n_kv_heads, s.d_head, s.d_hidden
+    layers = []
+    for _ in range(s.n_layers):
+        lw = {"w_kv": rn((d, 2 * nkv * dh), 0.02), "w_q": rn((d, nq * dh), 0.02), "w_o": rn((nq * dh, d), 0.02),
+              "w_gate": rn((d, s.d_mlp), 0.02), "w_up": rn((d, s.d_mlp), 0.02), "w_down": rn((s.d_mlp, d), 0.02),
+              "gamma_in": rn((d,), 0.02, 1.0), "gamma_mlp": rn((d,), 0.02, 1.0)}
+        if s.qk_norm:
+            lw["gamma_q"] = rn((dh,), 0.02, 1.0)
+            lw["gamma_k"] = rn((dh,), 0.02, 1.0)
+        layers.append(lw)
+    return {"embed": rn((s.vocab, d), 1.0), "lm_head": rn((d, s.vocab), 0.02), "gamma_final": rn((d,), 0.02, 1.0),
+            "layers": layers}
+
+
 class GpuStack:
-    def __init__(self, stack, weights, policy="full", budget=0, max_tokens=512):
+    def __init__(self, stack, weights, policy="full", budget=0, max_tokens=512, device_weights=False):
         assert policy in ("full", "kvdirect")
         self.s, self.policy, self.budget, self.max_tokens = stack, policy, int(budget), max_tokens
         s = stack
         self.kdim = s.n_kv_heads * s.d_head
-        self.embed = _dev(weights.embed)
-        self.lm_head = _dev(weights.lm_head)
-        self.g_final = _dev(weights.gamma_final).float()
-        self.lw = []
-        for lw in weights.layers:
-            d = {k: _dev(v) for k, v in lw.items()}
-            self.lw.append(d)
+        if device_weights:
+            self.embed, self.lm_head = weights["embed"], weights["lm_head"]
+            self.g_final = weights["gamma_final"].float()
+            self.lw = weights["layers"]
+        else:
+            self.embed = _dev(weights.embed)
+            self.lm_head = _dev(weights.lm_head)
+            self.g_final = _dev(weights.gamma_final).float()
+            self.lw = []
+            for lw in weights.layers:
+                d = {k: _dev(v) for k, v in lw.items()}
+                self.lw.append(d)
         desc = kvd.make_desc(s.n_layers, s.d_hidden, s.n_q_heads, s.n_kv_heads, s.d_head, s.rms_eps, s.qk_norm,
-                             s.rms_eps, s.rope_style, 1, max_tokens, 1)
+                             s.rms_eps, s.rope_style, 1, max_tokens, 64)
         self.ctx = kvd.Kvd(desc)
         for l in range(s.n_layers):
             ls = s.layer_shape(l)
@@ -65,12 +95,16 @@ class GpuStack:
         return xf * torch.rsqrt(xf.pow(2).mean(-1, keepdim=True) + self.s.rms_eps) * gamma.float()
 
     def _rope_q(self, q, pos, theta):
+        """q: [..., n_q, d_head] with `pos` an int or a list of positions (one per leading row)."""
         s = self.s
         half = s.d_head // 2
         key = float(theta)
         if key not in self.inv_freq:
             self.inv_freq[key] = torch.tensor([theta ** (-2.0 * i / s.d_head) for i in range(half)], dtype=torch.float64)
-        ang = (self.inv_freq[key] * pos)
+        if isinstance(pos, int):
+            ang = (self.inv_freq[key] * pos)
+        else:
+            ang = torch.tensor(pos, dtype=torch.float64)[:, None, None] * self.inv_freq[key]  # [U, 1, half]
         c, sn = torch.cos(ang).float().cuda(), torch.sin(ang).float().cuda()
         if s.rope_style == ROPE_HALF:
             a, b = q[..., :half], q[..., half:]
@@ -125,6 +159,51 @@ class GpuStack:
                 self.win_first[l] = max(self.win_first[l], pos + 1 - self.budget)  # evict the oldest
         self.t += 1
         hf = self._rms(h, self.g_final).to(torch.bfloat16)
+        return (hf @ self.lm_head).float().view(-1)
+
+    def prefill(self, tokens):
+        """Process a whole segment of tokens at once (every token attends to the keys up to its own
+        position: the decode-attention call is issued with one "sequence" per segment token).  Returns
+        the logits of the last token."""
+        s, ctx = self.s, self.ctx
+        U, p0 = len(tokens), self.t
+        assert p0 + U <= self.max_tokens
+        tok = torch.tensor(tokens, dtype=torch.long, device="cuda")
+        h = self.embed[tok].clone()  # [U, d] bf16
+        positions = list(range(p0, p0 + U))
+        pos_t = torch.arange(p0, p0 + U, dtype=torch.int32, device="cuda")
+        for l in range(s.n_layers):
+            lw, ls = self.lw[l], s.layer_shape(l)
+            ctx.kvd_checkpoint_residual(0, l, h, pos_t, U)
+            xb = self._rms(h, lw["gamma_in"]).to(torch.bfloat16)
+            q = (xb @ lw["w_q"]).float().view(U, s.n_q_heads, s.d_head)
+            if s.qk_norm:
+                q = q * torch.rsqrt(q.pow(2).mean(-1, keepdim=True) + s.rms_eps) * lw["gamma_q"].float()
+            q = self._rope_q(q, positions, ls.rope_theta).to(torch.bfloat16).contiguous()
+            kl, vl = self.k_live[l], self.v_live[l]
+            ctx.kvd_recompute_kv(l, h, pos_t, U, kl[p0:], vl[p0:], self.kdim)
+            lo_min = 0 if ls.sliding_window == 0 else max(0, p0 - ls.sliding_window + 1)
+            wf = min(self.win_first[l], p0) if self.policy == "kvdirect" else 0
+            segs = []
+            if self.policy == "kvdirect" and lo_min < wf:
+                n = wf - lo_min
+                ctx.kvd_recompute_kv(l, None, None, n, self.k_old, self.v_old, self.kdim, seq=0, first_row=lo_min)
+                self.recomputed_rows += n
+                segs.append((self.k_old, self.v_old, self.kdim, lo_min, n))
+            first_live = max(wf, lo_min) if self.policy == "kvdirect" else 0
+            segs.append((kl[first_live:], vl[first_live:], self.kdim, first_live, p0 + U - first_live))
+            out = torch.empty((U, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
+            for b0 in range(0, U, 64):
+                nb = min(64, U - b0)
+                ctx.kvd_decode_attention(l, nb, q[b0:], positions[b0:b0 + nb], [segs] * nb, 0.0, out[b0:])
+            h = (h.float() + (out.view(U, -1) @ lw["w_o"]).float()).to(torch.bfloat16)
+            xm = self._rms(h, lw["gamma_mlp"]).to(torch.bfloat16)
+            mlp = (self._act((xm @ lw["w_gate"]).float()) * (xm @ lw["w_up"]).float()).to(torch.bfloat16) @ lw["w_down"]
+            h = (h.float() + mlp.float()).to(torch.bfloat16)
+            if self.policy == "kvdirect":
+                self.win_first[l] = max(self.win_first[l], p0 + U - self.budget)
+        self.t += U
+        hf = self._rms(h[-1:], self.g_final).to(torch.bfloat16)
         return (hf @ self.lm_head).float().view(-1)
 
     def generate(self, prompt, n_new, forced=None):

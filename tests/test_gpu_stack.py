@@ -52,3 +52,19 @@ def test_gpu_stack_follows_the_oracle_stack(stack, ctx_len):
             decided += 1
             assert gt == ot, f"step {i}: margin {top2[1] - top2[0]} vs error {err}"
     assert decided >= 4, "too few steps with a clear margin to compare tokens"
+
+
+def test_multi_turn_session_matches_and_bounds_live_kv():
+    """Reduced form of the 20-turn session: 4 turns of (user segment prefilled at once + 12 greedy
+    tokens) on the small Gemma-patterned stack with a 16-token window."""
+    from session_config5 import run_session
+    from stack_harness import torch_stack_weights
+    stack = S_GEMMA
+    w = torch_stack_weights(stack, seed=5)
+    recs, ok = run_session(stack, w, turns=4, gen=12, window=16, seg_lo=24, seg_hi=64, max_tokens=4 * 76 + 8)
+    assert ok and all(r["token_match"] for r in recs)
+    kv_tok = 2 * stack.n_kv_heads * stack.d_head * 2
+    for r in recs:
+        assert r["kvdirect_live_kv_bytes"] <= stack.n_layers * 16 * kv_tok
+        assert r["full_cache_kv_bytes"] == stack.n_layers * r["tokens_so_far"] * kv_tok
+    assert recs[-1]["rows_recomputed_so_far"] > 0
