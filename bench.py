@@ -6,8 +6,8 @@ single decoder layer shaped like Gemma-3-4B (hidden 2560, 8 query / 4 KV heads, 
 key norm, RoPE base 1e6) with T = 4096 checkpointed tokens:
 
     kvd_checkpoint_residual (T rows)           STORE_RESIDUAL of Algorithm 1
-    kvd_recompute_kv        (T rows from store) Eq. 13-14: RMSNorm -> [W_K|W_V] GEMM -> key norm -> RoPE
-    kvd_recompute_kv        (1 row)             K_t, V_t of the current token
+    kvd_recompute_kv_step   (T rows from store  Eq. 13-14: RMSNorm -> [W_K|W_V] GEMM -> key norm -> RoPE,
+                             + 1 new row)       and K_t, V_t of the current token, in one launch
     kvd_decode_attention    (T + 1 keys)        Eq. 6-7, query at position T
 
 The JSON line printed by rank 0 follows the repository's bench contract; `value` is recomputed-KV
@@ -257,7 +257,7 @@ class Workload:
 
     def step(self, i, events=None):
         """One pass of the hot path on buffer set i % n_sets.  `events` (optional): 4 CUDA events
-        recorded around checkpoint / recompute / attention."""
+        recorded around checkpoint / recompute (stored rows + current token) / attention."""
         s, T, c = i % self.n_sets, self.T, self.ctx
         X, K, V = self.X[s], self.K[s], self.V[s]
         c.kvd_reset_sequence(s)
@@ -266,18 +266,16 @@ class Workload:
         c.kvd_checkpoint_residual(s, 0, X, self.pos, T)
         if events:
             events[1].record()
-        c.kvd_recompute_kv(0, None, None, T, K, V, self.kdim, seq=s, first_row=0)
+        # one launch: K/V of the T stored rows and (K_t, V_t) of the current token
+        c.kvd_recompute_kv_step(0, [(s, 0, T, K, V)], X[T:], self.pos[T:], 1, K[T:], V[T:], self.kdim)
         if events:
             events[2].record()
-        c.kvd_recompute_kv(0, X[T:], self.pos[T:], 1, K[T:], V[T:], self.kdim)
-        if events:
-            events[3].record()
         c.kvd_decode_attention(0, 1, self.q[s:s + 1], [T],
                                [[(K, V, self.kdim, 0, T), (K[T:], V[T:], self.kdim, T, 1)]], 0.0, self.out[s:s + 1])
         if events:
-            events[4].record()
+            events[3].record()
 
-    # the four launches of a step, individually (for per-kernel timing)
+    # the launches of a step, individually (for per-kernel timing)
     def k_checkpoint(self, i):
         s = i % self.n_sets
         self.ctx.kvd_reset_sequence(s)
@@ -287,6 +285,12 @@ class Workload:
         # rows come straight from the rotating residual buffers (same bytes as the stored copy)
         s = i % self.n_sets
         self.ctx.kvd_recompute_kv(0, self.X[s], self.pos, self.T, self.K[s], self.V[s], self.kdim)
+
+    def k_recompute_step(self, i):
+        # the step's launch: T rows from the store of set s (filled by the last step on it) + 1 new row
+        s, T = i % self.n_sets, self.T
+        self.ctx.kvd_recompute_kv_step(0, [(s, 0, T, self.K[s], self.V[s])], self.X[s][T:], self.pos[T:], 1,
+                                       self.K[s][T:], self.V[s][T:], self.kdim)
 
     def k_current(self, i):
         s, T = i % self.n_sets, self.T
@@ -371,7 +375,7 @@ def run_gpu(args):
     g_full = capture(n_sets)
     launches_per_step = (wl.ctx.kvd_launch_count() - l0) // n_sets
     g_rem = capture(steps % n_sets) if steps % n_sets else None
-    kev = [[GraphEvent() for _ in range(5)] for _ in range(n_sets)]
+    kev = [[GraphEvent() for _ in range(4)] for _ in range(n_sets)]
     g_ev = capture(n_sets, kev)
     for _ in range(2):
         g_full.replay()
@@ -389,19 +393,19 @@ def run_gpu(args):
         stop.record()
         barrier()
         # per-kernel durations: the same steps with event-record nodes between the kernels
-        t_k = [[], [], [], []]
+        t_k = [[], [], []]
         for _ in range(max(2, min(20, steps // n_sets))):
             g_ev.replay()
             torch.cuda.synchronize()
             for e in kev:
-                for j in range(4):
+                for j in range(3):
                     t_k[j].append(e[j].elapsed_ms(e[j + 1]))
     launches = launches_per_step * steps
     total_ms = start.elapsed_time(stop)
     status = wl.ctx.kvd_poll_status()
     if status != kvd.KVD_OK:
         raise RuntimeError(f"device status after the timed region: {kvd.status_string(status)}")
-    t_ckpt, t_gemm, t_kt, t_attn = (np.array(t) for t in t_k)
+    t_ckpt, t_gemm, t_attn = (np.array(t) for t in t_k)
     ms_per_step, value = aggregate_replicas(total_ms, T, steps, dist, "cuda")
 
     # ---- the read that recomputation replaces (graphs of n_sets calls, same rotation)
@@ -437,7 +441,8 @@ def run_gpu(args):
     # each kernel of the step on its own: a graph of n_sets back-to-back launches on rotating buffer
     # sets between two CUDA events (launch gaps included), averaged per launch
     iso_ms = {"checkpoint": timed_graph(wl.k_checkpoint, 10), "recompute": timed_graph(wl.k_recompute, 10),
-              "current_token_kv": timed_graph(wl.k_current, 10), "attention": timed_graph(wl.k_attention, 10)}
+              "recompute_with_current_token": timed_graph(wl.k_recompute_step, 10),
+              "current_token_kv_alone": timed_graph(wl.k_current, 10), "attention": timed_graph(wl.k_attention, 10)}
     read_attn_ms = timed_graph(wl.cached_read_step, 10)
     kv_copy_dst = torch.empty((2, T + 1, wl.kdim), dtype=torch.bfloat16, device="cuda")
 
@@ -467,8 +472,8 @@ def run_gpu(args):
         c = wl.ctx
         c.kvd_reset_sequence(s)
         c.kvd_checkpoint_residual(s, 0, xd, pos_dev, T)
-        c.kvd_recompute_kv(0, None, None, T, wl.K[s], wl.V[s], wl.kdim, seq=s, first_row=0)
-        c.kvd_recompute_kv(0, xd[T:], pos_dev[T:], 1, wl.K[s][T:], wl.V[s][T:], wl.kdim)
+        c.kvd_recompute_kv_step(0, [(s, 0, T, wl.K[s], wl.V[s])], xd[T:], pos_dev[T:], 1, wl.K[s][T:], wl.V[s][T:],
+                                wl.kdim)
         c.kvd_decode_attention(0, 1, q_dev, [T], [[(wl.K[s], wl.V[s], wl.kdim, 0, T), (wl.K[s][T:], wl.V[s][T:], wl.kdim, T, 1)]],
                                0.0, out_dev)
         out_pin.copy_(out_dev, non_blocking=True)
@@ -496,8 +501,8 @@ def run_gpu(args):
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": "gemma3-4b layer (d=2560, 8q/4kv heads, d_head=256, key norm, theta=1e6), "
                                    "T=4096 checkpointed tokens, batch 1 (config 2)",
-                       "step": "checkpoint T rows -> recompute K/V of T rows from the store -> K_t,V_t -> "
-                               "decode attention over T+1 keys",
+                       "step": "checkpoint T rows -> recompute K/V of T rows from the store + K_t,V_t of the current "
+                               "token (one launch) -> decode attention over T+1 keys",
                        "l2": f"inputs rotate over {n_sets} buffer sets (~{n_sets * 59} MB), larger than L2",
                        "launch": "steps replayed from CUDA graphs of the captured launch sequence",
                        "replicas": "independent replicas per GPU, no collective" if world > 1 else "single GPU"},
@@ -525,8 +530,7 @@ def run_gpu(args):
             "decode_step_us": {"total": ms_per_step * 1e3,
                                "isolated": {k: v * 1e3 for k, v in iso_ms.items()},
                                "in_step_with_event_nodes": {"checkpoint": float(np.mean(t_ckpt)) * 1e3,
-                                                            "recompute": float(np.mean(t_gemm)) * 1e3,
-                                                            "current_token_kv": float(np.mean(t_kt)) * 1e3,
+                                                            "recompute_with_current_token": float(np.mean(t_gemm)) * 1e3,
                                                             "attention": float(np.mean(t_attn)) * 1e3}},
             "cached_read": {"attention_over_stored_cache_us": read_attn_ms * 1e3,
                             "attention_gbs": attn_bytes / (read_attn_ms * 1e-3) / 1e9,

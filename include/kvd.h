@@ -165,6 +165,31 @@ kvd_status kvd_checkpoint_residual(kvd_ctx *ctx, int seq, int layer, const void 
 kvd_status kvd_recompute_kv(kvd_ctx *ctx, int layer, const void *rows, const int32_t *positions, int n, int seq,
                             int first_row, void *k_out, void *v_out, int64_t out_row_stride, void *stream);
 
+/* One range of checkpointed rows of one sequence, for kvd_recompute_kv_step. */
+typedef struct kvd_store_range {
+  int32_t seq;       /* sequence slot */
+  int32_t first_row; /* first stored row of (layer, seq) */
+  int32_t n;         /* rows; 0 = skip this entry */
+  int32_t reserved;  /* 0 */
+  void *k_out;       /* DEVICE bf16, row m of the range at [m*out_row_stride + h*d_head + c] */
+  void *v_out;
+} kvd_store_range;
+#define KVD_MAX_STORE_RANGES 64
+
+/* The K/V work of one decode step of one layer in ONE launch (Algorithm 1, inside the layer loop):
+ * RECOMPUTE_KV(C, l) for the evicted tokens of every sequence of the batch (Eq. 13-14) together
+ * with the projection that makes (K_t, V_t) of the new tokens.  Equivalent to one kvd_recompute_kv
+ * call per range plus one for `rows`, with identical output bits; the rows of all sources share
+ * the kernel's tile schedule, so single-token sources cost no launch of their own.
+ *   ranges    HOST array of n_ranges <= KVD_MAX_STORE_RANGES entries (read during the call only).
+ *   rows      DEVICE bf16 [n_rows, d_hidden] (16-byte aligned) with DEVICE int32 positions[n_rows],
+ *             results to k_rows_out / v_rows_out; n_rows == 0 leaves this source out.
+ *   out_row_stride applies to every output (elements, multiple of 8, >= n_kv*d_head).
+ * Errors as kvd_recompute_kv; nothing is launched when any entry is rejected. */
+kvd_status kvd_recompute_kv_step(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
+                                 const void *rows, const int32_t *positions, int n_rows, void *k_rows_out,
+                                 void *v_rows_out, int64_t out_row_stride, void *stream);
+
 /* ATTENTION(Q, K_all, V_all) of Algorithm 1 for one new token per sequence (Eq. 6-7).
  *   q      DEVICE bf16 [batch, n_q_heads, d_head], already normalised and rotated to q_pos.
  *   q_pos  HOST int32 [batch]: position of each sequence's query token.

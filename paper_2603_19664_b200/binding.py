@@ -32,9 +32,15 @@ KVD_MAX_SEGMENTS = 4
 EXPORTED_SYMBOLS = (
     "kvd_create", "kvd_destroy", "kvd_set_layer", "kvd_store_bytes", "kvd_attach_store", "kvd_reset_sequence",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
+    "kvd_recompute_kv_step",
     "kvd_decode_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
     "kvd_status_string", "kvd_version",
 )
+
+
+class kvd_store_range(ctypes.Structure):
+    _fields_ = [("seq", ctypes.c_int32), ("first_row", ctypes.c_int32), ("n", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("k_out", ctypes.c_void_p), ("v_out", ctypes.c_void_p)]
 
 
 class kvd_model_desc(ctypes.Structure):
@@ -106,6 +112,8 @@ def load() -> ctypes.CDLL:
     lib.kvd_checkpoint_residual.restype = i32
     lib.kvd_recompute_kv.argtypes = [vp, i32, vp, vp, i32, i32, i32, vp, vp, i64, vp]
     lib.kvd_recompute_kv.restype = i32
+    lib.kvd_recompute_kv_step.argtypes = [vp, i32, ctypes.POINTER(kvd_store_range), i32, vp, vp, i32, vp, vp, i64, vp]
+    lib.kvd_recompute_kv_step.restype = i32
     lib.kvd_decode_attention.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
                                          ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
     lib.kvd_decode_attention.restype = i32
@@ -259,6 +267,17 @@ class Kvd:
         self._check(self._lib.kvd_recompute_kv(self._h, layer, _ptr(rows), _ptr(positions), n, seq, first_row,
                                                _ptr(k_out), _ptr(v_out), out_row_stride, _stream(stream)),
                     "kvd_recompute_kv")
+
+    def kvd_recompute_kv_step(self, layer: int, ranges: Sequence[Tuple[int, int, int, object, object]], rows,
+                              positions, n_rows: int, k_rows_out, v_rows_out, out_row_stride: int, stream=None) -> None:
+        """ranges: (seq, first_row, n, k_out, v_out) per sequence; rows/positions: the new tokens (or None, 0)."""
+        arr = (kvd_store_range * max(len(ranges), 1))()
+        for i, (seq, first_row, n, k_out, v_out) in enumerate(ranges):
+            arr[i].seq, arr[i].first_row, arr[i].n, arr[i].reserved = int(seq), int(first_row), int(n), 0
+            arr[i].k_out, arr[i].v_out = _ptr(k_out), _ptr(v_out)
+        self._check(self._lib.kvd_recompute_kv_step(self._h, layer, arr, len(ranges), _ptr(rows), _ptr(positions),
+                                                    n_rows, _ptr(k_rows_out), _ptr(v_rows_out), out_row_stride,
+                                                    _stream(stream)), "kvd_recompute_kv_step")
 
     def kvd_decode_attention(self, layer: int, batch: int, q, q_pos: Sequence[int],
                              segs: Sequence[Sequence[Segment]], scale: float, out, stream=None) -> None:

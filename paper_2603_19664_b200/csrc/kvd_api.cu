@@ -168,6 +168,25 @@ static kvd_status encode_2d(kvd_ctx *ctx, CUtensorMap *map, const void *base, ui
   return KVD_OK;
 }
 
+// Row source of the recompute GEMM as a 3-D map [slabs][rows][d_hidden]; box = one 128 x 64 tile.
+static kvd_status encode_rows_3d(kvd_ctx *ctx, CUtensorMap *map, const void *base, uint64_t d_hidden, uint64_t rows,
+                                 uint64_t slabs) {
+  cuuint64_t dims[3] = {d_hidden, rows, slabs};
+  cuuint64_t strides[2] = {d_hidden * 2, rows * d_hidden * 2};
+  cuuint32_t box[3] = {RC_BLOCK_K, RC_BLOCK_M, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    char buf[64];
+    snprintf(buf, sizeof buf, "cuTensorMapEncodeTiled (rows) failed: %d", static_cast<int>(r));
+    ctx->last_error = buf;
+    return KVD_ERR_CUDA;
+  }
+  return KVD_OK;
+}
+
 // (cos, sin) tables of Eq. 11-12 split as position = 16*hi + lo; built in double on the host.
 // hi is row-major [hi][pair]; lo is pair-major [pair][lo] so that neighbouring positions read
 // neighbouring shared-memory words.
@@ -259,6 +278,16 @@ extern "C" kvd_status kvd_attach_store(kvd_ctx *ctx, void *arena, size_t bytes, 
   ctx->store_pos = reinterpret_cast<int32_t *>(static_cast<uint8_t *>(arena) + round_up(slots * d.d_hidden * 2, 256));
   ctx->layers_stored = layers_stored;
   ctx->rows_stored.assign(static_cast<size_t>(layers_stored) * d.max_seqs, 0);
+  ctx->store_maps.resize(layers_stored);
+  for (int l = 0; l < layers_stored; ++l) {
+    const __nv_bfloat16 *base = ctx->store_rows + static_cast<size_t>(l) * d.max_seqs * d.max_tokens_per_seq * d.d_hidden;
+    kvd_status st = encode_rows_3d(ctx, &ctx->store_maps[l], base, d.d_hidden, d.max_tokens_per_seq, d.max_seqs);
+    if (st != KVD_OK) {
+      ctx->store_rows = nullptr;
+      ctx->layers_stored = 0;
+      return st;
+    }
+  }
   return KVD_OK;
 }
 
@@ -319,48 +348,65 @@ extern "C" kvd_status kvd_checkpoint_residual(kvd_ctx *ctx, int seq, int layer, 
   return st;
 }
 
-extern "C" kvd_status kvd_recompute_kv(kvd_ctx *ctx, int layer, const void *rows, const int32_t *positions, int n,
-                                       int seq, int first_row, void *k_out, void *v_out, int64_t out_row_stride,
-                                       void *stream_) {
-  if (!ctx || n < 0) return KVD_ERR_INVALID_ARG;
-  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+// Shared body of kvd_recompute_kv and kvd_recompute_kv_step: validate, build the job table (store
+// ranges first, then the caller's rows), launch once.
+static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
+                                   const void *rows, const int32_t *positions, int n_rows, void *k_rows_out,
+                                   void *v_rows_out, int64_t out_row_stride, cudaStream_t stream) {
   const LayerState &ls = ctx->layers[layer];
-  if (!ls.set) return KVD_ERR_STATE;
-  if (n == 0) return KVD_OK;
-  if (!k_out || !v_out) return KVD_ERR_INVALID_ARG;
   const kvd_model_desc &d = ctx->desc;
   const int kdim = d.n_kv_heads * d.d_head;
   if (out_row_stride < kdim) return KVD_ERR_INVALID_ARG;
-  if (out_row_stride % 8 != 0 || !aligned16(k_out) || !aligned16(v_out)) return KVD_ERR_ALIGNMENT;
-  const __nv_bfloat16 *a_rows;
-  const int32_t *a_pos;
-  if (rows) {
-    if (!positions) return KVD_ERR_INVALID_ARG;
-    if (!aligned16(rows)) return KVD_ERR_ALIGNMENT;
-    a_rows = static_cast<const __nv_bfloat16 *>(rows);
-    a_pos = positions;
-  } else {
-    if (positions) return KVD_ERR_INVALID_ARG;
-    if (!ctx->store_rows) return KVD_ERR_STATE;
-    if (seq < 0 || seq >= d.max_seqs || layer >= ctx->layers_stored || first_row < 0) return KVD_ERR_INVALID_ARG;
-    const int have = ctx->rows_stored[static_cast<size_t>(layer) * d.max_seqs + seq];
-    if (first_row + n > have) return KVD_ERR_CAPACITY;
-    const size_t slot = store_slot(ctx, layer, seq) + first_row;
-    a_rows = ctx->store_rows + slot * d.d_hidden;
-    a_pos = ctx->store_pos + slot;
-  }
-  CUtensorMap tmap_a;
-  kvd_status st = encode_2d(ctx, &tmap_a, a_rows, d.d_hidden, static_cast<uint64_t>(n), RC_BLOCK_K, RC_BLOCK_M);
-  if (st != KVD_OK) return st;
+  if (out_row_stride % 8 != 0) return KVD_ERR_ALIGNMENT;
   RecomputeParams p;
-  p.M = n;
+  int n_jobs = 0, mb = 0;
+  bool any_store = false;
+  for (int i = 0; i < n_ranges; ++i) {
+    const kvd_store_range &r = ranges[i];
+    if (r.n < 0) return KVD_ERR_INVALID_ARG;
+    if (r.n == 0) continue;
+    if (!ctx->store_rows) return KVD_ERR_STATE;
+    if (r.seq < 0 || r.seq >= d.max_seqs || layer >= ctx->layers_stored || r.first_row < 0) return KVD_ERR_INVALID_ARG;
+    if (!r.k_out || !r.v_out) return KVD_ERR_INVALID_ARG;
+    if (!aligned16(r.k_out) || !aligned16(r.v_out)) return KVD_ERR_ALIGNMENT;
+    const int have = ctx->rows_stored[static_cast<size_t>(layer) * d.max_seqs + r.seq];
+    if (r.first_row > have || r.n > have - r.first_row) return KVD_ERR_CAPACITY;
+    RcJob &J = p.jobs[n_jobs++];
+    J.mb_start = mb;
+    J.n = r.n;
+    J.row0 = r.first_row;
+    J.slab = r.seq;
+    J.positions = ctx->store_pos + store_slot(ctx, layer, r.seq) + r.first_row;
+    J.k_out = static_cast<__nv_bfloat16 *>(r.k_out);
+    J.v_out = static_cast<__nv_bfloat16 *>(r.v_out);
+    mb += (r.n + 2 * RC_BLOCK_M - 1) / (2 * RC_BLOCK_M);  // 256-row tiles, 128 rows per CTA of a pair
+    any_store = true;
+  }
+  CUtensorMap tmap_rows;
+  if (n_rows > 0) {
+    if (!rows || !positions || !k_rows_out || !v_rows_out) return KVD_ERR_INVALID_ARG;
+    if (!aligned16(rows) || !aligned16(k_rows_out) || !aligned16(v_rows_out)) return KVD_ERR_ALIGNMENT;
+    kvd_status st = encode_rows_3d(ctx, &tmap_rows, rows, d.d_hidden, static_cast<uint64_t>(n_rows), 1);
+    if (st != KVD_OK) return st;
+    RcJob &J = p.jobs[n_jobs++];
+    J.mb_start = mb;
+    J.n = n_rows;
+    J.row0 = 0;
+    J.slab = -1;
+    J.positions = positions;
+    J.k_out = static_cast<__nv_bfloat16 *>(k_rows_out);
+    J.v_out = static_cast<__nv_bfloat16 *>(v_rows_out);
+    mb += (n_rows + 2 * RC_BLOCK_M - 1) / (2 * RC_BLOCK_M);
+  }
+  if (n_jobs == 0) return KVD_OK;
+  // the kernel is handed both maps; an unused one aliases the other
+  const CUtensorMap &tmap_store = any_store ? ctx->store_maps[layer] : tmap_rows;
+  const CUtensorMap &tmap_ext = n_rows > 0 ? tmap_rows : ctx->store_maps[layer];
+  p.n_jobs = n_jobs;
   p.num_k_blocks = d.d_hidden / RC_BLOCK_K;
-  p.num_m_blocks = (n + 2 * RC_BLOCK_M - 1) / (2 * RC_BLOCK_M);  // 256-row tiles, 128 rows per CTA of a pair
+  p.num_m_blocks = mb;
   p.num_n_blocks = 2 * kdim / ctx->block_n;
   p.k_cols = kdim;
-  p.positions = a_pos;
-  p.k_out = static_cast<__nv_bfloat16 *>(k_out);
-  p.v_out = static_cast<__nv_bfloat16 *>(v_out);
   p.out_row_stride = out_row_stride;
   p.inv_d_hidden = 1.0f / static_cast<float>(d.d_hidden);
   p.rms_eps = d.rms_eps;
@@ -379,7 +425,43 @@ extern "C" kvd_status kvd_recompute_kv(kvd_ctx *ctx, int layer, const void *rows
     const size_t ctas = 2 * static_cast<size_t>(tiles < ctx->num_sms / 2 ? tiles : ctx->num_sms / 2);
     if (ctas * RC_TRACE_TILES * RC_TRACE_FIELDS * sizeof(long long) <= ctx->trace_bytes) p.trace = ctx->trace;
   }
-  return launch_recompute(ctx, ls, tmap_a, p, static_cast<cudaStream_t>(stream_));
+  return launch_recompute(ctx, ls, tmap_store, tmap_ext, p, stream);
+}
+
+extern "C" kvd_status kvd_recompute_kv(kvd_ctx *ctx, int layer, const void *rows, const int32_t *positions, int n,
+                                       int seq, int first_row, void *k_out, void *v_out, int64_t out_row_stride,
+                                       void *stream_) {
+  if (!ctx || n < 0) return KVD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  if (!ctx->layers[layer].set) return KVD_ERR_STATE;
+  if (n == 0) return KVD_OK;
+  if (!k_out || !v_out) return KVD_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (rows) {
+    if (!positions) return KVD_ERR_INVALID_ARG;
+    return recompute_launch(ctx, layer, nullptr, 0, rows, positions, n, k_out, v_out, out_row_stride, stream);
+  }
+  if (positions) return KVD_ERR_INVALID_ARG;
+  if (!ctx->store_rows) return KVD_ERR_STATE;
+  kvd_store_range r;
+  r.seq = seq;
+  r.first_row = first_row;
+  r.n = n;
+  r.reserved = 0;
+  r.k_out = k_out;
+  r.v_out = v_out;
+  return recompute_launch(ctx, layer, &r, 1, nullptr, nullptr, 0, nullptr, nullptr, out_row_stride, stream);
+}
+
+extern "C" kvd_status kvd_recompute_kv_step(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
+                                            const void *rows, const int32_t *positions, int n_rows, void *k_rows_out,
+                                            void *v_rows_out, int64_t out_row_stride, void *stream_) {
+  if (!ctx || n_ranges < 0 || n_rows < 0) return KVD_ERR_INVALID_ARG;
+  if (n_ranges > KVD_MAX_STORE_RANGES || (n_ranges > 0 && !ranges)) return KVD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  if (!ctx->layers[layer].set) return KVD_ERR_STATE;
+  return recompute_launch(ctx, layer, ranges, n_ranges, rows, positions, n_rows, k_rows_out, v_rows_out, out_row_stride,
+                          static_cast<cudaStream_t>(stream_));
 }
 
 extern "C" kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, const void *q, const int32_t *q_pos,

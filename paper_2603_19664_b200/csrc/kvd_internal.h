@@ -28,15 +28,25 @@ constexpr int RC_TRACE_TILES = 8;    // tiles per CTA recorded when a trace buff
 constexpr int RC_TRACE_FIELDS = 16;  // int64 slots per (CTA, tile); see kvd_set_trace
 constexpr int RC_THREADS = 320;  // warp 2 TMA, warp 3 MMA, warps 0,1,8,9 row statistics, warps 4-7 epilogue
 
+constexpr int RC_MAX_JOBS = 65;  // row sources per launch: up to 64 store ranges and one caller buffer
+
+// One source of rows inside a launch.  Jobs own consecutive runs of 256-row blocks.
+struct RcJob {
+  int mb_start;  // first 256-row block of this job in the launch
+  int n;         // rows
+  int row0;      // first row: index into the store slab, or 0 for a caller buffer
+  int slab;      // store slab (sequence slot of this layer), or -1: rows come from the caller's buffer
+  const int32_t *positions;  // [n]
+  __nv_bfloat16 *k_out;      // row m of the job at k_out + m * out_row_stride
+  __nv_bfloat16 *v_out;
+};
+
 struct RecomputeParams {
-  int M;          // rows
+  int n_jobs;
   int num_k_blocks;  // d_hidden / 64
-  int num_m_blocks;
+  int num_m_blocks;  // over all jobs
   int num_n_blocks;
   int k_cols;  // n_kv * d_head: fused columns below this index are keys, the rest values
-  const int32_t *positions;  // [M]
-  __nv_bfloat16 *k_out;
-  __nv_bfloat16 *v_out;
   long long out_row_stride;
   float inv_d_hidden;
   float rms_eps;
@@ -50,6 +60,7 @@ struct RecomputeParams {
   int *status;
   unsigned long long timeout_ns;
   long long *trace;  // nullptr unless a trace buffer is attached
+  RcJob jobs[RC_MAX_JOBS];
 };
 
 // ------------------------------------------------------------------------------ decode attention
@@ -165,6 +176,7 @@ struct kvd_ctx {
   int32_t *store_pos = nullptr;
   int layers_stored = 0;
   std::vector<int> rows_stored;  // [layers_stored * max_seqs]
+  std::vector<CUtensorMap> store_maps;  // per stored layer: [max_seqs][max_tokens_per_seq][d_hidden]
   // attention scratch
   float *part_o = nullptr;
   float *part_ml = nullptr;
@@ -184,8 +196,8 @@ struct kvd_ctx {
 
 namespace kvd {
 // launchers implemented next to their kernels
-kvd_status launch_recompute(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_a, const RecomputeParams &p,
-                            cudaStream_t stream);
+kvd_status launch_recompute(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
+                            const CUtensorMap &tmap_rows, const RecomputeParams &p, cudaStream_t stream);
 kvd_status launch_attention(kvd_ctx *ctx, const AttnLaunch &L, int d_head, int group, cudaStream_t stream);
 kvd_status launch_prepare_weights(kvd_ctx *ctx, const __nv_bfloat16 *w, const __nv_bfloat16 *gamma, __nv_bfloat16 *wt,
                                   int d_hidden, int n_cols, cudaStream_t stream);

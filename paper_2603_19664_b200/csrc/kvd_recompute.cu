@@ -1,6 +1,8 @@
 // Fused K/V recomputation kernel (paper Eq. 13-14 with Eq. 1-2 and Eq. 11-12 folded in).
 //
 //   Y[M, 2*n_kv*d_head] = X[M, d_hidden] * W'          W' = diag(gamma) W_kv, bf16, K-major
+//   (the M rows of one launch may come from several sources -- ranges of the residual store of
+//    several sequences plus one caller buffer; each source owns a run of 256-row blocks)
 //   y <- y / sqrt(mean_i x_i^2 + eps)                   RMSNorm applied after the contraction
 //   K heads: optional RMS norm over d_head, scale gamma_k, rotation by the row's position
 //   K, V stored as bf16
@@ -116,8 +118,8 @@ __device__ __forceinline__ void umma_kblock_pair(uint32_t d_tmem, uint32_t a_lo,
 
 template <int BLOCK_N, int D_HEAD, bool TRACE>
 __global__ void __launch_bounds__(RC_THREADS, 1)
-kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                     const RecomputeParams p) {
+kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __grid_constant__ CUtensorMap tmap_rows,
+                     const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ RecomputeParams p) {
   using Cfg = RcCfg<BLOCK_N, D_HEAD>;
   constexpr int STAGES = Cfg::STAGES;
   static_assert(BLOCK_N % D_HEAD == 0, "a tile must hold whole heads");
@@ -152,19 +154,29 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
   // epilogue nothing overlaps) is a cheap value tile.  Falls back to row-major order when a tile
   // mixes key and value heads.
   const int nk_tiles = (p.k_cols % BLOCK_N == 0) ? p.k_cols / BLOCK_N : 0;
-  auto tile_coords = [&](int t, int &m0, int &n0) {
+  // tile -> (job, first row of this CTA's 128 rows within the job, first fused column)
+  auto tile_coords = [&](int t, int &job, int &m0, int &n0) {
+    int mb;
     if (nk_tiles == 0) {
-      m0 = (t / p.num_n_blocks) * (2 * RC_BLOCK_M);
+      mb = t / p.num_n_blocks;
       n0 = (t % p.num_n_blocks) * BLOCK_N;
     } else if (t < p.num_m_blocks * nk_tiles) {
-      m0 = (t / nk_tiles) * (2 * RC_BLOCK_M);
+      mb = t / nk_tiles;
       n0 = (t % nk_tiles) * BLOCK_N;
     } else {
       const int u = t - p.num_m_blocks * nk_tiles, nv = p.num_n_blocks - nk_tiles;
-      m0 = (u / nv) * (2 * RC_BLOCK_M);
+      mb = u / nv;
       n0 = (nk_tiles + u % nv) * BLOCK_N;
     }
-    m0 += static_cast<int>(cta_rank) * RC_BLOCK_M;  // this CTA's 128 rows of the 256-row tile
+    // jobs own consecutive runs of 256-row blocks: the last job whose first block is <= mb
+    int lo = 0, hi = p.n_jobs;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (p.jobs[mid].mb_start <= mb) lo = mid;
+      else hi = mid;
+    }
+    job = lo;
+    m0 = (mb - p.jobs[lo].mb_start) * (2 * RC_BLOCK_M) + static_cast<int>(cta_rank) * RC_BLOCK_M;
   };
   const unsigned long long tmo = p.timeout_ns;
 
@@ -182,7 +194,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     }
     *s_abort = 0;
     fence_mbar_init();
-    prefetch_tensormap(&tmap_a);
+    prefetch_tensormap(&tmap_store);
+    prefetch_tensormap(&tmap_rows);
     prefetch_tensormap(&tmap_b);
   }
   if (threadIdx.x < D_HEAD) s_gamma_k[threadIdx.x] = p.gamma_k ? p.gamma_k[threadIdx.x] : 1.0f;
@@ -208,9 +221,14 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       bool ok = true;
       int ti = 0;
       for (int t = cluster_id; t < num_tiles && ok; t += num_clusters, ++ti) {
-        int m0, n0;
-        tile_coords(t, m0, n0);
+        int job, m0, n0;
+        tile_coords(t, job, m0, n0);
         n0 += b_row_off;
+        // rows come from a slab of the residual store or from the caller's buffer (slab 0 of its map)
+        const int slab = p.jobs[job].slab;
+        const CUtensorMap *tmap_a = slab < 0 ? &tmap_rows : &tmap_store;
+        const int a_slab = slab < 0 ? 0 : slab;
+        m0 += p.jobs[job].row0;
         long long waited = 0;
         trace_put<TRACE>(p.trace, ti, 1);
         for (int k0 = 0; k0 < p.num_k_blocks * RC_BLOCK_K; k0 += RC_BLOCK_K) {
@@ -222,7 +240,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
           }
           if (TRACE) waited += clock64() - w0;
           mbar_arrive_expect_tx(full, Cfg::STAGE_BYTES);
-          tma_load_2d(dst, &tmap_a, full, k0, m0);
+          tma_load_3d(dst, tmap_a, full, k0, m0, a_slab);
           tma_load_2d(dst + Cfg::A_BYTES, &tmap_b, full, k0, n0);
           ++n_issued;
           full += 8u;
@@ -417,8 +435,9 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     uint32_t aph = 0;
     int ti = 0;
     for (int t = cluster_id; t < num_tiles; t += num_clusters, ++ti) {
-      int m0, n0;
-      tile_coords(t, m0, n0);
+      int job, m0, n0;
+      tile_coords(t, job, m0, n0);
+      const RcJob &J = p.jobs[job];
       // warp-uniform outcome: tcgen05.ld below is an aligned instruction
       if (!warp_wait(bar_tmem_full(a), aph, s_abort, tmo, lane) || !warp_wait(bar_stats_full(a), aph, s_abort, tmo, lane)) {
         raise(p.status, STATUS_TIMEOUT, s_abort);
@@ -427,9 +446,9 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
       tc_fence_after();
       if (TRACE && threadIdx.x == 4 * 32) trace_put<TRACE>(p.trace, ti, 6);
       const int m = m0 + row;
-      const bool valid = m < p.M;
+      const bool valid = m < J.n;
       const float rstd = s_rstd[a * RC_BLOCK_M + row];
-      int pos = valid ? p.positions[m] : 0;
+      int pos = valid ? J.positions[m] : 0;
       if (pos < 0 || pos >= p.max_pos) {
         atomicOr(p.status, STATUS_POSITION);
         pos = pos < 0 ? 0 : p.max_pos - 1;
@@ -446,7 +465,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         const uint32_t tcol = acc + hh * D_HEAD;
         if (col0 >= p.k_cols) {
           // ---- value head (Eq. 14): scale by 1/rms and store
-          __nv_bfloat16 *dst = p.v_out + static_cast<size_t>(m) * p.out_row_stride + (col0 - p.k_cols);
+          __nv_bfloat16 *dst = J.v_out + static_cast<size_t>(m) * p.out_row_stride + (col0 - p.k_cols);
 #pragma unroll 1
           for (int c = 0; c < D_HEAD / 32; ++c) {
             uint32_t r[32];
@@ -464,7 +483,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
           }
         } else {
           // ---- key head (Eq. 13): 1/rms, optional key norm, rotation R_pos
-          __nv_bfloat16 *dst = p.k_out + static_cast<size_t>(m) * p.out_row_stride + col0;
+          __nv_bfloat16 *dst = J.k_out + static_cast<size_t>(m) * p.out_row_stride + col0;
           float kscale = rstd;
           if (p.qk_norm) {
             float ss = 0.f;
@@ -589,8 +608,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
 
 // ------------------------------------------------------------------------------ host launcher
 template <int BLOCK_N, int D_HEAD, bool TRACE>
-static kvd_status launch_impl(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_a, const RecomputeParams &p,
-                              cudaStream_t stream) {
+static kvd_status launch_impl(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
+                              const CUtensorMap &tmap_rows, const RecomputeParams &p, cudaStream_t stream) {
   using Cfg = RcCfg<BLOCK_N, D_HEAD>;
   auto kern = kvd_recompute_kernel<BLOCK_N, D_HEAD, TRACE>;
   static bool configured[64] = {};
@@ -615,29 +634,29 @@ static kvd_status launch_impl(kvd_ctx *ctx, const LayerState &ls, const CUtensor
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  cudaError_t le = cudaLaunchKernelEx(&cfg, kern, tmap_a, ls.tmap_b, p);
+  cudaError_t le = cudaLaunchKernelEx(&cfg, kern, tmap_store, tmap_rows, ls.tmap_b, p);
   if (le != cudaSuccess) return cuda_fail(ctx, le, "launch recompute");
   ctx->launches += 1;
   return KVD_OK;
 }
 
 template <int BLOCK_N, int D_HEAD>
-static kvd_status launch_sel(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_a, const RecomputeParams &p,
-                             cudaStream_t stream) {
-  if (p.trace != nullptr) return launch_impl<BLOCK_N, D_HEAD, true>(ctx, ls, tmap_a, p, stream);
-  return launch_impl<BLOCK_N, D_HEAD, false>(ctx, ls, tmap_a, p, stream);
+static kvd_status launch_sel(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
+                             const CUtensorMap &tmap_rows, const RecomputeParams &p, cudaStream_t stream) {
+  if (p.trace != nullptr) return launch_impl<BLOCK_N, D_HEAD, true>(ctx, ls, tmap_store, tmap_rows, p, stream);
+  return launch_impl<BLOCK_N, D_HEAD, false>(ctx, ls, tmap_store, tmap_rows, p, stream);
 }
 
-kvd_status launch_recompute(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_a, const RecomputeParams &p,
-                            cudaStream_t stream) {
+kvd_status launch_recompute(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
+                            const CUtensorMap &tmap_rows, const RecomputeParams &p, cudaStream_t stream) {
   const int dh = ctx->desc.d_head;
   if (ctx->block_n == 256) {
-    if (dh == 256) return launch_sel<256, 256>(ctx, ls, tmap_a, p, stream);
-    if (dh == 128) return launch_sel<256, 128>(ctx, ls, tmap_a, p, stream);
-    if (dh == 64) return launch_sel<256, 64>(ctx, ls, tmap_a, p, stream);
+    if (dh == 256) return launch_sel<256, 256>(ctx, ls, tmap_store, tmap_rows, p, stream);
+    if (dh == 128) return launch_sel<256, 128>(ctx, ls, tmap_store, tmap_rows, p, stream);
+    if (dh == 64) return launch_sel<256, 64>(ctx, ls, tmap_store, tmap_rows, p, stream);
   } else if (ctx->block_n == 128) {
-    if (dh == 128) return launch_sel<128, 128>(ctx, ls, tmap_a, p, stream);
-    if (dh == 64) return launch_sel<128, 64>(ctx, ls, tmap_a, p, stream);
+    if (dh == 128) return launch_sel<128, 128>(ctx, ls, tmap_store, tmap_rows, p, stream);
+    if (dh == 64) return launch_sel<128, 64>(ctx, ls, tmap_store, tmap_rows, p, stream);
   }
   return KVD_ERR_SHAPE;
 }

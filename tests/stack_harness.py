@@ -136,16 +136,20 @@ class GpuStack:
             q = self._rope_q(q, pos, ls.rope_theta).to(torch.bfloat16).view(1, s.n_q_heads, s.d_head).contiguous()
             # hot path: K_t, V_t of the current token, written at its position in the live storage
             kl, vl = self.k_live[l], self.v_live[l]
-            ctx.kvd_recompute_kv(l, h, pos_t, 1, kl[pos:], vl[pos:], self.kdim)
             lo = 0 if ls.sliding_window == 0 else max(0, pos - ls.sliding_window + 1)
             wf = self.win_first[l] if self.policy == "kvdirect" else 0
             wf = min(wf, pos)
             segs = []
             if self.policy == "kvdirect" and lo < wf:
-                n = wf - lo  # evicted tokens this layer still attends to: RECOMPUTE_KV(C, l)
-                ctx.kvd_recompute_kv(l, None, None, n, self.k_old, self.v_old, self.kdim, seq=0, first_row=lo)
+                # evicted tokens this layer still attends to: RECOMPUTE_KV(C, l), in the same launch
+                # as K_t, V_t of the current token
+                n = wf - lo
+                ctx.kvd_recompute_kv_step(l, [(0, lo, n, self.k_old, self.v_old)], h, pos_t, 1, kl[pos:], vl[pos:],
+                                          self.kdim)
                 self.recomputed_rows += n
                 segs.append((self.k_old, self.v_old, self.kdim, lo, n))
+            else:
+                ctx.kvd_recompute_kv(l, h, pos_t, 1, kl[pos:], vl[pos:], self.kdim)
             first_live = max(wf, lo) if self.policy == "kvdirect" else 0
             segs.append((kl[first_live:], vl[first_live:], self.kdim, first_live, pos + 1 - first_live))
             out = torch.empty((1, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")

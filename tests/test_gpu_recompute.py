@@ -187,6 +187,112 @@ def test_checkpoint_store_roundtrip_and_recompute_from_store():
     assert ctx.kvd_rows_stored(0, 1) == 0
 
 
+@pytest.mark.parametrize("shape", [SMOLLM2_135M, GEMMA3_4B_GLOBAL], ids=lambda s: s.name)
+def test_step_call_matches_separate_calls_bit_for_bit(shape):
+    """kvd_recompute_kv_step: ranges of three sequences (ragged, non-zero first rows, one empty) plus
+    new-token rows in one launch == one kvd_recompute_kv call per source, and within tolerance of
+    the oracle; rows after each range's end are left untouched."""
+    ctx, w = open_layer(shape, max_tokens=1024, max_seqs=4, with_store=True)
+    kdim = shape.n_kv_heads * shape.d_head
+    n_seq = [700, 300, 0, 513]
+    Xs, Ps = [], []
+    for s, n in enumerate(n_seq):
+        X = make_residuals(shape, max(n, 1), seed=40 + s)[:n]
+        pos = (np.arange(n) + 3 * s).astype(np.int32)
+        Xs.append(X)
+        Ps.append(pos)
+        if n:
+            ctx.kvd_checkpoint_residual(s, 0, dev(X), torch.from_numpy(pos).cuda(), n)
+    ranges_spec = [(0, 37, 600), (1, 0, 300), (2, 0, 0), (3, 256, 257)]
+    Xn = make_residuals(shape, 3, seed=50)
+    pn = np.array([700, 303, 519], np.int32)
+    xn, pnd = dev(Xn), torch.from_numpy(pn).cuda()
+
+    def outputs():
+        ks = [torch.full((n + 2, kdim), -7.0, dtype=torch.bfloat16, device="cuda") for (_, _, n) in ranges_spec]
+        vs = [torch.full((n + 2, kdim), -7.0, dtype=torch.bfloat16, device="cuda") for (_, _, n) in ranges_spec]
+        kn = torch.full((3 + 2, kdim), -7.0, dtype=torch.bfloat16, device="cuda")
+        vn = torch.full((3 + 2, kdim), -7.0, dtype=torch.bfloat16, device="cuda")
+        return ks, vs, kn, vn
+
+    ks, vs, kn, vn = outputs()
+    launches = ctx.kvd_launch_count()
+    ctx.kvd_recompute_kv_step(0, [(s, f, n, ks[i], vs[i]) for i, (s, f, n) in enumerate(ranges_spec)], xn, pnd, 3,
+                              kn, vn, kdim)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    assert ctx.kvd_launch_count() == launches + 1
+    ks2, vs2, kn2, vn2 = outputs()
+    for i, (s, f, n) in enumerate(ranges_spec):
+        ctx.kvd_recompute_kv(0, None, None, n, ks2[i], vs2[i], kdim, seq=s, first_row=f)
+    ctx.kvd_recompute_kv(0, xn, pnd, 3, kn2, vn2, kdim)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    for a, b in zip(ks + vs + [kn, vn], ks2 + vs2 + [kn2, vn2]):
+        assert torch.equal(a, b)
+    sentinel = host_bits(torch.full((1,), -7.0, dtype=torch.bfloat16))[0]
+    for i, (s, f, n) in enumerate(ranges_spec):
+        assert np.all(host_bits(ks[i])[n:] == sentinel) and np.all(host_bits(vs[i])[n:] == sentinel)
+        if n:
+            Kr, Vr = oracle_kv(shape, w, Xs[s][f:f + n], Ps[s][f:f + n])
+            check(shape, ks[i][:n], vs[i][:n], Kr, Vr)
+    assert np.all(host_bits(kn)[3:] == sentinel) and np.all(host_bits(vn)[3:] == sentinel)
+    Kr, Vr = oracle_kv(shape, w, Xn, pn)
+    check(shape, kn[:3], vn[:3], Kr, Vr)
+    # ranges only; rows only
+    ks3, vs3, kn3, vn3 = outputs()
+    ctx.kvd_recompute_kv_step(0, [(s, f, n, ks3[i], vs3[i]) for i, (s, f, n) in enumerate(ranges_spec)], None, None, 0,
+                              None, None, kdim)
+    ctx.kvd_recompute_kv_step(0, [], xn, pnd, 3, kn3, vn3, kdim)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    for a, b in zip(ks + vs + [kn, vn], ks3 + vs3 + [kn3, vn3]):
+        assert torch.equal(a, b)
+    # a range past the stored rows rejects the whole call before anything is launched
+    launches = ctx.kvd_launch_count()
+    with pytest.raises(kvd.KvdError) as e:
+        ctx.kvd_recompute_kv_step(0, [(0, 0, 10, ks[0], vs[0]), (1, 290, 11, ks[1], vs[1])], xn, pnd, 3, kn, vn, kdim)
+    assert e.value.status == 4
+    with pytest.raises(kvd.KvdError) as e:
+        ctx.kvd_recompute_kv_step(0, [(0, 0, 1, ks[0], vs[0])] * 65, None, None, 0, None, None, kdim)
+    assert e.value.status == 1
+    assert ctx.kvd_launch_count() == launches
+
+
+def test_step_call_with_64_sequences():
+    """A batch of 64 sequences with different evicted lengths and 64 new tokens in one launch."""
+    shape = TINY_GQA
+    ctx, w = open_layer(shape, max_tokens=640, max_seqs=64, max_batch=64, with_store=True)
+    kdim = shape.n_kv_heads * shape.d_head
+    rng = np.random.default_rng(77)
+    lens = rng.integers(1, 600, size=64)
+    ranges, refs = [], []
+    for s in range(64):
+        n = int(lens[s])
+        X = make_residuals(shape, n, seed=900 + s)
+        pos = np.arange(n, dtype=np.int32)
+        ctx.kvd_checkpoint_residual(s, 0, dev(X), torch.from_numpy(pos).cuda(), n)
+        k = torch.zeros((n, kdim), dtype=torch.bfloat16, device="cuda")
+        v = torch.zeros_like(k)
+        ranges.append((s, 0, n, k, v))
+        refs.append((X, pos))
+    Xn = make_residuals(shape, 64, seed=990)
+    pn = lens.astype(np.int32)
+    kn = torch.zeros((64, kdim), dtype=torch.bfloat16, device="cuda")
+    vn = torch.zeros_like(kn)
+    ctx.kvd_recompute_kv_step(0, ranges, dev(Xn), torch.from_numpy(pn).cuda(), 64, kn, vn, kdim)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    for s in (0, 1, 17, 40, 63):
+        Kr, Vr = oracle_kv(shape, w, *refs[s])
+        check(shape, ranges[s][3], ranges[s][4], Kr, Vr)
+    Kr, Vr = oracle_kv(shape, w, Xn, pn)
+    check(shape, kn, vn, Kr, Vr)
+    # every range equals the single-source call
+    for s in (5, 33, 62):
+        n = int(lens[s])
+        k = torch.zeros((n, kdim), dtype=torch.bfloat16, device="cuda")
+        v = torch.zeros_like(k)
+        ctx.kvd_recompute_kv(0, None, None, n, k, v, kdim, seq=s, first_row=0)
+        assert torch.equal(k, ranges[s][3]) and torch.equal(v, ranges[s][4])
+
+
 def test_argument_errors_and_position_flag():
     shape = TINY_GQA
     ctx, w = open_layer(shape, max_tokens=1024)
