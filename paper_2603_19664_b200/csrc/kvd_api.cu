@@ -68,22 +68,15 @@ extern "C" size_t kvd_store_bytes(const kvd_model_desc *d, int layers_stored) {
   return round_up(slots * d->d_hidden * 2, 256) + round_up(slots * 4, 256);
 }
 
-// chunk partials plus first-level group partials of one sequence
+// chunk partials of one sequence
 static size_t parts_per_seq(const kvd_model_desc *d) {
-  const size_t chunks = attn_max_chunks(d->d_head, d->n_kv_heads, d->max_tokens_per_seq);
-  return chunks + (chunks + AT_MERGE_GROUP - 1) / AT_MERGE_GROUP + 1;
-}
-static size_t groups_per_seq(const kvd_model_desc *d) {
-  const size_t chunks = attn_max_chunks(d->d_head, d->n_kv_heads, d->max_tokens_per_seq);
-  return (chunks + AT_MERGE_GROUP - 1) / AT_MERGE_GROUP + 1;
+  return attn_max_chunks(d->d_head, d->n_kv_heads, d->max_tokens_per_seq);
 }
 
 extern "C" size_t kvd_workspace_bytes(const kvd_model_desc *d) {
   if (check_desc(d) != KVD_OK) return 0;
   const size_t parts = static_cast<size_t>(d->max_batch) * parts_per_seq(d);
-  const size_t counters = static_cast<size_t>(d->max_batch) * d->n_kv_heads * (1 + groups_per_seq(d));
-  return round_up(parts * d->n_q_heads * d->d_head * 4, 256) + round_up(parts * d->n_q_heads * 2 * 4, 256) +
-         round_up(counters * 4, 256);
+  return round_up(parts * d->n_q_heads * d->d_head * 4, 256) + round_up(parts * d->n_q_heads * 2 * 4, 256);
 }
 
 extern "C" kvd_status kvd_create(const kvd_model_desc *desc, kvd_ctx **out) {
@@ -314,13 +307,6 @@ extern "C" kvd_status kvd_attach_workspace(kvd_ctx *ctx, void *ws, size_t bytes)
   ctx->part_o = static_cast<float *>(ws);
   uint8_t *base = static_cast<uint8_t *>(ws);
   ctx->part_ml = reinterpret_cast<float *>(base + round_up(parts * d.n_q_heads * d.d_head * 4, 256));
-  ctx->counters = reinterpret_cast<int *>(base + round_up(parts * d.n_q_heads * d.d_head * 4, 256) +
-                                          round_up(parts * d.n_q_heads * 2 * 4, 256));
-  // the per-(sequence, head) arrival counters must start at zero; kernels leave them at zero
-  ctx->max_groups = static_cast<int>(groups_per_seq(&d));
-  cudaError_t e = cudaMemset(ctx->counters, 0,
-                             static_cast<size_t>(d.max_batch) * d.n_kv_heads * (1 + ctx->max_groups) * 4);
-  if (e != cudaSuccess) return cuda_fail(ctx, e, "kvd_attach_workspace memset");
   ctx->max_parts = static_cast<int>(parts);
   ctx->workspace_bytes = need;
   return KVD_OK;
@@ -532,7 +518,6 @@ extern "C" kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, c
       S.lo_pos = lo;
       S.hi_pos = hi;
       S.part_base = parts;
-      S.group_base = 0;
       if (max_last < 0 || hi < lo) {
         S.n_chunks = 0;
         S.iters = 1;
@@ -546,14 +531,7 @@ extern "C" kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, c
       }
       parts += S.n_chunks;
     }
-    int groups = 0;
-    for (int i = 0; i < nb; ++i) {  // group partials live behind the launch's chunk partials
-      L.seq[i].group_base = parts + groups;
-      groups += (L.seq[i].n_chunks + AT_MERGE_GROUP - 1) / AT_MERGE_GROUP;
-    }
-    if (parts + groups > ctx->max_parts) return KVD_ERR_CAPACITY;
-    L.max_groups = ctx->max_groups;
-    L.cnt1_off = d.max_batch * d.n_kv_heads;
+    if (parts > ctx->max_parts) return KVD_ERR_CAPACITY;
     L.n_seqs = nb;
     L.total_chunks = parts;
     L.n_q = d.n_q_heads;
@@ -562,17 +540,8 @@ extern "C" kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, c
     L.out = static_cast<__nv_bfloat16 *>(out) + static_cast<size_t>(b0) * d.n_q_heads * d.d_head;
     L.part_o = ctx->part_o;
     L.part_ml = ctx->part_ml;
-    L.counters = ctx->counters;
-    L.seq0 = b0;
     L.scale_log2e = sc * 1.4426950408889634f;
-    // sequences without a visible key launch no work: their output is all zeros
-    for (int i = 0; i < nb; ++i) {
-      if (L.seq[i].n_chunks == 0) {
-        cudaError_t me = cudaMemsetAsync(L.out + static_cast<size_t>(i) * d.n_q_heads * d.d_head, 0,
-                                         static_cast<size_t>(d.n_q_heads) * d.d_head * 2, stream);
-        if (me != cudaSuccess) return cuda_fail(ctx, me, "zero output");
-      }
-    }
+    // sequences without a visible key stream nothing; the merge kernel writes their zeros
     kvd_status st = launch_attention(ctx, L, d.d_head, group, stream);
     if (st != KVD_OK) return st;
   }

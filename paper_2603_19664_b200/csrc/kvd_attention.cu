@@ -6,9 +6,10 @@
 // coalesced 16-byte loads, every lane owning 8 channels, and serves all query heads of the group
 // from the same loads.  Scores of 8 keys at a time are reduced across the lanes of a key with a
 // transposing shuffle butterfly, the softmax runs online in base 2, and each CTA writes one partial
-// (max, sum, unnormalised output) per query head.  The CTA that finishes last for a (sequence, KV
-// head) -- found with one atomic counter, no waiting -- merges that head group's partials in chunk
-// order and writes the output, so a decode step is a single launch.
+// (max, sum, unnormalised output) per query head.  A second, small kernel merges each head group's
+// partials in chunk order and writes the output.  CTAs are 16 warps (one per SM): a long sequence
+// then yields only 148 / n_kv partials per head, few enough for a single merge level that costs
+// one round trip to the L2.
 //
 // Which chunk, warp, lane group and slot a key lands in is a function of its position only, and the
 // merge runs in chunk order, so the output bits do not depend on how the keys are spread over
@@ -86,15 +87,16 @@ __device__ __forceinline__ float reduce8_transposed(const float (&v)[8], int lig
 }
 
 template <int D_HEAD, int G, int NSEQ>
-__global__ void __launch_bounds__(AT_THREADS, 4) kvd_attn_split_kernel(const __grid_constant__ AttnLaunchT<NSEQ> P) {
+__global__ void __launch_bounds__(AT_THREADS, 1) kvd_attn_split_kernel(const __grid_constant__ AttnLaunchT<NSEQ> P) {
   constexpr int LPK = D_HEAD / 8;         // lanes per key
   constexpr int KPL = 32 / LPK;           // keys per warp-wide load
   constexpr int U = AT_UNROLL;            // keys per lane group per iteration
   constexpr int NPART = AT_WARPS * KPL;   // lane groups per CTA
-  __shared__ float s_o[NPART][G][D_HEAD];
-  __shared__ float s_m[NPART][G];
-  __shared__ float s_l[NPART][G];
-  __shared__ int s_last;
+  // per lane group: unnormalised output, maximum, sum (AttnSmem<D_HEAD, G>::BYTES of dynamic shared memory)
+  extern __shared__ __align__(16) float at_smem[];
+  float (*s_o)[G][D_HEAD] = reinterpret_cast<float (*)[G][D_HEAD]>(at_smem);
+  float (*s_m)[G] = reinterpret_cast<float (*)[G]>(at_smem + NPART * G * D_HEAD);
+  float (*s_l)[G] = s_m + NPART;
 
   // ---- which (sequence, chunk) is this CTA's?
   int si = 0;
@@ -273,9 +275,9 @@ __global__ void __launch_bounds__(AT_THREADS, 4) kvd_attn_split_kernel(const __g
     if (__any_sync(0xffffffffu, vmask != 0u)) compute(kr, vr, vmask);
   };
 
-  // One buffer of loads per iteration; latency is hidden by the other CTAs resident on the SM (the
-  // kernel is capped at 128 registers so that four fit), which measured faster than register double
-  // buffering or a shared-memory ring at half the occupancy.
+  // One buffer of loads per iteration; latency is hidden by the other 15 warps of the CTA (the
+  // kernel is capped at 128 registers so that 16 warps fit an SM), which measured faster than
+  // register double buffering or a shared-memory ring at half the occupancy.
   {
     uint4 ka[U], va[U];
     uint32_t ma = 0;
@@ -310,11 +312,11 @@ __global__ void __launch_bounds__(AT_THREADS, 4) kvd_attn_split_kernel(const __g
   for (int idx = threadIdx.x; idx < G * D_HEAD; idx += AT_THREADS) {
     const int g = idx / D_HEAD, c = idx % D_HEAD;
     float M = -CUDART_INF_F;
-#pragma unroll
+#pragma unroll 8
     for (int pp = 0; pp < NPART; ++pp) M = fmaxf(M, s_m[pp][g]);
     const float Mu = (M == -CUDART_INF_F) ? 0.f : M;
     float o = 0.f, l = 0.f;
-#pragma unroll
+#pragma unroll 8
     for (int pp = 0; pp < NPART; ++pp) {
       const float w = exp2f(s_m[pp][g] - Mu);
       o = fmaf(w, s_o[pp][g][c], o);
@@ -327,151 +329,165 @@ __global__ void __launch_bounds__(AT_THREADS, 4) kvd_attn_split_kernel(const __g
       P.part_ml[hq * 2 + 1] = l;
     }
   }
+}
 
-  // ---- two-level merge without waiting.  Chunks are grouped 16 at a time by chunk index (one group
-  // of everything when there are at most 64); the CTA
-  // that arrives last on a group's counter merges that group's partials into one group partial (this
-  // happens while other groups are still streaming), and the CTA that completes the last group merges
-  // the group partials and writes the output.  Grouping and order depend on chunk indices only.
+// Second kernel of a decode step: one CTA per (sequence, KV head) merges that head group's chunk
+// partials in chunk order and writes the output.  A separate launch instead of a "last CTA merges"
+// tail: every dependent global-memory hop (partial -> fence -> counter -> merge) measured above a
+// microsecond, which the streaming CTAs would spend idle on their SM; the kernel boundary costs about
+// as much once per step and needs no counters.  A sequence without a visible key gets zeros.
+template <int D_HEAD, int G, int NSEQ>
+__global__ void __launch_bounds__(AT_THREADS, 1) kvd_attn_merge_kernel(const __grid_constant__ AttnLaunchT<NSEQ> P) {
+  extern __shared__ __align__(16) float at_smem[];
+  float (*s_o)[G][D_HEAD] = reinterpret_cast<float (*)[G][D_HEAD]>(at_smem);  // [AT_WARPS]
+  float (*s_l)[G] = reinterpret_cast<float (*)[G]>(at_smem + AT_WARPS * G * D_HEAD);
+  const int si = blockIdx.x / P.n_kv, kvh = blockIdx.x % P.n_kv;
+  const AttnSeq &S = P.seq[si];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // Every warp finds the maximum of each head by itself (lanes over partials, shuffles -- no block
+  // barrier), then sums a contiguous sixteenth of the partials scaled to it, each lane owning CPL
+  // channels of every head; the warp results are added in warp order.  All loads of a warp's first
+  // PF partials are issued before the maxima are known, so the merge costs about one round trip to
+  // the L2.
   constexpr int CPL = D_HEAD / 32;  // channels per lane
-  float *s_M = &s_m[0][0];          // [G] maximum used for scaling (0 when nothing is visible)
-  float *s_Mraw = &s_m[1][0];       // [G] the maximum itself (NPART >= 4 rows are available)
+  // partials fetched ahead (bounded by the registers they take)
+  constexpr int PF = 64 / (G * CPL) >= 4 ? 4 : (64 / (G * CPL) >= 1 ? 64 / (G * CPL) : 1);
+  const int count = S.n_chunks;
+  const float *ml0 = P.part_ml + (static_cast<size_t>(S.part_base) * P.n_q + kvh * G) * 2;
+  const float *po0 = P.part_o + (static_cast<size_t>(S.part_base) * P.n_q + kvh * G) * D_HEAD;
   const size_t ml_stride = static_cast<size_t>(P.n_q) * 2, po_stride = static_cast<size_t>(P.n_q) * D_HEAD;
-
-  // Merge `count` consecutive partials starting at part index `first` for this CTA's head group.
-  // Pass 1: the maximum of each head.  Pass 2: every warp sums a contiguous quarter of the partials
-  // scaled to the common maximum, each lane owning CPL channels of every head; the four warp results
-  // are added in warp order.  The result becomes the partial `dst` or, normalised, the output.
-  auto merge = [&](size_t first, int count, bool final, size_t dst) {
-    const float *ml0 = P.part_ml + (first * P.n_q + kvh * G) * 2;
-    const float *po0 = P.part_o + (first * P.n_q + kvh * G) * D_HEAD;
-    __syncthreads();
+  const int per_warp = (count + AT_WARPS - 1) / AT_WARPS;
+  const int c_begin = warp * per_warp;
+  const int c_end = c_begin + per_warp < count ? c_begin + per_warp : count;
+  float vbuf[PF][G][CPL];
+  float2 mlbuf[PF][G];
+  auto fetch = [&](int ch, float (&d)[G][CPL], float2 (&dm)[G]) {
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      float mx = -CUDART_INF_F;
-      for (int ch = threadIdx.x; ch < count; ch += AT_THREADS) mx = fmaxf(mx, __ldcg(ml0 + ch * ml_stride + g * 2));
+      dm[g] = __ldcg(reinterpret_cast<const float2 *>(ml0 + ch * ml_stride + g * 2));
+      const float *src = po0 + ch * po_stride + g * D_HEAD + lane * CPL;
+      if constexpr (CPL == 2) {
+        const float2 v = __ldcg(reinterpret_cast<const float2 *>(src));
+        d[g][0] = v.x;
+        d[g][1] = v.y;
+      } else {
 #pragma unroll
-      for (int msk = 16; msk >= 1; msk >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, msk));
-      if (lane == 0) s_l[warp][g] = mx;
-    }
-    __syncthreads();
-    if (threadIdx.x < G) {
-      float mx = s_l[0][threadIdx.x];
-#pragma unroll
-      for (int w = 1; w < AT_WARPS; ++w) mx = fmaxf(mx, s_l[w][threadIdx.x]);
-      s_Mraw[threadIdx.x] = mx;
-      s_M[threadIdx.x] = (mx == -CUDART_INF_F) ? 0.f : mx;
-    }
-    __syncthreads();
-    {
-      float o[G][CPL], l[G];
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        l[g] = 0.f;
-#pragma unroll
-        for (int e = 0; e < CPL; ++e) o[g][e] = 0.f;
+        for (int e = 0; e < CPL; e += 4) {
+          const float4 v = __ldcg(reinterpret_cast<const float4 *>(src + e));
+          d[g][e] = v.x;
+          d[g][e + 1] = v.y;
+          d[g][e + 2] = v.z;
+          d[g][e + 3] = v.w;
+        }
       }
-      const int per_warp = (count + AT_WARPS - 1) / AT_WARPS;
-      const int c_begin = warp * per_warp;
-      const int c_end = c_begin + per_warp < count ? c_begin + per_warp : count;
-#pragma unroll 4
-      for (int ch = c_begin; ch < c_end; ++ch) {
+    }
+  };
+#pragma unroll
+  for (int i = 0; i < PF; ++i)
+    if (c_begin + i < c_end) fetch(c_begin + i, vbuf[i], mlbuf[i]);
+  float Mu[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    float mx = -CUDART_INF_F;
+    for (int ch = lane; ch < count; ch += 32) mx = fmaxf(mx, __ldcg(ml0 + ch * ml_stride + g * 2));
+#pragma unroll
+    for (int msk = 16; msk >= 1; msk >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, msk));
+    Mu[g] = (mx == -CUDART_INF_F) ? 0.f : mx;
+  }
+  float o[G][CPL], l[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    l[g] = 0.f;
+#pragma unroll
+    for (int e = 0; e < CPL; ++e) o[g][e] = 0.f;
+  }
+  for (int base = c_begin; base < c_end; base += PF) {
+#pragma unroll
+    for (int i = 0; i < PF; ++i) {
+      const int ch = base + i;
+      if (ch < c_end) {
 #pragma unroll
         for (int g = 0; g < G; ++g) {
-          const float2 mlv = __ldcg(reinterpret_cast<const float2 *>(ml0 + ch * ml_stride + g * 2));
-          const float w = exp2f(mlv.x - s_M[g]);
-          l[g] = fmaf(w, mlv.y, l[g]);
-          const float *src = po0 + ch * po_stride + g * D_HEAD + lane * CPL;
-          if constexpr (CPL == 2) {
-            const float2 v = __ldcg(reinterpret_cast<const float2 *>(src));
-            o[g][0] = fmaf(w, v.x, o[g][0]);
-            o[g][1] = fmaf(w, v.y, o[g][1]);
-          } else {
+          const float w = exp2f(mlbuf[i][g].x - Mu[g]);
+          l[g] = fmaf(w, mlbuf[i][g].y, l[g]);
 #pragma unroll
-            for (int e = 0; e < CPL; e += 4) {
-              const float4 v = __ldcg(reinterpret_cast<const float4 *>(src + e));
-              o[g][e] = fmaf(w, v.x, o[g][e]);
-              o[g][e + 1] = fmaf(w, v.y, o[g][e + 1]);
-              o[g][e + 2] = fmaf(w, v.z, o[g][e + 2]);
-              o[g][e + 3] = fmaf(w, v.w, o[g][e + 3]);
-            }
-          }
+          for (int e = 0; e < CPL; ++e) o[g][e] = fmaf(w, vbuf[i][g][e], o[g][e]);
         }
-      }
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        if (lane == 0) s_l[warp][g] = l[g];
-#pragma unroll
-        for (int e = 0; e < CPL; ++e) s_o[warp][g][lane * CPL + e] = o[g][e];
+        if (ch + PF < c_end) fetch(ch + PF, vbuf[i], mlbuf[i]);
       }
     }
-    __syncthreads();
-    for (int idx = threadIdx.x; idx < G * D_HEAD; idx += AT_THREADS) {
-      const int g = idx / D_HEAD, c = idx % D_HEAD;
-      float o = s_o[0][g][c], l = s_l[0][g];
-#pragma unroll
-      for (int w = 1; w < AT_WARPS; ++w) {
-        o += s_o[w][g][c];
-        l += s_l[w][g];
-      }
-      if (final) {
-        const float r = l > 0.f ? o / l : 0.f;
-        P.out[(static_cast<size_t>(si) * P.n_q + kvh * G + g) * D_HEAD + c] = __float2bfloat16_rn(r);
-      } else {
-        const size_t hq = dst * P.n_q + kvh * G + g;
-        P.part_o[hq * D_HEAD + c] = o;
-        if (c == 0) {
-          P.part_ml[hq * 2] = s_Mraw[g];
-          P.part_ml[hq * 2 + 1] = l;
-        }
-      }
-    }
-  };
-
-  // arrive on `cnt`; true for the CTA that is the `expected`-th (last) arrival, which also resets it
-  auto arrive_last = [&](int *cnt, int expected) -> bool {
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      const int old = atomicAdd(cnt, 1);
-      s_last = (old == expected - 1) ? 1 : 0;
-      if (s_last) *cnt = 0;  // ready for the next call
-    }
-    __syncthreads();
-    const bool last = s_last != 0;
-    if (last) __threadfence();
-    return last;
-  };
-
-  // up to 64 chunks are merged in one go (a second level would only add latency)
-  const int gsz = S.n_chunks <= 64 ? 64 : AT_MERGE_GROUP;
-  const int n_groups = (S.n_chunks + gsz - 1) / gsz;
-  const int grp_idx = chunk / gsz;
-  const int grp_size = S.n_chunks - grp_idx * gsz < gsz ? S.n_chunks - grp_idx * gsz : gsz;
-  const int head_slot = (P.seq0 + si) * P.n_kv + kvh;
-  int *cnt1 = P.counters + P.cnt1_off + static_cast<size_t>(head_slot) * P.max_groups + grp_idx;
-  int *cnt2 = P.counters + head_slot;
-  if (!arrive_last(cnt1, grp_size)) return;
-  const size_t first = static_cast<size_t>(S.part_base) + static_cast<size_t>(grp_idx) * gsz;
-  if (n_groups == 1) {
-    merge(first, grp_size, true, 0);
-    return;
   }
-  merge(first, grp_size, false, static_cast<size_t>(S.group_base) + grp_idx);
-  if (!arrive_last(cnt2, n_groups)) return;
-  merge(static_cast<size_t>(S.group_base), n_groups, true, 0);
+  // the warp sums are added in warp order
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    if (lane == 0) s_l[warp][g] = l[g];
+#pragma unroll
+    for (int e = 0; e < CPL; ++e) s_o[warp][g][lane * CPL + e] = o[g][e];
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < G * D_HEAD; idx += AT_THREADS) {
+    const int g = idx / D_HEAD, c = idx % D_HEAD;
+    float ov = s_o[0][g][c], lv = s_l[0][g];
+#pragma unroll
+    for (int w = 1; w < AT_WARPS; ++w) {
+      ov += s_o[w][g][c];
+      lv += s_l[w][g];
+    }
+    const float r = lv > 0.f ? ov / lv : 0.f;
+    P.out[(static_cast<size_t>(si) * P.n_q + kvh * G + g) * D_HEAD + c] = __float2bfloat16_rn(r);
+  }
+}
+
+// dynamic shared memory of the kernel and its one-time opt-in (sizes above 48 KB need it)
+template <int D_HEAD, int G>
+struct AttnSmem {
+  static constexpr int NPART = AT_WARPS * (32 / (D_HEAD / 8));
+  static constexpr int BYTES = NPART * G * (D_HEAD + 2) * 4;
+  static constexpr int MERGE_BYTES = AT_WARPS * G * (D_HEAD + 1) * 4;
+};
+template <int D_HEAD, int G, int NSEQ>
+static cudaError_t attn_configure() {
+  static bool done[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (!done[dev & 63]) {
+    e = cudaFuncSetAttribute(kvd_attn_split_kernel<D_HEAD, G, NSEQ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             AttnSmem<D_HEAD, G>::BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(kvd_attn_merge_kernel<D_HEAD, G, NSEQ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             AttnSmem<D_HEAD, G>::MERGE_BYTES);
+    if (e != cudaSuccess) return e;
+    done[dev & 63] = true;
+  }
+  return cudaSuccess;
+}
+// the two launches of a decode step: stream + partials, then merge
+template <int D_HEAD, int G, int NSEQ>
+static cudaError_t attn_launch_pair(const AttnLaunchT<NSEQ> &S, cudaStream_t stream) {
+  cudaError_t e = attn_configure<D_HEAD, G, NSEQ>();
+  if (e != cudaSuccess) return e;
+  if (S.total_chunks > 0) {
+    kvd_attn_split_kernel<D_HEAD, G, NSEQ>
+        <<<S.total_chunks * S.n_kv, AT_THREADS, AttnSmem<D_HEAD, G>::BYTES, stream>>>(S);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  kvd_attn_merge_kernel<D_HEAD, G, NSEQ>
+      <<<S.n_seqs * S.n_kv, AT_THREADS, AttnSmem<D_HEAD, G>::MERGE_BYTES, stream>>>(S);
+  return cudaGetLastError();
 }
 
 template <int D_HEAD, int G, int NSEQ>
 static kvd_status launch_attn_impl(kvd_ctx *ctx, const AttnLaunch &L, cudaStream_t stream) {
-  if (L.total_chunks > 0) {
+  if (L.n_seqs > 0) {
     static thread_local AttnLaunchT<NSEQ> S;
     static_cast<AttnLaunchHead &>(S) = static_cast<const AttnLaunchHead &>(L);
     for (int i = 0; i < L.n_seqs; ++i) S.seq[i] = L.seq[i];
-    kvd_attn_split_kernel<D_HEAD, G, NSEQ><<<L.total_chunks * L.n_kv, AT_THREADS, 0, stream>>>(S);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = attn_launch_pair<D_HEAD, G, NSEQ>(S, stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch attention");
-    ctx->launches += 1;
+    ctx->launches += L.total_chunks > 0 ? 2 : 1;
   }
   return KVD_OK;
 }
@@ -508,7 +524,7 @@ kvd_status launch_attention(kvd_ctx *ctx, const AttnLaunch &L, int d_head, int g
 // ------------------------------------------------------------------------------------------------
 // kvd_decode_attention_static: decode attention for callers that cannot allocate device memory.
 //
-// The split partials and the arrival counters live in the file-scope device array below instead of
+// The split partials live in the file-scope device array below instead of
 // a caller-provided workspace.  Every GPU that loads this library holds the array until the process
 // exits.  All calls share it, so two calls whose kernels overlap on one GPU race on it.
 // ------------------------------------------------------------------------------------------------
@@ -544,8 +560,11 @@ static kvd_status static_launch_g(const AttnLaunch &L, cudaStream_t stream) {
   static thread_local AttnLaunchT<AT_MAX_SEQS> S;
   static_cast<AttnLaunchHead &>(S) = static_cast<const AttnLaunchHead &>(L);
   for (int i = 0; i < L.n_seqs; ++i) S.seq[i] = L.seq[i];
-  kvd_attn_split_kernel<D_HEAD, G, AT_MAX_SEQS><<<L.total_chunks * L.n_kv, AT_THREADS, 0, stream>>>(S);
-  return cudaGetLastError() == cudaSuccess ? KVD_OK : KVD_ERR_CUDA;
+  if (attn_launch_pair<D_HEAD, G, AT_MAX_SEQS>(S, stream) != cudaSuccess) {
+    cudaGetLastError();
+    return KVD_ERR_CUDA;
+  }
+  return KVD_OK;
 }
 
 template <int D_HEAD>
@@ -578,7 +597,7 @@ extern "C" kvd_status kvd_decode_attention_static(int n_q_heads, int n_kv_heads,
   if (batch == 0) return KVD_OK;
   if (!q || !q_pos || !out || (n_segs > 0 && !segs)) return KVD_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(q) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u)) return KVD_ERR_ALIGNMENT;
-  // ---- limits of the fixed scratch: one launch, counters for batch * n_kv heads, room for every partial
+  // ---- limits of the fixed scratch: one launch pair, room for every partial
   if (batch > AT_MAX_SEQS) return KVD_ERR_CAPACITY;
   if (static_cast<size_t>(batch) * n_kv_heads > 1024) return KVD_ERR_CAPACITY;
   const int kdim = n_kv_heads * d_head;
@@ -632,7 +651,6 @@ extern "C" kvd_status kvd_decode_attention_static(int n_q_heads, int n_kv_heads,
     S.lo_pos = lo;
     S.hi_pos = hi;
     S.part_base = parts;
-    S.group_base = 0;
     if (max_last < 0 || hi < lo) {
       S.n_chunks = 0;
       S.iters = 1;
@@ -645,54 +663,25 @@ extern "C" kvd_status kvd_decode_attention_static(int n_q_heads, int n_kv_heads,
     }
     parts += S.n_chunks;
   }
-  // first-level group partials live behind the chunk partials; one counter per (sequence, KV head)
-  // and one per (sequence, KV head, group)
-  int groups = 0, max_groups = 1;
-  for (int b = 0; b < batch; ++b) {
-    const int g = (L.seq[b].n_chunks + AT_MERGE_GROUP - 1) / AT_MERGE_GROUP;
-    L.seq[b].group_base = parts + groups;
-    groups += g;
-    if (g > max_groups) max_groups = g;
-  }
-  const size_t all_parts = static_cast<size_t>(parts) + groups;
-  const size_t counter_bytes =
-      (static_cast<size_t>(batch) * n_kv_heads * (1 + max_groups) * sizeof(int) + 255) / 256 * 256;
+  // one partial per chunk
+  const size_t all_parts = static_cast<size_t>(parts);
   const size_t ml_bytes = (all_parts * n_q_heads * 2 * sizeof(float) + 255) / 256 * 256;
   const size_t o_bytes = all_parts * n_q_heads * d_head * sizeof(float);
-  if (counter_bytes + ml_bytes + o_bytes > static_cast<size_t>(KVD_STATIC_SCRATCH_BYTES)) return KVD_ERR_CAPACITY;
+  if (ml_bytes + o_bytes > static_cast<size_t>(KVD_STATIC_SCRATCH_BYTES)) return KVD_ERR_CAPACITY;
 
   unsigned char *scratch = nullptr;
   kvd_status st = static_scratch_address(&scratch);  // first call on a device: symbol look-up
   if (st != KVD_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  // the arrival counters must start at zero whatever an earlier call left behind
-  if (cudaMemsetAsync(scratch, 0, counter_bytes, stream) != cudaSuccess) {
-    cudaGetLastError();
-    return KVD_ERR_CUDA;
-  }
   L.n_seqs = batch;
   L.total_chunks = parts;
   L.n_q = n_q_heads;
   L.n_kv = n_kv_heads;
-  L.seq0 = 0;
-  L.max_groups = max_groups;
-  L.cnt1_off = batch * n_kv_heads;
   L.scale_log2e = (scale > 0.f ? scale : 1.0f / sqrtf(static_cast<float>(d_head))) * 1.4426950408889634f;
   L.q = static_cast<const __nv_bfloat16 *>(q);
   L.out = static_cast<__nv_bfloat16 *>(out);
-  L.counters = reinterpret_cast<int *>(scratch);
-  L.part_ml = reinterpret_cast<float *>(scratch + counter_bytes);
-  L.part_o = reinterpret_cast<float *>(scratch + counter_bytes + ml_bytes);
-  for (int b = 0; b < batch; ++b) {
-    if (L.seq[b].n_chunks == 0) {  // no visible key: the output is all zeros
-      if (cudaMemsetAsync(L.out + static_cast<size_t>(b) * n_q_heads * d_head, 0,
-                          static_cast<size_t>(n_q_heads) * d_head * 2, stream) != cudaSuccess) {
-        cudaGetLastError();
-        return KVD_ERR_CUDA;
-      }
-    }
-  }
-  if (parts == 0) return KVD_OK;
+  L.part_ml = reinterpret_cast<float *>(scratch);
+  L.part_o = reinterpret_cast<float *>(scratch + ml_bytes);
   switch (d_head) {
     case 64: return static_launch_d<64>(L, group, stream);
     case 128: return static_launch_d<128>(L, group, stream);

@@ -64,10 +64,9 @@ struct RecomputeParams {
 };
 
 // ------------------------------------------------------------------------------ decode attention
-constexpr int AT_THREADS = 128;
-constexpr int AT_WARPS = 4;
+constexpr int AT_THREADS = 512;
+constexpr int AT_WARPS = 16;
 constexpr int AT_UNROLL = 8;          // keys per lane group per iteration
-constexpr int AT_MERGE_GROUP = 16;    // chunk partials merged per first-level group
 constexpr int AT_MAX_SEQS = 64;       // sequences per launch (bounded by the kernel parameter space)
 
 struct AttnSeq {
@@ -83,7 +82,6 @@ struct AttnSeq {
   int n_chunks;
   int part_base;    // index of this sequence's first partial in the scratch
   int iters;        // warp iterations per chunk
-  int group_base;   // index of this sequence's first group partial in the scratch
 };
 
 // Launch-wide fields, followed by the per-sequence descriptors.  The kernel takes the variant whose
@@ -94,15 +92,11 @@ struct AttnLaunchHead {
   int total_chunks;
   int n_q;
   int n_kv;
-  int seq0;                // index of the launch's first sequence in the batch (counter addressing)
-  int max_groups;          // stride of the per-group counters
-  int cnt1_off;            // offset (ints) of the per-group counters inside `counters`
   float scale_log2e;
   const __nv_bfloat16 *q;  // [n_seqs, n_q, d_head] (already offset to the launch's first sequence)
   __nv_bfloat16 *out;      // [n_seqs, n_q, d_head]
   float *part_o;           // [parts][n_q][d_head]
   float *part_ml;          // [parts][n_q][2]
-  int *counters;           // [max_batch][n_kv] then [max_batch][n_kv][max_groups], zero between calls
 };
 template <int NSEQ>
 struct AttnLaunchT : AttnLaunchHead {
@@ -112,21 +106,19 @@ typedef AttnLaunchT<AT_MAX_SEQS> AttnLaunch;
 
 // keys per chunk for a head size and iteration count
 inline int attn_keys_per_warp_iter(int d_head) { return (32 / (d_head / 8)) * AT_UNROLL; }
-// Iterations per chunk.  Short spans (<= 8192 keys) are cut into at most 64 chunks per (sequence, KV
-// head): there a CTA's prologue, combine and merge bookkeeping cost as much as streaming a few dozen
-// keys, so fat chunks win.  Longer spans are cut so that one sequence yields about 592 work units
-// (chunks x KV heads) -- four CTAs on each of a B200's 148 SMs -- which keeps every SM equally
-// loaded when the batch is 1.  A function of the model and of the visible span only, so a full
-// cache and a recomputed + window + current layout of the same positions are split identically,
-// and a sequence's result does not depend on what else is in the batch.
-inline int attn_target_chunks(int n_kv, int span) {
-  if (span <= 8192) return 64;
-  const int t = 592 / n_kv;
-  return t > 16 ? t : 16;
+// Iterations per chunk.  The visible span is cut so that one sequence yields about 148 work units
+// (chunks x KV heads) -- one 16-warp CTA on each of a B200's SMs -- which keeps every SM equally
+// loaded when the batch is 1 and leaves few enough partials per head for a single merge level.  A
+// function of the model and of the visible span only, so a full cache and a recomputed + window +
+// current layout of the same positions are split identically, and a sequence's result does not
+// depend on what else is in the batch.
+inline int attn_target_chunks(int n_kv) {
+  const int t = 148 / n_kv;
+  return t > 1 ? t : 1;
 }
 inline int attn_iters_for_span(int d_head, int n_kv, int span) {
   const int per_iter = attn_keys_per_warp_iter(d_head) * AT_WARPS;
-  const long long per_chunk_min = static_cast<long long>(per_iter) * attn_target_chunks(n_kv, span);
+  const long long per_chunk_min = static_cast<long long>(per_iter) * attn_target_chunks(n_kv);
   long long iters = (span + per_chunk_min - 1) / per_chunk_min;
   if (iters < 1) iters = 1;
   if (iters > 64) iters = 64;
@@ -136,8 +128,7 @@ inline int attn_chunk_keys(int d_head, int iters) { return attn_keys_per_warp_it
 inline int attn_max_chunks(int d_head, int n_kv, int max_tokens) {
   const int per_iter = attn_keys_per_warp_iter(d_head) * AT_WARPS;
   const int capped = max_tokens / (per_iter * 64) + 2;  // once the iteration count is capped
-  int target = attn_target_chunks(n_kv, max_tokens);
-  if (target < 64) target = 64;
+  const int target = attn_target_chunks(n_kv);
   return (capped > target ? capped : target) + 2;
 }
 
@@ -180,10 +171,8 @@ struct kvd_ctx {
   // attention scratch
   float *part_o = nullptr;
   float *part_ml = nullptr;
-  int *counters = nullptr;
   size_t workspace_bytes = 0;
   int max_parts = 0;
-  int max_groups = 0;
   int *d_status = nullptr;
   uint64_t launches = 0;
   uint64_t prepared_bytes = 0;

@@ -86,7 +86,7 @@ def test_static_scratch_matches_workspace_path_on_two_calls_in_a_row():
     K, V = make_kv(shape, T, seed=80)
     k, v = dev(K), dev(V)
     kdim = shape.n_kv_heads * shape.d_head
-    big = 16
+    big = 64
     qb = dev(make_query(shape, big, seed=43))
     out = torch.full((big, shape.n_q_heads, shape.d_head), 5.0, dtype=torch.bfloat16, device="cuda")
     st = kvd.kvd_decode_attention_static(shape.n_q_heads, shape.n_kv_heads, shape.d_head, 0, big, qb, [T - 1] * big,
