@@ -15,6 +15,7 @@
 // merge runs in chunk order, so the output bits do not depend on how the keys are spread over
 // segments.
 #include <math_constants.h>
+#include <string.h>
 
 #include "kvd_internal.h"
 #include "kvd_ptx.cuh"
@@ -92,6 +93,10 @@ __global__ void __launch_bounds__(AT_THREADS, 1) kvd_attn_split_kernel(const __g
   constexpr int KPL = 32 / LPK;           // keys per warp-wide load
   constexpr int U = AT_UNROLL;            // keys per lane group per iteration
   constexpr int NPART = AT_WARPS * KPL;   // lane groups per CTA
+  // The merge kernel is launched as a programmatic dependent of this one: once every CTA of this
+  // grid has started, its CTAs may take SMs that become free and wait there (griddepcontrol.wait)
+  // for this grid to complete, so its launch latency is off the critical path.
+  grid_launch_dependents();
   // per lane group: unnormalised output, maximum, sum (AttnSmem<D_HEAD, G>::BYTES of dynamic shared memory)
   extern __shared__ __align__(16) float at_smem[];
   float (*s_o)[G][D_HEAD] = reinterpret_cast<float (*)[G][D_HEAD]>(at_smem);
@@ -120,6 +125,8 @@ __global__ void __launch_bounds__(AT_THREADS, 1) kvd_attn_split_kernel(const __g
   const int chunk_keys = KPL * U * AT_WARPS * S.iters;
   const int chunk_pos0 = S.chunk0_pos + chunk * chunk_keys;
 
+  // everything above used kernel parameters only; K, V and q may come from the preceding kernel
+  grid_dependency_wait();
   // ---- query of every head of the group, pre-multiplied by scale * log2(e)
   uint64_t qf[G][4];  // channel pairs (2j, 2j+1)
 #pragma unroll
@@ -344,6 +351,10 @@ __global__ void __launch_bounds__(AT_THREADS, 1) kvd_attn_merge_kernel(const __g
   const int si = blockIdx.x / P.n_kv, kvh = blockIdx.x % P.n_kv;
   const AttnSeq &S = P.seq[si];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // wait until the preceding grid in the stream (the streaming kernel) has completed and its
+  // partials are visible
+  grid_launch_dependents();
+  grid_dependency_wait();
 
   // Every warp finds the maximum of each head by itself (lanes over partials, shuffles -- no block
   // barrier), then sums a contiguous sixteenth of the partials scaled to it, each lane owning CPL
@@ -468,15 +479,24 @@ template <int D_HEAD, int G, int NSEQ>
 static cudaError_t attn_launch_pair(const AttnLaunchT<NSEQ> &S, cudaStream_t stream) {
   cudaError_t e = attn_configure<D_HEAD, G, NSEQ>();
   if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.blockDim = dim3(AT_THREADS, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   if (S.total_chunks > 0) {
-    kvd_attn_split_kernel<D_HEAD, G, NSEQ>
-        <<<S.total_chunks * S.n_kv, AT_THREADS, AttnSmem<D_HEAD, G>::BYTES, stream>>>(S);
-    e = cudaGetLastError();
+    cfg.gridDim = dim3(S.total_chunks * S.n_kv, 1, 1);
+    cfg.dynamicSmemBytes = AttnSmem<D_HEAD, G>::BYTES;
+    e = cudaLaunchKernelEx(&cfg, kvd_attn_split_kernel<D_HEAD, G, NSEQ>, S);
     if (e != cudaSuccess) return e;
   }
-  kvd_attn_merge_kernel<D_HEAD, G, NSEQ>
-      <<<S.n_seqs * S.n_kv, AT_THREADS, AttnSmem<D_HEAD, G>::MERGE_BYTES, stream>>>(S);
-  return cudaGetLastError();
+  cfg.gridDim = dim3(S.n_seqs * S.n_kv, 1, 1);
+  cfg.dynamicSmemBytes = AttnSmem<D_HEAD, G>::MERGE_BYTES;
+  return cudaLaunchKernelEx(&cfg, kvd_attn_merge_kernel<D_HEAD, G, NSEQ>, S);
 }
 
 template <int D_HEAD, int G, int NSEQ>

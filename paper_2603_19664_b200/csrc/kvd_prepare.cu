@@ -39,6 +39,7 @@ __global__ void __launch_bounds__(256) kvd_checkpoint_kernel(const uint4 *__rest
                                                              long long n_vec, int n) {
   const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
   const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  grid_launch_dependents();  // the next kernel's set-up may overlap this copy
   for (long long i = tid; i < n_vec; i += stride) dst_rows[i] = rows[i];
   for (long long i = tid; i < n; i += stride) dst_pos[i] = pos[i];
 }

@@ -99,6 +99,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const void *tmap,
       : "memory");
 }
 
+// ------------------------------------------------------------------------------ dependent launch
+// A kernel launched with programmatic stream serialisation may start while its predecessor in the
+// stream is still running: everything up to grid_dependency_wait() (set-up that touches no global
+// memory the predecessor writes) overlaps with the predecessor's tail.  grid_launch_dependents()
+// lets the successor do the same with this kernel.  Both are no-ops for ordinary launches.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+
 // ------------------------------------------------------------------------------ tcgen05 / TMEM
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_result, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(ncols)

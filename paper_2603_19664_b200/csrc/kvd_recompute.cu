@@ -209,6 +209,10 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   cluster_sync_all();  // barriers of both CTAs are initialised before anyone signals across the pair
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
+  // The set-up above read only kernel parameters and tables written at kvd_set_layer time, so it may
+  // overlap the tail of the preceding kernel; rows, positions and outputs are touched from here on.
+  grid_launch_dependents();
+  grid_dependency_wait();
   if (threadIdx.x == 0) trace_put<TRACE>(p.trace, 0, 11);
 
   if (warp == 2) {
@@ -627,13 +631,15 @@ static kvd_status launch_impl(kvd_ctx *ctx, const LayerState &ls, const CUtensor
   cfg.blockDim = dim3(RC_THREADS, 1, 1);
   cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   cudaError_t le = cudaLaunchKernelEx(&cfg, kern, tmap_store, tmap_rows, ls.tmap_b, p);
   if (le != cudaSuccess) return cuda_fail(ctx, le, "launch recompute");
   ctx->launches += 1;
