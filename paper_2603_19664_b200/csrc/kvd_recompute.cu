@@ -38,7 +38,7 @@ namespace kvd {
 
 template <int BLOCK_N, int D_HEAD>
 struct RcCfg {
-  static constexpr int STAGES = BLOCK_N == 256 ? 6 : 8;
+  static constexpr int STAGES = BLOCK_N == 256 ? 7 : 9;  // all the shared memory an SM has: the ring is latency-bound
   static constexpr int A_BYTES = RC_BLOCK_M * RC_BLOCK_K * 2;
   static constexpr int B_ROWS = BLOCK_N / 2;  // this CTA's half of the W' tile
   static constexpr int B_BYTES = B_ROWS * RC_BLOCK_K * 2;
@@ -46,10 +46,9 @@ struct RcCfg {
   static constexpr int TMEM_COLS = 2 * BLOCK_N;
   // barriers: full[S], empty[S], peer_full[S], tmem_full[2], tmem_empty[2], stats_full[2], rstd_free[2]
   static constexpr int NUM_BARS = 3 * STAGES + 8;
-  static constexpr int ROPE_LO_BYTES = (D_HEAD / 2) * ROPE_LO_SIZE * 8;  // [pair][position low bits] (cos, sin)
-  static constexpr int TAIL_BYTES =
-      NUM_BARS * 8 + 16 /*tmem ptr, abort*/ + 2 * RC_BLOCK_M * 4 /*rstd*/ + 256 * 4 /*gamma_k*/ + ROPE_LO_BYTES;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + TAIL_BYTES + 1024 /*alignment slack*/;
+  static constexpr int TAIL_BYTES = NUM_BARS * 8 + 16 /*tmem ptr, abort*/ + 2 * RC_BLOCK_M * 4 /*rstd*/ + 256 * 4 /*gamma_k*/;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + TAIL_BYTES;  // the base must be 1024-byte aligned
+  static_assert(SMEM_BYTES <= 232448, "more shared memory than an SM offers");
 };
 
 // Optional per-tile timeline (SM clock cycles) for performance analysis; see kvd_set_trace.
@@ -124,15 +123,18 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   constexpr int STAGES = Cfg::STAGES;
   static_assert(BLOCK_N % D_HEAD == 0, "a tile must hold whole heads");
 
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  extern __shared__ __align__(1024) uint8_t smem[];
+  // the 128-byte swizzle pattern is anchored at 1024-byte boundaries; there is no slack to realign
+  if ((smem_u32(smem) & 1023u) != 0u) {
+    if (threadIdx.x == 0) atomicOr(p.status, STATUS_TIMEOUT);
+    return;
+  }
   uint8_t *tail = smem + STAGES * Cfg::STAGE_BYTES;
   uint64_t *bars = reinterpret_cast<uint64_t *>(tail);
   uint32_t *s_tmem = reinterpret_cast<uint32_t *>(tail + Cfg::NUM_BARS * 8);
   volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
   float *s_rstd = reinterpret_cast<float *>(tail + Cfg::NUM_BARS * 8 + 16);
   float *s_gamma_k = s_rstd + 2 * RC_BLOCK_M;
-  float2 *s_rope_lo = reinterpret_cast<float2 *>(s_gamma_k + 256);
 
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_base = smem_u32(bars);
@@ -199,8 +201,6 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
     prefetch_tensormap(&tmap_b);
   }
   if (threadIdx.x < D_HEAD) s_gamma_k[threadIdx.x] = p.gamma_k ? p.gamma_k[threadIdx.x] : 1.0f;
-  for (int i = threadIdx.x; i < Cfg::ROPE_LO_BYTES / 16; i += RC_THREADS)
-    reinterpret_cast<float4 *>(s_rope_lo)[i] = reinterpret_cast<const float4 *>(p.rope_lo)[i];
   if (warp == 3) {
     tmem_alloc_pair(smem_u32(s_tmem), Cfg::TMEM_COLS);
     tmem_relinquish_pair();
@@ -457,10 +457,11 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
         atomicOr(p.status, STATUS_POSITION);
         pos = pos < 0 ? 0 : p.max_pos - 1;
       }
-      // (cos, sin) of pos * f_i = angle sum of the entries for (pos & ~15) [global, shared by 16
-      // neighbouring positions] and (pos & 15) [shared memory, laid out [pair][low bits]]
+      // (cos, sin) of pos * f_i = angle sum of the entries for (pos & ~15) [shared by 16 neighbouring
+      // positions] and (pos & 15) [laid out [pair][low bits]: the 32 rows of a warp read one 128-byte
+      // line per pair, which stays in L1]
       const float4 *t_hi = reinterpret_cast<const float4 *>(p.rope_hi + static_cast<size_t>(pos >> ROPE_LO_BITS) * HALF);
-      const float2 *t_lo = s_rope_lo + (pos & (ROPE_LO_SIZE - 1));
+      const float2 *t_lo = p.rope_lo + (pos & (ROPE_LO_SIZE - 1));
       const uint32_t acc = tmem_base + lane_field + a * BLOCK_N;
 
 #pragma unroll 1
@@ -524,7 +525,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
 #pragma unroll
               for (int j = 0; j < 8; j += 2) {
                 const int i = c * 8 + j;  // pairs i and i + 1
-                const float2 l0 = t_lo[i * ROPE_LO_SIZE], l1 = t_lo[(i + 1) * ROPE_LO_SIZE];
+                const float2 l0 = __ldg(t_lo + i * ROPE_LO_SIZE), l1 = __ldg(t_lo + (i + 1) * ROPE_LO_SIZE);
                 const float4 hh4 = h[j >> 1];
                 const float c0 = fmaf(hh4.x, l0.x, -hh4.y * l0.y), s0 = fmaf(hh4.y, l0.x, hh4.x * l0.y);
                 const float c1 = fmaf(hh4.z, l1.x, -hh4.w * l1.y), s1 = fmaf(hh4.w, l1.x, hh4.z * l1.y);
@@ -562,7 +563,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
 #pragma unroll
               for (int j = 0; j < 16; j += 2) {
                 const int i = c * 16 + j;  // pairs (i, i + HALF) and (i + 1, i + 1 + HALF)
-                const float2 l0 = t_lo[i * ROPE_LO_SIZE], l1 = t_lo[(i + 1) * ROPE_LO_SIZE];
+                const float2 l0 = __ldg(t_lo + i * ROPE_LO_SIZE), l1 = __ldg(t_lo + (i + 1) * ROPE_LO_SIZE);
                 const float4 hh4 = h[j >> 1];
                 const float c0 = fmaf(hh4.x, l0.x, -hh4.y * l0.y), s0 = fmaf(hh4.y, l0.x, hh4.x * l0.y);
                 const float c1 = fmaf(hh4.z, l1.x, -hh4.w * l1.y), s1 = fmaf(hh4.w, l1.x, hh4.z * l1.y);
