@@ -639,7 +639,8 @@ def run_stack_configs(args):
     """Hot-path timing of the stack-shaped configurations: the 34-layer Gemma-3-4B-shaped stack
     (context 2048, 256 live K/V, batch 1..64: KV-Direct decode step against a full-cache step) and the
     Qwen3-4B-shaped long-context case (36 layers, context 32768, batch 8, 512 live K/V).  Only the
-    library's kernels are timed; one layer of each kind is measured and multiplied by the layer count."""
+    library's kernels are timed (CUDA graphs of the launch sequence, stored K/V rotating over sets that
+    exceed the L2); one layer of each kind is measured and multiplied by the layer count."""
     import torch
     import paper_2603_19664_b200 as kvd
     from kvd_synth import GEMMA3_4B_GLOBAL, GEMMA3_4B_LOCAL, QWEN3_4B, make_layer_weights
@@ -651,39 +652,57 @@ def run_stack_configs(args):
     def dev(bits):
         return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
 
-    def timed(fn, reps=5):
-        for _ in range(2):
-            fn()
+    side = torch.cuda.Stream()
+
+    def timed_graph(fn, n_sets, reps=5):
+        """us per call of fn(i), i rotating over n_sets input sets, replayed from a CUDA graph."""
+        for i in range(n_sets):
+            fn(i)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for i in range(n_sets):
+                fn(i)
+        g.replay()
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         for _ in range(reps):
-            fn()
+            g.replay()
         b.record()
         torch.cuda.synchronize()
-        return a.elapsed_time(b) / reps * 1e3  # us
+        return a.elapsed_time(b) / (reps * n_sets) * 1e3
 
     def layer_case(shape, ctx_len, budget, batch):
-        """(kvdirect_us, fullcache_us, detail) for one layer: decode step of `batch` sequences at position ctx_len."""
+        """One layer, decode step of `batch` sequences at position ctx_len.  KV-Direct: recompute the
+        evicted rows of every sequence from the residual store together with K_t, V_t of the new tokens
+        (one launch), then attention over recomputed + window + current segments.  Full cache: K_t, V_t,
+        then attention over the stored K/V.  Stored K/V rotate over enough sets to exceed the L2."""
         kdim = shape.n_kv_heads * shape.d_head
         lo = 0 if shape.sliding_window == 0 else max(0, ctx_len - shape.sliding_window + 1)
         n_old = max(0, ctx_len - budget - lo)  # evicted positions [lo, ctx_len - budget) this layer attends to
         w = make_layer_weights(shape)
         desc = kvd.make_desc(1, shape.d_hidden, shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.rms_eps,
-                             shape.qk_norm, shape.rms_eps, shape.rope_style, 1, ctx_len + 8, batch)
+                             shape.qk_norm, shape.rms_eps, shape.rope_style, batch, ctx_len + 8, batch)
         c = kvd.Kvd(desc)
         tw, tg = dev(w.w_kv), dev(w.gamma_in)
         tk = dev(w.gamma_k) if w.gamma_k is not None else None
         c.kvd_set_layer(0, tw, tg, tk, shape.rope_theta, shape.sliding_window)
         ws = torch.empty(kvd.kvd_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
         c.kvd_attach_workspace(ws)
+        arena = torch.empty(kvd.kvd_store_bytes(desc, 1), dtype=torch.uint8, device="cuda")
+        c.kvd_attach_store(arena, 1)
+        xs = torch.randn((ctx_len, shape.d_hidden), device="cuda").to(torch.bfloat16)
+        ps = torch.arange(ctx_len, device="cuda", dtype=torch.int32)
+        for b in range(batch):
+            c.kvd_checkpoint_residual(b, 0, xs, ps, ctx_len)  # STORE_RESIDUAL of the whole context
         M = batch * n_old
-        X = torch.randn((max(M, 1), shape.d_hidden), device="cuda").to(torch.bfloat16)
-        pos = (torch.arange(max(M, 1), device="cuda", dtype=torch.int32) % max(n_old, 1)) + lo
         Ko = torch.empty((max(M, 1), kdim), device="cuda", dtype=torch.bfloat16)
         Vo = torch.empty_like(Ko)
-        Kf = torch.randn((batch, ctx_len + 1, kdim), device="cuda").to(torch.bfloat16)  # stored cache / window / current
-        Vf = torch.randn((batch, ctx_len + 1, kdim), device="cuda").to(torch.bfloat16)
+        set_bytes = 2 * batch * (ctx_len + 1) * kdim * 2
+        n_sets = max(2, min(24, -(-300_000_000 // set_bytes)))
+        Kf = [torch.randn((batch, ctx_len + 1, kdim), device="cuda").to(torch.bfloat16) for _ in range(n_sets)]
+        Vf = [torch.randn((batch, ctx_len + 1, kdim), device="cuda").to(torch.bfloat16) for _ in range(n_sets)]
         xc = torch.randn((batch, shape.d_hidden), device="cuda").to(torch.bfloat16)
         pc = torch.full((batch,), ctx_len, device="cuda", dtype=torch.int32)
         kc = torch.empty((batch, kdim), device="cuda", dtype=torch.bfloat16)
@@ -691,39 +710,67 @@ def run_stack_configs(args):
         q = torch.randn((batch, shape.n_q_heads, shape.d_head), device="cuda").to(torch.bfloat16)
         out = torch.empty_like(q)
         wf = ctx_len - budget
-        segs_kvd = [[(Ko[b * n_old:], Vo[b * n_old:], kdim, lo, n_old), (Kf[b, wf:], Vf[b, wf:], kdim, wf, budget),
-                     (kc[b:], vc[b:], kdim, ctx_len, 1)] for b in range(batch)]
-        first_full = lo
-        segs_full = [[(Kf[b, first_full:], Vf[b, first_full:], kdim, first_full, ctx_len + 1 - first_full)]
-                     for b in range(batch)]
+        ranges = [(b, lo, n_old, Ko[b * n_old:], Vo[b * n_old:]) for b in range(batch)] if n_old > 0 else []
+        segs_kvd = [[[(Ko[b * n_old:], Vo[b * n_old:], kdim, lo, n_old), (Kf[s][b, wf:], Vf[s][b, wf:], kdim, wf, budget),
+                      (kc[b:], vc[b:], kdim, ctx_len, 1)] for b in range(batch)] for s in range(n_sets)]
+        segs_full = [[[(Kf[s][b, lo:], Vf[s][b, lo:], kdim, lo, ctx_len + 1 - lo)] for b in range(batch)]
+                     for s in range(n_sets)]
         qpos = [ctx_len] * batch
-        t_rec = timed(lambda: c.kvd_recompute_kv(0, X, pos, M, Ko, Vo, kdim)) if M > 0 else 0.0
-        t_cur = timed(lambda: c.kvd_recompute_kv(0, xc, pc, batch, kc, vc, kdim))
-        t_att = timed(lambda: c.kvd_decode_attention(0, batch, q, qpos, segs_kvd, 0.0, out))
-        t_full = timed(lambda: c.kvd_decode_attention(0, batch, q, qpos, segs_full, 0.0, out))
+
+        def rec(i):
+            c.kvd_recompute_kv_step(0, ranges, xc, pc, batch, kc, vc, kdim)
+
+        def cur(i):
+            c.kvd_recompute_kv(0, xc, pc, batch, kc, vc, kdim)
+
+        def att(i):
+            c.kvd_decode_attention(0, batch, q, qpos, segs_kvd[i % n_sets], 0.0, out)
+
+        def att_full(i):
+            c.kvd_decode_attention(0, batch, q, qpos, segs_full[i % n_sets], 0.0, out)
+
+        def layer_kvd(i):
+            rec(i)
+            att(i)
+
+        def layer_full(i):
+            cur(i)
+            att_full(i)
+
+        # memory-bound cases first, each after a short pause: a long run of GEMMs at the power cap
+        # leaves the clocks low for whatever is measured next
+        def rested(fn):
+            torch.cuda.synchronize()
+            time.sleep(0.3)
+            return timed_graph(fn, n_sets)
+        rec(0)  # the K/V that the KV-Direct attention reads
+        t_cur, t_att, t_full = rested(cur), rested(att), rested(att_full)
+        t_layer_full = rested(layer_full)
+        t_rec, t_layer_kvd = rested(rec), rested(layer_kvd)
         assert c.kvd_poll_status() == kvd.KVD_OK
-        flops = 4.0 * M * shape.n_kv_heads * shape.d_hidden * shape.d_head
+        flops = 4.0 * (M + batch) * shape.n_kv_heads * shape.d_hidden * shape.d_head
         keys = batch * (ctx_len + 1 - lo)
         byts = keys * 4 * shape.n_kv_heads * shape.d_head
         c.close()
-        return {"rows_recomputed": M, "recompute_us": t_rec, "recompute_tflops": flops / t_rec / 1e6 if M else None,
-                "current_kv_us": t_cur, "attention_us": t_att, "attention_gbs": byts / t_att / 1e3,
-                "fullcache_attention_us": t_full, "fullcache_attention_gbs": byts / t_full / 1e3}
+        return {"rows_recomputed": M, "kv_buffer_sets": n_sets,
+                "recompute_with_current_us": t_rec, "recompute_tflops": flops / t_rec / 1e6,
+                "current_kv_only_us": t_cur, "attention_us": t_att, "attention_gbs": byts / t_att / 1e3,
+                "fullcache_attention_us": t_full, "fullcache_attention_gbs": byts / t_full / 1e3,
+                "kvdirect_layer_us": t_layer_kvd, "fullcache_layer_us": t_layer_full}
 
     result = {"peaks": peaks, "gemma3_4b_stack_ctx2048_window256": [], "qwen3_4b_ctx32768_batch8_window512": None}
     for batch in (1, 4, 16, 64):
         g = layer_case(GEMMA3_4B_GLOBAL, 2048, 256, batch)
         l = layer_case(GEMMA3_4B_LOCAL, 2048, 256, batch)
-        kvd_step = 5 * (g["recompute_us"] + g["current_kv_us"] + g["attention_us"]) + \
-            29 * (l["recompute_us"] + l["current_kv_us"] + l["attention_us"])
-        full_step = 5 * (g["current_kv_us"] + g["fullcache_attention_us"]) + \
-            29 * (l["current_kv_us"] + l["fullcache_attention_us"])
+        kvd_step = 5 * g["kvdirect_layer_us"] + 29 * l["kvdirect_layer_us"]
+        full_step = 5 * g["fullcache_layer_us"] + 29 * l["fullcache_layer_us"]
         result["gemma3_4b_stack_ctx2048_window256"].append(
             {"batch": batch, "kvdirect_decode_step_us": kvd_step, "fullcache_decode_step_us": full_step,
              "ratio": kvd_step / full_step, "recomputed_tokens_per_s": batch * (5 * g["rows_recomputed"] // batch +
              29 * l["rows_recomputed"] // batch) / (kvd_step * 1e-6), "global_layer": g, "local_layer": l})
     qw = layer_case(QWEN3_4B, 32768, 512, 8)
-    qw["step_us_36_layers"] = 36 * (qw["recompute_us"] + qw["current_kv_us"] + qw["attention_us"])
+    qw["step_us_36_layers"] = 36 * qw["kvdirect_layer_us"]
+    qw["fullcache_step_us_36_layers"] = 36 * qw["fullcache_layer_us"]
     qw["recompute_frac_of_sustained_peak"] = qw["recompute_tflops"] / peaks["bf16_tflops_sustained"]
     qw["recompute_frac_of_burst_peak"] = qw["recompute_tflops"] / peaks["bf16_tflops"]
     qw["attention_frac_of_hbm_peak"] = qw["attention_gbs"] / peaks["hbm_gbs"]

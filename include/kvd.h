@@ -12,6 +12,8 @@
  *                            row's stored position (Eq. 11-12).  The same call produces the current
  *                            token's (K_t, V_t), so "first pass" and "recomputed" K/V are the output
  *                            of one routine and are bit-identical for the same row and position.
+ *   kvd_recompute_kv_step    the K/V work of one decode step of a layer in one launch: RECOMPUTE_KV
+ *                            for the evicted ranges of every sequence plus (K_t, V_t) of the new tokens.
  *   kvd_decode_attention     ATTENTION(Q, K_all, V_all) for one query token per sequence (Eq. 6-7)
  *                            over the CONCAT of up to four position-contiguous K/V segments
  *                            (recomputed, live window, current token), grouped-query heads,
@@ -209,7 +211,7 @@ kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, const void *
  * cannot allocate device memory at all -- code running inside someone else's memory pool or under a
  * fixed memory budget, a plug-in whose host forbids cudaMalloc after start-up, a process that must
  * not disturb an allocator's bookkeeping.  It needs no context and no workspace: the split partials
- * and the arrival counters live in a fixed array of KVD_STATIC_SCRATCH_BYTES compiled into the
+ * live in a fixed array of KVD_STATIC_SCRATCH_BYTES compiled into the
  * library, which every GPU that loads the library holds until the process exits.
  *   - Shapes are passed directly (d_head in {64, 128, 256}, group size n_q_heads / n_kv_heads in
  *     {1, 2, 3, 4, 8}); q, q_pos, segs, scale, out and the visibility rule are those of
@@ -221,9 +223,9 @@ kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, const void *
  *   - It calls no cudaMalloc / cudaFree and no library routine that allocates.  The first call on a
  *     device looks up the array's device address (cudaGetSymbolAddress) with that device current;
  *     make that first call outside any stream capture.
- *   - All calls share the array and it keeps the previous call's contents; the counters are cleared
- *     on `stream` at the start of every call.  Calls whose kernels can overlap on one GPU (different
- *     streams, different host threads) race on the array: serialise them on one stream. */
+ *   - All calls share the array and it keeps the previous call's contents; every call overwrites
+ *     the part it reads, so nothing has to be cleared.  Calls whose kernels can overlap on one GPU
+ *     (different streams, different host threads) race on the array: serialise them on one stream. */
 #define KVD_STATIC_SCRATCH_BYTES (8u << 20)
 kvd_status kvd_decode_attention_static(int n_q_heads, int n_kv_heads, int d_head, int sliding_window, int batch,
                                        const void *q, const int32_t *q_pos, const kvd_kv_segment *segs, int n_segs,

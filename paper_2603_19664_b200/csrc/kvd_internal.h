@@ -5,6 +5,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
 
 #include <map>
 #include <string>
@@ -184,6 +185,17 @@ struct kvd_ctx {
 };
 
 namespace kvd {
+// Kernels are launched as programmatic dependents of their predecessor in the stream unless the
+// environment variable KVD_SERIAL_LAUNCH says otherwise: a bit mask, 1 = recompute kernel, 2 = attention
+// streaming kernel, 4 = attention merge kernel get plain stream ordering instead.
+inline int serial_launch_mask() {
+  static const int mask = [] {
+    const char *e = getenv("KVD_SERIAL_LAUNCH");
+    return e ? atoi(e) : 0;
+  }();
+  return mask;
+}
+
 // launchers implemented next to their kernels
 kvd_status launch_recompute(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
                             const CUtensorMap &tmap_rows, const RecomputeParams &p, cudaStream_t stream);

@@ -638,7 +638,7 @@ static kvd_status launch_impl(kvd_ctx *ctx, const LayerState &ls, const CUtensor
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].val.programmaticStreamSerializationAllowed = (serial_launch_mask() & 1) ? 0 : 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   cudaError_t le = cudaLaunchKernelEx(&cfg, kern, tmap_store, tmap_rows, ls.tmap_b, p);

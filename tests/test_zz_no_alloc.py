@@ -2,8 +2,8 @@
 
 Some users of this library run where cudaMalloc is off limits -- inside another framework's memory
 pool, under a fixed device-memory budget, or in a plug-in whose host forbids allocation after
-start-up.  For them the library offers one entry point whose scratch (split partials and arrival
-counters) is a fixed array compiled into the library instead of a caller-provided workspace.
+start-up.  For them the library offers one entry point whose scratch (the split partials) is a
+fixed array compiled into the library instead of a caller-provided workspace.
 
 This file is collected last on purpose: a run that stops at the first failure has then already run
 every other test.  The test calls the entry point through the C ABI twice in a row with different
