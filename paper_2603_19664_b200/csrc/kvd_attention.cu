@@ -88,7 +88,7 @@ __device__ __forceinline__ float reduce8_transposed(const float (&v)[8], int lig
 }
 
 template <int D_HEAD, int G, int NSEQ>
-__global__ void __launch_bounds__(AT_THREADS, 1) kvd_attn_split_kernel(const __grid_constant__ AttnLaunchT<NSEQ> P) {
+__global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM) kvd_attn_split_kernel(const __grid_constant__ AttnLaunchT<NSEQ> P) {
   constexpr int LPK = D_HEAD / 8;         // lanes per key
   constexpr int KPL = 32 / LPK;           // keys per warp-wide load
   constexpr int U = AT_UNROLL;            // keys per lane group per iteration
@@ -338,115 +338,117 @@ __global__ void __launch_bounds__(AT_THREADS, 1) kvd_attn_split_kernel(const __g
   }
 }
 
-// Second kernel of a decode step: one CTA per (sequence, KV head) merges that head group's chunk
-// partials in chunk order and writes the output.  A separate launch instead of a "last CTA merges"
-// tail: every dependent global-memory hop (partial -> fence -> counter -> merge) measured above a
-// microsecond, which the streaming CTAs would spend idle on their SM; the kernel boundary costs about
-// as much once per step and needs no counters.  A sequence without a visible key gets zeros.
+// Second kernel of a decode step: the chunk partials of every (sequence, KV head) are merged in chunk
+// order and the output written.  A separate launch instead of a "last CTA merges" tail: every
+// dependent global-memory hop (partial -> fence -> counter -> merge) measured above a microsecond,
+// which the streaming CTAs would spend idle on their SM; the kernel boundary costs about as much
+// once per step and needs no counters.  A sequence without a visible key gets zeros.
+//
+// One CTA per (sequence, KV head, slice of 64 channels).  Warp w merges the w-th group of consecutive
+// partials of its head group, each lane owning two channels of every head: a partial costs a lane 4*G
+// registers, a group is as many partials as fit 64 registers (attn_merge_group(G)), all fetched at
+// once, so a warp's work is one round trip to the L2; the warp results are added in warp order.  The
+// launch has as many warps per CTA as its longest sequence has groups (at most 16; beyond that a warp
+// takes several groups, 16 apart); a shorter sequence leaves the extra warps idle, so its summation
+// order depends on its own chunk count only.
 template <int D_HEAD, int G, int NSEQ>
-__global__ void __launch_bounds__(AT_THREADS, 1) kvd_attn_merge_kernel(const __grid_constant__ AttnLaunchT<NSEQ> P) {
-  extern __shared__ __align__(16) float at_smem[];
-  float (*s_o)[G][D_HEAD] = reinterpret_cast<float (*)[G][D_HEAD]>(at_smem);  // [AT_WARPS]
-  float (*s_l)[G] = reinterpret_cast<float (*)[G]>(at_smem + AT_WARPS * G * D_HEAD);
-  const int si = blockIdx.x / P.n_kv, kvh = blockIdx.x % P.n_kv;
+__global__ void __launch_bounds__(AT_MERGE_THREADS)
+    kvd_attn_merge_kernel(const __grid_constant__ AttnLaunchT<NSEQ> P) {
+  constexpr int SLICES = D_HEAD / AT_MERGE_SLICE;
+  constexpr int PF = attn_merge_group(G);
+  __shared__ float s_o[AT_MERGE_WARPS][G][AT_MERGE_SLICE];
+  __shared__ float s_l[AT_MERGE_WARPS][G];
+  const int slice = blockIdx.x % SLICES;
+  const int head_slot = blockIdx.x / SLICES;
+  const int si = head_slot / P.n_kv, kvh = head_slot % P.n_kv;
   const AttnSeq &S = P.seq[si];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  grid_launch_dependents();
   // wait until the preceding grid in the stream (the streaming kernel) has completed and its
   // partials are visible
-  grid_launch_dependents();
   grid_dependency_wait();
 
-  // Every warp finds the maximum of each head by itself (lanes over partials, shuffles -- no block
-  // barrier), then sums a contiguous sixteenth of the partials scaled to it, each lane owning CPL
-  // channels of every head; the warp results are added in warp order.  All loads of a warp's first
-  // PF partials are issued before the maxima are known, so the merge costs about one round trip to
-  // the L2.
-  constexpr int CPL = D_HEAD / 32;  // channels per lane
-  // partials fetched ahead (bounded by the registers they take)
-  constexpr int PF = 64 / (G * CPL) >= 4 ? 4 : (64 / (G * CPL) >= 1 ? 64 / (G * CPL) : 1);
   const int count = S.n_chunks;
+  const int n_groups = (count + PF - 1) / PF;
+  const int warps_used = n_groups < AT_MERGE_WARPS ? n_groups : AT_MERGE_WARPS;
   const float *ml0 = P.part_ml + (static_cast<size_t>(S.part_base) * P.n_q + kvh * G) * 2;
-  const float *po0 = P.part_o + (static_cast<size_t>(S.part_base) * P.n_q + kvh * G) * D_HEAD;
+  const float *po0 = P.part_o + (static_cast<size_t>(S.part_base) * P.n_q + kvh * G) * D_HEAD +
+                     slice * AT_MERGE_SLICE + lane * 2;
   const size_t ml_stride = static_cast<size_t>(P.n_q) * 2, po_stride = static_cast<size_t>(P.n_q) * D_HEAD;
-  const int per_warp = (count + AT_WARPS - 1) / AT_WARPS;
-  const int c_begin = warp * per_warp;
-  const int c_end = c_begin + per_warp < count ? c_begin + per_warp : count;
-  float vbuf[PF][G][CPL];
-  float2 mlbuf[PF][G];
-  auto fetch = [&](int ch, float (&d)[G][CPL], float2 (&dm)[G]) {
+  if (warp < warps_used) {
+    float2 vbuf[PF][G], mlbuf[PF][G];
+    auto fetch_group = [&](int grp) {
+#pragma unroll
+      for (int i = 0; i < PF; ++i) {
+        const int ch = grp * PF + i;
+        if (ch < count) {
+#pragma unroll
+          for (int g = 0; g < G; ++g) {
+            mlbuf[i][g] = __ldcg(reinterpret_cast<const float2 *>(ml0 + ch * ml_stride + g * 2));
+            vbuf[i][g] = __ldcg(reinterpret_cast<const float2 *>(po0 + ch * po_stride + g * D_HEAD));
+          }
+        }
+      }
+    };
+    fetch_group(warp);
+    // the maximum of each head over all partials: lanes over partials (the first 256 loaded before
+    // any is used), then shuffles -- every warp by itself, no block barrier
+    float Mu[G];
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      dm[g] = __ldcg(reinterpret_cast<const float2 *>(ml0 + ch * ml_stride + g * 2));
-      const float *src = po0 + ch * po_stride + g * D_HEAD + lane * CPL;
-      if constexpr (CPL == 2) {
-        const float2 v = __ldcg(reinterpret_cast<const float2 *>(src));
-        d[g][0] = v.x;
-        d[g][1] = v.y;
-      } else {
+      float mv[8];
 #pragma unroll
-        for (int e = 0; e < CPL; e += 4) {
-          const float4 v = __ldcg(reinterpret_cast<const float4 *>(src + e));
-          d[g][e] = v.x;
-          d[g][e + 1] = v.y;
-          d[g][e + 2] = v.z;
-          d[g][e + 3] = v.w;
+      for (int i = 0; i < 8; ++i) {
+        const int ch = lane + 32 * i;
+        mv[i] = ch < count ? __ldcg(ml0 + ch * ml_stride + g * 2) : -CUDART_INF_F;
+      }
+      float mx = fmaxf(fmaxf(fmaxf(mv[0], mv[1]), fmaxf(mv[2], mv[3])), fmaxf(fmaxf(mv[4], mv[5]), fmaxf(mv[6], mv[7])));
+      for (int ch = lane + 256; ch < count; ch += 32) mx = fmaxf(mx, __ldcg(ml0 + ch * ml_stride + g * 2));
+#pragma unroll
+      for (int msk = 16; msk >= 1; msk >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, msk));
+      Mu[g] = (mx == -CUDART_INF_F) ? 0.f : mx;
+    }
+    float2 o[G];
+    float l[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      l[g] = 0.f;
+      o[g] = make_float2(0.f, 0.f);
+    }
+    for (int grp = warp; grp < n_groups; grp += AT_MERGE_WARPS) {
+      if (grp != warp) fetch_group(grp);
+#pragma unroll
+      for (int i = 0; i < PF; ++i) {
+        if (grp * PF + i < count) {
+#pragma unroll
+          for (int g = 0; g < G; ++g) {
+            const float w = exp2f(mlbuf[i][g].x - Mu[g]);
+            l[g] = fmaf(w, mlbuf[i][g].y, l[g]);
+            o[g].x = fmaf(w, vbuf[i][g].x, o[g].x);
+            o[g].y = fmaf(w, vbuf[i][g].y, o[g].y);
+          }
         }
       }
     }
-  };
 #pragma unroll
-  for (int i = 0; i < PF; ++i)
-    if (c_begin + i < c_end) fetch(c_begin + i, vbuf[i], mlbuf[i]);
-  float Mu[G];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    float mx = -CUDART_INF_F;
-    for (int ch = lane; ch < count; ch += 32) mx = fmaxf(mx, __ldcg(ml0 + ch * ml_stride + g * 2));
-#pragma unroll
-    for (int msk = 16; msk >= 1; msk >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, msk));
-    Mu[g] = (mx == -CUDART_INF_F) ? 0.f : mx;
-  }
-  float o[G][CPL], l[G];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    l[g] = 0.f;
-#pragma unroll
-    for (int e = 0; e < CPL; ++e) o[g][e] = 0.f;
-  }
-  for (int base = c_begin; base < c_end; base += PF) {
-#pragma unroll
-    for (int i = 0; i < PF; ++i) {
-      const int ch = base + i;
-      if (ch < c_end) {
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-          const float w = exp2f(mlbuf[i][g].x - Mu[g]);
-          l[g] = fmaf(w, mlbuf[i][g].y, l[g]);
-#pragma unroll
-          for (int e = 0; e < CPL; ++e) o[g][e] = fmaf(w, vbuf[i][g][e], o[g][e]);
-        }
-        if (ch + PF < c_end) fetch(ch + PF, vbuf[i], mlbuf[i]);
-      }
+    for (int g = 0; g < G; ++g) {
+      if (lane == 0) s_l[warp][g] = l[g];
+      s_o[warp][g][lane * 2] = o[g].x;
+      s_o[warp][g][lane * 2 + 1] = o[g].y;
     }
-  }
-  // the warp sums are added in warp order
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    if (lane == 0) s_l[warp][g] = l[g];
-#pragma unroll
-    for (int e = 0; e < CPL; ++e) s_o[warp][g][lane * CPL + e] = o[g][e];
   }
   __syncthreads();
-  for (int idx = threadIdx.x; idx < G * D_HEAD; idx += AT_THREADS) {
-    const int g = idx / D_HEAD, c = idx % D_HEAD;
-    float ov = s_o[0][g][c], lv = s_l[0][g];
-#pragma unroll
-    for (int w = 1; w < AT_WARPS; ++w) {
+  // the warp sums are added in warp order
+  for (int idx = threadIdx.x; idx < G * AT_MERGE_SLICE; idx += blockDim.x) {
+    const int g = idx / AT_MERGE_SLICE, c = idx % AT_MERGE_SLICE;
+    float ov = 0.f, lv = 0.f;
+    for (int w = 0; w < warps_used; ++w) {
       ov += s_o[w][g][c];
       lv += s_l[w][g];
     }
     const float r = lv > 0.f ? ov / lv : 0.f;
-    P.out[(static_cast<size_t>(si) * P.n_q + kvh * G + g) * D_HEAD + c] = __float2bfloat16_rn(r);
+    P.out[(static_cast<size_t>(si) * P.n_q + kvh * G + g) * D_HEAD + slice * AT_MERGE_SLICE + c] =
+        __float2bfloat16_rn(r);
   }
 }
 
@@ -455,7 +457,6 @@ template <int D_HEAD, int G>
 struct AttnSmem {
   static constexpr int NPART = AT_WARPS * (32 / (D_HEAD / 8));
   static constexpr int BYTES = NPART * G * (D_HEAD + 2) * 4;
-  static constexpr int MERGE_BYTES = AT_WARPS * G * (D_HEAD + 1) * 4;
 };
 template <int D_HEAD, int G, int NSEQ>
 static cudaError_t attn_configure() {
@@ -466,9 +467,6 @@ static cudaError_t attn_configure() {
   if (!done[dev & 63]) {
     e = cudaFuncSetAttribute(kvd_attn_split_kernel<D_HEAD, G, NSEQ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              AttnSmem<D_HEAD, G>::BYTES);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(kvd_attn_merge_kernel<D_HEAD, G, NSEQ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             AttnSmem<D_HEAD, G>::MERGE_BYTES);
     if (e != cudaSuccess) return e;
     done[dev & 63] = true;
   }
@@ -481,7 +479,6 @@ static cudaError_t attn_launch_pair(const AttnLaunchT<NSEQ> &S, cudaStream_t str
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cfg.blockDim = dim3(AT_THREADS, 1, 1);
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -494,13 +491,20 @@ static cudaError_t attn_launch_pair(const AttnLaunchT<NSEQ> &S, cudaStream_t str
   if (S.total_chunks > 0) {
     attr[0].val.programmaticStreamSerializationAllowed = (small && !(serial_launch_mask() & 2)) ? 1 : 0;
     cfg.gridDim = dim3(S.total_chunks * S.n_kv, 1, 1);
+    cfg.blockDim = dim3(AT_THREADS, 1, 1);
     cfg.dynamicSmemBytes = AttnSmem<D_HEAD, G>::BYTES;
     e = cudaLaunchKernelEx(&cfg, kvd_attn_split_kernel<D_HEAD, G, NSEQ>, S);
     if (e != cudaSuccess) return e;
   }
   attr[0].val.programmaticStreamSerializationAllowed = (small && !(serial_launch_mask() & 4)) ? 1 : 0;
-  cfg.gridDim = dim3(S.n_seqs * S.n_kv, 1, 1);
-  cfg.dynamicSmemBytes = AttnSmem<D_HEAD, G>::MERGE_BYTES;
+  // as many warps per merge CTA as the longest sequence of the launch has groups of partials
+  int max_chunks = 1;
+  for (int i = 0; i < S.n_seqs; ++i) max_chunks = S.seq[i].n_chunks > max_chunks ? S.seq[i].n_chunks : max_chunks;
+  int merge_warps = (max_chunks + attn_merge_group(G) - 1) / attn_merge_group(G);
+  if (merge_warps > AT_MERGE_WARPS) merge_warps = AT_MERGE_WARPS;
+  cfg.gridDim = dim3(S.n_seqs * S.n_kv * (D_HEAD / AT_MERGE_SLICE), 1, 1);
+  cfg.blockDim = dim3(32 * merge_warps, 1, 1);
+  cfg.dynamicSmemBytes = 0;
   return cudaLaunchKernelEx(&cfg, kvd_attn_merge_kernel<D_HEAD, G, NSEQ>, S);
 }
 

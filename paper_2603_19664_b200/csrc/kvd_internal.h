@@ -65,8 +65,14 @@ struct RecomputeParams {
 };
 
 // ------------------------------------------------------------------------------ decode attention
-constexpr int AT_THREADS = 512;
-constexpr int AT_WARPS = 16;
+constexpr int AT_THREADS = 128;        // streaming kernel
+constexpr int AT_WARPS = 4;
+constexpr int AT_CTAS_PER_SM = 4;      // 128 registers per thread
+constexpr int AT_MERGE_THREADS = 640;  // merge kernel: at most 20 warps (102 registers each)
+constexpr int AT_MERGE_WARPS = 20;
+constexpr int AT_MERGE_SLICE = 64;     // channels per merge CTA
+// partials one warp of the merge kernel fetches at once: 4*G registers each, 64 registers in all
+constexpr int attn_merge_group(int g) { return 16 / g >= 1 ? 16 / g : 1; }
 constexpr int AT_UNROLL = 8;          // keys per lane group per iteration
 constexpr int AT_MAX_SEQS = 64;       // sequences per launch (bounded by the kernel parameter space)
 
@@ -107,21 +113,24 @@ typedef AttnLaunchT<AT_MAX_SEQS> AttnLaunch;
 
 // keys per chunk for a head size and iteration count
 inline int attn_keys_per_warp_iter(int d_head) { return (32 / (d_head / 8)) * AT_UNROLL; }
-// Iterations per chunk.  The visible span is cut so that one sequence yields about 148 work units
-// (chunks x KV heads) -- one 16-warp CTA on each of a B200's SMs -- which keeps every SM equally
-// loaded when the batch is 1 and leaves few enough partials per head for a single merge level.  A
-// function of the model and of the visible span only, so a full cache and a recomputed + window +
-// current layout of the same positions are split identically, and a sequence's result does not
-// depend on what else is in the batch.
-inline int attn_target_chunks(int n_kv) {
-  const int t = 148 / n_kv;
-  return t > 1 ? t : 1;
+// Iterations per chunk.  Spans up to 8192 keys are cut into at most 128 chunks per (sequence, KV
+// head), longer ones so that one sequence yields about 592 work units (chunks x KV heads) -- four
+// CTAs on each of a B200's 148 SMs -- which keeps every SM equally loaded when the batch is 1.  A
+// chunk is at least two iterations: a CTA's prologue and combine cost as much as streaming a few
+// dozen keys, and in batched launches one-iteration CTAs measured 20 % slower.  A function of the
+// model and of the visible span only, so a full cache and a recomputed + window + current layout
+// of the same positions are split identically, and a sequence's result does not depend on what
+// else is in the batch.
+inline int attn_target_chunks(int n_kv, int span) {
+  if (span <= 8192) return 128;
+  const int t = (148 * AT_CTAS_PER_SM) / n_kv;
+  return t > 16 ? t : 16;
 }
 inline int attn_iters_for_span(int d_head, int n_kv, int span) {
   const int per_iter = attn_keys_per_warp_iter(d_head) * AT_WARPS;
-  const long long per_chunk_min = static_cast<long long>(per_iter) * attn_target_chunks(n_kv);
+  const long long per_chunk_min = static_cast<long long>(per_iter) * attn_target_chunks(n_kv, span);
   long long iters = (span + per_chunk_min - 1) / per_chunk_min;
-  if (iters < 1) iters = 1;
+  if (iters < 2) iters = 2;
   if (iters > 64) iters = 64;
   return static_cast<int>(iters);
 }
@@ -129,7 +138,8 @@ inline int attn_chunk_keys(int d_head, int iters) { return attn_keys_per_warp_it
 inline int attn_max_chunks(int d_head, int n_kv, int max_tokens) {
   const int per_iter = attn_keys_per_warp_iter(d_head) * AT_WARPS;
   const int capped = max_tokens / (per_iter * 64) + 2;  // once the iteration count is capped
-  const int target = attn_target_chunks(n_kv);
+  int target = attn_target_chunks(n_kv, max_tokens);
+  if (target < 128) target = 128;
   return (capped > target ? capped : target) + 2;
 }
 
