@@ -484,10 +484,10 @@ static cudaError_t attn_launch_pair(const AttnLaunchT<NSEQ> &S, cudaStream_t str
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  // Starting early pays for launches of a wave or two (the set-up hides under the predecessor's
-  // tail); with many-wave grids it measured slower (CTAs parked on SMs waiting for the predecessor:
-  // 12 us lost on a 20 us predecessor, 7 % on back-to-back long calls), so those are ordered plainly.
-  const bool small = S.total_chunks * S.n_kv <= 2 * 148;
+  // Starting early pays for launches of up to one wave (the set-up hides under the predecessor's tail);
+  // a many-wave grid whose first CTAs sit on the SMs waiting slowed a short predecessor down in
+  // measurements (11 us lost on a 24 us predecessor), so those are ordered plainly.
+  const bool small = S.total_chunks * S.n_kv <= 148 * AT_CTAS_PER_SM;
   if (S.total_chunks > 0) {
     attr[0].val.programmaticStreamSerializationAllowed = (small && !(serial_launch_mask() & 2)) ? 1 : 0;
     cfg.gridDim = dim3(S.total_chunks * S.n_kv, 1, 1);
