@@ -338,6 +338,241 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM) kvd_attn_split_ker
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Streaming kernel for wide query groups (G >= 3, d_head <= 128).  With four or more query heads per
+// KV head the fp32 pipes, not the loads, bound the kernel above (about 45 warp instructions per key),
+// so the two products run on the tensor cores with the query heads padded to a 16-row tile:
+//     S (16 heads x 8 keys)         = Q (16 x d_head) * K^T            mma.m16n8k16, d_head/16 per 8 keys
+//     O^T (d_head x 8 heads)       += V^T (d_head x 8 keys) * P^T      mma.m16n8k8,  d_head/16 per 8 keys
+// Operands come straight from global memory with the same 16-byte loads: a contraction does not care
+// which channel (or key) sits in which slot as long as both operands agree, so each thread loads
+// contiguous 16-byte pieces and uses them as the fragment registers the instruction wants -- K pieces
+// as B fragments of the first product (the query is loaded the same way), pairs of V pieces of two
+// neighbouring keys, interleaved with two byte permutes, as A fragments of the second.  P is rounded
+// to bf16 for the second product (fp32 sums), as the scores' softmax weights are in any tensor-core
+// attention; the partials have the same format as those of the kernel above and go to the same merge.
+// Chunking, the position -> (chunk, warp, block) assignment and the masking rules are identical.
+__device__ __forceinline__ void mma_bf16_m16n8k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                  uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+               "{%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_bf16_m16n8k8(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5}, {%6}, {%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(b0));
+}
+
+template <int D_HEAD, int G, int NSEQ>
+__global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM)
+    kvd_attn_split_mma_kernel(const __grid_constant__ AttnLaunchT<NSEQ> P) {
+  static_assert(G >= 1 && G <= 8 && D_HEAD <= 128, "query heads are the 8 columns of the second product");
+  constexpr int LPK = D_HEAD / 8, KPL = 32 / LPK;
+  constexpr int WARP_KEYS = KPL * AT_UNROLL;  // keys per warp and iteration, as in the kernel above
+  constexpr int NBLK = WARP_KEYS / 8;         // blocks of 8 keys
+  constexpr int KP = D_HEAD / 32;             // 16-byte pieces of a key row per thread (first product)
+  constexpr int VP = D_HEAD / 64;             // 16-byte pieces of a value row per thread (second product)
+  constexpr int MB = D_HEAD / 16;             // 16-channel blocks of the output
+  __shared__ float s_o[AT_WARPS][G][D_HEAD];
+  __shared__ float s_m[AT_WARPS][G];
+  __shared__ float s_l[AT_WARPS][G];
+  grid_launch_dependents();
+
+  int si = 0;
+  {
+    int lo = 0, hi = P.n_seqs - 1;
+    const int b = blockIdx.x / P.n_kv;
+    while (lo < hi) {  // last sequence whose first partial index is <= b
+      const int mid = (lo + hi + 1) >> 1;
+      if (P.seq[mid].part_base - P.seq[0].part_base <= b) lo = mid; else hi = mid - 1;
+    }
+    si = lo;
+  }
+  const AttnSeq &S = P.seq[si];
+  const int chunk = blockIdx.x / P.n_kv - (S.part_base - P.seq[0].part_base);
+  const int kvh = blockIdx.x % P.n_kv;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g8 = lane >> 2;  // fragment row / column index: query head, key of a block, channel group
+  const int t = lane & 3;    // fragment pair index
+  const int chunk_keys = WARP_KEYS * AT_WARPS * S.iters;
+  const int chunk_pos0 = S.chunk0_pos + chunk * chunk_keys;
+
+  grid_dependency_wait();
+  // ---- query rows as A fragments: thread (g8, t) holds channels [32 j + 8 t, 32 j + 8 t + 8) of head g8
+  uint32_t qa[KP][4];
+#pragma unroll
+  for (int j = 0; j < KP; ++j) {
+    uint4 w = make_uint4(0u, 0u, 0u, 0u);
+    if (g8 < G)
+      w = *reinterpret_cast<const uint4 *>(P.q + (static_cast<size_t>(si) * P.n_q + kvh * G + g8) * D_HEAD + 32 * j + 8 * t);
+    qa[j][0] = w.x;
+    qa[j][1] = w.y;
+    qa[j][2] = w.z;
+    qa[j][3] = w.w;
+  }
+  float m_run = -CUDART_INF_F, l_run = 0.f;  // of head g8 (threads with g8 >= G carry padding)
+  float oacc[MB][4];                         // O^T: rows = channels of this thread's group, columns = heads 2t, 2t+1
+#pragma unroll
+  for (int mb = 0; mb < MB; ++mb)
+#pragma unroll
+    for (int r = 0; r < 4; ++r) oacc[mb][r] = 0.f;
+
+  const size_t head_el = static_cast<size_t>(kvh) * D_HEAD;
+  int fast_seg = -1;
+#pragma unroll
+  for (int sg = 0; sg < KVD_MAX_SEGMENTS; ++sg)
+    if (chunk_pos0 >= S.first[sg] && chunk_pos0 + chunk_keys <= S.first[sg] + S.len[sg]) fast_seg = sg;
+  const bool fast = fast_seg >= 0 && chunk_pos0 >= S.lo_pos && chunk_pos0 + chunk_keys - 1 <= S.hi_pos;
+  const __nv_bfloat16 *fk = P.q, *fv = P.q;
+  long long fstride = 0;
+  if (fast) {
+    fstride = S.stride[fast_seg];
+    const size_t off = static_cast<size_t>(chunk_pos0 - S.first[fast_seg]) * fstride + head_el;
+    fk = S.k[fast_seg] + off;
+    fv = S.v[fast_seg] + off;
+  }
+  // row pointers (K, V) of the key at chunk-relative position rel, or null when it is not visible
+  auto locate = [&](int rel, const __nv_bfloat16 *&kp, const __nv_bfloat16 *&vp) {
+    kp = vp = nullptr;
+    if (fast) {
+      kp = fk + static_cast<size_t>(rel) * fstride;
+      vp = fv + static_cast<size_t>(rel) * fstride;
+      return;
+    }
+    const int pos = chunk_pos0 + rel;
+    if (pos >= S.lo_pos && pos <= S.hi_pos) {
+#pragma unroll
+      for (int sg = 0; sg < KVD_MAX_SEGMENTS; ++sg) {
+        const int r = pos - S.first[sg];
+        if (r >= 0 && r < S.len[sg]) {
+          const size_t off = static_cast<size_t>(r) * S.stride[sg] + head_el;
+          kp = S.k[sg] + off;
+          vp = S.v[sg] + off;
+        }
+      }
+    }
+  };
+
+  for (int it = 0; it < S.iters; ++it) {
+    const int rel0 = (it * AT_WARPS + warp) * WARP_KEYS;
+    // ---- all loads of the iteration: per block, the key row of key g8 (first product) and the value
+    // rows of keys 2t and 2t+1 (second product); invisible keys read as zeros
+    uint4 kr[NBLK][KP], vr[NBLK][2][VP];
+    uint32_t vmask = 0;  // bit 2b + i: key 8b + 2t + i is visible
+#pragma unroll
+    for (int b = 0; b < NBLK; ++b) {
+      const __nv_bfloat16 *kp, *vp_unused, *kp_unused, *vp0, *vp1;
+      locate(rel0 + 8 * b + g8, kp, vp_unused);
+      locate(rel0 + 8 * b + 2 * t, kp_unused, vp0);
+      locate(rel0 + 8 * b + 2 * t + 1, kp_unused, vp1);
+#pragma unroll
+      for (int j = 0; j < KP; ++j)
+        kr[b][j] = kp ? ldg_stream(kp + 32 * j + 8 * t) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int i = 0; i < VP; ++i) {
+        vr[b][0][i] = vp0 ? ldg_stream(vp0 + 64 * i + 8 * g8) : make_uint4(0u, 0u, 0u, 0u);
+        vr[b][1][i] = vp1 ? ldg_stream(vp1 + 64 * i + 8 * g8) : make_uint4(0u, 0u, 0u, 0u);
+      }
+      vmask |= (vp0 ? 1u : 0u) << (2 * b);
+      vmask |= (vp1 ? 1u : 0u) << (2 * b + 1);
+    }
+    if (!__any_sync(0xffffffffu, vmask != 0u)) continue;  // nothing visible in this warp's keys
+
+#pragma unroll
+    for (int b = 0; b < NBLK; ++b) {
+      // ---- scores of 8 keys for (up to) 8 heads
+      float sc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int j = 0; j < KP; ++j) {
+        mma_bf16_m16n8k16(sc, qa[j][0], 0u, qa[j][1], 0u, kr[b][j].x, kr[b][j].y);
+        mma_bf16_m16n8k16(sc, qa[j][2], 0u, qa[j][3], 0u, kr[b][j].z, kr[b][j].w);
+      }
+      // thread (g8, t): head g8, keys 2t and 2t+1 of the block
+      const float s0 = ((vmask >> (2 * b)) & 1u) ? sc[0] * P.scale_log2e : -CUDART_INF_F;
+      const float s1 = ((vmask >> (2 * b + 1)) & 1u) ? sc[1] * P.scale_log2e : -CUDART_INF_F;
+      float bmax = fmaxf(s0, s1);
+      bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
+      bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
+      const float m_new = fmaxf(m_run, bmax);
+      const float m_use = (m_new == -CUDART_INF_F) ? 0.f : m_new;
+      const float corr = exp2f(m_run - m_use);  // 0 while nothing has been seen
+      const float p0 = exp2f(s0 - m_use), p1 = exp2f(s1 - m_use);
+      l_run = fmaf(l_run, corr, p0 + p1);
+      m_run = m_new;
+      const uint32_t pk = pack_bf16(p0, p1);  // B fragment of the second product: keys 2t, 2t+1, head g8
+      // ---- rescale the accumulators when a maximum moved (columns are heads 2t and 2t+1)
+      const float c_even = __shfl_sync(0xffffffffu, corr, (2 * t) * 4);
+      const float c_odd = __shfl_sync(0xffffffffu, corr, (2 * t + 1) * 4);
+      if (__any_sync(0xffffffffu, c_even != 1.0f || c_odd != 1.0f)) {
+#pragma unroll
+        for (int mb = 0; mb < MB; ++mb) {
+          oacc[mb][0] *= c_even;
+          oacc[mb][1] *= c_odd;
+          oacc[mb][2] *= c_even;
+          oacc[mb][3] *= c_odd;
+        }
+      }
+      // ---- weighted values: A fragment rows are this thread's channels 64 i + 8 g8 + 2 e (+1), taken
+      // from keys 2t (low half) and 2t+1 (high half)
+#pragma unroll
+      for (int i = 0; i < VP; ++i) {
+        const uint32_t v0[4] = {vr[b][0][i].x, vr[b][0][i].y, vr[b][0][i].z, vr[b][0][i].w};
+        const uint32_t v1[4] = {vr[b][1][i].x, vr[b][1][i].y, vr[b][1][i].z, vr[b][1][i].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const uint32_t a0 = __byte_perm(v0[e], v1[e], 0x5410);  // channel 2e of both keys
+          const uint32_t a1 = __byte_perm(v0[e], v1[e], 0x7632);  // channel 2e + 1 of both keys
+          mma_bf16_m16n8k8(oacc[4 * i + e], a0, a1, pk);
+        }
+      }
+    }
+  }
+
+  // ---- one partial per warp into shared memory, then the CTA's partial as in the kernel above
+  {
+    float l = l_run;
+    l += __shfl_xor_sync(0xffffffffu, l, 1);
+    l += __shfl_xor_sync(0xffffffffu, l, 2);
+    if (t == 0 && g8 < G) {
+      s_m[warp][g8] = m_run;
+      s_l[warp][g8] = l;
+    }
+#pragma unroll
+    for (int mb = 0; mb < MB; ++mb) {
+      const int ch = 64 * (mb >> 2) + 8 * g8 + 2 * (mb & 3);
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int head = 2 * t + (r & 1);
+        if (head < G) s_o[warp][head][ch + (r >> 1)] = oacc[mb][r];
+      }
+    }
+  }
+  __syncthreads();
+  const size_t pidx = static_cast<size_t>(S.part_base + chunk);
+  for (int idx = threadIdx.x; idx < G * D_HEAD; idx += AT_THREADS) {
+    const int g = idx / D_HEAD, c = idx % D_HEAD;
+    float M = -CUDART_INF_F;
+#pragma unroll
+    for (int pp = 0; pp < AT_WARPS; ++pp) M = fmaxf(M, s_m[pp][g]);
+    const float Mu = (M == -CUDART_INF_F) ? 0.f : M;
+    float o = 0.f, l = 0.f;
+#pragma unroll
+    for (int pp = 0; pp < AT_WARPS; ++pp) {
+      const float w = exp2f(s_m[pp][g] - Mu);
+      o = fmaf(w, s_o[pp][g][c], o);
+      l = fmaf(w, s_l[pp][g], l);
+    }
+    const size_t hq = pidx * P.n_q + kvh * G + g;
+    P.part_o[hq * D_HEAD + c] = o;
+    if (c == 0) {
+      P.part_ml[hq * 2] = M;
+      P.part_ml[hq * 2 + 1] = l;
+    }
+  }
+}
+
 // Second kernel of a decode step: the chunk partials of every (sequence, KV head) are merged in chunk
 // order and the output written.  A separate launch instead of a "last CTA merges" tail: every
 // dependent global-memory hop (partial -> fence -> counter -> merge) measured above a microsecond,
@@ -465,9 +700,11 @@ static cudaError_t attn_configure() {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (!done[dev & 63]) {
-    e = cudaFuncSetAttribute(kvd_attn_split_kernel<D_HEAD, G, NSEQ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             AttnSmem<D_HEAD, G>::BYTES);
-    if (e != cudaSuccess) return e;
+    if constexpr (!(G >= 3 && D_HEAD <= 128)) {
+      e = cudaFuncSetAttribute(kvd_attn_split_kernel<D_HEAD, G, NSEQ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               AttnSmem<D_HEAD, G>::BYTES);
+      if (e != cudaSuccess) return e;
+    }
     done[dev & 63] = true;
   }
   return cudaSuccess;
@@ -492,8 +729,13 @@ static cudaError_t attn_launch_pair(const AttnLaunchT<NSEQ> &S, cudaStream_t str
     attr[0].val.programmaticStreamSerializationAllowed = (small && !(serial_launch_mask() & 2)) ? 1 : 0;
     cfg.gridDim = dim3(S.total_chunks * S.n_kv, 1, 1);
     cfg.blockDim = dim3(AT_THREADS, 1, 1);
-    cfg.dynamicSmemBytes = AttnSmem<D_HEAD, G>::BYTES;
-    e = cudaLaunchKernelEx(&cfg, kvd_attn_split_kernel<D_HEAD, G, NSEQ>, S);
+    if constexpr (G >= 3 && D_HEAD <= 128) {
+      cfg.dynamicSmemBytes = 0;
+      e = cudaLaunchKernelEx(&cfg, kvd_attn_split_mma_kernel<D_HEAD, G, NSEQ>, S);
+    } else {
+      cfg.dynamicSmemBytes = AttnSmem<D_HEAD, G>::BYTES;
+      e = cudaLaunchKernelEx(&cfg, kvd_attn_split_kernel<D_HEAD, G, NSEQ>, S);
+    }
     if (e != cudaSuccess) return e;
   }
   attr[0].val.programmaticStreamSerializationAllowed = (small && !(serial_launch_mask() & 4)) ? 1 : 0;
