@@ -11,7 +11,7 @@ import torch
 
 import oracle
 import paper_2603_19664_b200 as kvd
-from kvd_synth import (GEMMA3_4B_GLOBAL, GEMMA3_4B_LOCAL, QWEN3_4B, SMOLLM2_135M, TINY_GQA, TINY_MHA, bf16_to_f64,
+from kvd_synth import (LayerShape, GEMMA3_4B_GLOBAL, GEMMA3_4B_LOCAL, QWEN3_4B, SMOLLM2_135M, TINY_GQA, TINY_MHA, bf16_to_f64,
                        make_kv, make_query, make_residuals)
 from gpu_util import dev, host_bits, host_f64, open_layer, oracle_kv
 
@@ -123,6 +123,38 @@ def test_batch_with_mixed_lengths_windows_and_gaps():
     ref = oracle_attention(shape, q, qpos, segs)
     for b in range(5):
         attn_check(host_f64(out)[b], ref[b])
+
+
+# every supported group size on both streaming kernels (fp32 pipes; tensor cores for 3+ query heads per
+# KV head at d_head <= 128), including the widest group and a sliding window
+WIDE_SHAPES = [LayerShape("g8-d128", 256, 16, 2, 128, 1e-6, False, 1.0e4),
+               LayerShape("g8-d64", 256, 8, 1, 64, 1e-6, False, 1.0e4, 300),
+               LayerShape("g3-d128", 256, 6, 2, 128, 1e-6, False, 1.0e4),
+               LayerShape("g4-d256", 256, 8, 2, 256, 1e-6, False, 1.0e4),
+               LayerShape("g8-d256", 256, 8, 1, 256, 1e-6, False, 1.0e4),
+               LayerShape("g1-d128", 256, 2, 2, 128, 1e-6, False, 1.0e4)]
+
+
+@pytest.mark.parametrize("shape", WIDE_SHAPES, ids=lambda s: s.name)
+def test_group_sizes_on_both_streaming_kernels(shape):
+    ctx, _ = open_layer(shape, max_tokens=8192, max_batch=3)
+    lens = [5000, 777, 9]
+    q = make_query(shape, 3, seed=31)
+    segs, qpos = [], []
+    for b, T in enumerate(lens):
+        K, V = make_kv(shape, T, seed=310 + b)
+        cut = max(1, T - 100)
+        segs.append([(K[:cut], V[:cut], 0), (K[cut:], V[cut:], cut)])
+        qpos.append(T - 1)
+    out = gpu_attention(ctx, shape, q, qpos, segs)
+    attn_check(host_f64(out), oracle_attention(shape, q, qpos, segs))
+    # one segment per sequence: identical bits
+    segs1 = []
+    for b, T in enumerate(lens):
+        K, V = make_kv(shape, T, seed=310 + b)
+        segs1.append([(K, V, 0)])
+    out1 = gpu_attention(ctx, shape, q, qpos, segs1)
+    assert torch.equal(out, out1)
 
 
 @pytest.mark.parametrize("shape", [TINY_GQA, SMOLLM2_135M, GEMMA3_4B_GLOBAL, QWEN3_4B], ids=lambda s: s.name)
