@@ -134,7 +134,11 @@ kvd_status kvd_set_layer(kvd_ctx *ctx, int layer, const kvd_layer_desc *ldesc, v
 size_t kvd_store_bytes(const kvd_model_desc *desc, int layers_stored);
 
 /* Hand the context a caller-owned DEVICE arena (256-byte aligned, >= kvd_store_bytes) for the
- * residual store C of Algorithm 1.  Resets all row counts to zero. */
+ * residual store C of Algorithm 1.  Resets all row counts to zero.
+ * Layout (the arena stays the caller's, who may read it): residual rows as bf16
+ * [layers_stored][max_seqs][max_tokens_per_seq][d_hidden] from the start of the arena, then, at the
+ * next multiple of 256 bytes, their positions as int32 [layers_stored][max_seqs][max_tokens_per_seq].
+ * Row r of (layer, seq) is valid for r < kvd_rows_stored(ctx, layer, seq). */
 kvd_status kvd_attach_store(kvd_ctx *ctx, void *arena, size_t bytes, int layers_stored);
 
 /* Forget the rows of one sequence (all layers) so that its slot can be reused. */

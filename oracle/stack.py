@@ -4,12 +4,16 @@ The model is the paper's pre-norm block (Eq. 3-9): RMSNorm -> Q/K/V projections 
 softmax attention -> W_o -> residual add; RMSNorm -> gated MLP -> residual add; then a final
 RMSNorm, the vocabulary projection and a greedy argmax (lowest index wins ties).
 
-Two cache policies share every line of the model:
+Three cache policies share every line of the model:
   * ``full``      -- append (K_t, V_t) of every token, never evict;
   * ``kvdirect``  -- keep at most B live entries per layer; the keys and values of evicted tokens
                      are rebuilt each step from the checkpointed residual row that entered the
                      layer (Eq. 13-14), then concatenated [rebuilt, live window, current] as in
                      Algorithm 1.  B = 0 is allowed.
+  * ``chained``   -- as ``kvdirect`` but with ONE checkpointed row per token, the row entering
+                     layer 0 (the d_hidden * b bytes per token of Eq. 24): every step the evicted
+                     tokens are carried through the layers again, so that at layer l their rows
+                     h^(l), and from them their keys and values, exist while that layer runs.
 K and V of the current token and of rebuilt tokens come from the same oracle routine
 (``oracle.recompute_kv``), which treats rows independently, so Proposition 3.2's "same operations
 in the same order" holds literally and the two policies must agree bit for bit.
@@ -52,59 +56,84 @@ class OracleStack:
     def __init__(self, shape, weights_f64: Dict, policy: str = "full", budget: int = 0):
         """``shape`` is a kvd_synth.StackShape-like object; ``weights_f64`` maps
         'embed', 'lm_head', 'gamma_final' and 'layers' (list of dicts) to float64 arrays."""
-        assert policy in ("full", "kvdirect")
+        assert policy in ("full", "kvdirect", "chained")
         self.s = shape
         self.w = weights_f64
         self.policy = policy
         self.budget = int(budget)
         self.layers = [LayerState() for _ in range(shape.n_layers)]
         self.t = 0  # next position
+        self.rows0: List[np.ndarray] = []  # "chained": the one checkpointed row per token
+        self.replayed_rows = 0
         self.trace_kv: Optional[List[List]] = None  # when set: per layer list of (K_t, V_t) as first computed
+
+    # -- one token through one layer, given the keys/values before it ------------------------------
+    def _block(self, l: int, h: np.ndarray, pos: int, segments_before: List):
+        """Eq. 3-9 for the row ``h`` entering layer ``l`` at position ``pos``.  ``segments_before``
+        are (K, V, first_pos) runs of the keys at earlier positions.  Returns (row leaving the layer,
+        K_t, V_t)."""
+        s, lw, ls = self.s, self.w["layers"][l], self.s.layer_shape(l)
+        scale = 1.0 / np.sqrt(float(s.d_head))
+        xb = rmsnorm(h, lw["gamma_in"], s.rms_eps)
+        q = (xb @ lw["w_q"]).reshape(s.n_q_heads, s.d_head)
+        for hh in range(s.n_q_heads):
+            if s.qk_norm:
+                q[hh] = rmsnorm(q[hh], lw["gamma_q"], s.rms_eps)
+            q[hh] = rope(q[hh], pos, ls.rope_theta, s.rope_style)
+        k_t, v_t = self._kv_rows(l, [h], [pos])
+        heads = decode_attention(q, pos, list(segments_before) + [(k_t, v_t, pos)], scale, ls.sliding_window)
+        h = h + heads.reshape(-1) @ lw["w_o"]  # Eq. 8
+        xm = rmsnorm(h, lw["gamma_mlp"], s.rms_eps)
+        h = h + (_act(xm @ lw["w_gate"], s.activation) * (xm @ lw["w_up"])) @ lw["w_down"]  # Eq. 9
+        return h, k_t, v_t
 
     # -- one decoding step (Algorithm 1) -------------------------------------------------------
     def step(self, token: int) -> np.ndarray:
         s, w = self.s, self.w
         pos = self.t
         h = w["embed"][token].copy()
-        scale = 1.0 / np.sqrt(float(s.d_head))
+        chained = self.policy == "chained"
+        if chained:
+            self.rows0.append(h.copy())  # the only checkpoint: the row entering layer 0
+            n_ev = min(self.layers[0].win_first, pos) if self.layers[0].win_k else pos
+            ev_rows = [self.rows0[j] for j in range(n_ev)]  # evicted tokens' rows entering the current layer
         for l in range(s.n_layers):
-            lw = w["layers"][l]
             ls = s.layer_shape(l)
             st = self.layers[l]
-            st.rows.append(h.copy())  # STORE_RESIDUAL: the row entering layer l
-            # current-token projections (Eq. 3-5)
-            xb = rmsnorm(h, lw["gamma_in"], s.rms_eps)
-            q = (xb @ lw["w_q"]).reshape(s.n_q_heads, s.d_head)
-            for hh in range(s.n_q_heads):
-                if s.qk_norm:
-                    q[hh] = rmsnorm(q[hh], lw["gamma_q"], s.rms_eps)
-                q[hh] = rope(q[hh], pos, ls.rope_theta, s.rope_style)
-            k_t, v_t = self._kv(l, [pos])
-            if self.trace_kv is not None:
-                self.trace_kv[l].append((k_t[0].copy(), v_t[0].copy()))
+            if not chained:
+                st.rows.append(h.copy())  # STORE_RESIDUAL: the row entering layer l
             # which past positions does this layer need?
             lo = 0 if ls.sliding_window == 0 else max(0, pos - ls.sliding_window + 1)
             segments = []
             win_lo = st.win_first
             n_win = len(st.win_k)
-            if self.policy == "kvdirect":
+            if chained:
+                if n_ev > 0:
+                    k_ev, v_ev = self._kv_rows(l, ev_rows, list(range(n_ev)))  # RECOMPUTE_KV from h^(l)
+                    if lo < n_ev:
+                        segments.append((k_ev[lo:], v_ev[lo:], lo))
+            elif self.policy == "kvdirect":
                 old = list(range(lo, min(win_lo, pos))) if n_win > 0 else list(range(lo, pos))
                 if old:
                     k_old, v_old = self._kv(l, old)  # RECOMPUTE_KV(C, l)
                     segments.append((k_old, v_old, old[0]))
             if n_win > 0:
                 segments.append((np.stack(st.win_k), np.stack(st.win_v), win_lo))
-            segments.append((k_t, v_t, pos))
-            heads = decode_attention(q, pos, segments, scale, ls.sliding_window)
-            h = h + heads.reshape(-1) @ lw["w_o"]  # Eq. 8
-            xm = rmsnorm(h, lw["gamma_mlp"], s.rms_eps)
-            h = h + (_act(xm @ lw["w_gate"], s.activation) * (xm @ lw["w_up"])) @ lw["w_down"]  # Eq. 9
+            h, k_t, v_t = self._block(l, h, pos, segments)
+            if self.trace_kv is not None:
+                self.trace_kv[l].append((k_t[0].copy(), v_t[0].copy()))
+            if chained and n_ev > 0 and l + 1 < s.n_layers:
+                # the evicted tokens' own step through this layer, in position order: token j sees
+                # the evicted keys before it
+                ev_rows = [self._block(l, ev_rows[j], j, [(k_ev[:j], v_ev[:j], 0)] if j > 0 else [])[0]
+                           for j in range(n_ev)]
+                self.replayed_rows += n_ev
             # cache update, then eviction of the oldest entries
             if n_win == 0:
                 st.win_first = pos
             st.win_k.append(k_t[0])
             st.win_v.append(v_t[0])
-            if self.policy == "kvdirect":
+            if self.policy != "full":
                 while len(st.win_k) > self.budget:
                     st.win_k.pop(0)
                     st.win_v.pop(0)
@@ -113,13 +142,15 @@ class OracleStack:
         hf = rmsnorm(h, w["gamma_final"], s.rms_eps)
         return hf @ w["lm_head"]
 
-    def _kv(self, l: int, positions: List[int]):
+    def _kv_rows(self, l: int, rows: List[np.ndarray], positions: List[int]):
         s, lw, ls = self.s, self.w["layers"][l], self.s.layer_shape(l)
+        return recompute_kv(np.stack(rows), np.asarray(positions, dtype=np.int32), lw["gamma_in"], lw["w_kv"],
+                            s.n_kv_heads, s.d_head, s.rms_eps, ls.rope_theta,
+                            lw.get("gamma_k") if s.qk_norm else None, s.rms_eps, s.rope_style)
+
+    def _kv(self, l: int, positions: List[int]):
         st = self.layers[l]
-        X = np.stack([st.rows[p] for p in positions])
-        return recompute_kv(X, np.asarray(positions, dtype=np.int32), lw["gamma_in"], lw["w_kv"], s.n_kv_heads,
-                            s.d_head, s.rms_eps, ls.rope_theta, lw.get("gamma_k") if s.qk_norm else None,
-                            s.rms_eps, s.rope_style)
+        return self._kv_rows(l, [st.rows[p] for p in positions], positions)
 
     # -- greedy generation ---------------------------------------------------------------------
     def generate(self, prompt: List[int], n_new: int, forced: Optional[List[int]] = None):

@@ -6,11 +6,20 @@ rotation, W_o, the gated MLP, the final norm, the vocabulary projection and the 
 torch arithmetic: it is scaffolding that both cache policies share line for line, needed only to
 produce realistic residual streams and to turn attention outputs into tokens.
 
-Two cache policies, as in the oracle's stack:
+Cache policies, as in the oracle's stack:
   * "full"      every token's K/V is kept; attention reads one stored segment;
   * "kvdirect"  at most B live K/V entries per layer; the K/V of evicted tokens are rebuilt every
                 step from the checkpointed residual rows (kvd_recompute_kv from the store) and
                 attention reads [rebuilt, live window incl. current].
+  * GpuStackChained: one checkpointed row per token (the row entering layer 0), B live K/V entries
+                per layer; every step the evicted prefix is carried through the layers again, layer by
+                layer next to the new tokens, so that each layer's K/V of the evicted tokens exist only
+                while that layer runs.  This is the variant whose memory is Eq. 24 / Eq. 28.
+
+`exact_scaffold=True` makes the scaffold's matrix products and norms accumulate in fp64 before
+rounding to bf16: their bf16 results then do not depend on how many rows are processed at once
+(the library's kernels have that property by construction), which the chained variant needs to
+reproduce the first pass bit for bit when it replays tokens in different batches.
 """
 import math
 
@@ -51,9 +60,11 @@ def torch_stack_weights(stack, seed=0):
 
 
 class GpuStack:
-    def __init__(self, stack, weights, policy="full", budget=0, max_tokens=512, device_weights=False):
+    def __init__(self, stack, weights, policy="full", budget=0, max_tokens=512, device_weights=False,
+                 exact_scaffold=False, layers_stored=None):
         assert policy in ("full", "kvdirect")
         self.s, self.policy, self.budget, self.max_tokens = stack, policy, int(budget), max_tokens
+        self.exact = bool(exact_scaffold)
         s = stack
         self.kdim = s.n_kv_heads * s.d_head
         if device_weights:
@@ -77,8 +88,9 @@ class GpuStack:
                                    self.lw[l].get("gamma_k") if s.qk_norm else None, ls.rope_theta, ls.sliding_window)
         self.ws = torch.empty(kvd.kvd_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
         self.ctx.kvd_attach_workspace(self.ws)
-        self.arena = torch.empty(kvd.kvd_store_bytes(desc, s.n_layers), dtype=torch.uint8, device="cuda")
-        self.ctx.kvd_attach_store(self.arena, s.n_layers)
+        n_stored = s.n_layers if layers_stored is None else layers_stored
+        self.arena = torch.empty(kvd.kvd_store_bytes(desc, n_stored), dtype=torch.uint8, device="cuda")
+        self.ctx.kvd_attach_store(self.arena, n_stored)
         # K/V storage indexed by position: the full cache, or the live window of the bounded policy
         self.k_live = [torch.zeros((max_tokens, self.kdim), dtype=torch.bfloat16, device="cuda") for _ in range(s.n_layers)]
         self.v_live = [torch.zeros((max_tokens, self.kdim), dtype=torch.bfloat16, device="cuda") for _ in range(s.n_layers)]
@@ -91,8 +103,41 @@ class GpuStack:
         self.inv_freq = {}
 
     def _rms(self, x, gamma):
+        if self.exact:
+            xd = x.double()
+            return (xd * torch.rsqrt(xd.pow(2).mean(-1, keepdim=True) + self.s.rms_eps) * gamma.double()).float()
         xf = x.float()
         return xf * torch.rsqrt(xf.pow(2).mean(-1, keepdim=True) + self.s.rms_eps) * gamma.float()
+
+    def _mm(self, x, w):
+        """bf16 x @ bf16 w -> bf16 (fp64 accumulation when exact_scaffold)."""
+        if self.exact:
+            return (x.double() @ w.double()).to(torch.bfloat16)
+        return x @ w
+
+    def _qnorm(self, q, gamma_q):
+        if self.exact:
+            qd = q.double()
+            return (qd * torch.rsqrt(qd.pow(2).mean(-1, keepdim=True) + self.s.rms_eps) * gamma_q.double()).float()
+        return q * torch.rsqrt(q.pow(2).mean(-1, keepdim=True) + self.s.rms_eps) * gamma_q.float()
+
+    def _queries(self, l, h, positions):
+        """Scaffold: normalised, rotated bf16 queries [U, n_q, d_head] of residual rows h [U, d]."""
+        s, lw, ls = self.s, self.lw[l], self.s.layer_shape(l)
+        xb = self._rms(h, lw["gamma_in"]).to(torch.bfloat16)
+        q = self._mm(xb, lw["w_q"]).float().view(h.shape[0], s.n_q_heads, s.d_head)
+        if s.qk_norm:
+            q = self._qnorm(q, lw["gamma_q"])
+        return self._rope_q(q, positions, ls.rope_theta).to(torch.bfloat16).contiguous()
+
+    def _after_attention(self, l, h, out):
+        """Scaffold: W_o, residual add, gated MLP, residual add (Eq. 8-9) for rows h [U, d]."""
+        lw = self.lw[l]
+        h = (h.float() + self._mm(out.view(h.shape[0], -1), lw["w_o"]).float()).to(torch.bfloat16)
+        xm = self._rms(h, lw["gamma_mlp"]).to(torch.bfloat16)
+        gate = self._act(self._mm(xm, lw["w_gate"]).float()) * self._mm(xm, lw["w_up"]).float()
+        mlp = self._mm(gate.to(torch.bfloat16), lw["w_down"])
+        return (h.float() + mlp.float()).to(torch.bfloat16)
 
     def _rope_q(self, q, pos, theta):
         """q: [..., n_q, d_head] with `pos` an int or a list of positions (one per leading row)."""
@@ -129,11 +174,7 @@ class GpuStack:
             lw, ls = self.lw[l], s.layer_shape(l)
             ctx.kvd_checkpoint_residual(0, l, h, pos_t, 1)  # STORE_RESIDUAL: the row entering layer l
             # scaffold: query
-            xb = self._rms(h, lw["gamma_in"]).to(torch.bfloat16)
-            q = (xb @ lw["w_q"]).float().view(s.n_q_heads, s.d_head)
-            if s.qk_norm:
-                q = q * torch.rsqrt(q.pow(2).mean(-1, keepdim=True) + s.rms_eps) * lw["gamma_q"].float()
-            q = self._rope_q(q, pos, ls.rope_theta).to(torch.bfloat16).view(1, s.n_q_heads, s.d_head).contiguous()
+            q = self._queries(l, h, [pos])
             # hot path: K_t, V_t of the current token, written at its position in the live storage
             kl, vl = self.k_live[l], self.v_live[l]
             lo = 0 if ls.sliding_window == 0 else max(0, pos - ls.sliding_window + 1)
@@ -155,15 +196,15 @@ class GpuStack:
             out = torch.empty((1, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
             ctx.kvd_decode_attention(l, 1, q, [pos], [segs], 0.0, out)
             # scaffold: W_o, MLP
-            h = (h.float() + (out.view(1, -1) @ lw["w_o"]).float()).to(torch.bfloat16)
-            xm = self._rms(h, lw["gamma_mlp"]).to(torch.bfloat16)
-            mlp = (self._act((xm @ lw["w_gate"]).float()) * (xm @ lw["w_up"]).float()).to(torch.bfloat16) @ lw["w_down"]
-            h = (h.float() + mlp.float()).to(torch.bfloat16)
+            h = self._after_attention(l, h, out)
             if self.policy == "kvdirect":
                 self.win_first[l] = max(self.win_first[l], pos + 1 - self.budget)  # evict the oldest
         self.t += 1
-        hf = self._rms(h, self.g_final).to(torch.bfloat16)
-        return (hf @ self.lm_head).float().view(-1)
+        return self._logits(h)
+
+    def _logits(self, h_last):
+        hf = self._rms(h_last, self.g_final).to(torch.bfloat16)
+        return self._mm(hf, self.lm_head).float().view(-1)
 
     def prefill(self, tokens):
         """Process a whole segment of tokens at once (every token attends to the keys up to its own
@@ -179,11 +220,7 @@ class GpuStack:
         for l in range(s.n_layers):
             lw, ls = self.lw[l], s.layer_shape(l)
             ctx.kvd_checkpoint_residual(0, l, h, pos_t, U)
-            xb = self._rms(h, lw["gamma_in"]).to(torch.bfloat16)
-            q = (xb @ lw["w_q"]).float().view(U, s.n_q_heads, s.d_head)
-            if s.qk_norm:
-                q = q * torch.rsqrt(q.pow(2).mean(-1, keepdim=True) + s.rms_eps) * lw["gamma_q"].float()
-            q = self._rope_q(q, positions, ls.rope_theta).to(torch.bfloat16).contiguous()
+            q = self._queries(l, h, positions)
             kl, vl = self.k_live[l], self.v_live[l]
             ctx.kvd_recompute_kv(l, h, pos_t, U, kl[p0:], vl[p0:], self.kdim)
             lo_min = 0 if ls.sliding_window == 0 else max(0, p0 - ls.sliding_window + 1)
@@ -200,15 +237,11 @@ class GpuStack:
             for b0 in range(0, U, 64):
                 nb = min(64, U - b0)
                 ctx.kvd_decode_attention(l, nb, q[b0:], positions[b0:b0 + nb], [segs] * nb, 0.0, out[b0:])
-            h = (h.float() + (out.view(U, -1) @ lw["w_o"]).float()).to(torch.bfloat16)
-            xm = self._rms(h, lw["gamma_mlp"]).to(torch.bfloat16)
-            mlp = (self._act((xm @ lw["w_gate"]).float()) * (xm @ lw["w_up"]).float()).to(torch.bfloat16) @ lw["w_down"]
-            h = (h.float() + mlp.float()).to(torch.bfloat16)
+            h = self._after_attention(l, h, out)
             if self.policy == "kvdirect":
                 self.win_first[l] = max(self.win_first[l], p0 + U - self.budget)
         self.t += U
-        hf = self._rms(h[-1:], self.g_final).to(torch.bfloat16)
-        return (hf @ self.lm_head).float().view(-1)
+        return self._logits(h[-1:])
 
     def generate(self, prompt, n_new, forced=None):
         logits = None
@@ -233,3 +266,72 @@ class GpuStack:
                 "checkpoint_bytes_per_layer_rows": self.ctx.kvd_memory_stats()["checkpoint_bytes_used"],
                 "eq28_bytes": 2 * min(B, T) * s.n_layers * s.n_kv_heads * s.d_head * 2 + max(T - B, 0) * s.d_hidden * 2,
                 "full_cache_bytes": s.n_layers * T * kv_tok}
+
+
+class GpuStackChained(GpuStack):
+    """One checkpointed residual row per token (the row entering layer 0) and a window of B live K/V
+    entries per layer.  Every call carries the evicted prefix [0, first live position) through the
+    layers again next to the new tokens: at layer l the K/V of the evicted tokens are recomputed from
+    their current rows (the same kvd_recompute_kv as ever), serve the new tokens' attention and the
+    evicted tokens' own causal attention, and are dropped when the rows move on to layer l + 1."""
+
+    def __init__(self, stack, weights, budget=0, max_tokens=512, device_weights=False, exact_scaffold=True):
+        super().__init__(stack, weights, policy="kvdirect", budget=budget, max_tokens=max_tokens,
+                         device_weights=device_weights, exact_scaffold=exact_scaffold, layers_stored=1)
+        # the layer-0 rows as the library stores them (documented arena layout)
+        self.rows0 = self.arena[:max_tokens * stack.d_hidden * 2].view(torch.bfloat16).view(max_tokens, stack.d_hidden)
+        self.replayed_rows = 0
+
+    def step(self, token):
+        return self.prefill([int(token)])
+
+    def prefill(self, tokens):
+        s, ctx = self.s, self.ctx
+        U, p0 = len(tokens), self.t
+        assert p0 + U <= self.max_tokens
+        tok = torch.tensor(tokens, dtype=torch.long, device="cuda")
+        h_new = self.embed[tok].clone()
+        pos_new = list(range(p0, p0 + U))
+        pos_new_t = torch.arange(p0, p0 + U, dtype=torch.int32, device="cuda")
+        ctx.kvd_checkpoint_residual(0, 0, h_new, pos_new_t, U)  # STORE_RESIDUAL: one row per token
+        N = min(self.win_first[0], p0)  # evicted prefix [0, N); the windows of all layers move together
+        h_old = self.rows0[:N].clone() if N > 0 else None
+        pos_old = list(range(N))
+        pos_old_t = torch.arange(N, dtype=torch.int32, device="cuda")
+        for l in range(s.n_layers):
+            ls = s.layer_shape(l)
+            kl, vl = self.k_live[l], self.v_live[l]
+            ctx.kvd_recompute_kv(l, h_new, pos_new_t, U, kl[p0:], vl[p0:], self.kdim)
+            segs_new = []
+            if N > 0:
+                # RECOMPUTE_KV for the evicted tokens from their rows as they enter this layer
+                ctx.kvd_recompute_kv(l, h_old, pos_old_t, N, self.k_old, self.v_old, self.kdim)
+                self.recomputed_rows += N
+                segs_new.append((self.k_old, self.v_old, self.kdim, 0, N))
+            segs_new.append((kl[N:], vl[N:], self.kdim, N, p0 + U - N))
+            q_new = self._queries(l, h_new, pos_new)
+            out_new = torch.empty((U, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
+            for b0 in range(0, U, 64):
+                nb = min(64, U - b0)
+                ctx.kvd_decode_attention(l, nb, q_new[b0:], pos_new[b0:b0 + nb], [segs_new] * nb, 0.0, out_new[b0:])
+            if N > 0 and l + 1 < s.n_layers:
+                # the evicted tokens' own step through this layer: each attends to the evicted keys up
+                # to its own position (the position mask does the rest)
+                q_old = self._queries(l, h_old, pos_old)
+                out_old = torch.empty((N, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
+                segs_old = [(self.k_old, self.v_old, self.kdim, 0, N)]
+                for b0 in range(0, N, 64):
+                    nb = min(64, N - b0)
+                    ctx.kvd_decode_attention(l, nb, q_old[b0:], pos_old[b0:b0 + nb], [segs_old] * nb, 0.0, out_old[b0:])
+                h_old = self._after_attention(l, h_old, out_old)
+                self.replayed_rows += N
+            h_new = self._after_attention(l, h_new, out_new)
+        for l in range(s.n_layers):
+            self.win_first[l] = max(self.win_first[l], p0 + U - self.budget)
+        self.t += U
+        return self._logits(h_new[-1:])
+
+    def memory_report(self):
+        rep = super().memory_report()
+        rep["checkpoint_bytes_single_row"] = rep.pop("checkpoint_bytes_per_layer_rows")
+        return rep

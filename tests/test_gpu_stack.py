@@ -12,7 +12,7 @@ import torch
 
 from kvd_synth import S_GEMMA, S_QWEN, S_SMOL, bf16_to_f64, make_stack_weights, make_token_ids
 from oracle.stack import OracleStack, weights_to_f64
-from stack_harness import GpuStack
+from stack_harness import GpuStack, GpuStackChained
 
 pytestmark = pytest.mark.gpu
 
@@ -68,3 +68,41 @@ def test_multi_turn_session_matches_and_bounds_live_kv():
         assert r["kvdirect_live_kv_bytes"] <= stack.n_layers * 16 * kv_tok
         assert r["full_cache_kv_bytes"] == stack.n_layers * r["tokens_so_far"] * kv_tok
     assert recs[-1]["rows_recomputed_so_far"] > 0
+
+
+@pytest.mark.parametrize("stack,ctx_len", [(S_GEMMA, 72), (S_QWEN, 48), (S_SMOL, 48)], ids=lambda x: getattr(x, "name", x))
+def test_single_checkpoint_chained_recompute_is_token_and_bit_identical_to_full_cache(stack, ctx_len):
+    """One checkpointed row per token: each step the evicted prefix is carried through all layers
+    again (prompt prefilled in two segments, then 16 greedy tokens).  Tokens and logits must equal the
+    full-cache run bit for bit, and the checkpoint memory is Eq. 24's d_hidden * b per token."""
+    w = make_stack_weights(stack)
+    prompt = make_token_ids(ctx_len, stack.vocab, seed=4).tolist()
+    cut = ctx_len // 3
+
+    def run(m):
+        m.prefill(prompt[:cut])
+        logits = m.prefill(prompt[cut:])
+        toks, lgs = [], []
+        for i in range(16):
+            nxt = int(torch.argmax(logits).item())
+            toks.append(nxt)
+            lgs.append(logits.clone())
+            if i + 1 < 16:
+                logits = m.step(nxt)
+        assert m.ctx.kvd_poll_status() == 0
+        return toks, lgs
+
+    ref_tokens, ref_logits = run(GpuStack(stack, w, "full", exact_scaffold=True))
+    assert len(set(ref_tokens)) > 2, "degenerate generation would prove nothing"
+    for B in (0, 8, 40):
+        m = GpuStackChained(stack, w, budget=B)
+        toks, logits = run(m)
+        assert toks == ref_tokens, f"budget {B}"
+        for a, b in zip(logits, ref_logits):
+            assert torch.equal(a, b), f"budget {B}: logits differ"
+        assert m.replayed_rows > 0 and m.recomputed_rows > 0
+        rep = m.memory_report()
+        assert rep["checkpoint_bytes_single_row"] == m.t * (stack.d_hidden * 2 + 4)
+        assert rep["live_kv_bytes"] == stack.n_layers * min(B, m.t) * 2 * stack.n_kv_heads * stack.d_head * 2
+        # Eq. 28 with b = 2 bytes: B tokens of K/V plus one residual row per evicted token
+        assert rep["eq28_bytes"] == rep["live_kv_bytes"] + max(m.t - B, 0) * stack.d_hidden * 2

@@ -77,6 +77,30 @@ def test_greedy_tokens_identical_at_every_budget(stack, ctx):
             assert np.array_equal(a, b), f"budget {B}: logits differ"
 
 
+@pytest.mark.parametrize("stack,ctx", [(S_GEMMA, 40), (S_QWEN, 32), (S_SMOL, 32)], ids=lambda x: getattr(x, "name", x))
+def test_single_checkpoint_chained_recompute_is_exact(stack, ctx):
+    """One checkpointed row per token (Eq. 24's d_hidden * b bytes): carrying the evicted tokens
+    through the layers again every step reproduces the full-cache logits bit for bit (Prop. 3.2
+    applied layer after layer), and what is held matches Eq. 28."""
+    w = _weights(stack)
+    prompt = make_token_ids(ctx, stack.vocab, seed=2).tolist()
+    ref_tokens, ref_logits = OracleStack(stack, w, "full").generate(prompt, 12)
+    assert len(set(ref_tokens)) > 2
+    for B in (0, 8):
+        m = OracleStack(stack, w, "chained", B)
+        toks, logits = m.generate(prompt, 12)
+        assert toks == ref_tokens, f"budget {B}"
+        for a, b in zip(logits, ref_logits):
+            assert np.array_equal(a, b), f"budget {B}: logits differ"
+        assert m.replayed_rows > 0
+        T = m.t
+        assert len(m.rows0) == T and all(len(st.rows) == 0 for st in m.layers)
+        assert all(len(st.win_k) == min(B, T) for st in m.layers)
+        held = (len(m.rows0) - min(B, T)) * stack.d_hidden * 2 + \
+            sum(len(st.win_k) for st in m.layers) * 2 * stack.n_kv_heads * stack.d_head * 2
+        assert held == cost_model.total_memory(T, B, stack.n_layers, stack.n_kv_heads, stack.d_head, stack.d_hidden)
+
+
 def test_window_without_recompute_is_not_lossless():
     # the comparison the paper draws (Section 5.6): dropping evicted tokens changes the output
     stack = S_QWEN
