@@ -222,7 +222,8 @@ kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, const void *
  *     kvd_decode_attention; sliding_window is the layer's window (0 = global).
  *   - The result is bit-identical to kvd_decode_attention on the same inputs.
  *   - Limits: batch <= 64 and batch * n_kv_heads <= 1024; the partials of all sequences together
- *     (up to about 148 / n_kv_heads chunks per sequence and KV head, n_q_heads * (d_head + 2) floats each) must fit
+ *     (at most 130 chunks per sequence and KV head up to 8192 visible keys, about 592 / n_kv_heads
+ *     beyond, n_q_heads * (d_head + 2) floats each) must fit
  *     the array.  A request beyond that returns KVD_ERR_CAPACITY and launches nothing.
  *   - It calls no cudaMalloc / cudaFree and no library routine that allocates.  The first call on a
  *     device looks up the array's device address (cudaGetSymbolAddress) with that device current;

@@ -7,9 +7,9 @@
 // from the same loads.  Scores of 8 keys at a time are reduced across the lanes of a key with a
 // transposing shuffle butterfly, the softmax runs online in base 2, and each CTA writes one partial
 // (max, sum, unnormalised output) per query head.  A second, small kernel merges each head group's
-// partials in chunk order and writes the output.  CTAs are 16 warps (one per SM): a long sequence
-// then yields only 148 / n_kv partials per head, few enough for a single merge level that costs
-// one round trip to the L2.
+// partials in chunk order and writes the output.  Streaming CTAs are four warps, four per SM: the
+// CTAs of an SM overlap each other's start-up and combine phases, which matters in batched launches
+// of many waves.
 //
 // Which chunk, warp, lane group and slot a key lands in is a function of its position only, and the
 // merge runs in chunk order, so the output bits do not depend on how the keys are spread over
@@ -282,8 +282,8 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM) kvd_attn_split_ker
     if (__any_sync(0xffffffffu, vmask != 0u)) compute(kr, vr, vmask);
   };
 
-  // One buffer of loads per iteration; latency is hidden by the other 15 warps of the CTA (the
-  // kernel is capped at 128 registers so that 16 warps fit an SM), which measured faster than
+  // One buffer of loads per iteration; latency is hidden by the other 15 warps resident on the SM
+  // (the kernel is capped at 128 registers so that four CTAs fit), which measured faster than
   // register double buffering or a shared-memory ring at half the occupancy.
   {
     uint4 ka[U], va[U];

@@ -106,3 +106,80 @@ def test_single_checkpoint_chained_recompute_is_token_and_bit_identical_to_full_
         assert rep["live_kv_bytes"] == stack.n_layers * min(B, m.t) * 2 * stack.n_kv_heads * stack.d_head * 2
         # Eq. 28 with b = 2 bytes: B tokens of K/V plus one residual row per evicted token
         assert rep["eq28_bytes"] == rep["live_kv_bytes"] + max(m.t - B, 0) * stack.d_hidden * 2
+
+
+@pytest.mark.parametrize("stack", [S_GEMMA, S_QWEN, S_SMOL], ids=lambda x: x.name)
+def test_reconstruction_is_bit_exact_at_every_length(stack):
+    """Section 5.1 on the GPU (random-init stacks): K/V captured while a cached forward pass runs
+    equal, bit for bit, K/V rebuilt afterwards from the checkpointed residual rows, at sequence
+    lengths 16 ... 256 and in every layer (max |dK| = max |dV| = 0)."""
+    w = make_stack_weights(stack)
+    kdim = stack.n_kv_heads * stack.d_head
+    for length in (16, 32, 64, 128, 256):
+        prompt = make_token_ids(length, stack.vocab, seed=10 + length).tolist()
+        m = GpuStack(stack, w, "full", max_tokens=264)
+        # the first half at once, the rest token by token: cached K/V come from launches of different sizes
+        m.prefill(prompt[:length // 2])
+        for tok in prompt[length // 2:]:
+            m.step(tok)
+        for l in range(stack.n_layers):
+            k = torch.empty((length, kdim), dtype=torch.bfloat16, device="cuda")
+            v = torch.empty_like(k)
+            m.ctx.kvd_recompute_kv(l, None, None, length, k, v, kdim, seq=0, first_row=0)
+            assert torch.equal(k, m.k_live[l][:length]) and torch.equal(v, m.v_live[l][:length]), (length, l)
+        assert m.ctx.kvd_poll_status() == 0
+        m.ctx.close()
+
+
+def test_residual_rows_determine_the_output():
+    """The residual-patching check (Section 5.4) in KV-Direct terms: a model that holds no K/V at all
+    (B = 0) and whose checkpointed rows from layer l on are replaced by a donor's continues exactly as
+    the donor does from that layer -- given the donor's row entering layer l for the next token, the
+    patched recipient's logits equal the donor's bit for bit."""
+    stack = S_GEMMA
+    w = make_stack_weights(stack)
+    donor_prompt = make_token_ids(40, stack.vocab, seed=21).tolist()
+    recip_prompt = make_token_ids(40, stack.vocab, seed=22).tolist()
+    donor = GpuStack(stack, w, "kvdirect", 0, max_tokens=64)
+    recip = GpuStack(stack, w, "kvdirect", 0, max_tokens=64)
+    donor.prefill(donor_prompt)
+    recip.prefill(recip_prompt)
+    nxt = 7
+    ref = donor.step(nxt)
+    plain = recip.step(nxt)
+    assert not torch.equal(ref, plain)
+    # patch: from layer l on the recipient's rows (all positions, including the token just processed)
+    # become the donor's; both arenas share one layout
+    l0 = 2
+    rows_per_layer = 64 * stack.d_hidden * 2
+    recip.arena[l0 * rows_per_layer:stack.n_layers * rows_per_layer].copy_(
+        donor.arena[l0 * rows_per_layer:stack.n_layers * rows_per_layer])
+    # the next token: take the donor's row entering layer l0 and run layers l0.. on the recipient
+    tok2 = 11
+    h_d, out_d = _step_from_layer(donor, tok2, 0, None)
+    rows_entering = h_d  # rows entering each layer on the donor
+    _, out_r = _step_from_layer(recip, tok2, l0, rows_entering[l0])
+    assert torch.equal(out_d, out_r)
+
+
+def _step_from_layer(m, token, first_layer, h_in):
+    """One decoding step of a B = 0 model starting at `first_layer` with residual row `h_in` (or from
+    the embedding when first_layer is 0).  Returns (rows entering each layer, logits)."""
+    s, ctx, pos = m.s, m.ctx, m.t
+    h = m.embed[token].clone().view(1, -1) if first_layer == 0 else h_in.clone()
+    pos_t = torch.tensor([pos], dtype=torch.int32, device="cuda")
+    entering = {}
+    for l in range(first_layer, s.n_layers):
+        entering[l] = h.clone()
+        ls = s.layer_shape(l)
+        q = m._queries(l, h, [pos])
+        lo = 0 if ls.sliding_window == 0 else max(0, pos - ls.sliding_window + 1)
+        kc = torch.empty((1, m.kdim), dtype=torch.bfloat16, device="cuda")
+        vc = torch.empty_like(kc)
+        n = pos - lo
+        ctx.kvd_recompute_kv_step(l, [(0, lo, n, m.k_old, m.v_old)], h, pos_t, 1, kc, vc, m.kdim)
+        out = torch.empty((1, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
+        ctx.kvd_decode_attention(l, 1, q, [pos], [[(m.k_old, m.v_old, m.kdim, lo, n), (kc, vc, m.kdim, pos, 1)]], 0.0, out)
+        h = m._after_attention(l, h, out)
+    assert ctx.kvd_poll_status() == 0
+    return entering, m._logits(h)
