@@ -32,6 +32,12 @@
  *     are recorded in a device status word that kvd_poll_status reads.
  *   - bf16 everywhere a tensor is stored; fp32 accumulation and fp32 epilogue arithmetic.
  *   - There is no CPU fallback: without a CUDA device of compute capability 10.x kvd_create fails.
+ *   - Kernels after the first of a call sequence are launched as programmatic dependents of their
+ *     predecessor in the stream (their set-up overlaps its tail; they wait for its completion before
+ *     touching its results), which is transparent to callers and to stream capture.  Environment:
+ *     KVD_SERIAL_LAUNCH (bit mask: 1 recompute, 2 attention streaming, 4 attention merge) restores
+ *     plain stream ordering for those kernels; KVD_SPIN_LIMIT_MS (read by kvd_create) bounds every
+ *     in-kernel pipeline wait (default 2000 ms).
  */
 #ifndef KVD_H_
 #define KVD_H_
