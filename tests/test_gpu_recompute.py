@@ -293,6 +293,50 @@ def test_step_call_with_64_sequences():
         assert torch.equal(k, ranges[s][3]) and torch.equal(v, ranges[s][4])
 
 
+def test_step_sequence_in_a_cuda_graph_on_a_side_stream_matches_eager():
+    """checkpoint -> recompute (store range + new token) -> attention, captured into a CUDA graph on a
+    non-default stream (the kernels are programmatic dependents of one another) and replayed several
+    times, gives the bits of the eager sequence on the default stream."""
+    shape = GEMMA3_4B_GLOBAL
+    T = 600
+    ctx, w = open_layer(shape, max_tokens=1024, max_seqs=2, with_store=True)
+    kdim = shape.n_kv_heads * shape.d_head
+    X = dev(make_residuals(shape, T + 1, seed=61, outliers=True))
+    pos = torch.arange(T + 1, dtype=torch.int32, device="cuda")
+    q = torch.randn((1, shape.n_q_heads, shape.d_head), device="cuda").to(torch.bfloat16)
+
+    def sequence(seq, K, V, out):
+        ctx.kvd_reset_sequence(seq)
+        ctx.kvd_checkpoint_residual(seq, 0, X, pos, T)
+        ctx.kvd_recompute_kv_step(0, [(seq, 0, T, K, V)], X[T:], pos[T:], 1, K[T:], V[T:], kdim)
+        ctx.kvd_decode_attention(0, 1, q, [T], [[(K, V, kdim, 0, T), (K[T:], V[T:], kdim, T, 1)]], 0.0, out)
+
+    def buffers():
+        return (torch.zeros((T + 1, kdim), dtype=torch.bfloat16, device="cuda"),
+                torch.zeros((T + 1, kdim), dtype=torch.bfloat16, device="cuda"),
+                torch.zeros((1, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda"))
+
+    K0, V0, o0 = buffers()
+    sequence(0, K0, V0, o0)
+    torch.cuda.synchronize()
+    K1, V1, o1 = buffers()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        sequence(1, K1, V1, o1)  # warm-up on the capture stream
+    side.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        sequence(1, K1, V1, o1)
+    for _ in range(3):
+        K1.zero_(); V1.zero_(); o1.zero_()
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(K1, K0) and torch.equal(V1, V0) and torch.equal(o1, o0)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+
+
 def test_argument_errors_and_position_flag():
     shape = TINY_GQA
     ctx, w = open_layer(shape, max_tokens=1024)
