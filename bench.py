@@ -810,6 +810,65 @@ def run_stack_configs(args):
     print(json.dumps({"stack_configs": result}), flush=True)
 
 
+def run_profile_qwen(args):
+    """A few eager launches of the Qwen3-4B-shaped layer's kernels for a profiler (a reduced form of
+    the long-context configuration: 16384 recomputed rows, decode attention over 2 x 16385 keys in
+    recomputed + window + current segments, 268 MB of K and V): no graphs, no measurements."""
+    import torch
+    import paper_2603_19664_b200 as kvd
+    from kvd_synth import QWEN3_4B as shape, make_layer_weights
+    from paper_2603_19664_b200.build import build
+    build()
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+
+    def dev(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+    batch, ctx_len, budget = 2, 16384, 512
+    kdim = shape.n_kv_heads * shape.d_head
+    w = make_layer_weights(shape)
+    desc = kvd.make_desc(1, shape.d_hidden, shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.rms_eps,
+                         shape.qk_norm, shape.rms_eps, shape.rope_style, batch, ctx_len + 8, batch)
+    c = kvd.Kvd(desc)
+    tw, tg, tk = dev(w.w_kv), dev(w.gamma_in), dev(w.gamma_k)
+    c.kvd_set_layer(0, tw, tg, tk, shape.rope_theta, 0)
+    ws = torch.empty(kvd.kvd_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+    c.kvd_attach_workspace(ws)
+    arena = torch.empty(kvd.kvd_store_bytes(desc, 1), dtype=torch.uint8, device="cuda")
+    c.kvd_attach_store(arena, 1)
+    xs = torch.randn((ctx_len, shape.d_hidden), device="cuda").to(torch.bfloat16)
+    ps = torch.arange(ctx_len, device="cuda", dtype=torch.int32)
+    for b in range(batch):
+        c.kvd_checkpoint_residual(b, 0, xs, ps, ctx_len)
+    n_old = ctx_len - budget
+    Ko = torch.empty((batch * n_old, kdim), device="cuda", dtype=torch.bfloat16)
+    Vo = torch.empty_like(Ko)
+    n_sets = 3
+    Kf = [torch.randn((batch, ctx_len + 1, kdim), device="cuda").to(torch.bfloat16) for _ in range(n_sets)]
+    Vf = [torch.randn((batch, ctx_len + 1, kdim), device="cuda").to(torch.bfloat16) for _ in range(n_sets)]
+    xc = torch.randn((batch, shape.d_hidden), device="cuda").to(torch.bfloat16)
+    pc = torch.full((batch,), ctx_len, device="cuda", dtype=torch.int32)
+    kc = torch.empty((batch, kdim), device="cuda", dtype=torch.bfloat16)
+    vc = torch.empty_like(kc)
+    q = torch.randn((batch, shape.n_q_heads, shape.d_head), device="cuda").to(torch.bfloat16)
+    out = torch.empty_like(q)
+    ranges = [(b, 0, n_old, Ko[b * n_old:], Vo[b * n_old:]) for b in range(batch)]
+    for i in range(max(args.steps, 1) + 2):
+        s = i % n_sets
+        c.kvd_recompute_kv_step(0, ranges, xc, pc, batch, kc, vc, kdim)
+        segs = [[(Ko[b * n_old:], Vo[b * n_old:], kdim, 0, n_old),
+                 (Kf[s][b, n_old:], Vf[s][b, n_old:], kdim, n_old, budget), (kc[b:], vc[b:], kdim, ctx_len, 1)]
+                for b in range(batch)]
+        c.kvd_decode_attention(0, batch, q, [ctx_len] * batch, segs, 0.0, out)
+        # the same keys from one stored segment (the cached-KV read)
+        c.kvd_decode_attention(0, batch, q, [ctx_len] * batch,
+                               [[(Kf[s][b], Vf[s][b], kdim, 0, ctx_len + 1)] for b in range(batch)], 0.0, out)
+    torch.cuda.synchronize()
+    assert c.kvd_poll_status() == kvd.KVD_OK
+    print(json.dumps({"profile_run": "qwen3-4b layer", "rows_recomputed": batch * n_old, "keys": batch * (ctx_len + 1),
+                      "launches": c.kvd_launch_count()}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -821,11 +880,15 @@ def main():
     ap.add_argument("--profile", action="store_true", help="eager launches only, for a run under a profiler")
     ap.add_argument("--profile-long-attn", action="store_true",
                     help="with --profile: also run decode attention over 32769 keys a few times")
+    ap.add_argument("--profile-qwen", action="store_true",
+                    help="eager launches of the Qwen3-4B-shaped layer's kernels (reduced long-context case) for a profiler")
     ap.add_argument("--stack-configs", action="store_true",
                     help="time the hot path of the stack-shaped configurations instead of the contract line")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.profile_qwen:
+        run_profile_qwen(args)
     elif args.stack_configs:
         run_stack_configs(args)
     else:
