@@ -1,0 +1,90 @@
+"""The long-context configuration at full size, in the launch shapes bench.py --stack-configs times:
+Qwen3-4B-shaped layer, batch 8, context 32768, 512 live K/V entries per sequence.
+
+One kvd_recompute_kv_step launch rebuilds 8 x 32256 evicted rows from the residual store together with
+the 8 new tokens; one kvd_decode_attention call attends over recomputed + window + current segments.
+The oracle checks sampled rows of K/V (first/last rows of tiles, a random sample, several sequences)
+and the attention output of two sequences computed from the keys the GPU produced.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2603_19664_b200 as kvd
+from kvd_synth import QWEN3_4B, bf16_to_f64, make_query, make_residuals
+from gpu_util import dev, host_f64, kv_errors, open_layer, oracle_kv
+
+pytestmark = pytest.mark.gpu
+
+
+def test_config4_full_size_sampled():
+    shape, batch, ctx_len, budget = QWEN3_4B, 8, 32768, 512
+    kdim = shape.n_kv_heads * shape.d_head
+    n_old = ctx_len - budget
+    ctx, w = open_layer(shape, max_tokens=ctx_len + 8, max_batch=batch, max_seqs=batch, with_store=True)
+    X = make_residuals(shape, ctx_len + batch, seed=44)  # the context rows, then one new row per sequence
+    x = dev(X)
+    pos = torch.arange(ctx_len, dtype=torch.int32, device="cuda")
+    for b in range(batch):
+        # every sequence checkpoints the same rows shifted by b, so that sequences differ
+        ctx.kvd_checkpoint_residual(b, 0, torch.roll(x[:ctx_len], shifts=-b, dims=0).contiguous(), pos, ctx_len)
+    Ko = torch.zeros((batch * n_old, kdim), dtype=torch.bfloat16, device="cuda")
+    Vo = torch.zeros_like(Ko)
+    kc = torch.zeros((batch, kdim), dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    pc = torch.full((batch,), ctx_len, dtype=torch.int32, device="cuda")
+    ranges = [(b, 0, n_old, Ko[b * n_old:], Vo[b * n_old:]) for b in range(batch)]
+    launches = ctx.kvd_launch_count()
+    ctx.kvd_recompute_kv_step(0, ranges, x[ctx_len:], pc, batch, kc, vc, kdim)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    assert ctx.kvd_launch_count() == launches + 1
+
+    # ---- K/V of sampled rows against the oracle
+    rng = np.random.default_rng(4)
+    for b in (0, 3, 7):
+        rows = np.unique(np.concatenate([[0, 1, 255, 256, 257, n_old - 257, n_old - 256, n_old - 1],
+                                         rng.choice(n_old, 40, replace=False)]))
+        src = (rows + b) % ctx_len  # the roll above
+        Kr, Vr = oracle_kv(shape, w, X[src], rows)
+        got_k = host_f64(Ko[b * n_old:(b + 1) * n_old][torch.from_numpy(rows).cuda()])
+        got_v = host_f64(Vo[b * n_old:(b + 1) * n_old][torch.from_numpy(rows).cuda()])
+        for name, g, r in (("K", got_k, Kr.reshape(len(rows), kdim)), ("V", got_v, Vr.reshape(len(rows), kdim))):
+            mx, rel = kv_errors(g, r)
+            assert mx <= 2e-2 and rel <= 1e-2, (b, name, mx, rel)
+    Kr, Vr = oracle_kv(shape, w, X[ctx_len:], np.full(batch, ctx_len))
+    for name, g, r in (("K", host_f64(kc), Kr.reshape(batch, kdim)), ("V", host_f64(vc), Vr.reshape(batch, kdim))):
+        mx, rel = kv_errors(g, r)
+        assert mx <= 2e-2 and rel <= 1e-2, ("current", name, mx, rel)
+
+    # ---- attention over recomputed + window + current segments (all 8 sequences in one call)
+    Kw = torch.randn((batch, budget, kdim), device="cuda").to(torch.bfloat16)
+    Vw = torch.randn((batch, budget, kdim), device="cuda").to(torch.bfloat16)
+    q_bits = make_query(shape, batch, seed=45)
+    q = dev(q_bits)
+    out = torch.zeros((batch, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda")
+    segs = [[(Ko[b * n_old:], Vo[b * n_old:], kdim, 0, n_old), (Kw[b], Vw[b], kdim, n_old, budget),
+             (kc[b:], vc[b:], kdim, ctx_len, 1)] for b in range(batch)]
+    ctx.kvd_decode_attention(0, batch, q, [ctx_len] * batch, segs, 0.0, out)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    for b in (0, 7):
+        def f64(t):
+            return host_f64(t).reshape(-1, shape.n_kv_heads, shape.d_head)
+        ref = oracle.decode_attention(bf16_to_f64(q_bits[b]).reshape(shape.n_q_heads, shape.d_head), ctx_len,
+                                      [(f64(Ko[b * n_old:(b + 1) * n_old]), f64(Vo[b * n_old:(b + 1) * n_old]), 0),
+                                       (f64(Kw[b]), f64(Vw[b]), n_old), (f64(kc[b:b + 1]), f64(vc[b:b + 1]), ctx_len)],
+                                      1.0 / math.sqrt(shape.d_head), 0)
+        got = host_f64(out[b]).reshape(ref.shape)
+        d = got - ref
+        assert np.linalg.norm(d) <= 1e-2 * np.linalg.norm(ref)
+        assert np.max(np.abs(d)) <= 1e-2 * np.max(np.abs(ref))
+    # the same keys from one stored segment per sequence give the same bits
+    Kfull = torch.cat([Ko.view(batch, n_old, kdim), Kw, kc.view(batch, 1, kdim)], dim=1).contiguous()
+    Vfull = torch.cat([Vo.view(batch, n_old, kdim), Vw, vc.view(batch, 1, kdim)], dim=1).contiguous()
+    out1 = torch.zeros_like(out)
+    ctx.kvd_decode_attention(0, batch, q, [ctx_len] * batch,
+                             [[(Kfull[b], Vfull[b], kdim, 0, ctx_len + 1)] for b in range(batch)], 0.0, out1)
+    assert torch.equal(out, out1)
+    ctx.close()
