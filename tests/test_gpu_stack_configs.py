@@ -1,4 +1,6 @@
-"""The long-context configuration at full size, in the launch shapes bench.py --stack-configs times:
+"""The stack-shaped configurations at full size, in the launch shapes bench.py --stack-configs times.
+
+Long context:
 Qwen3-4B-shaped layer, batch 8, context 32768, 512 live K/V entries per sequence.
 
 One kvd_recompute_kv_step launch rebuilds 8 x 32256 evicted rows from the residual store together with
@@ -87,4 +89,63 @@ def test_config4_full_size_sampled():
     ctx.kvd_decode_attention(0, batch, q, [ctx_len] * batch,
                              [[(Kfull[b], Vfull[b], kdim, 0, ctx_len + 1)] for b in range(batch)], 0.0, out1)
     assert torch.equal(out, out1)
+    ctx.close()
+
+
+@pytest.mark.parametrize("local", [False, True], ids=["global-layer", "local-layer"])
+def test_config3_batch64_full_size_sampled(local):
+    """The batched decode step of the 34-layer stack configuration at its largest batch: 64 sequences,
+    context 2048, 256 live K/V entries; one recompute launch for the 64 evicted ranges and the 64 new
+    tokens, one attention call over recomputed + window + current segments."""
+    from kvd_synth import GEMMA3_4B_GLOBAL, GEMMA3_4B_LOCAL
+    shape = GEMMA3_4B_LOCAL if local else GEMMA3_4B_GLOBAL
+    batch, ctx_len, budget = 64, 2048, 256
+    kdim = shape.n_kv_heads * shape.d_head
+    lo = 0 if shape.sliding_window == 0 else ctx_len - shape.sliding_window + 1
+    n_old = ctx_len - budget - lo
+    ctx, w = open_layer(shape, max_tokens=ctx_len + 8, max_batch=batch, max_seqs=batch, with_store=True)
+    X = make_residuals(shape, ctx_len + batch, seed=46, outliers=True)
+    x = dev(X)
+    pos = torch.arange(ctx_len, dtype=torch.int32, device="cuda")
+    for b in range(batch):
+        ctx.kvd_checkpoint_residual(b, 0, torch.roll(x[:ctx_len], shifts=-b, dims=0).contiguous(), pos, ctx_len)
+    Ko = torch.zeros((batch * n_old, kdim), dtype=torch.bfloat16, device="cuda")
+    Vo = torch.zeros_like(Ko)
+    kc = torch.zeros((batch, kdim), dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    pc = torch.full((batch,), ctx_len, dtype=torch.int32, device="cuda")
+    ranges = [(b, lo, n_old, Ko[b * n_old:], Vo[b * n_old:]) for b in range(batch)]
+    ctx.kvd_recompute_kv_step(0, ranges, x[ctx_len:], pc, batch, kc, vc, kdim)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    rng = np.random.default_rng(5)
+    for b in (0, 31, 63):
+        rows = np.unique(np.concatenate([[0, 1, 255, 256, n_old - 1], rng.choice(n_old, 30, replace=False)]))
+        src = (rows + lo + b) % ctx_len
+        Kr, Vr = oracle_kv(shape, w, X[src], rows + lo)
+        idx = torch.from_numpy(rows).cuda()
+        for name, g, r in (("K", host_f64(Ko[b * n_old:(b + 1) * n_old][idx]), Kr.reshape(len(rows), kdim)),
+                           ("V", host_f64(Vo[b * n_old:(b + 1) * n_old][idx]), Vr.reshape(len(rows), kdim))):
+            mx, rel = kv_errors(g, r)
+            assert mx <= 2e-2 and rel <= 1e-2, (b, name, mx, rel)
+    wf = ctx_len - budget
+    Kw = torch.randn((batch, budget, kdim), device="cuda").to(torch.bfloat16)
+    Vw = torch.randn((batch, budget, kdim), device="cuda").to(torch.bfloat16)
+    q_bits = make_query(shape, batch, seed=47)
+    q = dev(q_bits)
+    out = torch.zeros((batch, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda")
+    segs = [[(Ko[b * n_old:], Vo[b * n_old:], kdim, lo, n_old), (Kw[b], Vw[b], kdim, wf, budget),
+             (kc[b:], vc[b:], kdim, ctx_len, 1)] for b in range(batch)]
+    ctx.kvd_decode_attention(0, batch, q, [ctx_len] * batch, segs, 0.0, out)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+
+    def f64(t):
+        return host_f64(t).reshape(-1, shape.n_kv_heads, shape.d_head)
+    for b in (0, 17, 63):
+        ref = oracle.decode_attention(bf16_to_f64(q_bits[b]).reshape(shape.n_q_heads, shape.d_head), ctx_len,
+                                      [(f64(Ko[b * n_old:(b + 1) * n_old]), f64(Vo[b * n_old:(b + 1) * n_old]), lo),
+                                       (f64(Kw[b]), f64(Vw[b]), wf), (f64(kc[b:b + 1]), f64(vc[b:b + 1]), ctx_len)],
+                                      1.0 / math.sqrt(shape.d_head), shape.sliding_window)
+        d = host_f64(out[b]).reshape(ref.shape) - ref
+        assert np.linalg.norm(d) <= 1e-2 * np.linalg.norm(ref)
+        assert np.max(np.abs(d)) <= 1e-2 * np.max(np.abs(ref))
     ctx.close()
