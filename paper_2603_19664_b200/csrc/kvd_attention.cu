@@ -30,29 +30,6 @@ __device__ __forceinline__ uint4 ldg_stream(const void *p) {
   return r;
 }
 
-// Packed pairs of fp32 (sm_100 has two-wide fp32 FMA): halves the FMA count of the dot products and
-// of the weighted sum.
-__device__ __forceinline__ uint64_t pack2(float a, float b) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
-  return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float &a, float &b) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
-}
-__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-// the two bf16 halves of a 32-bit word as a packed pair of fp32
-__device__ __forceinline__ uint64_t bf16x2_to_f32x2(uint32_t w) { return pack2(bf16_lo(w), bf16_hi(w)); }
-
 // Sum each of the 8 values over the LPK lanes of a group; afterwards the lane whose index bits
 // (LPK/2, LPK/4, LPK/8) spell slot u holds the total of v[u].
 template <int LPK>

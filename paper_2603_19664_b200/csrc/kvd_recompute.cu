@@ -152,23 +152,39 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int num_tiles = p.num_m_blocks * p.num_n_blocks;
-  // Tile order: all key tiles first, then all value tiles, so that the last tile of a CTA (whose
-  // epilogue nothing overlaps) is a cheap value tile.  Falls back to row-major order when a tile
-  // mixes key and value heads.
+  // Tile order.  With more tiles than clusters a cluster works through "units" of two consecutive
+  // tiles that share a row block -- the key tile and the value tile of one head column -- so that the
+  // row statistics (whose shared-memory reads compete with the tensor cores' operand fetch: 12 % of
+  // the kernel's time when taken for every tile) are taken once per unit and reused; key first, so
+  // that the last tile of a CTA, whose epilogue nothing overlaps, is a cheap value tile.  (Units of
+  // all tiles of a row block measured slower: the units are then too few to balance the clusters.)
+  // With no more tiles than clusters every tile is its own unit, all key tiles first.  Falls back to
+  // row-major single tiles when a tile mixes key and value heads.
   const int nk_tiles = (p.k_cols % BLOCK_N == 0) ? p.k_cols / BLOCK_N : 0;
-  // tile -> (job, first row of this CTA's 128 rows within the job, first fused column)
-  auto tile_coords = [&](int t, int &job, int &m0, int &n0) {
+  const int unit_tiles = (nk_tiles != 0 && num_tiles > num_clusters) ? 2 : 1;
+  const int n_units = num_tiles / unit_tiles;
+  // i-th tile of this cluster -> (job, first row of this CTA's 128 rows within the job, first fused
+  // column, whether it opens a unit); false when the cluster has no i-th tile
+  auto tile_at = [&](int i, int &job, int &m0, int &n0, bool &first) -> bool {
+    const int unit = cluster_id + (i / unit_tiles) * num_clusters, j = i % unit_tiles;
+    if (unit >= n_units) return false;
+    first = j == 0;
     int mb;
     if (nk_tiles == 0) {
-      mb = t / p.num_n_blocks;
-      n0 = (t % p.num_n_blocks) * BLOCK_N;
-    } else if (t < p.num_m_blocks * nk_tiles) {
-      mb = t / nk_tiles;
-      n0 = (t % nk_tiles) * BLOCK_N;
+      mb = unit / p.num_n_blocks;
+      n0 = (unit % p.num_n_blocks) * BLOCK_N;
+    } else if (unit_tiles == 1) {
+      if (unit < p.num_m_blocks * nk_tiles) {
+        mb = unit / nk_tiles;
+        n0 = (unit % nk_tiles) * BLOCK_N;
+      } else {
+        const int u = unit - p.num_m_blocks * nk_tiles, nv = p.num_n_blocks - nk_tiles;
+        mb = u / nv;
+        n0 = (nk_tiles + u % nv) * BLOCK_N;
+      }
     } else {
-      const int u = t - p.num_m_blocks * nk_tiles, nv = p.num_n_blocks - nk_tiles;
-      mb = u / nv;
-      n0 = (nk_tiles + u % nv) * BLOCK_N;
+      mb = unit / nk_tiles;
+      n0 = (unit % nk_tiles + (j == 0 ? 0 : nk_tiles)) * BLOCK_N;
     }
     // jobs own consecutive runs of 256-row blocks: the last job whose first block is <= mb
     int lo = 0, hi = p.n_jobs;
@@ -179,6 +195,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
     }
     job = lo;
     m0 = (mb - p.jobs[lo].mb_start) * (2 * RC_BLOCK_M) + static_cast<int>(cta_rank) * RC_BLOCK_M;
+    return true;
   };
   const unsigned long long tmo = p.timeout_ns;
 
@@ -223,10 +240,9 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
       uint32_t full = bar_full(0), empty = bar_empty(0), dst = smem_base;
       const int b_row_off = static_cast<int>(cta_rank) * Cfg::B_ROWS;
       bool ok = true;
-      int ti = 0;
-      for (int t = cluster_id; t < num_tiles && ok; t += num_clusters, ++ti) {
-        int job, m0, n0;
-        tile_coords(t, job, m0, n0);
+      int job, m0, n0;
+      bool first_of_unit;
+      for (int ti = 0; ok && tile_at(ti, job, m0, n0, first_of_unit); ++ti) {
         n0 += b_row_off;
         // rows come from a slab of the residual store or from the caller's buffer (slab 0 of its map)
         const int slab = p.jobs[job].slab;
@@ -289,8 +305,9 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
       uint32_t ph = 0, aph = 0;
       uint32_t full = bar_full(0), peer = bar_peer_full(0), empty = bar_empty(0), a_lo = a_lo0;
       bool ok = true;
-      int ti = 0;
-      for (int t = cluster_id; t < num_tiles && ok; t += num_clusters, ++ti) {
+      int job_, m0_, n0_;
+      bool first_;
+      for (int ti = 0; ok && tile_at(ti, job_, m0_, n0_, first_); ++ti) {
         // both CTAs' epilogues have drained accumulator a
         if (!mbar_wait(bar_tmem_empty(a), aph ^ 1u, s_abort, tmo)) {
           raise(p.status, STATUS_TIMEOUT, s_abort);
@@ -300,7 +317,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
         const uint32_t d_tmem = tmem_base + a * BLOCK_N;
         long long waited = 0;
         trace_put<TRACE>(p.trace, ti, 4);
-        trace_put<TRACE>(p.trace, ti, 10, t);
+        trace_put<TRACE>(p.trace, ti, 10, (m0_ / (2 * RC_BLOCK_M)) * p.num_n_blocks + n0_ / BLOCK_N);
         for (int kb = 0; kb < p.num_k_blocks; ++kb) {
           const long long w0 = TRACE ? clock64() : 0;
           // stage s has landed here and (relayed) in the partner CTA
@@ -343,7 +360,9 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
       const uint32_t peer0 = map_to_cta(bar_peer_full(0), 0);
       uint32_t peer = peer0;
       bool ok = true;
-      for (int t = cluster_id; t < num_tiles && ok; t += num_clusters) {
+      int job_, m0_, n0_;
+      bool first_;
+      for (int ti = 0; ok && tile_at(ti, job_, m0_, n0_, first_); ++ti) {
         for (int kb = 0; kb < p.num_k_blocks; ++kb) {
           if (!mbar_wait(full, ph, s_abort, tmo)) {
             raise(p.status, STATUS_TIMEOUT, s_abort);
@@ -370,8 +389,10 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
     int s = 0, a = 0;
     uint32_t ph = 0, aph = 0;
     bool ok = true;
-    int ti = 0;
-    for (int t = cluster_id; t < num_tiles && ok; t += num_clusters, ++ti) {
+    int job_, m0_, n0_;
+    bool first_of_unit;
+    float rstd_row = 0.f;  // of this thread's row, kept for the other tiles of the unit
+    for (int ti = 0; ok && tile_at(ti, job_, m0_, n0_, first_of_unit); ++ti) {
       long long waited = 0;
       const long long st0 = TRACE ? clock64() : 0;
       // s_rstd[a] is free once the local epilogue that read it has finished with accumulator a
@@ -382,7 +403,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
       }
       // eight partial sums (one per element slot of a 16-byte chunk) keep the FMA chains short; they
       // are combined in a fixed order below, the same for every row
-      float ps[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      uint64_t ps2[4] = {0ull, 0ull, 0ull, 0ull};  // (ps0, ps1), (ps2, ps3), (ps4, ps5), (ps6, ps7): two-wide fp32 FMAs
       for (int kb = 0; kb < p.num_k_blocks; ++kb) {
         const long long w0 = TRACE ? clock64() : 0;
         if (!warp_wait(bar_full(s), ph, s_abort, tmo, lane)) {
@@ -392,6 +413,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
         }
         if (TRACE) waited += clock64() - w0;
         const uint32_t a_addr = smem_base + s * Cfg::STAGE_BYTES + row_off;
+        // (the same rows again in a later tile of the unit: only the stage hand-shake is needed)
+        if (first_of_unit) {
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
           // logical 16-byte chunk c of this row sits at chunk (c ^ (row % 8)) under the 128-byte swizzle
@@ -399,15 +422,12 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
           asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
                        : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
                        : "r"(a_addr + ((static_cast<uint32_t>(c) << 4) ^ sw)));
-          float x;
-          x = bf16_lo(w0); ps[0] = fmaf(x, x, ps[0]);
-          x = bf16_hi(w0); ps[1] = fmaf(x, x, ps[1]);
-          x = bf16_lo(w1); ps[2] = fmaf(x, x, ps[2]);
-          x = bf16_hi(w1); ps[3] = fmaf(x, x, ps[3]);
-          x = bf16_lo(w2); ps[4] = fmaf(x, x, ps[4]);
-          x = bf16_hi(w2); ps[5] = fmaf(x, x, ps[5]);
-          x = bf16_lo(w3); ps[6] = fmaf(x, x, ps[6]);
-          x = bf16_hi(w3); ps[7] = fmaf(x, x, ps[7]);
+          uint64_t x2;
+          x2 = bf16x2_to_f32x2(w0); ps2[0] = ffma2(x2, x2, ps2[0]);
+          x2 = bf16x2_to_f32x2(w1); ps2[1] = ffma2(x2, x2, ps2[1]);
+          x2 = bf16x2_to_f32x2(w2); ps2[2] = ffma2(x2, x2, ps2[2]);
+          x2 = bf16x2_to_f32x2(w3); ps2[3] = ffma2(x2, x2, ps2[3]);
+        }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_empty(s));
@@ -417,8 +437,12 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
         }
       }
       if (!ok) break;
+      float ps[8];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) unpack2(ps2[j], ps[2 * j], ps[2 * j + 1]);
       const float sum = ((ps[0] + ps[1]) + (ps[2] + ps[3])) + ((ps[4] + ps[5]) + (ps[6] + ps[7]));
-      s_rstd[a * RC_BLOCK_M + row] = 1.0f / sqrtf(sum * p.inv_d_hidden + p.rms_eps);
+      if (first_of_unit) rstd_row = 1.0f / sqrtf(sum * p.inv_d_hidden + p.rms_eps);
+      s_rstd[a * RC_BLOCK_M + row] = rstd_row;
       mbar_arrive(bar_stats_full(a));
       if (TRACE && threadIdx.x == 0) {
         trace_put<TRACE>(p.trace, ti, 8, waited);
@@ -437,10 +461,9 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
     constexpr int HALF = D_HEAD / 2;
     int a = 0;
     uint32_t aph = 0;
-    int ti = 0;
-    for (int t = cluster_id; t < num_tiles; t += num_clusters, ++ti) {
-      int job, m0, n0;
-      tile_coords(t, job, m0, n0);
+    int job, m0, n0;
+    bool first_of_unit;
+    for (int ti = 0; tile_at(ti, job, m0, n0, first_of_unit); ++ti) {
       const RcJob &J = p.jobs[job];
       // warp-uniform outcome: tcgen05.ld below is an aligned instruction
       if (!warp_wait(bar_tmem_full(a), aph, s_abort, tmo, lane) || !warp_wait(bar_stats_full(a), aph, s_abort, tmo, lane)) {
@@ -491,18 +514,27 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
           __nv_bfloat16 *dst = J.k_out + static_cast<size_t>(m) * p.out_row_stride + col0;
           float kscale = rstd;
           if (p.qk_norm) {
-            float ss = 0.f;
+            // sum of squares over the head in four chains (columns j mod 4), two-wide, combined in a
+            // fixed order: a single 256-long dependent chain would be pure latency
+            uint64_t ss2[2] = {0ull, 0ull};
+            const uint64_t rstd2 = pack2(rstd, rstd);
 #pragma unroll 1
             for (int c = 0; c < D_HEAD / 32; ++c) {
               uint32_t r[32];
               tmem_ld_x32(tcol + c * 32, r);
               tmem_wait_ld();
 #pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const float v = __uint_as_float(r[j]) * rstd;
-                ss = fmaf(v, v, ss);
+              for (int j = 0; j < 32; j += 4) {
+                const uint64_t v0 = fmul2(pack2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), rstd2);
+                const uint64_t v1 = fmul2(pack2(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])), rstd2);
+                ss2[0] = ffma2(v0, v0, ss2[0]);
+                ss2[1] = ffma2(v1, v1, ss2[1]);
               }
             }
+            float s0, s1, s2, s3;
+            unpack2(ss2[0], s0, s1);
+            unpack2(ss2[1], s2, s3);
+            const float ss = (s0 + s1) + (s2 + s3);
             kscale = rstd * (1.0f / sqrtf(ss * (1.0f / D_HEAD) + p.qk_eps));
           }
           if (p.rope_style == KVD_ROPE_INTERLEAVED) {
