@@ -157,6 +157,40 @@ def test_group_sizes_on_both_streaming_kernels(shape):
     assert torch.equal(out, out1)
 
 
+@pytest.mark.parametrize("shape", [TINY_GQA, SMOLLM2_135M, GEMMA3_4B_LOCAL, QWEN3_4B, WIDE_SHAPES[1]], ids=lambda s: s.name)
+def test_random_batches_of_random_layouts(shape):
+    """Seeded random batches: lengths from 1 to 6000, one to four segments cut at random places, some
+    with a gap or with keys beyond the query position, a random window override through the shape's own
+    window -- every sequence against the oracle, and each sequence alone gives the bits it has in the batch."""
+    rng = np.random.default_rng(1234 + shape.d_head + shape.n_q_heads)
+    ctx, _ = open_layer(shape, max_tokens=8192, max_batch=7)
+    for case in range(4):
+        batch = int(rng.integers(1, 8))
+        q = make_query(shape, batch, seed=500 + case)
+        segs, qpos = [], []
+        for b in range(batch):
+            T = int(rng.choice([1, 2, 31, 33, 200, 1025, 2500, 6000]))
+            K, V = make_kv(shape, T, seed=600 + 10 * case + b)
+            n_cuts = int(rng.integers(0, 4))
+            cuts = sorted(set(int(c) for c in rng.integers(1, T, size=n_cuts))) if T > 1 else []
+            bounds = [0] + cuts + [T]
+            gap = int(rng.integers(0, 2)) * 7  # shift everything after the first segment: a hole in the positions
+            row = []
+            for i in range(len(bounds) - 1):
+                lo, hi = bounds[i], bounds[i + 1]
+                row.append((K[lo:hi], V[lo:hi], lo + (gap if i > 0 else 0)))
+            last_pos = T - 1 + (gap if len(bounds) > 2 else 0)
+            qpos.append(max(0, last_pos - int(rng.integers(0, 3))))  # sometimes keys after the query
+            segs.append(row)
+        out = gpu_attention(ctx, shape, q, qpos, segs)
+        ref = oracle_attention(shape, q, qpos, segs)
+        for b in range(batch):
+            attn_check(host_f64(out)[b], ref[b])
+        b = int(rng.integers(0, batch))
+        alone = gpu_attention(ctx, shape, q[b:b + 1], qpos[b:b + 1], segs[b:b + 1])
+        assert torch.equal(alone[0], out[b])
+
+
 @pytest.mark.parametrize("shape", [TINY_GQA, SMOLLM2_135M, GEMMA3_4B_GLOBAL, QWEN3_4B], ids=lambda s: s.name)
 def test_segment_layout_does_not_change_the_bits(shape):
     """One stored segment (a full cache) and the same keys cut into recomputed / window / current
