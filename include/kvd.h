@@ -156,6 +156,14 @@ int kvd_rows_stored(const kvd_ctx *ctx, int layer, int seq);
 /* Bytes of attention scratch for the context's max_batch / max_tokens_per_seq. */
 size_t kvd_workspace_bytes(const kvd_model_desc *desc);
 
+/* How decode attention splits one sequence: the keys at positions first_visible .. last_visible (after
+ * the window and the query position have been applied) are cut into chunks aligned to multiples of
+ * *chunk_keys; returns the number of chunks (= partials per KV head that the call keeps in its scratch)
+ * and, if not NULL, stores the chunk length.  A function of its arguments only: the split of a sequence
+ * does not depend on the segment layout or on the rest of the batch.  Host-only; 0 on bad arguments
+ * (d_head not in {64, 128, 256}, n_kv_heads < 1, an empty or negative range). */
+int kvd_attention_split(int d_head, int n_kv_heads, int first_visible, int last_visible, int *chunk_keys);
+
 /* Hand the context a caller-owned DEVICE workspace (256-byte aligned, >= kvd_workspace_bytes). */
 kvd_status kvd_attach_workspace(kvd_ctx *ctx, void *workspace, size_t bytes);
 

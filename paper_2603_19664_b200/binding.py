@@ -31,7 +31,7 @@ KVD_MAX_SEGMENTS = 4
 # every symbol include/kvd.h declares
 EXPORTED_SYMBOLS = (
     "kvd_create", "kvd_destroy", "kvd_set_layer", "kvd_store_bytes", "kvd_attach_store", "kvd_reset_sequence",
-    "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
+    "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
     "kvd_recompute_kv_step",
     "kvd_decode_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
     "kvd_status_string", "kvd_version",
@@ -108,6 +108,8 @@ def load() -> ctypes.CDLL:
     lib.kvd_workspace_bytes.restype = sz
     lib.kvd_attach_workspace.argtypes = [vp, vp, sz]
     lib.kvd_attach_workspace.restype = i32
+    lib.kvd_attention_split.argtypes = [i32, i32, i32, i32, ctypes.POINTER(ctypes.c_int32)]
+    lib.kvd_attention_split.restype = i32
     lib.kvd_checkpoint_residual.argtypes = [vp, i32, i32, vp, vp, i32, vp]
     lib.kvd_checkpoint_residual.restype = i32
     lib.kvd_recompute_kv.argtypes = [vp, i32, vp, vp, i32, i32, i32, vp, vp, i64, vp]
@@ -161,6 +163,13 @@ def kvd_store_bytes(desc: kvd_model_desc, layers_stored: int) -> int:
 
 def kvd_workspace_bytes(desc: kvd_model_desc) -> int:
     return int(load().kvd_workspace_bytes(ctypes.byref(desc)))
+
+
+def kvd_attention_split(d_head: int, n_kv_heads: int, first_visible: int, last_visible: int) -> Tuple[int, int]:
+    """(number of chunks, keys per chunk) of one sequence's visible range; (0, 0) on bad arguments."""
+    ck = ctypes.c_int32(0)
+    n = int(load().kvd_attention_split(d_head, n_kv_heads, first_visible, last_visible, ctypes.byref(ck)))
+    return n, int(ck.value)
 
 
 def _ptr(t) -> int:

@@ -79,6 +79,15 @@ extern "C" size_t kvd_workspace_bytes(const kvd_model_desc *d) {
   return round_up(parts * d->n_q_heads * d->d_head * 4, 256) + round_up(parts * d->n_q_heads * 2 * 4, 256);
 }
 
+extern "C" int kvd_attention_split(int d_head, int n_kv_heads, int first_visible, int last_visible, int *chunk_keys) {
+  if ((d_head != 64 && d_head != 128 && d_head != 256) || n_kv_heads < 1) return 0;
+  if (first_visible < 0 || last_visible < first_visible) return 0;
+  const int iters = attn_iters_for_span(d_head, n_kv_heads, last_visible - first_visible + 1);
+  const int ck = attn_chunk_keys(d_head, iters);
+  if (chunk_keys) *chunk_keys = ck;
+  return last_visible / ck - first_visible / ck + 1;
+}
+
 extern "C" kvd_status kvd_create(const kvd_model_desc *desc, kvd_ctx **out) {
   if (!out) return KVD_ERR_INVALID_ARG;
   *out = nullptr;

@@ -53,3 +53,44 @@ def test_create_rejects_bad_arguments_before_touching_a_device():
     assert lib.kvd_poll_status(None, None) == binding.KVD_ERR_INVALID_ARG
     assert lib.kvd_rows_stored(None, 0, 0) == -1
     assert lib.kvd_launch_count(None) == 0
+
+
+def test_attention_split_is_a_function_of_the_visible_range_only():
+    """Host logic of the split decode attention uses: bounded chunk counts, chunks of at least two
+    iterations aligned to absolute position, full coverage, one wave of CTAs for a long single
+    sequence; bad arguments give 0."""
+    assert kvd.kvd_attention_split(96, 4, 0, 10) == (0, 0)
+    assert kvd.kvd_attention_split(256, 0, 0, 10)[0] == 0
+    assert kvd.kvd_attention_split(256, 4, 5, 4)[0] == 0
+    assert kvd.kvd_attention_split(256, 4, -1, 4)[0] == 0
+    for d_head, n_kv, per_iter in ((256, 4, 32), (128, 8, 64), (64, 3, 128)):
+        for span in (1, 2, 31, 33, 257, 1024, 1025, 2049, 4097, 8192, 8193, 32769, 131073, 1000003):
+            for lo in (0, 7, 1000, 123457):
+                hi = lo + span - 1
+                n, ck = kvd.kvd_attention_split(d_head, n_kv, lo, hi)
+                assert ck % per_iter == 0 and ck >= 2 * per_iter   # whole iterations, at least two
+                assert ck <= 64 * per_iter                                # iteration count is capped
+                assert (lo // ck + n - 1) * ck <= hi < (lo // ck + n) * ck  # the chunks cover [lo, hi]
+                if span <= 8192:
+                    assert n <= 130
+                elif ck < 64 * per_iter:
+                    assert n <= 592 // n_kv + 2
+                # the same visible range in any segment layout or batch gives the same split: it is a pure function
+                assert (n, ck) == kvd.kvd_attention_split(d_head, n_kv, lo, hi)
+    # a long single sequence of the Gemma-shaped layer: one wave of four CTAs per SM
+    n, ck = kvd.kvd_attention_split(256, 4, 0, 32768)
+    assert 4 * n <= 4 * 148 and n >= 140 and ck == 224
+
+
+def test_entry_points_reject_null_contexts_and_bad_shapes_without_a_device():
+    lib = binding.load()
+    assert lib.kvd_recompute_kv_step(None, 0, None, 0, None, None, 0, None, None, 0, None) == binding.KVD_ERR_INVALID_ARG
+    assert lib.kvd_recompute_kv(None, 0, None, None, 0, 0, 0, None, None, 0, None) == binding.KVD_ERR_INVALID_ARG
+    assert lib.kvd_decode_attention(None, 0, 0, None, None, None, 0, 0.0, None, None) == binding.KVD_ERR_INVALID_ARG
+    # the allocation-free entry point validates shapes and limits on the host before it looks for a device
+    qp = (ctypes.c_int32 * 1)(0)
+    assert lib.kvd_decode_attention_static(8, 4, 96, 0, 1, None, qp, None, 0, 0.0, None, None) == binding.KVD_ERR_SHAPE
+    assert lib.kvd_decode_attention_static(7, 4, 128, 0, 1, None, qp, None, 0, 0.0, None, None) == binding.KVD_ERR_SHAPE
+    assert lib.kvd_decode_attention_static(8, 4, 128, -1, 1, None, qp, None, 0, 0.0, None, None) == binding.KVD_ERR_INVALID_ARG
+    assert lib.kvd_decode_attention_static(8, 4, 128, 0, 0, None, None, None, 0, 0.0, None, None) == binding.KVD_OK  # empty batch
+    assert lib.kvd_decode_attention_static(8, 4, 128, 0, 1, None, qp, None, 0, 0.0, None, None) == binding.KVD_ERR_INVALID_ARG
