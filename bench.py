@@ -282,7 +282,13 @@ class Workload:
         self.ctx.kvd_checkpoint_residual(s, 0, self.X[s], self.pos, self.T)
 
     def k_recompute(self, i):
-        # rows come straight from the rotating residual buffers (same bytes as the stored copy)
+        # RECOMPUTE_KV of Algorithm 1: T checkpointed rows of set s (filled by the last step on it)
+        s = i % self.n_sets
+        self.ctx.kvd_recompute_kv(0, None, None, self.T, self.K[s], self.V[s], self.kdim, seq=s, first_row=0)
+
+    def k_recompute_rows(self, i):
+        # the same rows handed over by the caller instead (a prefill-shaped call: their statistics are
+        # taken by a small kernel of their own first, two launches)
         s = i % self.n_sets
         self.ctx.kvd_recompute_kv(0, self.X[s], self.pos, self.T, self.K[s], self.V[s], self.kdim)
 
@@ -442,6 +448,7 @@ def run_gpu(args):
     # sets between two CUDA events (launch gaps included), averaged per launch
     iso_ms = {"checkpoint": timed_graph(wl.k_checkpoint, 10), "recompute": timed_graph(wl.k_recompute, 10),
               "recompute_with_current_token": timed_graph(wl.k_recompute_step, 10),
+              "recompute_from_caller_rows": timed_graph(wl.k_recompute_rows, 10),
               "current_token_kv_alone": timed_graph(wl.k_current, 10), "attention": timed_graph(wl.k_attention, 10)}
     read_attn_ms = timed_graph(wl.cached_read_step, 10)
     kv_copy_dst = torch.empty((2, T + 1, wl.kdim), dtype=torch.bfloat16, device="cuda")

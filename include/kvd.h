@@ -136,14 +136,17 @@ void kvd_destroy(kvd_ctx *ctx);
  * composed with Eq. 13-14: (x / rms * gamma) W = (x W') / rms.  Enqueues on `stream` and waits for it. */
 kvd_status kvd_set_layer(kvd_ctx *ctx, int layer, const kvd_layer_desc *ldesc, void *stream);
 
-/* Bytes the residual store needs for `layers_stored` layers (rows + positions). */
+/* Bytes the residual store needs for `layers_stored` layers (rows + positions + row statistics). */
 size_t kvd_store_bytes(const kvd_model_desc *desc, int layers_stored);
 
 /* Hand the context a caller-owned DEVICE arena (256-byte aligned, >= kvd_store_bytes) for the
  * residual store C of Algorithm 1.  Resets all row counts to zero.
  * Layout (the arena stays the caller's, who may read it): residual rows as bf16
  * [layers_stored][max_seqs][max_tokens_per_seq][d_hidden] from the start of the arena, then, at the
- * next multiple of 256 bytes, their positions as int32 [layers_stored][max_seqs][max_tokens_per_seq].
+ * next multiple of 256 bytes, their positions as int32 [layers_stored][max_seqs][max_tokens_per_seq],
+ * then, again at the next multiple of 256 bytes, the sum of squares of each row as fp32 in the same
+ * shape (the RMSNorm statistic of Eq. 2, taken once when the row is checkpointed and read back by every
+ * recomputation; a caller that writes rows into the arena itself must write these too).
  * Row r of (layer, seq) is valid for r < kvd_rows_stored(ctx, layer, seq). */
 kvd_status kvd_attach_store(kvd_ctx *ctx, void *arena, size_t bytes, int layers_stored);
 
@@ -168,7 +171,8 @@ int kvd_attention_split(int d_head, int n_kv_heads, int first_visible, int last_
 kvd_status kvd_attach_workspace(kvd_ctx *ctx, void *workspace, size_t bytes);
 
 /* STORE_RESIDUAL(C, l): append n residual rows (DEVICE bf16 [n, d_hidden], 16-byte aligned) and
- * their absolute positions (DEVICE int32 [n]) to the store of (layer, seq).
+ * their absolute positions (DEVICE int32 [n]) to the store of (layer, seq), together with each row's
+ * sum of squares (taken in the one fixed order that recomputation from caller rows uses as well).
  * KVD_ERR_CAPACITY when the rows do not fit; KVD_ERR_STATE without an attached store. */
 kvd_status kvd_checkpoint_residual(kvd_ctx *ctx, int seq, int layer, const void *rows, const int32_t *positions,
                                    int n, void *stream);

@@ -65,7 +65,8 @@ extern "C" const char *kvd_status_string(kvd_status s) {
 extern "C" size_t kvd_store_bytes(const kvd_model_desc *d, int layers_stored) {
   if (check_desc(d) != KVD_OK || layers_stored <= 0) return 0;
   const size_t slots = static_cast<size_t>(layers_stored) * d->max_seqs * d->max_tokens_per_seq;
-  return round_up(slots * d->d_hidden * 2, 256) + round_up(slots * 4, 256);
+  // rows, then positions, then the rows' sums of squares, each region starting at a 256-byte multiple
+  return round_up(slots * d->d_hidden * 2, 256) + 2 * round_up(slots * 4, 256);
 }
 
 // chunk partials of one sequence
@@ -122,7 +123,14 @@ extern "C" kvd_status kvd_create(const kvd_model_desc *desc, kvd_ctx **out) {
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
   cudaError_t e = cudaMalloc(&ctx->d_status, sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int));
+  if (e == cudaSuccess) {
+    // scratch for the statistics of caller rows (one fp32 per row, at most one full batch of rows)
+    ctx->ext_sumsq_rows = static_cast<size_t>(desc->max_seqs) * desc->max_tokens_per_seq;
+    e = cudaMalloc(&ctx->ext_sumsq, ctx->ext_sumsq_rows * sizeof(float));
+    if (e == cudaSuccess) ctx->prepared_bytes += ctx->ext_sumsq_rows * sizeof(float);
+  }
   if (e != cudaSuccess) {
+    cudaFree(ctx->d_status);
     delete ctx;
     return KVD_ERR_CUDA;
   }
@@ -148,6 +156,7 @@ extern "C" void kvd_destroy(kvd_ctx *ctx) {
     if (kv.second.lo) cudaFree(kv.second.lo);
   }
   if (ctx->d_status) cudaFree(ctx->d_status);
+  if (ctx->ext_sumsq) cudaFree(ctx->ext_sumsq);
   cudaGetLastError();
   delete ctx;
 }
@@ -278,6 +287,7 @@ extern "C" kvd_status kvd_attach_store(kvd_ctx *ctx, void *arena, size_t bytes, 
   const size_t slots = static_cast<size_t>(layers_stored) * d.max_seqs * d.max_tokens_per_seq;
   ctx->store_rows = static_cast<__nv_bfloat16 *>(arena);
   ctx->store_pos = reinterpret_cast<int32_t *>(static_cast<uint8_t *>(arena) + round_up(slots * d.d_hidden * 2, 256));
+  ctx->store_sumsq = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(ctx->store_pos) + round_up(slots * 4, 256));
   ctx->layers_stored = layers_stored;
   ctx->rows_stored.assign(static_cast<size_t>(layers_stored) * d.max_seqs, 0);
   ctx->store_maps.resize(layers_stored);
@@ -337,8 +347,8 @@ extern "C" kvd_status kvd_checkpoint_residual(kvd_ctx *ctx, int seq, int layer, 
   if (count + n > ctx->desc.max_tokens_per_seq) return KVD_ERR_CAPACITY;
   const size_t slot = store_slot(ctx, layer, seq) + count;
   kvd_status st = launch_checkpoint(ctx, static_cast<const __nv_bfloat16 *>(rows), positions,
-                                    ctx->store_rows + slot * ctx->desc.d_hidden, ctx->store_pos + slot, n,
-                                    ctx->desc.d_hidden, static_cast<cudaStream_t>(stream_));
+                                    ctx->store_rows + slot * ctx->desc.d_hidden, ctx->store_pos + slot,
+                                    ctx->store_sumsq + slot, n, ctx->desc.d_hidden, static_cast<cudaStream_t>(stream_));
   if (st == KVD_OK) count += n;
   return st;
 }
@@ -372,6 +382,7 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
     J.row0 = r.first_row;
     J.slab = r.seq;
     J.positions = ctx->store_pos + store_slot(ctx, layer, r.seq) + r.first_row;
+    J.sumsq = ctx->store_sumsq + store_slot(ctx, layer, r.seq) + r.first_row;
     J.k_out = static_cast<__nv_bfloat16 *>(r.k_out);
     J.v_out = static_cast<__nv_bfloat16 *>(r.v_out);
     mb += (r.n + 2 * RC_BLOCK_M - 1) / (2 * RC_BLOCK_M);  // 256-row tiles, 128 rows per CTA of a pair
@@ -389,6 +400,15 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
     J.row0 = 0;
     J.slab = -1;
     J.positions = positions;
+    J.sumsq = nullptr;
+    if (n_rows > RC_INLINE_STAT_ROWS && static_cast<size_t>(n_rows) <= ctx->ext_sumsq_rows) {
+      // too many rows for the statistics warps of the main kernel: take the statistics first (same
+      // function, same bits).  The scratch is shared by the calls on this context, which are
+      // stream-ordered by contract.
+      st = launch_rowstats(ctx, static_cast<const __nv_bfloat16 *>(rows), ctx->ext_sumsq, n_rows, d.d_hidden, stream);
+      if (st != KVD_OK) return st;
+      J.sumsq = ctx->ext_sumsq;
+    }
     J.k_out = static_cast<__nv_bfloat16 *>(k_rows_out);
     J.v_out = static_cast<__nv_bfloat16 *>(v_rows_out);
     mb += (n_rows + 2 * RC_BLOCK_M - 1) / (2 * RC_BLOCK_M);
@@ -414,6 +434,11 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
   p.gamma_k = d.qk_norm ? ls.gamma_k : nullptr;
   p.status = ctx->d_status;
   p.timeout_ns = ctx->timeout_ns;
+  p.ext_rows = static_cast<const __nv_bfloat16 *>(rows);
+  p.row_chunks = d.d_hidden / 8;
+  p.wide_store = out_row_stride % 16 == 0;
+  for (int i = 0; i < n_jobs; ++i)
+    if (((reinterpret_cast<uintptr_t>(p.jobs[i].k_out) | reinterpret_cast<uintptr_t>(p.jobs[i].v_out)) & 31u) != 0) p.wide_store = 0;
   p.trace = nullptr;
   if (ctx->trace) {
     const int tiles = p.num_m_blocks * p.num_n_blocks;
@@ -568,7 +593,7 @@ extern "C" kvd_status kvd_memory_stats(const kvd_ctx *ctx, kvd_mem_stats *out) {
     rows_total += layer_rows;
     if (layer_rows > tokens) tokens = layer_rows;
   }
-  out->checkpoint_bytes_used = rows_total * (static_cast<uint64_t>(d.d_hidden) * 2 + 4);
+  out->checkpoint_bytes_used = rows_total * (static_cast<uint64_t>(d.d_hidden) * 2 + 8);  // row, position, sum of squares
   out->checkpoint_bytes_capacity = ctx->layers_stored > 0 ? kvd_store_bytes(&d, ctx->layers_stored) : 0;
   out->workspace_bytes = ctx->workspace_bytes;
   out->prepared_weight_bytes = ctx->prepared_bytes;

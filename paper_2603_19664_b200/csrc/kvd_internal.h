@@ -25,6 +25,9 @@ constexpr int ROPE_LO_SIZE = 1 << ROPE_LO_BITS;
 // ------------------------------------------------------------------------------ recompute GEMM
 constexpr int RC_BLOCK_M = 128;
 constexpr int RC_BLOCK_K = 64;
+// caller rows up to this count have their statistics taken inside the recompute kernel (its four
+// statistics warps cover them under the main loop of one tile pair); more rows get a kernel of their own
+constexpr int RC_INLINE_STAT_ROWS = 64;
 constexpr int RC_TRACE_TILES = 8;    // tiles per CTA recorded when a trace buffer is attached
 constexpr int RC_TRACE_FIELDS = 16;  // int64 slots per (CTA, tile); see kvd_set_trace
 constexpr int RC_THREADS = 320;  // warp 2 TMA, warp 3 MMA, warps 0,1,8,9 row statistics, warps 4-7 epilogue
@@ -38,6 +41,7 @@ struct RcJob {
   int row0;      // first row: index into the store slab, or 0 for a caller buffer
   int slab;      // store slab (sequence slot of this layer), or -1: rows come from the caller's buffer
   const int32_t *positions;  // [n]
+  const float *sumsq;        // [n] sum of squares of each row (store ranges), nullptr for the caller's rows
   __nv_bfloat16 *k_out;      // row m of the job at k_out + m * out_row_stride
   __nv_bfloat16 *v_out;
 };
@@ -61,6 +65,9 @@ struct RecomputeParams {
   int *status;
   unsigned long long timeout_ns;
   long long *trace;  // nullptr unless a trace buffer is attached
+  const __nv_bfloat16 *ext_rows;  // the caller's rows (job with slab < 0), [n][d_hidden]
+  int row_chunks;                 // d_hidden / 8: 16-byte chunks per row
+  int wide_store;                 // outputs are 32-byte aligned: 32-byte stores
   RcJob jobs[RC_MAX_JOBS];
 };
 
@@ -176,6 +183,9 @@ struct kvd_ctx {
   // residual store
   __nv_bfloat16 *store_rows = nullptr;
   int32_t *store_pos = nullptr;
+  float *store_sumsq = nullptr;
+  float *ext_sumsq = nullptr;     // statistics of caller rows taken ahead of the recompute kernel
+  size_t ext_sumsq_rows = 0;
   int layers_stored = 0;
   std::vector<int> rows_stored;  // [layers_stored * max_seqs]
   std::vector<CUtensorMap> store_maps;  // per stored layer: [max_seqs][max_tokens_per_seq][d_hidden]
@@ -213,8 +223,10 @@ kvd_status launch_attention(kvd_ctx *ctx, const AttnLaunch &L, int d_head, int g
 kvd_status launch_prepare_weights(kvd_ctx *ctx, const __nv_bfloat16 *w, const __nv_bfloat16 *gamma, __nv_bfloat16 *wt,
                                   int d_hidden, int n_cols, cudaStream_t stream);
 kvd_status launch_convert_gamma(kvd_ctx *ctx, const __nv_bfloat16 *g, float *out, int n, cudaStream_t stream);
+kvd_status launch_rowstats(kvd_ctx *ctx, const __nv_bfloat16 *rows, float *sumsq, int n, int d_hidden,
+                           cudaStream_t stream);
 kvd_status launch_checkpoint(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, __nv_bfloat16 *dst_rows,
-                             int32_t *dst_pos, int n, int d_hidden, cudaStream_t stream);
+                             int32_t *dst_pos, float *dst_sumsq, int n, int d_hidden, cudaStream_t stream);
 kvd_status launch_selftest_timeout(kvd_ctx *ctx, unsigned long long timeout_ns, cudaStream_t stream);
 kvd_status cuda_fail(kvd_ctx *ctx, cudaError_t e, const char *where);
 }  // namespace kvd

@@ -32,16 +32,48 @@ __global__ void kvd_convert_gamma_kernel(const __nv_bfloat16 *__restrict__ g, fl
   if (i < n) out[i] = __bfloat162float(g[i]);
 }
 
-// Copy n rows of d_hidden bf16 (16 bytes per thread-iteration) and their positions into the store.
+// Copy n rows of d_hidden bf16 and their positions into the store, one warp per row; the warp also
+// takes the row's sum of squares (the RMSNorm statistic of Eq. 2), which the recompute kernel reads
+// back instead of taking it again for every recomputation.
 __global__ void __launch_bounds__(256) kvd_checkpoint_kernel(const uint4 *__restrict__ rows,
                                                              const int32_t *__restrict__ pos,
                                                              uint4 *__restrict__ dst_rows, int32_t *__restrict__ dst_pos,
-                                                             long long n_vec, int n) {
-  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
-  const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+                                                             float *__restrict__ dst_sumsq, int row_chunks, int n) {
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
   grid_launch_dependents();  // the next kernel's set-up may overlap this copy
-  for (long long i = tid; i < n_vec; i += stride) dst_rows[i] = rows[i];
-  for (long long i = tid; i < n; i += stride) dst_pos[i] = pos[i];
+  for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n; r += warps) {
+    const size_t off = static_cast<size_t>(r) * row_chunks;
+    const uint4 *const src[1] = {rows + off};
+    uint4 *const dst[1] = {dst_rows + off};
+    float ss[1];
+    warp_rows_sumsq<1, 8, true>(src, dst, row_chunks, lane, ss);
+    if (lane == 0) {
+      dst_sumsq[r] = ss[0];
+      dst_pos[r] = pos[r];
+    }
+  }
+}
+
+// Sums of squares of n caller rows (no copy), two rows per warp and pass: what kvd_recompute_kv takes
+// ahead of the main kernel when the caller hands it more rows than that kernel's statistics warps
+// can cover under the main loop.
+__global__ void __launch_bounds__(256) kvd_rowstats_kernel(const uint4 *__restrict__ rows, float *__restrict__ sumsq,
+                                                           int row_chunks, int n) {
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  grid_launch_dependents();
+  for (int r = ((blockIdx.x * blockDim.x + threadIdx.x) >> 5) * 2; r < n; r += 2 * warps) {
+    const int r1 = r + 1 < n ? r + 1 : r;
+    const uint4 *const src[2] = {rows + static_cast<size_t>(r) * row_chunks, rows + static_cast<size_t>(r1) * row_chunks};
+    uint4 *const none[2] = {nullptr, nullptr};
+    float ss[2];
+    warp_rows_sumsq<2, 8, false>(src, none, row_chunks, lane, ss);
+    if (lane == 0) {
+      sumsq[r] = ss[0];
+      sumsq[r1] = ss[1];
+    }
+  }
 }
 
 // Self-test of the bounded wait: one thread waits on an mbarrier that nothing ever arrives on.  The
@@ -84,16 +116,29 @@ kvd_status launch_convert_gamma(kvd_ctx *ctx, const __nv_bfloat16 *g, float *out
 }
 
 kvd_status launch_checkpoint(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, __nv_bfloat16 *dst_rows,
-                             int32_t *dst_pos, int n, int d_hidden, cudaStream_t stream) {
-  const long long n_vec = static_cast<long long>(n) * d_hidden / 8;
-  long long blocks = (n_vec + 255) / 256;
+                             int32_t *dst_pos, float *dst_sumsq, int n, int d_hidden, cudaStream_t stream) {
+  long long blocks = (static_cast<long long>(n) + 7) / 8;  // eight warps, one row each per pass
   const long long cap = static_cast<long long>(ctx->num_sms) * 8;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   kvd_checkpoint_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
-      reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint4 *>(dst_rows), dst_pos, n_vec, n);
+      reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint4 *>(dst_rows), dst_pos, dst_sumsq, d_hidden / 8, n);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "launch checkpoint");
+  ctx->launches += 1;
+  return KVD_OK;
+}
+
+kvd_status launch_rowstats(kvd_ctx *ctx, const __nv_bfloat16 *rows, float *sumsq, int n, int d_hidden,
+                           cudaStream_t stream) {
+  long long blocks = (static_cast<long long>(n) + 15) / 16;  // eight warps, two rows each per pass
+  const long long cap = static_cast<long long>(ctx->num_sms) * 8;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  kvd_rowstats_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(reinterpret_cast<const uint4 *>(rows), sumsq,
+                                                                         d_hidden / 8, n);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "launch rowstats");
   ctx->launches += 1;
   return KVD_OK;
 }

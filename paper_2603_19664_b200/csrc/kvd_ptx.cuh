@@ -99,6 +99,22 @@ __device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const void *tmap,
       : "memory");
 }
 
+// The same loads issued by either CTA of a pair (cta_group::2): the completion may be counted on a
+// barrier of the partner CTA (`bar` is then a shared::cluster address obtained with map_to_cta).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t smem_dst, const void *tmap, uint32_t bar, int32_t c0, int32_t c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t smem_dst, const void *tmap, uint32_t bar, int32_t c0, int32_t c1,
+                                                 int32_t c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
 // ------------------------------------------------------------------------------ dependent launch
 // A kernel launched with programmatic stream serialisation may start while its predecessor in the
 // stream is still running: everything up to grid_dependency_wait() (set-up that touches no global
@@ -273,5 +289,66 @@ __device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
 }
 // the two bf16 halves of a 32-bit word as a packed pair of fp32
 __device__ __forceinline__ uint64_t bf16x2_to_f32x2(uint32_t w) { return pack2(bf16_lo(w), bf16_hi(w)); }
+
+// ------------------------------------------------------------------------------ row statistic (Eq. 2)
+// Sum of squares of one row of bf16 values (n_chunks 16-byte chunks), taken by a whole warp: lane l
+// squares chunks l, l + 32, ... in ascending order into eight partial sums (one per element slot of
+// a chunk, as four two-wide FMAs), adds the eight in a fixed tree, and the 32 lane sums are combined
+// by an xor butterfly (16, 8, 4, 2, 1), so every lane returns the same bits.  With COPY the chunks
+// are also written to `dst`.  (FMAs and adds are explicit: the compiler cannot re-associate them.)  The checkpoint kernel and the recompute kernel both take the statistic
+// with this one function: its bits do not depend on which of them saw the row.
+__device__ __forceinline__ void sumsq_chunk(uint64_t (&ps2)[4], const uint4 &v) {
+  uint64_t x2;
+  x2 = bf16x2_to_f32x2(v.x); ps2[0] = ffma2(x2, x2, ps2[0]);
+  x2 = bf16x2_to_f32x2(v.y); ps2[1] = ffma2(x2, x2, ps2[1]);
+  x2 = bf16x2_to_f32x2(v.z); ps2[2] = ffma2(x2, x2, ps2[2]);
+  x2 = bf16x2_to_f32x2(v.w); ps2[3] = ffma2(x2, x2, ps2[3]);
+}
+template <int R, int B, bool COPY>
+__device__ __forceinline__ void warp_rows_sumsq(const uint4 *const (&src)[R], uint4 *const (&dst)[R], int n_chunks, int lane,
+                                                float (&out)[R]) {
+  // R rows side by side, B loads per row in flight per lane; each row's arithmetic is the sequence
+  // described above whatever R and B are
+  uint64_t ps2[R][4];
+#pragma unroll
+  for (int r = 0; r < R; ++r)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) ps2[r][j] = 0ull;
+  int c = lane;
+  for (; c + 32 * (B - 1) < n_chunks; c += 32 * B) {
+    uint4 v[R][B];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int j = 0; j < B; ++j) v[r][j] = __ldg(src[r] + c + 32 * j);
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int j = 0; j < B; ++j) {
+        if (COPY) dst[r][c + 32 * j] = v[r][j];
+        sumsq_chunk(ps2[r], v[r][j]);
+      }
+  }
+  for (; c < n_chunks; c += 32) {
+    uint4 v[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) v[r] = __ldg(src[r] + c);
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      if (COPY) dst[r][c] = v[r];
+      sumsq_chunk(ps2[r], v[r]);
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    float ps[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) unpack2(ps2[r][j], ps[2 * j], ps[2 * j + 1]);
+    float sum = ((ps[0] + ps[1]) + (ps[2] + ps[3])) + ((ps[4] + ps[5]) + (ps[6] + ps[7]));
+#pragma unroll
+    for (int k = 16; k >= 1; k >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, k);
+    out[r] = sum;
+  }
+}
 
 }  // namespace kvd

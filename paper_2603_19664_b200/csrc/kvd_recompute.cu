@@ -10,14 +10,19 @@
 // Persistent CTA pairs (clusters of two, one CTA per SM) walk over 256 x BLOCK_N output tiles with
 // tcgen05.mma.cta_group::2: each CTA owns 128 rows of the tile and stages, per 64-wide k block, its
 // own 128x64 tile of X plus HALF of the BLOCK_Nx64 tile of W'; the tensor cores of the pair read
-// both halves, so a k block costs each SM 32 KB of L2 traffic instead of 48 KB.  Warp roles:
-//   warp 2         TMA producer (one lane; local tiles, local barrier)
-//   warp 3         even CTA: one lane issues the MMAs for the pair and commits to both CTAs' barriers
-//                  odd CTA:  one lane relays "my stage has landed" to the even CTA; owns TMEM alloc
-//   warps 0,1,8,9  row statistics: each thread sums x^2 of one row from the X tiles as they land
+// both halves, so a k block costs each SM 32 KB of L2 traffic instead of 48 KB.  Both CTAs' loads
+// count their bytes on ONE barrier per stage, in the even CTA, which that CTA's producer arms for
+// the pair: the MMA issuer waits on a single barrier and nothing has to be relayed across the pair.
+// Warp roles:
+//   warp 2         TMA producer (one lane)
+//   warp 3         even CTA: one lane issues the MMAs for the pair and commits to both CTAs' barriers;
+//                  owns the TMEM allocation
+//   warps 0,1,8,9  row statistics 1/rms(x): read back from the store for checkpointed rows (taken
+//                  when the row was checkpointed), taken from global memory for the caller's rows
 //   warps 4-7      epilogue: tcgen05.ld the fp32 accumulator, normalise, rotate, convert, store
-// Warp w runs on scheduler w % 4, so the two single-thread roles (warps 2, 3) share their scheduler
-// with one epilogue warp only; the statistics warps sit on the other two schedulers.
+// Nothing but the tensor cores reads the operand ring, so a stage is free again as soon as the MMAs
+// that read it have retired.  Warp w runs on scheduler w % 4, so the two single-thread roles (warps
+// 2, 3) share their scheduler with one epilogue warp only.
 // The accumulator is double-buffered in TMEM (2 x BLOCK_N columns) so the epilogue of tile i
 // overlaps the main loop of tile i+1.
 //
@@ -26,9 +31,10 @@
 // (incremental addresses, one asm block per k block).  Every wait is bounded; on expiry the kernel records STATUS_TIMEOUT and drains.
 //
 // Bit-reproducibility: the k loop always runs over all of d_hidden in ascending order with one MMA
-// shape, row sums are taken thread-locally in a fixed order, the key norm is reduced by the single
-// thread that owns the row, and cos/sin depend on (position, channel) only.  A row's output bits
-// are therefore independent of M and of the row's index.
+// shape, a row's sum of squares is taken by one function in one fixed order wherever it is taken
+// (warp_row_sumsq), the key norm is reduced by the single thread that owns the row, and cos/sin
+// depend on (position, channel) only.  A row's output bits are therefore independent of M, of the
+// row's index and of whether it came from the store or from the caller.
 #include <string.h>
 
 #include "kvd_internal.h"
@@ -44,8 +50,8 @@ struct RcCfg {
   static constexpr int B_BYTES = B_ROWS * RC_BLOCK_K * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = 2 * BLOCK_N;
-  // barriers: full[S], empty[S], peer_full[S], tmem_full[2], tmem_empty[2], stats_full[2], rstd_free[2]
-  static constexpr int NUM_BARS = 3 * STAGES + 8;
+  // barriers: full[S] (used in the even CTA), empty[S], tmem_full[2], tmem_empty[2], stats_full[2], rstd_free[2]
+  static constexpr int NUM_BARS = 2 * STAGES + 9;  // + stats_x: the four statistics warps among themselves
   static constexpr int TAIL_BYTES = NUM_BARS * 8 + 16 /*tmem ptr, abort*/ + 2 * RC_BLOCK_M * 4 /*rstd*/ + 256 * 4 /*gamma_k*/;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + TAIL_BYTES;  // the base must be 1024-byte aligned
   static_assert(SMEM_BYTES <= 232448, "more shared memory than an SM offers");
@@ -115,6 +121,29 @@ __device__ __forceinline__ void umma_kblock_pair(uint32_t d_tmem, uint32_t a_lo,
       : "memory");
 }
 
+// Output stores.  Each epilogue thread owns one row, so the 32 lanes of a store instruction write 32
+// different lines and the instruction occupies the SM's load/store data path once per lane -- cycles
+// the operand ring's TMA writes and the tensor cores' operand reads compete for.  32-byte stores halve
+// the instruction count, and not allocating the lines in L1 (nothing reads them back) halves the
+// data-path cycles again.  `o` holds n16 * 4 packed words.
+template <int N16>
+__device__ __forceinline__ void store_row_piece(__nv_bfloat16 *dst, const uint32_t *o, bool wide) {
+  if (wide) {
+#pragma unroll
+    for (int j = 0; j < N16 / 2; ++j)
+      asm volatile("st.global.L1::no_allocate.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + 16 * j),
+                   "r"(o[8 * j]), "r"(o[8 * j + 1]), "r"(o[8 * j + 2]), "r"(o[8 * j + 3]), "r"(o[8 * j + 4]),
+                   "r"(o[8 * j + 5]), "r"(o[8 * j + 6]), "r"(o[8 * j + 7])
+                   : "memory");
+  } else {
+#pragma unroll
+    for (int j = 0; j < N16; ++j)
+      asm volatile("st.global.L1::no_allocate.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(dst + 8 * j), "r"(o[4 * j]),
+                   "r"(o[4 * j + 1]), "r"(o[4 * j + 2]), "r"(o[4 * j + 3])
+                   : "memory");
+  }
+}
+
 template <int BLOCK_N, int D_HEAD, bool TRACE>
 __global__ void __launch_bounds__(RC_THREADS, 1)
 kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __grid_constant__ CUtensorMap tmap_rows,
@@ -140,11 +169,11 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   const uint32_t bar_base = smem_u32(bars);
   auto bar_full = [&](int s) { return bar_base + 8u * s; };
   auto bar_empty = [&](int s) { return bar_base + 8u * (STAGES + s); };
-  auto bar_peer_full = [&](int s) { return bar_base + 8u * (2 * STAGES + s); };  // even CTA only
-  auto bar_tmem_full = [&](int a) { return bar_base + 8u * (3 * STAGES + a); };
-  auto bar_tmem_empty = [&](int a) { return bar_base + 8u * (3 * STAGES + 2 + a); };  // even CTA only
-  auto bar_stats_full = [&](int a) { return bar_base + 8u * (3 * STAGES + 4 + a); };
-  auto bar_rstd_free = [&](int a) { return bar_base + 8u * (3 * STAGES + 6 + a); };
+  auto bar_tmem_full = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+  auto bar_tmem_empty = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };  // even CTA only
+  auto bar_stats_full = [&](int a) { return bar_base + 8u * (2 * STAGES + 4 + a); };
+  auto bar_rstd_free = [&](int a) { return bar_base + 8u * (2 * STAGES + 6 + a); };
+  const uint32_t bar_stats_x = bar_base + 8u * (2 * STAGES + 8);
   const uint32_t cta_rank = cluster_ctarank();  // 0: issues the MMAs, 1: its partner
   const int cluster_id = static_cast<int>(blockIdx.x >> 1);
   const int num_clusters = static_cast<int>(gridDim.x >> 1);
@@ -154,9 +183,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   const int num_tiles = p.num_m_blocks * p.num_n_blocks;
   // Tile order.  With more tiles than clusters a cluster works through "units" of two consecutive
   // tiles that share a row block -- the key tile and the value tile of one head column -- so that the
-  // row statistics (whose shared-memory reads compete with the tensor cores' operand fetch: 12 % of
-  // the kernel's time when taken for every tile) are taken once per unit and reused; key first, so
-  // that the last tile of a CTA, whose epilogue nothing overlaps, is a cheap value tile.  (Units of
+  // row statistics are fetched once per unit and reused; key first, so that the last tile of a CTA,
+  // whose epilogue nothing overlaps, is a cheap value tile.  (Units of
   // all tiles of a row block measured slower: the units are then too few to balance the clusters.)
   // With no more tiles than clusters every tile is its own unit, all key tiles first.  Falls back to
   // row-major single tiles when a tile mixes key and value heads.
@@ -201,9 +229,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(bar_full(s), 1);
-      mbar_init(bar_empty(s), 1 + 4);  // MMA commit + one arrival per statistics warp
-      mbar_init(bar_peer_full(s), 1);  // the partner's relay
+      mbar_init(bar_full(s), 1);   // the even CTA's producer arms it with the bytes of both CTAs
+      mbar_init(bar_empty(s), 1);  // the MMA commit
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(bar_tmem_full(a), 1);
@@ -211,6 +238,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
       mbar_init(bar_stats_full(a), RC_BLOCK_M);  // one arrival per statistics thread
       mbar_init(bar_rstd_free(a), 4);            // one arrival per local epilogue warp
     }
+    mbar_init(bar_stats_x, 4);  // one arrival per statistics warp
     *s_abort = 0;
     fence_mbar_init();
     prefetch_tensormap(&tmap_store);
@@ -237,7 +265,9 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
     if (lane == 0) {
       int s = 0, n_issued = 0;
       uint32_t ph = 0;
-      uint32_t full = bar_full(0), empty = bar_empty(0), dst = smem_base;
+      // the stage barrier lives in the even CTA; `full` is its address as seen from this CTA
+      const uint32_t full0 = map_to_cta(bar_full(0), 0);
+      uint32_t full = full0, empty = bar_empty(0), dst = smem_base;
       const int b_row_off = static_cast<int>(cta_rank) * Cfg::B_ROWS;
       bool ok = true;
       int job, m0, n0;
@@ -259,9 +289,9 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
             break;
           }
           if (TRACE) waited += clock64() - w0;
-          mbar_arrive_expect_tx(full, Cfg::STAGE_BYTES);
-          tma_load_3d(dst, tmap_a, full, k0, m0, a_slab);
-          tma_load_2d(dst + Cfg::A_BYTES, &tmap_b, full, k0, n0);
+          if (cta_rank == 0) mbar_arrive_expect_tx(bar_full(s), 2 * Cfg::STAGE_BYTES);
+          tma_load_3d_pair(dst, tmap_a, full, k0, m0, a_slab);
+          tma_load_2d_pair(dst + Cfg::A_BYTES, &tmap_b, full, k0, n0);
           ++n_issued;
           full += 8u;
           empty += 8u;
@@ -269,7 +299,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
           if (++s == STAGES) {
             s = 0;
             ph ^= 1u;
-            full = bar_full(0);
+            full = full0;
             empty = bar_empty(0);
             dst = smem_base;
           }
@@ -278,17 +308,24 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
         trace_put<TRACE>(p.trace, ti, 2);
       }
       if (!ok) {
-        // leave no bulk copy in flight behind us: wait (bounded) for every load already issued.
-        // Stages below s were last filled in the current round (parity ph), the others in the
-        // previous round.
-        for (int i = 0; i < STAGES; ++i) {
-          if (n_issued > i) {
-            const uint32_t par = i < s ? ph : ph ^ 1u;
-            const unsigned long long t0 = globaltimer_ns();
-            while (!mbar_try_wait(bar_full(i), par)) {
-              if (globaltimer_ns() - t0 > 100000000ull) break;
+        // leave no bulk copy in flight behind us.  The even CTA waits (bounded) for every stage it
+        // armed: stages below s were last filled in the current round (parity ph), the others in the
+        // previous round; a stage completes only when the partner's bytes have landed too.  The odd
+        // CTA cannot watch the barrier; it gives its copies a bounded time that exceeds any load
+        // latency by orders of magnitude, and neither CTA leaves before the cluster barrier below.
+        if (cta_rank == 0) {
+          for (int i = 0; i < STAGES; ++i) {
+            if (n_issued > i) {
+              const uint32_t par = i < s ? ph : ph ^ 1u;
+              const unsigned long long t0 = globaltimer_ns();
+              while (!mbar_try_wait(bar_full(i), par)) {
+                if (globaltimer_ns() - t0 > 100000000ull) break;
+              }
             }
           }
+        } else {
+          const unsigned long long t0 = globaltimer_ns();
+          while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
         }
       }
     }
@@ -303,7 +340,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
       constexpr uint32_t stage_units = Cfg::STAGE_BYTES >> 4, b_off_units = Cfg::A_BYTES >> 4;
       int s = 0, a = 0;
       uint32_t ph = 0, aph = 0;
-      uint32_t full = bar_full(0), peer = bar_peer_full(0), empty = bar_empty(0), a_lo = a_lo0;
+      uint32_t full = bar_full(0), empty = bar_empty(0), a_lo = a_lo0;
       bool ok = true;
       int job_, m0_, n0_;
       bool first_;
@@ -320,8 +357,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
         trace_put<TRACE>(p.trace, ti, 10, (m0_ / (2 * RC_BLOCK_M)) * p.num_n_blocks + n0_ / BLOCK_N);
         for (int kb = 0; kb < p.num_k_blocks; ++kb) {
           const long long w0 = TRACE ? clock64() : 0;
-          // stage s has landed here and (relayed) in the partner CTA
-          if (!mbar_wait(full, ph, s_abort, tmo) || !mbar_wait(peer, ph, s_abort, tmo)) {
+          // stage s has landed in both CTAs
+          if (!mbar_wait(full, ph, s_abort, tmo)) {
             raise(p.status, STATUS_TIMEOUT, s_abort);
             ok = false;
             break;
@@ -330,14 +367,12 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
           tc_fence_after();
           umma_kblock_pair(d_tmem, a_lo, a_lo + b_off_units, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
           full += 8u;
-          peer += 8u;
           empty += 8u;
           a_lo += stage_units;
           if (++s == STAGES) {
             s = 0;
             ph ^= 1u;
             full = bar_full(0);
-            peer = bar_peer_full(0);
             empty = bar_empty(0);
             a_lo = a_lo0;
           }
@@ -351,49 +386,18 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
           aph ^= 1u;
         }
       }
-    } else if (lane == 0) {
-      // ---------------------------------------------------------------- relay (odd CTA)
-      // tells the MMA issuer that this CTA's copy of stage s has landed
-      int s = 0;
-      uint32_t ph = 0;
-      uint32_t full = bar_full(0);
-      const uint32_t peer0 = map_to_cta(bar_peer_full(0), 0);
-      uint32_t peer = peer0;
-      bool ok = true;
-      int job_, m0_, n0_;
-      bool first_;
-      for (int ti = 0; ok && tile_at(ti, job_, m0_, n0_, first_); ++ti) {
-        for (int kb = 0; kb < p.num_k_blocks; ++kb) {
-          if (!mbar_wait(full, ph, s_abort, tmo)) {
-            raise(p.status, STATUS_TIMEOUT, s_abort);
-            ok = false;
-            break;
-          }
-          mbar_arrive_cluster(peer);
-          full += 8u;
-          peer += 8u;
-          if (++s == STAGES) {
-            s = 0;
-            ph ^= 1u;
-            full = bar_full(0);
-            peer = peer0;
-          }
-        }
-      }
     }
   } else if (warp < 2 || warp >= 8) {
     // ------------------------------------------------------------------ row statistics (Eq. 2)
-    const int row = (warp < 2 ? warp : warp - 6) * 32 + lane;  // warps 0, 1, 8, 9 -> rows 0..127
-    const uint32_t row_off = row * 128u;
-    const uint32_t sw = (row & 7u) << 4;
-    int s = 0, a = 0;
-    uint32_t ph = 0, aph = 0;
-    bool ok = true;
-    int job_, m0_, n0_;
+    const int w4 = warp < 2 ? warp : warp - 6;  // warps 0, 1, 8, 9 -> rows 32 * w4 .. 32 * w4 + 31
+    const int row = w4 * 32 + lane;
+    int a = 0;
+    uint32_t aph = 0;
+    int job, m0, n0_;
     bool first_of_unit;
     float rstd_row = 0.f;  // of this thread's row, kept for the other tiles of the unit
-    for (int ti = 0; ok && tile_at(ti, job_, m0_, n0_, first_of_unit); ++ti) {
-      long long waited = 0;
+    uint32_t xph = 0;      // phase of the statistics warps' own barrier
+    for (int ti = 0; tile_at(ti, job, m0, n0_, first_of_unit); ++ti) {
       const long long st0 = TRACE ? clock64() : 0;
       // s_rstd[a] is free once the local epilogue that read it has finished with accumulator a
       // the whole warp takes the same branch: aligned instructions follow
@@ -401,51 +405,45 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
         raise(p.status, STATUS_TIMEOUT, s_abort);
         break;
       }
-      // eight partial sums (one per element slot of a 16-byte chunk) keep the FMA chains short; they
-      // are combined in a fixed order below, the same for every row
-      uint64_t ps2[4] = {0ull, 0ull, 0ull, 0ull};  // (ps0, ps1), (ps2, ps3), (ps4, ps5), (ps6, ps7): two-wide fp32 FMAs
-      for (int kb = 0; kb < p.num_k_blocks; ++kb) {
-        const long long w0 = TRACE ? clock64() : 0;
-        if (!warp_wait(bar_full(s), ph, s_abort, tmo, lane)) {
-          raise(p.status, STATUS_TIMEOUT, s_abort);
-          ok = false;
-          break;
-        }
-        if (TRACE) waited += clock64() - w0;
-        const uint32_t a_addr = smem_base + s * Cfg::STAGE_BYTES + row_off;
-        // (the same rows again in a later tile of the unit: only the stage hand-shake is needed)
-        if (first_of_unit) {
+      if (first_of_unit) {
+        const RcJob &J = p.jobs[job];
+        const int n_here = J.n - m0;  // rows of this CTA's 128 that exist (may exceed 128)
+        if (J.sumsq != nullptr) {
+          // checkpointed rows (or caller rows whose statistics a kernel of their own took): the sum of
+          // squares is read back
+          const float sum = row < n_here ? __ldg(J.sumsq + m0 + row) : 0.f;
+          rstd_row = 1.0f / sqrtf(sum * p.inv_d_hidden + p.rms_eps);
+        } else {
+          // a few caller rows: the four warps share them in groups of four rows (group g -> warp g % 4),
+          // leave 1/rms in s_rstd[a] and meet on a barrier before every thread picks up its own row.
+          // Rows past the end of the job read the job's last row instead (no branch inside a group).
+          const uint4 *base = reinterpret_cast<const uint4 *>(p.ext_rows) + static_cast<size_t>(m0) * p.row_chunks;
+#pragma unroll 1
+          for (int g = w4; g < 32 && 4 * g < n_here; g += 4) {
+            const uint4 *src[4];
+            uint4 *const none[4] = {nullptr, nullptr, nullptr, nullptr};
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          // logical 16-byte chunk c of this row sits at chunk (c ^ (row % 8)) under the 128-byte swizzle
-          uint32_t w0, w1, w2, w3;
-          asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                       : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3)
-                       : "r"(a_addr + ((static_cast<uint32_t>(c) << 4) ^ sw)));
-          uint64_t x2;
-          x2 = bf16x2_to_f32x2(w0); ps2[0] = ffma2(x2, x2, ps2[0]);
-          x2 = bf16x2_to_f32x2(w1); ps2[1] = ffma2(x2, x2, ps2[1]);
-          x2 = bf16x2_to_f32x2(w2); ps2[2] = ffma2(x2, x2, ps2[2]);
-          x2 = bf16x2_to_f32x2(w3); ps2[3] = ffma2(x2, x2, ps2[3]);
-        }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_empty(s));
-        if (++s == STAGES) {
-          s = 0;
-          ph ^= 1u;
+            for (int i = 0; i < 4; ++i) src[i] = base + static_cast<size_t>(4 * g + i < n_here ? 4 * g + i : n_here - 1) * p.row_chunks;
+            float ss[4];
+            warp_rows_sumsq<4, 4, false>(src, none, p.row_chunks, lane, ss);
+            const float mine = lane == 0 ? ss[0] : lane == 1 ? ss[1] : lane == 2 ? ss[2] : ss[3];
+            if (lane < 4 && 4 * g + lane < n_here)
+              s_rstd[a * RC_BLOCK_M + 4 * g + lane] = 1.0f / sqrtf(mine * p.inv_d_hidden + p.rms_eps);
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_stats_x);
+          if (!warp_wait(bar_stats_x, xph, s_abort, tmo, lane)) {
+            raise(p.status, STATUS_TIMEOUT, s_abort);
+            break;
+          }
+          xph ^= 1u;
+          rstd_row = row < n_here ? s_rstd[a * RC_BLOCK_M + row] : 0.f;
         }
       }
-      if (!ok) break;
-      float ps[8];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) unpack2(ps2[j], ps[2 * j], ps[2 * j + 1]);
-      const float sum = ((ps[0] + ps[1]) + (ps[2] + ps[3])) + ((ps[4] + ps[5]) + (ps[6] + ps[7]));
-      if (first_of_unit) rstd_row = 1.0f / sqrtf(sum * p.inv_d_hidden + p.rms_eps);
       s_rstd[a * RC_BLOCK_M + row] = rstd_row;
       mbar_arrive(bar_stats_full(a));
       if (TRACE && threadIdx.x == 0) {
-        trace_put<TRACE>(p.trace, ti, 8, waited);
+        trace_put<TRACE>(p.trace, ti, 8, 0);
         trace_put<TRACE>(p.trace, ti, 9, clock64() - st0);
       }
       if (++a == 2) {
@@ -474,6 +472,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
       if (TRACE && threadIdx.x == 4 * 32) trace_put<TRACE>(p.trace, ti, 6);
       const int m = m0 + row;
       const bool valid = m < J.n;
+      const bool wide = p.wide_store != 0;
       const float rstd = s_rstd[a * RC_BLOCK_M + row];
       int pos = valid ? J.positions[m] : 0;
       if (pos < 0 || pos >= p.max_pos) {
@@ -503,11 +502,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
 #pragma unroll
             for (int j = 0; j < 16; ++j)
               o[j] = pack_bf16(__uint_as_float(r[2 * j]) * rstd, __uint_as_float(r[2 * j + 1]) * rstd);
-            if (valid) {
-              uint4 *d4 = reinterpret_cast<uint4 *>(dst + c * 32);
-#pragma unroll
-              for (int j = 0; j < 4; ++j) d4[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
-            }
+            if (valid) store_row_piece<4>(dst + c * 32, o, wide);
           }
         } else {
           // ---- key head (Eq. 13): 1/rms, optional key norm, rotation R_pos
@@ -568,11 +563,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
                 o[j] = pack_bf16(fmaf(a0, c0, -b0 * s0), fmaf(a0, s0, b0 * c0));
                 o[j + 1] = pack_bf16(fmaf(a1, c1, -b1 * s1), fmaf(a1, s1, b1 * c1));
               }
-              if (valid) {
-                uint4 *d4 = reinterpret_cast<uint4 *>(dst + c * 16);
-                d4[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                d4[1] = make_uint4(o[4], o[5], o[6], o[7]);
-              }
+              if (valid) store_row_piece<2>(dst + c * 16, o, wide);
             }
           } else {
             constexpr int NC = HALF / 16;  // 16 pairs (i, i + HALF) per step
@@ -607,12 +598,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
                 ob[j >> 1] = pack_bf16(fmaf(a0, s0, b0 * c0), fmaf(a1, s1, b1 * c1));
               }
               if (valid) {
-                uint4 *da = reinterpret_cast<uint4 *>(dst + c * 16);
-                uint4 *db = reinterpret_cast<uint4 *>(dst + HALF + c * 16);
-                da[0] = make_uint4(oa[0], oa[1], oa[2], oa[3]);
-                da[1] = make_uint4(oa[4], oa[5], oa[6], oa[7]);
-                db[0] = make_uint4(ob[0], ob[1], ob[2], ob[3]);
-                db[1] = make_uint4(ob[4], ob[5], ob[6], ob[7]);
+                store_row_piece<2>(dst + c * 16, oa, wide);
+                store_row_piece<2>(dst + HALF + c * 16, ob, wide);
               }
             }
           }

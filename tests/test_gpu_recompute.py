@@ -166,7 +166,7 @@ def test_checkpoint_store_roundtrip_and_recompute_from_store():
     ctx.kvd_checkpoint_residual(1, 0, x[100:], p[100:], 200)
     assert ctx.kvd_rows_stored(0, 1) == 300 and ctx.kvd_rows_stored(0, 0) == 100
     stats = ctx.kvd_memory_stats()
-    assert stats["checkpoint_bytes_used"] == 400 * (shape.d_hidden * 2 + 4)
+    assert stats["checkpoint_bytes_used"] == 400 * (shape.d_hidden * 2 + 8)
     assert stats["eq24_residual_bytes_per_token"] == shape.d_hidden * 2
     K, V = run_gpu(ctx, shape, X, pos)
     k = torch.zeros((250, kdim), dtype=torch.bfloat16, device="cuda")

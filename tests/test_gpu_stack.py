@@ -102,7 +102,7 @@ def test_single_checkpoint_chained_recompute_is_token_and_bit_identical_to_full_
             assert torch.equal(a, b), f"budget {B}: logits differ"
         assert m.replayed_rows > 0 and m.recomputed_rows > 0
         rep = m.memory_report()
-        assert rep["checkpoint_bytes_single_row"] == m.t * (stack.d_hidden * 2 + 4)
+        assert rep["checkpoint_bytes_single_row"] == m.t * (stack.d_hidden * 2 + 8)
         assert rep["live_kv_bytes"] == stack.n_layers * min(B, m.t) * 2 * stack.n_kv_heads * stack.d_head * 2
         # Eq. 28 with b = 2 bytes: B tokens of K/V plus one residual row per evicted token
         assert rep["eq28_bytes"] == rep["live_kv_bytes"] + max(m.t - B, 0) * stack.d_hidden * 2
@@ -154,6 +154,12 @@ def test_residual_rows_determine_the_output():
     rows_per_layer = 64 * stack.d_hidden * 2
     recip.arena[l0 * rows_per_layer:stack.n_layers * rows_per_layer].copy_(
         donor.arena[l0 * rows_per_layer:stack.n_layers * rows_per_layer])
+    # ... and with the rows their stored statistics (the third region of the arena: rows, positions,
+    # sums of squares, each starting at a 256-byte multiple)
+    slots = stack.n_layers * 64
+    ru = lambda x: (x + 255) // 256 * 256
+    ss0 = ru(slots * stack.d_hidden * 2) + ru(slots * 4)
+    recip.arena[ss0 + l0 * 64 * 4:ss0 + slots * 4].copy_(donor.arena[ss0 + l0 * 64 * 4:ss0 + slots * 4])
     # the next token: take the donor's row entering layer l0 and run layers l0.. on the recipient
     tok2 = 11
     h_d, out_d = _step_from_layer(donor, tok2, 0, None)
