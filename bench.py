@@ -594,12 +594,14 @@ def run_sweep(wl, peaks):
     from kvd_synth import make_layer_weights  # noqa: F401
     import paper_2603_19664_b200 as kvd
     desc = kvd.make_desc(1, shape.d_hidden, shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.rms_eps,
-                         shape.qk_norm, shape.rms_eps, shape.rope_style, 1, big_T + 8, 1)
+                         shape.qk_norm, shape.rms_eps, shape.rope_style, 5, big_T + 8, 1)
     ctx = kvd.Kvd(desc)
     ctx.kvd_set_layer(0, wl.w_kv, wl.g_in, wl.g_k, shape.rope_theta, 0)
     ws = torch.empty(kvd.kvd_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
     ctx.kvd_attach_workspace(ws)
     n_sets = 5
+    arena = torch.empty(kvd.kvd_store_bytes(desc, 1), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_store(arena, 1)
     X = [torch.randn((big_T, shape.d_hidden), device="cuda", dtype=torch.float32).to(torch.bfloat16) for _ in range(n_sets)]
     K = [torch.randn((big_T + 1, kdim), device="cuda", dtype=torch.float32).to(torch.bfloat16) for _ in range(n_sets)]
     V = [torch.randn((big_T + 1, kdim), device="cuda", dtype=torch.float32).to(torch.bfloat16) for _ in range(n_sets)]
@@ -607,6 +609,8 @@ def run_sweep(wl, peaks):
     Vo = torch.empty_like(Ko)
     dst = torch.empty((2, big_T, kdim), device="cuda", dtype=torch.bfloat16)
     pos = torch.arange(big_T, dtype=torch.int32, device="cuda")
+    for s_ in range(n_sets):  # the rows are recomputed from the store, as the method does (set = sequence slot)
+        ctx.kvd_checkpoint_residual(s_, 0, X[s_], pos, big_T)
     q = wl.q[:1]
     out = wl.out[:1]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
@@ -648,7 +652,7 @@ def run_sweep(wl, peaks):
 
     for T in (1, 10, 50, 100, 256, 500, 512, 1024, 2048, 4096, 8192, 16384, 32768):
         def f_rec(i):
-            ctx.kvd_recompute_kv(0, X[i % n_sets], pos, T, Ko, Vo, kdim)
+            ctx.kvd_recompute_kv(0, None, None, T, Ko, Vo, kdim, seq=i % n_sets, first_row=0)
 
         def f_att(i):
             ctx.kvd_decode_attention(0, 1, q, [T], [[(K[i % n_sets], V[i % n_sets], kdim, 0, T + 1)]], 0.0, out)

@@ -47,7 +47,7 @@ __global__ void __launch_bounds__(256) kvd_checkpoint_kernel(const uint4 *__rest
     const uint4 *const src[1] = {rows + off};
     uint4 *const dst[1] = {dst_rows + off};
     float ss[1];
-    warp_rows_sumsq<1, 8, true>(src, dst, row_chunks, lane, ss);
+    warp_rows_sumsq<1, 10, true>(src, dst, row_chunks, lane, ss);  // all of a 2560-wide row in flight at once
     if (lane == 0) {
       dst_sumsq[r] = ss[0];
       dst_pos[r] = pos[r];

@@ -258,7 +258,10 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   // overlap the tail of the preceding kernel; rows, positions and outputs are touched from here on.
   grid_launch_dependents();
   grid_dependency_wait();
-  if (threadIdx.x == 0) trace_put<TRACE>(p.trace, 0, 11);
+  if (threadIdx.x == 0) {
+    trace_put<TRACE>(p.trace, 0, 11);
+    if (TRACE) trace_put<TRACE>(p.trace, 0, 12, static_cast<long long>(globaltimer_ns()));
+  }
 
   if (warp == 2) {
     // ------------------------------------------------------------------ TMA producer
@@ -624,6 +627,10 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   // nobody may leave while the partner can still signal into this CTA's shared memory
   tc_fence_before();
   cluster_sync_all();
+  if (TRACE && threadIdx.x == 0) {
+    trace_put<TRACE>(p.trace, 0, 13, static_cast<long long>(globaltimer_ns()));
+    trace_put<TRACE>(p.trace, 0, 14);
+  }
   if (warp == 3) {
     tc_fence_after();
     tmem_dealloc_pair(tmem_base, Cfg::TMEM_COLS);
