@@ -185,7 +185,12 @@ kvd_status kvd_checkpoint_residual(kvd_ctx *ctx, int seq, int layer, const void 
  *   k_out, v_out: DEVICE bf16; row m, head h, channel c at [m*out_row_stride + h*d_head + c]
  *                 (out_row_stride in elements, multiple of 8, >= n_kv*d_head; bases 16-byte aligned).
  * n == 0 is a no-op.  Output bits for a row depend only on that row, its position and the layer,
- * never on n or on the row's index in the batch. */
+ * never on n, on the row's index in the batch, or on whether the row came from the store or from the
+ * caller.  Rows from the store use the statistic stored with them; for more than 64 caller rows the call
+ * first launches a small kernel that takes their statistics into a scratch of the context (calls on one
+ * context are stream-ordered by contract: they must not overlap on different streams).  Outputs whose
+ * bases are 32-byte aligned and whose row stride is a multiple of 16 elements are written with 32-byte
+ * stores (a little faster); 16-byte alignment is all that is required. */
 kvd_status kvd_recompute_kv(kvd_ctx *ctx, int layer, const void *rows, const int32_t *positions, int n, int seq,
                             int first_row, void *k_out, void *v_out, int64_t out_row_stride, void *stream);
 
