@@ -187,6 +187,63 @@ def test_checkpoint_store_roundtrip_and_recompute_from_store():
     assert ctx.kvd_rows_stored(0, 1) == 0
 
 
+def test_row_statistic_kept_in_the_store_is_the_sum_of_squares():
+    """The third region of the arena (rows, positions, sums of squares, each starting at a 256-byte
+    multiple) holds the RMSNorm statistic of Eq. 2 for every checkpointed row."""
+    shape = GEMMA3_4B_GLOBAL
+    max_tokens, n = 384, 300
+    desc = kvd.make_desc(1, shape.d_hidden, shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.rms_eps,
+                         shape.qk_norm, shape.rms_eps, shape.rope_style, 2, max_tokens, 1)
+    ctx = kvd.Kvd(desc)
+    arena = torch.zeros(kvd.kvd_store_bytes(desc, 1), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_store(arena, 1)
+    X = make_residuals(shape, n, seed=17, outliers=True)
+    pos = np.arange(n) + 3
+    x, p = dev(X), torch.from_numpy(pos.astype(np.int32)).cuda()
+    ctx.kvd_checkpoint_residual(1, 0, x[:7], p[:7], 7)      # two appends to sequence slot 1
+    ctx.kvd_checkpoint_residual(1, 0, x[7:], p[7:], n - 7)
+    torch.cuda.synchronize()
+    slots = 2 * max_tokens
+    ru = lambda b: (b + 255) // 256 * 256
+    rows_bytes, pos_bytes = ru(slots * shape.d_hidden * 2), ru(slots * 4)
+    assert arena.numel() == rows_bytes + 2 * pos_bytes
+    a = arena.cpu().numpy()
+    got_rows = a[:rows_bytes].view(np.uint16).reshape(-1, shape.d_hidden)[max_tokens:max_tokens + n]
+    got_pos = a[rows_bytes:rows_bytes + pos_bytes].view(np.int32)[max_tokens:max_tokens + n]
+    got_ss = a[rows_bytes + pos_bytes:].view(np.float32)[max_tokens:max_tokens + n]
+    assert np.array_equal(got_rows, X) and np.array_equal(got_pos, pos)
+    from kvd_synth import bf16_to_f64
+    ref = np.sum(bf16_to_f64(X) ** 2, axis=1)
+    assert np.max(np.abs(got_ss - ref) / ref) < 1e-6   # fp32 accumulation of 2560 exact squares
+
+
+@pytest.mark.parametrize("shape", [SMOLLM2_135M, GEMMA3_4B_GLOBAL], ids=lambda s: s.name)
+def test_output_bits_do_not_depend_on_output_alignment_or_row_count_path(shape):
+    """32-byte-aligned outputs take 32-byte stores, others 16-byte stores; 1..64 caller rows have their
+    statistics taken inside the kernel, more by a kernel of their own: the bits must not change."""
+    ctx, w = open_layer(shape, max_tokens=1024)
+    kdim = shape.n_kv_heads * shape.d_head
+    T = 300
+    X = make_residuals(shape, T, seed=18, outliers=True)
+    pos = np.arange(T) + 40
+    K, V = run_gpu(ctx, shape, X, pos)
+    Kb, Vb = host_bits(K), host_bits(V)
+    for n in (1, 3, 33, 64, 65, 129, T):
+        x, p = dev(X[:n]), torch.from_numpy(pos[:n].astype(np.int32)).cuda()
+        stride = kdim + 8                       # rows 16-byte but not 32-byte aligned
+        kbuf = torch.full((n * stride + 8,), -7.0, dtype=torch.bfloat16, device="cuda")
+        vbuf = torch.full((n * stride + 8,), -7.0, dtype=torch.bfloat16, device="cuda")
+        ctx._check(ctx._lib.kvd_recompute_kv(ctx._h, 0, x.data_ptr(), p.data_ptr(), n, 0, 0, kbuf.data_ptr() + 16,
+                                             vbuf.data_ptr() + 16, stride, None), "kvd_recompute_kv")
+        assert ctx.kvd_poll_status() == kvd.KVD_OK
+        k = host_bits(kbuf[8:].view(n, stride))
+        v = host_bits(vbuf[8:].view(n, stride))
+        assert np.array_equal(k[:, :kdim], Kb[:n]) and np.array_equal(v[:, :kdim], Vb[:n]), n
+        pad = host_bits(torch.full((1,), -7.0, dtype=torch.bfloat16))[0]
+        assert np.all(k[:, kdim:] == pad) and np.all(v[:, kdim:] == pad)   # nothing written between rows
+        assert host_bits(kbuf[:8]).tolist() == [pad] * 8
+
+
 @pytest.mark.parametrize("shape", [SMOLLM2_135M, GEMMA3_4B_GLOBAL], ids=lambda s: s.name)
 def test_step_call_matches_separate_calls_bit_for_bit(shape):
     """kvd_recompute_kv_step: ranges of three sequences (ragged, non-zero first rows, one empty) plus
