@@ -234,6 +234,31 @@ kvd_status kvd_recompute_kv_step(kvd_ctx *ctx, int layer, const kvd_store_range 
 kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, const void *q, const int32_t *q_pos,
                                 const kvd_kv_segment *segs, int n_segs, float scale, void *out, void *stream);
 
+/* RECOMPUTE_KV and ATTENTION of Algorithm 1 in one pass for the evicted tokens (Eq. 13-14 feeding
+ * Eq. 6-7): the keys and values rebuilt from the residual rows of ranges[b] are consumed inside the
+ * recompute kernel -- the rotated key of a row is multiplied with the queries of its KV head, the value
+ * tile is produced transposed and summed over rows with the softmax weights -- and never written to
+ * memory.  The result for sequence b is attention over [keys recomputed from ranges[b]] united with the
+ * live segments segs[b][*] (window, current token), as kvd_recompute_kv_step followed by
+ * kvd_decode_attention would give it, up to rounding: the recomputed part is split by 256-row blocks
+ * instead of position chunks and its values are not rounded to bf16 on the way, so the bits differ from
+ * the two-call path (same tolerances against the definition).  Use the two-call path where bit-identical
+ * outputs across cache policies are required.
+ *   ranges  HOST [batch]: rows first_row .. first_row+n-1 of the store of (layer, ranges[b].seq); k_out and
+ *           v_out are ignored; n == 0 leaves a sequence with its live segments only.  Visibility of a
+ *           recomputed key follows its stored position (<= q_pos[b], inside the layer's window).
+ *   rows, positions, n_rows, k_rows_out, v_rows_out, out_row_stride: the new tokens, exactly as in
+ *           kvd_recompute_kv_step -- their K and V ARE written (the live segments usually point at them).
+ *   q, q_pos, segs, n_segs, scale, out: as in kvd_decode_attention; batch <= KVD_MAX_STORE_RANGES.
+ * Three launches (recompute+attend, live segments, merge).  KVD_ERR_UNSUPPORTED, with nothing launched,
+ * for shapes the fused kernel is not built for (it exists for 256-column tiles with d_head 256 and 1 or 2
+ * query heads per KV head, or d_head 128 and 1, 2 or 4); needs the store and the workspace attached. */
+kvd_status kvd_decode_attention_recompute(kvd_ctx *ctx, int layer, int batch, const void *q, const int32_t *q_pos,
+                                          const kvd_store_range *ranges, const void *rows,
+                                          const int32_t *positions, int n_rows, void *k_rows_out, void *v_rows_out,
+                                          int64_t out_row_stride, const kvd_kv_segment *segs, int n_segs,
+                                          float scale, void *out, void *stream);
+
 /* No counterpart in the paper: the same decode attention as kvd_decode_attention for callers that
  * cannot allocate device memory at all -- code running inside someone else's memory pool or under a
  * fixed memory budget, a plug-in whose host forbids cudaMalloc after start-up, a process that must

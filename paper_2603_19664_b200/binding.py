@@ -31,6 +31,7 @@ KVD_MAX_SEGMENTS = 4
 # every symbol include/kvd.h declares
 EXPORTED_SYMBOLS = (
     "kvd_create", "kvd_destroy", "kvd_set_layer", "kvd_store_bytes", "kvd_attach_store", "kvd_reset_sequence",
+    "kvd_decode_attention_recompute",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
     "kvd_recompute_kv_step",
     "kvd_decode_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
@@ -119,6 +120,10 @@ def load() -> ctypes.CDLL:
     lib.kvd_decode_attention.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
                                          ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
     lib.kvd_decode_attention.restype = i32
+    lib.kvd_decode_attention_recompute.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
+                                                   ctypes.POINTER(kvd_store_range), vp, vp, i32, vp, vp, i64,
+                                                   ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
+    lib.kvd_decode_attention_recompute.restype = i32
     lib.kvd_decode_attention_static.argtypes = [i32, i32, i32, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
                                                 ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
     lib.kvd_decode_attention_static.restype = i32
@@ -305,6 +310,22 @@ class Kvd:
                     e.k, e.v, e.row_stride, e.first_pos, e.len = None, None, 0, 0, 0
         self._check(self._lib.kvd_decode_attention(self._h, layer, batch, _ptr(q), pos_arr, seg_arr, n_segs,
                                                    float(scale), _ptr(out), _stream(stream)), "kvd_decode_attention")
+
+    def kvd_decode_attention_recompute(self, layer: int, batch: int, q, q_pos: Sequence[int],
+                                       ranges: Sequence[Tuple[int, int, int]], rows, positions, n_rows: int,
+                                       k_rows_out, v_rows_out, out_row_stride: int,
+                                       segs: Sequence[Sequence[Segment]], scale: float, out, stream=None) -> None:
+        """ranges: (seq, first_row, n) per sequence -- attended inside the recompute kernel; rows/positions:
+        the new tokens (their K/V are written); segs: the live segments, as for kvd_decode_attention."""
+        n_segs, pos_arr, seg_arr = _marshal_segments(batch, q_pos, segs)
+        arr = (kvd_store_range * max(len(ranges), 1))()
+        for i, (seq, first_row, n) in enumerate(ranges):
+            arr[i].seq, arr[i].first_row, arr[i].n, arr[i].reserved = int(seq), int(first_row), int(n), 0
+            arr[i].k_out, arr[i].v_out = None, None
+        self._check(self._lib.kvd_decode_attention_recompute(
+            self._h, layer, batch, _ptr(q), pos_arr, arr, _ptr(rows), _ptr(positions), n_rows, _ptr(k_rows_out),
+            _ptr(v_rows_out), out_row_stride, seg_arr, n_segs, float(scale), _ptr(out), _stream(stream)),
+            "kvd_decode_attention_recompute")
 
     def kvd_memory_stats(self) -> dict:
         ms = kvd_mem_stats()

@@ -71,7 +71,9 @@ extern "C" size_t kvd_store_bytes(const kvd_model_desc *d, int layers_stored) {
 
 // chunk partials of one sequence
 static size_t parts_per_seq(const kvd_model_desc *d) {
-  return attn_max_chunks(d->d_head, d->n_kv_heads, d->max_tokens_per_seq);
+  // the streaming kernel's chunks plus, for kvd_decode_attention_recompute, one partial per 256-row block
+  // of a recomputed range
+  return attn_max_chunks(d->d_head, d->n_kv_heads, d->max_tokens_per_seq) + (d->max_tokens_per_seq + 255) / 256;
 }
 
 extern "C" size_t kvd_workspace_bytes(const kvd_model_desc *d) {
@@ -355,15 +357,19 @@ extern "C" kvd_status kvd_checkpoint_residual(kvd_ctx *ctx, int seq, int layer, 
 
 // Shared body of kvd_recompute_kv and kvd_recompute_kv_step: validate, build the job table (store
 // ranges first, then the caller's rows), launch once.
+// With `fused` (one RcAttend per range, q == nullptr for a range that is to be stored as usual) the
+// ranges that carry a query are attended inside the kernel instead of being written.
 static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
                                    const void *rows, const int32_t *positions, int n_rows, void *k_rows_out,
-                                   void *v_rows_out, int64_t out_row_stride, cudaStream_t stream) {
+                                   void *v_rows_out, int64_t out_row_stride, cudaStream_t stream,
+                                   const RcAttend *fused = nullptr, const AttnLaunchHead *fused_head = nullptr) {
   const LayerState &ls = ctx->layers[layer];
   const kvd_model_desc &d = ctx->desc;
   const int kdim = d.n_kv_heads * d.d_head;
   if (out_row_stride < kdim) return KVD_ERR_INVALID_ARG;
   if (out_row_stride % 8 != 0) return KVD_ERR_ALIGNMENT;
   RecomputeParams p;
+  static thread_local FusedParams fp;  // large: keep it off the stack
   int n_jobs = 0, mb = 0;
   bool any_store = false;
   for (int i = 0; i < n_ranges; ++i) {
@@ -372,8 +378,12 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
     if (r.n == 0) continue;
     if (!ctx->store_rows) return KVD_ERR_STATE;
     if (r.seq < 0 || r.seq >= d.max_seqs || layer >= ctx->layers_stored || r.first_row < 0) return KVD_ERR_INVALID_ARG;
-    if (!r.k_out || !r.v_out) return KVD_ERR_INVALID_ARG;
-    if (!aligned16(r.k_out) || !aligned16(r.v_out)) return KVD_ERR_ALIGNMENT;
+    const bool attends = fused && fused[i].q != nullptr;
+    if (!attends) {
+      if (!r.k_out || !r.v_out) return KVD_ERR_INVALID_ARG;
+      if (!aligned16(r.k_out) || !aligned16(r.v_out)) return KVD_ERR_ALIGNMENT;
+    }
+    if (fused) fp.att[n_jobs] = fused[i];
     const int have = ctx->rows_stored[static_cast<size_t>(layer) * d.max_seqs + r.seq];
     if (r.first_row > have || r.n > have - r.first_row) return KVD_ERR_CAPACITY;
     RcJob &J = p.jobs[n_jobs++];
@@ -394,6 +404,7 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
     if (!aligned16(rows) || !aligned16(k_rows_out) || !aligned16(v_rows_out)) return KVD_ERR_ALIGNMENT;
     kvd_status st = encode_rows_3d(ctx, &tmap_rows, rows, d.d_hidden, static_cast<uint64_t>(n_rows), 1);
     if (st != KVD_OK) return st;
+    if (fused) fp.att[n_jobs].q = nullptr;  // the caller's rows are stored
     RcJob &J = p.jobs[n_jobs++];
     J.mb_start = mb;
     J.n = n_rows;
@@ -445,6 +456,13 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
     const size_t ctas = 2 * static_cast<size_t>(tiles < ctx->num_sms / 2 ? tiles : ctx->num_sms / 2);
     if (ctas * RC_TRACE_TILES * RC_TRACE_FIELDS * sizeof(long long) <= ctx->trace_bytes) p.trace = ctx->trace;
   }
+  if (fused) {
+    fp.part_o = fused_head->part_o;
+    fp.part_ml = fused_head->part_ml;
+    fp.n_q = fused_head->n_q;
+    fp.scale_log2e = fused_head->scale_log2e;
+    return launch_recompute_fused(ctx, ls, tmap_store, tmap_ext, p, fp, stream);
+  }
   return launch_recompute(ctx, ls, tmap_store, tmap_ext, p, stream);
 }
 
@@ -484,22 +502,11 @@ extern "C" kvd_status kvd_recompute_kv_step(kvd_ctx *ctx, int layer, const kvd_s
                           static_cast<cudaStream_t>(stream_));
 }
 
-extern "C" kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, const void *q, const int32_t *q_pos,
-                                           const kvd_kv_segment *segs, int n_segs, float scale, void *out,
-                                           void *stream_) {
-  if (!ctx || batch < 0 || n_segs < 0 || n_segs > KVD_MAX_SEGMENTS) return KVD_ERR_INVALID_ARG;
-  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
-  const LayerState &ls = ctx->layers[layer];
-  if (!ls.set) return KVD_ERR_STATE;
-  if (!ctx->part_o) return KVD_ERR_STATE;
-  if (batch == 0) return KVD_OK;
-  if (!q || !q_pos || !out || (n_segs > 0 && !segs)) return KVD_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(out)) return KVD_ERR_ALIGNMENT;
+// Validate the segments of `batch` sequences (nothing is launched on an error).
+static kvd_status check_segments(const kvd_ctx *ctx, int batch, const int32_t *q_pos, const kvd_kv_segment *segs,
+                                 int n_segs) {
   const kvd_model_desc &d = ctx->desc;
-  if (batch > d.max_batch) return KVD_ERR_CAPACITY;
   const int kdim = d.n_kv_heads * d.d_head;
-  const int group = d.n_q_heads / d.n_kv_heads;
-  // ---- validate every segment before anything is launched
   for (int b = 0; b < batch; ++b) {
     if (q_pos[b] < 0) return KVD_ERR_INVALID_ARG;
     for (int s = 0; s < n_segs; ++s) {
@@ -516,70 +523,156 @@ extern "C" kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, c
       }
     }
   }
+  return KVD_OK;
+}
+
+// Describe one launch over sequences b0 .. b0 + nb - 1 (nb <= AT_MAX_SEQS): segments, visible range, the
+// split into chunks and the slots of the partial arrays.  pre_parts[b] (may be NULL) slots are left
+// in front of a sequence's chunks for partials that another kernel writes (fused recompute); the
+// merge kernel combines them with the chunks, in slot order.
+static kvd_status build_attn_launch(kvd_ctx *ctx, const LayerState &ls, int b0, int nb, const void *q,
+                                    const int32_t *q_pos, const kvd_kv_segment *segs, int n_segs, float scale,
+                                    void *out, const int *pre_parts, AttnLaunch &L) {
+  const kvd_model_desc &d = ctx->desc;
+  int parts = 0, slots = 0;
+  for (int i = 0; i < nb; ++i) {
+    const int b = b0 + i;
+    AttnSeq &S = L.seq[i];
+    int min_first = INT32_MAX, max_last = -1;
+    for (int s = 0; s < KVD_MAX_SEGMENTS; ++s) {
+      S.k[s] = S.v[s] = nullptr;
+      S.stride[s] = 0;
+      S.first[s] = 0;
+      S.len[s] = 0;
+      if (s < n_segs) {
+        const kvd_kv_segment &sg = segs[static_cast<size_t>(b) * n_segs + s];
+        if (sg.len > 0) {
+          S.k[s] = static_cast<const __nv_bfloat16 *>(sg.k);
+          S.v[s] = static_cast<const __nv_bfloat16 *>(sg.v);
+          S.stride[s] = sg.row_stride;
+          S.first[s] = sg.first_pos;
+          S.len[s] = sg.len;
+          if (sg.first_pos < min_first) min_first = sg.first_pos;
+          if (sg.first_pos + sg.len - 1 > max_last) max_last = sg.first_pos + sg.len - 1;
+        }
+      }
+    }
+    S.q_pos = q_pos[b];
+    int lo = ls.window > 0 ? S.q_pos - ls.window + 1 : 0;
+    if (lo < 0) lo = 0;
+    if (min_first > lo) lo = min_first;
+    int hi = S.q_pos < max_last ? S.q_pos : max_last;
+    S.lo_pos = lo;
+    S.hi_pos = hi;
+    S.part_base = parts;
+    if (max_last < 0 || hi < lo) {
+      S.n_chunks = 0;
+      S.iters = 1;
+      S.chunk0_pos = 0;
+    } else {
+      // the split depends on the visible position range only
+      S.iters = attn_iters_for_span(d.d_head, d.n_kv_heads, hi - lo + 1);
+      const int ck = attn_chunk_keys(d.d_head, S.iters);
+      S.chunk0_pos = lo / ck * ck;
+      S.n_chunks = hi / ck - lo / ck + 1;
+    }
+    const int pre = pre_parts ? pre_parts[b] : 0;
+    S.merge_base = slots;
+    S.slot_base = slots + pre;
+    S.merge_count = pre + S.n_chunks;
+    slots += S.merge_count;
+    parts += S.n_chunks;
+  }
+  if (slots > ctx->max_parts) return KVD_ERR_CAPACITY;
   const float sc = scale > 0.f ? scale : 1.0f / sqrtf(static_cast<float>(d.d_head));
+  L.n_seqs = nb;
+  L.total_chunks = parts;
+  L.n_q = d.n_q_heads;
+  L.n_kv = d.n_kv_heads;
+  L.q = static_cast<const __nv_bfloat16 *>(q) + static_cast<size_t>(b0) * d.n_q_heads * d.d_head;
+  L.out = static_cast<__nv_bfloat16 *>(out) + static_cast<size_t>(b0) * d.n_q_heads * d.d_head;
+  L.part_o = ctx->part_o;
+  L.part_ml = ctx->part_ml;
+  L.scale_log2e = sc * 1.4426950408889634f;
+  return KVD_OK;
+}
+
+extern "C" kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, const void *q, const int32_t *q_pos,
+                                           const kvd_kv_segment *segs, int n_segs, float scale, void *out,
+                                           void *stream_) {
+  if (!ctx || batch < 0 || n_segs < 0 || n_segs > KVD_MAX_SEGMENTS) return KVD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  const LayerState &ls = ctx->layers[layer];
+  if (!ls.set) return KVD_ERR_STATE;
+  if (!ctx->part_o) return KVD_ERR_STATE;
+  if (batch == 0) return KVD_OK;
+  if (!q || !q_pos || !out || (n_segs > 0 && !segs)) return KVD_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out)) return KVD_ERR_ALIGNMENT;
+  const kvd_model_desc &d = ctx->desc;
+  if (batch > d.max_batch) return KVD_ERR_CAPACITY;
+  const int group = d.n_q_heads / d.n_kv_heads;
+  kvd_status st = check_segments(ctx, batch, q_pos, segs, n_segs);
+  if (st != KVD_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   static thread_local AttnLaunch L;  // large: keep it off the stack
   for (int b0 = 0; b0 < batch; b0 += AT_MAX_SEQS) {
     const int nb = batch - b0 < AT_MAX_SEQS ? batch - b0 : AT_MAX_SEQS;
-    int parts = 0;
-    for (int i = 0; i < nb; ++i) {
-      const int b = b0 + i;
-      AttnSeq &S = L.seq[i];
-      int min_first = INT32_MAX, max_last = -1;
-      for (int s = 0; s < KVD_MAX_SEGMENTS; ++s) {
-        S.k[s] = S.v[s] = nullptr;
-        S.stride[s] = 0;
-        S.first[s] = 0;
-        S.len[s] = 0;
-        if (s < n_segs) {
-          const kvd_kv_segment &sg = segs[static_cast<size_t>(b) * n_segs + s];
-          if (sg.len > 0) {
-            S.k[s] = static_cast<const __nv_bfloat16 *>(sg.k);
-            S.v[s] = static_cast<const __nv_bfloat16 *>(sg.v);
-            S.stride[s] = sg.row_stride;
-            S.first[s] = sg.first_pos;
-            S.len[s] = sg.len;
-            if (sg.first_pos < min_first) min_first = sg.first_pos;
-            if (sg.first_pos + sg.len - 1 > max_last) max_last = sg.first_pos + sg.len - 1;
-          }
-        }
-      }
-      S.q_pos = q_pos[b];
-      int lo = ls.window > 0 ? S.q_pos - ls.window + 1 : 0;
-      if (lo < 0) lo = 0;
-      if (min_first > lo) lo = min_first;
-      int hi = S.q_pos < max_last ? S.q_pos : max_last;
-      S.lo_pos = lo;
-      S.hi_pos = hi;
-      S.part_base = parts;
-      if (max_last < 0 || hi < lo) {
-        S.n_chunks = 0;
-        S.iters = 1;
-        S.chunk0_pos = 0;
-      } else {
-        // the split depends on the visible position range only
-        S.iters = attn_iters_for_span(d.d_head, d.n_kv_heads, hi - lo + 1);
-        const int ck = attn_chunk_keys(d.d_head, S.iters);
-        S.chunk0_pos = lo / ck * ck;
-        S.n_chunks = hi / ck - lo / ck + 1;
-      }
-      parts += S.n_chunks;
-    }
-    if (parts > ctx->max_parts) return KVD_ERR_CAPACITY;
-    L.n_seqs = nb;
-    L.total_chunks = parts;
-    L.n_q = d.n_q_heads;
-    L.n_kv = d.n_kv_heads;
-    L.q = static_cast<const __nv_bfloat16 *>(q) + static_cast<size_t>(b0) * d.n_q_heads * d.d_head;
-    L.out = static_cast<__nv_bfloat16 *>(out) + static_cast<size_t>(b0) * d.n_q_heads * d.d_head;
-    L.part_o = ctx->part_o;
-    L.part_ml = ctx->part_ml;
-    L.scale_log2e = sc * 1.4426950408889634f;
+    st = build_attn_launch(ctx, ls, b0, nb, q, q_pos, segs, n_segs, scale, out, nullptr, L);
+    if (st != KVD_OK) return st;
     // sequences without a visible key stream nothing; the merge kernel writes their zeros
-    kvd_status st = launch_attention(ctx, L, d.d_head, group, stream);
+    st = launch_attention(ctx, L, d.d_head, group, stream);
     if (st != KVD_OK) return st;
   }
   return KVD_OK;
+}
+
+// Decode attention over [K/V recomputed from store ranges] + [live segments], the recomputed part
+// inside the recompute kernel (its K/V never reach memory); see kvd.h.
+extern "C" kvd_status kvd_decode_attention_recompute(kvd_ctx *ctx, int layer, int batch, const void *q,
+                                                     const int32_t *q_pos, const kvd_store_range *ranges,
+                                                     const void *rows, const int32_t *positions, int n_rows,
+                                                     void *k_rows_out, void *v_rows_out, int64_t out_row_stride,
+                                                     const kvd_kv_segment *segs, int n_segs, float scale,
+                                                     void *out, void *stream_) {
+  if (!ctx || batch < 0 || n_segs < 0 || n_segs > KVD_MAX_SEGMENTS || n_rows < 0) return KVD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  const LayerState &ls = ctx->layers[layer];
+  if (!ls.set) return KVD_ERR_STATE;
+  if (!ctx->part_o || !ctx->store_rows) return KVD_ERR_STATE;
+  const kvd_model_desc &d = ctx->desc;
+  const int group = d.n_q_heads / d.n_kv_heads, kdim = d.n_kv_heads * d.d_head;
+  // shapes the fused kernel is built for (nothing is launched otherwise)
+  if (ctx->block_n != 256 || kdim % 256 != 0 || !((d.d_head == 256 && (group == 1 || group == 2)) ||
+                                                   (d.d_head == 128 && (group == 1 || group == 2 || group == 4))))
+    return KVD_ERR_UNSUPPORTED;
+  if (batch == 0 && n_rows == 0) return KVD_OK;
+  if (batch > 0 && (!q || !q_pos || !out || !ranges || (n_segs > 0 && !segs))) return KVD_ERR_INVALID_ARG;
+  if (batch > 0 && (!aligned16(q) || !aligned16(out))) return KVD_ERR_ALIGNMENT;
+  if (batch > d.max_batch || batch > KVD_MAX_STORE_RANGES) return KVD_ERR_CAPACITY;
+  kvd_status st = check_segments(ctx, batch, q_pos, segs, n_segs);
+  if (st != KVD_OK) return st;
+  int pre[KVD_MAX_STORE_RANGES];
+  for (int b = 0; b < batch; ++b) {
+    if (ranges[b].n < 0) return KVD_ERR_INVALID_ARG;
+    pre[b] = (ranges[b].n + 2 * RC_BLOCK_M - 1) / (2 * RC_BLOCK_M);  // one partial per 256-row block
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  static thread_local AttnLaunch L;  // large: keep it off the stack
+  st = build_attn_launch(ctx, ls, 0, batch, q, q_pos, segs, n_segs, scale, out, pre, L);
+  if (st != KVD_OK) return st;
+  RcAttend att[KVD_MAX_STORE_RANGES];
+  for (int b = 0; b < batch; ++b) {
+    att[b].q = static_cast<const __nv_bfloat16 *>(q) + static_cast<size_t>(b) * d.n_q_heads * d.d_head;
+    att[b].q_pos = q_pos[b];
+    att[b].lo_pos = ls.window > 0 && q_pos[b] - ls.window + 1 > 0 ? q_pos[b] - ls.window + 1 : 0;
+    att[b].part_base = L.seq[b].merge_base;
+    att[b].reserved = 0;
+  }
+  st = recompute_launch(ctx, layer, ranges, batch, rows, positions, n_rows, k_rows_out, v_rows_out,
+                        out_row_stride > 0 ? out_row_stride : kdim, stream, att, &L);
+  if (st != KVD_OK) return st;
+  if (batch == 0) return KVD_OK;
+  return launch_attention(ctx, L, d.d_head, group, stream);
 }
 
 extern "C" kvd_status kvd_memory_stats(const kvd_ctx *ctx, kvd_mem_stats *out) {

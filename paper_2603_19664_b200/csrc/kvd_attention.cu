@@ -292,7 +292,7 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM) kvd_attn_split_ker
     }
   }
   __syncthreads();
-  const size_t pidx = static_cast<size_t>(S.part_base + chunk);
+  const size_t pidx = static_cast<size_t>(S.slot_base + chunk);
   for (int idx = threadIdx.x; idx < G * D_HEAD; idx += AT_THREADS) {
     const int g = idx / D_HEAD, c = idx % D_HEAD;
     float M = -CUDART_INF_F;
@@ -527,7 +527,7 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM)
     }
   }
   __syncthreads();
-  const size_t pidx = static_cast<size_t>(S.part_base + chunk);
+  const size_t pidx = static_cast<size_t>(S.slot_base + chunk);
   for (int idx = threadIdx.x; idx < G * D_HEAD; idx += AT_THREADS) {
     const int g = idx / D_HEAD, c = idx % D_HEAD;
     float M = -CUDART_INF_F;
@@ -580,11 +580,11 @@ __global__ void __launch_bounds__(AT_MERGE_THREADS)
   // partials are visible
   grid_dependency_wait();
 
-  const int count = S.n_chunks;
+  const int count = S.merge_count;
   const int n_groups = (count + PF - 1) / PF;
   const int warps_used = n_groups < AT_MERGE_WARPS ? n_groups : AT_MERGE_WARPS;
-  const float *ml0 = P.part_ml + (static_cast<size_t>(S.part_base) * P.n_q + kvh * G) * 2;
-  const float *po0 = P.part_o + (static_cast<size_t>(S.part_base) * P.n_q + kvh * G) * D_HEAD +
+  const float *ml0 = P.part_ml + (static_cast<size_t>(S.merge_base) * P.n_q + kvh * G) * 2;
+  const float *po0 = P.part_o + (static_cast<size_t>(S.merge_base) * P.n_q + kvh * G) * D_HEAD +
                      slice * AT_MERGE_SLICE + lane * 2;
   const size_t ml_stride = static_cast<size_t>(P.n_q) * 2, po_stride = static_cast<size_t>(P.n_q) * D_HEAD;
   if (warp < warps_used) {
@@ -718,7 +718,7 @@ static cudaError_t attn_launch_pair(const AttnLaunchT<NSEQ> &S, cudaStream_t str
   attr[0].val.programmaticStreamSerializationAllowed = (small && !(serial_launch_mask() & 4)) ? 1 : 0;
   // as many warps per merge CTA as the longest sequence of the launch has groups of partials
   int max_chunks = 1;
-  for (int i = 0; i < S.n_seqs; ++i) max_chunks = S.seq[i].n_chunks > max_chunks ? S.seq[i].n_chunks : max_chunks;
+  for (int i = 0; i < S.n_seqs; ++i) max_chunks = S.seq[i].merge_count > max_chunks ? S.seq[i].merge_count : max_chunks;
   int merge_warps = (max_chunks + attn_merge_group(G) - 1) / attn_merge_group(G);
   if (merge_warps > AT_MERGE_WARPS) merge_warps = AT_MERGE_WARPS;
   cfg.gridDim = dim3(S.n_seqs * S.n_kv * (D_HEAD / AT_MERGE_SLICE), 1, 1);
@@ -909,6 +909,8 @@ extern "C" kvd_status kvd_decode_attention_static(int n_q_heads, int n_kv_heads,
       S.chunk0_pos = lo / ck * ck;
       S.n_chunks = hi / ck - lo / ck + 1;
     }
+    S.slot_base = S.merge_base = S.part_base;
+    S.merge_count = S.n_chunks;
     parts += S.n_chunks;
   }
   // one partial per chunk

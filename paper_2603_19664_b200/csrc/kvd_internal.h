@@ -71,6 +71,24 @@ struct RecomputeParams {
   RcJob jobs[RC_MAX_JOBS];
 };
 
+// Fused recompute + attention (the recomputed K/V of a store range are consumed inside the kernel and
+// never written): per job, the query of the range's sequence and where its partials go.
+struct RcAttend {
+  const __nv_bfloat16 *q;  // [n_q][d_head] of the job's sequence; nullptr: plain job, K and V are stored
+  int q_pos;               // position of the query
+  int lo_pos;              // first visible position (sliding window), 0 without a window
+  int part_base;           // slot of the job's first 256-row block in the partial arrays
+  int reserved;
+};
+struct FusedParams {
+  float *part_o;   // [slot][n_q][d_head] unnormalised outputs
+  float *part_ml;  // [slot][n_q][2] (max in log2 units, sum)
+  int n_q;
+  float scale_log2e;
+  RcAttend att[RC_MAX_JOBS];
+};
+struct NoFusedParams {};
+
 // ------------------------------------------------------------------------------ decode attention
 constexpr int AT_THREADS = 128;        // streaming kernel
 constexpr int AT_WARPS = 4;
@@ -94,8 +112,11 @@ struct AttnSeq {
   int hi_pos;       // last visible position (<= q_pos)
   int chunk0_pos;   // position of the first key of chunk 0 (multiple of the chunk size)
   int n_chunks;
-  int part_base;    // index of this sequence's first partial in the scratch
+  int part_base;    // chunks of the sequences before this one in the launch (the flattened grid)
   int iters;        // warp iterations per chunk
+  int slot_base;    // slot of this sequence's chunk 0 in the partial arrays
+  int merge_base;   // first slot and number of slots the merge kernel combines for this sequence: the
+  int merge_count;  // streaming kernel's chunks, preceded by partials of the fused recompute kernel if any
 };
 
 // Launch-wide fields, followed by the per-sequence descriptors.  The kernel takes the variant whose
@@ -219,6 +240,9 @@ inline int serial_launch_mask() {
 // launchers implemented next to their kernels
 kvd_status launch_recompute(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
                             const CUtensorMap &tmap_rows, const RecomputeParams &p, cudaStream_t stream);
+kvd_status launch_recompute_fused(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
+                                  const CUtensorMap &tmap_rows, const RecomputeParams &p, const FusedParams &fp,
+                                  cudaStream_t stream);
 kvd_status launch_attention(kvd_ctx *ctx, const AttnLaunch &L, int d_head, int group, cudaStream_t stream);
 kvd_status launch_prepare_weights(kvd_ctx *ctx, const __nv_bfloat16 *w, const __nv_bfloat16 *gamma, __nv_bfloat16 *wt,
                                   int d_hidden, int n_cols, cudaStream_t stream);

@@ -35,24 +35,38 @@
 // (warp_row_sumsq), the key norm is reduced by the single thread that owns the row, and cos/sin
 // depend on (position, channel) only.  A row's output bits are therefore independent of M, of the
 // row's index and of whether it came from the store or from the caller.
+#include <math_constants.h>
 #include <string.h>
+
+#include <type_traits>
 
 #include "kvd_internal.h"
 #include "kvd_ptx.cuh"
 
 namespace kvd {
 
-template <int BLOCK_N, int D_HEAD>
+// FG = 0: the plain kernel (K and V are stored).  FG > 0: the fused variant for models with FG query
+// heads per KV head -- jobs that carry a query attend over their rows inside the kernel (see the
+// epilogue); it gives one ring stage to the score buffers.
+template <int BLOCK_N, int D_HEAD, int FG = 0>
 struct RcCfg {
-  static constexpr int STAGES = BLOCK_N == 256 ? 7 : 9;  // all the shared memory an SM has: the ring is latency-bound
+  static constexpr bool FUSED = FG > 0;
+  static constexpr int STAGES = FUSED ? 6 : (BLOCK_N == 256 ? 7 : 9);  // all the shared memory an SM has: the ring is latency-bound
   static constexpr int A_BYTES = RC_BLOCK_M * RC_BLOCK_K * 2;
   static constexpr int B_ROWS = BLOCK_N / 2;  // this CTA's half of the W' tile
   static constexpr int B_BYTES = B_ROWS * RC_BLOCK_K * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = 2 * BLOCK_N;
   // barriers: full[S] (used in the even CTA), empty[S], tmem_full[2], tmem_empty[2], stats_full[2], rstd_free[2]
-  static constexpr int NUM_BARS = 2 * STAGES + 9;  // + stats_x: the four statistics warps among themselves
-  static constexpr int TAIL_BYTES = NUM_BARS * 8 + 16 /*tmem ptr, abort*/ + 2 * RC_BLOCK_M * 4 /*rstd*/ + 256 * 4 /*gamma_k*/;
+  // + stats_x (the four statistics warps among themselves); fused: + scores[2] (both CTAs' epilogue
+  // threads), epi (the four epilogue warps among themselves)
+  static constexpr int NUM_BARS = 2 * STAGES + 9 + (FUSED ? 3 : 0);
+  static constexpr int BAR_BYTES = (NUM_BARS * 8 + 15) / 16 * 16;
+  // fused: scores / weights [2 units][heads of the tile x FG][256 rows of the pair], 1/rms of the 256 rows
+  // [2 units][256], partial sums of the weights [heads x FG][4 warps]
+  static constexpr int GT = (BLOCK_N / D_HEAD) * (FUSED ? FG : 0);
+  static constexpr int FUSED_BYTES = FUSED ? (2 * GT * 256 + 2 * 256 + GT * 4) * 4 : 0;
+  static constexpr int TAIL_BYTES = BAR_BYTES + 16 /*tmem ptr, abort*/ + 2 * RC_BLOCK_M * 4 /*rstd*/ + 256 * 4 /*gamma_k*/ + FUSED_BYTES;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + TAIL_BYTES;  // the base must be 1024-byte aligned
   static_assert(SMEM_BYTES <= 232448, "more shared memory than an SM offers");
 };
@@ -74,6 +88,25 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, const v
                                           unsigned long long timeout_ns, int lane) {
   int ok = 1;
   if (lane == 0) ok = mbar_wait(bar, parity, abort_flag, timeout_ns) ? 1 : 0;
+  ok = __shfl_sync(0xffffffffu, ok, 0);
+  return ok != 0;
+}
+
+// The same wait with a cluster-scope acquire, for barriers whose arrivals publish data that threads of
+// the partner CTA wrote.
+__device__ __forceinline__ bool warp_wait_cluster(uint32_t bar, uint32_t parity, const volatile int *abort_flag,
+                                                  unsigned long long timeout_ns, int lane) {
+  int ok = 1;
+  if (lane == 0 && !mbar_try_wait_cluster(bar, parity)) {
+    const unsigned long long t0 = globaltimer_ns();
+    uint32_t it = 0;
+    while (!mbar_try_wait_cluster(bar, parity)) {
+      if (((++it) & 31u) == 0u && (*abort_flag != 0 || globaltimer_ns() - t0 > timeout_ns)) {
+        ok = 0;
+        break;
+      }
+    }
+  }
   ok = __shfl_sync(0xffffffffu, ok, 0);
   return ok != 0;
 }
@@ -144,12 +177,14 @@ __device__ __forceinline__ void store_row_piece(__nv_bfloat16 *dst, const uint32
   }
 }
 
-template <int BLOCK_N, int D_HEAD, bool TRACE>
+template <int BLOCK_N, int D_HEAD, bool TRACE, int FG>
 __global__ void __launch_bounds__(RC_THREADS, 1)
 kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __grid_constant__ CUtensorMap tmap_rows,
-                     const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ RecomputeParams p) {
-  using Cfg = RcCfg<BLOCK_N, D_HEAD>;
+                     const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ RecomputeParams p,
+                     const __grid_constant__ std::conditional_t<(FG > 0), FusedParams, NoFusedParams> f) {
+  using Cfg = RcCfg<BLOCK_N, D_HEAD, FG>;
   constexpr int STAGES = Cfg::STAGES;
+  constexpr bool FUSED = FG > 0;
   static_assert(BLOCK_N % D_HEAD == 0, "a tile must hold whole heads");
 
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -160,10 +195,13 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   }
   uint8_t *tail = smem + STAGES * Cfg::STAGE_BYTES;
   uint64_t *bars = reinterpret_cast<uint64_t *>(tail);
-  uint32_t *s_tmem = reinterpret_cast<uint32_t *>(tail + Cfg::NUM_BARS * 8);
+  uint32_t *s_tmem = reinterpret_cast<uint32_t *>(tail + Cfg::BAR_BYTES);
   volatile int *s_abort = reinterpret_cast<volatile int *>(s_tmem + 1);
-  float *s_rstd = reinterpret_cast<float *>(tail + Cfg::NUM_BARS * 8 + 16);
+  float *s_rstd = reinterpret_cast<float *>(tail + Cfg::BAR_BYTES + 16);
   float *s_gamma_k = s_rstd + 2 * RC_BLOCK_M;
+  float *s_sc = s_gamma_k + 256;                 // fused: [2][GT][256]
+  float *s_rall = s_sc + 2 * Cfg::GT * 256;      // fused: [2][256]
+  float *s_lsum = s_rall + 2 * 256;              // fused: [GT][4]
 
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_base = smem_u32(bars);
@@ -174,6 +212,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   auto bar_stats_full = [&](int a) { return bar_base + 8u * (2 * STAGES + 4 + a); };
   auto bar_rstd_free = [&](int a) { return bar_base + 8u * (2 * STAGES + 6 + a); };
   const uint32_t bar_stats_x = bar_base + 8u * (2 * STAGES + 8);
+  auto bar_scores = [&](int u) { return bar_base + 8u * (2 * STAGES + 9 + u); };  // fused only
+  const uint32_t bar_epi = bar_base + 8u * (2 * STAGES + 11);                       // fused only
   const uint32_t cta_rank = cluster_ctarank();  // 0: issues the MMAs, 1: its partner
   const int cluster_id = static_cast<int>(blockIdx.x >> 1);
   const int num_clusters = static_cast<int>(gridDim.x >> 1);
@@ -189,7 +229,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   // With no more tiles than clusters every tile is its own unit, all key tiles first.  Falls back to
   // row-major single tiles when a tile mixes key and value heads.
   const int nk_tiles = (p.k_cols % BLOCK_N == 0) ? p.k_cols / BLOCK_N : 0;
-  const int unit_tiles = (nk_tiles != 0 && num_tiles > num_clusters) ? 2 : 1;
+  // (the fused variant always pairs the key tile with the value tile: the scores of the one weight the other)
+  const int unit_tiles = (nk_tiles != 0 && (FUSED || num_tiles > num_clusters)) ? 2 : 1;
   const int n_units = num_tiles / unit_tiles;
   // i-th tile of this cluster -> (job, first row of this CTA's 128 rows within the job, first fused
   // column, whether it opens a unit); false when the cluster has no i-th tile
@@ -239,6 +280,11 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
       mbar_init(bar_rstd_free(a), 4);            // one arrival per local epilogue warp
     }
     mbar_init(bar_stats_x, 4);  // one arrival per statistics warp
+    if (FUSED) {
+      mbar_init(bar_scores(0), 256);  // one arrival per epilogue thread of both CTAs
+      mbar_init(bar_scores(1), 256);
+      mbar_init(bar_epi, 4);          // one arrival per local epilogue warp
+    }
     *s_abort = 0;
     fence_mbar_init();
     prefetch_tensormap(&tmap_store);
@@ -355,6 +401,11 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
         }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + a * BLOCK_N;
+        // fused, value tile of a unit whose job attends: the operands change places, the accumulator
+        // holds V transposed (lanes = the pair's 256 value channels, columns = the pair's 256 rows), so
+        // that the weighted sum over rows is a sum along columns, local to a thread
+        bool swap_ab = false;
+        if constexpr (FUSED) swap_ab = !first_ && f.att[job_].q != nullptr;
         long long waited = 0;
         trace_put<TRACE>(p.trace, ti, 4);
         trace_put<TRACE>(p.trace, ti, 10, (m0_ / (2 * RC_BLOCK_M)) * p.num_n_blocks + n0_ / BLOCK_N);
@@ -368,7 +419,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
           }
           if (TRACE) waited += clock64() - w0;
           tc_fence_after();
-          umma_kblock_pair(d_tmem, a_lo, a_lo + b_off_units, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
+          if (FUSED && swap_ab) umma_kblock_pair(d_tmem, a_lo + b_off_units, a_lo, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
+          else umma_kblock_pair(d_tmem, a_lo, a_lo + b_off_units, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
           full += 8u;
           empty += 8u;
           a_lo += stage_units;
@@ -460,12 +512,29 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
     const int row = quarter * 32 + lane;
     const uint32_t lane_field = static_cast<uint32_t>(quarter * 32) << 16;
     constexpr int HALF = D_HEAD / 2;
+    constexpr int NG = FUSED ? FG : 1;
     int a = 0;
     uint32_t aph = 0;
+    uint32_t sph[2] = {0u, 0u}, eph = 0;  // fused: phases of the score barriers and of the epilogue warps' barrier
     int job, m0, n0;
     bool first_of_unit;
     for (int ti = 0; tile_at(ti, job, m0, n0, first_of_unit); ++ti) {
       const RcJob &J = p.jobs[job];
+      // fused: does this tile's job attend (K and V are consumed here) or is it a plain job?
+      bool attend = false;
+      int q_pos = 0, lo_pos = 0, part_base = 0;
+      const __nv_bfloat16 *qrow = nullptr;
+      if constexpr (FUSED) {
+        const RcAttend &A = f.att[job];
+        attend = A.q != nullptr;
+        qrow = A.q;
+        q_pos = A.q_pos;
+        lo_pos = A.lo_pos;
+        part_base = A.part_base;
+      }
+      const int ubuf = (ti >> 1) & 1;  // fused: score buffer of this unit
+      float f_scale = 0.f;
+      if constexpr (FUSED) f_scale = f.scale_log2e;
       // warp-uniform outcome: tcgen05.ld below is an aligned instruction
       if (!warp_wait(bar_tmem_full(a), aph, s_abort, tmo, lane) || !warp_wait(bar_stats_full(a), aph, s_abort, tmo, lane)) {
         raise(p.status, STATUS_TIMEOUT, s_abort);
@@ -488,6 +557,109 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
       const float4 *t_hi = reinterpret_cast<const float4 *>(p.rope_hi + static_cast<size_t>(pos >> ROPE_LO_BITS) * HALF);
       const float2 *t_lo = p.rope_lo + (pos & (ROPE_LO_SIZE - 1));
       const uint32_t acc = tmem_base + lane_field + a * BLOCK_N;
+      const bool visible = valid && pos <= q_pos && pos >= lo_pos;  // fused: does the query see this row's key
+      bool ok = true;
+
+      if (FUSED && attend && !first_of_unit) {
+        // ---- fused, value tile (Eq. 14 into Eq. 7): the accumulator holds V transposed and unscaled --
+        // this thread's lane is value channel ch of the 256-wide tile, column r is row r of the pair's
+        // 256 rows.  out[ch] = sum_r w[r] * acc[ch][r] with w[r] = exp2(score[r] - max) / rms(x_r).
+        constexpr int GT = Cfg::GT;
+        constexpr int WPH = D_HEAD >= 128 ? 4 : D_HEAD / 32;  // local epilogue warps that share a head
+        constexpr int RPW = 256 / WPH;                          // rows whose weights each of them makes
+        const int ch = static_cast<int>(cta_rank) * RC_BLOCK_M + row;
+        const int hh = ch / D_HEAD, cih = ch % D_HEAD, wi = quarter % WPH;
+        float *sc = s_sc + (ubuf * GT + hh * NG) * 256;
+        const float *ra = s_rall + ubuf * 256;
+        auto epi_sync = [&]() -> bool {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_epi);
+          const bool good = warp_wait(bar_epi, eph, s_abort, tmo, lane);
+          eph ^= 1u;
+          return good;
+        };
+        // the scores and 1/rms of all 256 rows (both CTAs' key-tile epilogues) have arrived
+        if (!warp_wait_cluster(bar_scores(ubuf), sph[ubuf], s_abort, tmo, lane)) {
+          raise(p.status, STATUS_TIMEOUT, s_abort);
+          break;
+        }
+        sph[ubuf] ^= 1u;
+        float mx[NG], lsum[NG], o[NG];
+#pragma unroll
+        for (int g = 0; g < NG; ++g) {
+          float mv = -CUDART_INF_F;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) mv = fmaxf(mv, sc[g * 256 + lane + 32 * k]);
+#pragma unroll
+          for (int msk = 16; msk >= 1; msk >>= 1) mv = fmaxf(mv, __shfl_xor_sync(0xffffffffu, mv, msk));
+          mx[g] = mv;
+        }
+        if (!epi_sync()) {  // every warp has its maxima before the scores become weights
+          raise(p.status, STATUS_TIMEOUT, s_abort);
+          break;
+        }
+#pragma unroll
+        for (int g = 0; g < NG; ++g) {
+          float lp = 0.f;
+#pragma unroll
+          for (int k = 0; k < RPW / 32; ++k) {
+            const int r = wi * RPW + lane + 32 * k;
+            const float pw = mx[g] == -CUDART_INF_F ? 0.f : exp2f(sc[g * 256 + r] - mx[g]);
+            lp += pw;
+            sc[g * 256 + r] = pw * ra[r];
+          }
+#pragma unroll
+          for (int msk = 16; msk >= 1; msk >>= 1) lp += __shfl_xor_sync(0xffffffffu, lp, msk);
+          if (lane == 0) s_lsum[(hh * NG + g) * 4 + wi] = lp;
+        }
+        if (!epi_sync()) {
+          raise(p.status, STATUS_TIMEOUT, s_abort);
+          break;
+        }
+#pragma unroll
+        for (int g = 0; g < NG; ++g) {
+          float l = 0.f;
+#pragma unroll
+          for (int w = 0; w < WPH; ++w) l += s_lsum[(hh * NG + g) * 4 + w];
+          lsum[g] = l;
+          o[g] = 0.f;
+        }
+        // rows past the end of the job hold whatever the store holds there (possibly NaN patterns):
+        // their weight is zero, but 0 * NaN is not, so those columns are skipped or zeroed
+        const int nvalid = J.n - (m0 - static_cast<int>(cta_rank) * RC_BLOCK_M);
+#pragma unroll 1
+        for (int c8 = 0; c8 < 8 && c8 * 32 < nvalid; ++c8) {
+          uint32_t r[32];
+          tmem_ld_x32(acc + c8 * 32, r);
+          tmem_wait_ld();
+          if (c8 * 32 + 32 > nvalid) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c8 * 32 + j >= nvalid) r[j] = 0u;
+          }
+#pragma unroll
+          for (int g = 0; g < NG; ++g) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              const float4 w4 = *reinterpret_cast<const float4 *>(sc + g * 256 + c8 * 32 + j);
+              o[g] = fmaf(w4.x, __uint_as_float(r[j]), o[g]);
+              o[g] = fmaf(w4.y, __uint_as_float(r[j + 1]), o[g]);
+              o[g] = fmaf(w4.z, __uint_as_float(r[j + 2]), o[g]);
+              o[g] = fmaf(w4.w, __uint_as_float(r[j + 3]), o[g]);
+            }
+          }
+        }
+        if constexpr (FUSED) {
+          const size_t slot = static_cast<size_t>(part_base) + (m0 - static_cast<int>(cta_rank) * RC_BLOCK_M) / (2 * RC_BLOCK_M);
+          const int kvh = (n0 - p.k_cols) / D_HEAD + hh;
+#pragma unroll
+          for (int g = 0; g < NG; ++g) {
+            const size_t qh = slot * f.n_q + static_cast<size_t>(kvh) * NG + g;
+            f.part_o[qh * D_HEAD + cih] = o[g];
+            if (cih == 0) *reinterpret_cast<float2 *>(f.part_ml + qh * 2) = make_float2(mx[g], lsum[g]);
+          }
+        }
+      } else {
 
 #pragma unroll 1
       for (int hh = 0; hh < BLOCK_N / D_HEAD; ++hh) {
@@ -511,6 +683,13 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
           // ---- key head (Eq. 13): 1/rms, optional key norm, rotation R_pos
           __nv_bfloat16 *dst = J.k_out + static_cast<size_t>(m) * p.out_row_stride + col0;
           float kscale = rstd;
+          // fused, attending job: the rotated key (rounded to bf16 like a stored one) is not written but
+          // multiplied with the NG queries of this KV head (Eq. 6); two-wide partial sums per query
+          uint64_t sdot[NG];
+#pragma unroll
+          for (int g = 0; g < NG; ++g) sdot[g] = 0ull;
+          const uint4 *qh = nullptr;  // the queries of this KV head: [NG][D_HEAD] bf16
+          if (FUSED && attend) qh = reinterpret_cast<const uint4 *>(qrow + static_cast<size_t>(col0 / D_HEAD) * NG * D_HEAD);
           if (p.qk_norm) {
             // sum of squares over the head in four chains (columns j mod 4), two-wide, combined in a
             // fixed order: a single 256-long dependent chain would be pure latency
@@ -566,7 +745,17 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
                 o[j] = pack_bf16(fmaf(a0, c0, -b0 * s0), fmaf(a0, s0, b0 * c0));
                 o[j + 1] = pack_bf16(fmaf(a1, c1, -b1 * s1), fmaf(a1, s1, b1 * c1));
               }
-              if (valid) store_row_piece<2>(dst + c * 16, o, wide);
+              if (FUSED && attend) {
+#pragma unroll
+                for (int g = 0; g < NG; ++g) {
+                  const uint4 q0 = __ldg(qh + (g * D_HEAD + c * 16) / 8), q1 = __ldg(qh + (g * D_HEAD + c * 16) / 8 + 1);
+                  const uint32_t qw[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+#pragma unroll
+                  for (int w = 0; w < 8; ++w) sdot[g] = ffma2(bf16x2_to_f32x2(o[w]), bf16x2_to_f32x2(qw[w]), sdot[g]);
+                }
+              } else if (valid) {
+                store_row_piece<2>(dst + c * 16, o, wide);
+              }
             }
           } else {
             constexpr int NC = HALF / 16;  // 16 pairs (i, i + HALF) per step
@@ -600,14 +789,52 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
                 oa[j >> 1] = pack_bf16(fmaf(a0, c0, -b0 * s0), fmaf(a1, c1, -b1 * s1));
                 ob[j >> 1] = pack_bf16(fmaf(a0, s0, b0 * c0), fmaf(a1, s1, b1 * c1));
               }
-              if (valid) {
+              if (FUSED && attend) {
+#pragma unroll
+                for (int g = 0; g < NG; ++g) {
+                  const uint4 a0 = __ldg(qh + (g * D_HEAD + c * 16) / 8), a1 = __ldg(qh + (g * D_HEAD + c * 16) / 8 + 1);
+                  const uint4 b0 = __ldg(qh + (g * D_HEAD + HALF + c * 16) / 8), b1 = __ldg(qh + (g * D_HEAD + HALF + c * 16) / 8 + 1);
+                  const uint32_t qa[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                  const uint32_t qb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+                  for (int w = 0; w < 8; ++w) {
+                    sdot[g] = ffma2(bf16x2_to_f32x2(oa[w]), bf16x2_to_f32x2(qa[w]), sdot[g]);
+                    sdot[g] = ffma2(bf16x2_to_f32x2(ob[w]), bf16x2_to_f32x2(qb[w]), sdot[g]);
+                  }
+                }
+              } else if (valid) {
                 store_row_piece<2>(dst + c * 16, oa, wide);
                 store_row_piece<2>(dst + HALF + c * 16, ob, wide);
               }
             }
           }
+          if (FUSED && attend) {
+            // the scores of this row (log2 units, -inf when the query does not see the key) go to both
+            // CTAs of the pair: the value tile's epilogue needs those of all 256 rows
+#pragma unroll
+            for (int g = 0; g < NG; ++g) {
+              float lo, hi;
+              unpack2(sdot[g], lo, hi);
+              float sv = (lo + hi) * f_scale;
+              if (!visible) sv = -CUDART_INF_F;
+              float *dstp = s_sc + (ubuf * Cfg::GT + hh * NG + g) * 256 + static_cast<int>(cta_rank) * RC_BLOCK_M + row;
+              *dstp = sv;
+              st_cluster_f32(map_to_cta(smem_u32(dstp), cta_rank ^ 1u), sv);
+            }
+          }
         }
       }
+      if (FUSED && attend) {
+        // 1/rms of the row, then "this thread's scores are in place" to both CTAs (a release at cluster
+        // scope: the partner's value-tile epilogue reads what was just stored into its shared memory)
+        float *rp = s_rall + ubuf * 256 + static_cast<int>(cta_rank) * RC_BLOCK_M + row;
+        *rp = rstd;
+        st_cluster_f32(map_to_cta(smem_u32(rp), cta_rank ^ 1u), rstd);
+        mbar_arrive(bar_scores(ubuf));
+        mbar_arrive_cluster_release(map_to_cta(bar_scores(ubuf), cta_rank ^ 1u));
+      }
+      }
+      if (!ok) break;
       // accumulator a (and s_rstd[a]) may be overwritten now
       tc_fence_before();
       __syncwarp();
@@ -638,20 +865,22 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
 }
 
 // ------------------------------------------------------------------------------ host launcher
-template <int BLOCK_N, int D_HEAD, bool TRACE>
+template <int BLOCK_N, int D_HEAD, bool TRACE, int FG>
 static kvd_status launch_impl(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
-                              const CUtensorMap &tmap_rows, const RecomputeParams &p, cudaStream_t stream) {
-  using Cfg = RcCfg<BLOCK_N, D_HEAD>;
-  auto kern = kvd_recompute_kernel<BLOCK_N, D_HEAD, TRACE>;
+                              const CUtensorMap &tmap_rows, const RecomputeParams &p, const FusedParams *fp,
+                              cudaStream_t stream) {
+  using Cfg = RcCfg<BLOCK_N, D_HEAD, FG>;
+  auto kern = kvd_recompute_kernel<BLOCK_N, D_HEAD, TRACE, FG>;
   static bool configured[64] = {};
   if (!configured[ctx->device & 63]) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaFuncSetAttribute(recompute)");
     configured[ctx->device & 63] = true;
   }
-  const int tiles = p.num_m_blocks * p.num_n_blocks;
+  // plain: one cluster per tile at most; fused: per unit of a key tile and a value tile
+  const int work = FG > 0 ? p.num_m_blocks * p.num_n_blocks / 2 : p.num_m_blocks * p.num_n_blocks;
   const int max_clusters = ctx->num_sms / 2;
-  const int clusters = tiles < max_clusters ? tiles : max_clusters;
+  const int clusters = work < max_clusters ? work : max_clusters;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(2 * clusters, 1, 1);
@@ -667,31 +896,52 @@ static kvd_status launch_impl(kvd_ctx *ctx, const LayerState &ls, const CUtensor
   attr[1].val.programmaticStreamSerializationAllowed = (serial_launch_mask() & 1) ? 0 : 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  cudaError_t le = cudaLaunchKernelEx(&cfg, kern, tmap_store, tmap_rows, ls.tmap_b, p);
+  cudaError_t le;
+  if constexpr (FG > 0) le = cudaLaunchKernelEx(&cfg, kern, tmap_store, tmap_rows, ls.tmap_b, p, *fp);
+  else le = cudaLaunchKernelEx(&cfg, kern, tmap_store, tmap_rows, ls.tmap_b, p, NoFusedParams());
   if (le != cudaSuccess) return cuda_fail(ctx, le, "launch recompute");
   ctx->launches += 1;
   return KVD_OK;
 }
 
-template <int BLOCK_N, int D_HEAD>
+template <int BLOCK_N, int D_HEAD, int FG = 0>
 static kvd_status launch_sel(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
-                             const CUtensorMap &tmap_rows, const RecomputeParams &p, cudaStream_t stream) {
-  if (p.trace != nullptr) return launch_impl<BLOCK_N, D_HEAD, true>(ctx, ls, tmap_store, tmap_rows, p, stream);
-  return launch_impl<BLOCK_N, D_HEAD, false>(ctx, ls, tmap_store, tmap_rows, p, stream);
+                             const CUtensorMap &tmap_rows, const RecomputeParams &p, const FusedParams *fp,
+                             cudaStream_t stream) {
+  if constexpr (FG == 0) {
+    if (p.trace != nullptr) return launch_impl<BLOCK_N, D_HEAD, true, 0>(ctx, ls, tmap_store, tmap_rows, p, fp, stream);
+  }
+  return launch_impl<BLOCK_N, D_HEAD, false, FG>(ctx, ls, tmap_store, tmap_rows, p, fp, stream);
 }
 
 kvd_status launch_recompute(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
                             const CUtensorMap &tmap_rows, const RecomputeParams &p, cudaStream_t stream) {
   const int dh = ctx->desc.d_head;
   if (ctx->block_n == 256) {
-    if (dh == 256) return launch_sel<256, 256>(ctx, ls, tmap_store, tmap_rows, p, stream);
-    if (dh == 128) return launch_sel<256, 128>(ctx, ls, tmap_store, tmap_rows, p, stream);
-    if (dh == 64) return launch_sel<256, 64>(ctx, ls, tmap_store, tmap_rows, p, stream);
+    if (dh == 256) return launch_sel<256, 256>(ctx, ls, tmap_store, tmap_rows, p, nullptr, stream);
+    if (dh == 128) return launch_sel<256, 128>(ctx, ls, tmap_store, tmap_rows, p, nullptr, stream);
+    if (dh == 64) return launch_sel<256, 64>(ctx, ls, tmap_store, tmap_rows, p, nullptr, stream);
   } else if (ctx->block_n == 128) {
-    if (dh == 128) return launch_sel<128, 128>(ctx, ls, tmap_store, tmap_rows, p, stream);
-    if (dh == 64) return launch_sel<128, 64>(ctx, ls, tmap_store, tmap_rows, p, stream);
+    if (dh == 128) return launch_sel<128, 128>(ctx, ls, tmap_store, tmap_rows, p, nullptr, stream);
+    if (dh == 64) return launch_sel<128, 64>(ctx, ls, tmap_store, tmap_rows, p, nullptr, stream);
   }
   return KVD_ERR_SHAPE;
+}
+
+// The fused variant exists for 256-column tiles and the head sizes / group sizes of the model shapes
+// this library is built around; KVD_ERR_UNSUPPORTED otherwise (the caller falls back to
+// kvd_recompute_kv + kvd_decode_attention).
+kvd_status launch_recompute_fused(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
+                                  const CUtensorMap &tmap_rows, const RecomputeParams &p, const FusedParams &fp,
+                                  cudaStream_t stream) {
+  const int dh = ctx->desc.d_head, g = ctx->desc.n_q_heads / ctx->desc.n_kv_heads;
+  if (ctx->block_n != 256 || p.k_cols % 256 != 0) return KVD_ERR_UNSUPPORTED;
+  if (dh == 256 && g == 2) return launch_sel<256, 256, 2>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
+  if (dh == 256 && g == 1) return launch_sel<256, 256, 1>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
+  if (dh == 128 && g == 4) return launch_sel<256, 128, 4>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
+  if (dh == 128 && g == 2) return launch_sel<256, 128, 2>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
+  if (dh == 128 && g == 1) return launch_sel<256, 128, 1>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
+  return KVD_ERR_UNSUPPORTED;
 }
 
 }  // namespace kvd
