@@ -309,6 +309,20 @@ class Workload:
                                       [[(K, V, self.kdim, 0, T), (K[T:], V[T:], self.kdim, T, 1)]], 0.0,
                                       self.out[s:s + 1])
 
+    def k_two_call(self, i):
+        # recompute (T stored rows + the current token) followed by attention: the step's two K/V launches
+        self.k_recompute_step(i)
+        self.k_attention(i)
+
+    def k_fused(self, i):
+        # the same work with the recomputed K/V consumed inside the recompute kernel (never written):
+        # kvd_decode_attention_recompute; only the current token's K_t, V_t are stored and read back
+        s, T = i % self.n_sets, self.T
+        K, V = self.K[s], self.V[s]
+        self.ctx.kvd_decode_attention_recompute(0, 1, self.q[s:s + 1], [T], [(s, 0, T)], self.X[s][T:], self.pos[T:], 1,
+                                                K[T:], V[T:], self.kdim, [[(K[T:], V[T:], self.kdim, T, 1)]], 0.0,
+                                                self.out[s:s + 1])
+
     def cached_read_step(self, i):
         """What KV-Direct replaces: attention over the stored cache of T + 1 keys in one segment."""
         s, T = i % self.n_sets, self.T
@@ -449,7 +463,9 @@ def run_gpu(args):
     iso_ms = {"checkpoint": timed_graph(wl.k_checkpoint, 10), "recompute": timed_graph(wl.k_recompute, 10),
               "recompute_with_current_token": timed_graph(wl.k_recompute_step, 10),
               "recompute_from_caller_rows": timed_graph(wl.k_recompute_rows, 10),
-              "current_token_kv_alone": timed_graph(wl.k_current, 10), "attention": timed_graph(wl.k_attention, 10)}
+              "current_token_kv_alone": timed_graph(wl.k_current, 10), "attention": timed_graph(wl.k_attention, 10),
+              "recompute_then_attention_two_calls": timed_graph(wl.k_two_call, 10),
+              "recompute_fused_into_attention": timed_graph(wl.k_fused, 10)}
     read_attn_ms = timed_graph(wl.cached_read_step, 10)
     kv_copy_dst = torch.empty((2, T + 1, wl.kdim), dtype=torch.bfloat16, device="cuda")
 
@@ -780,6 +796,16 @@ def run_stack_configs(args):
             cur(i)
             att_full(i)
 
+        # the KV-Direct layer with the recompute fused into attention (recomputed K/V never written):
+        # evicted ranges attended inside the recompute kernel, window + current token as live segments
+        segs_live = [[[(Kf[s][b, wf:], Vf[s][b, wf:], kdim, wf, budget), (kc[b:], vc[b:], kdim, ctx_len, 1)]
+                      for b in range(batch)] for s in range(n_sets)]
+        franges = [(b, lo, n_old) for b in range(batch)]
+
+        def layer_fused(i):
+            c.kvd_decode_attention_recompute(0, batch, q, qpos, franges, xc, pc, batch, kc, vc, kdim,
+                                             segs_live[i % n_sets], 0.0, out)
+
         # memory-bound cases first, each after a short pause: a long run of GEMMs at the power cap
         # leaves the clocks low for whatever is measured next
         def rested(fn):
@@ -790,6 +816,7 @@ def run_stack_configs(args):
         t_cur, t_att, t_full = rested(cur), rested(att), rested(att_full)
         t_layer_full = rested(layer_full)
         t_rec, t_layer_kvd = rested(rec), rested(layer_kvd)
+        t_layer_fused = rested(layer_fused)
         assert c.kvd_poll_status() == kvd.KVD_OK
         flops = 4.0 * (M + batch) * shape.n_kv_heads * shape.d_hidden * shape.d_head
         keys = batch * (ctx_len + 1 - lo)
@@ -799,7 +826,8 @@ def run_stack_configs(args):
                 "recompute_with_current_us": t_rec, "recompute_tflops": flops / t_rec / 1e6,
                 "current_kv_only_us": t_cur, "attention_us": t_att, "attention_gbs": byts / t_att / 1e3,
                 "fullcache_attention_us": t_full, "fullcache_attention_gbs": byts / t_full / 1e3,
-                "kvdirect_layer_us": t_layer_kvd, "fullcache_layer_us": t_layer_full}
+                "kvdirect_layer_us": t_layer_kvd, "kvdirect_fused_layer_us": t_layer_fused,
+                "fullcache_layer_us": t_layer_full}
 
     result = {"peaks": peaks, "gemma3_4b_stack_ctx2048_window256": [], "qwen3_4b_ctx32768_batch8_window512": None}
     for batch in (1, 4, 16, 64):
@@ -808,11 +836,14 @@ def run_stack_configs(args):
         kvd_step = 5 * g["kvdirect_layer_us"] + 29 * l["kvdirect_layer_us"]
         full_step = 5 * g["fullcache_layer_us"] + 29 * l["fullcache_layer_us"]
         result["gemma3_4b_stack_ctx2048_window256"].append(
-            {"batch": batch, "kvdirect_decode_step_us": kvd_step, "fullcache_decode_step_us": full_step,
+            {"batch": batch, "kvdirect_decode_step_us": kvd_step,
+             "kvdirect_fused_decode_step_us": 5 * g["kvdirect_fused_layer_us"] + 29 * l["kvdirect_fused_layer_us"],
+             "fullcache_decode_step_us": full_step,
              "ratio": kvd_step / full_step, "recomputed_tokens_per_s": batch * (5 * g["rows_recomputed"] // batch +
              29 * l["rows_recomputed"] // batch) / (kvd_step * 1e-6), "global_layer": g, "local_layer": l})
     qw = layer_case(QWEN3_4B, 32768, 512, 8)
     qw["step_us_36_layers"] = 36 * qw["kvdirect_layer_us"]
+    qw["fused_step_us_36_layers"] = 36 * qw["kvdirect_fused_layer_us"]
     qw["fullcache_step_us_36_layers"] = 36 * qw["fullcache_layer_us"]
     qw["recompute_frac_of_sustained_peak"] = qw["recompute_tflops"] / peaks["bf16_tflops_sustained"]
     qw["recompute_frac_of_burst_peak"] = qw["recompute_tflops"] / peaks["bf16_tflops"]
