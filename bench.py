@@ -905,6 +905,12 @@ def run_profile_qwen(args):
         # the same keys from one stored segment (the cached-KV read)
         c.kvd_decode_attention(0, batch, q, [ctx_len] * batch,
                                [[(Kf[s][b], Vf[s][b], kdim, 0, ctx_len + 1)] for b in range(batch)], 0.0, out)
+        # the KV-Direct layer again with the recompute fused into attention (every second launch of the
+        # recompute kernel in this run is the fused variant)
+        c.kvd_decode_attention_recompute(0, batch, q, [ctx_len] * batch, [(b, 0, n_old) for b in range(batch)], xc, pc,
+                                         batch, kc, vc, kdim,
+                                         [[(Kf[s][b, n_old:], Vf[s][b, n_old:], kdim, n_old, budget),
+                                           (kc[b:], vc[b:], kdim, ctx_len, 1)] for b in range(batch)], 0.0, out)
     torch.cuda.synchronize()
     assert c.kvd_poll_status() == kvd.KVD_OK
     print(json.dumps({"profile_run": "qwen3-4b layer", "rows_recomputed": batch * n_old, "keys": batch * (ctx_len + 1),
