@@ -219,6 +219,36 @@ kvd_status kvd_recompute_kv_step(kvd_ctx *ctx, int layer, const kvd_store_range 
                                  const void *rows, const int32_t *positions, int n_rows, void *k_rows_out,
                                  void *v_rows_out, int64_t out_row_stride, void *stream);
 
+/* ---- FP8 checkpoints (lower-precision residual rows and weights: the second future-work item of the
+ * paper's Section 6, which fixes no format; this is the definition this library implements) ----
+ * A residual row x (bf16) is stored as E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits,
+ * largest finite value 448) with one fp32 scale per row:
+ *     s_x = max|x| / 448,    code_k = e4m3(x_k / s_x)   round to nearest even, saturating, both steps in fp32,
+ * together with its position and the sum of squares of the ORIGINAL row (1/rms of Eq. 2 is not affected by
+ * the quantisation).  The folded weights W' = gamma (.) W_kv get one scale for the whole matrix,
+ * s_w = max|W'| / 448, code = e4m3(W' / s_w) (prepared by kvd_set_layer next to the bf16 copy).
+ * RECOMPUTE_KV from such rows is Eq. 13-14 on the dequantised operands,
+ *     y = (s_x s_w / rms(x)) * sum_k code_x[k] code_w[k][:],   then key norm and rotation as usual,
+ * with the code products accumulated on the tensor cores (kind f8f6f4, fp32 accumulation).  Per token and
+ * layer the store holds d_hidden + 12 bytes instead of 2 d_hidden + 8.  The result is NOT the bf16 result:
+ * each operand carries up to 2^-4 relative error, a few per cent of the outputs' rms after the contraction
+ * (measured in the tests); exactness claims (Prop. 3.2) do not carry over, determinism does (a row's bits
+ * do not depend on the batch it is recomputed in).
+ * The FP8 store is a second, independent arena (layout: codes uint8 [layers][max_seqs][max_tokens][d_hidden],
+ * then positions int32, sums of squares fp32, scales fp32, each [layers][max_seqs][max_tokens] and each
+ * region starting at a 256-byte multiple); kvd_reset_sequence clears a sequence in both stores.
+ * kvd_store_bytes_fp8 returns 0 for shapes the variant does not support (d_hidden % 16 != 0). */
+size_t kvd_store_bytes_fp8(const kvd_model_desc *desc, int layers_stored);
+kvd_status kvd_attach_store_fp8(kvd_ctx *ctx, void *arena, size_t bytes, int layers_stored);
+int kvd_rows_stored_fp8(const kvd_ctx *ctx, int layer, int seq);
+/* Append n rows (DEVICE bf16 [n, d_hidden], 16-byte aligned; DEVICE int32 positions[n]) in quantised form. */
+kvd_status kvd_checkpoint_residual_fp8(kvd_ctx *ctx, int seq, int layer, const void *rows, const int32_t *positions,
+                                       int n, void *stream);
+/* RECOMPUTE_KV for ranges of the FP8 store (as kvd_recompute_kv_step without caller rows): K and V (bf16) of
+ * rows first_row .. first_row+n-1 of every range to its k_out / v_out. */
+kvd_status kvd_recompute_kv_fp8(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
+                                int64_t out_row_stride, void *stream);
+
 /* ATTENTION(Q, K_all, V_all) of Algorithm 1 for one new token per sequence (Eq. 6-7).
  *   q      DEVICE bf16 [batch, n_q_heads, d_head], already normalised and rotated to q_pos.
  *   q_pos  HOST int32 [batch]: position of each sequence's query token.

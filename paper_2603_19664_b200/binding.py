@@ -32,6 +32,7 @@ KVD_MAX_SEGMENTS = 4
 EXPORTED_SYMBOLS = (
     "kvd_create", "kvd_destroy", "kvd_set_layer", "kvd_store_bytes", "kvd_attach_store", "kvd_reset_sequence",
     "kvd_decode_attention_recompute",
+    "kvd_store_bytes_fp8", "kvd_attach_store_fp8", "kvd_rows_stored_fp8", "kvd_checkpoint_residual_fp8", "kvd_recompute_kv_fp8",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
     "kvd_recompute_kv_step",
     "kvd_decode_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
@@ -120,6 +121,16 @@ def load() -> ctypes.CDLL:
     lib.kvd_decode_attention.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
                                          ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
     lib.kvd_decode_attention.restype = i32
+    lib.kvd_store_bytes_fp8.argtypes = [ctypes.POINTER(kvd_model_desc), i32]
+    lib.kvd_store_bytes_fp8.restype = sz
+    lib.kvd_attach_store_fp8.argtypes = [vp, vp, sz, i32]
+    lib.kvd_attach_store_fp8.restype = i32
+    lib.kvd_rows_stored_fp8.argtypes = [vp, i32, i32]
+    lib.kvd_rows_stored_fp8.restype = i32
+    lib.kvd_checkpoint_residual_fp8.argtypes = [vp, i32, i32, vp, vp, i32, vp]
+    lib.kvd_checkpoint_residual_fp8.restype = i32
+    lib.kvd_recompute_kv_fp8.argtypes = [vp, i32, ctypes.POINTER(kvd_store_range), i32, i64, vp]
+    lib.kvd_recompute_kv_fp8.restype = i32
     lib.kvd_decode_attention_recompute.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
                                                    ctypes.POINTER(kvd_store_range), vp, vp, i32, vp, vp, i64,
                                                    ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
@@ -164,6 +175,10 @@ def make_desc(n_layers: int, d_hidden: int, n_q_heads: int, n_kv_heads: int, d_h
 
 def kvd_store_bytes(desc: kvd_model_desc, layers_stored: int) -> int:
     return int(load().kvd_store_bytes(ctypes.byref(desc), layers_stored))
+
+
+def kvd_store_bytes_fp8(desc: kvd_model_desc, layers_stored: int) -> int:
+    return int(load().kvd_store_bytes_fp8(ctypes.byref(desc), layers_stored))
 
 
 def kvd_workspace_bytes(desc: kvd_model_desc) -> int:
@@ -326,6 +341,28 @@ class Kvd:
             self._h, layer, batch, _ptr(q), pos_arr, arr, _ptr(rows), _ptr(positions), n_rows, _ptr(k_rows_out),
             _ptr(v_rows_out), out_row_stride, seg_arr, n_segs, float(scale), _ptr(out), _stream(stream)),
             "kvd_decode_attention_recompute")
+
+    def kvd_attach_store_fp8(self, arena, layers_stored: int) -> None:
+        self._keep.append(arena)
+        self._check(self._lib.kvd_attach_store_fp8(self._h, _ptr(arena), arena.numel() * arena.element_size(),
+                                                   layers_stored), "kvd_attach_store_fp8")
+
+    def kvd_rows_stored_fp8(self, layer: int, seq: int) -> int:
+        return int(self._lib.kvd_rows_stored_fp8(self._h, layer, seq))
+
+    def kvd_checkpoint_residual_fp8(self, seq: int, layer: int, rows, positions, n: int, stream=None) -> None:
+        self._check(self._lib.kvd_checkpoint_residual_fp8(self._h, seq, layer, _ptr(rows), _ptr(positions), n,
+                                                          _stream(stream)), "kvd_checkpoint_residual_fp8")
+
+    def kvd_recompute_kv_fp8(self, layer: int, ranges: Sequence[Tuple[int, int, int, object, object]],
+                             out_row_stride: int, stream=None) -> None:
+        """ranges: (seq, first_row, n, k_out, v_out) over the FP8 store."""
+        arr = (kvd_store_range * max(len(ranges), 1))()
+        for i, (seq, first_row, n, k_out, v_out) in enumerate(ranges):
+            arr[i].seq, arr[i].first_row, arr[i].n, arr[i].reserved = int(seq), int(first_row), int(n), 0
+            arr[i].k_out, arr[i].v_out = _ptr(k_out), _ptr(v_out)
+        self._check(self._lib.kvd_recompute_kv_fp8(self._h, layer, arr, len(ranges), out_row_stride, _stream(stream)),
+                    "kvd_recompute_kv_fp8")
 
     def kvd_memory_stats(self) -> dict:
         ms = kvd_mem_stats()

@@ -152,6 +152,8 @@ extern "C" void kvd_destroy(kvd_ctx *ctx) {
   for (auto &l : ctx->layers) {
     if (l.wt) cudaFree(l.wt);
     if (l.gamma_k) cudaFree(l.gamma_k);
+    if (l.wt8) cudaFree(l.wt8);
+    if (l.w_scale8) cudaFree(l.w_scale8);
   }
   for (auto &kv : ctx->rope_cache) {
     if (kv.second.hi) cudaFree(kv.second.hi);
@@ -159,17 +161,20 @@ extern "C" void kvd_destroy(kvd_ctx *ctx) {
   }
   if (ctx->d_status) cudaFree(ctx->d_status);
   if (ctx->ext_sumsq) cudaFree(ctx->ext_sumsq);
+  if (ctx->amax_scratch) cudaFree(ctx->amax_scratch);
   cudaGetLastError();
   delete ctx;
 }
 
+// (eb = bytes per element: 2 for bf16, 1 for the FP8 variant's codes; a box row is 128 bytes either way)
 static kvd_status encode_2d(kvd_ctx *ctx, CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer,
-                            uint32_t box_inner, uint32_t box_outer) {
+                            uint32_t box_inner, uint32_t box_outer, int eb = 2) {
   cuuint64_t dims[2] = {inner, outer};
-  cuuint64_t strides[1] = {inner * 2};
+  cuuint64_t strides[1] = {inner * eb};
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+  CUresult r = ctx->encode(map, eb == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
+                           const_cast<void *>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
@@ -183,12 +188,13 @@ static kvd_status encode_2d(kvd_ctx *ctx, CUtensorMap *map, const void *base, ui
 
 // Row source of the recompute GEMM as a 3-D map [slabs][rows][d_hidden]; box = one 128 x 64 tile.
 static kvd_status encode_rows_3d(kvd_ctx *ctx, CUtensorMap *map, const void *base, uint64_t d_hidden, uint64_t rows,
-                                 uint64_t slabs) {
+                                 uint64_t slabs, int eb = 2) {
   cuuint64_t dims[3] = {d_hidden, rows, slabs};
-  cuuint64_t strides[2] = {d_hidden * 2, rows * d_hidden * 2};
-  cuuint32_t box[3] = {RC_BLOCK_K, RC_BLOCK_M, 1};
+  cuuint64_t strides[2] = {d_hidden * eb, rows * d_hidden * eb};
+  cuuint32_t box[3] = {static_cast<cuuint32_t>(RC_BLOCK_K * 2 / eb), RC_BLOCK_M, 1};
   cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+  CUresult r = ctx->encode(map, eb == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 3,
+                           const_cast<void *>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
@@ -272,6 +278,22 @@ extern "C" kvd_status kvd_set_layer(kvd_ctx *ctx, int layer, const kvd_layer_des
   if (st != KVD_OK) return st;
   st = encode_2d(ctx, &ls.tmap_b, ls.wt, d.d_hidden, n_cols, RC_BLOCK_K, ctx->block_n / 2);  // half tile per CTA
   if (st != KVD_OK) return st;
+  // the FP8 variant's copy of W' (E4M3 codes and one scale); rows of d_hidden bytes must be TMA-addressable
+  if (d.d_hidden % 16 == 0) {
+    if (!ls.wt8) {
+      e = cudaMalloc(&ls.wt8, static_cast<size_t>(n_cols) * d.d_hidden);
+      if (e == cudaSuccess) e = cudaMalloc(&ls.w_scale8, sizeof(float));
+      if (e == cudaSuccess && !ctx->amax_scratch) e = cudaMalloc(&ctx->amax_scratch, sizeof(unsigned));
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMalloc(fp8 weights)");
+      ctx->prepared_bytes += static_cast<size_t>(n_cols) * d.d_hidden + sizeof(float);
+    }
+    st = launch_prepare_weights_fp8(ctx, static_cast<const __nv_bfloat16 *>(ld->w_kv),
+                                    static_cast<const __nv_bfloat16 *>(ld->gamma_in), ls.wt8, d.d_hidden, n_cols,
+                                    ctx->amax_scratch, ls.w_scale8, stream);
+    if (st != KVD_OK) return st;
+    st = encode_2d(ctx, &ls.tmap_b8, ls.wt8, d.d_hidden, n_cols, 2 * RC_BLOCK_K, ctx->block_n / 2, 1);
+    if (st != KVD_OK) return st;
+  }
   e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "kvd_set_layer sync");
   ls.theta = ld->rope_theta;
@@ -307,8 +329,9 @@ extern "C" kvd_status kvd_attach_store(kvd_ctx *ctx, void *arena, size_t bytes, 
 
 extern "C" kvd_status kvd_reset_sequence(kvd_ctx *ctx, int seq) {
   if (!ctx || seq < 0 || seq >= ctx->desc.max_seqs) return KVD_ERR_INVALID_ARG;
-  if (!ctx->store_rows) return KVD_ERR_STATE;
+  if (!ctx->store_rows && !ctx->store8_codes) return KVD_ERR_STATE;
   for (int l = 0; l < ctx->layers_stored; ++l) ctx->rows_stored[static_cast<size_t>(l) * ctx->desc.max_seqs + seq] = 0;
+  for (int l = 0; l < ctx->layers_stored8; ++l) ctx->rows_stored8[static_cast<size_t>(l) * ctx->desc.max_seqs + seq] = 0;
   return KVD_OK;
 }
 
@@ -393,6 +416,7 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
     J.slab = r.seq;
     J.positions = ctx->store_pos + store_slot(ctx, layer, r.seq) + r.first_row;
     J.sumsq = ctx->store_sumsq + store_slot(ctx, layer, r.seq) + r.first_row;
+    J.scale = nullptr;
     J.k_out = static_cast<__nv_bfloat16 *>(r.k_out);
     J.v_out = static_cast<__nv_bfloat16 *>(r.v_out);
     mb += (r.n + 2 * RC_BLOCK_M - 1) / (2 * RC_BLOCK_M);  // 256-row tiles, 128 rows per CTA of a pair
@@ -412,6 +436,7 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
     J.slab = -1;
     J.positions = positions;
     J.sumsq = nullptr;
+    J.scale = nullptr;
     if (n_rows > RC_INLINE_STAT_ROWS && static_cast<size_t>(n_rows) <= ctx->ext_sumsq_rows) {
       // too many rows for the statistics warps of the main kernel: take the statistics first (same
       // function, same bits).  The scratch is shared by the calls on this context, which are
@@ -446,6 +471,7 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
   p.status = ctx->d_status;
   p.timeout_ns = ctx->timeout_ns;
   p.ext_rows = static_cast<const __nv_bfloat16 *>(rows);
+  p.w_scale = nullptr;
   p.row_chunks = d.d_hidden / 8;
   p.wide_store = out_row_stride % 16 == 0;
   for (int i = 0; i < n_jobs; ++i)
@@ -464,6 +490,130 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
     return launch_recompute_fused(ctx, ls, tmap_store, tmap_ext, p, fp, stream);
   }
   return launch_recompute(ctx, ls, tmap_store, tmap_ext, p, stream);
+}
+
+// ------------------------------------------------------------------------------ FP8 checkpoints
+extern "C" size_t kvd_store_bytes_fp8(const kvd_model_desc *d, int layers_stored) {
+  if (check_desc(d) != KVD_OK || layers_stored <= 0 || d->d_hidden % 16 != 0) return 0;
+  const size_t slots = static_cast<size_t>(layers_stored) * d->max_seqs * d->max_tokens_per_seq;
+  // codes, then positions, sums of squares and scales, each region starting at a 256-byte multiple
+  return round_up(slots * d->d_hidden, 256) + 3 * round_up(slots * 4, 256);
+}
+
+extern "C" kvd_status kvd_attach_store_fp8(kvd_ctx *ctx, void *arena, size_t bytes, int layers_stored) {
+  if (!ctx || !arena || layers_stored <= 0 || layers_stored > ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(arena) & 255u) != 0) return KVD_ERR_ALIGNMENT;
+  const size_t need = kvd_store_bytes_fp8(&ctx->desc, layers_stored);
+  if (need == 0) return KVD_ERR_SHAPE;
+  if (bytes < need) return KVD_ERR_CAPACITY;
+  const kvd_model_desc &d = ctx->desc;
+  const size_t slots = static_cast<size_t>(layers_stored) * d.max_seqs * d.max_tokens_per_seq;
+  uint8_t *base = static_cast<uint8_t *>(arena);
+  ctx->store8_codes = base;
+  ctx->store8_pos = reinterpret_cast<int32_t *>(base + round_up(slots * d.d_hidden, 256));
+  ctx->store8_sumsq = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(ctx->store8_pos) + round_up(slots * 4, 256));
+  ctx->store8_scale = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(ctx->store8_sumsq) + round_up(slots * 4, 256));
+  ctx->layers_stored8 = layers_stored;
+  ctx->rows_stored8.assign(static_cast<size_t>(layers_stored) * d.max_seqs, 0);
+  ctx->store8_maps.resize(layers_stored);
+  for (int l = 0; l < layers_stored; ++l) {
+    const uint8_t *lb = ctx->store8_codes + static_cast<size_t>(l) * d.max_seqs * d.max_tokens_per_seq * d.d_hidden;
+    kvd_status st = encode_rows_3d(ctx, &ctx->store8_maps[l], lb, d.d_hidden, d.max_tokens_per_seq, d.max_seqs, 1);
+    if (st != KVD_OK) {
+      ctx->store8_codes = nullptr;
+      ctx->layers_stored8 = 0;
+      return st;
+    }
+  }
+  return KVD_OK;
+}
+
+extern "C" int kvd_rows_stored_fp8(const kvd_ctx *ctx, int layer, int seq) {
+  if (!ctx || !ctx->store8_codes || layer < 0 || layer >= ctx->layers_stored8 || seq < 0 || seq >= ctx->desc.max_seqs)
+    return -1;
+  return ctx->rows_stored8[static_cast<size_t>(layer) * ctx->desc.max_seqs + seq];
+}
+
+extern "C" kvd_status kvd_checkpoint_residual_fp8(kvd_ctx *ctx, int seq, int layer, const void *rows,
+                                                  const int32_t *positions, int n, void *stream_) {
+  if (!ctx || n < 0) return KVD_ERR_INVALID_ARG;
+  if (!ctx->store8_codes) return KVD_ERR_STATE;
+  if (seq < 0 || seq >= ctx->desc.max_seqs || layer < 0 || layer >= ctx->layers_stored8) return KVD_ERR_INVALID_ARG;
+  if (n == 0) return KVD_OK;
+  if (!rows || !positions) return KVD_ERR_INVALID_ARG;
+  if (!aligned16(rows)) return KVD_ERR_ALIGNMENT;
+  int &count = ctx->rows_stored8[static_cast<size_t>(layer) * ctx->desc.max_seqs + seq];
+  if (count + n > ctx->desc.max_tokens_per_seq) return KVD_ERR_CAPACITY;
+  const size_t slot = store_slot(ctx, layer, seq) + count;
+  kvd_status st = launch_checkpoint_fp8(ctx, static_cast<const __nv_bfloat16 *>(rows), positions,
+                                        ctx->store8_codes + slot * ctx->desc.d_hidden, ctx->store8_pos + slot,
+                                        ctx->store8_sumsq + slot, ctx->store8_scale + slot, n, ctx->desc.d_hidden,
+                                        static_cast<cudaStream_t>(stream_));
+  if (st == KVD_OK) count += n;
+  return st;
+}
+
+extern "C" kvd_status kvd_recompute_kv_fp8(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
+                                           int64_t out_row_stride, void *stream_) {
+  if (!ctx || n_ranges < 0 || n_ranges > KVD_MAX_STORE_RANGES || (n_ranges > 0 && !ranges)) return KVD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  const LayerState &ls = ctx->layers[layer];
+  if (!ls.set || !ctx->store8_codes || !ls.wt8) return KVD_ERR_STATE;
+  if (layer >= ctx->layers_stored8) return KVD_ERR_INVALID_ARG;
+  const kvd_model_desc &d = ctx->desc;
+  const int kdim = d.n_kv_heads * d.d_head;
+  if (out_row_stride < kdim) return KVD_ERR_INVALID_ARG;
+  if (out_row_stride % 8 != 0) return KVD_ERR_ALIGNMENT;
+  RecomputeParams p;
+  int n_jobs = 0, mb = 0;
+  for (int i = 0; i < n_ranges; ++i) {
+    const kvd_store_range &r = ranges[i];
+    if (r.n < 0) return KVD_ERR_INVALID_ARG;
+    if (r.n == 0) continue;
+    if (r.seq < 0 || r.seq >= d.max_seqs || r.first_row < 0) return KVD_ERR_INVALID_ARG;
+    if (!r.k_out || !r.v_out) return KVD_ERR_INVALID_ARG;
+    if (!aligned16(r.k_out) || !aligned16(r.v_out)) return KVD_ERR_ALIGNMENT;
+    const int have = ctx->rows_stored8[static_cast<size_t>(layer) * d.max_seqs + r.seq];
+    if (r.first_row > have || r.n > have - r.first_row) return KVD_ERR_CAPACITY;
+    const size_t slot = store_slot(ctx, layer, r.seq) + r.first_row;
+    RcJob &J = p.jobs[n_jobs++];
+    J.mb_start = mb;
+    J.n = r.n;
+    J.row0 = r.first_row;
+    J.slab = r.seq;
+    J.positions = ctx->store8_pos + slot;
+    J.sumsq = ctx->store8_sumsq + slot;
+    J.scale = ctx->store8_scale + slot;
+    J.k_out = static_cast<__nv_bfloat16 *>(r.k_out);
+    J.v_out = static_cast<__nv_bfloat16 *>(r.v_out);
+    mb += (r.n + 2 * RC_BLOCK_M - 1) / (2 * RC_BLOCK_M);
+  }
+  if (n_jobs == 0) return KVD_OK;
+  p.n_jobs = n_jobs;
+  p.num_k_blocks = (d.d_hidden + 2 * RC_BLOCK_K - 1) / (2 * RC_BLOCK_K);  // 128 channels per k block; the tail reads zeros
+  p.num_m_blocks = mb;
+  p.num_n_blocks = 2 * kdim / ctx->block_n;
+  p.k_cols = kdim;
+  p.out_row_stride = out_row_stride;
+  p.inv_d_hidden = 1.0f / static_cast<float>(d.d_hidden);
+  p.rms_eps = d.rms_eps;
+  p.qk_norm = d.qk_norm;
+  p.qk_eps = d.qk_norm_eps;
+  p.rope_style = d.rope_style;
+  p.rope_hi = ls.rope.hi;
+  p.rope_lo = ls.rope.lo;
+  p.max_pos = ls.rope.n_hi * ROPE_LO_SIZE < d.max_tokens_per_seq ? ls.rope.n_hi * ROPE_LO_SIZE : d.max_tokens_per_seq;
+  p.gamma_k = d.qk_norm ? ls.gamma_k : nullptr;
+  p.status = ctx->d_status;
+  p.timeout_ns = ctx->timeout_ns;
+  p.trace = nullptr;
+  p.ext_rows = nullptr;
+  p.row_chunks = d.d_hidden / 8;
+  p.w_scale = ls.w_scale8;
+  p.wide_store = out_row_stride % 16 == 0;
+  for (int i = 0; i < n_jobs; ++i)
+    if (((reinterpret_cast<uintptr_t>(p.jobs[i].k_out) | reinterpret_cast<uintptr_t>(p.jobs[i].v_out)) & 31u) != 0) p.wide_store = 0;
+  return launch_recompute_fp8(ctx, ls, ctx->store8_maps[layer], p, static_cast<cudaStream_t>(stream_));
 }
 
 extern "C" kvd_status kvd_recompute_kv(kvd_ctx *ctx, int layer, const void *rows, const int32_t *positions, int n,

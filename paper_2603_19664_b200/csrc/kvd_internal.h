@@ -42,6 +42,7 @@ struct RcJob {
   int slab;      // store slab (sequence slot of this layer), or -1: rows come from the caller's buffer
   const int32_t *positions;  // [n]
   const float *sumsq;        // [n] sum of squares of each row (store ranges), nullptr for the caller's rows
+  const float *scale;        // [n] FP8 store: the rows' quantisation scales; nullptr for bf16 rows
   __nv_bfloat16 *k_out;      // row m of the job at k_out + m * out_row_stride
   __nv_bfloat16 *v_out;
 };
@@ -68,6 +69,7 @@ struct RecomputeParams {
   const __nv_bfloat16 *ext_rows;  // the caller's rows (job with slab < 0), [n][d_hidden]
   int row_chunks;                 // d_hidden / 8: 16-byte chunks per row
   int wide_store;                 // outputs are 32-byte aligned: 32-byte stores
+  const float *w_scale;           // FP8 variant: the weight matrix's quantisation scale (one float), else nullptr
   RcJob jobs[RC_MAX_JOBS];
 };
 
@@ -190,6 +192,10 @@ struct LayerState {
   int window = 0;
   RopeTable rope;
   CUtensorMap tmap_b;
+  // FP8 variant: E4M3 codes of W' / w_scale8, K-major; one scale for the matrix (device float)
+  uint8_t *wt8 = nullptr;
+  float *w_scale8 = nullptr;
+  CUtensorMap tmap_b8;
 };
 
 }  // namespace kvd
@@ -210,6 +216,15 @@ struct kvd_ctx {
   int layers_stored = 0;
   std::vector<int> rows_stored;  // [layers_stored * max_seqs]
   std::vector<CUtensorMap> store_maps;  // per stored layer: [max_seqs][max_tokens_per_seq][d_hidden]
+  // FP8 residual store (separate arena): codes, positions, sums of squares of the original rows, scales
+  uint8_t *store8_codes = nullptr;
+  int32_t *store8_pos = nullptr;
+  float *store8_sumsq = nullptr;
+  float *store8_scale = nullptr;
+  int layers_stored8 = 0;
+  std::vector<int> rows_stored8;
+  std::vector<CUtensorMap> store8_maps;
+  unsigned *amax_scratch = nullptr;  // one word, used while weights are prepared
   // attention scratch
   float *part_o = nullptr;
   float *part_ml = nullptr;
@@ -249,6 +264,14 @@ kvd_status launch_prepare_weights(kvd_ctx *ctx, const __nv_bfloat16 *w, const __
 kvd_status launch_convert_gamma(kvd_ctx *ctx, const __nv_bfloat16 *g, float *out, int n, cudaStream_t stream);
 kvd_status launch_rowstats(kvd_ctx *ctx, const __nv_bfloat16 *rows, float *sumsq, int n, int d_hidden,
                            cudaStream_t stream);
+kvd_status launch_checkpoint_fp8(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, uint8_t *dst_codes,
+                                 int32_t *dst_pos, float *dst_sumsq, float *dst_scale, int n, int d_hidden,
+                                 cudaStream_t stream);
+kvd_status launch_prepare_weights_fp8(kvd_ctx *ctx, const __nv_bfloat16 *w, const __nv_bfloat16 *gamma, uint8_t *wt8,
+                                      int d_hidden, int n_cols, unsigned *amax_scratch, float *scale_out,
+                                      cudaStream_t stream);
+kvd_status launch_recompute_fp8(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
+                                const RecomputeParams &p, cudaStream_t stream);
 kvd_status launch_checkpoint(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, __nv_bfloat16 *dst_rows,
                              int32_t *dst_pos, float *dst_sumsq, int n, int d_hidden, cudaStream_t stream);
 kvd_status launch_selftest_timeout(kvd_ctx *ctx, unsigned long long timeout_ns, cudaStream_t stream);

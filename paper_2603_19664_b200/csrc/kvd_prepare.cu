@@ -1,4 +1,6 @@
 // One-time weight preparation and the residual-checkpoint append (STORE_RESIDUAL of Algorithm 1).
+#include <cuda_fp8.h>
+
 #include "kvd_internal.h"
 #include "kvd_ptx.cuh"
 
@@ -76,6 +78,104 @@ __global__ void __launch_bounds__(256) kvd_rowstats_kernel(const uint4 *__restri
   }
 }
 
+// ------------------------------------------------------------------------------ FP8 checkpoints
+// The lower-precision variant (the paper's Section 6 names it as future work and fixes no format; the
+// definition is in kvd.h): a row is stored as E4M3 codes with one fp32 scale, s = max|x| / 448,
+// code = e4m3(x / s) rounded to nearest even and saturating, scale and quotient in IEEE fp32.  The row's
+// sum of squares is taken from the ORIGINAL row with the shared function, so 1/rms is not affected.
+__device__ __forceinline__ uint32_t e4m3x4(float a, float b, float c, float d) {
+  const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(a, b), __NV_SATFINITE, __NV_E4M3);
+  const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(c, d), __NV_SATFINITE, __NV_E4M3);
+  return lo | (hi << 16);
+}
+__global__ void __launch_bounds__(256) kvd_checkpoint_fp8_kernel(const uint4 *__restrict__ rows,
+                                                                 const int32_t *__restrict__ pos,
+                                                                 uint2 *__restrict__ dst_codes,
+                                                                 int32_t *__restrict__ dst_pos,
+                                                                 float *__restrict__ dst_sumsq,
+                                                                 float *__restrict__ dst_scale, int row_chunks, int n) {
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  grid_launch_dependents();
+  for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n; r += warps) {
+    const size_t off = static_cast<size_t>(r) * row_chunks;
+    const uint4 *const src[1] = {rows + off};
+    uint4 *const none[1] = {nullptr};
+    float ss[1];
+    warp_rows_sumsq<1, 10, false>(src, none, row_chunks, lane, ss);
+    // largest magnitude of the row (the row is read again: it sits in L1 / L2)
+    float amax = 0.f;
+    for (int c = lane; c < row_chunks; c += 32) {
+      const uint4 v = __ldg(rows + off + c);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) amax = fmaxf(amax, fmaxf(fabsf(bf16_lo(w[j])), fabsf(bf16_hi(w[j]))));
+    }
+#pragma unroll
+    for (int k = 16; k >= 1; k >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, k));
+    const float scale = __fdiv_rn(fmaxf(amax, 1e-30f), 448.0f);
+    for (int c = lane; c < row_chunks; c += 32) {
+      const uint4 v = __ldg(rows + off + c);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+      float q[8];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        q[2 * j] = __fdiv_rn(bf16_lo(w[j]), scale);
+        q[2 * j + 1] = __fdiv_rn(bf16_hi(w[j]), scale);
+      }
+      dst_codes[off + c] = make_uint2(e4m3x4(q[0], q[1], q[2], q[3]), e4m3x4(q[4], q[5], q[6], q[7]));
+    }
+    if (lane == 0) {
+      dst_sumsq[r] = ss[0];
+      dst_scale[r] = scale;
+      dst_pos[r] = pos[r];
+    }
+  }
+}
+
+// W' = gamma (.) W in fp32 (exact for bf16 inputs): its largest magnitude, then the E4M3 codes of
+// W' / s_w, s_w = max|W'| / 448, stored K-major like the bf16 copy.
+__global__ void __launch_bounds__(256) kvd_weights_amax_kernel(const __nv_bfloat16 *__restrict__ w,
+                                                               const __nv_bfloat16 *__restrict__ gamma, int d_hidden,
+                                                               int n_cols, unsigned *__restrict__ amax_bits) {
+  float m = 0.f;
+  const size_t total = static_cast<size_t>(d_hidden) * n_cols;
+  for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+       i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    const int k = static_cast<int>(i / n_cols);
+    m = fmaxf(m, fabsf(__bfloat162float(gamma[k]) * __bfloat162float(w[i])));
+  }
+#pragma unroll
+  for (int k = 16; k >= 1; k >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, k));
+  if ((threadIdx.x & 31) == 0) atomicMax(amax_bits, __float_as_uint(m));  // non-negative floats order like their bits
+}
+__global__ void __launch_bounds__(256) kvd_prepare_weights_fp8_kernel(const __nv_bfloat16 *__restrict__ w,
+                                                                      const __nv_bfloat16 *__restrict__ gamma,
+                                                                      uint8_t *__restrict__ wt8, int d_hidden, int n_cols,
+                                                                      const unsigned *__restrict__ amax_bits,
+                                                                      float *__restrict__ scale_out) {
+  __shared__ float tile[32][33];
+  const float scale = __fdiv_rn(fmaxf(__uint_as_float(*amax_bits), 1e-30f), 448.0f);
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *scale_out = scale;
+  const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // 32 x 8
+  for (int r = ty; r < 32; r += 8) {
+    const int k = k0 + r, n = n0 + tx;
+    float v = 0.f;
+    if (k < d_hidden && n < n_cols)
+      v = __bfloat162float(gamma[k]) * __bfloat162float(w[static_cast<size_t>(k) * n_cols + n]);
+    tile[r][tx] = v;
+  }
+  __syncthreads();
+  for (int r = ty; r < 32; r += 8) {
+    const int n = n0 + r, k = k0 + tx;
+    if (k < d_hidden && n < n_cols) {
+      const uint32_t c = __nv_cvt_float2_to_fp8x2(make_float2(__fdiv_rn(tile[tx][r], scale), 0.f), __NV_SATFINITE, __NV_E4M3);
+      wt8[static_cast<size_t>(n) * d_hidden + k] = static_cast<uint8_t>(c & 0xffu);
+    }
+  }
+}
+
 // Self-test of the bounded wait: one thread waits on an mbarrier that nothing ever arrives on.  The
 // wait gives up after `timeout_ns`, records STATUS_TIMEOUT and the kernel returns normally.
 __global__ void kvd_selftest_timeout_kernel(int *status, unsigned long long timeout_ns) {
@@ -140,6 +240,37 @@ kvd_status launch_rowstats(kvd_ctx *ctx, const __nv_bfloat16 *rows, float *sumsq
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "launch rowstats");
   ctx->launches += 1;
+  return KVD_OK;
+}
+
+kvd_status launch_checkpoint_fp8(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, uint8_t *dst_codes,
+                                 int32_t *dst_pos, float *dst_sumsq, float *dst_scale, int n, int d_hidden,
+                                 cudaStream_t stream) {
+  long long blocks = (static_cast<long long>(n) + 7) / 8;
+  const long long cap = static_cast<long long>(ctx->num_sms) * 8;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  kvd_checkpoint_fp8_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+      reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint2 *>(dst_codes), dst_pos, dst_sumsq, dst_scale,
+      d_hidden / 8, n);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "launch checkpoint_fp8");
+  ctx->launches += 1;
+  return KVD_OK;
+}
+
+// amax_scratch: one zeroed unsigned on the device; scale_out: one float on the device
+kvd_status launch_prepare_weights_fp8(kvd_ctx *ctx, const __nv_bfloat16 *w, const __nv_bfloat16 *gamma, uint8_t *wt8,
+                                      int d_hidden, int n_cols, unsigned *amax_scratch, float *scale_out,
+                                      cudaStream_t stream) {
+  cudaError_t e = cudaMemsetAsync(amax_scratch, 0, sizeof(unsigned), stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "memset amax");
+  kvd_weights_amax_kernel<<<ctx->num_sms * 4, 256, 0, stream>>>(w, gamma, d_hidden, n_cols, amax_scratch);
+  dim3 grid((n_cols + 31) / 32, (d_hidden + 31) / 32);
+  kvd_prepare_weights_fp8_kernel<<<grid, 256, 0, stream>>>(w, gamma, wt8, d_hidden, n_cols, amax_scratch, scale_out);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "launch prepare_weights_fp8");
+  ctx->launches += 2;
   return KVD_OK;
 }
 

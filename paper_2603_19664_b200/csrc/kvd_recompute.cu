@@ -120,39 +120,43 @@ __device__ __forceinline__ void raise(int *status, int bit, volatile int *abort_
 // stage in both CTAs.  a_lo / b_lo are the low words of the shared-memory descriptors of the stage
 // (the K step advances the start-address field by 32 bytes = 2 units); desc_hi is their common
 // high word.  `acc_first` = 0 makes the first step overwrite the accumulator.
-__device__ __forceinline__ void umma_kblock_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
-                                                 uint32_t idesc, uint32_t acc_first, uint32_t bar_empty) {
-  asm volatile(
-      "{\n\t"
-      ".reg .pred p, t;\n\t"
-      ".reg .b64 da, db;\n\t"
-      ".reg .b32 la, lb;\n\t"
-      "setp.ne.b32 p, %5, 0;\n\t"
-      "setp.eq.b32 t, 0, 0;\n\t"
-      "mov.b64 da, {%1, %3};\n\t"
-      "mov.b64 db, {%2, %3};\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t"
-      "add.u32 la, %1, 2;\n\t"
-      "add.u32 lb, %2, 2;\n\t"
-      "mov.b64 da, {la, %3};\n\t"
-      "mov.b64 db, {lb, %3};\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, t;\n\t"
-      "add.u32 la, %1, 4;\n\t"
-      "add.u32 lb, %2, 4;\n\t"
-      "mov.b64 da, {la, %3};\n\t"
-      "mov.b64 db, {lb, %3};\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, t;\n\t"
-      "add.u32 la, %1, 6;\n\t"
-      "add.u32 lb, %2, 6;\n\t"
-      "mov.b64 da, {la, %3};\n\t"
-      "mov.b64 db, {lb, %3};\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, t;\n\t"
-      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%6], %7;\n\t"
-      "}"
-      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc_first), "r"(bar_empty),
-        "h"(static_cast<uint16_t>(3))
-      : "memory");
+#define KVD_DEFINE_UMMA_KBLOCK(NAME, KIND) \
+__device__ __forceinline__ void NAME(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, \
+                                                 uint32_t idesc, uint32_t acc_first, uint32_t bar_empty) { \
+  asm volatile( \
+      "{\n\t" \
+      ".reg .pred p, t;\n\t" \
+      ".reg .b64 da, db;\n\t" \
+      ".reg .b32 la, lb;\n\t" \
+      "setp.ne.b32 p, %5, 0;\n\t" \
+      "setp.eq.b32 t, 0, 0;\n\t" \
+      "mov.b64 da, {%1, %3};\n\t" \
+      "mov.b64 db, {%2, %3};\n\t" \
+      "tcgen05.mma.cta_group::2.kind::" KIND " [%0], da, db, %4, p;\n\t" \
+      "add.u32 la, %1, 2;\n\t" \
+      "add.u32 lb, %2, 2;\n\t" \
+      "mov.b64 da, {la, %3};\n\t" \
+      "mov.b64 db, {lb, %3};\n\t" \
+      "tcgen05.mma.cta_group::2.kind::" KIND " [%0], da, db, %4, t;\n\t" \
+      "add.u32 la, %1, 4;\n\t" \
+      "add.u32 lb, %2, 4;\n\t" \
+      "mov.b64 da, {la, %3};\n\t" \
+      "mov.b64 db, {lb, %3};\n\t" \
+      "tcgen05.mma.cta_group::2.kind::" KIND " [%0], da, db, %4, t;\n\t" \
+      "add.u32 la, %1, 6;\n\t" \
+      "add.u32 lb, %2, 6;\n\t" \
+      "mov.b64 da, {la, %3};\n\t" \
+      "mov.b64 db, {lb, %3};\n\t" \
+      "tcgen05.mma.cta_group::2.kind::" KIND " [%0], da, db, %4, t;\n\t" \
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%6], %7;\n\t" \
+      "}" \
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc_first), "r"(bar_empty), \
+        "h"(static_cast<uint16_t>(3)) \
+      : "memory"); \
 }
+KVD_DEFINE_UMMA_KBLOCK(umma_kblock_pair, "f16")        // bf16 operands: 64 channels = four K=16 steps
+KVD_DEFINE_UMMA_KBLOCK(umma_kblock_pair_f8, "f8f6f4")  // E4M3 operands: 128 channels = four K=32 steps
+#undef KVD_DEFINE_UMMA_KBLOCK
 
 // Output stores.  Each epilogue thread owns one row, so the 32 lanes of a store instruction write 32
 // different lines and the instruction occupies the SM's load/store data path once per lane -- cycles
@@ -177,7 +181,10 @@ __device__ __forceinline__ void store_row_piece(__nv_bfloat16 *dst, const uint32
   }
 }
 
-template <int BLOCK_N, int D_HEAD, bool TRACE, int FG>
+// EB = bytes per operand element: 2 = bf16 rows and weights, 1 = the FP8 variant (E4M3 codes of rows and
+// weights; a k block is then 128 channels in the same 128-byte rows, the MMA kind f8f6f4, and the rows'
+// and the matrix's quantisation scales ride in the per-row factor that the statistics warps hand over).
+template <int BLOCK_N, int D_HEAD, bool TRACE, int FG, int EB = 2>
 __global__ void __launch_bounds__(RC_THREADS, 1)
 kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __grid_constant__ CUtensorMap tmap_rows,
                      const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ RecomputeParams p,
@@ -185,6 +192,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   using Cfg = RcCfg<BLOCK_N, D_HEAD, FG>;
   constexpr int STAGES = Cfg::STAGES;
   constexpr bool FUSED = FG > 0;
+  static_assert(EB == 2 || (EB == 1 && FG == 0), "the fused variant exists for bf16 operands only");
+  constexpr int KB_ELEMS = RC_BLOCK_K * 2 / EB;  // channels per k block
   static_assert(BLOCK_N % D_HEAD == 0, "a tile must hold whole heads");
 
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -330,7 +339,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
         m0 += p.jobs[job].row0;
         long long waited = 0;
         trace_put<TRACE>(p.trace, ti, 1);
-        for (int k0 = 0; k0 < p.num_k_blocks * RC_BLOCK_K; k0 += RC_BLOCK_K) {
+        for (int k0 = 0; k0 < p.num_k_blocks * KB_ELEMS; k0 += KB_ELEMS) {
           const long long w0 = TRACE ? clock64() : 0;
           if (!mbar_wait(empty, ph ^ 1u, s_abort, tmo)) {
             raise(p.status, STATUS_TIMEOUT, s_abort);
@@ -381,7 +390,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   } else if (warp == 3) {
     if (lane == 0 && cta_rank == 0) {
       // ---------------------------------------------------------------- MMA issuer (even CTA)
-      constexpr uint32_t idesc = umma_idesc_bf16_f32(2 * RC_BLOCK_M, BLOCK_N);
+      constexpr uint32_t idesc = EB == 2 ? umma_idesc_bf16_f32(2 * RC_BLOCK_M, BLOCK_N) : umma_idesc_e4m3_f32(2 * RC_BLOCK_M, BLOCK_N);
       // descriptor words for 128-byte-swizzled K-major tiles: low = start address >> 4 | LBO field (1),
       // high = SBO (1024 B >> 4) | version 1 (bit 46) | swizzle mode 2 (bits 61-63)
       constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
@@ -419,7 +428,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
           }
           if (TRACE) waited += clock64() - w0;
           tc_fence_after();
-          if (FUSED && swap_ab) umma_kblock_pair(d_tmem, a_lo + b_off_units, a_lo, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
+          if (EB == 1) umma_kblock_pair_f8(d_tmem, a_lo, a_lo + b_off_units, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
+          else if (FUSED && swap_ab) umma_kblock_pair(d_tmem, a_lo + b_off_units, a_lo, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
           else umma_kblock_pair(d_tmem, a_lo, a_lo + b_off_units, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
           full += 8u;
           empty += 8u;
@@ -468,6 +478,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
           // squares is read back
           const float sum = row < n_here ? __ldg(J.sumsq + m0 + row) : 0.f;
           rstd_row = 1.0f / sqrtf(sum * p.inv_d_hidden + p.rms_eps);
+          // FP8 rows: the accumulator is a sum of code products; row scale and matrix scale go with 1/rms
+          if (EB == 1) rstd_row *= (row < n_here ? __ldg(J.scale + m0 + row) : 0.f) * __ldg(p.w_scale);
         } else {
           // a few caller rows: the four warps share them in groups of four rows (group g -> warp g % 4),
           // leave 1/rms in s_rstd[a] and meet on a barrier before every thread picks up its own row.
@@ -865,12 +877,13 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
 }
 
 // ------------------------------------------------------------------------------ host launcher
-template <int BLOCK_N, int D_HEAD, bool TRACE, int FG>
+template <int BLOCK_N, int D_HEAD, bool TRACE, int FG, int EB = 2>
 static kvd_status launch_impl(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
                               const CUtensorMap &tmap_rows, const RecomputeParams &p, const FusedParams *fp,
                               cudaStream_t stream) {
   using Cfg = RcCfg<BLOCK_N, D_HEAD, FG>;
-  auto kern = kvd_recompute_kernel<BLOCK_N, D_HEAD, TRACE, FG>;
+  auto kern = kvd_recompute_kernel<BLOCK_N, D_HEAD, TRACE, FG, EB>;
+  const CUtensorMap &tmap_b = EB == 1 ? ls.tmap_b8 : ls.tmap_b;
   static bool configured[64] = {};
   if (!configured[ctx->device & 63]) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
@@ -897,8 +910,8 @@ static kvd_status launch_impl(kvd_ctx *ctx, const LayerState &ls, const CUtensor
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   cudaError_t le;
-  if constexpr (FG > 0) le = cudaLaunchKernelEx(&cfg, kern, tmap_store, tmap_rows, ls.tmap_b, p, *fp);
-  else le = cudaLaunchKernelEx(&cfg, kern, tmap_store, tmap_rows, ls.tmap_b, p, NoFusedParams());
+  if constexpr (FG > 0) le = cudaLaunchKernelEx(&cfg, kern, tmap_store, tmap_rows, tmap_b, p, *fp);
+  else le = cudaLaunchKernelEx(&cfg, kern, tmap_store, tmap_rows, tmap_b, p, NoFusedParams());
   if (le != cudaSuccess) return cuda_fail(ctx, le, "launch recompute");
   ctx->launches += 1;
   return KVD_OK;
@@ -942,6 +955,21 @@ kvd_status launch_recompute_fused(kvd_ctx *ctx, const LayerState &ls, const CUte
   if (dh == 128 && g == 2) return launch_sel<256, 128, 2>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
   if (dh == 128 && g == 1) return launch_sel<256, 128, 1>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
   return KVD_ERR_UNSUPPORTED;
+}
+
+// The FP8 variant: rows and weights as E4M3 codes (tmap_store is the FP8 store's map).
+kvd_status launch_recompute_fp8(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
+                                const RecomputeParams &p, cudaStream_t stream) {
+  const int dh = ctx->desc.d_head;
+  if (ctx->block_n == 256) {
+    if (dh == 256) return launch_impl<256, 256, false, 0, 1>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
+    if (dh == 128) return launch_impl<256, 128, false, 0, 1>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
+    if (dh == 64) return launch_impl<256, 64, false, 0, 1>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
+  } else if (ctx->block_n == 128) {
+    if (dh == 128) return launch_impl<128, 128, false, 0, 1>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
+    if (dh == 64) return launch_impl<128, 64, false, 0, 1>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
+  }
+  return KVD_ERR_SHAPE;
 }
 
 }  // namespace kvd
