@@ -243,6 +243,9 @@ class Workload:
         self.ctx.kvd_attach_workspace(self.ws)
         self.arena = torch.empty(kvd.kvd_store_bytes(self.desc, 1), dtype=torch.uint8, device="cuda")
         self.ctx.kvd_attach_store(self.arena, 1)
+        # the FP8 checkpoint variant's store (a second arena), filled once per set below
+        self.arena8 = torch.empty(kvd.kvd_store_bytes_fp8(self.desc, 1), dtype=torch.uint8, device="cuda")
+        self.ctx.kvd_attach_store_fp8(self.arena8, 1)
         x_bits = make_residuals(shape, T + 1, seed=2, outliers=True)
         self.x_host_bits = x_bits
         x0 = dev(x_bits)
@@ -308,6 +311,16 @@ class Workload:
         self.ctx.kvd_decode_attention(0, 1, self.q[s:s + 1], [T],
                                       [[(K, V, self.kdim, 0, T), (K[T:], V[T:], self.kdim, T, 1)]], 0.0,
                                       self.out[s:s + 1])
+
+    def k_checkpoint_fp8(self, i):
+        s = i % self.n_sets
+        self.ctx.kvd_reset_sequence_fp8(s)
+        self.ctx.kvd_checkpoint_residual_fp8(s, 0, self.X[s], self.pos, self.T)
+
+    def k_recompute_fp8(self, i):
+        # RECOMPUTE_KV from E4M3 checkpoints (rows and weights as FP8 codes, tensor-core kind f8f6f4)
+        s = i % self.n_sets
+        self.ctx.kvd_recompute_kv_fp8(0, [(s, 0, self.T, self.K[s], self.V[s])], self.kdim)
 
     def k_two_call(self, i):
         # recompute (T stored rows + the current token) followed by attention: the step's two K/V launches
@@ -464,6 +477,8 @@ def run_gpu(args):
               "recompute_with_current_token": timed_graph(wl.k_recompute_step, 10),
               "recompute_from_caller_rows": timed_graph(wl.k_recompute_rows, 10),
               "current_token_kv_alone": timed_graph(wl.k_current, 10), "attention": timed_graph(wl.k_attention, 10),
+              "checkpoint_fp8": timed_graph(wl.k_checkpoint_fp8, 10),
+              "recompute_from_fp8_checkpoints": timed_graph(wl.k_recompute_fp8, 10),
               "recompute_then_attention_two_calls": timed_graph(wl.k_two_call, 10),
               "recompute_fused_into_attention": timed_graph(wl.k_fused, 10)}
     read_attn_ms = timed_graph(wl.cached_read_step, 10)
@@ -585,6 +600,15 @@ def run_gpu(args):
                          "in_step_us": float(np.mean(t_gemm)) * 1e3,
                          "timing": "graph of back-to-back launches on rotating inputs, CUDA events, per launch",
                          "frac_of_sustained": flops / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]},
+            # the FP8 checkpoint variant of the same launch: same flop count, E4M3 operands; its peak is the
+            # measured bf16 peak times the nominal fp8 : bf16 ratio of 2 (no fp8 GEMM was measured on this machine)
+            "roofline_fp8": {"kernel": "kvd_recompute_kernel<256,256,...,EB=1> (E4M3 rows and weights)", "bound": "tensor",
+                             "achieved": flops / (iso_ms["recompute_from_fp8_checkpoints"] * 1e-3) / 1e12,
+                             "peak": 2 * peaks["bf16_tflops"], "unit": "TFLOP/s",
+                             "frac": flops / (iso_ms["recompute_from_fp8_checkpoints"] * 1e-3) / 1e12 / (2 * peaks["bf16_tflops"]),
+                             "peak_source": peaks["source"] + " bf16 burst x 2 (nominal fp8 ratio)",
+                             "avg_launch_us": iso_ms["recompute_from_fp8_checkpoints"] * 1e3,
+                             "checkpoint_bytes_per_token": shape.d_hidden + 12, "traffic": None},
             "roofline_attention": {"kernel": "kvd_attn_split_kernel<256,2> + merge", "bound": "hbm",
                                    "achieved": attn_bytes / (attn_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                                    "unit": "GB/s", "frac": attn_bytes / (attn_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],

@@ -223,10 +223,10 @@ kvd_status kvd_recompute_kv_step(kvd_ctx *ctx, int layer, const kvd_store_range 
  * paper's Section 6, which fixes no format; this is the definition this library implements) ----
  * A residual row x (bf16) is stored as E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits,
  * largest finite value 448) with one fp32 scale per row:
- *     s_x = max|x| / 448,    code_k = e4m3(x_k / s_x)   round to nearest even, saturating, both steps in fp32,
+ *     s_x = max|x| / 448,    code_k = e4m3(x_k * (448 / max|x|))   round to nearest even, saturating, all in fp32,
  * together with its position and the sum of squares of the ORIGINAL row (1/rms of Eq. 2 is not affected by
  * the quantisation).  The folded weights W' = gamma (.) W_kv get one scale for the whole matrix,
- * s_w = max|W'| / 448, code = e4m3(W' / s_w) (prepared by kvd_set_layer next to the bf16 copy).
+ * s_w = max|W'| / 448, code = e4m3(W' * (448 / max|W'|)) (prepared by kvd_set_layer next to the bf16 copy).
  * RECOMPUTE_KV from such rows is Eq. 13-14 on the dequantised operands,
  *     y = (s_x s_w / rms(x)) * sum_k code_x[k] code_w[k][:],   then key norm and rotation as usual,
  * with the code products accumulated on the tensor cores (kind f8f6f4, fp32 accumulation).  Per token and
@@ -236,11 +236,12 @@ kvd_status kvd_recompute_kv_step(kvd_ctx *ctx, int layer, const kvd_store_range 
  * do not depend on the batch it is recomputed in).
  * The FP8 store is a second, independent arena (layout: codes uint8 [layers][max_seqs][max_tokens][d_hidden],
  * then positions int32, sums of squares fp32, scales fp32, each [layers][max_seqs][max_tokens] and each
- * region starting at a 256-byte multiple); kvd_reset_sequence clears a sequence in both stores.
+ * region starting at a 256-byte multiple) with row counts of its own (kvd_reset_sequence_fp8).
  * kvd_store_bytes_fp8 returns 0 for shapes the variant does not support (d_hidden % 16 != 0). */
 size_t kvd_store_bytes_fp8(const kvd_model_desc *desc, int layers_stored);
 kvd_status kvd_attach_store_fp8(kvd_ctx *ctx, void *arena, size_t bytes, int layers_stored);
 int kvd_rows_stored_fp8(const kvd_ctx *ctx, int layer, int seq);
+kvd_status kvd_reset_sequence_fp8(kvd_ctx *ctx, int seq);
 /* Append n rows (DEVICE bf16 [n, d_hidden], 16-byte aligned; DEVICE int32 positions[n]) in quantised form. */
 kvd_status kvd_checkpoint_residual_fp8(kvd_ctx *ctx, int seq, int layer, const void *rows, const int32_t *positions,
                                        int n, void *stream);

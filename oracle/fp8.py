@@ -4,11 +4,13 @@ The paper names lower-precision checkpoints as future work (its Section 6, secon
 format, so the variant is defined here and in include/kvd.h:
 
   * a residual row x (bf16) is stored as E4M3 codes with one fp32 scale per row,
-        s_x = max(|x|) / 448,   code_k = e4m3_rne_sat(x_k / s_x)       (both steps in fp32),
+        s_x = max(|x|) / 448,   code_k = e4m3_rne_sat(x_k * r_x),  r_x = 448 / max(|x|)   (all in fp32),
     together with the row's sum of squares taken from the ORIGINAL row (the RMSNorm statistic of Eq. 2 is
     not affected by the quantisation);
   * the folded weights W' = gamma (.) W_kv (Eq. 1 composed with Eq. 13-14) are stored as E4M3 codes with one
-    fp32 scale for the whole matrix, s_w = max|W'| / 448, code = e4m3_rne_sat(W' / s_w), W' formed in fp32;
+    fp32 scale for the whole matrix, s_w = max|W'| / 448, code = e4m3_rne_sat(W' * (448 / max|W'|)), W' and
+    the reciprocal formed in fp32 (a multiplication by the rounded reciprocal, not a division: one division
+    per row instead of one per element on the GPU; the decoded value is still code * s);
   * RECOMPUTE_KV then is Eq. 13-14 on the dequantised operands:
         y = (s_x s_w / rms(x)) * sum_k code_x[k] code_w[k][:]      followed by key norm and rotation as usual.
 
@@ -18,7 +20,7 @@ no infinities, largest finite value 448, subnormal step 2^-9, round to nearest e
 own float8_e4m3fn conversion on the CPU as an independent library routine.
 
 The codes are an encoding decided in floating point, so both sides take that decision in the same
-precision: the scale, the division and the rounding input are fp32 here exactly as in the kernel.
+precision: the scale, the reciprocal, the product and the rounding input are fp32 here exactly as in the kernel.
 """
 from __future__ import annotations
 
@@ -48,8 +50,10 @@ def quantize_rows(X_f64: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
     fp64 [n]) with row r represented by values[r] * scales[r].  Scale and quotient are formed in fp32."""
     X = np.asarray(X_f64, dtype=np.float32)
     amax = np.max(np.abs(X), axis=1)
-    s = (np.maximum(amax, np.float32(1e-30)) / np.float32(E4M3_MAX)).astype(np.float32)
-    quot = (X / s[:, None]).astype(np.float32)
+    amax = np.maximum(amax, np.float32(1e-30))
+    s = (amax / np.float32(E4M3_MAX)).astype(np.float32)
+    r = (np.float32(E4M3_MAX) / amax).astype(np.float32)
+    quot = (X * r[:, None]).astype(np.float32)
     return e4m3_round(quot.astype(np.float64)), s.astype(np.float64)
 
 
@@ -58,8 +62,9 @@ def quantize_weights(gamma_f64: np.ndarray, W_f64: np.ndarray) -> Tuple[np.ndarr
     the E4M3 grid [d_hidden, n_cols] as fp64, scale)."""
     Wp = (np.asarray(gamma_f64, dtype=np.float32)[:, None] * np.asarray(W_f64, dtype=np.float32)).astype(np.float32)
     amax = np.float32(np.max(np.abs(Wp)))
-    s = np.float32(max(amax, np.float32(1e-30))) / np.float32(E4M3_MAX)
-    quot = (Wp / s).astype(np.float32)
+    amax = np.float32(max(amax, np.float32(1e-30)))
+    s = amax / np.float32(E4M3_MAX)
+    quot = (Wp * (np.float32(E4M3_MAX) / amax)).astype(np.float32)
     return e4m3_round(quot.astype(np.float64)), float(s)
 
 

@@ -32,7 +32,7 @@ KVD_MAX_SEGMENTS = 4
 EXPORTED_SYMBOLS = (
     "kvd_create", "kvd_destroy", "kvd_set_layer", "kvd_store_bytes", "kvd_attach_store", "kvd_reset_sequence",
     "kvd_decode_attention_recompute",
-    "kvd_store_bytes_fp8", "kvd_attach_store_fp8", "kvd_rows_stored_fp8", "kvd_checkpoint_residual_fp8", "kvd_recompute_kv_fp8",
+    "kvd_store_bytes_fp8", "kvd_attach_store_fp8", "kvd_rows_stored_fp8", "kvd_reset_sequence_fp8", "kvd_checkpoint_residual_fp8", "kvd_recompute_kv_fp8",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
     "kvd_recompute_kv_step",
     "kvd_decode_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
@@ -127,6 +127,8 @@ def load() -> ctypes.CDLL:
     lib.kvd_attach_store_fp8.restype = i32
     lib.kvd_rows_stored_fp8.argtypes = [vp, i32, i32]
     lib.kvd_rows_stored_fp8.restype = i32
+    lib.kvd_reset_sequence_fp8.argtypes = [vp, i32]
+    lib.kvd_reset_sequence_fp8.restype = i32
     lib.kvd_checkpoint_residual_fp8.argtypes = [vp, i32, i32, vp, vp, i32, vp]
     lib.kvd_checkpoint_residual_fp8.restype = i32
     lib.kvd_recompute_kv_fp8.argtypes = [vp, i32, ctypes.POINTER(kvd_store_range), i32, i64, vp]
@@ -346,6 +348,9 @@ class Kvd:
         self._keep.append(arena)
         self._check(self._lib.kvd_attach_store_fp8(self._h, _ptr(arena), arena.numel() * arena.element_size(),
                                                    layers_stored), "kvd_attach_store_fp8")
+
+    def kvd_reset_sequence_fp8(self, seq: int) -> None:
+        self._check(self._lib.kvd_reset_sequence_fp8(self._h, seq), "kvd_reset_sequence_fp8")
 
     def kvd_rows_stored_fp8(self, layer: int, seq: int) -> int:
         return int(self._lib.kvd_rows_stored_fp8(self._h, layer, seq))

@@ -329,8 +329,14 @@ extern "C" kvd_status kvd_attach_store(kvd_ctx *ctx, void *arena, size_t bytes, 
 
 extern "C" kvd_status kvd_reset_sequence(kvd_ctx *ctx, int seq) {
   if (!ctx || seq < 0 || seq >= ctx->desc.max_seqs) return KVD_ERR_INVALID_ARG;
-  if (!ctx->store_rows && !ctx->store8_codes) return KVD_ERR_STATE;
+  if (!ctx->store_rows) return KVD_ERR_STATE;
   for (int l = 0; l < ctx->layers_stored; ++l) ctx->rows_stored[static_cast<size_t>(l) * ctx->desc.max_seqs + seq] = 0;
+  return KVD_OK;
+}
+
+extern "C" kvd_status kvd_reset_sequence_fp8(kvd_ctx *ctx, int seq) {
+  if (!ctx || seq < 0 || seq >= ctx->desc.max_seqs) return KVD_ERR_INVALID_ARG;
+  if (!ctx->store8_codes) return KVD_ERR_STATE;
   for (int l = 0; l < ctx->layers_stored8; ++l) ctx->rows_stored8[static_cast<size_t>(l) * ctx->desc.max_seqs + seq] = 0;
   return KVD_OK;
 }

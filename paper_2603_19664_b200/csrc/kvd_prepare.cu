@@ -81,13 +81,16 @@ __global__ void __launch_bounds__(256) kvd_rowstats_kernel(const uint4 *__restri
 // ------------------------------------------------------------------------------ FP8 checkpoints
 // The lower-precision variant (the paper's Section 6 names it as future work and fixes no format; the
 // definition is in kvd.h): a row is stored as E4M3 codes with one fp32 scale, s = max|x| / 448,
-// code = e4m3(x / s) rounded to nearest even and saturating, scale and quotient in IEEE fp32.  The row's
+// code = e4m3(x * (448 / max|x|)) rounded to nearest even and saturating, everything in IEEE fp32.  The row's
 // sum of squares is taken from the ORIGINAL row with the shared function, so 1/rms is not affected.
 __device__ __forceinline__ uint32_t e4m3x4(float a, float b, float c, float d) {
   const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(a, b), __NV_SATFINITE, __NV_E4M3);
   const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(c, d), __NV_SATFINITE, __NV_E4M3);
   return lo | (hi << 16);
 }
+// CPL > 0: rows of at most 32 * CPL chunks are held in registers (one pass over memory); CPL = 0: any
+// width, the row is read three times (it sits in L1 / L2 after the first).  The arithmetic is the same.
+template <int CPL>
 __global__ void __launch_bounds__(256) kvd_checkpoint_fp8_kernel(const uint4 *__restrict__ rows,
                                                                  const int32_t *__restrict__ pos,
                                                                  uint2 *__restrict__ dst_codes,
@@ -97,37 +100,66 @@ __global__ void __launch_bounds__(256) kvd_checkpoint_fp8_kernel(const uint4 *__
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   grid_launch_dependents();
+  auto chunk_amax = [](const uint4 &v, float amax) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) amax = fmaxf(amax, fmaxf(fabsf(bf16_lo(w[j])), fabsf(bf16_hi(w[j]))));
+    return amax;
+  };
+  auto chunk_codes = [](const uint4 &v, float recip) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    float q[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      q[2 * j] = __fmul_rn(bf16_lo(w[j]), recip);
+      q[2 * j + 1] = __fmul_rn(bf16_hi(w[j]), recip);
+    }
+    return make_uint2(e4m3x4(q[0], q[1], q[2], q[3]), e4m3x4(q[4], q[5], q[6], q[7]));
+  };
   for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n; r += warps) {
     const size_t off = static_cast<size_t>(r) * row_chunks;
-    const uint4 *const src[1] = {rows + off};
-    uint4 *const none[1] = {nullptr};
-    float ss[1];
-    warp_rows_sumsq<1, 10, false>(src, none, row_chunks, lane, ss);
-    // largest magnitude of the row (the row is read again: it sits in L1 / L2)
-    float amax = 0.f;
-    for (int c = lane; c < row_chunks; c += 32) {
-      const uint4 v = __ldg(rows + off + c);
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    float ss, amax = 0.f;
+    if constexpr (CPL > 0) {
+      uint4 v[CPL];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) amax = fmaxf(amax, fmaxf(fabsf(bf16_lo(w[j])), fabsf(bf16_hi(w[j]))));
-    }
-#pragma unroll
-    for (int k = 16; k >= 1; k >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, k));
-    const float scale = __fdiv_rn(fmaxf(amax, 1e-30f), 448.0f);
-    for (int c = lane; c < row_chunks; c += 32) {
-      const uint4 v = __ldg(rows + off + c);
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-      float q[8];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        q[2 * j] = __fdiv_rn(bf16_lo(w[j]), scale);
-        q[2 * j + 1] = __fdiv_rn(bf16_hi(w[j]), scale);
+      for (int i = 0; i < CPL; ++i) {
+        const int c = lane + 32 * i;
+        v[i] = c < row_chunks ? __ldg(rows + off + c) : make_uint4(0u, 0u, 0u, 0u);
       }
-      dst_codes[off + c] = make_uint2(e4m3x4(q[0], q[1], q[2], q[3]), e4m3x4(q[4], q[5], q[6], q[7]));
+      // the lane's chunks in ascending order, as warp_rows_sumsq takes them (absent chunks add exact zeros)
+      uint64_t ps2[4] = {0ull, 0ull, 0ull, 0ull};
+#pragma unroll
+      for (int i = 0; i < CPL; ++i) {
+        sumsq_chunk(ps2, v[i]);
+        amax = chunk_amax(v[i], amax);
+      }
+      ss = sumsq_finish(ps2);
+#pragma unroll
+      for (int k = 16; k >= 1; k >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, k));
+      amax = fmaxf(amax, 1e-30f);
+      const float scale = __fdiv_rn(amax, 448.0f), recip = __fdiv_rn(448.0f, amax);
+#pragma unroll
+      for (int i = 0; i < CPL; ++i) {
+        const int c = lane + 32 * i;
+        if (c < row_chunks) dst_codes[off + c] = chunk_codes(v[i], recip);
+      }
+      if (lane == 0) dst_scale[r] = scale;
+    } else {
+      const uint4 *const src[1] = {rows + off};
+      uint4 *const none[1] = {nullptr};
+      float s1[1];
+      warp_rows_sumsq<1, 10, false>(src, none, row_chunks, lane, s1);
+      ss = s1[0];
+      for (int c = lane; c < row_chunks; c += 32) amax = chunk_amax(__ldg(rows + off + c), amax);
+#pragma unroll
+      for (int k = 16; k >= 1; k >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, k));
+      amax = fmaxf(amax, 1e-30f);
+      const float scale = __fdiv_rn(amax, 448.0f), recip = __fdiv_rn(448.0f, amax);
+      for (int c = lane; c < row_chunks; c += 32) dst_codes[off + c] = chunk_codes(__ldg(rows + off + c), recip);
+      if (lane == 0) dst_scale[r] = scale;
     }
     if (lane == 0) {
-      dst_sumsq[r] = ss[0];
-      dst_scale[r] = scale;
+      dst_sumsq[r] = ss;
       dst_pos[r] = pos[r];
     }
   }
@@ -155,7 +187,8 @@ __global__ void __launch_bounds__(256) kvd_prepare_weights_fp8_kernel(const __nv
                                                                       const unsigned *__restrict__ amax_bits,
                                                                       float *__restrict__ scale_out) {
   __shared__ float tile[32][33];
-  const float scale = __fdiv_rn(fmaxf(__uint_as_float(*amax_bits), 1e-30f), 448.0f);
+  const float amax = fmaxf(__uint_as_float(*amax_bits), 1e-30f);
+  const float scale = __fdiv_rn(amax, 448.0f), recip = __fdiv_rn(448.0f, amax);
   if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *scale_out = scale;
   const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // 32 x 8
@@ -170,7 +203,7 @@ __global__ void __launch_bounds__(256) kvd_prepare_weights_fp8_kernel(const __nv
   for (int r = ty; r < 32; r += 8) {
     const int n = n0 + r, k = k0 + tx;
     if (k < d_hidden && n < n_cols) {
-      const uint32_t c = __nv_cvt_float2_to_fp8x2(make_float2(__fdiv_rn(tile[tx][r], scale), 0.f), __NV_SATFINITE, __NV_E4M3);
+      const uint32_t c = __nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(tile[tx][r], recip), 0.f), __NV_SATFINITE, __NV_E4M3);
       wt8[static_cast<size_t>(n) * d_hidden + k] = static_cast<uint8_t>(c & 0xffu);
     }
   }
@@ -250,9 +283,15 @@ kvd_status launch_checkpoint_fp8(kvd_ctx *ctx, const __nv_bfloat16 *rows, const 
   const long long cap = static_cast<long long>(ctx->num_sms) * 8;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  kvd_checkpoint_fp8_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
-      reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint2 *>(dst_codes), dst_pos, dst_sumsq, dst_scale,
-      d_hidden / 8, n);
+  const int row_chunks = d_hidden / 8;
+  if (row_chunks <= 320)
+    kvd_checkpoint_fp8_kernel<10><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+        reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint2 *>(dst_codes), dst_pos, dst_sumsq, dst_scale,
+        row_chunks, n);
+  else
+    kvd_checkpoint_fp8_kernel<0><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+        reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint2 *>(dst_codes), dst_pos, dst_sumsq, dst_scale,
+        row_chunks, n);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "launch checkpoint_fp8");
   ctx->launches += 1;

@@ -329,6 +329,16 @@ __device__ __forceinline__ void sumsq_chunk(uint64_t (&ps2)[4], const uint4 &v) 
   x2 = bf16x2_to_f32x2(v.z); ps2[2] = ffma2(x2, x2, ps2[2]);
   x2 = bf16x2_to_f32x2(v.w); ps2[3] = ffma2(x2, x2, ps2[3]);
 }
+// the eight partial sums of a lane in a fixed tree, then the xor butterfly over the warp
+__device__ __forceinline__ float sumsq_finish(const uint64_t (&ps2)[4]) {
+  float ps[8];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) unpack2(ps2[j], ps[2 * j], ps[2 * j + 1]);
+  float sum = ((ps[0] + ps[1]) + (ps[2] + ps[3])) + ((ps[4] + ps[5]) + (ps[6] + ps[7]));
+#pragma unroll
+  for (int k = 16; k >= 1; k >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, k);
+  return sum;
+}
 template <int R, int B, bool COPY>
 __device__ __forceinline__ void warp_rows_sumsq(const uint4 *const (&src)[R], uint4 *const (&dst)[R], int n_chunks, int lane,
                                                 float (&out)[R]) {
@@ -365,15 +375,7 @@ __device__ __forceinline__ void warp_rows_sumsq(const uint4 *const (&src)[R], ui
     }
   }
 #pragma unroll
-  for (int r = 0; r < R; ++r) {
-    float ps[8];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) unpack2(ps2[r][j], ps[2 * j], ps[2 * j + 1]);
-    float sum = ((ps[0] + ps[1]) + (ps[2] + ps[3])) + ((ps[4] + ps[5]) + (ps[6] + ps[7]));
-#pragma unroll
-    for (int k = 16; k >= 1; k >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, k);
-    out[r] = sum;
-  }
+  for (int r = 0; r < R; ++r) out[r] = sumsq_finish(ps2[r]);
 }
 
 }  // namespace kvd

@@ -63,6 +63,15 @@ def test_stored_codes_scales_and_statistics_equal_the_oracles_quantisation():
     assert np.array_equal(got_pos, pos)
     ref = np.sum(Xf ** 2, axis=1)
     assert np.max(np.abs(got_ss - ref) / ref) < 1e-6
+    # the statistic has the bits the bf16 store keeps for the same rows (one function takes it everywhere)
+    arena16 = torch.zeros(kvd.kvd_store_bytes(ctx.desc, 1), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_store(arena16, 1)
+    ctx.kvd_checkpoint_residual(1, 0, x, p, n)
+    torch.cuda.synchronize()
+    a16 = arena16.cpu().numpy()
+    r_bytes = ru(slots * shape.d_hidden * 2)
+    ss16 = a16[r_bytes + f_bytes:].view(np.float32)[max_tokens:max_tokens + n]
+    assert np.array_equal(ss16.view(np.uint32), got_ss.view(np.uint32))
 
 
 @pytest.mark.parametrize("shape,n", [(GEMMA3_4B_GLOBAL, 300), (GEMMA3_4B_GLOBAL, 1), (QWEN3_4B, 700), (SMOLLM2_135M, 130)],
