@@ -381,6 +381,10 @@ def run_gpu(args):
         # plain eager launches for a profiler: no graphs, no auxiliary measurements
         for i in range(steps):
             wl.step(warmup + i)
+        # the FP8 checkpoint variant of the same layer: quantising checkpoint + recompute, two sets
+        for i in range(2):
+            wl.k_checkpoint_fp8(i)
+            wl.k_recompute_fp8(i)
         barrier()
         if args.profile_long_attn:
             # a few eager decode-attention calls over 32769 keys (134 MB each, larger than L2)
