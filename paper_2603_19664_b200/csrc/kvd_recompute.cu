@@ -28,13 +28,21 @@
 //
 // The producer and the MMA issuer are single threads whose loop must finish well inside the 512
 // clocks a k block of MMAs takes; their loops are therefore kept to a few dozen instructions
-// (incremental addresses, one asm block per k block).  Every wait is bounded; on expiry the kernel records STATUS_TIMEOUT and drains.
+// (incremental addresses, one asm block per k block).  Every wait is bounded; on expiry the kernel
+// records STATUS_TIMEOUT and drains.
 //
 // Bit-reproducibility: the k loop always runs over all of d_hidden in ascending order with one MMA
 // shape, a row's sum of squares is taken by one function in one fixed order wherever it is taken
-// (warp_row_sumsq), the key norm is reduced by the single thread that owns the row, and cos/sin
+// (warp_rows_sumsq), the key norm is reduced by the single thread that owns the row, and cos/sin
 // depend on (position, channel) only.  A row's output bits are therefore independent of M, of the
 // row's index and of whether it came from the store or from the caller.
+//
+// Variants of the one kernel (template arguments):
+//   FG > 0  recompute fused into attention (kvd_decode_attention_recompute): for a job that carries a
+//           query the key tile's epilogue turns keys into scores and the value tile is produced
+//           transposed and reduced with the softmax weights; nothing of K or V is written.
+//   EB = 1  FP8 checkpoints (kvd_recompute_kv_fp8): rows and weights are E4M3 codes, a k block is 128
+//           channels, the MMA kind is f8f6f4; the scales ride in the per-row factor of the epilogue.
 #include <math_constants.h>
 #include <string.h>
 
@@ -48,10 +56,18 @@ namespace kvd {
 // FG = 0: the plain kernel (K and V are stored).  FG > 0: the fused variant for models with FG query
 // heads per KV head -- jobs that carry a query attend over their rows inside the kernel (see the
 // epilogue); it gives one ring stage to the score buffers.
-template <int BLOCK_N, int D_HEAD, int FG = 0>
+// LOSM: the low rotation table (d_head/2 pairs x 16 positions, 64 B per channel) sits in shared memory
+// instead of being read through L1.  The table and the high table's rows do not fit the L1 that is left
+// beside the ring (a third of the epilogue's global loads miss, and a key tile's epilogue spends more
+// than half its time on them); in shared memory the table costs a ring stage.  Launches whose key-tile
+// epilogues are exposed (one tile per cluster; the FP8 variant, whose main loop is shorter than that
+// epilogue; the fused variant, which has given a stage away already) take LOSM, the others the seventh
+// stage.  The arithmetic is the same either way.
+template <int BLOCK_N, int D_HEAD, int FG = 0, bool LOSM = false>
 struct RcCfg {
   static constexpr bool FUSED = FG > 0;
-  static constexpr int STAGES = FUSED ? 6 : (BLOCK_N == 256 ? 7 : 9);  // all the shared memory an SM has: the ring is latency-bound
+  static_assert(!FUSED || LOSM, "the fused variant keeps the low table in shared memory");
+  static constexpr int STAGES = (BLOCK_N == 256 ? 7 : 9) - ((FUSED || LOSM) ? 1 : 0);  // all the shared memory an SM has: the ring is latency-bound
   static constexpr int A_BYTES = RC_BLOCK_M * RC_BLOCK_K * 2;
   static constexpr int B_ROWS = BLOCK_N / 2;  // this CTA's half of the W' tile
   static constexpr int B_BYTES = B_ROWS * RC_BLOCK_K * 2;
@@ -66,7 +82,8 @@ struct RcCfg {
   // [2 units][256], partial sums of the weights [heads x FG][4 warps]
   static constexpr int GT = (BLOCK_N / D_HEAD) * (FUSED ? FG : 0);
   static constexpr int FUSED_BYTES = FUSED ? (2 * GT * 256 + 2 * 256 + GT * 4) * 4 : 0;
-  static constexpr int TAIL_BYTES = BAR_BYTES + 16 /*tmem ptr, abort*/ + 2 * RC_BLOCK_M * 4 /*rstd*/ + 256 * 4 /*gamma_k*/ + FUSED_BYTES;
+  static constexpr int LO_BYTES = LOSM ? (D_HEAD / 2) * ROPE_LO_SIZE * 8 : 0;
+  static constexpr int TAIL_BYTES = BAR_BYTES + 16 /*tmem ptr, abort*/ + 2 * RC_BLOCK_M * 4 /*rstd*/ + 256 * 4 /*gamma_k*/ + FUSED_BYTES + LO_BYTES;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + TAIL_BYTES;  // the base must be 1024-byte aligned
   static_assert(SMEM_BYTES <= 232448, "more shared memory than an SM offers");
 };
@@ -184,12 +201,12 @@ __device__ __forceinline__ void store_row_piece(__nv_bfloat16 *dst, const uint32
 // EB = bytes per operand element: 2 = bf16 rows and weights, 1 = the FP8 variant (E4M3 codes of rows and
 // weights; a k block is then 128 channels in the same 128-byte rows, the MMA kind f8f6f4, and the rows'
 // and the matrix's quantisation scales ride in the per-row factor that the statistics warps hand over).
-template <int BLOCK_N, int D_HEAD, bool TRACE, int FG, int EB = 2>
+template <int BLOCK_N, int D_HEAD, bool TRACE, int FG, int EB = 2, bool LOSM = (FG > 0)>
 __global__ void __launch_bounds__(RC_THREADS, 1)
 kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __grid_constant__ CUtensorMap tmap_rows,
                      const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ RecomputeParams p,
                      const __grid_constant__ std::conditional_t<(FG > 0), FusedParams, NoFusedParams> f) {
-  using Cfg = RcCfg<BLOCK_N, D_HEAD, FG>;
+  using Cfg = RcCfg<BLOCK_N, D_HEAD, FG, LOSM>;
   constexpr int STAGES = Cfg::STAGES;
   constexpr bool FUSED = FG > 0;
   static_assert(EB == 2 || (EB == 1 && FG == 0), "the fused variant exists for bf16 operands only");
@@ -211,6 +228,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   float *s_sc = s_gamma_k + 256;                 // fused: [2][GT][256]
   float *s_rall = s_sc + 2 * Cfg::GT * 256;      // fused: [2][256]
   float *s_lsum = s_rall + 2 * 256;              // fused: [GT][4]
+  // LOSM: the low rotation table [pair][16], behind whatever precedes it in this variant's tail
+  float2 *s_lo = reinterpret_cast<float2 *>(FUSED ? s_lsum + Cfg::GT * 4 : s_gamma_k + 256);
 
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_base = smem_u32(bars);
@@ -301,6 +320,12 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
     prefetch_tensormap(&tmap_b);
   }
   if (threadIdx.x < D_HEAD) s_gamma_k[threadIdx.x] = p.gamma_k ? p.gamma_k[threadIdx.x] : 1.0f;
+  if constexpr (LOSM) {
+    // (written at kvd_set_layer time: may be read before the dependency wait below)
+    const uint4 *src = reinterpret_cast<const uint4 *>(p.rope_lo);
+    uint4 *dstl = reinterpret_cast<uint4 *>(s_lo);
+    for (int i = threadIdx.x; i < Cfg::LO_BYTES / 16; i += RC_THREADS) dstl[i] = __ldg(src + i);
+  }
   if (warp == 3) {
     tmem_alloc_pair(smem_u32(s_tmem), Cfg::TMEM_COLS);
     tmem_relinquish_pair();
@@ -567,7 +592,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
       // positions] and (pos & 15) [laid out [pair][low bits]: the 32 rows of a warp read one 128-byte
       // line per pair, which stays in L1]
       const float4 *t_hi = reinterpret_cast<const float4 *>(p.rope_hi + static_cast<size_t>(pos >> ROPE_LO_BITS) * HALF);
-      const float2 *t_lo = p.rope_lo + (pos & (ROPE_LO_SIZE - 1));
+      const float2 *t_lo = (LOSM ? static_cast<const float2 *>(s_lo) : p.rope_lo) + (pos & (ROPE_LO_SIZE - 1));
       const uint32_t acc = tmem_base + lane_field + a * BLOCK_N;
       const bool visible = valid && pos <= q_pos && pos >= lo_pos;  // fused: does the query see this row's key
       bool ok = true;
@@ -746,7 +771,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
 #pragma unroll
               for (int j = 0; j < 8; j += 2) {
                 const int i = c * 8 + j;  // pairs i and i + 1
-                const float2 l0 = __ldg(t_lo + i * ROPE_LO_SIZE), l1 = __ldg(t_lo + (i + 1) * ROPE_LO_SIZE);
+                const float2 l0 = LOSM ? t_lo[i * ROPE_LO_SIZE] : __ldg(t_lo + i * ROPE_LO_SIZE), l1 = LOSM ? t_lo[(i + 1) * ROPE_LO_SIZE] : __ldg(t_lo + (i + 1) * ROPE_LO_SIZE);
                 const float4 hh4 = h[j >> 1];
                 const float c0 = fmaf(hh4.x, l0.x, -hh4.y * l0.y), s0 = fmaf(hh4.y, l0.x, hh4.x * l0.y);
                 const float c1 = fmaf(hh4.z, l1.x, -hh4.w * l1.y), s1 = fmaf(hh4.w, l1.x, hh4.z * l1.y);
@@ -790,7 +815,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
 #pragma unroll
               for (int j = 0; j < 16; j += 2) {
                 const int i = c * 16 + j;  // pairs (i, i + HALF) and (i + 1, i + 1 + HALF)
-                const float2 l0 = __ldg(t_lo + i * ROPE_LO_SIZE), l1 = __ldg(t_lo + (i + 1) * ROPE_LO_SIZE);
+                const float2 l0 = LOSM ? t_lo[i * ROPE_LO_SIZE] : __ldg(t_lo + i * ROPE_LO_SIZE), l1 = LOSM ? t_lo[(i + 1) * ROPE_LO_SIZE] : __ldg(t_lo + (i + 1) * ROPE_LO_SIZE);
                 const float4 hh4 = h[j >> 1];
                 const float c0 = fmaf(hh4.x, l0.x, -hh4.y * l0.y), s0 = fmaf(hh4.y, l0.x, hh4.x * l0.y);
                 const float c1 = fmaf(hh4.z, l1.x, -hh4.w * l1.y), s1 = fmaf(hh4.w, l1.x, hh4.z * l1.y);
@@ -877,12 +902,12 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
 }
 
 // ------------------------------------------------------------------------------ host launcher
-template <int BLOCK_N, int D_HEAD, bool TRACE, int FG, int EB = 2>
+template <int BLOCK_N, int D_HEAD, bool TRACE, int FG, int EB = 2, bool LOSM = (FG > 0)>
 static kvd_status launch_impl(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
                               const CUtensorMap &tmap_rows, const RecomputeParams &p, const FusedParams *fp,
                               cudaStream_t stream) {
-  using Cfg = RcCfg<BLOCK_N, D_HEAD, FG>;
-  auto kern = kvd_recompute_kernel<BLOCK_N, D_HEAD, TRACE, FG, EB>;
+  using Cfg = RcCfg<BLOCK_N, D_HEAD, FG, LOSM>;
+  auto kern = kvd_recompute_kernel<BLOCK_N, D_HEAD, TRACE, FG, EB, LOSM>;
   const CUtensorMap &tmap_b = EB == 1 ? ls.tmap_b8 : ls.tmap_b;
   static bool configured[64] = {};
   if (!configured[ctx->device & 63]) {
@@ -923,6 +948,9 @@ static kvd_status launch_sel(kvd_ctx *ctx, const LayerState &ls, const CUtensorM
                              cudaStream_t stream) {
   if constexpr (FG == 0) {
     if (p.trace != nullptr) return launch_impl<BLOCK_N, D_HEAD, true, 0>(ctx, ls, tmap_store, tmap_rows, p, fp, stream);
+    // one tile per cluster at most: every key tile's epilogue is exposed -> the low table from shared memory
+    if (p.num_m_blocks * p.num_n_blocks <= ctx->num_sms / 2)
+      return launch_impl<BLOCK_N, D_HEAD, false, 0, 2, true>(ctx, ls, tmap_store, tmap_rows, p, fp, stream);
   }
   return launch_impl<BLOCK_N, D_HEAD, false, FG>(ctx, ls, tmap_store, tmap_rows, p, fp, stream);
 }
@@ -962,12 +990,12 @@ kvd_status launch_recompute_fp8(kvd_ctx *ctx, const LayerState &ls, const CUtens
                                 const RecomputeParams &p, cudaStream_t stream) {
   const int dh = ctx->desc.d_head;
   if (ctx->block_n == 256) {
-    if (dh == 256) return launch_impl<256, 256, false, 0, 1>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
-    if (dh == 128) return launch_impl<256, 128, false, 0, 1>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
-    if (dh == 64) return launch_impl<256, 64, false, 0, 1>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
+    if (dh == 256) return launch_impl<256, 256, false, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
+    if (dh == 128) return launch_impl<256, 128, false, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
+    if (dh == 64) return launch_impl<256, 64, false, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
   } else if (ctx->block_n == 128) {
-    if (dh == 128) return launch_impl<128, 128, false, 0, 1>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
-    if (dh == 64) return launch_impl<128, 64, false, 0, 1>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
+    if (dh == 128) return launch_impl<128, 128, false, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
+    if (dh == 64) return launch_impl<128, 64, false, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
   }
   return KVD_ERR_SHAPE;
 }
