@@ -844,6 +844,16 @@ extern "C" kvd_status kvd_memory_stats(const kvd_ctx *ctx, kvd_mem_stats *out) {
   }
   out->checkpoint_bytes_used = rows_total * (static_cast<uint64_t>(d.d_hidden) * 2 + 8);  // row, position, sum of squares
   out->checkpoint_bytes_capacity = ctx->layers_stored > 0 ? kvd_store_bytes(&d, ctx->layers_stored) : 0;
+  // the FP8 store counts too: codes, position, sum of squares, scale
+  uint64_t rows8 = 0;
+  for (int l = 0; l < ctx->layers_stored8; ++l) {
+    uint64_t layer_rows = 0;
+    for (int s = 0; s < d.max_seqs; ++s) layer_rows += ctx->rows_stored8[static_cast<size_t>(l) * d.max_seqs + s];
+    rows8 += layer_rows;
+    if (layer_rows > tokens) tokens = layer_rows;
+  }
+  out->checkpoint_bytes_used += rows8 * (static_cast<uint64_t>(d.d_hidden) + 12);
+  out->checkpoint_bytes_capacity += ctx->layers_stored8 > 0 ? kvd_store_bytes_fp8(&d, ctx->layers_stored8) : 0;
   out->workspace_bytes = ctx->workspace_bytes;
   out->prepared_weight_bytes = ctx->prepared_bytes;
   out->tokens_stored = tokens;

@@ -47,6 +47,7 @@ def test_stored_codes_scales_and_statistics_equal_the_oracles_quantisation():
     ctx.kvd_checkpoint_residual_fp8(1, 0, x[11:], p[11:], n - 11)
     torch.cuda.synchronize()
     assert ctx.kvd_rows_stored_fp8(0, 1) == n and ctx.kvd_rows_stored_fp8(0, 0) == 0
+    assert ctx.kvd_memory_stats()["checkpoint_bytes_used"] == n * (shape.d_hidden + 12)
     slots = 2 * max_tokens
     ru = lambda b: (b + 255) // 256 * 256
     c_bytes, f_bytes = ru(slots * shape.d_hidden), ru(slots * 4)
@@ -97,6 +98,29 @@ def test_recompute_from_fp8_checkpoints_follows_the_fp8_oracle(shape, n):
     for name, g, r in (("K", host_f64(k)[:n], Ke.reshape(n, kdim)), ("V", host_f64(v)[:n], Ve.reshape(n, kdim))):
         rel = np.linalg.norm(g - r) / np.linalg.norm(r)
         assert rel < 0.08, (name, rel)
+
+
+def test_fp8_recompute_at_the_bench_size_sampled_against_the_fp8_oracle():
+    """T = 4096 rows of the Gemma-3-4B-shaped layer (the configuration bench.py times), a seeded sample of rows
+    plus the first and last row of every 128-row block class against the FP8 oracle."""
+    shape = GEMMA3_4B_GLOBAL
+    T = 4096
+    ctx, w, arena = open_fp8(shape, T + 8)
+    kdim = shape.n_kv_heads * shape.d_head
+    X = make_residuals(shape, T, seed=34, outliers=True)
+    pos = np.arange(T)
+    x, p = dev(X), torch.from_numpy(pos.astype(np.int32)).cuda()
+    ctx.kvd_checkpoint_residual_fp8(0, 0, x, p, T)
+    k = torch.zeros((T, kdim), dtype=torch.bfloat16, device="cuda")
+    v = torch.zeros_like(k)
+    ctx.kvd_recompute_kv_fp8(0, [(0, 0, T, k, v)], kdim)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    rows = np.unique(np.concatenate([np.random.default_rng(5).choice(T, 512, replace=False),
+                                     [0, 127, 128, 255, 256, 2047, 2048, T - 129, T - 128, T - 1]]))
+    Kr, Vr = oracle_fp8_kv(shape, w, X[rows], pos[rows])
+    for name, g, r in (("K", host_f64(k)[rows], Kr.reshape(len(rows), kdim)), ("V", host_f64(v)[rows], Vr.reshape(len(rows), kdim))):
+        mx, rel = kv_errors(g, r)
+        assert mx <= 2e-2 and rel <= 1e-2, (name, mx, rel)
 
 
 def test_fp8_recompute_bits_do_not_depend_on_the_batch():

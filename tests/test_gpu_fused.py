@@ -113,6 +113,13 @@ def test_fused_matches_the_oracle_and_the_two_call_path(shape, n_old, n_live):
     attn_check(f, two, "fused vs two-call")
 
 
+def test_fused_at_the_bench_size():
+    # the configuration bench.py times: 4096 evicted rows + the current token, Gemma-3-4B-shaped global layer
+    f, two, ref = run_case(GEMMA3_4B_GLOBAL, [4096], 0, max_tokens=4104, seed=8)
+    attn_check(f, ref, "fused vs oracle")
+    attn_check(f, two, "fused vs two-call")
+
+
 def test_fused_batch_with_ragged_ranges_and_an_empty_one():
     f, two, ref = run_case(GEMMA3_4B_GLOBAL, [300, 0, 513, 40], 16, pos0_list=[0, 5, 11, 1000], seed=7)
     attn_check(f, ref, "fused vs oracle")
