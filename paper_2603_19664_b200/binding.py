@@ -31,7 +31,7 @@ KVD_MAX_SEGMENTS = 4
 # every symbol include/kvd.h declares
 EXPORTED_SYMBOLS = (
     "kvd_create", "kvd_destroy", "kvd_set_layer", "kvd_store_bytes", "kvd_attach_store", "kvd_reset_sequence",
-    "kvd_decode_attention_recompute",
+    "kvd_decode_attention_recompute", "kvd_set_dtype",
     "kvd_store_bytes_fp8", "kvd_attach_store_fp8", "kvd_rows_stored_fp8", "kvd_reset_sequence_fp8", "kvd_checkpoint_residual_fp8", "kvd_recompute_kv_fp8",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
     "kvd_recompute_kv_step",
@@ -121,6 +121,8 @@ def load() -> ctypes.CDLL:
     lib.kvd_decode_attention.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
                                          ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
     lib.kvd_decode_attention.restype = i32
+    lib.kvd_set_dtype.argtypes = [vp, i32]
+    lib.kvd_set_dtype.restype = i32
     lib.kvd_store_bytes_fp8.argtypes = [ctypes.POINTER(kvd_model_desc), i32]
     lib.kvd_store_bytes_fp8.restype = sz
     lib.kvd_attach_store_fp8.argtypes = [vp, vp, sz, i32]
@@ -343,6 +345,10 @@ class Kvd:
             self._h, layer, batch, _ptr(q), pos_arr, arr, _ptr(rows), _ptr(positions), n_rows, _ptr(k_rows_out),
             _ptr(v_rows_out), out_row_stride, seg_arr, n_segs, float(scale), _ptr(out), _stream(stream)),
             "kvd_decode_attention_recompute")
+
+    def kvd_set_dtype(self, dtype: int) -> None:
+        """0 = bf16 (default), 1 = fp16 (checkpoint / recompute entry points only); before any kvd_set_layer."""
+        self._check(self._lib.kvd_set_dtype(self._h, dtype), "kvd_set_dtype")
 
     def kvd_attach_store_fp8(self, arena, layers_stored: int) -> None:
         self._keep.append(arena)

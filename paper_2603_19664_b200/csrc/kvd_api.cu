@@ -244,6 +244,16 @@ static kvd_status get_rope(kvd_ctx *ctx, float theta, RopeTable *out) {
   return KVD_OK;
 }
 
+extern "C" kvd_status kvd_set_dtype(kvd_ctx *ctx, int dtype) {
+  if (!ctx || (dtype != KVD_DTYPE_BF16 && dtype != KVD_DTYPE_F16)) return KVD_ERR_INVALID_ARG;
+  for (const LayerState &l : ctx->layers)
+    if (l.set) return KVD_ERR_STATE;  // weights are prepared in the element type: choose it first
+  for (int c : ctx->rows_stored)
+    if (c != 0) return KVD_ERR_STATE;
+  ctx->dtype = dtype;
+  return KVD_OK;
+}
+
 extern "C" kvd_status kvd_set_layer(kvd_ctx *ctx, int layer, const kvd_layer_desc *ld, void *stream_) {
   if (!ctx || !ld) return KVD_ERR_INVALID_ARG;
   if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
@@ -279,7 +289,7 @@ extern "C" kvd_status kvd_set_layer(kvd_ctx *ctx, int layer, const kvd_layer_des
   st = encode_2d(ctx, &ls.tmap_b, ls.wt, d.d_hidden, n_cols, RC_BLOCK_K, ctx->block_n / 2);  // half tile per CTA
   if (st != KVD_OK) return st;
   // the FP8 variant's copy of W' (E4M3 codes and one scale); rows of d_hidden bytes must be TMA-addressable
-  if (d.d_hidden % 16 == 0) {
+  if (d.d_hidden % 16 == 0 && ctx->dtype == KVD_DTYPE_BF16) {
     if (!ls.wt8) {
       e = cudaMalloc(&ls.wt8, static_cast<size_t>(n_cols) * d.d_hidden);
       if (e == cudaSuccess) e = cudaMalloc(&ls.w_scale8, sizeof(float));
@@ -544,6 +554,7 @@ extern "C" kvd_status kvd_checkpoint_residual_fp8(kvd_ctx *ctx, int seq, int lay
                                                   const int32_t *positions, int n, void *stream_) {
   if (!ctx || n < 0) return KVD_ERR_INVALID_ARG;
   if (!ctx->store8_codes) return KVD_ERR_STATE;
+  if (ctx->dtype != KVD_DTYPE_BF16) return KVD_ERR_UNSUPPORTED;  // the quantiser reads bf16 rows
   if (seq < 0 || seq >= ctx->desc.max_seqs || layer < 0 || layer >= ctx->layers_stored8) return KVD_ERR_INVALID_ARG;
   if (n == 0) return KVD_OK;
   if (!rows || !positions) return KVD_ERR_INVALID_ARG;
@@ -761,6 +772,7 @@ extern "C" kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, c
   const LayerState &ls = ctx->layers[layer];
   if (!ls.set) return KVD_ERR_STATE;
   if (!ctx->part_o) return KVD_ERR_STATE;
+  if (ctx->dtype != KVD_DTYPE_BF16) return KVD_ERR_UNSUPPORTED;  // attention reads bf16 K/V
   if (batch == 0) return KVD_OK;
   if (!q || !q_pos || !out || (n_segs > 0 && !segs)) return KVD_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(out)) return KVD_ERR_ALIGNMENT;
@@ -795,6 +807,7 @@ extern "C" kvd_status kvd_decode_attention_recompute(kvd_ctx *ctx, int layer, in
   const LayerState &ls = ctx->layers[layer];
   if (!ls.set) return KVD_ERR_STATE;
   if (!ctx->part_o || !ctx->store_rows) return KVD_ERR_STATE;
+  if (ctx->dtype != KVD_DTYPE_BF16) return KVD_ERR_UNSUPPORTED;
   const kvd_model_desc &d = ctx->desc;
   const int group = d.n_q_heads / d.n_kv_heads, kdim = d.n_kv_heads * d.d_head;
   // shapes the fused kernel is built for (nothing is launched otherwise)

@@ -205,6 +205,7 @@ struct kvd_ctx {
   int device = 0;
   int num_sms = 0;
   int block_n = 0;
+  int dtype = 0;  // 16-bit element type of rows, weights and K/V: 0 bf16, 1 fp16 (recompute path only)
   std::vector<kvd::LayerState> layers;
   std::map<uint32_t, kvd::RopeTable> rope_cache;  // keyed by the bits of theta
   // residual store

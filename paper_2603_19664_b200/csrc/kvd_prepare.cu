@@ -6,11 +6,24 @@
 
 namespace kvd {
 
+// a 16-bit element (bf16 or fp16 bits) as float, and back (round to nearest even)
+template <int DT>
+__device__ __forceinline__ float elem_to_float(uint16_t bits) {
+  if constexpr (DT == 0) return __uint_as_float(static_cast<uint32_t>(bits) << 16);
+  else return __half2float(__ushort_as_half(bits));
+}
+template <int DT>
+__device__ __forceinline__ uint16_t float_to_elem(float v) {
+  if constexpr (DT == 0) return __bfloat16_as_ushort(__float2bfloat16_rn(v));
+  else return __half_as_ushort(__float2half_rn(v));
+}
+
 // wt[n][k] = bf16( gamma[k] * w[k][n] ): fold the RMSNorm scale of Eq. 1 into the projection of
 // Eq. 13-14 and store the result K-major so that both GEMM operands are read along d_hidden.
-__global__ void __launch_bounds__(256) kvd_prepare_weights_kernel(const __nv_bfloat16 *__restrict__ w,
-                                                                  const __nv_bfloat16 *__restrict__ gamma,
-                                                                  __nv_bfloat16 *__restrict__ wt, int d_hidden,
+template <int DT>
+__global__ void __launch_bounds__(256) kvd_prepare_weights_kernel(const uint16_t *__restrict__ w,
+                                                                  const uint16_t *__restrict__ gamma,
+                                                                  uint16_t *__restrict__ wt, int d_hidden,
                                                                   int n_cols) {
   __shared__ float tile[32][33];
   const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
@@ -19,24 +32,26 @@ __global__ void __launch_bounds__(256) kvd_prepare_weights_kernel(const __nv_bfl
     const int k = k0 + r, n = n0 + tx;
     float v = 0.f;
     if (k < d_hidden && n < n_cols)
-      v = __bfloat162float(gamma[k]) * __bfloat162float(w[static_cast<size_t>(k) * n_cols + n]);
+      v = elem_to_float<DT>(gamma[k]) * elem_to_float<DT>(w[static_cast<size_t>(k) * n_cols + n]);
     tile[r][tx] = v;
   }
   __syncthreads();
   for (int r = ty; r < 32; r += 8) {
     const int n = n0 + r, k = k0 + tx;
-    if (k < d_hidden && n < n_cols) wt[static_cast<size_t>(n) * d_hidden + k] = __float2bfloat16_rn(tile[tx][r]);
+    if (k < d_hidden && n < n_cols) wt[static_cast<size_t>(n) * d_hidden + k] = float_to_elem<DT>(tile[tx][r]);
   }
 }
 
-__global__ void kvd_convert_gamma_kernel(const __nv_bfloat16 *__restrict__ g, float *__restrict__ out, int n) {
+template <int DT>
+__global__ void kvd_convert_gamma_kernel(const uint16_t *__restrict__ g, float *__restrict__ out, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) out[i] = __bfloat162float(g[i]);
+  if (i < n) out[i] = elem_to_float<DT>(g[i]);
 }
 
 // Copy n rows of d_hidden bf16 and their positions into the store, one warp per row; the warp also
 // takes the row's sum of squares (the RMSNorm statistic of Eq. 2), which the recompute kernel reads
 // back instead of taking it again for every recomputation.
+template <int DT>
 __global__ void __launch_bounds__(256) kvd_checkpoint_kernel(const uint4 *__restrict__ rows,
                                                              const int32_t *__restrict__ pos,
                                                              uint4 *__restrict__ dst_rows, int32_t *__restrict__ dst_pos,
@@ -49,7 +64,7 @@ __global__ void __launch_bounds__(256) kvd_checkpoint_kernel(const uint4 *__rest
     const uint4 *const src[1] = {rows + off};
     uint4 *const dst[1] = {dst_rows + off};
     float ss[1];
-    warp_rows_sumsq<1, 10, true>(src, dst, row_chunks, lane, ss);  // all of a 2560-wide row in flight at once
+    warp_rows_sumsq<1, 10, true, DT>(src, dst, row_chunks, lane, ss);  // all of a 2560-wide row in flight at once
     if (lane == 0) {
       dst_sumsq[r] = ss[0];
       dst_pos[r] = pos[r];
@@ -60,6 +75,7 @@ __global__ void __launch_bounds__(256) kvd_checkpoint_kernel(const uint4 *__rest
 // Sums of squares of n caller rows (no copy), two rows per warp and pass: what kvd_recompute_kv takes
 // ahead of the main kernel when the caller hands it more rows than that kernel's statistics warps
 // can cover under the main loop.
+template <int DT>
 __global__ void __launch_bounds__(256) kvd_rowstats_kernel(const uint4 *__restrict__ rows, float *__restrict__ sumsq,
                                                            int row_chunks, int n) {
   const int lane = threadIdx.x & 31;
@@ -70,7 +86,7 @@ __global__ void __launch_bounds__(256) kvd_rowstats_kernel(const uint4 *__restri
     const uint4 *const src[2] = {rows + static_cast<size_t>(r) * row_chunks, rows + static_cast<size_t>(r1) * row_chunks};
     uint4 *const none[2] = {nullptr, nullptr};
     float ss[2];
-    warp_rows_sumsq<2, 8, false>(src, none, row_chunks, lane, ss);
+    warp_rows_sumsq<2, 8, false, DT>(src, none, row_chunks, lane, ss);
     if (lane == 0) {
       sumsq[r] = ss[0];
       sumsq[r1] = ss[1];
@@ -233,7 +249,10 @@ kvd_status launch_selftest_timeout(kvd_ctx *ctx, unsigned long long timeout_ns, 
 kvd_status launch_prepare_weights(kvd_ctx *ctx, const __nv_bfloat16 *w, const __nv_bfloat16 *gamma, __nv_bfloat16 *wt,
                                   int d_hidden, int n_cols, cudaStream_t stream) {
   dim3 grid((n_cols + 31) / 32, (d_hidden + 31) / 32);
-  kvd_prepare_weights_kernel<<<grid, 256, 0, stream>>>(w, gamma, wt, d_hidden, n_cols);
+  const uint16_t *w16 = reinterpret_cast<const uint16_t *>(w), *g16 = reinterpret_cast<const uint16_t *>(gamma);
+  uint16_t *wt16 = reinterpret_cast<uint16_t *>(wt);
+  if (ctx->dtype == 1) kvd_prepare_weights_kernel<1><<<grid, 256, 0, stream>>>(w16, g16, wt16, d_hidden, n_cols);
+  else kvd_prepare_weights_kernel<0><<<grid, 256, 0, stream>>>(w16, g16, wt16, d_hidden, n_cols);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "launch prepare_weights");
   ctx->launches += 1;
@@ -241,7 +260,9 @@ kvd_status launch_prepare_weights(kvd_ctx *ctx, const __nv_bfloat16 *w, const __
 }
 
 kvd_status launch_convert_gamma(kvd_ctx *ctx, const __nv_bfloat16 *g, float *out, int n, cudaStream_t stream) {
-  kvd_convert_gamma_kernel<<<(n + 127) / 128, 128, 0, stream>>>(g, out, n);
+  const uint16_t *g16 = reinterpret_cast<const uint16_t *>(g);
+  if (ctx->dtype == 1) kvd_convert_gamma_kernel<1><<<(n + 127) / 128, 128, 0, stream>>>(g16, out, n);
+  else kvd_convert_gamma_kernel<0><<<(n + 127) / 128, 128, 0, stream>>>(g16, out, n);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "launch convert_gamma");
   ctx->launches += 1;
@@ -254,8 +275,12 @@ kvd_status launch_checkpoint(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int3
   const long long cap = static_cast<long long>(ctx->num_sms) * 8;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  kvd_checkpoint_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
-      reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint4 *>(dst_rows), dst_pos, dst_sumsq, d_hidden / 8, n);
+  if (ctx->dtype == 1)
+    kvd_checkpoint_kernel<1><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+        reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint4 *>(dst_rows), dst_pos, dst_sumsq, d_hidden / 8, n);
+  else
+    kvd_checkpoint_kernel<0><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+        reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint4 *>(dst_rows), dst_pos, dst_sumsq, d_hidden / 8, n);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "launch checkpoint");
   ctx->launches += 1;
@@ -268,8 +293,12 @@ kvd_status launch_rowstats(kvd_ctx *ctx, const __nv_bfloat16 *rows, float *sumsq
   const long long cap = static_cast<long long>(ctx->num_sms) * 8;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  kvd_rowstats_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(reinterpret_cast<const uint4 *>(rows), sumsq,
-                                                                         d_hidden / 8, n);
+  if (ctx->dtype == 1)
+    kvd_rowstats_kernel<1><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(reinterpret_cast<const uint4 *>(rows), sumsq,
+                                                                              d_hidden / 8, n);
+  else
+    kvd_rowstats_kernel<0><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(reinterpret_cast<const uint4 *>(rows), sumsq,
+                                                                              d_hidden / 8, n);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "launch rowstats");
   ctx->launches += 1;

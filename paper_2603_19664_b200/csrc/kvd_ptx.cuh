@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 
 namespace kvd {
@@ -279,6 +280,10 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(int m, int n) {
          (static_cast<uint32_t>(m >> 4) << 24);
 }
 
+// kind::f16 with fp16 A and B (format code 0 in both fields).
+__host__ __device__ constexpr uint32_t umma_idesc_f16_f32(int m, int n) {
+  return (1u << 4) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
+}
 // The same for kind::f8f6f4 with E4M3 A and B (format code 0 in both fields).
 __host__ __device__ constexpr uint32_t umma_idesc_e4m3_f32(int m, int n) {
   return (1u << 4) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
@@ -315,6 +320,27 @@ __device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
 // the two bf16 halves of a 32-bit word as a packed pair of fp32
 __device__ __forceinline__ uint64_t bf16x2_to_f32x2(uint32_t w) { return pack2(bf16_lo(w), bf16_hi(w)); }
 
+// 16-bit element type of rows, weights and outputs: DT = 0 bf16 (the default everywhere), DT = 1 fp16 (the
+// recompute path only: the dtype-invariance check of the paper's Section 5.1)
+template <int DT>
+__device__ __forceinline__ uint64_t x2_to_f32x2(uint32_t w) {
+  if constexpr (DT == 0) {
+    return bf16x2_to_f32x2(w);
+  } else {
+    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w));
+    return pack2(f.x, f.y);
+  }
+}
+template <int DT>
+__device__ __forceinline__ uint32_t pack_out(float lo, float hi) {
+  if constexpr (DT == 0) {
+    return pack_bf16(lo, hi);
+  } else {
+    const __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&v);
+  }
+}
+
 // ------------------------------------------------------------------------------ row statistic (Eq. 2)
 // Sum of squares of one row of bf16 values (n_chunks 16-byte chunks), taken by a whole warp: lane l
 // squares chunks l, l + 32, ... in ascending order into eight partial sums (one per element slot of
@@ -322,12 +348,13 @@ __device__ __forceinline__ uint64_t bf16x2_to_f32x2(uint32_t w) { return pack2(b
 // by an xor butterfly (16, 8, 4, 2, 1), so every lane returns the same bits.  With COPY the chunks
 // are also written to `dst`.  (FMAs and adds are explicit: the compiler cannot re-associate them.)  The checkpoint kernel and the recompute kernel both take the statistic
 // with this one function: its bits do not depend on which of them saw the row.
+template <int DT = 0>
 __device__ __forceinline__ void sumsq_chunk(uint64_t (&ps2)[4], const uint4 &v) {
   uint64_t x2;
-  x2 = bf16x2_to_f32x2(v.x); ps2[0] = ffma2(x2, x2, ps2[0]);
-  x2 = bf16x2_to_f32x2(v.y); ps2[1] = ffma2(x2, x2, ps2[1]);
-  x2 = bf16x2_to_f32x2(v.z); ps2[2] = ffma2(x2, x2, ps2[2]);
-  x2 = bf16x2_to_f32x2(v.w); ps2[3] = ffma2(x2, x2, ps2[3]);
+  x2 = x2_to_f32x2<DT>(v.x); ps2[0] = ffma2(x2, x2, ps2[0]);
+  x2 = x2_to_f32x2<DT>(v.y); ps2[1] = ffma2(x2, x2, ps2[1]);
+  x2 = x2_to_f32x2<DT>(v.z); ps2[2] = ffma2(x2, x2, ps2[2]);
+  x2 = x2_to_f32x2<DT>(v.w); ps2[3] = ffma2(x2, x2, ps2[3]);
 }
 // the eight partial sums of a lane in a fixed tree, then the xor butterfly over the warp
 __device__ __forceinline__ float sumsq_finish(const uint64_t (&ps2)[4]) {
@@ -339,7 +366,7 @@ __device__ __forceinline__ float sumsq_finish(const uint64_t (&ps2)[4]) {
   for (int k = 16; k >= 1; k >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, k);
   return sum;
 }
-template <int R, int B, bool COPY>
+template <int R, int B, bool COPY, int DT = 0>
 __device__ __forceinline__ void warp_rows_sumsq(const uint4 *const (&src)[R], uint4 *const (&dst)[R], int n_chunks, int lane,
                                                 float (&out)[R]) {
   // R rows side by side, B loads per row in flight per lane; each row's arithmetic is the sequence
@@ -361,7 +388,7 @@ __device__ __forceinline__ void warp_rows_sumsq(const uint4 *const (&src)[R], ui
 #pragma unroll
       for (int j = 0; j < B; ++j) {
         if (COPY) dst[r][c + 32 * j] = v[r][j];
-        sumsq_chunk(ps2[r], v[r][j]);
+        sumsq_chunk<DT>(ps2[r], v[r][j]);
       }
   }
   for (; c < n_chunks; c += 32) {
@@ -371,7 +398,7 @@ __device__ __forceinline__ void warp_rows_sumsq(const uint4 *const (&src)[R], ui
 #pragma unroll
     for (int r = 0; r < R; ++r) {
       if (COPY) dst[r][c] = v[r];
-      sumsq_chunk(ps2[r], v[r]);
+      sumsq_chunk<DT>(ps2[r], v[r]);
     }
   }
 #pragma unroll

@@ -201,7 +201,8 @@ __device__ __forceinline__ void store_row_piece(__nv_bfloat16 *dst, const uint32
 // EB = bytes per operand element: 2 = bf16 rows and weights, 1 = the FP8 variant (E4M3 codes of rows and
 // weights; a k block is then 128 channels in the same 128-byte rows, the MMA kind f8f6f4, and the rows'
 // and the matrix's quantisation scales ride in the per-row factor that the statistics warps hand over).
-template <int BLOCK_N, int D_HEAD, bool TRACE, int FG, int EB = 2, bool LOSM = (FG > 0)>
+// DT = 1: fp16 rows, weights and outputs instead of bf16 (plain variant only).
+template <int BLOCK_N, int D_HEAD, bool TRACE, int FG, int EB = 2, bool LOSM = (FG > 0), int DT = 0>
 __global__ void __launch_bounds__(RC_THREADS, 1)
 kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __grid_constant__ CUtensorMap tmap_rows,
                      const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ RecomputeParams p,
@@ -210,6 +211,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   constexpr int STAGES = Cfg::STAGES;
   constexpr bool FUSED = FG > 0;
   static_assert(EB == 2 || (EB == 1 && FG == 0), "the fused variant exists for bf16 operands only");
+  static_assert(DT == 0 || (FG == 0 && EB == 2), "fp16 exists for the plain variant only");
   constexpr int KB_ELEMS = RC_BLOCK_K * 2 / EB;  // channels per k block
   static_assert(BLOCK_N % D_HEAD == 0, "a tile must hold whole heads");
 
@@ -415,7 +417,9 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   } else if (warp == 3) {
     if (lane == 0 && cta_rank == 0) {
       // ---------------------------------------------------------------- MMA issuer (even CTA)
-      constexpr uint32_t idesc = EB == 2 ? umma_idesc_bf16_f32(2 * RC_BLOCK_M, BLOCK_N) : umma_idesc_e4m3_f32(2 * RC_BLOCK_M, BLOCK_N);
+      constexpr uint32_t idesc = EB == 1   ? umma_idesc_e4m3_f32(2 * RC_BLOCK_M, BLOCK_N)
+                                 : DT == 1 ? umma_idesc_f16_f32(2 * RC_BLOCK_M, BLOCK_N)
+                                           : umma_idesc_bf16_f32(2 * RC_BLOCK_M, BLOCK_N);
       // descriptor words for 128-byte-swizzled K-major tiles: low = start address >> 4 | LBO field (1),
       // high = SBO (1024 B >> 4) | version 1 (bit 46) | swizzle mode 2 (bits 61-63)
       constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
@@ -517,7 +521,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
 #pragma unroll
             for (int i = 0; i < 4; ++i) src[i] = base + static_cast<size_t>(4 * g + i < n_here ? 4 * g + i : n_here - 1) * p.row_chunks;
             float ss[4];
-            warp_rows_sumsq<4, 4, false>(src, none, p.row_chunks, lane, ss);
+            warp_rows_sumsq<4, 4, false, DT>(src, none, p.row_chunks, lane, ss);
             const float mine = lane == 0 ? ss[0] : lane == 1 ? ss[1] : lane == 2 ? ss[2] : ss[3];
             if (lane < 4 && 4 * g + lane < n_here)
               s_rstd[a * RC_BLOCK_M + 4 * g + lane] = 1.0f / sqrtf(mine * p.inv_d_hidden + p.rms_eps);
@@ -713,7 +717,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
             uint32_t o[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-              o[j] = pack_bf16(__uint_as_float(r[2 * j]) * rstd, __uint_as_float(r[2 * j + 1]) * rstd);
+              o[j] = pack_out<DT>(__uint_as_float(r[2 * j]) * rstd, __uint_as_float(r[2 * j + 1]) * rstd);
             if (valid) store_row_piece<4>(dst + c * 32, o, wide);
           }
         } else {
@@ -779,8 +783,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
                 const float b0 = __uint_as_float(r[2 * j + 1]) * kscale * s_gamma_k[c * 16 + 2 * j + 1];
                 const float a1 = __uint_as_float(r[2 * j + 2]) * kscale * s_gamma_k[c * 16 + 2 * j + 2];
                 const float b1 = __uint_as_float(r[2 * j + 3]) * kscale * s_gamma_k[c * 16 + 2 * j + 3];
-                o[j] = pack_bf16(fmaf(a0, c0, -b0 * s0), fmaf(a0, s0, b0 * c0));
-                o[j + 1] = pack_bf16(fmaf(a1, c1, -b1 * s1), fmaf(a1, s1, b1 * c1));
+                o[j] = pack_out<DT>(fmaf(a0, c0, -b0 * s0), fmaf(a0, s0, b0 * c0));
+                o[j + 1] = pack_out<DT>(fmaf(a1, c1, -b1 * s1), fmaf(a1, s1, b1 * c1));
               }
               if (FUSED && attend) {
 #pragma unroll
@@ -823,8 +827,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
                 const float b0 = __uint_as_float(rb[j]) * kscale * s_gamma_k[i + HALF];
                 const float a1 = __uint_as_float(ra[j + 1]) * kscale * s_gamma_k[i + 1];
                 const float b1 = __uint_as_float(rb[j + 1]) * kscale * s_gamma_k[i + 1 + HALF];
-                oa[j >> 1] = pack_bf16(fmaf(a0, c0, -b0 * s0), fmaf(a1, c1, -b1 * s1));
-                ob[j >> 1] = pack_bf16(fmaf(a0, s0, b0 * c0), fmaf(a1, s1, b1 * c1));
+                oa[j >> 1] = pack_out<DT>(fmaf(a0, c0, -b0 * s0), fmaf(a1, c1, -b1 * s1));
+                ob[j >> 1] = pack_out<DT>(fmaf(a0, s0, b0 * c0), fmaf(a1, s1, b1 * c1));
               }
               if (FUSED && attend) {
 #pragma unroll
@@ -902,12 +906,12 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
 }
 
 // ------------------------------------------------------------------------------ host launcher
-template <int BLOCK_N, int D_HEAD, bool TRACE, int FG, int EB = 2, bool LOSM = (FG > 0)>
+template <int BLOCK_N, int D_HEAD, bool TRACE, int FG, int EB = 2, bool LOSM = (FG > 0), int DT = 0>
 static kvd_status launch_impl(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
                               const CUtensorMap &tmap_rows, const RecomputeParams &p, const FusedParams *fp,
                               cudaStream_t stream) {
   using Cfg = RcCfg<BLOCK_N, D_HEAD, FG, LOSM>;
-  auto kern = kvd_recompute_kernel<BLOCK_N, D_HEAD, TRACE, FG, EB, LOSM>;
+  auto kern = kvd_recompute_kernel<BLOCK_N, D_HEAD, TRACE, FG, EB, LOSM, DT>;
   const CUtensorMap &tmap_b = EB == 1 ? ls.tmap_b8 : ls.tmap_b;
   static bool configured[64] = {};
   if (!configured[ctx->device & 63]) {
@@ -947,6 +951,8 @@ static kvd_status launch_sel(kvd_ctx *ctx, const LayerState &ls, const CUtensorM
                              const CUtensorMap &tmap_rows, const RecomputeParams &p, const FusedParams *fp,
                              cudaStream_t stream) {
   if constexpr (FG == 0) {
+    // fp16 contexts: one variant (low table in shared memory) for all launch sizes
+    if (ctx->dtype == 1) return launch_impl<BLOCK_N, D_HEAD, false, 0, 2, true, 1>(ctx, ls, tmap_store, tmap_rows, p, fp, stream);
     if (p.trace != nullptr) return launch_impl<BLOCK_N, D_HEAD, true, 0>(ctx, ls, tmap_store, tmap_rows, p, fp, stream);
     // one tile per cluster at most: every key tile's epilogue is exposed -> the low table from shared memory
     if (p.num_m_blocks * p.num_n_blocks <= ctx->num_sms / 2)
