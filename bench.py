@@ -336,6 +336,26 @@ class Workload:
                                                 K[T:], V[T:], self.kdim, [[(K[T:], V[T:], self.kdim, T, 1)]], 0.0,
                                                 self.out[s:s + 1])
 
+    def append_current_fp8(self):
+        # the current token joins the FP8 store of every set (row T), once, outside any timed region
+        for s in range(self.n_sets):
+            if self.ctx.kvd_rows_stored_fp8(0, s) == self.T:
+                self.ctx.kvd_checkpoint_residual_fp8(s, 0, self.X[s][self.T:], self.pos[self.T:], 1)
+
+    def k_two_call_fp8(self, i):
+        # nothing kept: K/V of all T + 1 tokens rebuilt from their FP8 checkpoints, then attention over them
+        s, T = i % self.n_sets, self.T
+        K, V = self.K[s], self.V[s]
+        self.ctx.kvd_recompute_kv_fp8(0, [(s, 0, T + 1, K, V)], self.kdim)
+        self.ctx.kvd_decode_attention(0, 1, self.q[s:s + 1], [T], [[(K, V, self.kdim, 0, T + 1)]], 0.0,
+                                      self.out[s:s + 1])
+
+    def k_fused_fp8(self, i):
+        # the same with the rebuilt K/V consumed inside the recompute kernel: kvd_decode_attention_recompute_fp8
+        s, T = i % self.n_sets, self.T
+        self.ctx.kvd_decode_attention_recompute_fp8(0, 1, self.q[s:s + 1], [T], [(s, 0, T + 1)], [], self.kdim, [[]],
+                                                    0.0, self.out[s:s + 1])
+
     def cached_read_step(self, i):
         """What KV-Direct replaces: attention over the stored cache of T + 1 keys in one segment."""
         s, T = i % self.n_sets, self.T
@@ -485,6 +505,9 @@ def run_gpu(args):
               "recompute_from_fp8_checkpoints": timed_graph(wl.k_recompute_fp8, 10),
               "recompute_then_attention_two_calls": timed_graph(wl.k_two_call, 10),
               "recompute_fused_into_attention": timed_graph(wl.k_fused, 10)}
+    wl.append_current_fp8()
+    iso_ms["recompute_fp8_then_attention_two_calls"] = timed_graph(wl.k_two_call_fp8, 10)
+    iso_ms["recompute_fp8_fused_into_attention"] = timed_graph(wl.k_fused_fp8, 10)
     read_attn_ms = timed_graph(wl.cached_read_step, 10)
     kv_copy_dst = torch.empty((2, T + 1, wl.kdim), dtype=torch.bfloat16, device="cuda")
 

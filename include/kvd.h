@@ -299,6 +299,20 @@ kvd_status kvd_decode_attention_recompute(kvd_ctx *ctx, int layer, int batch, co
                                           int64_t out_row_stride, const kvd_kv_segment *segs, int n_segs,
                                           float scale, void *out, void *stream);
 
+/* The same with the evicted tokens taken from the FP8 store (kvd_checkpoint_residual_fp8): ranges[b] (HOST
+ * [batch], rows of the FP8 store of (layer, ranges[b].seq); k_out / v_out ignored) are rebuilt with E4M3
+ * operands and attended inside the recompute kernel.  There are no caller rows here: the new tokens are
+ * quantised into the FP8 store first and either belong to ranges[b] (nothing is kept: a cache budget of
+ * zero) or are listed in store_ranges (HOST [n_store_ranges], batch + n_store_ranges <=
+ * KVD_MAX_STORE_RANGES), whose K and V ARE written to their k_out / v_out (row stride out_row_stride) for
+ * the live segments to point at.  Result: attention over [keys of ranges[b]] united with segs[b][*], with
+ * the tolerance and the definition of kvd_recompute_kv_fp8.  Shapes and attachments as above, the FP8
+ * store in place of the bf16 one. */
+kvd_status kvd_decode_attention_recompute_fp8(kvd_ctx *ctx, int layer, int batch, const void *q, const int32_t *q_pos,
+                                              const kvd_store_range *ranges, const kvd_store_range *store_ranges,
+                                              int n_store_ranges, int64_t out_row_stride, const kvd_kv_segment *segs,
+                                              int n_segs, float scale, void *out, void *stream);
+
 /* No counterpart in the paper: the same decode attention as kvd_decode_attention for callers that
  * cannot allocate device memory at all -- code running inside someone else's memory pool or under a
  * fixed memory budget, a plug-in whose host forbids cudaMalloc after start-up, a process that must

@@ -31,7 +31,7 @@ KVD_MAX_SEGMENTS = 4
 # every symbol include/kvd.h declares
 EXPORTED_SYMBOLS = (
     "kvd_create", "kvd_destroy", "kvd_set_layer", "kvd_store_bytes", "kvd_attach_store", "kvd_reset_sequence",
-    "kvd_decode_attention_recompute", "kvd_set_dtype",
+    "kvd_decode_attention_recompute", "kvd_decode_attention_recompute_fp8", "kvd_set_dtype",
     "kvd_store_bytes_fp8", "kvd_attach_store_fp8", "kvd_rows_stored_fp8", "kvd_reset_sequence_fp8", "kvd_checkpoint_residual_fp8", "kvd_recompute_kv_fp8",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
     "kvd_recompute_kv_step",
@@ -139,6 +139,11 @@ def load() -> ctypes.CDLL:
                                                    ctypes.POINTER(kvd_store_range), vp, vp, i32, vp, vp, i64,
                                                    ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
     lib.kvd_decode_attention_recompute.restype = i32
+    lib.kvd_decode_attention_recompute_fp8.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
+                                                       ctypes.POINTER(kvd_store_range), ctypes.POINTER(kvd_store_range),
+                                                       i32, i64, ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float,
+                                                       vp, vp]
+    lib.kvd_decode_attention_recompute_fp8.restype = i32
     lib.kvd_decode_attention_static.argtypes = [i32, i32, i32, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
                                                 ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
     lib.kvd_decode_attention_static.restype = i32
@@ -345,6 +350,26 @@ class Kvd:
             self._h, layer, batch, _ptr(q), pos_arr, arr, _ptr(rows), _ptr(positions), n_rows, _ptr(k_rows_out),
             _ptr(v_rows_out), out_row_stride, seg_arr, n_segs, float(scale), _ptr(out), _stream(stream)),
             "kvd_decode_attention_recompute")
+
+    def kvd_decode_attention_recompute_fp8(self, layer: int, batch: int, q, q_pos: Sequence[int],
+                                           ranges: Sequence[Tuple[int, int, int]],
+                                           store_ranges: Sequence[Tuple[int, int, int, object, object]],
+                                           out_row_stride: int, segs: Sequence[Sequence[Segment]], scale: float, out,
+                                           stream=None) -> None:
+        """ranges: (seq, first_row, n) of the FP8 store per sequence -- attended inside the recompute kernel;
+        store_ranges: (seq, first_row, n, k_out, v_out) of the FP8 store whose K/V are written."""
+        n_segs, pos_arr, seg_arr = _marshal_segments(batch, q_pos, segs)
+        arr = (kvd_store_range * max(len(ranges), 1))()
+        for i, (seq, first_row, n) in enumerate(ranges):
+            arr[i].seq, arr[i].first_row, arr[i].n, arr[i].reserved = int(seq), int(first_row), int(n), 0
+            arr[i].k_out, arr[i].v_out = None, None
+        sarr = (kvd_store_range * max(len(store_ranges), 1))()
+        for i, (seq, first_row, n, k_out, v_out) in enumerate(store_ranges):
+            sarr[i].seq, sarr[i].first_row, sarr[i].n, sarr[i].reserved = int(seq), int(first_row), int(n), 0
+            sarr[i].k_out, sarr[i].v_out = _ptr(k_out), _ptr(v_out)
+        self._check(self._lib.kvd_decode_attention_recompute_fp8(
+            self._h, layer, batch, _ptr(q), pos_arr, arr, sarr, len(store_ranges), out_row_stride, seg_arr, n_segs,
+            float(scale), _ptr(out), _stream(stream)), "kvd_decode_attention_recompute_fp8")
 
     def kvd_set_dtype(self, dtype: int) -> None:
         """0 = bf16 (default), 1 = fp16 (checkpoint / recompute entry points only); before any kvd_set_layer."""

@@ -570,10 +570,12 @@ extern "C" kvd_status kvd_checkpoint_residual_fp8(kvd_ctx *ctx, int seq, int lay
   return st;
 }
 
-extern "C" kvd_status kvd_recompute_kv_fp8(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
-                                           int64_t out_row_stride, void *stream_) {
-  if (!ctx || n_ranges < 0 || n_ranges > KVD_MAX_STORE_RANGES || (n_ranges > 0 && !ranges)) return KVD_ERR_INVALID_ARG;
-  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+// Shared body of kvd_recompute_kv_fp8 and kvd_decode_attention_recompute_fp8: validate, build the
+// job table from ranges of the FP8 store, launch once.  With `fused` (one RcAttend per range, q ==
+// nullptr for a range whose K/V are written) the ranges that carry a query are attended in the kernel.
+static kvd_status recompute_launch_fp8(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
+                                       int64_t out_row_stride, cudaStream_t stream, const RcAttend *fused = nullptr,
+                                       const AttnLaunchHead *fused_head = nullptr) {
   const LayerState &ls = ctx->layers[layer];
   if (!ls.set || !ctx->store8_codes || !ls.wt8) return KVD_ERR_STATE;
   if (layer >= ctx->layers_stored8) return KVD_ERR_INVALID_ARG;
@@ -582,14 +584,19 @@ extern "C" kvd_status kvd_recompute_kv_fp8(kvd_ctx *ctx, int layer, const kvd_st
   if (out_row_stride < kdim) return KVD_ERR_INVALID_ARG;
   if (out_row_stride % 8 != 0) return KVD_ERR_ALIGNMENT;
   RecomputeParams p;
+  static thread_local FusedParams fp;  // large: keep it off the stack
   int n_jobs = 0, mb = 0;
   for (int i = 0; i < n_ranges; ++i) {
     const kvd_store_range &r = ranges[i];
     if (r.n < 0) return KVD_ERR_INVALID_ARG;
     if (r.n == 0) continue;
     if (r.seq < 0 || r.seq >= d.max_seqs || r.first_row < 0) return KVD_ERR_INVALID_ARG;
-    if (!r.k_out || !r.v_out) return KVD_ERR_INVALID_ARG;
-    if (!aligned16(r.k_out) || !aligned16(r.v_out)) return KVD_ERR_ALIGNMENT;
+    const bool attends = fused && fused[i].q != nullptr;
+    if (!attends) {
+      if (!r.k_out || !r.v_out) return KVD_ERR_INVALID_ARG;
+      if (!aligned16(r.k_out) || !aligned16(r.v_out)) return KVD_ERR_ALIGNMENT;
+    }
+    if (fused) fp.att[n_jobs] = fused[i];
     const int have = ctx->rows_stored8[static_cast<size_t>(layer) * d.max_seqs + r.seq];
     if (r.first_row > have || r.n > have - r.first_row) return KVD_ERR_CAPACITY;
     const size_t slot = store_slot(ctx, layer, r.seq) + r.first_row;
@@ -630,7 +637,21 @@ extern "C" kvd_status kvd_recompute_kv_fp8(kvd_ctx *ctx, int layer, const kvd_st
   p.wide_store = out_row_stride % 16 == 0;
   for (int i = 0; i < n_jobs; ++i)
     if (((reinterpret_cast<uintptr_t>(p.jobs[i].k_out) | reinterpret_cast<uintptr_t>(p.jobs[i].v_out)) & 31u) != 0) p.wide_store = 0;
-  return launch_recompute_fp8(ctx, ls, ctx->store8_maps[layer], p, static_cast<cudaStream_t>(stream_));
+  if (fused) {
+    fp.part_o = fused_head->part_o;
+    fp.part_ml = fused_head->part_ml;
+    fp.n_q = fused_head->n_q;
+    fp.scale_log2e = fused_head->scale_log2e;
+    return launch_recompute_fused(ctx, ls, ctx->store8_maps[layer], ctx->store8_maps[layer], p, fp, stream, 1);
+  }
+  return launch_recompute_fp8(ctx, ls, ctx->store8_maps[layer], p, stream);
+}
+
+extern "C" kvd_status kvd_recompute_kv_fp8(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
+                                           int64_t out_row_stride, void *stream_) {
+  if (!ctx || n_ranges < 0 || n_ranges > KVD_MAX_STORE_RANGES || (n_ranges > 0 && !ranges)) return KVD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  return recompute_launch_fp8(ctx, layer, ranges, n_ranges, out_row_stride, static_cast<cudaStream_t>(stream_));
 }
 
 extern "C" kvd_status kvd_recompute_kv(kvd_ctx *ctx, int layer, const void *rows, const int32_t *positions, int n,
@@ -839,6 +860,60 @@ extern "C" kvd_status kvd_decode_attention_recompute(kvd_ctx *ctx, int layer, in
   }
   st = recompute_launch(ctx, layer, ranges, batch, rows, positions, n_rows, k_rows_out, v_rows_out,
                         out_row_stride > 0 ? out_row_stride : kdim, stream, att, &L);
+  if (st != KVD_OK) return st;
+  if (batch == 0) return KVD_OK;
+  return launch_attention(ctx, L, d.d_head, group, stream);
+}
+
+// The same over the FP8 store: ranges[b] is attended by query b; store_ranges are written as K/V.
+extern "C" kvd_status kvd_decode_attention_recompute_fp8(kvd_ctx *ctx, int layer, int batch, const void *q,
+                                                         const int32_t *q_pos, const kvd_store_range *ranges,
+                                                         const kvd_store_range *store_ranges, int n_store_ranges,
+                                                         int64_t out_row_stride, const kvd_kv_segment *segs,
+                                                         int n_segs, float scale, void *out, void *stream_) {
+  if (!ctx || batch < 0 || n_segs < 0 || n_segs > KVD_MAX_SEGMENTS || n_store_ranges < 0) return KVD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  const LayerState &ls = ctx->layers[layer];
+  if (!ls.set) return KVD_ERR_STATE;
+  if (!ctx->part_o || !ctx->store8_codes || !ls.wt8) return KVD_ERR_STATE;
+  if (ctx->dtype != KVD_DTYPE_BF16) return KVD_ERR_UNSUPPORTED;
+  const kvd_model_desc &d = ctx->desc;
+  const int group = d.n_q_heads / d.n_kv_heads, kdim = d.n_kv_heads * d.d_head;
+  if (ctx->block_n != 256 || kdim % 256 != 0 || !((d.d_head == 256 && (group == 1 || group == 2)) ||
+                                                   (d.d_head == 128 && (group == 1 || group == 2 || group == 4))))
+    return KVD_ERR_UNSUPPORTED;
+  if (batch == 0 && n_store_ranges == 0) return KVD_OK;
+  if (batch > 0 && (!q || !q_pos || !out || !ranges || (n_segs > 0 && !segs))) return KVD_ERR_INVALID_ARG;
+  if (n_store_ranges > 0 && !store_ranges) return KVD_ERR_INVALID_ARG;
+  if (batch > 0 && (!aligned16(q) || !aligned16(out))) return KVD_ERR_ALIGNMENT;
+  if (batch > d.max_batch || batch + n_store_ranges > KVD_MAX_STORE_RANGES) return KVD_ERR_CAPACITY;
+  kvd_status st = check_segments(ctx, batch, q_pos, segs, n_segs);
+  if (st != KVD_OK) return st;
+  int pre[KVD_MAX_STORE_RANGES];
+  for (int b = 0; b < batch; ++b) {
+    if (ranges[b].n < 0) return KVD_ERR_INVALID_ARG;
+    pre[b] = (ranges[b].n + 2 * RC_BLOCK_M - 1) / (2 * RC_BLOCK_M);  // one partial per 256-row block
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  static thread_local AttnLaunch L;  // large: keep it off the stack
+  st = build_attn_launch(ctx, ls, 0, batch, q, q_pos, segs, n_segs, scale, out, pre, L);
+  if (st != KVD_OK) return st;
+  kvd_store_range all[KVD_MAX_STORE_RANGES];
+  RcAttend att[KVD_MAX_STORE_RANGES];
+  for (int b = 0; b < batch; ++b) {
+    all[b] = ranges[b];
+    att[b].q = static_cast<const __nv_bfloat16 *>(q) + static_cast<size_t>(b) * d.n_q_heads * d.d_head;
+    att[b].q_pos = q_pos[b];
+    att[b].lo_pos = ls.window > 0 && q_pos[b] - ls.window + 1 > 0 ? q_pos[b] - ls.window + 1 : 0;
+    att[b].part_base = L.seq[b].merge_base;
+    att[b].reserved = 0;
+  }
+  for (int i = 0; i < n_store_ranges; ++i) {
+    all[batch + i] = store_ranges[i];
+    att[batch + i] = RcAttend{};
+  }
+  st = recompute_launch_fp8(ctx, layer, all, batch + n_store_ranges, out_row_stride > 0 ? out_row_stride : kdim, stream,
+                            att, &L);
   if (st != KVD_OK) return st;
   if (batch == 0) return KVD_OK;
   return launch_attention(ctx, L, d.d_head, group, stream);

@@ -258,7 +258,7 @@ kvd_status launch_recompute(kvd_ctx *ctx, const LayerState &ls, const CUtensorMa
                             const CUtensorMap &tmap_rows, const RecomputeParams &p, cudaStream_t stream);
 kvd_status launch_recompute_fused(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
                                   const CUtensorMap &tmap_rows, const RecomputeParams &p, const FusedParams &fp,
-                                  cudaStream_t stream);
+                                  cudaStream_t stream, int eb = 2);
 kvd_status launch_attention(kvd_ctx *ctx, const AttnLaunch &L, int d_head, int group, cudaStream_t stream);
 kvd_status launch_prepare_weights(kvd_ctx *ctx, const __nv_bfloat16 *w, const __nv_bfloat16 *gamma, __nv_bfloat16 *wt,
                                   int d_hidden, int n_cols, cudaStream_t stream);

@@ -210,8 +210,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   using Cfg = RcCfg<BLOCK_N, D_HEAD, FG, LOSM>;
   constexpr int STAGES = Cfg::STAGES;
   constexpr bool FUSED = FG > 0;
-  static_assert(EB == 2 || (EB == 1 && FG == 0), "the fused variant exists for bf16 operands only");
-  static_assert(DT == 0 || (FG == 0 && EB == 2), "fp16 exists for the plain variant only");
+  static_assert(DT == 0 || (FG == 0 && EB == 2), "fp16 exists for the plain bf16-sized variant only");
   constexpr int KB_ELEMS = RC_BLOCK_K * 2 / EB;  // channels per k block
   static_assert(BLOCK_N % D_HEAD == 0, "a tile must hold whole heads");
 
@@ -457,7 +456,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
           }
           if (TRACE) waited += clock64() - w0;
           tc_fence_after();
-          if (EB == 1) umma_kblock_pair_f8(d_tmem, a_lo, a_lo + b_off_units, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
+          if (EB == 1 && FUSED && swap_ab) umma_kblock_pair_f8(d_tmem, a_lo + b_off_units, a_lo, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
+          else if (EB == 1) umma_kblock_pair_f8(d_tmem, a_lo, a_lo + b_off_units, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
           else if (FUSED && swap_ab) umma_kblock_pair(d_tmem, a_lo + b_off_units, a_lo, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
           else umma_kblock_pair(d_tmem, a_lo, a_lo + b_off_units, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
           full += 8u;
@@ -980,9 +980,17 @@ kvd_status launch_recompute(kvd_ctx *ctx, const LayerState &ls, const CUtensorMa
 // kvd_recompute_kv + kvd_decode_attention).
 kvd_status launch_recompute_fused(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
                                   const CUtensorMap &tmap_rows, const RecomputeParams &p, const FusedParams &fp,
-                                  cudaStream_t stream) {
+                                  cudaStream_t stream, int eb) {
   const int dh = ctx->desc.d_head, g = ctx->desc.n_q_heads / ctx->desc.n_kv_heads;
   if (ctx->block_n != 256 || p.k_cols % 256 != 0) return KVD_ERR_UNSUPPORTED;
+  if (eb == 1) {  // rows and weights as E4M3 codes (the FP8 store)
+    if (dh == 256 && g == 2) return launch_impl<256, 256, false, 2, 1>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
+    if (dh == 256 && g == 1) return launch_impl<256, 256, false, 1, 1>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
+    if (dh == 128 && g == 4) return launch_impl<256, 128, false, 4, 1>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
+    if (dh == 128 && g == 2) return launch_impl<256, 128, false, 2, 1>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
+    if (dh == 128 && g == 1) return launch_impl<256, 128, false, 1, 1>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
+    return KVD_ERR_UNSUPPORTED;
+  }
   if (dh == 256 && g == 2) return launch_sel<256, 256, 2>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
   if (dh == 256 && g == 1) return launch_sel<256, 256, 1>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
   if (dh == 128 && g == 4) return launch_sel<256, 128, 4>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);

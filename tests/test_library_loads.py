@@ -89,6 +89,8 @@ def test_entry_points_reject_null_contexts_and_bad_shapes_without_a_device():
     assert lib.kvd_decode_attention(None, 0, 0, None, None, None, 0, 0.0, None, None) == binding.KVD_ERR_INVALID_ARG
     assert lib.kvd_decode_attention_recompute(None, 0, 0, None, None, None, None, None, 0, None, None, 0, None, 0, 0.0,
                                               None, None) == binding.KVD_ERR_INVALID_ARG
+    assert lib.kvd_decode_attention_recompute_fp8(None, 0, 0, None, None, None, None, 0, 0, None, 0, 0.0, None,
+                                                  None) == binding.KVD_ERR_INVALID_ARG
     # the allocation-free entry point validates shapes and limits on the host before it looks for a device
     qp = (ctypes.c_int32 * 1)(0)
     assert lib.kvd_decode_attention_static(8, 4, 96, 0, 1, None, qp, None, 0, 0.0, None, None) == binding.KVD_ERR_SHAPE
