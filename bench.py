@@ -717,8 +717,11 @@ def run_sweep(wl, peaks):
     Vo = torch.empty_like(Ko)
     dst = torch.empty((2, big_T, kdim), device="cuda", dtype=torch.bfloat16)
     pos = torch.arange(big_T, dtype=torch.int32, device="cuda")
+    arena8 = torch.empty(kvd.kvd_store_bytes_fp8(desc, 1), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_store_fp8(arena8, 1)
     for s_ in range(n_sets):  # the rows are recomputed from the store, as the method does (set = sequence slot)
         ctx.kvd_checkpoint_residual(s_, 0, X[s_], pos, big_T)
+        ctx.kvd_checkpoint_residual_fp8(s_, 0, X[s_], pos, big_T)
     q = wl.q[:1]
     out = wl.out[:1]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
@@ -769,8 +772,32 @@ def run_sweep(wl, peaks):
             dst[0, :T].copy_(K[i % n_sets][:T])
             dst[1, :T].copy_(V[i % n_sets][:T])
 
+        # recompute + attention over the T rebuilt keys: two calls against the fused call, bf16 and FP8 checkpoints
+        def f_two(i):
+            ctx.kvd_recompute_kv(0, None, None, T, Ko, Vo, kdim, seq=i % n_sets, first_row=0)
+            ctx.kvd_decode_attention(0, 1, q, [T], [[(Ko, Vo, kdim, 0, T)]], 0.0, out)
+
+        def f_fused(i):
+            ctx.kvd_decode_attention_recompute(0, 1, q, [T], [(i % n_sets, 0, T)], None, None, 0, None, None, kdim,
+                                               [[]], 0.0, out)
+
+        def f_rec8(i):
+            ctx.kvd_recompute_kv_fp8(0, [(i % n_sets, 0, T, Ko, Vo)], kdim)
+
+        def f_two8(i):
+            ctx.kvd_recompute_kv_fp8(0, [(i % n_sets, 0, T, Ko, Vo)], kdim)
+            ctx.kvd_decode_attention(0, 1, q, [T], [[(Ko, Vo, kdim, 0, T)]], 0.0, out)
+
+        def f_fused8(i):
+            ctx.kvd_decode_attention_recompute_fp8(0, 1, q, [T], [(i % n_sets, 0, T)], [], kdim, [[]], 0.0, out)
+
         rec, att, cpy = timed(f_rec), timed(f_att), timed(f_cp)
         rec_g, att_g, cpy_g = replayed(f_rec), replayed(f_att), replayed(f_cp)
+        variants = {"recompute_fp8_replay_us": replayed(f_rec8) * 1e3,
+                    "recompute_then_attention_replay_us": replayed(f_two) * 1e3,
+                    "fused_replay_us": replayed(f_fused) * 1e3,
+                    "recompute_fp8_then_attention_replay_us": replayed(f_two8) * 1e3,
+                    "fused_fp8_replay_us": replayed(f_fused8) * 1e3}
         flops = 4.0 * T * shape.n_kv_heads * shape.d_hidden * shape.d_head
         byts = T * 4 * shape.n_kv_heads * shape.d_head
         rows.append({"T": T,
@@ -781,7 +808,7 @@ def run_sweep(wl, peaks):
                      "recompute_replay_us": rec_g * 1e3, "recompute_replay_tflops": flops / (rec_g * 1e-3) / 1e12,
                      "attention_replay_us": att_g * 1e3, "attention_replay_gbs": byts / (att_g * 1e-3) / 1e9,
                      "copy_replay_us": cpy_g * 1e3, "ratio_replay_recompute_over_copy": rec_g / cpy_g,
-                     "ratio_replay_recompute_over_attention_read": rec_g / att_g})
+                     "ratio_replay_recompute_over_attention_read": rec_g / att_g, **variants})
     ctx.close()
     return rows
 
