@@ -872,8 +872,11 @@ def run_stack_configs(args):
         c.kvd_attach_store(arena, 1)
         xs = torch.randn((ctx_len, shape.d_hidden), device="cuda").to(torch.bfloat16)
         ps = torch.arange(ctx_len, device="cuda", dtype=torch.int32)
+        arena8 = torch.empty(kvd.kvd_store_bytes_fp8(desc, 1), dtype=torch.uint8, device="cuda")
+        c.kvd_attach_store_fp8(arena8, 1)
         for b in range(batch):
             c.kvd_checkpoint_residual(b, 0, xs, ps, ctx_len)  # STORE_RESIDUAL of the whole context
+            c.kvd_checkpoint_residual_fp8(b, 0, xs, ps, ctx_len)  # and as E4M3 checkpoints (second store)
         M = batch * n_old
         Ko = torch.empty((max(M, 1), kdim), device="cuda", dtype=torch.bfloat16)
         Vo = torch.empty_like(Ko)
@@ -925,6 +928,17 @@ def run_stack_configs(args):
             c.kvd_decode_attention_recompute(0, batch, q, qpos, franges, xc, pc, batch, kc, vc, kdim,
                                              segs_live[i % n_sets], 0.0, out)
 
+        # the same two layer forms with the evicted rows taken from the FP8 store; K_t, V_t of the new tokens
+        # still come from their bf16 rows (a launch of their own, as in the full-cache layer)
+        def layer_fp8(i):
+            cur(i)
+            c.kvd_recompute_kv_fp8(0, ranges, kdim)
+            att(i)
+
+        def layer_fp8_fused(i):
+            cur(i)
+            c.kvd_decode_attention_recompute_fp8(0, batch, q, qpos, franges, [], kdim, segs_live[i % n_sets], 0.0, out)
+
         # memory-bound cases first, each after a short pause: a long run of GEMMs at the power cap
         # leaves the clocks low for whatever is measured next
         def rested(fn):
@@ -936,6 +950,7 @@ def run_stack_configs(args):
         t_layer_full = rested(layer_full)
         t_rec, t_layer_kvd = rested(rec), rested(layer_kvd)
         t_layer_fused = rested(layer_fused)
+        t_layer_fp8, t_layer_fp8_fused = rested(layer_fp8), rested(layer_fp8_fused)
         assert c.kvd_poll_status() == kvd.KVD_OK
         flops = 4.0 * (M + batch) * shape.n_kv_heads * shape.d_hidden * shape.d_head
         keys = batch * (ctx_len + 1 - lo)
@@ -946,6 +961,7 @@ def run_stack_configs(args):
                 "current_kv_only_us": t_cur, "attention_us": t_att, "attention_gbs": byts / t_att / 1e3,
                 "fullcache_attention_us": t_full, "fullcache_attention_gbs": byts / t_full / 1e3,
                 "kvdirect_layer_us": t_layer_kvd, "kvdirect_fused_layer_us": t_layer_fused,
+                "kvdirect_fp8_layer_us": t_layer_fp8, "kvdirect_fp8_fused_layer_us": t_layer_fp8_fused,
                 "fullcache_layer_us": t_layer_full}
 
     result = {"peaks": peaks, "gemma3_4b_stack_ctx2048_window256": [], "qwen3_4b_ctx32768_batch8_window512": None}
@@ -957,12 +973,16 @@ def run_stack_configs(args):
         result["gemma3_4b_stack_ctx2048_window256"].append(
             {"batch": batch, "kvdirect_decode_step_us": kvd_step,
              "kvdirect_fused_decode_step_us": 5 * g["kvdirect_fused_layer_us"] + 29 * l["kvdirect_fused_layer_us"],
+             "kvdirect_fp8_decode_step_us": 5 * g["kvdirect_fp8_layer_us"] + 29 * l["kvdirect_fp8_layer_us"],
+             "kvdirect_fp8_fused_decode_step_us": 5 * g["kvdirect_fp8_fused_layer_us"] + 29 * l["kvdirect_fp8_fused_layer_us"],
              "fullcache_decode_step_us": full_step,
              "ratio": kvd_step / full_step, "recomputed_tokens_per_s": batch * (5 * g["rows_recomputed"] // batch +
              29 * l["rows_recomputed"] // batch) / (kvd_step * 1e-6), "global_layer": g, "local_layer": l})
     qw = layer_case(QWEN3_4B, 32768, 512, 8)
     qw["step_us_36_layers"] = 36 * qw["kvdirect_layer_us"]
     qw["fused_step_us_36_layers"] = 36 * qw["kvdirect_fused_layer_us"]
+    qw["fp8_step_us_36_layers"] = 36 * qw["kvdirect_fp8_layer_us"]
+    qw["fp8_fused_step_us_36_layers"] = 36 * qw["kvdirect_fp8_fused_layer_us"]
     qw["fullcache_step_us_36_layers"] = 36 * qw["fullcache_layer_us"]
     qw["recompute_frac_of_sustained_peak"] = qw["recompute_tflops"] / peaks["bf16_tflops_sustained"]
     qw["recompute_frac_of_burst_peak"] = qw["recompute_tflops"] / peaks["bf16_tflops"]
