@@ -405,6 +405,10 @@ def run_gpu(args):
         for i in range(2):
             wl.k_checkpoint_fp8(i)
             wl.k_recompute_fp8(i)
+        # and the FP8 checkpoints rebuilt and attended in one kernel (T + 1 rows, nothing kept)
+        wl.append_current_fp8()
+        for i in range(2):
+            wl.k_fused_fp8(i)
         barrier()
         if args.profile_long_attn:
             # a few eager decode-attention calls over 32769 keys (134 MB each, larger than L2)
