@@ -43,6 +43,8 @@
 //           transposed and reduced with the softmax weights; nothing of K or V is written.
 //   EB = 1  FP8 checkpoints (kvd_recompute_kv_fp8): rows and weights are E4M3 codes, a k block is 128
 //           channels, the MMA kind is f8f6f4; the scales ride in the per-row factor of the epilogue.
+//           Combines with FG > 0 (kvd_decode_attention_recompute_fp8).
+//   DT = 1  fp16 rows, weights and outputs (kvd_set_dtype), plain variant only.
 #include <math_constants.h>
 #include <string.h>
 
