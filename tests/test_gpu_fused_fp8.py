@@ -147,3 +147,33 @@ def test_fused_fp8_is_refused_without_its_store_and_for_other_shapes():
         ctx.kvd_decode_attention_recompute_fp8(0, 1, q, [0], [(0, 0, 0)], [], shape.n_kv_heads * shape.d_head, [[]], 0.0, out)
     assert e.value.status == 6
     assert ctx.kvd_poll_status() == kvd.KVD_OK
+
+
+def test_fused_fp8_decode_loop_with_nothing_kept_crosses_a_block_boundary():
+    """Twelve decode steps of one sequence whose every token lives in the FP8 store only: the new row is
+    quantised in, then all rows (250 -> 262, across the 256-row block boundary) are rebuilt and attended."""
+    shape = GEMMA3_4B_GLOBAL
+    ctx, w = open_layer(shape, max_tokens=512)
+    arena = torch.zeros(kvd.kvd_store_bytes_fp8(ctx.desc, 1), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_store_fp8(arena, 1)
+    kdim = shape.n_kv_heads * shape.d_head
+    n0, steps = 250, 12
+    X = make_residuals(shape, n0 + steps, seed=77, outliers=True)
+    pos = np.arange(n0 + steps)
+    x, p = dev(X), torch.from_numpy(pos.astype(np.int32)).cuda()
+    q_bits = make_query(shape, steps, seed=78)
+    q = dev(q_bits)
+    Kr, Vr = oracle_fp8_kv(shape, w, X, pos)
+    Kr = Kr.reshape(-1, shape.n_kv_heads, shape.d_head)
+    Vr = Vr.reshape(-1, shape.n_kv_heads, shape.d_head)
+    ctx.kvd_checkpoint_residual_fp8(0, 0, x[:n0], p[:n0], n0)
+    out = torch.zeros((1, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda")
+    for t in range(steps):
+        n = n0 + t + 1
+        ctx.kvd_checkpoint_residual_fp8(0, 0, x[n - 1:n], p[n - 1:n], 1)
+        assert ctx.kvd_rows_stored_fp8(0, 0) == n
+        ctx.kvd_decode_attention_recompute_fp8(0, 1, q[t:t + 1], [n - 1], [(0, 0, n)], [], kdim, [[]], 0.0, out)
+        ref = oracle.decode_attention(bf16_to_f64(q_bits[t]), n - 1, [(Kr[:n], Vr[:n], 0)],
+                                      1.0 / math.sqrt(shape.d_head), shape.sliding_window)
+        attn_check(host_f64(out)[0], ref, f"step {t}")
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
