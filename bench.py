@@ -932,16 +932,27 @@ def run_stack_configs(args):
             c.kvd_decode_attention_recompute(0, batch, q, qpos, franges, xc, pc, batch, kc, vc, kdim,
                                              segs_live[i % n_sets], 0.0, out)
 
-        # the same two layer forms with the evicted rows taken from the FP8 store; K_t, V_t of the new tokens
-        # still come from their bf16 rows (a launch of their own, as in the full-cache layer)
+        # the same two layer forms with the evicted rows taken from the FP8 store.  K_t, V_t of the new tokens:
+        # up to 8 sequences -- from their quantised rows in the FP8 store, inside the same launch (one 256-row
+        # block per sequence); larger batches -- from their bf16 rows in a launch of their own, as in the
+        # full-cache layer
+        new_in_store = batch <= 8
+        if new_in_store:
+            for b in range(batch):
+                c.kvd_checkpoint_residual_fp8(b, 0, xc[b:b + 1], pc[b:b + 1], 1)
+        new_ranges = [(b, ctx_len, 1, kc[b:], vc[b:]) for b in range(batch)] if new_in_store else []
+
         def layer_fp8(i):
-            cur(i)
-            c.kvd_recompute_kv_fp8(0, ranges, kdim)
+            if not new_in_store:
+                cur(i)
+            c.kvd_recompute_kv_fp8(0, ranges + new_ranges, kdim)
             att(i)
 
         def layer_fp8_fused(i):
-            cur(i)
-            c.kvd_decode_attention_recompute_fp8(0, batch, q, qpos, franges, [], kdim, segs_live[i % n_sets], 0.0, out)
+            if not new_in_store:
+                cur(i)
+            c.kvd_decode_attention_recompute_fp8(0, batch, q, qpos, franges, new_ranges, kdim, segs_live[i % n_sets],
+                                                 0.0, out)
 
         # memory-bound cases first, each after a short pause: a long run of GEMMs at the power cap
         # leaves the clocks low for whatever is measured next
