@@ -394,6 +394,38 @@ extern "C" kvd_status kvd_checkpoint_residual(kvd_ctx *ctx, int seq, int layer, 
   return st;
 }
 
+// The launch parameters every variant of the recompute kernel shares (jobs are filled in by the caller).
+static void fill_launch_params(const kvd_ctx *ctx, const LayerState &ls, RecomputeParams &p, int n_jobs, int m_blocks,
+                               int k_blocks, int64_t out_row_stride) {
+  const kvd_model_desc &d = ctx->desc;
+  const int kdim = d.n_kv_heads * d.d_head;
+  p.n_jobs = n_jobs;
+  p.num_k_blocks = k_blocks;
+  p.num_m_blocks = m_blocks;
+  p.num_n_blocks = 2 * kdim / ctx->block_n;
+  p.k_cols = kdim;
+  p.out_row_stride = out_row_stride;
+  p.inv_d_hidden = 1.0f / static_cast<float>(d.d_hidden);
+  p.rms_eps = d.rms_eps;
+  p.qk_norm = d.qk_norm;
+  p.qk_eps = d.qk_norm_eps;
+  p.rope_style = d.rope_style;
+  p.rope_hi = ls.rope.hi;
+  p.rope_lo = ls.rope.lo;
+  p.max_pos = ls.rope.n_hi * ROPE_LO_SIZE < d.max_tokens_per_seq ? ls.rope.n_hi * ROPE_LO_SIZE : d.max_tokens_per_seq;
+  p.gamma_k = d.qk_norm ? ls.gamma_k : nullptr;
+  p.status = ctx->d_status;
+  p.timeout_ns = ctx->timeout_ns;
+  p.trace = nullptr;
+  p.ext_rows = nullptr;
+  p.w_scale = nullptr;
+  p.row_chunks = d.d_hidden / 8;
+  // 32-byte stores need every output row 32-byte aligned
+  p.wide_store = out_row_stride % 16 == 0;
+  for (int i = 0; i < n_jobs; ++i)
+    if (((reinterpret_cast<uintptr_t>(p.jobs[i].k_out) | reinterpret_cast<uintptr_t>(p.jobs[i].v_out)) & 31u) != 0) p.wide_store = 0;
+}
+
 // Shared body of kvd_recompute_kv and kvd_recompute_kv_step: validate, build the job table (store
 // ranges first, then the caller's rows), launch once.
 // With `fused` (one RcAttend per range, q == nullptr for a range that is to be stored as usual) the
@@ -469,30 +501,8 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
   // the kernel is handed both maps; an unused one aliases the other
   const CUtensorMap &tmap_store = any_store ? ctx->store_maps[layer] : tmap_rows;
   const CUtensorMap &tmap_ext = n_rows > 0 ? tmap_rows : ctx->store_maps[layer];
-  p.n_jobs = n_jobs;
-  p.num_k_blocks = d.d_hidden / RC_BLOCK_K;
-  p.num_m_blocks = mb;
-  p.num_n_blocks = 2 * kdim / ctx->block_n;
-  p.k_cols = kdim;
-  p.out_row_stride = out_row_stride;
-  p.inv_d_hidden = 1.0f / static_cast<float>(d.d_hidden);
-  p.rms_eps = d.rms_eps;
-  p.qk_norm = d.qk_norm;
-  p.qk_eps = d.qk_norm_eps;
-  p.rope_style = d.rope_style;
-  p.rope_hi = ls.rope.hi;
-  p.rope_lo = ls.rope.lo;
-  p.max_pos = ls.rope.n_hi * ROPE_LO_SIZE < d.max_tokens_per_seq ? ls.rope.n_hi * ROPE_LO_SIZE : d.max_tokens_per_seq;
-  p.gamma_k = d.qk_norm ? ls.gamma_k : nullptr;
-  p.status = ctx->d_status;
-  p.timeout_ns = ctx->timeout_ns;
+  fill_launch_params(ctx, ls, p, n_jobs, mb, d.d_hidden / RC_BLOCK_K, out_row_stride);
   p.ext_rows = static_cast<const __nv_bfloat16 *>(rows);
-  p.w_scale = nullptr;
-  p.row_chunks = d.d_hidden / 8;
-  p.wide_store = out_row_stride % 16 == 0;
-  for (int i = 0; i < n_jobs; ++i)
-    if (((reinterpret_cast<uintptr_t>(p.jobs[i].k_out) | reinterpret_cast<uintptr_t>(p.jobs[i].v_out)) & 31u) != 0) p.wide_store = 0;
-  p.trace = nullptr;
   if (ctx->trace) {
     const int tiles = p.num_m_blocks * p.num_n_blocks;
     const size_t ctas = 2 * static_cast<size_t>(tiles < ctx->num_sms / 2 ? tiles : ctx->num_sms / 2);
@@ -613,30 +623,9 @@ static kvd_status recompute_launch_fp8(kvd_ctx *ctx, int layer, const kvd_store_
     mb += (r.n + 2 * RC_BLOCK_M - 1) / (2 * RC_BLOCK_M);
   }
   if (n_jobs == 0) return KVD_OK;
-  p.n_jobs = n_jobs;
-  p.num_k_blocks = (d.d_hidden + 2 * RC_BLOCK_K - 1) / (2 * RC_BLOCK_K);  // 128 channels per k block; the tail reads zeros
-  p.num_m_blocks = mb;
-  p.num_n_blocks = 2 * kdim / ctx->block_n;
-  p.k_cols = kdim;
-  p.out_row_stride = out_row_stride;
-  p.inv_d_hidden = 1.0f / static_cast<float>(d.d_hidden);
-  p.rms_eps = d.rms_eps;
-  p.qk_norm = d.qk_norm;
-  p.qk_eps = d.qk_norm_eps;
-  p.rope_style = d.rope_style;
-  p.rope_hi = ls.rope.hi;
-  p.rope_lo = ls.rope.lo;
-  p.max_pos = ls.rope.n_hi * ROPE_LO_SIZE < d.max_tokens_per_seq ? ls.rope.n_hi * ROPE_LO_SIZE : d.max_tokens_per_seq;
-  p.gamma_k = d.qk_norm ? ls.gamma_k : nullptr;
-  p.status = ctx->d_status;
-  p.timeout_ns = ctx->timeout_ns;
-  p.trace = nullptr;
-  p.ext_rows = nullptr;
-  p.row_chunks = d.d_hidden / 8;
+  // 128 channels per k block; the tail reads zeros
+  fill_launch_params(ctx, ls, p, n_jobs, mb, (d.d_hidden + 2 * RC_BLOCK_K - 1) / (2 * RC_BLOCK_K), out_row_stride);
   p.w_scale = ls.w_scale8;
-  p.wide_store = out_row_stride % 16 == 0;
-  for (int i = 0; i < n_jobs; ++i)
-    if (((reinterpret_cast<uintptr_t>(p.jobs[i].k_out) | reinterpret_cast<uintptr_t>(p.jobs[i].v_out)) & 31u) != 0) p.wide_store = 0;
   if (fused) {
     fp.part_o = fused_head->part_o;
     fp.part_ml = fused_head->part_ml;
