@@ -131,11 +131,12 @@ kvd_status kvd_create(const kvd_model_desc *desc, kvd_ctx **out);
 /* Release everything the context allocated (prepared weights, tables).  Synchronises the device. */
 void kvd_destroy(kvd_ctx *ctx);
 
-/* Element type of residual rows, weights and K/V outputs.  bf16 is the default and the only type the
- * attention, fused and FP8 entry points accept (KVD_ERR_UNSUPPORTED otherwise); fp16 exists for
- * kvd_checkpoint_residual / kvd_recompute_kv / kvd_recompute_kv_step -- the reconstruction identities
- * (Eq. 13-14) do not depend on the element type, and the bitwise recompute-equals-first-pass check of the
- * paper's Section 5.1 is run in both.  Call before any kvd_set_layer / checkpoint (KVD_ERR_STATE after). */
+/* Element type of residual rows, weights, K/V, queries and attention outputs.  bf16 is the default and the
+ * only type the fused, FP8 and static entry points accept (KVD_ERR_UNSUPPORTED otherwise); fp16 exists for
+ * kvd_checkpoint_residual / kvd_recompute_kv / kvd_recompute_kv_step / kvd_decode_attention -- the
+ * reconstruction identities (Eq. 13-14) do not depend on the element type, and the bitwise
+ * recompute-equals-first-pass check of the paper's Section 5.1 is run in both.  Call before any
+ * kvd_set_layer / checkpoint (KVD_ERR_STATE after). */
 #define KVD_DTYPE_BF16 0
 #define KVD_DTYPE_F16 1
 kvd_status kvd_set_dtype(kvd_ctx *ctx, int dtype);

@@ -372,7 +372,7 @@ class Kvd:
             float(scale), _ptr(out), _stream(stream)), "kvd_decode_attention_recompute_fp8")
 
     def kvd_set_dtype(self, dtype: int) -> None:
-        """0 = bf16 (default), 1 = fp16 (checkpoint / recompute entry points only); before any kvd_set_layer."""
+        """0 = bf16 (default), 1 = fp16 (checkpoint, recompute and kvd_decode_attention); before any kvd_set_layer."""
         self._check(self._lib.kvd_set_dtype(self._h, dtype), "kvd_set_dtype")
 
     def kvd_attach_store_fp8(self, arena, layers_stored: int) -> None:

@@ -782,7 +782,6 @@ extern "C" kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, c
   const LayerState &ls = ctx->layers[layer];
   if (!ls.set) return KVD_ERR_STATE;
   if (!ctx->part_o) return KVD_ERR_STATE;
-  if (ctx->dtype != KVD_DTYPE_BF16) return KVD_ERR_UNSUPPORTED;  // attention reads bf16 K/V
   if (batch == 0) return KVD_OK;
   if (!q || !q_pos || !out || (n_segs > 0 && !segs)) return KVD_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(out)) return KVD_ERR_ALIGNMENT;

@@ -64,7 +64,8 @@ __device__ __forceinline__ float reduce8_transposed(const float (&v)[8], int lig
   return w1;
 }
 
-template <int D_HEAD, int G, int NSEQ>
+// DT: element type of q, K, V and the output (0 = bf16, 1 = fp16; kvd_set_dtype).
+template <int D_HEAD, int G, int NSEQ, int DT = 0>
 __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM) kvd_attn_split_kernel(const __grid_constant__ AttnLaunchT<NSEQ> P) {
   constexpr int LPK = D_HEAD / 8;         // lanes per key
   constexpr int KPL = 32 / LPK;           // keys per warp-wide load
@@ -110,10 +111,11 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM) kvd_attn_split_ker
   for (int g = 0; g < G; ++g) {
     const __nv_bfloat16 *qp = P.q + (static_cast<size_t>(si) * P.n_q + kvh * G + g) * D_HEAD + lig * 8;
     const uint4 w = *reinterpret_cast<const uint4 *>(qp);
-    qf[g][0] = pack2(bf16_lo(w.x) * P.scale_log2e, bf16_hi(w.x) * P.scale_log2e);
-    qf[g][1] = pack2(bf16_lo(w.y) * P.scale_log2e, bf16_hi(w.y) * P.scale_log2e);
-    qf[g][2] = pack2(bf16_lo(w.z) * P.scale_log2e, bf16_hi(w.z) * P.scale_log2e);
-    qf[g][3] = pack2(bf16_lo(w.w) * P.scale_log2e, bf16_hi(w.w) * P.scale_log2e);
+    const uint64_t sc2 = pack2(P.scale_log2e, P.scale_log2e);
+    qf[g][0] = fmul2(x2_to_f32x2<DT>(w.x), sc2);
+    qf[g][1] = fmul2(x2_to_f32x2<DT>(w.y), sc2);
+    qf[g][2] = fmul2(x2_to_f32x2<DT>(w.z), sc2);
+    qf[g][3] = fmul2(x2_to_f32x2<DT>(w.w), sc2);
   }
 
   float m_run[G], l_run[G];
@@ -192,8 +194,8 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM) kvd_attn_split_ker
     float part[G][U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const uint64_t k0 = bf16x2_to_f32x2(kr[u].x), k1 = bf16x2_to_f32x2(kr[u].y);
-      const uint64_t k2 = bf16x2_to_f32x2(kr[u].z), k3 = bf16x2_to_f32x2(kr[u].w);
+      const uint64_t k0 = x2_to_f32x2<DT>(kr[u].x), k1 = x2_to_f32x2<DT>(kr[u].y);
+      const uint64_t k2 = x2_to_f32x2<DT>(kr[u].z), k3 = x2_to_f32x2<DT>(kr[u].w);
 #pragma unroll
       for (int g = 0; g < G; ++g) {
         // even and odd channels accumulate side by side, then are added
@@ -241,8 +243,8 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM) kvd_attn_split_ker
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const uint64_t v0 = bf16x2_to_f32x2(vr[u].x), v1 = bf16x2_to_f32x2(vr[u].y);
-      const uint64_t v2 = bf16x2_to_f32x2(vr[u].z), v3 = bf16x2_to_f32x2(vr[u].w);
+      const uint64_t v0 = x2_to_f32x2<DT>(vr[u].x), v1 = x2_to_f32x2<DT>(vr[u].y);
+      const uint64_t v2 = x2_to_f32x2<DT>(vr[u].z), v3 = x2_to_f32x2<DT>(vr[u].w);
 #pragma unroll
       for (int g = 0; g < G; ++g) {
         const uint64_t p2 = pack2(pb[g][u], pb[g][u]);
@@ -329,20 +331,33 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM) kvd_attn_split_ker
 // to bf16 for the second product (fp32 sums), as the scores' softmax weights are in any tensor-core
 // attention; the partials have the same format as those of the kernel above and go to the same merge.
 // Chunking, the position -> (chunk, warp, block) assignment and the masking rules are identical.
-__device__ __forceinline__ void mma_bf16_m16n8k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                                  uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
-               "{%0, %1, %2, %3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+template <int DT>
+__device__ __forceinline__ void mma_x16_m16n8k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                 uint32_t b0, uint32_t b1) {
+  if constexpr (DT == 0)
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+                 "{%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  else
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+                 "{%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ void mma_bf16_m16n8k8(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
-  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5}, {%6}, {%0, %1, %2, %3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a0), "r"(a1), "r"(b0));
+template <int DT>
+__device__ __forceinline__ void mma_x16_m16n8k8(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+  if constexpr (DT == 0)
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5}, {%6}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(b0));
+  else
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5}, {%6}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(b0));
 }
 
-template <int D_HEAD, int G, int NSEQ>
+template <int D_HEAD, int G, int NSEQ, int DT = 0>
 __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM)
     kvd_attn_split_mma_kernel(const __grid_constant__ AttnLaunchT<NSEQ> P) {
   static_assert(G >= 1 && G <= 8 && D_HEAD <= 128, "query heads are the 8 columns of the second product");
@@ -463,8 +478,8 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM)
       float sc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int j = 0; j < KP; ++j) {
-        mma_bf16_m16n8k16(sc, qa[j][0], 0u, qa[j][1], 0u, kr[b][j].x, kr[b][j].y);
-        mma_bf16_m16n8k16(sc, qa[j][2], 0u, qa[j][3], 0u, kr[b][j].z, kr[b][j].w);
+        mma_x16_m16n8k16<DT>(sc, qa[j][0], 0u, qa[j][1], 0u, kr[b][j].x, kr[b][j].y);
+        mma_x16_m16n8k16<DT>(sc, qa[j][2], 0u, qa[j][3], 0u, kr[b][j].z, kr[b][j].w);
       }
       // thread (g8, t): head g8, keys 2t and 2t+1 of the block
       const float s0 = ((vmask >> (2 * b)) & 1u) ? sc[0] * P.scale_log2e : -CUDART_INF_F;
@@ -478,7 +493,7 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM)
       const float p0 = exp2f(s0 - m_use), p1 = exp2f(s1 - m_use);
       l_run = fmaf(l_run, corr, p0 + p1);
       m_run = m_new;
-      const uint32_t pk = pack_bf16(p0, p1);  // B fragment of the second product: keys 2t, 2t+1, head g8
+      const uint32_t pk = pack_out<DT>(p0, p1);  // B fragment of the second product: keys 2t, 2t+1, head g8
       // ---- rescale the accumulators when a maximum moved (columns are heads 2t and 2t+1)
       const float c_even = __shfl_sync(0xffffffffu, corr, (2 * t) * 4);
       const float c_odd = __shfl_sync(0xffffffffu, corr, (2 * t + 1) * 4);
@@ -501,7 +516,7 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM)
         for (int e = 0; e < 4; ++e) {
           const uint32_t a0 = __byte_perm(v0[e], v1[e], 0x5410);  // channel 2e of both keys
           const uint32_t a1 = __byte_perm(v0[e], v1[e], 0x7632);  // channel 2e + 1 of both keys
-          mma_bf16_m16n8k8(oacc[4 * i + e], a0, a1, pk);
+          mma_x16_m16n8k8<DT>(oacc[4 * i + e], a0, a1, pk);
         }
       }
     }
@@ -563,7 +578,7 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM)
 // launch has as many warps per CTA as its longest sequence has groups (at most 16; beyond that a warp
 // takes several groups, 16 apart); a shorter sequence leaves the extra warps idle, so its summation
 // order depends on its own chunk count only.
-template <int D_HEAD, int G, int NSEQ>
+template <int D_HEAD, int G, int NSEQ, int DT = 0>
 __global__ void __launch_bounds__(AT_MERGE_THREADS)
     kvd_attn_merge_kernel(const __grid_constant__ AttnLaunchT<NSEQ> P) {
   constexpr int SLICES = D_HEAD / AT_MERGE_SLICE;
@@ -659,8 +674,9 @@ __global__ void __launch_bounds__(AT_MERGE_THREADS)
       lv += s_l[w][g];
     }
     const float r = lv > 0.f ? ov / lv : 0.f;
-    P.out[(static_cast<size_t>(si) * P.n_q + kvh * G + g) * D_HEAD + slice * AT_MERGE_SLICE + c] =
-        __float2bfloat16_rn(r);
+    const size_t oi = (static_cast<size_t>(si) * P.n_q + kvh * G + g) * D_HEAD + slice * AT_MERGE_SLICE + c;
+    if constexpr (DT == 0) P.out[oi] = __float2bfloat16_rn(r);
+    else reinterpret_cast<__half *>(P.out)[oi] = __float2half_rn(r);
   }
 }
 
@@ -670,7 +686,7 @@ struct AttnSmem {
   static constexpr int NPART = AT_WARPS * (32 / (D_HEAD / 8));
   static constexpr int BYTES = NPART * G * (D_HEAD + 2) * 4;
 };
-template <int D_HEAD, int G, int NSEQ>
+template <int D_HEAD, int G, int NSEQ, int DT>
 static cudaError_t attn_configure() {
   static bool done[64] = {};
   int dev = 0;
@@ -678,7 +694,7 @@ static cudaError_t attn_configure() {
   if (e != cudaSuccess) return e;
   if (!done[dev & 63]) {
     if constexpr (!(G >= 3 && D_HEAD <= 128)) {
-      e = cudaFuncSetAttribute(kvd_attn_split_kernel<D_HEAD, G, NSEQ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      e = cudaFuncSetAttribute(kvd_attn_split_kernel<D_HEAD, G, NSEQ, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                AttnSmem<D_HEAD, G>::BYTES);
       if (e != cudaSuccess) return e;
     }
@@ -687,9 +703,9 @@ static cudaError_t attn_configure() {
   return cudaSuccess;
 }
 // the two launches of a decode step: stream + partials, then merge
-template <int D_HEAD, int G, int NSEQ>
+template <int D_HEAD, int G, int NSEQ, int DT = 0>
 static cudaError_t attn_launch_pair(const AttnLaunchT<NSEQ> &S, cudaStream_t stream) {
-  cudaError_t e = attn_configure<D_HEAD, G, NSEQ>();
+  cudaError_t e = attn_configure<D_HEAD, G, NSEQ, DT>();
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
@@ -708,10 +724,10 @@ static cudaError_t attn_launch_pair(const AttnLaunchT<NSEQ> &S, cudaStream_t str
     cfg.blockDim = dim3(AT_THREADS, 1, 1);
     if constexpr (G >= 3 && D_HEAD <= 128) {
       cfg.dynamicSmemBytes = 0;
-      e = cudaLaunchKernelEx(&cfg, kvd_attn_split_mma_kernel<D_HEAD, G, NSEQ>, S);
+      e = cudaLaunchKernelEx(&cfg, kvd_attn_split_mma_kernel<D_HEAD, G, NSEQ, DT>, S);
     } else {
       cfg.dynamicSmemBytes = AttnSmem<D_HEAD, G>::BYTES;
-      e = cudaLaunchKernelEx(&cfg, kvd_attn_split_kernel<D_HEAD, G, NSEQ>, S);
+      e = cudaLaunchKernelEx(&cfg, kvd_attn_split_kernel<D_HEAD, G, NSEQ, DT>, S);
     }
     if (e != cudaSuccess) return e;
   }
@@ -724,7 +740,7 @@ static cudaError_t attn_launch_pair(const AttnLaunchT<NSEQ> &S, cudaStream_t str
   cfg.gridDim = dim3(S.n_seqs * S.n_kv * (D_HEAD / AT_MERGE_SLICE), 1, 1);
   cfg.blockDim = dim3(32 * merge_warps, 1, 1);
   cfg.dynamicSmemBytes = 0;
-  return cudaLaunchKernelEx(&cfg, kvd_attn_merge_kernel<D_HEAD, G, NSEQ>, S);
+  return cudaLaunchKernelEx(&cfg, kvd_attn_merge_kernel<D_HEAD, G, NSEQ, DT>, S);
 }
 
 template <int D_HEAD, int G, int NSEQ>
@@ -733,7 +749,9 @@ static kvd_status launch_attn_impl(kvd_ctx *ctx, const AttnLaunch &L, cudaStream
     static thread_local AttnLaunchT<NSEQ> S;
     static_cast<AttnLaunchHead &>(S) = static_cast<const AttnLaunchHead &>(L);
     for (int i = 0; i < L.n_seqs; ++i) S.seq[i] = L.seq[i];
-    cudaError_t e = attn_launch_pair<D_HEAD, G, NSEQ>(S, stream);
+    // fp16 contexts (kvd_set_dtype): the same kernels reading and writing fp16
+    cudaError_t e = ctx->dtype == 1 ? attn_launch_pair<D_HEAD, G, NSEQ, 1>(S, stream)
+                                    : attn_launch_pair<D_HEAD, G, NSEQ, 0>(S, stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch attention");
     ctx->launches += L.total_chunks > 0 ? 2 : 1;
   }

@@ -320,8 +320,8 @@ __device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
 // the two bf16 halves of a 32-bit word as a packed pair of fp32
 __device__ __forceinline__ uint64_t bf16x2_to_f32x2(uint32_t w) { return pack2(bf16_lo(w), bf16_hi(w)); }
 
-// 16-bit element type of rows, weights and outputs: DT = 0 bf16 (the default everywhere), DT = 1 fp16 (the
-// recompute path only: the dtype-invariance check of the paper's Section 5.1)
+// 16-bit element type of rows, weights, K/V and outputs: DT = 0 bf16 (the default everywhere), DT = 1 fp16
+// (checkpoint, recompute and decode attention: the dtype-invariance check of the paper's Section 5.1)
 template <int DT>
 __device__ __forceinline__ uint64_t x2_to_f32x2(uint32_t w) {
   if constexpr (DT == 0) {

@@ -6,7 +6,8 @@ outputs:
     than bf16, so the bf16 tolerances hold with room to spare; a tighter relative bound is asserted too);
   * K/V recomputed from checkpointed rows equal, bit for bit, the K/V of the first pass at every length
     16 ... 256 and for single rows (max |dK| = max |dV| = 0), as in bf16;
-  * the entry points that read bf16 K/V refuse an fp16 context.
+  * decode attention on fp16 q, K, V follows the oracle too, with bits independent of the segment layout;
+  * the bf16-only entry points (fused, FP8) refuse an fp16 context.
 """
 import numpy as np
 import pytest
@@ -99,7 +100,59 @@ def test_fp16_reconstruction_is_bit_exact_at_every_length(shape):
         assert torch.equal(vr.view(torch.int16), vc.view(torch.int16)), length
 
 
-def test_fp16_context_is_refused_where_bf16_is_required_and_the_type_is_fixed_once_used():
+def rand_f16(shape_, seed, scale=1.0):
+    return (np.random.default_rng(seed).standard_normal(shape_) * scale).astype(np.float16)
+
+
+@pytest.mark.parametrize("shape,lens", [(GEMMA3_4B_GLOBAL, [1, 300, 2049]), (QWEN3_4B, [700, 5]), (SMOLLM2_135M, [1500])],
+                         ids=lambda v: getattr(v, "name", str(v)))
+def test_fp16_decode_attention_follows_the_oracle_and_ignores_the_segment_layout(shape, lens):
+    """fp16 q, K, V and output on both streaming kernels (fp32 pipes: Gemma shape; mma.sync: Qwen3 and SmolLM2
+    shapes): Eq. 6-7 against the fp64 oracle on the same fp16-valued inputs, and identical bits whether the keys
+    sit in one segment or in three."""
+    import math
+    batch = len(lens)
+    w = make_layer_weights(shape)
+    desc = kvd.make_desc(1, shape.d_hidden, shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.rms_eps,
+                         shape.qk_norm, shape.rms_eps, shape.rope_style, 1, 4096, batch)
+    ctx = kvd.Kvd(desc)
+    ctx.kvd_set_dtype(1)
+    ctx.kvd_set_layer(0, dev16(as_f16(w.w_kv)), dev16(as_f16(w.gamma_in)),
+                      dev16(as_f16(w.gamma_k)) if w.gamma_k is not None else None, shape.rope_theta, shape.sliding_window)
+    ws = torch.empty(kvd.kvd_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_workspace(ws)
+    kdim = shape.n_kv_heads * shape.d_head
+    q16 = rand_f16((batch, shape.n_q_heads, shape.d_head), 1)
+    q = dev16(q16)
+    Ks = [rand_f16((n, kdim), 10 + b) for b, n in enumerate(lens)]
+    Vs = [rand_f16((n, kdim), 20 + b) for b, n in enumerate(lens)]
+    kd, vd = [dev16(k) for k in Ks], [dev16(v) for v in Vs]
+    q_pos = [n - 1 for n in lens]
+    one = [[(kd[b], vd[b], kdim, 0, lens[b])] for b in range(batch)]
+    out1 = torch.zeros((batch, shape.n_q_heads, shape.d_head), dtype=torch.float16, device="cuda")
+    ctx.kvd_decode_attention(0, batch, q, q_pos, one, 0.0, out1)
+
+    def three(b):
+        n = lens[b]
+        a, c = n // 3, (2 * n) // 3
+        cuts = [(0, a), (a, c), (c, n)]
+        return [(kd[b][lo:], vd[b][lo:], kdim, lo, hi - lo) for lo, hi in cuts if hi > lo]
+    out3 = torch.zeros_like(out1)
+    ctx.kvd_decode_attention(0, batch, q, q_pos, [three(b) for b in range(batch)], 0.0, out3)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    assert torch.equal(out1.view(torch.int16), out3.view(torch.int16))
+    for b, n in enumerate(lens):
+        K = Ks[b].astype(np.float64).reshape(n, shape.n_kv_heads, shape.d_head)
+        V = Vs[b].astype(np.float64).reshape(n, shape.n_kv_heads, shape.d_head)
+        ref = oracle.decode_attention(q16[b].astype(np.float64), q_pos[b], [(K, V, 0)], 1.0 / math.sqrt(shape.d_head),
+                                      shape.sliding_window)
+        got = out1[b].cpu().numpy().astype(np.float64)
+        d = got - ref
+        assert np.linalg.norm(d) / np.linalg.norm(ref) <= 1e-2, b
+        assert np.max(np.abs(d)) <= 1e-2 * np.max(np.abs(ref)), b
+
+
+def test_fp16_context_is_refused_by_the_bf16_only_entry_points_and_the_type_is_fixed_once_used():
     shape = GEMMA3_4B_GLOBAL
     ctx, w16 = open_f16(shape, 256)
     with pytest.raises(kvd.KvdError) as e:        # a layer is set: too late to change the type
@@ -109,8 +162,47 @@ def test_fp16_context_is_refused_where_bf16_is_required_and_the_type_is_fixed_on
     ctx.kvd_attach_workspace(ws)
     kdim = shape.n_kv_heads * shape.d_head
     q = torch.zeros((1, shape.n_q_heads, shape.d_head), dtype=torch.float16, device="cuda")
-    k = torch.zeros((4, kdim), dtype=torch.float16, device="cuda")
-    with pytest.raises(kvd.KvdError) as e:
-        ctx.kvd_decode_attention(0, 1, q, [3], [[(k, k, kdim, 0, 4)]], 0.0, q)
+    with pytest.raises(kvd.KvdError) as e:        # the fused path reads bf16 queries and writes bf16
+        ctx.kvd_decode_attention_recompute(0, 1, q, [3], [(0, 0, 0)], None, None, 0, None, None, kdim, [[]], 0.0, q)
+    assert e.value.status == 6
+    x = torch.zeros((2, shape.d_hidden), dtype=torch.float16, device="cuda")
+    p = torch.zeros((2,), dtype=torch.int32, device="cuda")
+    arena = torch.zeros(kvd.kvd_store_bytes_fp8(ctx.desc, 1), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_store_fp8(arena, 1)
+    with pytest.raises(kvd.KvdError) as e:        # the quantiser reads bf16 rows
+        ctx.kvd_checkpoint_residual_fp8(0, 0, x, p, 2)
     assert e.value.status == 6
     assert ctx.kvd_poll_status() == kvd.KVD_OK
+
+
+def test_fp16_kvdirect_layer_equals_the_full_cache_layer_bit_for_bit():
+    """Section 5.1 in fp16, one layer: K/V of 300 tokens computed as a decode loop would (first pass), then the
+    first 250 evicted and rebuilt from their checkpointed rows; attention over [rebuilt] + [kept] + [current]
+    has the bits of attention over the first-pass cache."""
+    shape = GEMMA3_4B_GLOBAL
+    ctx, w16 = open_f16(shape, 512)
+    ws = torch.empty(kvd.kvd_workspace_bytes(ctx.desc), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_workspace(ws)
+    kdim = shape.n_kv_heads * shape.d_head
+    T, n_old = 300, 250
+    X16 = as_f16(make_residuals(shape, T, seed=91, outliers=True))
+    x, p = dev16(X16), torch.arange(T, dtype=torch.int32, device="cuda")
+    kc = torch.zeros((T, kdim), dtype=torch.float16, device="cuda")
+    vc = torch.zeros_like(kc)
+    ctx.kvd_recompute_kv(0, x[:200], p[:200], 200, kc, vc, kdim)            # "prefill"
+    for m in range(200, T):                                                  # "decode", one token at a time
+        ctx.kvd_recompute_kv(0, x[m:m + 1], p[m:m + 1], 1, kc[m:], vc[m:], kdim)
+    ctx.kvd_checkpoint_residual(0, 0, x[:n_old], p[:n_old], n_old)
+    kr = torch.zeros((n_old, kdim), dtype=torch.float16, device="cuda")
+    vr = torch.zeros_like(kr)
+    ctx.kvd_recompute_kv(0, None, None, n_old, kr, vr, kdim, seq=0, first_row=0)
+    q = dev16(rand_f16((1, shape.n_q_heads, shape.d_head), 5))
+    full = torch.zeros((1, shape.n_q_heads, shape.d_head), dtype=torch.float16, device="cuda")
+    kvdir = torch.zeros_like(full)
+    ctx.kvd_decode_attention(0, 1, q, [T - 1], [[(kc, vc, kdim, 0, T)]], 0.0, full)
+    ctx.kvd_decode_attention(0, 1, q, [T - 1], [[(kr, vr, kdim, 0, n_old), (kc[n_old:], vc[n_old:], kdim, n_old, T - 1 - n_old),
+                                                 (kc[T - 1:], vc[T - 1:], kdim, T - 1, 1)]], 0.0, kvdir)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    assert torch.equal(kr.view(torch.int16), kc[:n_old].view(torch.int16))
+    assert torch.equal(full.view(torch.int16), kvdir.view(torch.int16))
+    assert float(full.abs().max()) > 0
