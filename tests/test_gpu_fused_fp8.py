@@ -177,3 +177,25 @@ def test_fused_fp8_decode_loop_with_nothing_kept_crosses_a_block_boundary():
                                       1.0 / math.sqrt(shape.d_head), shape.sliding_window)
         attn_check(host_f64(out)[0], ref, f"step {t}")
     assert ctx.kvd_poll_status() == kvd.KVD_OK
+
+
+def test_fused_fp8_without_queries_only_stores_and_empty_call_launches_nothing():
+    shape = GEMMA3_4B_GLOBAL
+    ctx, w = open_layer(shape, max_tokens=512)
+    arena = torch.zeros(kvd.kvd_store_bytes_fp8(ctx.desc, 1), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_store_fp8(arena, 1)
+    kdim = shape.n_kv_heads * shape.d_head
+    n = 70
+    X = make_residuals(shape, n, seed=3, outliers=True)
+    x, p = dev(X), torch.arange(n, dtype=torch.int32, device="cuda")
+    ctx.kvd_checkpoint_residual_fp8(0, 0, x, p, n)
+    before = ctx.kvd_launch_count()
+    ctx.kvd_decode_attention_recompute_fp8(0, 0, None, [], [], [], kdim, [], 0.0, None)   # nothing to do
+    assert ctx.kvd_launch_count() == before
+    # batch 0 with ranges to store: the call is a plain FP8 recompute of those ranges
+    k1 = torch.zeros((n, kdim), dtype=torch.bfloat16, device="cuda"); v1 = torch.zeros_like(k1)
+    k2 = torch.zeros_like(k1); v2 = torch.zeros_like(k1)
+    ctx.kvd_decode_attention_recompute_fp8(0, 0, None, [], [], [(0, 0, n, k1, v1)], kdim, [], 0.0, None)
+    ctx.kvd_recompute_kv_fp8(0, [(0, 0, n, k2, v2)], kdim)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    assert torch.equal(k1, k2) and torch.equal(v1, v2) and float(k1.abs().max()) > 0
