@@ -133,13 +133,18 @@ void kvd_destroy(kvd_ctx *ctx);
 
 /* Element type of residual rows, weights, K/V, queries and attention outputs.  bf16 is the default and the
  * only type the fused, FP8 and static entry points accept (KVD_ERR_UNSUPPORTED otherwise); fp16 exists for
- * kvd_checkpoint_residual / kvd_recompute_kv / kvd_recompute_kv_step / kvd_decode_attention -- the
- * reconstruction identities (Eq. 13-14) do not depend on the element type, and the bitwise
- * recompute-equals-first-pass check of the paper's Section 5.1 is run in both.  Call before any
- * kvd_set_layer / checkpoint (KVD_ERR_STATE after). */
+ * kvd_checkpoint_residual / kvd_recompute_kv / kvd_recompute_kv_step / kvd_decode_attention, fp32 for the
+ * first three (rows, weights and K/V outputs are fp32, strides count fp32 elements, the tensor cores read the
+ * operands as TF32 and accumulate in fp32) -- the reconstruction identities (Eq. 13-14) do not depend on the
+ * element type, and the bitwise recompute-equals-first-pass check of the paper's Section 5.1 is run in all
+ * three.  Call before kvd_set_layer, kvd_attach_store (when the element size changes) and any checkpoint
+ * (KVD_ERR_STATE after). */
 #define KVD_DTYPE_BF16 0
 #define KVD_DTYPE_F16 1
+#define KVD_DTYPE_F32 2
 kvd_status kvd_set_dtype(kvd_ctx *ctx, int dtype);
+/* kvd_store_bytes for a context of the given element type (fp32 rows take twice the room). */
+size_t kvd_store_bytes_dtype(const kvd_model_desc *desc, int layers_stored, int dtype);
 
 /* Prepare layer `layer`: build W' = diag(gamma_in) * W_kv rounded to bf16 and stored K-major, the
  * fp32 key-norm scale, and the rotation tables for rope_theta.  Folding gamma into W is Eq. 1

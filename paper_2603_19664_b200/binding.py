@@ -31,7 +31,7 @@ KVD_MAX_SEGMENTS = 4
 # every symbol include/kvd.h declares
 EXPORTED_SYMBOLS = (
     "kvd_create", "kvd_destroy", "kvd_set_layer", "kvd_store_bytes", "kvd_attach_store", "kvd_reset_sequence",
-    "kvd_decode_attention_recompute", "kvd_decode_attention_recompute_fp8", "kvd_set_dtype",
+    "kvd_decode_attention_recompute", "kvd_decode_attention_recompute_fp8", "kvd_set_dtype", "kvd_store_bytes_dtype",
     "kvd_store_bytes_fp8", "kvd_attach_store_fp8", "kvd_rows_stored_fp8", "kvd_reset_sequence_fp8", "kvd_checkpoint_residual_fp8", "kvd_recompute_kv_fp8",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
     "kvd_recompute_kv_step",
@@ -100,6 +100,8 @@ def load() -> ctypes.CDLL:
     lib.kvd_set_layer.restype = i32
     lib.kvd_store_bytes.argtypes = [ctypes.POINTER(kvd_model_desc), i32]
     lib.kvd_store_bytes.restype = sz
+    lib.kvd_store_bytes_dtype.argtypes = [ctypes.POINTER(kvd_model_desc), i32, i32]
+    lib.kvd_store_bytes_dtype.restype = sz
     lib.kvd_attach_store.argtypes = [vp, vp, sz, i32]
     lib.kvd_attach_store.restype = i32
     lib.kvd_reset_sequence.argtypes = [vp, i32]
@@ -184,6 +186,10 @@ def make_desc(n_layers: int, d_hidden: int, n_q_heads: int, n_kv_heads: int, d_h
 
 def kvd_store_bytes(desc: kvd_model_desc, layers_stored: int) -> int:
     return int(load().kvd_store_bytes(ctypes.byref(desc), layers_stored))
+
+
+def kvd_store_bytes_dtype(desc: kvd_model_desc, layers_stored: int, dtype: int) -> int:
+    return int(load().kvd_store_bytes_dtype(ctypes.byref(desc), layers_stored, dtype))
 
 
 def kvd_store_bytes_fp8(desc: kvd_model_desc, layers_stored: int) -> int:
@@ -372,7 +378,8 @@ class Kvd:
             float(scale), _ptr(out), _stream(stream)), "kvd_decode_attention_recompute_fp8")
 
     def kvd_set_dtype(self, dtype: int) -> None:
-        """0 = bf16 (default), 1 = fp16 (checkpoint, recompute and kvd_decode_attention); before any kvd_set_layer."""
+        """0 = bf16 (default), 1 = fp16 (checkpoint, recompute and kvd_decode_attention), 2 = fp32 (checkpoint and
+        recompute); before kvd_set_layer and kvd_attach_store."""
         self._check(self._lib.kvd_set_dtype(self._h, dtype), "kvd_set_dtype")
 
     def kvd_attach_store_fp8(self, arena, layers_stored: int) -> None:

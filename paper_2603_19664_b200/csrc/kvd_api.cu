@@ -62,11 +62,18 @@ extern "C" const char *kvd_status_string(kvd_status s) {
   return "unknown status";
 }
 
-extern "C" size_t kvd_store_bytes(const kvd_model_desc *d, int layers_stored) {
+static inline int dtype_bytes(int dtype) { return dtype == KVD_DTYPE_F32 ? 4 : 2; }
+
+extern "C" size_t kvd_store_bytes_dtype(const kvd_model_desc *d, int layers_stored, int dtype) {
   if (check_desc(d) != KVD_OK || layers_stored <= 0) return 0;
+  if (dtype != KVD_DTYPE_BF16 && dtype != KVD_DTYPE_F16 && dtype != KVD_DTYPE_F32) return 0;
   const size_t slots = static_cast<size_t>(layers_stored) * d->max_seqs * d->max_tokens_per_seq;
   // rows, then positions, then the rows' sums of squares, each region starting at a 256-byte multiple
-  return round_up(slots * d->d_hidden * 2, 256) + 2 * round_up(slots * 4, 256);
+  return round_up(slots * d->d_hidden * dtype_bytes(dtype), 256) + 2 * round_up(slots * 4, 256);
+}
+
+extern "C" size_t kvd_store_bytes(const kvd_model_desc *d, int layers_stored) {
+  return kvd_store_bytes_dtype(d, layers_stored, KVD_DTYPE_BF16);
 }
 
 // chunk partials of one sequence
@@ -173,7 +180,7 @@ static kvd_status encode_2d(kvd_ctx *ctx, CUtensorMap *map, const void *base, ui
   cuuint64_t strides[1] = {inner * eb};
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = ctx->encode(map, eb == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
+  CUresult r = ctx->encode(map, eb == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : eb == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
                            const_cast<void *>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -193,7 +200,7 @@ static kvd_status encode_rows_3d(kvd_ctx *ctx, CUtensorMap *map, const void *bas
   cuuint64_t strides[2] = {d_hidden * eb, rows * d_hidden * eb};
   cuuint32_t box[3] = {static_cast<cuuint32_t>(RC_BLOCK_K * 2 / eb), RC_BLOCK_M, 1};
   cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = ctx->encode(map, eb == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 3,
+  CUresult r = ctx->encode(map, eb == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : eb == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 3,
                            const_cast<void *>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -245,9 +252,10 @@ static kvd_status get_rope(kvd_ctx *ctx, float theta, RopeTable *out) {
 }
 
 extern "C" kvd_status kvd_set_dtype(kvd_ctx *ctx, int dtype) {
-  if (!ctx || (dtype != KVD_DTYPE_BF16 && dtype != KVD_DTYPE_F16)) return KVD_ERR_INVALID_ARG;
+  if (!ctx || (dtype != KVD_DTYPE_BF16 && dtype != KVD_DTYPE_F16 && dtype != KVD_DTYPE_F32)) return KVD_ERR_INVALID_ARG;
   for (const LayerState &l : ctx->layers)
     if (l.set) return KVD_ERR_STATE;  // weights are prepared in the element type: choose it first
+  if (ctx->store_rows && dtype_bytes(dtype) != dtype_bytes(ctx->dtype)) return KVD_ERR_STATE;  // the store is laid out for it
   for (int c : ctx->rows_stored)
     if (c != 0) return KVD_ERR_STATE;
   ctx->dtype = dtype;
@@ -267,9 +275,9 @@ extern "C" kvd_status kvd_set_layer(kvd_ctx *ctx, int layer, const kvd_layer_des
   LayerState &ls = ctx->layers[layer];
   cudaError_t e;
   if (!ls.wt) {
-    e = cudaMalloc(&ls.wt, static_cast<size_t>(n_cols) * d.d_hidden * 2);
+    e = cudaMalloc(&ls.wt, static_cast<size_t>(n_cols) * d.d_hidden * dtype_bytes(ctx->dtype));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMalloc(prepared weights)");
-    ctx->prepared_bytes += static_cast<size_t>(n_cols) * d.d_hidden * 2;
+    ctx->prepared_bytes += static_cast<size_t>(n_cols) * d.d_hidden * dtype_bytes(ctx->dtype);
   }
   if (d.qk_norm && !ls.gamma_k) {
     e = cudaMalloc(&ls.gamma_k, d.d_head * sizeof(float));
@@ -286,7 +294,9 @@ extern "C" kvd_status kvd_set_layer(kvd_ctx *ctx, int layer, const kvd_layer_des
   }
   st = get_rope(ctx, ld->rope_theta, &ls.rope);
   if (st != KVD_OK) return st;
-  st = encode_2d(ctx, &ls.tmap_b, ls.wt, d.d_hidden, n_cols, RC_BLOCK_K, ctx->block_n / 2);  // half tile per CTA
+  // half tile per CTA, 128 bytes of channels per k block
+  st = encode_2d(ctx, &ls.tmap_b, ls.wt, d.d_hidden, n_cols, RC_BLOCK_K * 2 / dtype_bytes(ctx->dtype), ctx->block_n / 2,
+                 dtype_bytes(ctx->dtype));
   if (st != KVD_OK) return st;
   // the FP8 variant's copy of W' (E4M3 codes and one scale); rows of d_hidden bytes must be TMA-addressable
   if (d.d_hidden % 16 == 0 && ctx->dtype == KVD_DTYPE_BF16) {
@@ -315,19 +325,20 @@ extern "C" kvd_status kvd_set_layer(kvd_ctx *ctx, int layer, const kvd_layer_des
 extern "C" kvd_status kvd_attach_store(kvd_ctx *ctx, void *arena, size_t bytes, int layers_stored) {
   if (!ctx || !arena || layers_stored <= 0 || layers_stored > ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(arena) & 255u) != 0) return KVD_ERR_ALIGNMENT;
-  const size_t need = kvd_store_bytes(&ctx->desc, layers_stored);
+  const size_t need = kvd_store_bytes_dtype(&ctx->desc, layers_stored, ctx->dtype);
   if (bytes < need) return KVD_ERR_CAPACITY;
   const kvd_model_desc &d = ctx->desc;
+  const int es = dtype_bytes(ctx->dtype), ew = es / 2;  // store_rows counts 16-bit units
   const size_t slots = static_cast<size_t>(layers_stored) * d.max_seqs * d.max_tokens_per_seq;
   ctx->store_rows = static_cast<__nv_bfloat16 *>(arena);
-  ctx->store_pos = reinterpret_cast<int32_t *>(static_cast<uint8_t *>(arena) + round_up(slots * d.d_hidden * 2, 256));
+  ctx->store_pos = reinterpret_cast<int32_t *>(static_cast<uint8_t *>(arena) + round_up(slots * d.d_hidden * es, 256));
   ctx->store_sumsq = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(ctx->store_pos) + round_up(slots * 4, 256));
   ctx->layers_stored = layers_stored;
   ctx->rows_stored.assign(static_cast<size_t>(layers_stored) * d.max_seqs, 0);
   ctx->store_maps.resize(layers_stored);
   for (int l = 0; l < layers_stored; ++l) {
-    const __nv_bfloat16 *base = ctx->store_rows + static_cast<size_t>(l) * d.max_seqs * d.max_tokens_per_seq * d.d_hidden;
-    kvd_status st = encode_rows_3d(ctx, &ctx->store_maps[l], base, d.d_hidden, d.max_tokens_per_seq, d.max_seqs);
+    const __nv_bfloat16 *base = ctx->store_rows + static_cast<size_t>(l) * d.max_seqs * d.max_tokens_per_seq * d.d_hidden * ew;
+    kvd_status st = encode_rows_3d(ctx, &ctx->store_maps[l], base, d.d_hidden, d.max_tokens_per_seq, d.max_seqs, es);
     if (st != KVD_OK) {
       ctx->store_rows = nullptr;
       ctx->layers_stored = 0;
@@ -388,7 +399,7 @@ extern "C" kvd_status kvd_checkpoint_residual(kvd_ctx *ctx, int seq, int layer, 
   if (count + n > ctx->desc.max_tokens_per_seq) return KVD_ERR_CAPACITY;
   const size_t slot = store_slot(ctx, layer, seq) + count;
   kvd_status st = launch_checkpoint(ctx, static_cast<const __nv_bfloat16 *>(rows), positions,
-                                    ctx->store_rows + slot * ctx->desc.d_hidden, ctx->store_pos + slot,
+                                    ctx->store_rows + slot * ctx->desc.d_hidden * (dtype_bytes(ctx->dtype) / 2), ctx->store_pos + slot,
                                     ctx->store_sumsq + slot, n, ctx->desc.d_hidden, static_cast<cudaStream_t>(stream_));
   if (st == KVD_OK) count += n;
   return st;
@@ -419,9 +430,9 @@ static void fill_launch_params(const kvd_ctx *ctx, const LayerState &ls, Recompu
   p.trace = nullptr;
   p.ext_rows = nullptr;
   p.w_scale = nullptr;
-  p.row_chunks = d.d_hidden / 8;
+  p.row_chunks = d.d_hidden * dtype_bytes(ctx->dtype) / 16;
   // 32-byte stores need every output row 32-byte aligned
-  p.wide_store = out_row_stride % 16 == 0;
+  p.wide_store = out_row_stride * dtype_bytes(ctx->dtype) % 32 == 0;
   for (int i = 0; i < n_jobs; ++i)
     if (((reinterpret_cast<uintptr_t>(p.jobs[i].k_out) | reinterpret_cast<uintptr_t>(p.jobs[i].v_out)) & 31u) != 0) p.wide_store = 0;
 }
@@ -437,8 +448,9 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
   const LayerState &ls = ctx->layers[layer];
   const kvd_model_desc &d = ctx->desc;
   const int kdim = d.n_kv_heads * d.d_head;
+  const int es = dtype_bytes(ctx->dtype);
   if (out_row_stride < kdim) return KVD_ERR_INVALID_ARG;
-  if (out_row_stride % 8 != 0) return KVD_ERR_ALIGNMENT;
+  if (out_row_stride * es % 16 != 0) return KVD_ERR_ALIGNMENT;
   RecomputeParams p;
   static thread_local FusedParams fp;  // large: keep it off the stack
   int n_jobs = 0, mb = 0;
@@ -474,7 +486,7 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
   if (n_rows > 0) {
     if (!rows || !positions || !k_rows_out || !v_rows_out) return KVD_ERR_INVALID_ARG;
     if (!aligned16(rows) || !aligned16(k_rows_out) || !aligned16(v_rows_out)) return KVD_ERR_ALIGNMENT;
-    kvd_status st = encode_rows_3d(ctx, &tmap_rows, rows, d.d_hidden, static_cast<uint64_t>(n_rows), 1);
+    kvd_status st = encode_rows_3d(ctx, &tmap_rows, rows, d.d_hidden, static_cast<uint64_t>(n_rows), 1, es);
     if (st != KVD_OK) return st;
     if (fused) fp.att[n_jobs].q = nullptr;  // the caller's rows are stored
     RcJob &J = p.jobs[n_jobs++];
@@ -501,7 +513,7 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
   // the kernel is handed both maps; an unused one aliases the other
   const CUtensorMap &tmap_store = any_store ? ctx->store_maps[layer] : tmap_rows;
   const CUtensorMap &tmap_ext = n_rows > 0 ? tmap_rows : ctx->store_maps[layer];
-  fill_launch_params(ctx, ls, p, n_jobs, mb, d.d_hidden / RC_BLOCK_K, out_row_stride);
+  fill_launch_params(ctx, ls, p, n_jobs, mb, d.d_hidden * es / (2 * RC_BLOCK_K), out_row_stride);  // 128 bytes per k block
   p.ext_rows = static_cast<const __nv_bfloat16 *>(rows);
   if (ctx->trace) {
     const int tiles = p.num_m_blocks * p.num_n_blocks;
@@ -782,6 +794,7 @@ extern "C" kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, c
   const LayerState &ls = ctx->layers[layer];
   if (!ls.set) return KVD_ERR_STATE;
   if (!ctx->part_o) return KVD_ERR_STATE;
+  if (ctx->dtype == KVD_DTYPE_F32) return KVD_ERR_UNSUPPORTED;  // attention reads 16-bit K/V
   if (batch == 0) return KVD_OK;
   if (!q || !q_pos || !out || (n_segs > 0 && !segs)) return KVD_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(out)) return KVD_ERR_ALIGNMENT;
@@ -918,8 +931,8 @@ extern "C" kvd_status kvd_memory_stats(const kvd_ctx *ctx, kvd_mem_stats *out) {
     rows_total += layer_rows;
     if (layer_rows > tokens) tokens = layer_rows;
   }
-  out->checkpoint_bytes_used = rows_total * (static_cast<uint64_t>(d.d_hidden) * 2 + 8);  // row, position, sum of squares
-  out->checkpoint_bytes_capacity = ctx->layers_stored > 0 ? kvd_store_bytes(&d, ctx->layers_stored) : 0;
+  out->checkpoint_bytes_used = rows_total * (static_cast<uint64_t>(d.d_hidden) * dtype_bytes(ctx->dtype) + 8);  // row, position, sum of squares
+  out->checkpoint_bytes_capacity = ctx->layers_stored > 0 ? kvd_store_bytes_dtype(&d, ctx->layers_stored, ctx->dtype) : 0;
   // the FP8 store counts too: codes, position, sum of squares, scale
   uint64_t rows8 = 0;
   for (int l = 0; l < ctx->layers_stored8; ++l) {
@@ -933,9 +946,9 @@ extern "C" kvd_status kvd_memory_stats(const kvd_ctx *ctx, kvd_mem_stats *out) {
   out->workspace_bytes = ctx->workspace_bytes;
   out->prepared_weight_bytes = ctx->prepared_bytes;
   out->tokens_stored = tokens;
-  out->eq23_kv_bytes_per_token = 2ull * d.n_layers * d.n_kv_heads * d.d_head * 2;
-  out->eq24_residual_bytes_per_token = static_cast<uint64_t>(d.d_hidden) * 2;
-  out->per_layer_residual_bytes_per_token = static_cast<uint64_t>(d.n_layers) * d.d_hidden * 2;
+  out->eq23_kv_bytes_per_token = 2ull * d.n_layers * d.n_kv_heads * d.d_head * dtype_bytes(ctx->dtype);
+  out->eq24_residual_bytes_per_token = static_cast<uint64_t>(d.d_hidden) * dtype_bytes(ctx->dtype);
+  out->per_layer_residual_bytes_per_token = static_cast<uint64_t>(d.n_layers) * d.d_hidden * dtype_bytes(ctx->dtype);
   return KVD_OK;
 }
 

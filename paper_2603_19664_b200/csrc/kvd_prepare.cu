@@ -6,25 +6,35 @@
 
 namespace kvd {
 
-// a 16-bit element (bf16 or fp16 bits) as float, and back (round to nearest even)
+// an element (bf16, fp16 or fp32 bits) as float, and back (round to nearest even)
 template <int DT>
-__device__ __forceinline__ float elem_to_float(uint16_t bits) {
+struct ElemBits {
+  typedef uint16_t type;
+};
+template <>
+struct ElemBits<2> {
+  typedef uint32_t type;
+};
+template <int DT>
+__device__ __forceinline__ float elem_to_float(typename ElemBits<DT>::type bits) {
   if constexpr (DT == 0) return __uint_as_float(static_cast<uint32_t>(bits) << 16);
-  else return __half2float(__ushort_as_half(bits));
+  else if constexpr (DT == 1) return __half2float(__ushort_as_half(bits));
+  else return __uint_as_float(bits);
 }
 template <int DT>
-__device__ __forceinline__ uint16_t float_to_elem(float v) {
+__device__ __forceinline__ typename ElemBits<DT>::type float_to_elem(float v) {
   if constexpr (DT == 0) return __bfloat16_as_ushort(__float2bfloat16_rn(v));
-  else return __half_as_ushort(__float2half_rn(v));
+  else if constexpr (DT == 1) return __half_as_ushort(__float2half_rn(v));
+  else return __float_as_uint(v);
 }
 
 // wt[n][k] = bf16( gamma[k] * w[k][n] ): fold the RMSNorm scale of Eq. 1 into the projection of
 // Eq. 13-14 and store the result K-major so that both GEMM operands are read along d_hidden.
 template <int DT>
-__global__ void __launch_bounds__(256) kvd_prepare_weights_kernel(const uint16_t *__restrict__ w,
-                                                                  const uint16_t *__restrict__ gamma,
-                                                                  uint16_t *__restrict__ wt, int d_hidden,
-                                                                  int n_cols) {
+__global__ void __launch_bounds__(256) kvd_prepare_weights_kernel(const typename ElemBits<DT>::type *__restrict__ w,
+                                                                  const typename ElemBits<DT>::type *__restrict__ gamma,
+                                                                  typename ElemBits<DT>::type *__restrict__ wt,
+                                                                  int d_hidden, int n_cols) {
   __shared__ float tile[32][33];
   const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // 32 x 8
@@ -43,7 +53,7 @@ __global__ void __launch_bounds__(256) kvd_prepare_weights_kernel(const uint16_t
 }
 
 template <int DT>
-__global__ void kvd_convert_gamma_kernel(const uint16_t *__restrict__ g, float *__restrict__ out, int n) {
+__global__ void kvd_convert_gamma_kernel(const typename ElemBits<DT>::type *__restrict__ g, float *__restrict__ out, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) out[i] = elem_to_float<DT>(g[i]);
 }
@@ -251,7 +261,10 @@ kvd_status launch_prepare_weights(kvd_ctx *ctx, const __nv_bfloat16 *w, const __
   dim3 grid((n_cols + 31) / 32, (d_hidden + 31) / 32);
   const uint16_t *w16 = reinterpret_cast<const uint16_t *>(w), *g16 = reinterpret_cast<const uint16_t *>(gamma);
   uint16_t *wt16 = reinterpret_cast<uint16_t *>(wt);
-  if (ctx->dtype == 1) kvd_prepare_weights_kernel<1><<<grid, 256, 0, stream>>>(w16, g16, wt16, d_hidden, n_cols);
+  if (ctx->dtype == 2)
+    kvd_prepare_weights_kernel<2><<<grid, 256, 0, stream>>>(reinterpret_cast<const uint32_t *>(w), reinterpret_cast<const uint32_t *>(gamma),
+                                                            reinterpret_cast<uint32_t *>(wt), d_hidden, n_cols);
+  else if (ctx->dtype == 1) kvd_prepare_weights_kernel<1><<<grid, 256, 0, stream>>>(w16, g16, wt16, d_hidden, n_cols);
   else kvd_prepare_weights_kernel<0><<<grid, 256, 0, stream>>>(w16, g16, wt16, d_hidden, n_cols);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "launch prepare_weights");
@@ -261,7 +274,8 @@ kvd_status launch_prepare_weights(kvd_ctx *ctx, const __nv_bfloat16 *w, const __
 
 kvd_status launch_convert_gamma(kvd_ctx *ctx, const __nv_bfloat16 *g, float *out, int n, cudaStream_t stream) {
   const uint16_t *g16 = reinterpret_cast<const uint16_t *>(g);
-  if (ctx->dtype == 1) kvd_convert_gamma_kernel<1><<<(n + 127) / 128, 128, 0, stream>>>(g16, out, n);
+  if (ctx->dtype == 2) kvd_convert_gamma_kernel<2><<<(n + 127) / 128, 128, 0, stream>>>(reinterpret_cast<const uint32_t *>(g), out, n);
+  else if (ctx->dtype == 1) kvd_convert_gamma_kernel<1><<<(n + 127) / 128, 128, 0, stream>>>(g16, out, n);
   else kvd_convert_gamma_kernel<0><<<(n + 127) / 128, 128, 0, stream>>>(g16, out, n);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "launch convert_gamma");
@@ -275,7 +289,10 @@ kvd_status launch_checkpoint(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int3
   const long long cap = static_cast<long long>(ctx->num_sms) * 8;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  if (ctx->dtype == 1)
+  if (ctx->dtype == 2)
+    kvd_checkpoint_kernel<2><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+        reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint4 *>(dst_rows), dst_pos, dst_sumsq, d_hidden / 4, n);
+  else if (ctx->dtype == 1)
     kvd_checkpoint_kernel<1><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
         reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint4 *>(dst_rows), dst_pos, dst_sumsq, d_hidden / 8, n);
   else
@@ -293,7 +310,10 @@ kvd_status launch_rowstats(kvd_ctx *ctx, const __nv_bfloat16 *rows, float *sumsq
   const long long cap = static_cast<long long>(ctx->num_sms) * 8;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  if (ctx->dtype == 1)
+  if (ctx->dtype == 2)
+    kvd_rowstats_kernel<2><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(reinterpret_cast<const uint4 *>(rows), sumsq,
+                                                                              d_hidden / 4, n);
+  else if (ctx->dtype == 1)
     kvd_rowstats_kernel<1><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(reinterpret_cast<const uint4 *>(rows), sumsq,
                                                                               d_hidden / 8, n);
   else

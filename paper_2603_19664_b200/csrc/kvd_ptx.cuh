@@ -284,6 +284,11 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(int m, int n) {
 __host__ __device__ constexpr uint32_t umma_idesc_f16_f32(int m, int n) {
   return (1u << 4) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
 }
+// kind::tf32 with fp32 operands read as TF32 (format code 2 in both fields).
+__host__ __device__ constexpr uint32_t umma_idesc_tf32_f32(int m, int n) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>(m >> 4) << 24);
+}
 // The same for kind::f8f6f4 with E4M3 A and B (format code 0 in both fields).
 __host__ __device__ constexpr uint32_t umma_idesc_e4m3_f32(int m, int n) {
   return (1u << 4) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
@@ -320,8 +325,9 @@ __device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
 // the two bf16 halves of a 32-bit word as a packed pair of fp32
 __device__ __forceinline__ uint64_t bf16x2_to_f32x2(uint32_t w) { return pack2(bf16_lo(w), bf16_hi(w)); }
 
-// 16-bit element type of rows, weights, K/V and outputs: DT = 0 bf16 (the default everywhere), DT = 1 fp16
-// (checkpoint, recompute and decode attention: the dtype-invariance check of the paper's Section 5.1)
+// Element type of rows, weights, K/V and outputs: DT = 0 bf16 (the default everywhere), DT = 1 fp16
+// (checkpoint, recompute and decode attention), DT = 2 fp32 (checkpoint and recompute; the tensor cores read
+// the operands as TF32): the dtype-invariance check of the paper's Section 5.1
 template <int DT>
 __device__ __forceinline__ uint64_t x2_to_f32x2(uint32_t w) {
   if constexpr (DT == 0) {
@@ -329,6 +335,19 @@ __device__ __forceinline__ uint64_t x2_to_f32x2(uint32_t w) {
   } else {
     const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w));
     return pack2(f.x, f.y);
+  }
+}
+// Two neighbouring outputs into the word array of a row piece: one packed word for the 16-bit types, two
+// words for fp32.
+template <int DT>
+__device__ __forceinline__ uint32_t pack_out(float lo, float hi);
+template <int DT>
+__device__ __forceinline__ void emit_pair(uint32_t *o, int j, float lo, float hi) {
+  if constexpr (DT == 2) {
+    o[2 * j] = __float_as_uint(lo);
+    o[2 * j + 1] = __float_as_uint(hi);
+  } else {
+    o[j] = pack_out<DT>(lo, hi);
   }
 }
 template <int DT>
@@ -351,6 +370,11 @@ __device__ __forceinline__ uint32_t pack_out(float lo, float hi) {
 template <int DT = 0>
 __device__ __forceinline__ void sumsq_chunk(uint64_t (&ps2)[4], const uint4 &v) {
   uint64_t x2;
+  if constexpr (DT == 2) {  // four fp32 values per chunk: two of the four two-wide chains are used
+    x2 = pack2(__uint_as_float(v.x), __uint_as_float(v.y)); ps2[0] = ffma2(x2, x2, ps2[0]);
+    x2 = pack2(__uint_as_float(v.z), __uint_as_float(v.w)); ps2[1] = ffma2(x2, x2, ps2[1]);
+    return;
+  }
   x2 = x2_to_f32x2<DT>(v.x); ps2[0] = ffma2(x2, x2, ps2[0]);
   x2 = x2_to_f32x2<DT>(v.y); ps2[1] = ffma2(x2, x2, ps2[1]);
   x2 = x2_to_f32x2<DT>(v.z); ps2[2] = ffma2(x2, x2, ps2[2]);

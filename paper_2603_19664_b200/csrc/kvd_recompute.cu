@@ -175,6 +175,7 @@ __device__ __forceinline__ void NAME(uint32_t d_tmem, uint32_t a_lo, uint32_t b_
 }
 KVD_DEFINE_UMMA_KBLOCK(umma_kblock_pair, "f16")        // bf16 operands: 64 channels = four K=16 steps
 KVD_DEFINE_UMMA_KBLOCK(umma_kblock_pair_f8, "f8f6f4")  // E4M3 operands: 128 channels = four K=32 steps
+KVD_DEFINE_UMMA_KBLOCK(umma_kblock_pair_tf32, "tf32")  // fp32 operands read as TF32: 32 channels = four K=8 steps
 #undef KVD_DEFINE_UMMA_KBLOCK
 
 // Output stores.  Each epilogue thread owns one row, so the 32 lanes of a store instruction write 32
@@ -212,7 +213,9 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   using Cfg = RcCfg<BLOCK_N, D_HEAD, FG, LOSM>;
   constexpr int STAGES = Cfg::STAGES;
   constexpr bool FUSED = FG > 0;
-  static_assert(DT == 0 || (FG == 0 && EB == 2), "fp16 exists for the plain bf16-sized variant only");
+  static_assert(DT == 0 || (FG == 0 && ((DT == 1 && EB == 2) || (DT == 2 && EB == 4))),
+                "fp16 and fp32 exist for the plain variant only");
+  constexpr int EW = DT == 2 ? 2 : 1;  // 16-bit units per output element (output pointers count 16-bit units)
   constexpr int KB_ELEMS = RC_BLOCK_K * 2 / EB;  // channels per k block
   static_assert(BLOCK_N % D_HEAD == 0, "a tile must hold whole heads");
 
@@ -419,6 +422,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
     if (lane == 0 && cta_rank == 0) {
       // ---------------------------------------------------------------- MMA issuer (even CTA)
       constexpr uint32_t idesc = EB == 1   ? umma_idesc_e4m3_f32(2 * RC_BLOCK_M, BLOCK_N)
+                                 : EB == 4 ? umma_idesc_tf32_f32(2 * RC_BLOCK_M, BLOCK_N)
                                  : DT == 1 ? umma_idesc_f16_f32(2 * RC_BLOCK_M, BLOCK_N)
                                            : umma_idesc_bf16_f32(2 * RC_BLOCK_M, BLOCK_N);
       // descriptor words for 128-byte-swizzled K-major tiles: low = start address >> 4 | LBO field (1),
@@ -460,6 +464,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
           tc_fence_after();
           if (EB == 1 && FUSED && swap_ab) umma_kblock_pair_f8(d_tmem, a_lo + b_off_units, a_lo, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
           else if (EB == 1) umma_kblock_pair_f8(d_tmem, a_lo, a_lo + b_off_units, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
+          else if (EB == 4) umma_kblock_pair_tf32(d_tmem, a_lo, a_lo + b_off_units, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
           else if (FUSED && swap_ab) umma_kblock_pair(d_tmem, a_lo + b_off_units, a_lo, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
           else umma_kblock_pair(d_tmem, a_lo, a_lo + b_off_units, desc_hi, idesc, kb != 0 ? 1u : 0u, empty);
           full += 8u;
@@ -710,21 +715,21 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
         const uint32_t tcol = acc + hh * D_HEAD;
         if (col0 >= p.k_cols) {
           // ---- value head (Eq. 14): scale by 1/rms and store
-          __nv_bfloat16 *dst = J.v_out + static_cast<size_t>(m) * p.out_row_stride + (col0 - p.k_cols);
+          __nv_bfloat16 *dst = J.v_out + (static_cast<size_t>(m) * p.out_row_stride + (col0 - p.k_cols)) * EW;
 #pragma unroll 1
           for (int c = 0; c < D_HEAD / 32; ++c) {
             uint32_t r[32];
             tmem_ld_x32(tcol + c * 32, r);
             tmem_wait_ld();
-            uint32_t o[16];
+            uint32_t o[16 * EW];
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-              o[j] = pack_out<DT>(__uint_as_float(r[2 * j]) * rstd, __uint_as_float(r[2 * j + 1]) * rstd);
-            if (valid) store_row_piece<4>(dst + c * 32, o, wide);
+              emit_pair<DT>(o, j, __uint_as_float(r[2 * j]) * rstd, __uint_as_float(r[2 * j + 1]) * rstd);
+            if (valid) store_row_piece<4 * EW>(dst + c * 32 * EW, o, wide);
           }
         } else {
           // ---- key head (Eq. 13): 1/rms, optional key norm, rotation R_pos
-          __nv_bfloat16 *dst = J.k_out + static_cast<size_t>(m) * p.out_row_stride + col0;
+          __nv_bfloat16 *dst = J.k_out + (static_cast<size_t>(m) * p.out_row_stride + col0) * EW;
           float kscale = rstd;
           // fused, attending job: the rotated key (rounded to bf16 like a stored one) is not written but
           // multiplied with the NG queries of this KV head (Eq. 6); two-wide partial sums per query
@@ -773,7 +778,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
               uint32_t r[16];
               tmem_ld_x16(tcol + c * 16, r);
               tmem_wait_ld();
-              uint32_t o[8];
+              uint32_t o[8 * EW];
 #pragma unroll
               for (int j = 0; j < 8; j += 2) {
                 const int i = c * 8 + j;  // pairs i and i + 1
@@ -785,8 +790,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
                 const float b0 = __uint_as_float(r[2 * j + 1]) * kscale * s_gamma_k[c * 16 + 2 * j + 1];
                 const float a1 = __uint_as_float(r[2 * j + 2]) * kscale * s_gamma_k[c * 16 + 2 * j + 2];
                 const float b1 = __uint_as_float(r[2 * j + 3]) * kscale * s_gamma_k[c * 16 + 2 * j + 3];
-                o[j] = pack_out<DT>(fmaf(a0, c0, -b0 * s0), fmaf(a0, s0, b0 * c0));
-                o[j + 1] = pack_out<DT>(fmaf(a1, c1, -b1 * s1), fmaf(a1, s1, b1 * c1));
+                emit_pair<DT>(o, j, fmaf(a0, c0, -b0 * s0), fmaf(a0, s0, b0 * c0));
+                emit_pair<DT>(o, j + 1, fmaf(a1, c1, -b1 * s1), fmaf(a1, s1, b1 * c1));
               }
               if (FUSED && attend) {
 #pragma unroll
@@ -797,7 +802,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
                   for (int w = 0; w < 8; ++w) sdot[g] = ffma2(bf16x2_to_f32x2(o[w]), bf16x2_to_f32x2(qw[w]), sdot[g]);
                 }
               } else if (valid) {
-                store_row_piece<2>(dst + c * 16, o, wide);
+                store_row_piece<2 * EW>(dst + c * 16 * EW, o, wide);
               }
             }
           } else {
@@ -817,7 +822,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
               tmem_ld_x16(tcol + c * 16, ra);
               tmem_ld_x16(tcol + HALF + c * 16, rb);
               tmem_wait_ld();
-              uint32_t oa[8], ob[8];
+              uint32_t oa[8 * EW], ob[8 * EW];
 #pragma unroll
               for (int j = 0; j < 16; j += 2) {
                 const int i = c * 16 + j;  // pairs (i, i + HALF) and (i + 1, i + 1 + HALF)
@@ -829,8 +834,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
                 const float b0 = __uint_as_float(rb[j]) * kscale * s_gamma_k[i + HALF];
                 const float a1 = __uint_as_float(ra[j + 1]) * kscale * s_gamma_k[i + 1];
                 const float b1 = __uint_as_float(rb[j + 1]) * kscale * s_gamma_k[i + 1 + HALF];
-                oa[j >> 1] = pack_out<DT>(fmaf(a0, c0, -b0 * s0), fmaf(a1, c1, -b1 * s1));
-                ob[j >> 1] = pack_out<DT>(fmaf(a0, s0, b0 * c0), fmaf(a1, s1, b1 * c1));
+                emit_pair<DT>(oa, j >> 1, fmaf(a0, c0, -b0 * s0), fmaf(a1, c1, -b1 * s1));
+                emit_pair<DT>(ob, j >> 1, fmaf(a0, s0, b0 * c0), fmaf(a1, s1, b1 * c1));
               }
               if (FUSED && attend) {
 #pragma unroll
@@ -846,8 +851,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
                   }
                 }
               } else if (valid) {
-                store_row_piece<2>(dst + c * 16, oa, wide);
-                store_row_piece<2>(dst + HALF + c * 16, ob, wide);
+                store_row_piece<2 * EW>(dst + c * 16 * EW, oa, wide);
+                store_row_piece<2 * EW>(dst + (HALF + c * 16) * EW, ob, wide);
               }
             }
           }
@@ -953,8 +958,9 @@ static kvd_status launch_sel(kvd_ctx *ctx, const LayerState &ls, const CUtensorM
                              const CUtensorMap &tmap_rows, const RecomputeParams &p, const FusedParams *fp,
                              cudaStream_t stream) {
   if constexpr (FG == 0) {
-    // fp16 contexts: one variant (low table in shared memory) for all launch sizes
+    // fp16 and fp32 contexts: one variant (low table in shared memory) for all launch sizes
     if (ctx->dtype == 1) return launch_impl<BLOCK_N, D_HEAD, false, 0, 2, true, 1>(ctx, ls, tmap_store, tmap_rows, p, fp, stream);
+    if (ctx->dtype == 2) return launch_impl<BLOCK_N, D_HEAD, false, 0, 4, true, 2>(ctx, ls, tmap_store, tmap_rows, p, fp, stream);
     if (p.trace != nullptr) return launch_impl<BLOCK_N, D_HEAD, true, 0>(ctx, ls, tmap_store, tmap_rows, p, fp, stream);
     // one tile per cluster at most: every key tile's epilogue is exposed -> the low table from shared memory
     if (p.num_m_blocks * p.num_n_blocks <= ctx->num_sms / 2)
