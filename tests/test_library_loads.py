@@ -33,6 +33,9 @@ def test_size_queries_validate_shapes_without_a_device():
     good = kvd.make_desc(34, 2560, 8, 4, 256, 1e-6, True, 1e-6, max_seqs=2, max_tokens_per_seq=4096, max_batch=2)
     # rows + positions for 1 layer: 2 seqs * 4096 tokens * (2560 * 2 + 4) bytes
     assert kvd.kvd_store_bytes(good, 1) == 2 * 4096 * (2560 * 2 + 4 + 4)
+    assert kvd.kvd_store_bytes_dtype(good, 1, 1) == kvd.kvd_store_bytes(good, 1)      # fp16: the same room
+    assert kvd.kvd_store_bytes_dtype(good, 1, 2) == 2 * 4096 * (2560 * 4 + 4 + 4)     # fp32 rows
+    assert kvd.kvd_store_bytes_dtype(good, 1, 3) == 0
     assert kvd.kvd_workspace_bytes(good) > 0
     bad_head = kvd.make_desc(1, 2560, 8, 4, 96, 1e-6, True, 1e-6)
     assert kvd.kvd_store_bytes(bad_head, 1) == 0
