@@ -1012,6 +1012,7 @@ kvd_status launch_recompute_fp8(kvd_ctx *ctx, const LayerState &ls, const CUtens
                                 const RecomputeParams &p, cudaStream_t stream) {
   const int dh = ctx->desc.d_head;
   if (ctx->block_n == 256) {
+    if (dh == 256 && p.trace != nullptr) return launch_impl<256, 256, true, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
     if (dh == 256) return launch_impl<256, 256, false, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
     if (dh == 128) return launch_impl<256, 128, false, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
     if (dh == 64) return launch_impl<256, 64, false, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
