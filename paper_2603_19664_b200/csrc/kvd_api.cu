@@ -638,7 +638,7 @@ static kvd_status recompute_launch_fp8(kvd_ctx *ctx, int layer, const kvd_store_
   // 128 channels per k block; the tail reads zeros
   fill_launch_params(ctx, ls, p, n_jobs, mb, (d.d_hidden + 2 * RC_BLOCK_K - 1) / (2 * RC_BLOCK_K), out_row_stride);
   p.w_scale = ls.w_scale8;
-  if (ctx->trace && !fused) {
+  if (ctx->trace) {
     const int tiles = p.num_m_blocks * p.num_n_blocks;
     const size_t ctas = 2 * static_cast<size_t>(tiles < ctx->num_sms / 2 ? tiles : ctx->num_sms / 2);
     if (ctas * RC_TRACE_TILES * RC_TRACE_FIELDS * sizeof(long long) <= ctx->trace_bytes) p.trace = ctx->trace;

@@ -992,6 +992,7 @@ kvd_status launch_recompute_fused(kvd_ctx *ctx, const LayerState &ls, const CUte
   const int dh = ctx->desc.d_head, g = ctx->desc.n_q_heads / ctx->desc.n_kv_heads;
   if (ctx->block_n != 256 || p.k_cols % 256 != 0) return KVD_ERR_UNSUPPORTED;
   if (eb == 1) {  // rows and weights as E4M3 codes (the FP8 store)
+    if (dh == 256 && g == 2 && p.trace != nullptr) return launch_impl<256, 256, true, 2, 1>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
     if (dh == 256 && g == 2) return launch_impl<256, 256, false, 2, 1>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
     if (dh == 256 && g == 1) return launch_impl<256, 256, false, 1, 1>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
     if (dh == 128 && g == 4) return launch_impl<256, 128, false, 4, 1>(ctx, ls, tmap_store, tmap_rows, p, &fp, stream);
