@@ -365,7 +365,10 @@ kvd_status kvd_selftest_wait_timeout(kvd_ctx *ctx, int limit_ms, void *stream);
  *   3 cycles the MMA issuer waited for data            4/5 MMA issue start / end
  *   6/7 epilogue start / end     8 cycles the row-statistics warp waited   9 its total cycles
  *   10 tile index                11 (tile 0 only) kernel start
- * A call whose grid does not fit `bytes` records nothing.  No effect on results. */
+ *   12/13 (tile 0 only) global timer in ns at kernel start / end    14 (tile 0 only) kernel end
+ * A call whose grid does not fit `bytes` records nothing.  No effect on results.  Traced variants: the bf16
+ * kernel, and for the Gemma-3-4B head shape (d_head 256, 2 query heads per KV head) kvd_recompute_kv_fp8 and
+ * kvd_decode_attention_recompute_fp8; other variants ignore the hook. */
 kvd_status kvd_set_trace(kvd_ctx *ctx, void *buf, size_t bytes);
 
 /* Number of kernels this context has launched since creation (all entry points). */
