@@ -146,7 +146,7 @@ kvd_status kvd_set_dtype(kvd_ctx *ctx, int dtype);
 /* kvd_store_bytes for a context of the given element type (fp32 rows take twice the room). */
 size_t kvd_store_bytes_dtype(const kvd_model_desc *desc, int layers_stored, int dtype);
 
-/* Prepare layer `layer`: build W' = diag(gamma_in) * W_kv rounded to bf16 and stored K-major, the
+/* Prepare layer `layer`: build W' = diag(gamma_in) * W_kv rounded to the context's element type and stored K-major, the
  * fp32 key-norm scale, and the rotation tables for rope_theta.  Folding gamma into W is Eq. 1
  * composed with Eq. 13-14: (x / rms * gamma) W = (x W') / rms.  Enqueues on `stream` and waits for it. */
 kvd_status kvd_set_layer(kvd_ctx *ctx, int layer, const kvd_layer_desc *ldesc, void *stream);
