@@ -143,3 +143,12 @@ def test_fused_is_refused_for_shapes_it_is_not_built_for():
         ctx.kvd_decode_attention_recompute(0, 1, q, [0], [(0, 0, 0)], None, None, 0, None, None, kdim, [[]], 0.0, out)
     assert e.value.status == 6
     assert ctx.kvd_poll_status() == kvd.KVD_OK
+
+
+def test_fused_at_the_largest_batch():
+    # 64 sequences (the most one call takes), lengths 0 ... 600 evicted rows, 8 live keys each
+    lens = [int(v) for v in np.random.default_rng(11).integers(0, 601, size=64)]
+    lens[5], lens[40] = 0, 600
+    f, two, ref = run_case(GEMMA3_4B_GLOBAL, lens, 8, pos0_list=[3 * b for b in range(64)], max_tokens=1024, seed=12)
+    attn_check(f, ref, "fused vs oracle")
+    attn_check(f, two, "fused vs two-call")

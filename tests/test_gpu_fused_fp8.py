@@ -199,3 +199,25 @@ def test_fused_fp8_without_queries_only_stores_and_empty_call_launches_nothing()
     ctx.kvd_recompute_kv_fp8(0, [(0, 0, n, k2, v2)], kdim)
     assert ctx.kvd_poll_status() == kvd.KVD_OK
     assert torch.equal(k1, k2) and torch.equal(v1, v2) and float(k1.abs().max()) > 0
+
+
+def test_fused_fp8_at_the_largest_batch_without_stored_ranges():
+    # 64 sequences is the most one call takes when nothing is stored (batch + stored ranges <= 64)
+    lens = [int(v) for v in np.random.default_rng(13).integers(1, 500, size=64)]
+    f, two, ref = run_case(GEMMA3_4B_GLOBAL, lens, 0, pos0_list=[2 * b for b in range(64)], max_tokens=1024, seed=14,
+                           keep_nothing=True)
+    attn_check(f, ref, "fused vs oracle")
+    attn_check(f, two, "fused vs two-call")
+    # 33 sequences with one stored range each exceed the limit of 64 ranges per call
+    shape = GEMMA3_4B_GLOBAL
+    ctx, w = open_layer(shape, max_tokens=64, max_batch=33, max_seqs=33)
+    arena = torch.zeros(kvd.kvd_store_bytes_fp8(ctx.desc, 1), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_store_fp8(arena, 1)
+    kdim = shape.n_kv_heads * shape.d_head
+    q = dev(make_query(shape, 33, seed=1))
+    out = torch.zeros((33, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros((33, kdim), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(kvd.KvdError) as e:
+        ctx.kvd_decode_attention_recompute_fp8(0, 33, q, [0] * 33, [(b, 0, 0) for b in range(33)],
+                                               [(b, 0, 0, k[b:], k[b:]) for b in range(33)], kdim, [[] for _ in range(33)], 0.0, out)
+    assert e.value.status == 4
