@@ -932,27 +932,31 @@ def run_stack_configs(args):
             c.kvd_decode_attention_recompute(0, batch, q, qpos, franges, xc, pc, batch, kc, vc, kdim,
                                              segs_live[i % n_sets], 0.0, out)
 
-        # the same two layer forms with the evicted rows taken from the FP8 store.  K_t, V_t of the new tokens:
-        # up to 8 sequences -- from their quantised rows in the FP8 store, inside the same launch (one 256-row
-        # block per sequence); larger batches -- from their bf16 rows in a launch of their own, as in the
-        # full-cache layer
+        # the same two layer forms with the evicted rows taken from the FP8 store.  K_t, V_t of the new tokens
+        # come from their quantised rows inside the same launch: up to 8 sequences from the FP8 store (one
+        # 256-row block per sequence), larger batches from one contiguous buffer that kvd_quantize_rows_fp8 fills
+        # (one block for the whole batch; the small quantising launch is part of the timed layer)
         new_in_store = batch <= 8
         if new_in_store:
             for b in range(batch):
                 c.kvd_checkpoint_residual_fp8(b, 0, xc[b:b + 1], pc[b:b + 1], 1)
         new_ranges = [(b, ctx_len, 1, kc[b:], vc[b:]) for b in range(batch)] if new_in_store else []
+        codes_c = torch.empty((batch, shape.d_hidden), dtype=torch.uint8, device="cuda")
+        scales_c = torch.empty((batch,), dtype=torch.float32, device="cuda")
+        sumsq_c = torch.empty_like(scales_c)
+        new_rows = None if new_in_store else (codes_c, scales_c, sumsq_c, pc, batch, kc, vc)
 
         def layer_fp8(i):
             if not new_in_store:
-                cur(i)
-            c.kvd_recompute_kv_fp8(0, ranges + new_ranges, kdim)
+                c.kvd_quantize_rows_fp8(xc, batch, codes_c, scales_c, sumsq_c)
+            c.kvd_recompute_kv_fp8_rows(0, ranges + new_ranges, new_rows, kdim)
             att(i)
 
         def layer_fp8_fused(i):
             if not new_in_store:
-                cur(i)
-            c.kvd_decode_attention_recompute_fp8(0, batch, q, qpos, franges, new_ranges, kdim, segs_live[i % n_sets],
-                                                 0.0, out)
+                c.kvd_quantize_rows_fp8(xc, batch, codes_c, scales_c, sumsq_c)
+            c.kvd_decode_attention_recompute_fp8_rows(0, batch, q, qpos, franges, new_ranges, new_rows, kdim,
+                                                      segs_live[i % n_sets], 0.0, out)
 
         # memory-bound cases first, each after a short pause: a long run of GEMMs at the power cap
         # leaves the clocks low for whatever is measured next

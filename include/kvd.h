@@ -264,6 +264,28 @@ kvd_status kvd_checkpoint_residual_fp8(kvd_ctx *ctx, int seq, int layer, const v
  * rows first_row .. first_row+n-1 of every range to its k_out / v_out. */
 kvd_status kvd_recompute_kv_fp8(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
                                 int64_t out_row_stride, void *stream);
+/* Rows in the FP8 checkpoint format that live in the caller's memory instead of the store (the new tokens of a
+ * decode step: one contiguous buffer for the whole batch instead of one store range per sequence):
+ * kvd_quantize_rows_fp8 turns n bf16 rows (DEVICE [n, d_hidden], 16-byte aligned) into codes (DEVICE uint8
+ * [n, d_hidden], 16-byte aligned), scales and sums of squares (DEVICE fp32 [n]) exactly as
+ * kvd_checkpoint_residual_fp8 would store them; a kvd_fp8_rows (HOST struct of DEVICE pointers; positions int32
+ * [n]; k_out / v_out bf16 [n, out_row_stride], 16-byte aligned) hands them to the _rows forms of the FP8
+ * recompute calls, which write their K and V like those of a store range (same bits as from the store).
+ * rows == NULL or n == 0: no caller rows. */
+typedef struct {
+  const void *codes;
+  const float *scales;
+  const float *sumsq;
+  const int32_t *positions;
+  int32_t n;
+  int32_t reserved;
+  void *k_out;
+  void *v_out;
+} kvd_fp8_rows;
+kvd_status kvd_quantize_rows_fp8(kvd_ctx *ctx, const void *rows, int n, void *codes_out, float *scales_out,
+                                 float *sumsq_out, void *stream);
+kvd_status kvd_recompute_kv_fp8_rows(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
+                                     const kvd_fp8_rows *rows, int64_t out_row_stride, void *stream);
 
 /* ATTENTION(Q, K_all, V_all) of Algorithm 1 for one new token per sequence (Eq. 6-7).
  *   q      DEVICE bf16 [batch, n_q_heads, d_head], already normalised and rotated to q_pos.
@@ -318,6 +340,13 @@ kvd_status kvd_decode_attention_recompute_fp8(kvd_ctx *ctx, int layer, int batch
                                               const kvd_store_range *ranges, const kvd_store_range *store_ranges,
                                               int n_store_ranges, int64_t out_row_stride, const kvd_kv_segment *segs,
                                               int n_segs, float scale, void *out, void *stream);
+/* The same with caller-held quantised rows (see kvd_fp8_rows) stored next to store_ranges. */
+kvd_status kvd_decode_attention_recompute_fp8_rows(kvd_ctx *ctx, int layer, int batch, const void *q,
+                                                   const int32_t *q_pos, const kvd_store_range *ranges,
+                                                   const kvd_store_range *store_ranges, int n_store_ranges,
+                                                   const kvd_fp8_rows *rows, int64_t out_row_stride,
+                                                   const kvd_kv_segment *segs, int n_segs, float scale, void *out,
+                                                   void *stream);
 
 /* No counterpart in the paper: the same decode attention as kvd_decode_attention for callers that
  * cannot allocate device memory at all -- code running inside someone else's memory pool or under a

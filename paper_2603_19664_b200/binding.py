@@ -32,6 +32,7 @@ KVD_MAX_SEGMENTS = 4
 EXPORTED_SYMBOLS = (
     "kvd_create", "kvd_destroy", "kvd_set_layer", "kvd_store_bytes", "kvd_attach_store", "kvd_reset_sequence",
     "kvd_decode_attention_recompute", "kvd_decode_attention_recompute_fp8", "kvd_set_dtype", "kvd_store_bytes_dtype",
+    "kvd_quantize_rows_fp8", "kvd_recompute_kv_fp8_rows", "kvd_decode_attention_recompute_fp8_rows",
     "kvd_store_bytes_fp8", "kvd_attach_store_fp8", "kvd_rows_stored_fp8", "kvd_reset_sequence_fp8", "kvd_checkpoint_residual_fp8", "kvd_recompute_kv_fp8",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
     "kvd_recompute_kv_step",
@@ -43,6 +44,12 @@ EXPORTED_SYMBOLS = (
 class kvd_store_range(ctypes.Structure):
     _fields_ = [("seq", ctypes.c_int32), ("first_row", ctypes.c_int32), ("n", ctypes.c_int32),
                 ("reserved", ctypes.c_int32), ("k_out", ctypes.c_void_p), ("v_out", ctypes.c_void_p)]
+
+
+class kvd_fp8_rows(ctypes.Structure):
+    _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("sumsq", ctypes.c_void_p),
+                ("positions", ctypes.c_void_p), ("n", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("k_out", ctypes.c_void_p), ("v_out", ctypes.c_void_p)]
 
 
 class kvd_model_desc(ctypes.Structure):
@@ -146,6 +153,16 @@ def load() -> ctypes.CDLL:
                                                        i32, i64, ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float,
                                                        vp, vp]
     lib.kvd_decode_attention_recompute_fp8.restype = i32
+    lib.kvd_decode_attention_recompute_fp8_rows.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
+                                                            ctypes.POINTER(kvd_store_range), ctypes.POINTER(kvd_store_range),
+                                                            i32, ctypes.POINTER(kvd_fp8_rows), i64,
+                                                            ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
+    lib.kvd_decode_attention_recompute_fp8_rows.restype = i32
+    lib.kvd_quantize_rows_fp8.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    lib.kvd_quantize_rows_fp8.restype = i32
+    lib.kvd_recompute_kv_fp8_rows.argtypes = [vp, i32, ctypes.POINTER(kvd_store_range), i32, ctypes.POINTER(kvd_fp8_rows),
+                                              i64, vp]
+    lib.kvd_recompute_kv_fp8_rows.restype = i32
     lib.kvd_decode_attention_static.argtypes = [i32, i32, i32, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
                                                 ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
     lib.kvd_decode_attention_static.restype = i32
@@ -376,6 +393,50 @@ class Kvd:
         self._check(self._lib.kvd_decode_attention_recompute_fp8(
             self._h, layer, batch, _ptr(q), pos_arr, arr, sarr, len(store_ranges), out_row_stride, seg_arr, n_segs,
             float(scale), _ptr(out), _stream(stream)), "kvd_decode_attention_recompute_fp8")
+
+    @staticmethod
+    def _fp8_rows(rows):
+        """(codes, scales, sumsq, positions, n, k_out, v_out) -> kvd_fp8_rows, or None."""
+        if rows is None:
+            return None
+        codes, scales, sumsq, positions, n, k_out, v_out = rows
+        return kvd_fp8_rows(_ptr(codes), _ptr(scales), _ptr(sumsq), _ptr(positions), int(n), 0, _ptr(k_out), _ptr(v_out))
+
+    def kvd_quantize_rows_fp8(self, rows, n: int, codes_out, scales_out, sumsq_out, stream=None) -> None:
+        self._check(self._lib.kvd_quantize_rows_fp8(self._h, _ptr(rows), n, _ptr(codes_out), _ptr(scales_out),
+                                                    _ptr(sumsq_out), _stream(stream)), "kvd_quantize_rows_fp8")
+
+    def kvd_recompute_kv_fp8_rows(self, layer: int, ranges: Sequence[Tuple[int, int, int, object, object]], rows,
+                                  out_row_stride: int, stream=None) -> None:
+        """ranges as for kvd_recompute_kv_fp8; rows: (codes, scales, sumsq, positions, n, k_out, v_out) or None."""
+        arr = (kvd_store_range * max(len(ranges), 1))()
+        for i, (seq, first_row, n, k_out, v_out) in enumerate(ranges):
+            arr[i].seq, arr[i].first_row, arr[i].n, arr[i].reserved = int(seq), int(first_row), int(n), 0
+            arr[i].k_out, arr[i].v_out = _ptr(k_out), _ptr(v_out)
+        r = self._fp8_rows(rows)
+        self._check(self._lib.kvd_recompute_kv_fp8_rows(self._h, layer, arr, len(ranges), ctypes.byref(r) if r else None,
+                                                        out_row_stride, _stream(stream)), "kvd_recompute_kv_fp8_rows")
+
+    def kvd_decode_attention_recompute_fp8_rows(self, layer: int, batch: int, q, q_pos: Sequence[int],
+                                                ranges: Sequence[Tuple[int, int, int]],
+                                                store_ranges: Sequence[Tuple[int, int, int, object, object]], rows,
+                                                out_row_stride: int, segs: Sequence[Sequence[Segment]], scale: float,
+                                                out, stream=None) -> None:
+        """As kvd_decode_attention_recompute_fp8, plus caller-held quantised rows (see kvd_recompute_kv_fp8_rows)."""
+        n_segs, pos_arr, seg_arr = _marshal_segments(batch, q_pos, segs)
+        arr = (kvd_store_range * max(len(ranges), 1))()
+        for i, (seq, first_row, n) in enumerate(ranges):
+            arr[i].seq, arr[i].first_row, arr[i].n, arr[i].reserved = int(seq), int(first_row), int(n), 0
+            arr[i].k_out, arr[i].v_out = None, None
+        sarr = (kvd_store_range * max(len(store_ranges), 1))()
+        for i, (seq, first_row, n, k_out, v_out) in enumerate(store_ranges):
+            sarr[i].seq, sarr[i].first_row, sarr[i].n, sarr[i].reserved = int(seq), int(first_row), int(n), 0
+            sarr[i].k_out, sarr[i].v_out = _ptr(k_out), _ptr(v_out)
+        r = self._fp8_rows(rows)
+        self._check(self._lib.kvd_decode_attention_recompute_fp8_rows(
+            self._h, layer, batch, _ptr(q), pos_arr, arr, sarr, len(store_ranges), ctypes.byref(r) if r else None,
+            out_row_stride, seg_arr, n_segs, float(scale), _ptr(out), _stream(stream)),
+            "kvd_decode_attention_recompute_fp8_rows")
 
     def kvd_set_dtype(self, dtype: int) -> None:
         """0 = bf16 (default), 1 = fp16 (checkpoint, recompute and kvd_decode_attention), 2 = fp32 (checkpoint and

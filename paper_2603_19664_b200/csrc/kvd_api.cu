@@ -596,11 +596,13 @@ extern "C" kvd_status kvd_checkpoint_residual_fp8(kvd_ctx *ctx, int seq, int lay
 // job table from ranges of the FP8 store, launch once.  With `fused` (one RcAttend per range, q ==
 // nullptr for a range whose K/V are written) the ranges that carry a query are attended in the kernel.
 static kvd_status recompute_launch_fp8(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
-                                       int64_t out_row_stride, cudaStream_t stream, const RcAttend *fused = nullptr,
-                                       const AttnLaunchHead *fused_head = nullptr) {
+                                       const kvd_fp8_rows *rows, int64_t out_row_stride, cudaStream_t stream,
+                                       const RcAttend *fused = nullptr, const AttnLaunchHead *fused_head = nullptr) {
   const LayerState &ls = ctx->layers[layer];
-  if (!ls.set || !ctx->store8_codes || !ls.wt8) return KVD_ERR_STATE;
-  if (layer >= ctx->layers_stored8) return KVD_ERR_INVALID_ARG;
+  if (!ls.set || !ls.wt8) return KVD_ERR_STATE;
+  bool any_range = false;
+  for (int i = 0; i < n_ranges; ++i) any_range |= ranges[i].n > 0;
+  if (any_range && (!ctx->store8_codes || layer >= ctx->layers_stored8)) return ctx->store8_codes ? KVD_ERR_INVALID_ARG : KVD_ERR_STATE;
   const kvd_model_desc &d = ctx->desc;
   const int kdim = d.n_kv_heads * d.d_head;
   if (out_row_stride < kdim) return KVD_ERR_INVALID_ARG;
@@ -634,7 +636,33 @@ static kvd_status recompute_launch_fp8(kvd_ctx *ctx, int layer, const kvd_store_
     J.v_out = static_cast<__nv_bfloat16 *>(r.v_out);
     mb += (r.n + 2 * RC_BLOCK_M - 1) / (2 * RC_BLOCK_M);
   }
+  // the caller's own quantised rows (kvd_quantize_rows_fp8): one more job, always stored
+  CUtensorMap tmap_rows;
+  const bool have_rows = rows != nullptr && rows->n > 0;
+  if (rows != nullptr && rows->n < 0) return KVD_ERR_INVALID_ARG;
+  if (have_rows) {
+    if (!rows->codes || !rows->scales || !rows->sumsq || !rows->positions || !rows->k_out || !rows->v_out) return KVD_ERR_INVALID_ARG;
+    if (!aligned16(rows->codes) || !aligned16(rows->k_out) || !aligned16(rows->v_out)) return KVD_ERR_ALIGNMENT;
+    kvd_status st = encode_rows_3d(ctx, &tmap_rows, rows->codes, d.d_hidden, static_cast<uint64_t>(rows->n), 1, 1);
+    if (st != KVD_OK) return st;
+    if (fused) fp.att[n_jobs] = RcAttend{};
+    RcJob &J = p.jobs[n_jobs++];
+    J.mb_start = mb;
+    J.n = rows->n;
+    J.row0 = 0;
+    J.slab = -1;
+    J.positions = rows->positions;
+    J.sumsq = rows->sumsq;
+    J.scale = rows->scales;
+    J.k_out = static_cast<__nv_bfloat16 *>(rows->k_out);
+    J.v_out = static_cast<__nv_bfloat16 *>(rows->v_out);
+    mb += (rows->n + 2 * RC_BLOCK_M - 1) / (2 * RC_BLOCK_M);
+  }
   if (n_jobs == 0) return KVD_OK;
+  // the kernel is handed both maps; an unused one aliases the other
+  const bool any_store = n_jobs > (have_rows ? 1 : 0);
+  const CUtensorMap &map_store = any_store ? ctx->store8_maps[layer] : tmap_rows;
+  const CUtensorMap &map_rows = have_rows ? tmap_rows : ctx->store8_maps[layer];
   // 128 channels per k block; the tail reads zeros
   fill_launch_params(ctx, ls, p, n_jobs, mb, (d.d_hidden + 2 * RC_BLOCK_K - 1) / (2 * RC_BLOCK_K), out_row_stride);
   p.w_scale = ls.w_scale8;
@@ -648,16 +676,35 @@ static kvd_status recompute_launch_fp8(kvd_ctx *ctx, int layer, const kvd_store_
     fp.part_ml = fused_head->part_ml;
     fp.n_q = fused_head->n_q;
     fp.scale_log2e = fused_head->scale_log2e;
-    return launch_recompute_fused(ctx, ls, ctx->store8_maps[layer], ctx->store8_maps[layer], p, fp, stream, 1);
+    return launch_recompute_fused(ctx, ls, map_store, map_rows, p, fp, stream, 1);
   }
-  return launch_recompute_fp8(ctx, ls, ctx->store8_maps[layer], p, stream);
+  return launch_recompute_fp8(ctx, ls, map_store, map_rows, p, stream);
+}
+
+extern "C" kvd_status kvd_quantize_rows_fp8(kvd_ctx *ctx, const void *rows, int n, void *codes_out, float *scales_out,
+                                            float *sumsq_out, void *stream_) {
+  if (!ctx || n < 0) return KVD_ERR_INVALID_ARG;
+  if (ctx->dtype != KVD_DTYPE_BF16) return KVD_ERR_UNSUPPORTED;
+  if (ctx->desc.d_hidden % 16 != 0) return KVD_ERR_SHAPE;
+  if (n == 0) return KVD_OK;
+  if (!rows || !codes_out || !scales_out || !sumsq_out) return KVD_ERR_INVALID_ARG;
+  if (!aligned16(rows) || !aligned16(codes_out)) return KVD_ERR_ALIGNMENT;
+  return launch_checkpoint_fp8(ctx, static_cast<const __nv_bfloat16 *>(rows), nullptr, static_cast<uint8_t *>(codes_out),
+                               nullptr, sumsq_out, scales_out, n, ctx->desc.d_hidden, static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" kvd_status kvd_recompute_kv_fp8_rows(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
+                                                const kvd_fp8_rows *rows, int64_t out_row_stride, void *stream_) {
+  if (!ctx || n_ranges < 0 || n_ranges > KVD_MAX_STORE_RANGES || (n_ranges > 0 && !ranges)) return KVD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  return recompute_launch_fp8(ctx, layer, ranges, n_ranges, rows, out_row_stride, static_cast<cudaStream_t>(stream_));
 }
 
 extern "C" kvd_status kvd_recompute_kv_fp8(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
                                            int64_t out_row_stride, void *stream_) {
   if (!ctx || n_ranges < 0 || n_ranges > KVD_MAX_STORE_RANGES || (n_ranges > 0 && !ranges)) return KVD_ERR_INVALID_ARG;
   if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
-  return recompute_launch_fp8(ctx, layer, ranges, n_ranges, out_row_stride, static_cast<cudaStream_t>(stream_));
+  return recompute_launch_fp8(ctx, layer, ranges, n_ranges, nullptr, out_row_stride, static_cast<cudaStream_t>(stream_));
 }
 
 extern "C" kvd_status kvd_recompute_kv(kvd_ctx *ctx, int layer, const void *rows, const int32_t *positions, int n,
@@ -871,12 +918,14 @@ extern "C" kvd_status kvd_decode_attention_recompute(kvd_ctx *ctx, int layer, in
   return launch_attention(ctx, L, d.d_head, group, stream);
 }
 
-// The same over the FP8 store: ranges[b] is attended by query b; store_ranges are written as K/V.
-extern "C" kvd_status kvd_decode_attention_recompute_fp8(kvd_ctx *ctx, int layer, int batch, const void *q,
-                                                         const int32_t *q_pos, const kvd_store_range *ranges,
-                                                         const kvd_store_range *store_ranges, int n_store_ranges,
-                                                         int64_t out_row_stride, const kvd_kv_segment *segs,
-                                                         int n_segs, float scale, void *out, void *stream_) {
+// The same over the FP8 store: ranges[b] is attended by query b; store_ranges and the caller's quantised rows
+// are written as K/V.
+extern "C" kvd_status kvd_decode_attention_recompute_fp8_rows(kvd_ctx *ctx, int layer, int batch, const void *q,
+                                                              const int32_t *q_pos, const kvd_store_range *ranges,
+                                                              const kvd_store_range *store_ranges, int n_store_ranges,
+                                                              const kvd_fp8_rows *rows, int64_t out_row_stride,
+                                                              const kvd_kv_segment *segs, int n_segs, float scale,
+                                                              void *out, void *stream_) {
   if (!ctx || batch < 0 || n_segs < 0 || n_segs > KVD_MAX_SEGMENTS || n_store_ranges < 0) return KVD_ERR_INVALID_ARG;
   if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
   const LayerState &ls = ctx->layers[layer];
@@ -888,7 +937,7 @@ extern "C" kvd_status kvd_decode_attention_recompute_fp8(kvd_ctx *ctx, int layer
   if (ctx->block_n != 256 || kdim % 256 != 0 || !((d.d_head == 256 && (group == 1 || group == 2)) ||
                                                    (d.d_head == 128 && (group == 1 || group == 2 || group == 4))))
     return KVD_ERR_UNSUPPORTED;
-  if (batch == 0 && n_store_ranges == 0) return KVD_OK;
+  if (batch == 0 && n_store_ranges == 0 && (rows == nullptr || rows->n == 0)) return KVD_OK;
   if (batch > 0 && (!q || !q_pos || !out || !ranges || (n_segs > 0 && !segs))) return KVD_ERR_INVALID_ARG;
   if (n_store_ranges > 0 && !store_ranges) return KVD_ERR_INVALID_ARG;
   if (batch > 0 && (!aligned16(q) || !aligned16(out))) return KVD_ERR_ALIGNMENT;
@@ -918,11 +967,20 @@ extern "C" kvd_status kvd_decode_attention_recompute_fp8(kvd_ctx *ctx, int layer
     all[batch + i] = store_ranges[i];
     att[batch + i] = RcAttend{};
   }
-  st = recompute_launch_fp8(ctx, layer, all, batch + n_store_ranges, out_row_stride > 0 ? out_row_stride : kdim, stream,
-                            att, &L);
+  st = recompute_launch_fp8(ctx, layer, all, batch + n_store_ranges, rows, out_row_stride > 0 ? out_row_stride : kdim,
+                            stream, att, &L);
   if (st != KVD_OK) return st;
   if (batch == 0) return KVD_OK;
   return launch_attention(ctx, L, d.d_head, group, stream);
+}
+
+extern "C" kvd_status kvd_decode_attention_recompute_fp8(kvd_ctx *ctx, int layer, int batch, const void *q,
+                                                         const int32_t *q_pos, const kvd_store_range *ranges,
+                                                         const kvd_store_range *store_ranges, int n_store_ranges,
+                                                         int64_t out_row_stride, const kvd_kv_segment *segs,
+                                                         int n_segs, float scale, void *out, void *stream_) {
+  return kvd_decode_attention_recompute_fp8_rows(ctx, layer, batch, q, q_pos, ranges, store_ranges, n_store_ranges, nullptr,
+                                                 out_row_stride, segs, n_segs, scale, out, stream_);
 }
 
 extern "C" kvd_status kvd_memory_stats(const kvd_ctx *ctx, kvd_mem_stats *out) {

@@ -272,7 +272,7 @@ kvd_status launch_prepare_weights_fp8(kvd_ctx *ctx, const __nv_bfloat16 *w, cons
                                       int d_hidden, int n_cols, unsigned *amax_scratch, float *scale_out,
                                       cudaStream_t stream);
 kvd_status launch_recompute_fp8(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
-                                const RecomputeParams &p, cudaStream_t stream);
+                                const CUtensorMap &tmap_rows, const RecomputeParams &p, cudaStream_t stream);
 kvd_status launch_checkpoint(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, __nv_bfloat16 *dst_rows,
                              int32_t *dst_pos, float *dst_sumsq, int n, int d_hidden, cudaStream_t stream);
 kvd_status launch_selftest_timeout(kvd_ctx *ctx, unsigned long long timeout_ns, cudaStream_t stream);

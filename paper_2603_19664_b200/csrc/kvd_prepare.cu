@@ -186,7 +186,7 @@ __global__ void __launch_bounds__(256) kvd_checkpoint_fp8_kernel(const uint4 *__
     }
     if (lane == 0) {
       dst_sumsq[r] = ss;
-      dst_pos[r] = pos[r];
+      if (dst_pos != nullptr) dst_pos[r] = pos[r];  // (no positions when the rows are only quantised, not stored)
     }
   }
 }

@@ -1008,18 +1008,19 @@ kvd_status launch_recompute_fused(kvd_ctx *ctx, const LayerState &ls, const CUte
   return KVD_ERR_UNSUPPORTED;
 }
 
-// The FP8 variant: rows and weights as E4M3 codes (tmap_store is the FP8 store's map).
+// The FP8 variant: rows and weights as E4M3 codes (tmap_store is the FP8 store's map, tmap_rows the map of
+// the caller's quantised rows, or the store's again).
 kvd_status launch_recompute_fp8(kvd_ctx *ctx, const LayerState &ls, const CUtensorMap &tmap_store,
-                                const RecomputeParams &p, cudaStream_t stream) {
+                                const CUtensorMap &tmap_rows, const RecomputeParams &p, cudaStream_t stream) {
   const int dh = ctx->desc.d_head;
   if (ctx->block_n == 256) {
-    if (dh == 256 && p.trace != nullptr) return launch_impl<256, 256, true, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
-    if (dh == 256) return launch_impl<256, 256, false, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
-    if (dh == 128) return launch_impl<256, 128, false, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
-    if (dh == 64) return launch_impl<256, 64, false, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
+    if (dh == 256 && p.trace != nullptr) return launch_impl<256, 256, true, 0, 1, true>(ctx, ls, tmap_store, tmap_rows, p, nullptr, stream);
+    if (dh == 256) return launch_impl<256, 256, false, 0, 1, true>(ctx, ls, tmap_store, tmap_rows, p, nullptr, stream);
+    if (dh == 128) return launch_impl<256, 128, false, 0, 1, true>(ctx, ls, tmap_store, tmap_rows, p, nullptr, stream);
+    if (dh == 64) return launch_impl<256, 64, false, 0, 1, true>(ctx, ls, tmap_store, tmap_rows, p, nullptr, stream);
   } else if (ctx->block_n == 128) {
-    if (dh == 128) return launch_impl<128, 128, false, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
-    if (dh == 64) return launch_impl<128, 64, false, 0, 1, true>(ctx, ls, tmap_store, tmap_store, p, nullptr, stream);
+    if (dh == 128) return launch_impl<128, 128, false, 0, 1, true>(ctx, ls, tmap_store, tmap_rows, p, nullptr, stream);
+    if (dh == 64) return launch_impl<128, 64, false, 0, 1, true>(ctx, ls, tmap_store, tmap_rows, p, nullptr, stream);
   }
   return KVD_ERR_SHAPE;
 }

@@ -164,3 +164,45 @@ def test_fp8_argument_errors():
         ctx.kvd_recompute_kv_fp8(0, [(0, 0, 8, k, k)], kdim)
     assert e.value.status == 4
     assert ctx.kvd_poll_status() == kvd.KVD_OK
+
+
+def test_caller_held_quantised_rows_give_the_bits_of_rows_in_the_store():
+    """kvd_quantize_rows_fp8 + the _rows forms: the new tokens of a batch in one contiguous caller buffer instead
+    of one store range per sequence.  Codes, scales and statistics equal what the checkpoint stores; K/V from the
+    caller's rows equal K/V from the same rows in the store, alone and next to store ranges in one launch."""
+    shape = GEMMA3_4B_GLOBAL
+    ctx, w, arena = open_fp8(shape, 512, max_seqs=2)
+    kdim = shape.n_kv_heads * shape.d_head
+    n = 70
+    X = make_residuals(shape, n, seed=35, outliers=True)
+    pos = np.arange(n) + 100
+    x, p = dev(X), torch.from_numpy(pos.astype(np.int32)).cuda()
+    ctx.kvd_checkpoint_residual_fp8(0, 0, x, p, n)
+    codes = torch.zeros((n, shape.d_hidden), dtype=torch.uint8, device="cuda")
+    scales = torch.zeros((n,), dtype=torch.float32, device="cuda")
+    sumsq = torch.zeros_like(scales)
+    ctx.kvd_quantize_rows_fp8(x, n, codes, scales, sumsq)
+    torch.cuda.synchronize()
+    q_ref, s_ref = ofp8.quantize_rows(bf16_to_f64(X))
+    assert np.array_equal(LUT[codes.cpu().numpy()], q_ref) and np.array_equal(scales.cpu().numpy().astype(np.float64), s_ref)
+    a = arena.cpu().numpy()
+    ru = lambda b: (b + 255) // 256 * 256
+    slots = 2 * 512
+    c_bytes, f_bytes = ru(slots * shape.d_hidden), ru(slots * 4)
+    assert np.array_equal(a[:c_bytes].reshape(-1, shape.d_hidden)[:n], codes.cpu().numpy())
+    assert np.array_equal(a[c_bytes + f_bytes:c_bytes + 2 * f_bytes].view(np.uint32)[:n], sumsq.cpu().numpy().view(np.uint32))
+    # K/V: from the store, from the caller's rows, and both kinds of source in one launch
+    ks = torch.zeros((n, kdim), dtype=torch.bfloat16, device="cuda"); vs = torch.zeros_like(ks)
+    kc = torch.zeros_like(ks); vc = torch.zeros_like(ks)
+    ctx.kvd_recompute_kv_fp8(0, [(0, 0, n, ks, vs)], kdim)
+    ctx.kvd_recompute_kv_fp8_rows(0, [], (codes, scales, sumsq, p, n, kc, vc), kdim)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    assert torch.equal(ks, kc) and torch.equal(vs, vc) and float(kc.abs().max()) > 0
+    k1 = torch.zeros((40, kdim), dtype=torch.bfloat16, device="cuda"); v1 = torch.zeros_like(k1)
+    k2 = torch.zeros((3, kdim), dtype=torch.bfloat16, device="cuda"); v2 = torch.zeros_like(k2)
+    ctx.kvd_recompute_kv_fp8_rows(0, [(0, 5, 40, k1, v1)], (codes[60:], scales[60:], sumsq[60:], p[60:], 3, k2, v2), kdim)
+    assert torch.equal(k1, ks[5:45]) and torch.equal(v1, vs[5:45]) and torch.equal(k2, ks[60:63]) and torch.equal(v2, vs[60:63])
+    with pytest.raises(kvd.KvdError) as e:      # incomplete description of the rows
+        ctx.kvd_recompute_kv_fp8_rows(0, [], (codes, None, sumsq, p, n, kc, vc), kdim)
+    assert e.value.status == 1
+    assert ctx.kvd_poll_status() == kvd.KVD_OK

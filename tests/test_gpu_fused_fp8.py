@@ -221,3 +221,42 @@ def test_fused_fp8_at_the_largest_batch_without_stored_ranges():
         ctx.kvd_decode_attention_recompute_fp8(0, 33, q, [0] * 33, [(b, 0, 0) for b in range(33)],
                                                [(b, 0, 0, k[b:], k[b:]) for b in range(33)], kdim, [[] for _ in range(33)], 0.0, out)
     assert e.value.status == 4
+
+
+def test_fused_fp8_with_the_new_tokens_as_caller_held_rows():
+    """A batch of 5 sequences: evicted ranges attended inside the kernel, the new tokens handed over as one
+    contiguous buffer of quantised rows.  Same output and same K_t, V_t bits as with the new tokens in the store."""
+    shape = GEMMA3_4B_GLOBAL
+    lens = [300, 0, 513, 40, 129]
+    batch = len(lens)
+    ctx, w = open_layer(shape, max_tokens=1024, max_batch=batch, max_seqs=batch)
+    arena = torch.zeros(kvd.kvd_store_bytes_fp8(ctx.desc, 1), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_store_fp8(arena, 1)
+    kdim = shape.n_kv_heads * shape.d_head
+    q = dev(make_query(shape, batch, seed=21))
+    x_new = torch.empty((batch, shape.d_hidden), dtype=torch.bfloat16, device="cuda")
+    p_new = torch.empty((batch,), dtype=torch.int32, device="cuda")
+    for b, n in enumerate(lens):
+        X = dev(make_residuals(shape, n + 1, seed=300 + b, outliers=True))
+        p = torch.arange(n + 1, dtype=torch.int32, device="cuda") + 7 * b
+        ctx.kvd_checkpoint_residual_fp8(b, 0, X, p, n + 1)      # the new token too: the reference form reads it there
+        x_new[b].copy_(X[n])
+        p_new[b] = n + 7 * b
+    q_pos = [n + 7 * b for b, n in enumerate(lens)]
+    ranges = [(b, 0, n) for b, n in enumerate(lens)]
+    k_a = torch.zeros((batch, kdim), dtype=torch.bfloat16, device="cuda"); v_a = torch.zeros_like(k_a)
+    k_b = torch.zeros_like(k_a); v_b = torch.zeros_like(k_a)
+    out_a = torch.zeros((batch, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda")
+    out_b = torch.zeros_like(out_a)
+    live = lambda k, v: [[(k[b:], v[b:], kdim, q_pos[b], 1)] for b in range(batch)]
+    ctx.kvd_decode_attention_recompute_fp8(0, batch, q, q_pos, ranges, [(b, lens[b], 1, k_a[b:], v_a[b:]) for b in range(batch)],
+                                           kdim, live(k_a, v_a), 0.0, out_a)
+    codes = torch.zeros((batch, shape.d_hidden), dtype=torch.uint8, device="cuda")
+    scales = torch.zeros((batch,), dtype=torch.float32, device="cuda")
+    sumsq = torch.zeros_like(scales)
+    ctx.kvd_quantize_rows_fp8(x_new, batch, codes, scales, sumsq)
+    ctx.kvd_decode_attention_recompute_fp8_rows(0, batch, q, q_pos, ranges, [], (codes, scales, sumsq, p_new, batch, k_b, v_b),
+                                                kdim, live(k_b, v_b), 0.0, out_b)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    assert torch.equal(k_a, k_b) and torch.equal(v_a, v_b) and torch.equal(out_a, out_b)
+    assert float(out_a.abs().max()) > 0
