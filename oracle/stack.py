@@ -14,9 +14,13 @@ Three cache policies share every line of the model:
                      layer 0 (the d_hidden * b bytes per token of Eq. 24): every step the evicted
                      tokens are carried through the layers again, so that at layer l their rows
                      h^(l), and from them their keys and values, exist while that layer runs.
-K and V of the current token and of rebuilt tokens come from the same oracle routine
-(``oracle.recompute_kv``), which treats rows independently, so Proposition 3.2's "same operations
-in the same order" holds literally and the two policies must agree bit for bit.
+K_t and V_t of the token being processed follow the FORWARD equations (Eq. 4-5 with the rotation
+of Eq. 11-12), written out here in Python: RMSNorm, one dot product per output channel summed over
+the hidden index in ascending order, the per-head key norm, the rotation.  K and V of evicted
+tokens come from the RECONSTRUCTION routine (``oracle.recompute_kv``, Eq. 13-14, C).  The two are
+separate pieces of code that take the same operations in the same order, which is what
+Proposition 3.2 asserts makes them agree bit for bit; the tests check exactly that, so a slip in
+either one (a dropped scale, another rotation angle, a transposed weight) shows.
 
 Readings where Algorithm 1 is silent: W_o and the rotations are applied as Eq. 3-8 state; the
 current token's (K_t, V_t) joins the live window after attention, then the oldest entries are
@@ -28,6 +32,8 @@ from __future__ import annotations
 
 from dataclasses import dataclass, field
 from typing import Dict, List, Optional
+
+import math
 
 import numpy as np
 
@@ -80,7 +86,7 @@ class OracleStack:
             if s.qk_norm:
                 q[hh] = rmsnorm(q[hh], lw["gamma_q"], s.rms_eps)
             q[hh] = rope(q[hh], pos, ls.rope_theta, s.rope_style)
-        k_t, v_t = self._kv_rows(l, [h], [pos])
+        k_t, v_t = self._kv_forward(l, h, pos)
         heads = decode_attention(q, pos, list(segments_before) + [(k_t, v_t, pos)], scale, ls.sliding_window)
         h = h + heads.reshape(-1) @ lw["w_o"]  # Eq. 8
         xm = rmsnorm(h, lw["gamma_mlp"], s.rms_eps)
@@ -141,6 +147,41 @@ class OracleStack:
         self.t += 1
         hf = rmsnorm(h, w["gamma_final"], s.rms_eps)
         return hf @ w["lm_head"]
+
+    def _kv_forward(self, l: int, h: np.ndarray, pos: int):
+        """Eq. 4-5 for one token during its own forward pass: K_t = R_pos(keynorm(W_K^T RMSNorm(h))),
+        V_t = W_V^T RMSNorm(h), each [1, n_kv, d_head].  Python restatement, independent of the C
+        reconstruction routine; every sum runs over its index in ascending order."""
+        s, lw, ls = self.s, self.w["layers"][l], self.s.layer_shape(l)
+        d, kdim, dh = s.d_hidden, s.n_kv_heads * s.d_head, s.d_head
+        ms = 0.0
+        for i in range(d):  # Eq. 2
+            ms += float(h[i]) * float(h[i])
+        r = math.sqrt(ms / d + s.rms_eps)
+        xb = [float(h[i]) / r * float(lw["gamma_in"][i]) for i in range(d)]  # Eq. 1
+        w_kv = lw["w_kv"]
+        acc = np.zeros(2 * kdim, dtype=np.float64)
+        for i in range(d):  # Eq. 4-5 before the rotation: channel c receives its terms in ascending i
+            acc += xb[i] * w_kv[i]
+        k = acc[:kdim].reshape(s.n_kv_heads, dh).copy()
+        v = acc[kdim:].reshape(s.n_kv_heads, dh).copy()
+        half = dh // 2
+        for g in range(s.n_kv_heads):
+            if s.qk_norm:
+                ss = 0.0
+                for j in range(dh):
+                    ss += float(k[g, j]) * float(k[g, j])
+                rk = math.sqrt(ss / dh + s.rms_eps)
+                for j in range(dh):
+                    k[g, j] = float(k[g, j]) / rk * float(lw["gamma_k"][j])
+            for i in range(half):  # Eq. 11-12, pair i turned by pos * theta^(-2i/d_head)
+                phi = float(pos) * math.pow(ls.rope_theta, -2.0 * i / dh)
+                c, sn = math.cos(phi), math.sin(phi)
+                ia, ib = (i, i + half) if s.rope_style == ROPE_HALF else (2 * i, 2 * i + 1)
+                a, b = float(k[g, ia]), float(k[g, ib])
+                k[g, ia] = a * c - b * sn
+                k[g, ib] = a * sn + b * c
+        return k[None], v[None]
 
     def _kv_rows(self, l: int, rows: List[np.ndarray], positions: List[int]):
         s, lw, ls = self.s, self.w["layers"][l], self.s.layer_shape(l)
