@@ -19,8 +19,10 @@ no infinities, largest finite value 448, subnormal step 2^-9, round to nearest e
 (tests/test_oracle_fp8.py) are the value table implied by that definition, hand-picked ties, and PyTorch's
 own float8_e4m3fn conversion on the CPU as an independent library routine.
 
-The codes are an encoding decided in floating point, so both sides take that decision in the same
-precision: the scale, the reciprocal, the product and the rounding input are fp32 here exactly as in the kernel.
+The codes are an encoding decided in floating point, so the definition fixes the precision of that
+decision: the scale, the reciprocal, the product and the rounding input are fp32.  The definition is
+frozen: a change to this file's arithmetic has to name the reading of the paper that calls for it, never a
+property of an implementation.
 """
 from __future__ import annotations
 

@@ -3,7 +3,7 @@
   * the bounded-window policy with recomputation must give the same tokens AND bit-identical logits
     as the full-cache policy at every budget (Table 3 / Section 5.6 of the paper, on the GPU);
   * the GPU stack must follow the fp64 oracle stack: logits within bf16 error, and the same token
-    wherever the oracle's top-2 margin exceeds four times the observed logit error (the GPU run is
+    wherever the oracle's top-2 margin exceeds twice the observed logit error (the GPU run is
     teacher-forced with the oracle's tokens so that one near-tie cannot derail the comparison).
 """
 import numpy as np
@@ -35,23 +35,29 @@ def test_bounded_window_with_recompute_is_token_and_bit_identical_to_full_cache(
         assert rep["live_kv_bytes"] <= stack.n_layers * max(B, 0) * 2 * stack.n_kv_heads * stack.d_head * 2 or B >= m.t
 
 
-@pytest.mark.parametrize("stack,ctx_len", [(S_GEMMA, 48), (S_SMOL, 48)], ids=lambda x: getattr(x, "name", x))
+@pytest.mark.parametrize("stack,ctx_len", [(S_GEMMA, 48), (S_SMOL, 48), (S_QWEN, 48)], ids=lambda x: getattr(x, "name", x))
 def test_gpu_stack_follows_the_oracle_stack(stack, ctx_len):
     w = make_stack_weights(stack)
     prompt = make_token_ids(ctx_len, stack.vocab, seed=3).tolist()
     o_tokens, o_logits = OracleStack(stack, weights_to_f64(w, bf16_to_f64), "kvdirect", 8).generate(prompt, 16)
     g_tokens, g_logits = GpuStack(stack, w, "kvdirect", 8).generate(prompt, 16, forced=o_tokens)
     errs = [float(np.max(np.abs(g.cpu().numpy().astype(np.float64) - o))) for g, o in zip(g_logits, o_logits)]
+    rels = [float(np.linalg.norm(g.cpu().numpy().astype(np.float64) - o) / np.linalg.norm(o))
+            for g, o in zip(g_logits, o_logits)]
     err = max(errs)
     scale = max(float(np.max(np.abs(o))) for o in o_logits)
-    assert err <= 0.05 * scale, f"logit error {err} vs scale {scale}"
+    # Measured on these stacks (bf16 activations through 4-6 layers, fp32 accumulation): the largest logit error is
+    # 0.55-0.71 % of the largest logit and the relative Frobenius error 0.58-0.72 %; the bounds leave a margin of 1.4.
+    assert err <= 0.01 * scale, f"logit error {err} vs scale {scale}"
+    assert max(rels) <= 0.01, f"relative logit error {max(rels)}"
+    # two logits that are each off by at most err can change order only if they are closer than 2 err
     decided = 0
     for i, (o, gt, ot) in enumerate(zip(o_logits, g_tokens, o_tokens)):
         top2 = np.sort(o)[-2:]
-        if top2[1] - top2[0] > 4 * err:
+        if top2[1] - top2[0] > 2 * err:
             decided += 1
             assert gt == ot, f"step {i}: margin {top2[1] - top2[0]} vs error {err}"
-    assert decided >= 4, "too few steps with a clear margin to compare tokens"
+    assert decided >= 8, "too few steps with a clear margin to compare tokens"
 
 
 def test_multi_turn_session_matches_and_bounds_live_kv():
