@@ -38,7 +38,13 @@ EXPORTED_SYMBOLS = (
     "kvd_recompute_kv_step",
     "kvd_decode_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
     "kvd_status_string", "kvd_version",
+    # include/kvd_scaffold.h: the parts of a decoder layer around the hot path, for whole-stack tests and benchmarks
+    "kvd_scaffold_linear_create", "kvd_scaffold_linear_destroy", "kvd_scaffold_linear_out_cols", "kvd_scaffold_linear",
+    "kvd_scaffold_query_finish", "kvd_scaffold_add_rows", "kvd_scaffold_gated_act", "kvd_scaffold_embed",
+    "kvd_scaffold_argmax",
 )
+KVD_ACT_GELU_TANH = 0
+KVD_ACT_SILU = 1
 
 
 class kvd_store_range(ctypes.Structure):
@@ -182,6 +188,24 @@ def load() -> ctypes.CDLL:
     lib.kvd_status_string.restype = ctypes.c_char_p
     lib.kvd_version.argtypes = []
     lib.kvd_version.restype = ctypes.c_char_p
+    lib.kvd_scaffold_linear_create.argtypes = [vp, vp, vp, i32, i32, ctypes.c_float, vp, ctypes.POINTER(vp)]
+    lib.kvd_scaffold_linear_create.restype = i32
+    lib.kvd_scaffold_linear_destroy.argtypes = [vp, vp]
+    lib.kvd_scaffold_linear_destroy.restype = None
+    lib.kvd_scaffold_linear_out_cols.argtypes = [vp]
+    lib.kvd_scaffold_linear_out_cols.restype = i32
+    lib.kvd_scaffold_linear.argtypes = [vp, vp, vp, i32, vp, i64, vp]
+    lib.kvd_scaffold_linear.restype = i32
+    lib.kvd_scaffold_query_finish.argtypes = [vp, i32, vp, i64, vp, i32, vp, vp, vp]
+    lib.kvd_scaffold_query_finish.restype = i32
+    lib.kvd_scaffold_add_rows.argtypes = [vp, vp, vp, i64, i32, i32, vp]
+    lib.kvd_scaffold_add_rows.restype = i32
+    lib.kvd_scaffold_gated_act.argtypes = [vp, vp, i64, i32, i32, i32, vp, vp]
+    lib.kvd_scaffold_gated_act.restype = i32
+    lib.kvd_scaffold_embed.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
+    lib.kvd_scaffold_embed.restype = i32
+    lib.kvd_scaffold_argmax.argtypes = [vp, vp, i64, i32, i32, vp, vp]
+    lib.kvd_scaffold_argmax.restype = i32
     _lib = lib
     return lib
 
@@ -489,3 +513,55 @@ class Kvd:
 
     def kvd_launch_count(self) -> int:
         return int(self._lib.kvd_launch_count(self._h))
+
+    # ---- include/kvd_scaffold.h (marshalling only, like everything above)
+    def kvd_scaffold_linear_create(self, w, gamma, k: int, n: int, rms_eps: float = 0.0, stream=None) -> "Linear":
+        h = ctypes.c_void_p()
+        self._check(self._lib.kvd_scaffold_linear_create(self._h, _ptr(w), _ptr(gamma), k, n, float(rms_eps),
+                                                         _stream(stream), ctypes.byref(h)), "kvd_scaffold_linear_create")
+        return Linear(self, h, k, n, int(self._lib.kvd_scaffold_linear_out_cols(h)))
+
+    def kvd_scaffold_linear(self, lin: "Linear", x, m: int, out, out_row_stride: int, stream=None) -> None:
+        self._check(self._lib.kvd_scaffold_linear(self._h, lin._h, _ptr(x), m, _ptr(out), out_row_stride,
+                                                  _stream(stream)), "kvd_scaffold_linear")
+
+    def kvd_scaffold_query_finish(self, layer: int, q_in, in_row_stride: int, positions, m: int, gamma_q, q_out,
+                                  stream=None) -> None:
+        self._check(self._lib.kvd_scaffold_query_finish(self._h, layer, _ptr(q_in), in_row_stride, _ptr(positions), m,
+                                                        _ptr(gamma_q), _ptr(q_out), _stream(stream)),
+                    "kvd_scaffold_query_finish")
+
+    def kvd_scaffold_add_rows(self, h, y, y_row_stride: int, m: int, d: int, stream=None) -> None:
+        self._check(self._lib.kvd_scaffold_add_rows(self._h, _ptr(h), _ptr(y), y_row_stride, m, d, _stream(stream)),
+                    "kvd_scaffold_add_rows")
+
+    def kvd_scaffold_gated_act(self, gate_up, row_stride: int, m: int, width: int, activation: int, out,
+                               stream=None) -> None:
+        self._check(self._lib.kvd_scaffold_gated_act(self._h, _ptr(gate_up), row_stride, m, width, activation,
+                                                     _ptr(out), _stream(stream)), "kvd_scaffold_gated_act")
+
+    def kvd_scaffold_embed(self, table, tokens, m: int, d: int, vocab: int, out, stream=None) -> None:
+        self._check(self._lib.kvd_scaffold_embed(self._h, _ptr(table), _ptr(tokens), m, d, vocab, _ptr(out),
+                                                 _stream(stream)), "kvd_scaffold_embed")
+
+    def kvd_scaffold_argmax(self, logits, row_stride: int, m: int, n: int, tokens_out, stream=None) -> None:
+        self._check(self._lib.kvd_scaffold_argmax(self._h, _ptr(logits), row_stride, m, n, _ptr(tokens_out),
+                                                  _stream(stream)), "kvd_scaffold_argmax")
+
+
+class Linear:
+    """Handle of one prepared weight matrix (kvd_scaffold_linear_create); freed with its context or by close()."""
+
+    def __init__(self, ctx: Kvd, h, k: int, n: int, out_cols: int):
+        self._ctx, self._h, self.k, self.n, self.out_cols = ctx, h, k, n, out_cols
+
+    def close(self) -> None:
+        if self._h and getattr(self._ctx, "_h", None):
+            self._ctx._lib.kvd_scaffold_linear_destroy(self._ctx._h, self._h)
+        self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -168,14 +168,16 @@ extern "C" void kvd_destroy(kvd_ctx *ctx) {
   }
   if (ctx->d_status) cudaFree(ctx->d_status);
   if (ctx->ext_sumsq) cudaFree(ctx->ext_sumsq);
+  if (ctx->zero_pos) cudaFree(ctx->zero_pos);
   if (ctx->amax_scratch) cudaFree(ctx->amax_scratch);
   cudaGetLastError();
   delete ctx;
 }
 
 // (eb = bytes per element: 2 for bf16, 1 for the FP8 variant's codes; a box row is 128 bytes either way)
-static kvd_status encode_2d(kvd_ctx *ctx, CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer,
-                            uint32_t box_inner, uint32_t box_outer, int eb = 2) {
+namespace kvd {
+kvd_status encode_2d(kvd_ctx *ctx, CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer,
+                     uint32_t box_inner, uint32_t box_outer, int eb) {
   cuuint64_t dims[2] = {inner, outer};
   cuuint64_t strides[1] = {inner * eb};
   cuuint32_t box[2] = {box_inner, box_outer};
@@ -194,8 +196,8 @@ static kvd_status encode_2d(kvd_ctx *ctx, CUtensorMap *map, const void *base, ui
 }
 
 // Row source of the recompute GEMM as a 3-D map [slabs][rows][d_hidden]; box = one 128 x 64 tile.
-static kvd_status encode_rows_3d(kvd_ctx *ctx, CUtensorMap *map, const void *base, uint64_t d_hidden, uint64_t rows,
-                                 uint64_t slabs, int eb = 2) {
+kvd_status encode_rows_3d(kvd_ctx *ctx, CUtensorMap *map, const void *base, uint64_t d_hidden, uint64_t rows,
+                          uint64_t slabs, int eb) {
   cuuint64_t dims[3] = {d_hidden, rows, slabs};
   cuuint64_t strides[2] = {d_hidden * eb, rows * d_hidden * eb};
   cuuint32_t box[3] = {static_cast<cuuint32_t>(RC_BLOCK_K * 2 / eb), RC_BLOCK_M, 1};
@@ -216,7 +218,7 @@ static kvd_status encode_rows_3d(kvd_ctx *ctx, CUtensorMap *map, const void *bas
 // (cos, sin) tables of Eq. 11-12 split as position = 16*hi + lo; built in double on the host.
 // hi is row-major [hi][pair]; lo is pair-major [pair][lo] so that neighbouring positions read
 // neighbouring shared-memory words.
-static kvd_status get_rope(kvd_ctx *ctx, float theta, RopeTable *out) {
+kvd_status get_rope(kvd_ctx *ctx, float theta, RopeTable *out) {
   uint32_t key;
   memcpy(&key, &theta, 4);
   auto it = ctx->rope_cache.find(key);
@@ -250,6 +252,7 @@ static kvd_status get_rope(kvd_ctx *ctx, float theta, RopeTable *out) {
   *out = t;
   return KVD_OK;
 }
+}  // namespace kvd
 
 extern "C" kvd_status kvd_set_dtype(kvd_ctx *ctx, int dtype) {
   if (!ctx || (dtype != KVD_DTYPE_BF16 && dtype != KVD_DTYPE_F16 && dtype != KVD_DTYPE_F32)) return KVD_ERR_INVALID_ARG;

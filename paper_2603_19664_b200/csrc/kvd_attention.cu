@@ -17,6 +17,8 @@
 #include <math_constants.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "kvd_internal.h"
 #include "kvd_ptx.cuh"
 
@@ -802,22 +804,22 @@ namespace kvd {
 // Device address of g_kvd_static_scratch on the current device.  The array's name is only a host-side
 // handle; the address a kernel can use comes from cudaGetSymbolAddress, looked up once per device.
 static kvd_status static_scratch_address(unsigned char **out) {
-  static unsigned char *cached[64] = {};
+  static std::atomic<unsigned char *> cached[64] = {};  // host threads may make a device's first call together
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) {
     cudaGetLastError();
     return KVD_ERR_UNSUPPORTED;
   }
   if (dev < 0 || dev >= 64) return KVD_ERR_UNSUPPORTED;
-  if (cached[dev] == nullptr) {
+  if (cached[dev].load(std::memory_order_acquire) == nullptr) {
     void *p = nullptr;
     if (cudaGetSymbolAddress(&p, g_kvd_static_scratch) != cudaSuccess || p == nullptr) {
       cudaGetLastError();
       return KVD_ERR_CUDA;
     }
-    cached[dev] = static_cast<unsigned char *>(p);
+    cached[dev].store(static_cast<unsigned char *>(p), std::memory_order_release);
   }
-  *out = cached[dev];
+  *out = cached[dev].load(std::memory_order_acquire);
   return KVD_OK;
 }
 

@@ -214,6 +214,7 @@ struct kvd_ctx {
   float *store_sumsq = nullptr;
   float *ext_sumsq = nullptr;     // statistics of caller rows taken ahead of the recompute kernel
   size_t ext_sumsq_rows = 0;
+  int32_t *zero_pos = nullptr;    // ext_sumsq_rows zeros: the positions of rows that are not rotated (scaffold products)
   int layers_stored = 0;
   std::vector<int> rows_stored;  // [layers_stored * max_seqs]
   std::vector<CUtensorMap> store_maps;  // per stored layer: [max_seqs][max_tokens_per_seq][d_hidden]
@@ -277,4 +278,10 @@ kvd_status launch_checkpoint(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int3
                              int32_t *dst_pos, float *dst_sumsq, int n, int d_hidden, cudaStream_t stream);
 kvd_status launch_selftest_timeout(kvd_ctx *ctx, unsigned long long timeout_ns, cudaStream_t stream);
 kvd_status cuda_fail(kvd_ctx *ctx, cudaError_t e, const char *where);
+// host helpers shared by the entry points (kvd_api.cu)
+kvd_status encode_2d(kvd_ctx *ctx, CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer,
+                     uint32_t box_inner, uint32_t box_outer, int eb = 2);
+kvd_status encode_rows_3d(kvd_ctx *ctx, CUtensorMap *map, const void *base, uint64_t d_hidden, uint64_t rows,
+                          uint64_t slabs, int eb = 2);
+kvd_status get_rope(kvd_ctx *ctx, float theta, RopeTable *out);
 }  // namespace kvd

@@ -35,7 +35,7 @@ def run_session(stack, weights, turns, gen, window, seg_lo, seg_hi, max_tokens, 
     rng = np.random.Generator(np.random.PCG64(SEED_TOKENS + 77))
     segments = [rng.integers(0, stack.vocab, size=int(rng.integers(seg_lo, seg_hi + 1))).tolist() for _ in range(turns)]
     if chained:
-        full = GpuStack(stack, weights, "full", 0, max_tokens, device_weights, exact_scaffold=True)
+        full = GpuStack(stack, weights, "full", 0, max_tokens, device_weights)
         kvdir = GpuStackChained(stack, weights, window, max_tokens, device_weights)
     else:
         full = GpuStack(stack, weights, "full", 0, max_tokens, device_weights)
@@ -48,7 +48,7 @@ def run_session(stack, weights, turns, gen, window, seg_lo, seg_hi, max_tokens, 
             logits = m.prefill(segments[t])
             toks = []
             for _ in range(gen):
-                nxt = int(torch.argmax(logits).item())
+                nxt = m.greedy_token()
                 toks.append(nxt)
                 logits = m.step(nxt)
             torch.cuda.synchronize()

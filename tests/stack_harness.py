@@ -1,10 +1,12 @@
 """Test scaffold: a whole decoder stack driven one token at a time on the GPU (Algorithm 1).
 
 The hot path -- checkpointing residual rows, K/V (re)computation and decode attention -- goes through
-the C ABI of the library.  Everything around it (embedding lookup, Q projection with q-norm and
-rotation, W_o, the gated MLP, the final norm, the vocabulary projection and the argmax) is plain
-torch arithmetic: it is scaffolding that both cache policies share line for line, needed only to
-produce realistic residual streams and to turn attention outputs into tokens.
+the C ABI of the library (include/kvd.h).  Everything around it (embedding lookup, Q projection with
+q-norm and rotation, W_o, the gated MLP, the final norm, the vocabulary projection and the greedy
+pick) goes through the library's scaffold entry points (include/kvd_scaffold.h): the dense products
+run on the same tcgen05 kernel as the K/V projection, the small steps between them are plain kernels.
+torch only allocates device memory and copies tensors; no torch arithmetic is on the path.  Both
+cache policies share the scaffold line for line.
 
 Cache policies, as in the oracle's stack:
   * "full"      every token's K/V is kept; attention reads one stored segment;
@@ -16,18 +18,15 @@ Cache policies, as in the oracle's stack:
                 layer next to the new tokens, so that each layer's K/V of the evicted tokens exist only
                 while that layer runs.  This is the variant whose memory is Eq. 24 / Eq. 28.
 
-`exact_scaffold=True` makes the scaffold's matrix products and norms accumulate in fp64 before
-rounding to bf16: their bf16 results then do not depend on how many rows are processed at once
-(the library's kernels have that property by construction), which the chained variant needs to
-reproduce the first pass bit for bit when it replays tokens in different batches.
+A row's result in every scaffold step depends on that row alone (the dense products inherit this from
+the recompute kernel), so replaying tokens in batches of another size reproduces the first pass bit
+for bit -- which the chained variant relies on.
 """
-import math
-
 import numpy as np
 import torch
 
 import paper_2603_19664_b200 as kvd
-from kvd_synth import ROPE_HALF
+from paper_2603_19664_b200.binding import KVD_ACT_GELU_TANH, KVD_ACT_SILU
 
 
 def _dev(bits):
@@ -61,36 +60,40 @@ def torch_stack_weights(stack, seed=0):
 
 class GpuStack:
     def __init__(self, stack, weights, policy="full", budget=0, max_tokens=512, device_weights=False,
-                 exact_scaffold=False, layers_stored=None):
+                 layers_stored=None):
         assert policy in ("full", "kvdirect")
         self.s, self.policy, self.budget, self.max_tokens = stack, policy, int(budget), max_tokens
-        self.exact = bool(exact_scaffold)
         s = stack
         self.kdim = s.n_kv_heads * s.d_head
         if device_weights:
-            self.embed, self.lm_head = weights["embed"], weights["lm_head"]
-            self.g_final = weights["gamma_final"].float()
+            self.embed, lm_head, g_final = weights["embed"], weights["lm_head"], weights["gamma_final"]
             self.lw = weights["layers"]
         else:
-            self.embed = _dev(weights.embed)
-            self.lm_head = _dev(weights.lm_head)
-            self.g_final = _dev(weights.gamma_final).float()
-            self.lw = []
-            for lw in weights.layers:
-                d = {k: _dev(v) for k, v in lw.items()}
-                self.lw.append(d)
+            self.embed, lm_head, g_final = _dev(weights.embed), _dev(weights.lm_head), _dev(weights.gamma_final)
+            self.lw = [{k: _dev(v) for k, v in lw.items()} for lw in weights.layers]
         desc = kvd.make_desc(s.n_layers, s.d_hidden, s.n_q_heads, s.n_kv_heads, s.d_head, s.rms_eps, s.qk_norm,
                              s.rms_eps, s.rope_style, 1, max_tokens, 64)
-        self.ctx = kvd.Kvd(desc)
+        self.ctx = ctx = kvd.Kvd(desc)
+        self.act = KVD_ACT_SILU if s.activation == "silu" else KVD_ACT_GELU_TANH
+        self.lin = []
         for l in range(s.n_layers):
-            ls = s.layer_shape(l)
-            self.ctx.kvd_set_layer(l, self.lw[l]["w_kv"], self.lw[l]["gamma_in"],
-                                   self.lw[l].get("gamma_k") if s.qk_norm else None, ls.rope_theta, ls.sliding_window)
+            ls, lw = s.layer_shape(l), self.lw[l]
+            ctx.kvd_set_layer(l, lw["w_kv"], lw["gamma_in"], lw.get("gamma_k") if s.qk_norm else None, ls.rope_theta,
+                              ls.sliding_window)
+            # the scaffold's products, each prepared once: RMSNorm scales folded where a norm precedes the product
+            gate_up = torch.cat([lw["w_gate"], lw["w_up"]], dim=1).contiguous()
+            self.lin.append({
+                "q": ctx.kvd_scaffold_linear_create(lw["w_q"], lw["gamma_in"], s.d_hidden, s.n_q_heads * s.d_head, s.rms_eps),
+                "o": ctx.kvd_scaffold_linear_create(lw["w_o"], None, s.n_q_heads * s.d_head, s.d_hidden),
+                "gate_up": ctx.kvd_scaffold_linear_create(gate_up, lw["gamma_mlp"], s.d_hidden, 2 * s.d_mlp, s.rms_eps),
+                "down": ctx.kvd_scaffold_linear_create(lw["w_down"], None, s.d_mlp, s.d_hidden)})
+            del gate_up
+        self.lin_head = ctx.kvd_scaffold_linear_create(lm_head, g_final, s.d_hidden, s.vocab, s.rms_eps)
         self.ws = torch.empty(kvd.kvd_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
-        self.ctx.kvd_attach_workspace(self.ws)
+        ctx.kvd_attach_workspace(self.ws)
         n_stored = s.n_layers if layers_stored is None else layers_stored
         self.arena = torch.empty(kvd.kvd_store_bytes(desc, n_stored), dtype=torch.uint8, device="cuda")
-        self.ctx.kvd_attach_store(self.arena, n_stored)
+        ctx.kvd_attach_store(self.arena, n_stored)
         # K/V storage indexed by position: the full cache, or the live window of the bounded policy
         self.k_live = [torch.zeros((max_tokens, self.kdim), dtype=torch.bfloat16, device="cuda") for _ in range(s.n_layers)]
         self.v_live = [torch.zeros((max_tokens, self.kdim), dtype=torch.bfloat16, device="cuda") for _ in range(s.n_layers)]
@@ -99,82 +102,64 @@ class GpuStack:
         self.win_first = [0] * s.n_layers
         self.t = 0
         self.recomputed_rows = 0
-        # rotation angles for q (scaffold side), fp64 on the host like the library's tables
-        self.inv_freq = {}
+        self.logits_bf16 = None  # [1, padded vocab] of the last token processed
 
-    def _rms(self, x, gamma):
-        if self.exact:
-            xd = x.double()
-            return (xd * torch.rsqrt(xd.pow(2).mean(-1, keepdim=True) + self.s.rms_eps) * gamma.double()).float()
-        xf = x.float()
-        return xf * torch.rsqrt(xf.pow(2).mean(-1, keepdim=True) + self.s.rms_eps) * gamma.float()
-
-    def _mm(self, x, w):
-        """bf16 x @ bf16 w -> bf16 (fp64 accumulation when exact_scaffold)."""
-        if self.exact:
-            return (x.double() @ w.double()).to(torch.bfloat16)
-        return x @ w
-
-    def _qnorm(self, q, gamma_q):
-        if self.exact:
-            qd = q.double()
-            return (qd * torch.rsqrt(qd.pow(2).mean(-1, keepdim=True) + self.s.rms_eps) * gamma_q.double()).float()
-        return q * torch.rsqrt(q.pow(2).mean(-1, keepdim=True) + self.s.rms_eps) * gamma_q.float()
-
-    def _queries(self, l, h, positions):
-        """Scaffold: normalised, rotated bf16 queries [U, n_q, d_head] of residual rows h [U, d]."""
-        s, lw, ls = self.s, self.lw[l], self.s.layer_shape(l)
-        xb = self._rms(h, lw["gamma_in"]).to(torch.bfloat16)
-        q = self._mm(xb, lw["w_q"]).float().view(h.shape[0], s.n_q_heads, s.d_head)
-        if s.qk_norm:
-            q = self._qnorm(q, lw["gamma_q"])
-        return self._rope_q(q, positions, ls.rope_theta).to(torch.bfloat16).contiguous()
-
-    def _after_attention(self, l, h, out):
-        """Scaffold: W_o, residual add, gated MLP, residual add (Eq. 8-9) for rows h [U, d]."""
-        lw = self.lw[l]
-        h = (h.float() + self._mm(out.view(h.shape[0], -1), lw["w_o"]).float()).to(torch.bfloat16)
-        xm = self._rms(h, lw["gamma_mlp"]).to(torch.bfloat16)
-        gate = self._act(self._mm(xm, lw["w_gate"]).float()) * self._mm(xm, lw["w_up"]).float()
-        mlp = self._mm(gate.to(torch.bfloat16), lw["w_down"])
-        return (h.float() + mlp.float()).to(torch.bfloat16)
-
-    def _rope_q(self, q, pos, theta):
-        """q: [..., n_q, d_head] with `pos` an int or a list of positions (one per leading row)."""
-        s = self.s
-        half = s.d_head // 2
-        key = float(theta)
-        if key not in self.inv_freq:
-            self.inv_freq[key] = torch.tensor([theta ** (-2.0 * i / s.d_head) for i in range(half)], dtype=torch.float64)
-        if isinstance(pos, int):
-            ang = (self.inv_freq[key] * pos)
-        else:
-            ang = torch.tensor(pos, dtype=torch.float64)[:, None, None] * self.inv_freq[key]  # [U, 1, half]
-        c, sn = torch.cos(ang).float().cuda(), torch.sin(ang).float().cuda()
-        if s.rope_style == ROPE_HALF:
-            a, b = q[..., :half], q[..., half:]
-            return torch.cat([a * c - b * sn, a * sn + b * c], dim=-1)
-        a, b = q[..., 0::2], q[..., 1::2]
-        out = torch.empty_like(q)
-        out[..., 0::2] = a * c - b * sn
-        out[..., 1::2] = a * sn + b * c
+    # ---- scaffold steps (include/kvd_scaffold.h); every tensor made here is an output buffer
+    def _linear(self, lin, x):
+        m = x.shape[0]
+        out = torch.empty((m, lin.out_cols), dtype=torch.bfloat16, device="cuda")
+        self.ctx.kvd_scaffold_linear(lin, x, m, out, lin.out_cols)
         return out
 
-    def _act(self, x):
-        if self.s.activation == "silu":
-            return torch.nn.functional.silu(x)
-        return torch.nn.functional.gelu(x, approximate="tanh")
+    def _embed_rows(self, tokens):
+        tok = torch.tensor([int(t) for t in tokens], dtype=torch.int32, device="cuda")
+        h = torch.empty((len(tokens), self.s.d_hidden), dtype=torch.bfloat16, device="cuda")
+        self.ctx.kvd_scaffold_embed(self.embed, tok, len(tokens), self.s.d_hidden, self.s.vocab, h)
+        return h
+
+    def _queries(self, l, h, positions):
+        """Normalised, rotated bf16 queries [U, n_q, d_head] of residual rows h [U, d] (Eq. 3)."""
+        s, U = self.s, h.shape[0]
+        raw = self._linear(self.lin[l]["q"], h)
+        pos_t = positions if torch.is_tensor(positions) else torch.tensor(list(positions), dtype=torch.int32, device="cuda")
+        q = torch.empty((U, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
+        self.ctx.kvd_scaffold_query_finish(l, raw, raw.shape[1], pos_t, U, self.lw[l].get("gamma_q") if s.qk_norm else None, q)
+        return q
+
+    def _after_attention(self, l, h, out):
+        """W_o, residual add, gated MLP, residual add (Eq. 8-9) for rows h [U, d]; returns the new rows."""
+        s, ctx, U = self.s, self.ctx, h.shape[0]
+        h = h.clone()
+        y = self._linear(self.lin[l]["o"], out.view(U, -1))
+        ctx.kvd_scaffold_add_rows(h, y, y.shape[1], U, s.d_hidden)
+        gu = self._linear(self.lin[l]["gate_up"], h)
+        inner = torch.empty((U, s.d_mlp), dtype=torch.bfloat16, device="cuda")
+        ctx.kvd_scaffold_gated_act(gu, gu.shape[1], U, s.d_mlp, self.act, inner)
+        y = self._linear(self.lin[l]["down"], inner)
+        ctx.kvd_scaffold_add_rows(h, y, y.shape[1], U, s.d_hidden)
+        return h
+
+    def _logits(self, h_last):
+        """Final norm and vocabulary projection of one row; keeps the bf16 logits for greedy_token()."""
+        self.logits_bf16 = self._linear(self.lin_head, h_last)
+        return self.logits_bf16[0, :self.s.vocab].float()
+
+    def greedy_token(self):
+        """Index of the largest logit of the last processed token (lowest index on ties), picked on the GPU."""
+        tok = torch.empty((1,), dtype=torch.int32, device="cuda")
+        self.ctx.kvd_scaffold_argmax(self.logits_bf16, self.logits_bf16.shape[1], 1, self.s.vocab, tok)
+        return int(tok.item())
 
     def step(self, token):
         s, ctx, pos = self.s, self.ctx, self.t
         assert pos < self.max_tokens
-        h = self.embed[token].clone().view(1, -1)  # bf16 residual stream
+        h = self._embed_rows([token])  # bf16 residual stream
         pos_t = torch.tensor([pos], dtype=torch.int32, device="cuda")
         for l in range(s.n_layers):
             lw, ls = self.lw[l], s.layer_shape(l)
             ctx.kvd_checkpoint_residual(0, l, h, pos_t, 1)  # STORE_RESIDUAL: the row entering layer l
             # scaffold: query
-            q = self._queries(l, h, [pos])
+            q = self._queries(l, h, pos_t)
             # hot path: K_t, V_t of the current token, written at its position in the live storage
             kl, vl = self.k_live[l], self.v_live[l]
             lo = 0 if ls.sliding_window == 0 else max(0, pos - ls.sliding_window + 1)
@@ -202,10 +187,6 @@ class GpuStack:
         self.t += 1
         return self._logits(h)
 
-    def _logits(self, h_last):
-        hf = self._rms(h_last, self.g_final).to(torch.bfloat16)
-        return self._mm(hf, self.lm_head).float().view(-1)
-
     def prefill(self, tokens):
         """Process a whole segment of tokens at once (every token attends to the keys up to its own
         position: the decode-attention call is issued with one "sequence" per segment token).  Returns
@@ -213,14 +194,13 @@ class GpuStack:
         s, ctx = self.s, self.ctx
         U, p0 = len(tokens), self.t
         assert p0 + U <= self.max_tokens
-        tok = torch.tensor(tokens, dtype=torch.long, device="cuda")
-        h = self.embed[tok].clone()  # [U, d] bf16
+        h = self._embed_rows(tokens)  # [U, d] bf16
         positions = list(range(p0, p0 + U))
         pos_t = torch.arange(p0, p0 + U, dtype=torch.int32, device="cuda")
         for l in range(s.n_layers):
             lw, ls = self.lw[l], s.layer_shape(l)
             ctx.kvd_checkpoint_residual(0, l, h, pos_t, U)
-            q = self._queries(l, h, positions)
+            q = self._queries(l, h, pos_t)
             kl, vl = self.k_live[l], self.v_live[l]
             ctx.kvd_recompute_kv(l, h, pos_t, U, kl[p0:], vl[p0:], self.kdim)
             lo_min = 0 if ls.sliding_window == 0 else max(0, p0 - ls.sliding_window + 1)
@@ -249,7 +229,7 @@ class GpuStack:
             logits = self.step(int(tok))
         toks, lgs = [], []
         for i in range(n_new):
-            nxt = int(torch.argmax(logits).item())
+            nxt = self.greedy_token()
             toks.append(nxt)
             lgs.append(logits.clone())
             if i + 1 < n_new:
@@ -275,9 +255,9 @@ class GpuStackChained(GpuStack):
     their current rows (the same kvd_recompute_kv as ever), serve the new tokens' attention and the
     evicted tokens' own causal attention, and are dropped when the rows move on to layer l + 1."""
 
-    def __init__(self, stack, weights, budget=0, max_tokens=512, device_weights=False, exact_scaffold=True):
+    def __init__(self, stack, weights, budget=0, max_tokens=512, device_weights=False):
         super().__init__(stack, weights, policy="kvdirect", budget=budget, max_tokens=max_tokens,
-                         device_weights=device_weights, exact_scaffold=exact_scaffold, layers_stored=1)
+                         device_weights=device_weights, layers_stored=1)
         # the layer-0 rows as the library stores them (documented arena layout)
         self.rows0 = self.arena[:max_tokens * stack.d_hidden * 2].view(torch.bfloat16).view(max_tokens, stack.d_hidden)
         self.replayed_rows = 0
@@ -289,8 +269,7 @@ class GpuStackChained(GpuStack):
         s, ctx = self.s, self.ctx
         U, p0 = len(tokens), self.t
         assert p0 + U <= self.max_tokens
-        tok = torch.tensor(tokens, dtype=torch.long, device="cuda")
-        h_new = self.embed[tok].clone()
+        h_new = self._embed_rows(tokens)
         pos_new = list(range(p0, p0 + U))
         pos_new_t = torch.arange(p0, p0 + U, dtype=torch.int32, device="cuda")
         ctx.kvd_checkpoint_residual(0, 0, h_new, pos_new_t, U)  # STORE_RESIDUAL: one row per token
@@ -309,7 +288,7 @@ class GpuStackChained(GpuStack):
                 self.recomputed_rows += N
                 segs_new.append((self.k_old, self.v_old, self.kdim, 0, N))
             segs_new.append((kl[N:], vl[N:], self.kdim, N, p0 + U - N))
-            q_new = self._queries(l, h_new, pos_new)
+            q_new = self._queries(l, h_new, pos_new_t)
             out_new = torch.empty((U, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
             for b0 in range(0, U, 64):
                 nb = min(64, U - b0)
@@ -317,7 +296,7 @@ class GpuStackChained(GpuStack):
             if N > 0 and l + 1 < s.n_layers:
                 # the evicted tokens' own step through this layer: each attends to the evicted keys up
                 # to its own position (the position mask does the rest)
-                q_old = self._queries(l, h_old, pos_old)
+                q_old = self._queries(l, h_old, pos_old_t)
                 out_old = torch.empty((N, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
                 segs_old = [(self.k_old, self.v_old, self.kdim, 0, N)]
                 for b0 in range(0, N, 64):

@@ -14,8 +14,10 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def test_library_builds_and_exports_every_declared_symbol():
     path = build()
     lib = ctypes.CDLL(path)
-    header = open(os.path.join(ROOT, "include", "kvd.h")).read()
-    declared = set(re.findall(r"\b(kvd_[a-z_0-9]+)\s*\(", header))
+    declared = set()
+    for name in sorted(os.listdir(os.path.join(ROOT, "include"))):
+        if name.endswith(".h"):
+            declared |= set(re.findall(r"\b(kvd_[a-z_0-9]+)\s*\(", open(os.path.join(ROOT, "include", name)).read()))
     declared -= {"kvd_ctx", "kvd_fp8_rows"}
     assert declared == set(binding.EXPORTED_SYMBOLS)
     for name in sorted(declared):

@@ -8,14 +8,19 @@ fixed array compiled into the library instead of a caller-provided workspace.
 This file is collected last on purpose: a run that stops at the first failure has then already run
 every other test.  The test calls the entry point through the C ABI twice in a row with different
 inputs -- the second call starts with the first call's leftovers in the shared array -- and checks
-each output against kvd_decode_attention on the same inputs, plus the size limit.
+each output against kvd_decode_attention on the same inputs and against the fp64 oracle, plus the
+size limit.  It also checks the property the entry point exists for: across a call, the device's free
+memory and the bytes held by the test's own allocator stay what they were.  A last case runs the entry
+point in a process state where no library context and no workspace exist at all.
 """
+import math
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2603_19664_b200 as kvd
-from kvd_synth import GEMMA3_4B_LOCAL, QWEN3_4B, make_kv, make_query
+from kvd_synth import GEMMA3_4B_LOCAL, QWEN3_4B, bf16_to_f64, make_kv, make_query
 from gpu_util import dev, host_f64, open_layer
 
 pytestmark = pytest.mark.gpu
@@ -36,12 +41,36 @@ def _both(ctx, shape, q_bits, q_pos, seg_bits):
         segs.append(row)
     ref = torch.full((batch, shape.n_q_heads, shape.d_head), 3.0, dtype=torch.bfloat16, device="cuda")
     got = torch.full_like(ref, -3.0)
-    ctx.kvd_decode_attention(0, batch, q, q_pos, segs, 0.0, ref)
+    if ctx is not None:
+        ctx.kvd_decode_attention(0, batch, q, q_pos, segs, 0.0, ref)
+    # a kernel's first launch in a process may make the driver load its code; measure a warmed call
+    st = kvd.kvd_decode_attention_static(shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.sliding_window,
+                                         batch, q, q_pos, segs, 0.0, got)
+    assert st == kvd.KVD_OK, kvd.status_string(st)
+    got.fill_(-3.0)
+    torch.cuda.synchronize()
+    free0, held0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
     st = kvd.kvd_decode_attention_static(shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.sliding_window,
                                          batch, q, q_pos, segs, 0.0, got)
     assert st == kvd.KVD_OK, kvd.status_string(st)
     torch.cuda.synchronize()
-    return ref, got
+    free1, held1 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+    return ref, got, (free0, held0, free1, held1)
+
+
+def _oracle(shape, q_bits, q_pos, seg_bits):
+    outs = []
+    for b in range(q_bits.shape[0]):
+        segs = [(bf16_to_f64(K), bf16_to_f64(V), first) for (K, V, first) in seg_bits[b] if K.shape[0] > 0]
+        outs.append(oracle.decode_attention(bf16_to_f64(q_bits[b]), int(q_pos[b]), segs, 1.0 / math.sqrt(shape.d_head),
+                                            shape.sliding_window))
+    return np.stack(outs)
+
+
+def _check_oracle(got, want):
+    g = host_f64(got)
+    assert np.linalg.norm(g - want) <= 1e-2 * np.linalg.norm(want)
+    assert np.max(np.abs(g - want)) <= 1e-2 * np.max(np.abs(want))
 
 
 def _check(ref, got):
@@ -65,8 +94,9 @@ def test_static_scratch_matches_workspace_path_on_two_calls_in_a_row():
         cut = max(1, T - 257)
         segs.append([(K[:cut], V[:cut], 0), (K[cut:T - 1], V[cut:T - 1], cut), (K[T - 1:], V[T - 1:], T - 1)])
         qpos.append(T - 1)
-    ref, got = _both(ctx, shape, q, qpos, segs)
+    ref, got, _ = _both(ctx, shape, q, qpos, segs)  # the first call on a device also looks the array up
     _check(ref, got)
+    _check_oracle(got, _oracle(shape, q, qpos, segs))
     ctx.close()
 
     # call 2 right after: another model shape, longer context; the array still holds call 1's partials
@@ -78,8 +108,12 @@ def test_static_scratch_matches_workspace_path_on_two_calls_in_a_row():
         K, V = make_kv(shape, T, seed=70 + b)
         segs.append([(K, V, 0)])
         qpos.append(T - 1)
-    ref, got = _both(ctx, shape, q, qpos, segs)
+    ref, got, (free0, held0, free1, held1) = _both(ctx, shape, q, qpos, segs)
     _check(ref, got)
+    _check_oracle(got, _oracle(shape, q, qpos, segs))
+    # the call allocated nothing: neither from the driver nor from the allocator this test's tensors come from
+    assert free1 == free0, f"free device memory moved by {free0 - free1} bytes across the call"
+    assert held1 == held0
 
     # a request whose partials cannot fit the fixed array is refused, and nothing is launched
     T = 16000
@@ -99,3 +133,20 @@ def test_static_scratch_matches_workspace_path_on_two_calls_in_a_row():
                                          [[]] * 65, 0.0, out)
     assert st == 4
     ctx.close()
+
+
+def test_static_entry_point_needs_no_context_or_workspace():
+    # no kvd context alive, no workspace attached anywhere: shapes are passed directly
+    import gc
+    gc.collect()
+    shape = GEMMA3_4B_LOCAL
+    lens = [777, 2100]
+    q = make_query(shape, 2, seed=44)
+    segs, qpos = [], []
+    for b, T in enumerate(lens):
+        K, V = make_kv(shape, T, seed=90 + b)
+        segs.append([(K[:T - 1], V[:T - 1], 0), (K[T - 1:], V[T - 1:], T - 1)])
+        qpos.append(T - 1)
+    _, got, (free0, held0, free1, held1) = _both(None, shape, q, qpos, segs)
+    _check_oracle(got, _oracle(shape, q, qpos, segs))
+    assert free1 == free0 and held1 == held0
