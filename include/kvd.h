@@ -192,6 +192,14 @@ kvd_status kvd_attach_workspace(kvd_ctx *ctx, void *workspace, size_t bytes);
 kvd_status kvd_checkpoint_residual(kvd_ctx *ctx, int seq, int layer, const void *rows, const int32_t *positions,
                                    int n, void *stream);
 
+/* STORE_RESIDUAL(C, l) for one decode step of a batch, in ONE launch: row i of rows (DEVICE bf16
+ * [n, d_hidden], 16-byte aligned; positions DEVICE int32 [n]) is appended to the store of (layer, seqs[i]),
+ * exactly as kvd_checkpoint_residual would append it (same bits, same statistic).  seqs is a HOST array of
+ * n <= KVD_MAX_STORE_RANGES sequence slots; a slot may occur more than once (its rows are appended in order).
+ * Nothing is stored when any entry is rejected. */
+kvd_status kvd_checkpoint_residual_step(kvd_ctx *ctx, int layer, int n, const int32_t *seqs, const void *rows,
+                                        const int32_t *positions, void *stream);
+
 /* RECOMPUTE_KV(C, l), Eq. 13-14.
  *   rows != NULL: DEVICE bf16 [n, d_hidden] (16-byte aligned) with DEVICE int32 positions[n];
  *                 seq and first_row are ignored.  This is also how (K_t, V_t) of new tokens is made.

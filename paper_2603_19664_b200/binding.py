@@ -34,7 +34,7 @@ EXPORTED_SYMBOLS = (
     "kvd_decode_attention_recompute", "kvd_decode_attention_recompute_fp8", "kvd_set_dtype", "kvd_store_bytes_dtype",
     "kvd_quantize_rows_fp8", "kvd_recompute_kv_fp8_rows", "kvd_decode_attention_recompute_fp8_rows",
     "kvd_store_bytes_fp8", "kvd_attach_store_fp8", "kvd_rows_stored_fp8", "kvd_reset_sequence_fp8", "kvd_checkpoint_residual_fp8", "kvd_recompute_kv_fp8",
-    "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_recompute_kv",
+    "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_checkpoint_residual_step", "kvd_recompute_kv",
     "kvd_recompute_kv_step",
     "kvd_decode_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
     "kvd_status_string", "kvd_version",
@@ -129,6 +129,8 @@ def load() -> ctypes.CDLL:
     lib.kvd_attention_split.restype = i32
     lib.kvd_checkpoint_residual.argtypes = [vp, i32, i32, vp, vp, i32, vp]
     lib.kvd_checkpoint_residual.restype = i32
+    lib.kvd_checkpoint_residual_step.argtypes = [vp, i32, i32, ctypes.POINTER(ctypes.c_int32), vp, vp, vp]
+    lib.kvd_checkpoint_residual_step.restype = i32
     lib.kvd_recompute_kv.argtypes = [vp, i32, vp, vp, i32, i32, i32, vp, vp, i64, vp]
     lib.kvd_recompute_kv.restype = i32
     lib.kvd_recompute_kv_step.argtypes = [vp, i32, ctypes.POINTER(kvd_store_range), i32, vp, vp, i32, vp, vp, i64, vp]
@@ -346,6 +348,11 @@ class Kvd:
     def kvd_checkpoint_residual(self, seq: int, layer: int, rows, positions, n: int, stream=None) -> None:
         self._check(self._lib.kvd_checkpoint_residual(self._h, seq, layer, _ptr(rows), _ptr(positions), n,
                                                       _stream(stream)), "kvd_checkpoint_residual")
+
+    def kvd_checkpoint_residual_step(self, layer: int, seqs: Sequence[int], rows, positions, stream=None) -> None:
+        arr = (ctypes.c_int32 * max(len(seqs), 1))(*[int(s) for s in seqs])
+        self._check(self._lib.kvd_checkpoint_residual_step(self._h, layer, len(seqs), arr, _ptr(rows), _ptr(positions),
+                                                           _stream(stream)), "kvd_checkpoint_residual_step")
 
     def kvd_recompute_kv(self, layer: int, rows, positions, n: int, k_out, v_out, out_row_stride: int, seq: int = 0,
                          first_row: int = 0, stream=None) -> None:

@@ -408,6 +408,33 @@ extern "C" kvd_status kvd_checkpoint_residual(kvd_ctx *ctx, int seq, int layer, 
   return st;
 }
 
+extern "C" kvd_status kvd_checkpoint_residual_step(kvd_ctx *ctx, int layer, int n, const int32_t *seqs, const void *rows,
+                                                   const int32_t *positions, void *stream_) {
+  if (!ctx || n < 0) return KVD_ERR_INVALID_ARG;
+  if (!ctx->store_rows) return KVD_ERR_STATE;
+  if (layer < 0 || layer >= ctx->layers_stored) return KVD_ERR_INVALID_ARG;
+  if (n == 0) return KVD_OK;
+  if (n > KVD_MAX_STORE_RANGES) return KVD_ERR_CAPACITY;
+  if (!seqs || !rows || !positions) return KVD_ERR_INVALID_ARG;
+  if (!aligned16(rows)) return KVD_ERR_ALIGNMENT;
+  // validate everything before any count moves
+  std::vector<int> add(ctx->desc.max_seqs, 0);
+  CkptSlots slots;
+  for (int i = 0; i < n; ++i) {
+    const int s = seqs[i];
+    if (s < 0 || s >= ctx->desc.max_seqs) return KVD_ERR_INVALID_ARG;
+    const int count = ctx->rows_stored[static_cast<size_t>(layer) * ctx->desc.max_seqs + s] + add[s];
+    if (count + 1 > ctx->desc.max_tokens_per_seq) return KVD_ERR_CAPACITY;
+    slots.slot[i] = static_cast<long long>(store_slot(ctx, layer, s) + count);
+    add[s] += 1;
+  }
+  kvd_status st = launch_checkpoint_scatter(ctx, static_cast<const __nv_bfloat16 *>(rows), positions, slots, n,
+                                            ctx->desc.d_hidden, static_cast<cudaStream_t>(stream_));
+  if (st == KVD_OK)
+    for (int s = 0; s < ctx->desc.max_seqs; ++s) ctx->rows_stored[static_cast<size_t>(layer) * ctx->desc.max_seqs + s] += add[s];
+  return st;
+}
+
 // The launch parameters every variant of the recompute kernel shares (jobs are filled in by the caller).
 static void fill_launch_params(const kvd_ctx *ctx, const LayerState &ls, RecomputeParams &p, int n_jobs, int m_blocks,
                                int k_blocks, int64_t out_row_stride) {

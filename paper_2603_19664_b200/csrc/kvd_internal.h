@@ -32,6 +32,11 @@ constexpr int RC_TRACE_TILES = 8;    // tiles per CTA recorded when a trace buff
 constexpr int RC_TRACE_FIELDS = 16;  // int64 slots per (CTA, tile); see kvd_set_trace
 constexpr int RC_THREADS = 320;  // warp 2 TMA, warp 3 MMA, warps 0,1,8,9 row statistics, warps 4-7 epilogue
 
+// store slots of the rows of kvd_checkpoint_residual_step (one new row per sequence of a batch)
+struct CkptSlots {
+  long long slot[KVD_MAX_STORE_RANGES];
+};
+
 constexpr int RC_MAX_JOBS = 65;  // row sources per launch: up to 64 store ranges and one caller buffer
 
 // One source of rows inside a launch.  Jobs own consecutive runs of 256-row blocks.
@@ -276,6 +281,8 @@ kvd_status launch_recompute_fp8(kvd_ctx *ctx, const LayerState &ls, const CUtens
                                 const CUtensorMap &tmap_rows, const RecomputeParams &p, cudaStream_t stream);
 kvd_status launch_checkpoint(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, __nv_bfloat16 *dst_rows,
                              int32_t *dst_pos, float *dst_sumsq, int n, int d_hidden, cudaStream_t stream);
+kvd_status launch_checkpoint_scatter(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, const CkptSlots &slots,
+                                     int n, int d_hidden, cudaStream_t stream);
 kvd_status launch_selftest_timeout(kvd_ctx *ctx, unsigned long long timeout_ns, cudaStream_t stream);
 kvd_status cuda_fail(kvd_ctx *ctx, cudaError_t e, const char *where);
 // host helpers shared by the entry points (kvd_api.cu)

@@ -82,6 +82,31 @@ __global__ void __launch_bounds__(256) kvd_checkpoint_kernel(const uint4 *__rest
   }
 }
 
+// The same for one new row per sequence of a decode batch: row r goes to slot P.slot[r] of the store
+// (rows, positions and statistics are indexed by slot), so that a whole batch is appended in one launch.
+template <int DT>
+__global__ void __launch_bounds__(256) kvd_checkpoint_scatter_kernel(const uint4 *__restrict__ rows,
+                                                                     const int32_t *__restrict__ pos,
+                                                                     uint4 *__restrict__ store_rows,
+                                                                     int32_t *__restrict__ store_pos,
+                                                                     float *__restrict__ store_sumsq, int row_chunks, int n,
+                                                                     const __grid_constant__ CkptSlots P) {
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  grid_launch_dependents();
+  for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n; r += warps) {
+    const size_t slot = static_cast<size_t>(P.slot[r]);
+    const uint4 *const src[1] = {rows + static_cast<size_t>(r) * row_chunks};
+    uint4 *const dst[1] = {store_rows + slot * row_chunks};
+    float ss[1];
+    warp_rows_sumsq<1, 10, true, DT>(src, dst, row_chunks, lane, ss);
+    if (lane == 0) {
+      store_sumsq[slot] = ss[0];
+      store_pos[slot] = pos[r];
+    }
+  }
+}
+
 // Sums of squares of n caller rows (no copy), two rows per warp and pass: what kvd_recompute_kv takes
 // ahead of the main kernel when the caller hands it more rows than that kernel's statistics warps
 // can cover under the main loop.
@@ -300,6 +325,23 @@ kvd_status launch_checkpoint(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int3
         reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint4 *>(dst_rows), dst_pos, dst_sumsq, d_hidden / 8, n);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "launch checkpoint");
+  ctx->launches += 1;
+  return KVD_OK;
+}
+
+kvd_status launch_checkpoint_scatter(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, const CkptSlots &slots,
+                                     int n, int d_hidden, cudaStream_t stream) {
+  const unsigned blocks = static_cast<unsigned>((n + 7) / 8);  // eight warps, one row each
+  const uint4 *src = reinterpret_cast<const uint4 *>(rows);
+  uint4 *dst = reinterpret_cast<uint4 *>(ctx->store_rows);
+  if (ctx->dtype == 2)
+    kvd_checkpoint_scatter_kernel<2><<<blocks, 256, 0, stream>>>(src, pos, dst, ctx->store_pos, ctx->store_sumsq, d_hidden / 4, n, slots);
+  else if (ctx->dtype == 1)
+    kvd_checkpoint_scatter_kernel<1><<<blocks, 256, 0, stream>>>(src, pos, dst, ctx->store_pos, ctx->store_sumsq, d_hidden / 8, n, slots);
+  else
+    kvd_checkpoint_scatter_kernel<0><<<blocks, 256, 0, stream>>>(src, pos, dst, ctx->store_pos, ctx->store_sumsq, d_hidden / 8, n, slots);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "launch checkpoint (batch)");
   ctx->launches += 1;
   return KVD_OK;
 }

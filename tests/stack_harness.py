@@ -314,3 +314,154 @@ class GpuStackChained(GpuStack):
         rep = super().memory_report()
         rep["checkpoint_bytes_single_row"] = rep.pop("checkpoint_bytes_per_layer_rows")
         return rep
+
+
+class BatchStack:
+    """A decode batch on a whole stack: `batch` sequences, each with `ctx_len` tokens of context behind it,
+    decoding one token per sequence and step under either cache policy from ONE shared state.
+
+    The context is synthetic (the stacks are random-init anyway): every layer's checkpointed residual rows
+    are N(0, 1) draws, and the stored K/V of the full-cache arm are those rows' K/V (RECOMPUTE_KV into the
+    cache), which is the state Algorithm 1 would have left behind: rows in C, their K/V in the cache.  The
+    full-cache arm attends over the stored K/V; the KV-Direct arm keeps the last `window` positions of the
+    same buffers as its live window and rebuilds the evicted positions from the rows every step.  Both
+    arms share the scaffold, so their tokens must be identical.
+    """
+
+    def __init__(self, stack, weights, batch, ctx_len, window, max_steps=8, seed=0):
+        self.s, self.batch, self.ctx_len, self.window = stack, batch, ctx_len, window
+        s = stack
+        self.kdim = s.n_kv_heads * s.d_head
+        self.max_tokens = ctx_len + max_steps + 8
+        self.embed = weights["embed"]
+        self.lw = weights["layers"]
+        desc = kvd.make_desc(s.n_layers, s.d_hidden, s.n_q_heads, s.n_kv_heads, s.d_head, s.rms_eps, s.qk_norm,
+                             s.rms_eps, s.rope_style, batch, self.max_tokens, batch)
+        self.ctx = ctx = kvd.Kvd(desc)
+        self.act = KVD_ACT_SILU if s.activation == "silu" else KVD_ACT_GELU_TANH
+        self.lin = []
+        for l in range(s.n_layers):
+            ls, lw = s.layer_shape(l), self.lw[l]
+            ctx.kvd_set_layer(l, lw["w_kv"], lw["gamma_in"], lw.get("gamma_k") if s.qk_norm else None, ls.rope_theta,
+                              ls.sliding_window)
+            gate_up = torch.cat([lw["w_gate"], lw["w_up"]], dim=1).contiguous()
+            self.lin.append({
+                "q": ctx.kvd_scaffold_linear_create(lw["w_q"], lw["gamma_in"], s.d_hidden, s.n_q_heads * s.d_head, s.rms_eps),
+                "o": ctx.kvd_scaffold_linear_create(lw["w_o"], None, s.n_q_heads * s.d_head, s.d_hidden),
+                "gate_up": ctx.kvd_scaffold_linear_create(gate_up, lw["gamma_mlp"], s.d_hidden, 2 * s.d_mlp, s.rms_eps),
+                "down": ctx.kvd_scaffold_linear_create(lw["w_down"], None, s.d_mlp, s.d_hidden)})
+            del gate_up
+        self.lin_head = ctx.kvd_scaffold_linear_create(weights["lm_head"], weights["gamma_final"], s.d_hidden, s.vocab,
+                                                       s.rms_eps)
+        self.ws = torch.empty(kvd.kvd_workspace_bytes(desc), dtype=torch.uint8, device="cuda")
+        ctx.kvd_attach_workspace(self.ws)
+        self.arena = torch.empty(kvd.kvd_store_bytes(desc, s.n_layers), dtype=torch.uint8, device="cuda")
+        ctx.kvd_attach_store(self.arena, s.n_layers)
+        mt = self.max_tokens
+        self.k_cache = [torch.zeros((batch, mt, self.kdim), dtype=torch.bfloat16, device="cuda") for _ in range(s.n_layers)]
+        self.v_cache = [torch.zeros((batch, mt, self.kdim), dtype=torch.bfloat16, device="cuda") for _ in range(s.n_layers)]
+        n_old_max = max(ctx_len + max_steps - window, 1)
+        self.k_old = torch.zeros((batch, n_old_max, self.kdim), dtype=torch.bfloat16, device="cuda")
+        self.v_old = torch.zeros_like(self.k_old)
+        self.k_new = torch.zeros((batch, self.kdim), dtype=torch.bfloat16, device="cuda")
+        self.v_new = torch.zeros_like(self.k_new)
+        # ---- the context: rows into the store, their K/V into the cache
+        g = torch.Generator(device="cuda")
+        g.manual_seed(3000 + seed)
+        pos = torch.arange(ctx_len, dtype=torch.int32, device="cuda")
+        self.context_rows = {}  # (layer, seq) -> rows, kept for a few pairs so that tests can check K/V against the oracle
+        for l in range(s.n_layers):
+            for b in range(batch):
+                x = torch.randn((ctx_len, s.d_hidden), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+                ctx.kvd_checkpoint_residual(b, l, x, pos, ctx_len)
+                ctx.kvd_recompute_kv(l, None, None, ctx_len, self.k_cache[l][b], self.v_cache[l][b], self.kdim, seq=b,
+                                     first_row=0)
+                if b in (0, batch - 1) and l in (0, s.n_layers - 1):
+                    self.context_rows[(l, b)] = x
+        torch.cuda.synchronize()
+        # stand-ins for the scaffold's outputs when the hot path is timed by itself (step(..., scaffold=False))
+        self.h_fixed = torch.randn((batch, s.d_hidden), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        self.q_fixed = torch.randn((batch, s.n_q_heads, s.d_head), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        self.rows_in_store = ctx_len  # per (layer, sequence); grows with every KV-Direct step
+        self.recomputed_rows = 0
+
+    def _linear(self, lin, x):
+        m = x.shape[0]
+        out = torch.empty((m, lin.out_cols), dtype=torch.bfloat16, device="cuda")
+        self.ctx.kvd_scaffold_linear(lin, x, m, out, lin.out_cols)
+        return out
+
+    def step(self, tokens_dev, pos, policy, scaffold=True):
+        """One decode step of the whole batch at position `pos` (all sequences are equally long).
+        tokens_dev: DEVICE int32 [batch].  Returns the next tokens (DEVICE int32 [batch]) picked greedily.
+        scaffold=False runs the hot-path launches alone (queries and rows are then whatever the buffers
+        hold): used to time the library's part of the step by itself."""
+        s, ctx, B, kdim, mt = self.s, self.ctx, self.batch, self.kdim, self.max_tokens
+        pos_t = torch.full((B,), pos, dtype=torch.int32, device="cuda")
+        qpos = [pos] * B
+        h = torch.empty((B, s.d_hidden), dtype=torch.bfloat16, device="cuda")
+        if scaffold:
+            ctx.kvd_scaffold_embed(self.embed, tokens_dev, B, s.d_hidden, s.vocab, h)
+        else:
+            h.copy_(self.h_fixed)
+        q = torch.empty((B, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
+        out = torch.empty_like(q)
+        if not scaffold:
+            q.copy_(self.q_fixed)
+        wf = pos - self.window  # first live position of the KV-Direct arm after the previous step's eviction
+        for l in range(s.n_layers):
+            ls = s.layer_shape(l)
+            kc, vc = self.k_cache[l], self.v_cache[l]
+            lo = 0 if ls.sliding_window == 0 else max(0, pos - ls.sliding_window + 1)
+            if scaffold:
+                raw = self._linear(self.lin[l]["q"], h)
+                ctx.kvd_scaffold_query_finish(l, raw, raw.shape[1], pos_t, B, self.lw[l].get("gamma_q") if s.qk_norm else None, q)
+            if policy == "kvdirect":
+                ctx.kvd_checkpoint_residual_step(l, list(range(B)), h, pos_t)  # STORE_RESIDUAL, the whole batch at once
+                n_old = max(0, wf - lo)
+                ranges = [(b, lo, n_old, self.k_old[b], self.v_old[b]) for b in range(B)] if n_old > 0 else []
+                # RECOMPUTE_KV for the evicted positions of every sequence + K_t, V_t of the new tokens: one launch
+                # (one row stride for all outputs of the call, so K_t, V_t land in a [batch, kdim] buffer)
+                ctx.kvd_recompute_kv_step(l, ranges, h, pos_t, B, self.k_new, self.v_new, kdim)
+                self.recomputed_rows += B * n_old
+                first_live = max(wf, lo)
+                segs = [[(self.k_old[b], self.v_old[b], kdim, lo, n_old),
+                         (kc[b, first_live], vc[b, first_live], kdim, first_live, pos - first_live),
+                         (self.k_new[b], self.v_new[b], kdim, pos, 1)] for b in range(B)]
+                kv_new = True
+            else:
+                ctx.kvd_recompute_kv(l, h, pos_t, B, kc[0, pos], vc[0, pos], mt * kdim)
+                segs = [[(kc[b, lo], vc[b, lo], kdim, lo, pos + 1 - lo)] for b in range(B)]
+                kv_new = False
+            ctx.kvd_decode_attention(l, B, q, qpos, segs, 0.0, out)
+            if kv_new:  # the new entries join the live window (a device copy, after attention as in Algorithm 1)
+                kc[:, pos].copy_(self.k_new)
+                vc[:, pos].copy_(self.v_new)
+            if scaffold:
+                y = self._linear(self.lin[l]["o"], out.view(B, -1))
+                ctx.kvd_scaffold_add_rows(h, y, y.shape[1], B, s.d_hidden)
+                gu = self._linear(self.lin[l]["gate_up"], h)
+                inner = torch.empty((B, s.d_mlp), dtype=torch.bfloat16, device="cuda")
+                ctx.kvd_scaffold_gated_act(gu, gu.shape[1], B, s.d_mlp, self.act, inner)
+                y = self._linear(self.lin[l]["down"], inner)
+                ctx.kvd_scaffold_add_rows(h, y, y.shape[1], B, s.d_hidden)
+        nxt = torch.empty((B,), dtype=torch.int32, device="cuda")
+        if scaffold:
+            self.logits = self._linear(self.lin_head, h)
+            ctx.kvd_scaffold_argmax(self.logits, self.logits.shape[1], B, s.vocab, nxt)
+        return nxt
+
+    def decode(self, first_tokens, n_steps, policy):
+        """n_steps greedy steps from the context state; returns the tokens [n_steps][batch] as lists."""
+        assert policy in ("full", "kvdirect")
+        if policy == "kvdirect":
+            assert self.rows_in_store == self.ctx_len, "the KV-Direct arm appends to the store: run it once, last"
+        tok = torch.tensor(first_tokens, dtype=torch.int32, device="cuda")
+        outs = []
+        for i in range(n_steps):
+            tok = self.step(tok, self.ctx_len + i, policy)
+            outs.append(tok.tolist())
+        if policy == "kvdirect":
+            self.rows_in_store += n_steps
+        assert self.ctx.kvd_poll_status() == kvd.KVD_OK
+        return outs
