@@ -372,6 +372,21 @@ class Workload:
                                                 K[T:], V[T:], self.kdim, [[(K[T:], V[T:], self.kdim, T, 1)]], 0.0,
                                                 self.out[s:s + 1])
 
+    def append_current(self):
+        # the current token's row joins the bf16 store of every set (row T), once, outside any timed region
+        for s in range(self.n_sets):
+            if self.ctx.kvd_rows_stored(0, s) == self.T:
+                self.ctx.kvd_checkpoint_residual(s, 0, self.X[s][self.T:], self.pos[self.T:], 1)
+
+    def k_fused_folded(self, i):
+        # the fused call with the current token inside the attended range (its row is checkpointed like every
+        # token's): no live segment is left, so the streaming launch disappears -- recompute+attend, merge.
+        # K_t, V_t are still written (the caller's row rides in the same launch) for a window that keeps them.
+        s, T = i % self.n_sets, self.T
+        K, V = self.K[s], self.V[s]
+        self.ctx.kvd_decode_attention_recompute(0, 1, self.q[s:s + 1], [T], [(s, 0, T + 1)], self.X[s][T:], self.pos[T:], 1,
+                                                K[T:], V[T:], self.kdim, [[]], 0.0, self.out[s:s + 1])
+
     def append_current_fp8(self):
         # the current token joins the FP8 store of every set (row T), once, outside any timed region
         for s in range(self.n_sets):
@@ -556,6 +571,8 @@ def run_gpu(args):
               "recompute_from_fp8_checkpoints": timed_graph(wl.k_recompute_fp8, 10),
               "recompute_then_attention_two_calls": timed_graph(wl.k_two_call, 10),
               "recompute_fused_into_attention": timed_graph(wl.k_fused, 10)}
+    wl.append_current()
+    iso_ms["recompute_fused_into_attention_current_token_in_range"] = timed_graph(wl.k_fused_folded, 10)
     wl.append_current_fp8()
     iso_ms["recompute_fp8_then_attention_two_calls"] = timed_graph(wl.k_two_call_fp8, 10)
     iso_ms["recompute_fp8_fused_into_attention"] = timed_graph(wl.k_fused_fp8, 10)

@@ -326,7 +326,13 @@ kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, const void *
  *   rows, positions, n_rows, k_rows_out, v_rows_out, out_row_stride: the new tokens, exactly as in
  *           kvd_recompute_kv_step -- their K and V ARE written (the live segments usually point at them).
  *   q, q_pos, segs, n_segs, scale, out: as in kvd_decode_attention; batch <= KVD_MAX_STORE_RANGES.
- * Three launches (recompute+attend, live segments, merge).  KVD_ERR_UNSUPPORTED, with nothing launched,
+ *   The current token can be folded into the recomputed part: its row is checkpointed like every token's, so
+ *   ranges[b] may end with it (n counts it) while `rows` still makes its K_t, V_t for a window that keeps them;
+ *   when no live segment is left (n_segs == 0 or all lengths 0) the live-segment launch is skipped.
+ * Three launches (recompute+attend, live segments, merge), two without live segments.  The fused form pays
+ * where the recompute volume is large (kvd_fused_recompute_pays); below that the two-call sequence
+ * kvd_recompute_kv_step + kvd_decode_attention is faster, because a unit of work here is a key tile AND a
+ * value tile on one SM pair, where the plain kernel gives every tile its own.  KVD_ERR_UNSUPPORTED, with nothing launched,
  * for shapes the fused kernel is not built for (it exists for 256-column tiles with d_head 256 and 1 or 2
  * query heads per KV head, or d_head 128 and 1, 2 or 4); needs the store and the workspace attached. */
 kvd_status kvd_decode_attention_recompute(kvd_ctx *ctx, int layer, int batch, const void *q, const int32_t *q_pos,
@@ -334,6 +340,12 @@ kvd_status kvd_decode_attention_recompute(kvd_ctx *ctx, int layer, int batch, co
                                           const int32_t *positions, int n_rows, void *k_rows_out, void *v_rows_out,
                                           int64_t out_row_stride, const kvd_kv_segment *segs, int n_segs,
                                           float scale, void *out, void *stream);
+
+/* Host-only: 1 when the fused call (kvd_decode_attention_recompute, or its _fp8 forms when fp8 != 0) is expected
+ * to be at least as fast as recomputing into a buffer and attending over it in two calls, for `total_rows`
+ * evicted rows over all sequences of the launch; 0 otherwise or on bad arguments.  A rule fitted to
+ * measurements on B200 (bf16: from 16384 rows, FP8: from 4096 rows per launch), not a guarantee. */
+int kvd_fused_recompute_pays(const kvd_model_desc *desc, int64_t total_rows, int fp8);
 
 /* The same with the evicted tokens taken from the FP8 store (kvd_checkpoint_residual_fp8): ranges[b] (HOST
  * [batch], rows of the FP8 store of (layer, ranges[b].seq); k_out / v_out ignored) are rebuilt with E4M3

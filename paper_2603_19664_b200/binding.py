@@ -31,7 +31,7 @@ KVD_MAX_SEGMENTS = 4
 # every symbol include/kvd.h declares
 EXPORTED_SYMBOLS = (
     "kvd_create", "kvd_destroy", "kvd_set_layer", "kvd_store_bytes", "kvd_attach_store", "kvd_reset_sequence",
-    "kvd_decode_attention_recompute", "kvd_decode_attention_recompute_fp8", "kvd_set_dtype", "kvd_store_bytes_dtype",
+    "kvd_decode_attention_recompute", "kvd_fused_recompute_pays", "kvd_decode_attention_recompute_fp8", "kvd_set_dtype", "kvd_store_bytes_dtype",
     "kvd_quantize_rows_fp8", "kvd_recompute_kv_fp8_rows", "kvd_decode_attention_recompute_fp8_rows",
     "kvd_store_bytes_fp8", "kvd_attach_store_fp8", "kvd_rows_stored_fp8", "kvd_reset_sequence_fp8", "kvd_checkpoint_residual_fp8", "kvd_recompute_kv_fp8",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_checkpoint_residual_step", "kvd_recompute_kv",
@@ -138,6 +138,8 @@ def load() -> ctypes.CDLL:
     lib.kvd_decode_attention.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
                                          ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
     lib.kvd_decode_attention.restype = i32
+    lib.kvd_fused_recompute_pays.argtypes = [ctypes.POINTER(kvd_model_desc), i64, i32]
+    lib.kvd_fused_recompute_pays.restype = i32
     lib.kvd_set_dtype.argtypes = [vp, i32]
     lib.kvd_set_dtype.restype = i32
     lib.kvd_store_bytes_fp8.argtypes = [ctypes.POINTER(kvd_model_desc), i32]
@@ -241,6 +243,10 @@ def kvd_store_bytes_fp8(desc: kvd_model_desc, layers_stored: int) -> int:
 
 def kvd_workspace_bytes(desc: kvd_model_desc) -> int:
     return int(load().kvd_workspace_bytes(ctypes.byref(desc)))
+
+
+def kvd_fused_recompute_pays(desc: kvd_model_desc, total_rows: int, fp8: bool = False) -> bool:
+    return bool(load().kvd_fused_recompute_pays(ctypes.byref(desc), int(total_rows), 1 if fp8 else 0))
 
 
 def kvd_attention_split(d_head: int, n_kv_heads: int, first_visible: int, last_visible: int) -> Tuple[int, int]:

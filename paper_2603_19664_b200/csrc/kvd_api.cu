@@ -898,6 +898,16 @@ extern "C" kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, c
   return KVD_OK;
 }
 
+extern "C" int kvd_fused_recompute_pays(const kvd_model_desc *desc, int64_t total_rows, int fp8) {
+  if (check_desc(desc) != KVD_OK || total_rows <= 0) return 0;
+  const int group = desc->n_q_heads / desc->n_kv_heads, kdim = desc->n_kv_heads * desc->d_head;
+  // the shapes the fused kernel exists for
+  if (pick_block_n(desc) != 256 || kdim % 256 != 0 ||
+      !((desc->d_head == 256 && (group == 1 || group == 2)) || (desc->d_head == 128 && (group == 1 || group == 2 || group == 4))))
+    return 0;
+  return total_rows >= (fp8 ? 4096 : 16384) ? 1 : 0;
+}
+
 // Decode attention over [K/V recomputed from store ranges] + [live segments], the recomputed part
 // inside the recompute kernel (its K/V never reach memory); see kvd.h.
 extern "C" kvd_status kvd_decode_attention_recompute(kvd_ctx *ctx, int layer, int batch, const void *q,

@@ -67,8 +67,12 @@ __device__ __forceinline__ float reduce8_transposed(const float (&v)[8], int lig
 }
 
 // DT: element type of q, K, V and the output (0 = bf16, 1 = fp16; kvd_set_dtype).
-template <int D_HEAD, int G, int NSEQ, int DT = 0>
-__global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM) kvd_attn_split_kernel(const __grid_constant__ AttnLaunchT<NSEQ> P) {
+// ALLIN: for launches of at most two CTAs per SM whose chunks are two iterations long (a single sequence of
+// a few thousand keys), where nothing else on the SM hides a load's latency: the loads of both iterations are
+// issued before the query is fetched and before anything is computed, so a CTA pays one memory round trip
+// instead of three.  The arithmetic and its order are the same, hence the same bits.
+template <int D_HEAD, int G, int NSEQ, int DT = 0, bool ALLIN = false>
+__global__ void __launch_bounds__(AT_THREADS, ALLIN ? 2 : AT_CTAS_PER_SM) kvd_attn_split_kernel(const __grid_constant__ AttnLaunchT<NSEQ> P) {
   constexpr int LPK = D_HEAD / 8;         // lanes per key
   constexpr int KPL = 32 / LPK;           // keys per warp-wide load
   constexpr int U = AT_UNROLL;            // keys per lane group per iteration
@@ -109,16 +113,19 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM) kvd_attn_split_ker
   grid_dependency_wait();
   // ---- query of every head of the group, pre-multiplied by scale * log2(e)
   uint64_t qf[G][4];  // channel pairs (2j, 2j+1)
+  auto load_query = [&]() {
 #pragma unroll
-  for (int g = 0; g < G; ++g) {
-    const __nv_bfloat16 *qp = P.q + (static_cast<size_t>(si) * P.n_q + kvh * G + g) * D_HEAD + lig * 8;
-    const uint4 w = *reinterpret_cast<const uint4 *>(qp);
-    const uint64_t sc2 = pack2(P.scale_log2e, P.scale_log2e);
-    qf[g][0] = fmul2(x2_to_f32x2<DT>(w.x), sc2);
-    qf[g][1] = fmul2(x2_to_f32x2<DT>(w.y), sc2);
-    qf[g][2] = fmul2(x2_to_f32x2<DT>(w.z), sc2);
-    qf[g][3] = fmul2(x2_to_f32x2<DT>(w.w), sc2);
-  }
+    for (int g = 0; g < G; ++g) {
+      const __nv_bfloat16 *qp = P.q + (static_cast<size_t>(si) * P.n_q + kvh * G + g) * D_HEAD + lig * 8;
+      const uint4 w = *reinterpret_cast<const uint4 *>(qp);
+      const uint64_t sc2 = pack2(P.scale_log2e, P.scale_log2e);
+      qf[g][0] = fmul2(x2_to_f32x2<DT>(w.x), sc2);
+      qf[g][1] = fmul2(x2_to_f32x2<DT>(w.y), sc2);
+      qf[g][2] = fmul2(x2_to_f32x2<DT>(w.z), sc2);
+      qf[g][3] = fmul2(x2_to_f32x2<DT>(w.w), sc2);
+    }
+  };
+  if constexpr (!ALLIN) load_query();
 
   float m_run[G], l_run[G];
   uint64_t acc[G][4];  // channel pairs
@@ -263,10 +270,19 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM) kvd_attn_split_ker
     if (__any_sync(0xffffffffu, vmask != 0u)) compute(kr, vr, vmask);
   };
 
-  // One buffer of loads per iteration; latency is hidden by the other 15 warps resident on the SM
-  // (the kernel is capped at 128 registers so that four CTAs fit), which measured faster than
-  // register double buffering or a shared-memory ring at half the occupancy.
-  {
+  if constexpr (ALLIN) {
+    // both iterations' loads, then the query, then the arithmetic in the usual order
+    uint4 ka[U], va[U], kb[U], vb[U];
+    uint32_t ma = 0, mb = 0;
+    issue(0, ka, va, ma);
+    issue(1, kb, vb, mb);
+    load_query();
+    step(ka, va, ma);
+    step(kb, vb, mb);
+  } else {
+    // One buffer of loads per iteration; latency is hidden by the other 15 warps resident on the SM
+    // (the kernel is capped at 128 registers so that four CTAs fit), which measured faster than
+    // register double buffering or a shared-memory ring at half the occupancy.
     uint4 ka[U], va[U];
     uint32_t ma = 0;
     for (int it = 0; it < S.iters; ++it) {
@@ -606,16 +622,15 @@ __global__ void __launch_bounds__(AT_MERGE_THREADS)
   const size_t ml_stride = static_cast<size_t>(P.n_q) * 2, po_stride = static_cast<size_t>(P.n_q) * D_HEAD;
   if (warp < warps_used) {
     float2 vbuf[PF][G], mlbuf[PF][G];
+    // (a partial past the end re-reads the last one and is skipped below: no branch between the loads)
     auto fetch_group = [&](int grp) {
 #pragma unroll
       for (int i = 0; i < PF; ++i) {
-        const int ch = grp * PF + i;
-        if (ch < count) {
+        const int ch = grp * PF + i < count ? grp * PF + i : count - 1;
 #pragma unroll
-          for (int g = 0; g < G; ++g) {
-            mlbuf[i][g] = __ldcg(reinterpret_cast<const float2 *>(ml0 + ch * ml_stride + g * 2));
-            vbuf[i][g] = __ldcg(reinterpret_cast<const float2 *>(po0 + ch * po_stride + g * D_HEAD));
-          }
+        for (int g = 0; g < G; ++g) {
+          mlbuf[i][g] = __ldcg(reinterpret_cast<const float2 *>(ml0 + ch * ml_stride + g * 2));
+          vbuf[i][g] = __ldcg(reinterpret_cast<const float2 *>(po0 + ch * po_stride + g * D_HEAD));
         }
       }
     };
@@ -699,6 +714,11 @@ static cudaError_t attn_configure() {
       e = cudaFuncSetAttribute(kvd_attn_split_kernel<D_HEAD, G, NSEQ, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                AttnSmem<D_HEAD, G>::BYTES);
       if (e != cudaSuccess) return e;
+      if constexpr (G <= 2) {
+        e = cudaFuncSetAttribute(kvd_attn_split_kernel<D_HEAD, G, NSEQ, DT, true>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<D_HEAD, G>::BYTES);
+        if (e != cudaSuccess) return e;
+      }
     }
     done[dev & 63] = true;
   }
@@ -729,7 +749,15 @@ static cudaError_t attn_launch_pair(const AttnLaunchT<NSEQ> &S, cudaStream_t str
       e = cudaLaunchKernelEx(&cfg, kvd_attn_split_mma_kernel<D_HEAD, G, NSEQ, DT>, S);
     } else {
       cfg.dynamicSmemBytes = AttnSmem<D_HEAD, G>::BYTES;
-      e = cudaLaunchKernelEx(&cfg, kvd_attn_split_kernel<D_HEAD, G, NSEQ, DT>, S);
+      // at most two CTAs per SM, every chunk two iterations long: the variant that issues all loads at once
+      bool allin = G <= 2 && S.total_chunks * S.n_kv <= 148 * 2;
+      for (int i = 0; i < S.n_seqs; ++i) allin = allin && (S.seq[i].n_chunks == 0 || S.seq[i].iters == 2);
+      if constexpr (G <= 2) {
+        if (allin) e = cudaLaunchKernelEx(&cfg, kvd_attn_split_kernel<D_HEAD, G, NSEQ, DT, true>, S);
+        else e = cudaLaunchKernelEx(&cfg, kvd_attn_split_kernel<D_HEAD, G, NSEQ, DT>, S);
+      } else {
+        e = cudaLaunchKernelEx(&cfg, kvd_attn_split_kernel<D_HEAD, G, NSEQ, DT>, S);
+      }
     }
     if (e != cudaSuccess) return e;
   }

@@ -152,3 +152,33 @@ def test_fused_at_the_largest_batch():
     f, two, ref = run_case(GEMMA3_4B_GLOBAL, lens, 8, pos0_list=[3 * b for b in range(64)], max_tokens=1024, seed=12)
     attn_check(f, ref, "fused vs oracle")
     attn_check(f, two, "fused vs two-call")
+
+
+@pytest.mark.parametrize("shape,T", [(GEMMA3_4B_GLOBAL, 700), (QWEN3_4B, 1300)], ids=lambda x: getattr(x, "name", x))
+def test_fused_with_the_current_token_inside_the_range_needs_no_live_segment(shape, T):
+    """Budget zero, the form the benchmark times: every token's row is checkpointed, the current one included,
+    and ranges[b] covers all T + 1 of them; the caller's row still yields K_t, V_t (same bits as
+    kvd_recompute_kv), no segment is passed, and only two kernels run (recompute+attend, merge)."""
+    ctx, w = open_layer(shape, max_tokens=2048, with_store=True)
+    kdim = shape.n_kv_heads * shape.d_head
+    X = make_residuals(shape, T + 1, seed=77, outliers=True)
+    pos = np.arange(T + 1)
+    x, p = dev(X), torch.from_numpy(pos.astype(np.int32)).cuda()
+    ctx.kvd_checkpoint_residual(0, 0, x, p, T + 1)
+    q_bits = make_query(shape, 1, seed=77)
+    q = dev(q_bits)
+    out = torch.zeros((1, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda")
+    kc = torch.zeros((1, kdim), dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    n0 = ctx.kvd_launch_count()
+    ctx.kvd_decode_attention_recompute(0, 1, q, [T], [(0, 0, T + 1)], x[T:], p[T:], 1, kc, vc, kdim, [[]], 0.0, out)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    assert ctx.kvd_launch_count() - n0 == 2
+    Kr, Vr = oracle_kv(shape, w, X, pos)
+    ref = oracle.decode_attention(bf16_to_f64(q_bits[0]), T, [(Kr, Vr, 0)], 1.0 / math.sqrt(shape.d_head), shape.sliding_window)
+    attn_check(host_f64(out)[0], ref, "folded")
+    k2 = torch.zeros_like(kc)
+    v2 = torch.zeros_like(vc)
+    ctx.kvd_recompute_kv(0, x[T:], p[T:], 1, k2, v2, kdim)
+    assert torch.equal(kc, k2) and torch.equal(vc, v2)
+    ctx.close()

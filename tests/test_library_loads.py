@@ -103,3 +103,12 @@ def test_entry_points_reject_null_contexts_and_bad_shapes_without_a_device():
     assert lib.kvd_decode_attention_static(8, 4, 128, -1, 1, None, qp, None, 0, 0.0, None, None) == binding.KVD_ERR_INVALID_ARG
     assert lib.kvd_decode_attention_static(8, 4, 128, 0, 0, None, None, None, 0, 0.0, None, None) == binding.KVD_OK  # empty batch
     assert lib.kvd_decode_attention_static(8, 4, 128, 0, 1, None, qp, None, 0, 0.0, None, None) == binding.KVD_ERR_INVALID_ARG
+
+
+def test_fused_predicate_is_host_only_and_shape_aware():
+    gemma = kvd.make_desc(34, 2560, 8, 4, 256, 1e-6, True, 1e-6)
+    smol = kvd.make_desc(1, 576, 9, 3, 64, 1e-5, False, 1e-5)
+    assert not kvd.kvd_fused_recompute_pays(gemma, 4096) and kvd.kvd_fused_recompute_pays(gemma, 32768)
+    assert kvd.kvd_fused_recompute_pays(gemma, 4096, fp8=True) and not kvd.kvd_fused_recompute_pays(gemma, 1024, fp8=True)
+    assert not kvd.kvd_fused_recompute_pays(smol, 1 << 20)  # no fused kernel for this shape
+    assert not kvd.kvd_fused_recompute_pays(gemma, 0)
