@@ -61,7 +61,8 @@ typedef enum {
   KVD_ERR_UNSUPPORTED = 6, /* no usable device / driver entry point                        */
   KVD_ERR_CUDA = 7,        /* a CUDA runtime call failed; see kvd_last_cuda_error          */
   KVD_ERR_TIMEOUT = 8,     /* a bounded wait inside a kernel expired (from kvd_poll_status) */
-  KVD_ERR_POSITION = 9     /* a row's position was outside [0, max_tokens_per_seq)         */
+  KVD_ERR_POSITION = 9,    /* a row's position was outside [0, max_tokens_per_seq)         */
+  KVD_ERR_BOUNDS = 10      /* checking build only: a kernel met an index outside its table or buffer */
 } kvd_status;
 
 /* Pairing of channels rotated together by Eq. 11-12. */
@@ -396,8 +397,8 @@ kvd_status kvd_decode_attention_static(int n_q_heads, int n_kv_heads, int d_head
 /* Fill `out` with the byte counts described at kvd_mem_stats. */
 kvd_status kvd_memory_stats(const kvd_ctx *ctx, kvd_mem_stats *out);
 
-/* Wait for `stream`, read and clear the device status word.  KVD_OK, KVD_ERR_TIMEOUT or
- * KVD_ERR_POSITION. */
+/* Wait for `stream`, read and clear the device status word.  KVD_OK, KVD_ERR_TIMEOUT, KVD_ERR_POSITION or (checking
+ * build) KVD_ERR_BOUNDS. */
 kvd_status kvd_poll_status(kvd_ctx *ctx, void *stream);
 
 /* Self-test of the failure path: enqueue a one-thread kernel that waits (at most limit_ms, 1..1000)
@@ -406,6 +407,18 @@ kvd_status kvd_poll_status(kvd_ctx *ctx, void *stream);
  * kernel uses (its limit is 2 s, or KVD_SPIN_LIMIT_MS from the environment at kvd_create).  The device
  * stays usable. */
 kvd_status kvd_selftest_wait_timeout(kvd_ctx *ctx, int limit_ms, void *stream);
+
+/* The checking build (libkvd_check.so: the same sources compiled with -DKVD_CHECK; python -m
+ * paper_2603_19664_b200.build --check).  Its kernels test the indices they derive on the device -- the job and
+ * row block a tile belongs to, the rows of a store range, the slot of a residual row, the slot of an attention
+ * partial -- before they use them; a failed test sets a bit of the status word and SKIPS the access (nothing
+ * faults, the context stays usable), and kvd_poll_status then returns KVD_ERR_BOUNDS.  It stands in for a
+ * memory checker where none can be run; the release build contains none of these tests.
+ * kvd_build_has_checks: 1 in the checking build, 0 otherwise.
+ * kvd_selftest_bounds_check: runs one such test on an index that is out of range by construction (no memory is
+ * touched), so that a test suite can see the mechanism report; KVD_ERR_UNSUPPORTED in the release build. */
+int kvd_build_has_checks(void);
+kvd_status kvd_selftest_bounds_check(kvd_ctx *ctx, void *stream);
 
 /* Diagnostic hook: attach (buf != NULL) or detach (buf == NULL) a DEVICE buffer of int64 slots that
  * kvd_recompute_kv fills with a per-tile timeline in SM clock cycles: for CTA b and its i-th tile

@@ -12,7 +12,10 @@ import os
 from typing import List, Optional, Sequence, Tuple
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libkvd.so")
+# KVD_LIBRARY=check selects the checking build (libkvd_check.so: device-side index tests, see kvd.h); a path selects
+# that file.  Either way it is this library's own code: there is no other implementation to fall back to.
+_sel = os.environ.get("KVD_LIBRARY", "")
+LIB_PATH = (os.path.join(_HERE, "libkvd_check.so") if _sel == "check" else _sel) if _sel else os.path.join(_HERE, "libkvd.so")
 
 KVD_OK = 0
 KVD_ERR_INVALID_ARG = 1
@@ -24,6 +27,7 @@ KVD_ERR_UNSUPPORTED = 6
 KVD_ERR_CUDA = 7
 KVD_ERR_TIMEOUT = 8
 KVD_ERR_POSITION = 9
+KVD_ERR_BOUNDS = 10
 KVD_ROPE_INTERLEAVED = 0
 KVD_ROPE_HALF = 1
 KVD_MAX_SEGMENTS = 4
@@ -36,7 +40,7 @@ EXPORTED_SYMBOLS = (
     "kvd_store_bytes_fp8", "kvd_attach_store_fp8", "kvd_rows_stored_fp8", "kvd_reset_sequence_fp8", "kvd_checkpoint_residual_fp8", "kvd_recompute_kv_fp8",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_checkpoint_residual_step", "kvd_recompute_kv",
     "kvd_recompute_kv_step",
-    "kvd_decode_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
+    "kvd_decode_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_build_has_checks", "kvd_selftest_bounds_check", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
     "kvd_status_string", "kvd_version",
     # include/kvd_scaffold.h: the parts of a decoder layer around the hot path, for whole-stack tests and benchmarks
     "kvd_scaffold_linear_create", "kvd_scaffold_linear_destroy", "kvd_scaffold_linear_out_cols", "kvd_scaffold_linear",
@@ -182,6 +186,10 @@ def load() -> ctypes.CDLL:
     lib.kvd_poll_status.restype = i32
     lib.kvd_selftest_wait_timeout.argtypes = [vp, i32, vp]
     lib.kvd_selftest_wait_timeout.restype = i32
+    lib.kvd_build_has_checks.argtypes = []
+    lib.kvd_build_has_checks.restype = i32
+    lib.kvd_selftest_bounds_check.argtypes = [vp, vp]
+    lib.kvd_selftest_bounds_check.restype = i32
     lib.kvd_set_trace.argtypes = [vp, vp, sz]
     lib.kvd_set_trace.restype = i32
     lib.kvd_launch_count.argtypes = [vp]
@@ -220,6 +228,10 @@ def status_string(status: int) -> str:
 
 def kvd_version() -> str:
     return load().kvd_version().decode()
+
+
+def kvd_build_has_checks() -> bool:
+    return bool(load().kvd_build_has_checks())
 
 
 def make_desc(n_layers: int, d_hidden: int, n_q_heads: int, n_kv_heads: int, d_head: int, rms_eps: float,
@@ -516,6 +528,10 @@ class Kvd:
     def kvd_selftest_wait_timeout(self, limit_ms: int, stream=None) -> None:
         self._check(self._lib.kvd_selftest_wait_timeout(self._h, limit_ms, _stream(stream)),
                     "kvd_selftest_wait_timeout")
+
+    def kvd_selftest_bounds_check(self, stream=None) -> int:
+        """Returns the status (KVD_ERR_UNSUPPORTED in the release build) instead of raising."""
+        return int(self._lib.kvd_selftest_bounds_check(self._h, _stream(stream)))
 
     def kvd_set_trace(self, buf) -> None:
         if buf is None:

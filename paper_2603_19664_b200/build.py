@@ -1,4 +1,4 @@
-"""Build the CUDA library in-tree: ``python -m paper_2603_19664_b200.build``.
+"""Build the CUDA library in-tree: ``python -m paper_2603_19664_b200.build`` (``--check``: the checking build).
 
 Compiles every ``csrc/*.cu`` for sm_100a with nvcc into ``libkvd.so`` next to this file.  The CUDA
 runtime is linked statically and the driver API is reached through ``cudaGetDriverEntryPoint``, so
@@ -15,6 +15,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkvd.so")
+LIB_CHECK = os.path.join(HERE, "libkvd_check.so")  # the same sources with -DKVD_CHECK (device-side index tests)
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
          "--expt-relaxed-constexpr"]
@@ -29,24 +30,28 @@ def _deps():
         os.path.join(os.path.dirname(HERE), "include", "kvd.h")]
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB):
+def needs_build(check: bool = False) -> bool:
+    lib = LIB_CHECK if check else LIB
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     return any(os.path.getmtime(p) > t for p in _deps())
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not needs_build():
+def build(force: bool = False, verbose: bool = False, check: bool = False) -> str:
+    """Compile libkvd.so, or with ``check`` libkvd_check.so: the build whose kernels test the indices they
+    derive on the device and report through the status word instead of accessing out of range."""
+    LIB = LIB_CHECK if check else globals()["LIB"]
+    if not force and not needs_build(check):
         return LIB
-    objdir = os.path.join(HERE, "build")
+    objdir = os.path.join(HERE, "build", "check") if check else os.path.join(HERE, "build")
     os.makedirs(objdir, exist_ok=True)
     procs = []
     objs = []
     for src in _sources():
         obj = os.path.join(objdir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
-        cmd = [NVCC, *FLAGS, "-c", src, "-o", obj]
+        cmd = [NVCC, *FLAGS, *(["-DKVD_CHECK"] if check else []), "-c", src, "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
@@ -66,4 +71,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, check="--check" in sys.argv))

@@ -58,6 +58,7 @@ extern "C" const char *kvd_status_string(kvd_status s) {
     case KVD_ERR_CUDA: return "CUDA error";
     case KVD_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
     case KVD_ERR_POSITION: return "row position out of range";
+    case KVD_ERR_BOUNDS: return "an index test of the checking build failed";
   }
   return "unknown status";
 }
@@ -176,13 +177,21 @@ extern "C" void kvd_destroy(kvd_ctx *ctx) {
 
 // (eb = bytes per element: 2 for bf16, 1 for the FP8 variant's codes; a box row is 128 bytes either way)
 namespace kvd {
+// element type of a tensor map for `eb` bytes per element (16-bit maps follow the context's type; the copies
+// are bit-for-bit either way)
+static CUtensorMapDataType map_type(const kvd_ctx *ctx, int eb) {
+  if (eb == 4) return CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+  if (eb == 1) return CU_TENSOR_MAP_DATA_TYPE_UINT8;
+  return ctx->dtype == KVD_DTYPE_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+}
+
 kvd_status encode_2d(kvd_ctx *ctx, CUtensorMap *map, const void *base, uint64_t inner, uint64_t outer,
                      uint32_t box_inner, uint32_t box_outer, int eb) {
   cuuint64_t dims[2] = {inner, outer};
   cuuint64_t strides[1] = {inner * eb};
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = ctx->encode(map, eb == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : eb == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
+  CUresult r = ctx->encode(map, map_type(ctx, eb), 2,
                            const_cast<void *>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -202,7 +211,7 @@ kvd_status encode_rows_3d(kvd_ctx *ctx, CUtensorMap *map, const void *base, uint
   cuuint64_t strides[2] = {d_hidden * eb, rows * d_hidden * eb};
   cuuint32_t box[3] = {static_cast<cuuint32_t>(RC_BLOCK_K * 2 / eb), RC_BLOCK_M, 1};
   cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = ctx->encode(map, eb == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : eb == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 3,
+  CUresult r = ctx->encode(map, map_type(ctx, eb), 3,
                            const_cast<void *>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -260,6 +269,10 @@ extern "C" kvd_status kvd_set_dtype(kvd_ctx *ctx, int dtype) {
     if (l.set) return KVD_ERR_STATE;  // weights are prepared in the element type: choose it first
   if (ctx->store_rows && dtype_bytes(dtype) != dtype_bytes(ctx->dtype)) return KVD_ERR_STATE;  // the store is laid out for it
   for (int c : ctx->rows_stored)
+    if (c != 0) return KVD_ERR_STATE;
+  // the FP8 variant reads bf16 rows and bf16-folded weights: no other element type next to an FP8 store
+  if (dtype != KVD_DTYPE_BF16 && ctx->store8_codes) return KVD_ERR_STATE;
+  for (int c : ctx->rows_stored8)
     if (c != 0) return KVD_ERR_STATE;
   ctx->dtype = dtype;
   return KVD_OK;
@@ -460,6 +473,7 @@ static void fill_launch_params(const kvd_ctx *ctx, const LayerState &ls, Recompu
   p.trace = nullptr;
   p.ext_rows = nullptr;
   p.w_scale = nullptr;
+  p.store_rows = d.max_tokens_per_seq;
   p.row_chunks = d.d_hidden * dtype_bytes(ctx->dtype) / 16;
   // 32-byte stores need every output row 32-byte aligned
   p.wide_store = out_row_stride * dtype_bytes(ctx->dtype) % 32 == 0;
@@ -864,6 +878,8 @@ static kvd_status build_attn_launch(kvd_ctx *ctx, const LayerState &ls, int b0, 
   L.out = static_cast<__nv_bfloat16 *>(out) + static_cast<size_t>(b0) * d.n_q_heads * d.d_head;
   L.part_o = ctx->part_o;
   L.part_ml = ctx->part_ml;
+  L.status = ctx->d_status;
+  L.max_parts = ctx->max_parts;
   L.scale_log2e = sc * 1.4426950408889634f;
   return KVD_OK;
 }
@@ -1068,8 +1084,22 @@ extern "C" kvd_status kvd_poll_status(kvd_ctx *ctx, void *stream_) {
     if (e != cudaSuccess) return cuda_fail(ctx, e, "kvd_poll_status clear");
   }
   if (word & STATUS_TIMEOUT) return KVD_ERR_TIMEOUT;
+  if (word & STATUS_BOUNDS) return KVD_ERR_BOUNDS;
   if (word & STATUS_POSITION) return KVD_ERR_POSITION;
   return KVD_OK;
+}
+
+extern "C" int kvd_build_has_checks(void) {
+#ifdef KVD_CHECK
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+extern "C" kvd_status kvd_selftest_bounds_check(kvd_ctx *ctx, void *stream_) {
+  if (!ctx) return KVD_ERR_INVALID_ARG;
+  return launch_selftest_bounds(ctx, static_cast<cudaStream_t>(stream_));
 }
 
 extern "C" kvd_status kvd_selftest_wait_timeout(kvd_ctx *ctx, int limit_ms, void *stream_) {

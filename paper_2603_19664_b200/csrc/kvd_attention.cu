@@ -327,6 +327,7 @@ __global__ void __launch_bounds__(AT_THREADS, ALLIN ? 2 : AT_CTAS_PER_SM) kvd_at
       l = fmaf(w, s_l[pp][g], l);
     }
     const size_t hq = pidx * P.n_q + kvh * G + g;
+    if (!KVD_BOUNDS_OK(pidx < static_cast<size_t>(P.max_parts), P.status)) continue;  // checking build: the partial's slot
     P.part_o[hq * D_HEAD + c] = o;
     if (c == 0) {
       P.part_ml[hq * 2] = M;
@@ -575,6 +576,7 @@ __global__ void __launch_bounds__(AT_THREADS, AT_CTAS_PER_SM)
       l = fmaf(w, s_l[pp][g], l);
     }
     const size_t hq = pidx * P.n_q + kvh * G + g;
+    if (!KVD_BOUNDS_OK(pidx < static_cast<size_t>(P.max_parts), P.status)) continue;  // checking build: the partial's slot
     P.part_o[hq * D_HEAD + c] = o;
     if (c == 0) {
       P.part_ml[hq * 2] = M;
@@ -613,7 +615,8 @@ __global__ void __launch_bounds__(AT_MERGE_THREADS)
   // partials are visible
   grid_dependency_wait();
 
-  const int count = S.merge_count;
+  // (checking build: the slots to merge lie inside the partial arrays; otherwise nothing is merged)
+  const int count = KVD_BOUNDS_OK(S.merge_base >= 0 && S.merge_base + S.merge_count <= P.max_parts, P.status) ? S.merge_count : 0;
   const int n_groups = (count + PF - 1) / PF;
   const int warps_used = n_groups < AT_MERGE_WARPS ? n_groups : AT_MERGE_WARPS;
   const float *ml0 = P.part_ml + (static_cast<size_t>(S.merge_base) * P.n_q + kvh * G) * 2;
@@ -980,6 +983,8 @@ extern "C" kvd_status kvd_decode_attention_static(int n_q_heads, int n_kv_heads,
   L.out = static_cast<__nv_bfloat16 *>(out);
   L.part_ml = reinterpret_cast<float *>(scratch);
   L.part_o = reinterpret_cast<float *>(scratch + ml_bytes);
+  L.status = nullptr;
+  L.max_parts = parts;
   switch (d_head) {
     case 64: return static_launch_d<64>(L, group, stream);
     case 128: return static_launch_d<128>(L, group, stream);

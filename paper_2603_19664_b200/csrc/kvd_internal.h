@@ -18,6 +18,15 @@ namespace kvd {
 // device status word bits (written by kernels with atomicOr, read by kvd_poll_status)
 constexpr int STATUS_TIMEOUT = 1;
 constexpr int STATUS_POSITION = 2;
+constexpr int STATUS_BOUNDS = 4;  // checking build: an index test failed (the access was skipped)
+
+// Index tests of the checking build (-DKVD_CHECK): `if (KVD_BOUNDS_OK(cond, status)) access;`.  A failed test
+// records STATUS_BOUNDS and yields false, so the access is skipped; the release build compiles the test away.
+#ifdef KVD_CHECK
+#define KVD_BOUNDS_OK(cond, status) ((cond) ? true : ((status) != nullptr ? (atomicOr((status), kvd::STATUS_BOUNDS), false) : false))
+#else
+#define KVD_BOUNDS_OK(cond, status) (true)
+#endif
 
 constexpr int ROPE_LO_BITS = 4;  // position = hi * 16 + lo; one table per part
 constexpr int ROPE_LO_SIZE = 1 << ROPE_LO_BITS;
@@ -75,6 +84,7 @@ struct RecomputeParams {
   int row_chunks;                 // d_hidden / 8: 16-byte chunks per row
   int wide_store;                 // outputs are 32-byte aligned: 32-byte stores
   const float *w_scale;           // FP8 variant: the weight matrix's quantisation scale (one float), else nullptr
+  int store_rows;                 // rows per (layer, sequence) slab of the store (checking build)
   RcJob jobs[RC_MAX_JOBS];
 };
 
@@ -139,6 +149,8 @@ struct AttnLaunchHead {
   __nv_bfloat16 *out;      // [n_seqs, n_q, d_head]
   float *part_o;           // [parts][n_q][d_head]
   float *part_ml;          // [parts][n_q][2]
+  int *status;             // device status word (nullptr: none), used by the checking build
+  int max_parts;           // slots the partial arrays hold
 };
 template <int NSEQ>
 struct AttnLaunchT : AttnLaunchHead {
@@ -281,6 +293,7 @@ kvd_status launch_recompute_fp8(kvd_ctx *ctx, const LayerState &ls, const CUtens
                                 const CUtensorMap &tmap_rows, const RecomputeParams &p, cudaStream_t stream);
 kvd_status launch_checkpoint(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, __nv_bfloat16 *dst_rows,
                              int32_t *dst_pos, float *dst_sumsq, int n, int d_hidden, cudaStream_t stream);
+kvd_status launch_selftest_bounds(kvd_ctx *ctx, cudaStream_t stream);
 kvd_status launch_checkpoint_scatter(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, const CkptSlots &slots,
                                      int n, int d_hidden, cudaStream_t stream);
 kvd_status launch_selftest_timeout(kvd_ctx *ctx, unsigned long long timeout_ns, cudaStream_t stream);

@@ -65,11 +65,13 @@ template <int DT>
 __global__ void __launch_bounds__(256) kvd_checkpoint_kernel(const uint4 *__restrict__ rows,
                                                              const int32_t *__restrict__ pos,
                                                              uint4 *__restrict__ dst_rows, int32_t *__restrict__ dst_pos,
-                                                             float *__restrict__ dst_sumsq, int row_chunks, int n) {
+                                                             float *__restrict__ dst_sumsq, int row_chunks, int n,
+                                                             int capacity, int *status) {
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   grid_launch_dependents();  // the next kernel's set-up may overlap this copy
   for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n; r += warps) {
+    if (!KVD_BOUNDS_OK(r < capacity, status)) continue;  // checking build: the row fits the sequence's slab
     const size_t off = static_cast<size_t>(r) * row_chunks;
     const uint4 *const src[1] = {rows + off};
     uint4 *const dst[1] = {dst_rows + off};
@@ -90,11 +92,13 @@ __global__ void __launch_bounds__(256) kvd_checkpoint_scatter_kernel(const uint4
                                                                      uint4 *__restrict__ store_rows,
                                                                      int32_t *__restrict__ store_pos,
                                                                      float *__restrict__ store_sumsq, int row_chunks, int n,
+                                                                     long long total_slots, int *status,
                                                                      const __grid_constant__ CkptSlots P) {
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   grid_launch_dependents();
   for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n; r += warps) {
+    if (!KVD_BOUNDS_OK(P.slot[r] >= 0 && P.slot[r] < total_slots, status)) continue;  // checking build
     const size_t slot = static_cast<size_t>(P.slot[r]);
     const uint4 *const src[1] = {rows + static_cast<size_t>(r) * row_chunks};
     uint4 *const dst[1] = {store_rows + slot * row_chunks};
@@ -273,6 +277,26 @@ __global__ void kvd_selftest_timeout_kernel(int *status, unsigned long long time
   }
 }
 
+// Checking build: one index test that fails by construction (index 1 of a table of one entry); the access it
+// guards is skipped, so nothing is read or written out of range.
+__global__ void kvd_selftest_bounds_kernel(int *status, int *table) {
+  const int idx = 1, entries = 1;
+  if (KVD_BOUNDS_OK(idx < entries, status)) table[idx] = 0;
+}
+kvd_status launch_selftest_bounds(kvd_ctx *ctx, cudaStream_t stream) {
+#ifdef KVD_CHECK
+  kvd_selftest_bounds_kernel<<<1, 1, 0, stream>>>(ctx->d_status, ctx->d_status);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "launch selftest_bounds");
+  ctx->launches += 1;
+  return KVD_OK;
+#else
+  (void)ctx;
+  (void)stream;
+  return KVD_ERR_UNSUPPORTED;
+#endif
+}
+
 kvd_status launch_selftest_timeout(kvd_ctx *ctx, unsigned long long timeout_ns, cudaStream_t stream) {
   kvd_selftest_timeout_kernel<<<1, 32, 0, stream>>>(ctx->d_status, timeout_ns);
   cudaError_t e = cudaGetLastError();
@@ -310,19 +334,22 @@ kvd_status launch_convert_gamma(kvd_ctx *ctx, const __nv_bfloat16 *g, float *out
 
 kvd_status launch_checkpoint(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, __nv_bfloat16 *dst_rows,
                              int32_t *dst_pos, float *dst_sumsq, int n, int d_hidden, cudaStream_t stream) {
+  // rows left in the (layer, sequence) slab from dst on: what the checking build tests row indices against
+  const long long slot = dst_pos - ctx->store_pos;
+  const int capacity = ctx->desc.max_tokens_per_seq - static_cast<int>(slot % ctx->desc.max_tokens_per_seq);
   long long blocks = (static_cast<long long>(n) + 7) / 8;  // eight warps, one row each per pass
   const long long cap = static_cast<long long>(ctx->num_sms) * 8;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   if (ctx->dtype == 2)
     kvd_checkpoint_kernel<2><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
-        reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint4 *>(dst_rows), dst_pos, dst_sumsq, d_hidden / 4, n);
+        reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint4 *>(dst_rows), dst_pos, dst_sumsq, d_hidden / 4, n, capacity, ctx->d_status);
   else if (ctx->dtype == 1)
     kvd_checkpoint_kernel<1><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
-        reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint4 *>(dst_rows), dst_pos, dst_sumsq, d_hidden / 8, n);
+        reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint4 *>(dst_rows), dst_pos, dst_sumsq, d_hidden / 8, n, capacity, ctx->d_status);
   else
     kvd_checkpoint_kernel<0><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
-        reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint4 *>(dst_rows), dst_pos, dst_sumsq, d_hidden / 8, n);
+        reinterpret_cast<const uint4 *>(rows), pos, reinterpret_cast<uint4 *>(dst_rows), dst_pos, dst_sumsq, d_hidden / 8, n, capacity, ctx->d_status);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "launch checkpoint");
   ctx->launches += 1;
@@ -334,12 +361,13 @@ kvd_status launch_checkpoint_scatter(kvd_ctx *ctx, const __nv_bfloat16 *rows, co
   const unsigned blocks = static_cast<unsigned>((n + 7) / 8);  // eight warps, one row each
   const uint4 *src = reinterpret_cast<const uint4 *>(rows);
   uint4 *dst = reinterpret_cast<uint4 *>(ctx->store_rows);
+  const long long total = static_cast<long long>(ctx->layers_stored) * ctx->desc.max_seqs * ctx->desc.max_tokens_per_seq;
   if (ctx->dtype == 2)
-    kvd_checkpoint_scatter_kernel<2><<<blocks, 256, 0, stream>>>(src, pos, dst, ctx->store_pos, ctx->store_sumsq, d_hidden / 4, n, slots);
+    kvd_checkpoint_scatter_kernel<2><<<blocks, 256, 0, stream>>>(src, pos, dst, ctx->store_pos, ctx->store_sumsq, d_hidden / 4, n, total, ctx->d_status, slots);
   else if (ctx->dtype == 1)
-    kvd_checkpoint_scatter_kernel<1><<<blocks, 256, 0, stream>>>(src, pos, dst, ctx->store_pos, ctx->store_sumsq, d_hidden / 8, n, slots);
+    kvd_checkpoint_scatter_kernel<1><<<blocks, 256, 0, stream>>>(src, pos, dst, ctx->store_pos, ctx->store_sumsq, d_hidden / 8, n, total, ctx->d_status, slots);
   else
-    kvd_checkpoint_scatter_kernel<0><<<blocks, 256, 0, stream>>>(src, pos, dst, ctx->store_pos, ctx->store_sumsq, d_hidden / 8, n, slots);
+    kvd_checkpoint_scatter_kernel<0><<<blocks, 256, 0, stream>>>(src, pos, dst, ctx->store_pos, ctx->store_sumsq, d_hidden / 8, n, total, ctx->d_status, slots);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "launch checkpoint (batch)");
   ctx->launches += 1;

@@ -298,6 +298,13 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
     }
     job = lo;
     m0 = (mb - p.jobs[lo].mb_start) * (2 * RC_BLOCK_M) + static_cast<int>(cta_rank) * RC_BLOCK_M;
+    // checking build: the tile lies inside the job table, its job's row blocks and (for store ranges) the
+    // sequence's slab; a tile that does not is not processed by any role
+    if (!KVD_BOUNDS_OK(mb >= 0 && mb < p.num_m_blocks && lo >= 0 && lo < p.n_jobs && n0 >= 0 && n0 < p.num_n_blocks * BLOCK_N &&
+                           m0 - static_cast<int>(cta_rank) * RC_BLOCK_M < p.jobs[lo].n &&
+                           (p.jobs[lo].slab < 0 || p.jobs[lo].row0 + p.jobs[lo].n <= p.store_rows),
+                       p.status))
+      return false;
     return true;
   };
   const unsigned long long tmo = p.timeout_ns;

@@ -295,6 +295,7 @@ extern "C" kvd_status kvd_scaffold_linear(kvd_ctx *ctx, const kvd_linear *lin, c
   p.row_chunks = lin->k / 8;
   p.wide_store = (out_row_stride * 2 % 32 == 0) && ((reinterpret_cast<uintptr_t>(out) & 31u) == 0);
   p.w_scale = nullptr;
+  p.store_rows = m;
   return launch_recompute(ctx, lin->ls, tmap_rows, tmap_rows, p, stream);
 }
 

@@ -18,6 +18,7 @@ def pytest_sessionstart(session):
     try:
         from paper_2603_19664_b200.build import build
         build()
+        build(check=True)  # the checking build (device-side index tests), used by tests/test_gpu_check_build.py
     except Exception as e:  # noqa: BLE001
         sys.stderr.write(f"[conftest] building libkvd.so failed: {e}\n")
 

@@ -206,3 +206,22 @@ def test_fp16_kvdirect_layer_equals_the_full_cache_layer_bit_for_bit():
     assert torch.equal(kr.view(torch.int16), kc[:n_old].view(torch.int16))
     assert torch.equal(full.view(torch.int16), kvdir.view(torch.int16))
     assert float(full.abs().max()) > 0
+
+
+def test_element_type_cannot_change_next_to_an_fp8_store():
+    # the FP8 entry points quantise bf16 rows and use bf16-folded weights: a context that holds an FP8 store
+    # stays bf16 (KVD_ERR_STATE), before any layer is set and whether or not rows are stored yet
+    shape = GEMMA3_4B_GLOBAL
+    desc = kvd.make_desc(1, shape.d_hidden, shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.rms_eps, shape.qk_norm,
+                         shape.rms_eps, shape.rope_style, 1, 64, 1)
+    ctx = kvd.Kvd(desc)
+    ctx.kvd_set_dtype(1)
+    ctx.kvd_set_dtype(0)  # nothing holds a type yet: free to change
+    arena = torch.zeros(kvd.kvd_store_bytes_fp8(desc, 1), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_store_fp8(arena, 1)
+    for dt in (1, 2):
+        with pytest.raises(kvd.KvdError) as e:
+            ctx.kvd_set_dtype(dt)
+        assert e.value.status == 5
+    ctx.kvd_set_dtype(0)
+    ctx.close()
