@@ -243,6 +243,25 @@ kvd_status kvd_recompute_kv_step(kvd_ctx *ctx, int layer, const kvd_store_range 
                                  const void *rows, const int32_t *positions, int n_rows, void *k_rows_out,
                                  void *v_rows_out, int64_t out_row_stride, void *stream);
 
+/* Everything a decode step of one layer does to K/V and to the store, in ONE launch (Algorithm 1, inside the
+ * layer loop): STORE_RESIDUAL(C, l) for the new tokens, RECOMPUTE_KV(C, l) for the evicted ranges (Eq. 13-14) and
+ * (K_t, V_t) of the new tokens.  As kvd_recompute_kv_step, with two additions:
+ *   append_seqs  HOST int32 [n_rows] or NULL.  Not NULL: row i of `rows` is also appended to the store of
+ *                (layer, append_seqs[i]) -- rows, position and sum of squares, the same bits
+ *                kvd_checkpoint_residual would store -- by the warps of the kernel that read the rows for
+ *                their statistics anyway; n_rows <= 64 (KVD_ERR_CAPACITY beyond).  The appended rows are not
+ *                visible to `ranges` of the same call.
+ *   rows_out_row_stride  row stride (elements, multiple of 8, >= n_kv*d_head; <= 0 selects n_kv*d_head) of
+ *                k_rows_out / v_rows_out alone, so that the new tokens' K and V can be written straight into
+ *                a cache laid out [sequence][position][n_kv*d_head] (stride = positions per sequence x
+ *                n_kv*d_head, base = the slot of the current position) while the recomputed ranges go to a
+ *                scratch with out_row_stride.
+ * Output bits are those of the separate calls.  Nothing is launched or stored when any argument is rejected. */
+kvd_status kvd_decode_step_kv(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
+                              int64_t out_row_stride, const void *rows, const int32_t *positions, int n_rows,
+                              const int32_t *append_seqs, void *k_rows_out, void *v_rows_out,
+                              int64_t rows_out_row_stride, void *stream);
+
 /* ---- FP8 checkpoints (lower-precision residual rows and weights: the second future-work item of the
  * paper's Section 6, which fixes no format; this is the definition this library implements) ----
  * A residual row x (bf16) is stored as E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits,

@@ -38,7 +38,7 @@ EXPORTED_SYMBOLS = (
     "kvd_decode_attention_recompute", "kvd_fused_recompute_pays", "kvd_decode_attention_recompute_fp8", "kvd_set_dtype", "kvd_store_bytes_dtype",
     "kvd_quantize_rows_fp8", "kvd_recompute_kv_fp8_rows", "kvd_decode_attention_recompute_fp8_rows",
     "kvd_store_bytes_fp8", "kvd_attach_store_fp8", "kvd_rows_stored_fp8", "kvd_reset_sequence_fp8", "kvd_checkpoint_residual_fp8", "kvd_recompute_kv_fp8",
-    "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_checkpoint_residual_step", "kvd_recompute_kv",
+    "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_checkpoint_residual_step", "kvd_decode_step_kv", "kvd_recompute_kv",
     "kvd_recompute_kv_step",
     "kvd_decode_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_build_has_checks", "kvd_selftest_bounds_check", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
     "kvd_status_string", "kvd_version",
@@ -139,6 +139,9 @@ def load() -> ctypes.CDLL:
     lib.kvd_recompute_kv.restype = i32
     lib.kvd_recompute_kv_step.argtypes = [vp, i32, ctypes.POINTER(kvd_store_range), i32, vp, vp, i32, vp, vp, i64, vp]
     lib.kvd_recompute_kv_step.restype = i32
+    lib.kvd_decode_step_kv.argtypes = [vp, i32, ctypes.POINTER(kvd_store_range), i32, i64, vp, vp, i32,
+                                       ctypes.POINTER(ctypes.c_int32), vp, vp, i64, vp]
+    lib.kvd_decode_step_kv.restype = i32
     lib.kvd_decode_attention.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
                                          ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
     lib.kvd_decode_attention.restype = i32
@@ -388,6 +391,19 @@ class Kvd:
         self._check(self._lib.kvd_recompute_kv_step(self._h, layer, arr, len(ranges), _ptr(rows), _ptr(positions),
                                                     n_rows, _ptr(k_rows_out), _ptr(v_rows_out), out_row_stride,
                                                     _stream(stream)), "kvd_recompute_kv_step")
+
+    def kvd_decode_step_kv(self, layer: int, ranges: Sequence[Tuple[int, int, int, object, object]], out_row_stride: int,
+                           rows, positions, n_rows: int, append_seqs: Optional[Sequence[int]], k_rows_out, v_rows_out,
+                           rows_out_row_stride: int, stream=None) -> None:
+        """ranges as for kvd_recompute_kv_step; append_seqs: the sequence slot each new row is appended to, or None."""
+        arr = (kvd_store_range * max(len(ranges), 1))()
+        for i, (seq, first_row, n, k_out, v_out) in enumerate(ranges):
+            arr[i].seq, arr[i].first_row, arr[i].n, arr[i].reserved = int(seq), int(first_row), int(n), 0
+            arr[i].k_out, arr[i].v_out = _ptr(k_out), _ptr(v_out)
+        seqs = None if append_seqs is None else (ctypes.c_int32 * max(len(append_seqs), 1))(*[int(x) for x in append_seqs])
+        self._check(self._lib.kvd_decode_step_kv(self._h, layer, arr, len(ranges), out_row_stride, _ptr(rows),
+                                                 _ptr(positions), n_rows, seqs, _ptr(k_rows_out), _ptr(v_rows_out),
+                                                 rows_out_row_stride, _stream(stream)), "kvd_decode_step_kv")
 
     def kvd_decode_attention(self, layer: int, batch: int, q, q_pos: Sequence[int],
                              segs: Sequence[Sequence[Segment]], scale: float, out, stream=None) -> None:

@@ -473,6 +473,11 @@ static void fill_launch_params(const kvd_ctx *ctx, const LayerState &ls, Recompu
   p.trace = nullptr;
   p.ext_rows = nullptr;
   p.w_scale = nullptr;
+  p.rows_out_stride = out_row_stride;
+  p.append_n = 0;
+  p.append_rows = nullptr;
+  p.append_pos = nullptr;
+  p.append_sumsq = nullptr;
   p.store_rows = d.max_tokens_per_seq;
   p.row_chunks = d.d_hidden * dtype_bytes(ctx->dtype) / 16;
   // 32-byte stores need every output row 32-byte aligned
@@ -485,10 +490,17 @@ static void fill_launch_params(const kvd_ctx *ctx, const LayerState &ls, Recompu
 // ranges first, then the caller's rows), launch once.
 // With `fused` (one RcAttend per range, q == nullptr for a range that is to be stored as usual) the
 // ranges that carry a query are attended inside the kernel instead of being written.
+// `step` (kvd_decode_step_kv): a row stride of their own for the caller rows' outputs and, with append_seqs, the
+// rows' STORE_RESIDUAL in the same launch.
+struct StepExtra {
+  int64_t rows_out_stride;
+  const int32_t *append_seqs;  // HOST [n_rows] or nullptr
+};
 static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
                                    const void *rows, const int32_t *positions, int n_rows, void *k_rows_out,
                                    void *v_rows_out, int64_t out_row_stride, cudaStream_t stream,
-                                   const RcAttend *fused = nullptr, const AttnLaunchHead *fused_head = nullptr) {
+                                   const RcAttend *fused = nullptr, const AttnLaunchHead *fused_head = nullptr,
+                                   const StepExtra *step = nullptr) {
   const LayerState &ls = ctx->layers[layer];
   const kvd_model_desc &d = ctx->desc;
   const int kdim = d.n_kv_heads * d.d_head;
@@ -559,6 +571,33 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
   const CUtensorMap &tmap_ext = n_rows > 0 ? tmap_rows : ctx->store_maps[layer];
   fill_launch_params(ctx, ls, p, n_jobs, mb, d.d_hidden * es / (2 * RC_BLOCK_K), out_row_stride);  // 128 bytes per k block
   p.ext_rows = static_cast<const __nv_bfloat16 *>(rows);
+  std::vector<int> add;
+  if (step && n_rows > 0) {
+    if (step->rows_out_stride < kdim) return KVD_ERR_INVALID_ARG;
+    if (step->rows_out_stride * es % 16 != 0) return KVD_ERR_ALIGNMENT;
+    p.rows_out_stride = step->rows_out_stride;
+    if (step->rows_out_stride * es % 32 != 0) p.wide_store = 0;
+    if (step->append_seqs) {
+      // STORE_RESIDUAL of the new rows inside this launch: the host assigns the store slots, the statistics
+      // warps of the main kernel write rows, positions and sums of squares (everything validated before any count moves)
+      if (!ctx->store_rows) return KVD_ERR_STATE;
+      if (layer >= ctx->layers_stored) return KVD_ERR_INVALID_ARG;
+      if (n_rows > RC_INLINE_STAT_ROWS) return KVD_ERR_CAPACITY;
+      add.assign(d.max_seqs, 0);
+      for (int i = 0; i < n_rows; ++i) {
+        const int sq = step->append_seqs[i];
+        if (sq < 0 || sq >= d.max_seqs) return KVD_ERR_INVALID_ARG;
+        const int count = ctx->rows_stored[static_cast<size_t>(layer) * d.max_seqs + sq] + add[sq];
+        if (count + 1 > d.max_tokens_per_seq) return KVD_ERR_CAPACITY;
+        p.append_slot[i] = static_cast<long long>(store_slot(ctx, layer, sq) + count);
+        add[sq] += 1;
+      }
+      p.append_n = n_rows;
+      p.append_rows = reinterpret_cast<uint4 *>(ctx->store_rows);
+      p.append_pos = ctx->store_pos;
+      p.append_sumsq = ctx->store_sumsq;
+    }
+  }
   if (ctx->trace) {
     const int tiles = p.num_m_blocks * p.num_n_blocks;
     const size_t ctas = 2 * static_cast<size_t>(tiles < ctx->num_sms / 2 ? tiles : ctx->num_sms / 2);
@@ -571,7 +610,26 @@ static kvd_status recompute_launch(kvd_ctx *ctx, int layer, const kvd_store_rang
     fp.scale_log2e = fused_head->scale_log2e;
     return launch_recompute_fused(ctx, ls, tmap_store, tmap_ext, p, fp, stream);
   }
-  return launch_recompute(ctx, ls, tmap_store, tmap_ext, p, stream);
+  kvd_status st = launch_recompute(ctx, ls, tmap_store, tmap_ext, p, stream);
+  if (st == KVD_OK && p.append_n > 0)
+    for (int sq = 0; sq < d.max_seqs; ++sq) ctx->rows_stored[static_cast<size_t>(layer) * d.max_seqs + sq] += add[sq];
+  return st;
+}
+
+extern "C" kvd_status kvd_decode_step_kv(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
+                                         int64_t out_row_stride, const void *rows, const int32_t *positions, int n_rows,
+                                         const int32_t *append_seqs, void *k_rows_out, void *v_rows_out,
+                                         int64_t rows_out_row_stride, void *stream_) {
+  if (!ctx || n_ranges < 0 || n_ranges > KVD_MAX_STORE_RANGES || n_rows < 0) return KVD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  if (!ctx->layers[layer].set) return KVD_ERR_STATE;
+  if (n_ranges > 0 && !ranges) return KVD_ERR_INVALID_ARG;
+  const int kdim = ctx->desc.n_kv_heads * ctx->desc.d_head;
+  StepExtra ex;
+  ex.rows_out_stride = rows_out_row_stride > 0 ? rows_out_row_stride : kdim;
+  ex.append_seqs = append_seqs;
+  return recompute_launch(ctx, layer, ranges, n_ranges, rows, positions, n_rows, k_rows_out, v_rows_out,
+                          out_row_stride > 0 ? out_row_stride : kdim, static_cast<cudaStream_t>(stream_), nullptr, nullptr, &ex);
 }
 
 // ------------------------------------------------------------------------------ FP8 checkpoints

@@ -85,6 +85,14 @@ struct RecomputeParams {
   int wide_store;                 // outputs are 32-byte aligned: 32-byte stores
   const float *w_scale;           // FP8 variant: the weight matrix's quantisation scale (one float), else nullptr
   int store_rows;                 // rows per (layer, sequence) slab of the store (checking build)
+  long long rows_out_stride;      // row stride of the caller rows' K/V outputs (the store ranges use out_row_stride)
+  // STORE_RESIDUAL riding in the launch (kvd_decode_step_kv): caller row i is also written to slot append_slot[i]
+  // of the store (rows, position, statistic), by the statistics warps that read it anyway
+  int append_n;                   // 0: nothing is appended
+  uint4 *append_rows;             // the store's rows, 16-byte chunks; slot s at append_rows + s * row_chunks
+  int32_t *append_pos;
+  float *append_sumsq;
+  long long append_slot[RC_INLINE_STAT_ROWS];
   RcJob jobs[RC_MAX_JOBS];
 };
 

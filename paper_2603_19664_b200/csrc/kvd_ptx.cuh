@@ -365,7 +365,7 @@ __device__ __forceinline__ uint32_t pack_out(float lo, float hi) {
 // squares chunks l, l + 32, ... in ascending order into eight partial sums (one per element slot of
 // a chunk, as four two-wide FMAs), adds the eight in a fixed tree, and the 32 lane sums are combined
 // by an xor butterfly (16, 8, 4, 2, 1), so every lane returns the same bits.  With COPY the chunks
-// are also written to `dst`.  (FMAs and adds are explicit: the compiler cannot re-associate them.)  The checkpoint kernel and the recompute kernel both take the statistic
+// are also written to `dst` (rows whose `dst` is null are only summed).  (FMAs and adds are explicit: the compiler cannot re-associate them.)  The checkpoint kernel and the recompute kernel both take the statistic
 // with this one function: its bits do not depend on which of them saw the row.
 template <int DT = 0>
 __device__ __forceinline__ void sumsq_chunk(uint64_t (&ps2)[4], const uint4 &v) {
@@ -411,7 +411,7 @@ __device__ __forceinline__ void warp_rows_sumsq(const uint4 *const (&src)[R], ui
     for (int r = 0; r < R; ++r)
 #pragma unroll
       for (int j = 0; j < B; ++j) {
-        if (COPY) dst[r][c + 32 * j] = v[r][j];
+        if (COPY && dst[r] != nullptr) dst[r][c + 32 * j] = v[r][j];
         sumsq_chunk<DT>(ps2[r], v[r][j]);
       }
   }
@@ -421,7 +421,7 @@ __device__ __forceinline__ void warp_rows_sumsq(const uint4 *const (&src)[R], ui
     for (int r = 0; r < R; ++r) v[r] = __ldg(src[r] + c);
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      if (COPY) dst[r][c] = v[r];
+      if (COPY && dst[r] != nullptr) dst[r][c] = v[r];
       sumsq_chunk<DT>(ps2[r], v[r]);
     }
   }

@@ -528,17 +528,32 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
           // leave 1/rms in s_rstd[a] and meet on a barrier before every thread picks up its own row.
           // Rows past the end of the job read the job's last row instead (no branch inside a group).
           const uint4 *base = reinterpret_cast<const uint4 *>(p.ext_rows) + static_cast<size_t>(m0) * p.row_chunks;
+          // STORE_RESIDUAL in the same launch: the tile of the first column block also writes the rows it reads
+          // (with their positions and statistics) into the store slots the host assigned to them
+          const bool append = p.append_n > 0 && n0_ == 0;
 #pragma unroll 1
           for (int g = w4; g < 32 && 4 * g < n_here; g += 4) {
             const uint4 *src[4];
-            uint4 *const none[4] = {nullptr, nullptr, nullptr, nullptr};
+            uint4 *dst[4] = {nullptr, nullptr, nullptr, nullptr};
 #pragma unroll
-            for (int i = 0; i < 4; ++i) src[i] = base + static_cast<size_t>(4 * g + i < n_here ? 4 * g + i : n_here - 1) * p.row_chunks;
+            for (int i = 0; i < 4; ++i) {
+              const int r = 4 * g + i;
+              src[i] = base + static_cast<size_t>(r < n_here ? r : n_here - 1) * p.row_chunks;
+              if (append && r < n_here && m0 + r < p.append_n)
+                dst[i] = p.append_rows + static_cast<size_t>(p.append_slot[m0 + r]) * p.row_chunks;
+            }
             float ss[4];
-            warp_rows_sumsq<4, 4, false, DT>(src, none, p.row_chunks, lane, ss);
+            if (append) warp_rows_sumsq<4, 4, true, DT>(src, dst, p.row_chunks, lane, ss);
+            else warp_rows_sumsq<4, 4, false, DT>(src, dst, p.row_chunks, lane, ss);
             const float mine = lane == 0 ? ss[0] : lane == 1 ? ss[1] : lane == 2 ? ss[2] : ss[3];
-            if (lane < 4 && 4 * g + lane < n_here)
+            if (lane < 4 && 4 * g + lane < n_here) {
               s_rstd[a * RC_BLOCK_M + 4 * g + lane] = 1.0f / sqrtf(mine * p.inv_d_hidden + p.rms_eps);
+              if (append && m0 + 4 * g + lane < p.append_n) {
+                const long long slot = p.append_slot[m0 + 4 * g + lane];
+                p.append_sumsq[slot] = mine;
+                p.append_pos[slot] = J.positions[m0 + 4 * g + lane];
+              }
+            }
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_stats_x);
@@ -600,6 +615,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
       const int m = m0 + row;
       const bool valid = m < J.n;
       const bool wide = p.wide_store != 0;
+      const long long out_stride = J.slab < 0 ? p.rows_out_stride : p.out_row_stride;  // the caller's rows may go elsewhere
       const float rstd = s_rstd[a * RC_BLOCK_M + row];
       int pos = valid ? J.positions[m] : 0;
       if (pos < 0 || pos >= p.max_pos) {
@@ -722,7 +738,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
         const uint32_t tcol = acc + hh * D_HEAD;
         if (col0 >= p.k_cols) {
           // ---- value head (Eq. 14): scale by 1/rms and store
-          __nv_bfloat16 *dst = J.v_out + (static_cast<size_t>(m) * p.out_row_stride + (col0 - p.k_cols)) * EW;
+          __nv_bfloat16 *dst = J.v_out + (static_cast<size_t>(m) * out_stride + (col0 - p.k_cols)) * EW;
 #pragma unroll 1
           for (int c = 0; c < D_HEAD / 32; ++c) {
             uint32_t r[32];
@@ -736,7 +752,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
           }
         } else {
           // ---- key head (Eq. 13): 1/rms, optional key norm, rotation R_pos
-          __nv_bfloat16 *dst = J.k_out + (static_cast<size_t>(m) * p.out_row_stride + col0) * EW;
+          __nv_bfloat16 *dst = J.k_out + (static_cast<size_t>(m) * out_stride + col0) * EW;
           float kscale = rstd;
           // fused, attending job: the rotated key (rounded to bf16 like a stored one) is not written but
           // multiplied with the NG queries of this KV head (Eq. 6); two-wide partial sums per query

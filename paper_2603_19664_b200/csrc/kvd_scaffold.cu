@@ -295,6 +295,11 @@ extern "C" kvd_status kvd_scaffold_linear(kvd_ctx *ctx, const kvd_linear *lin, c
   p.row_chunks = lin->k / 8;
   p.wide_store = (out_row_stride * 2 % 32 == 0) && ((reinterpret_cast<uintptr_t>(out) & 31u) == 0);
   p.w_scale = nullptr;
+  p.rows_out_stride = out_row_stride;
+  p.append_n = 0;
+  p.append_rows = nullptr;
+  p.append_pos = nullptr;
+  p.append_sumsq = nullptr;
   p.store_rows = m;
   return launch_recompute(ctx, lin->ls, tmap_rows, tmap_rows, p, stream);
 }

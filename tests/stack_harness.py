@@ -363,8 +363,6 @@ class BatchStack:
         n_old_max = max(ctx_len + max_steps - window, 1)
         self.k_old = torch.zeros((batch, n_old_max, self.kdim), dtype=torch.bfloat16, device="cuda")
         self.v_old = torch.zeros_like(self.k_old)
-        self.k_new = torch.zeros((batch, self.kdim), dtype=torch.bfloat16, device="cuda")
-        self.v_new = torch.zeros_like(self.k_new)
         # ---- the context: rows into the store, their K/V into the cache
         g = torch.Generator(device="cuda")
         g.manual_seed(3000 + seed)
@@ -417,26 +415,19 @@ class BatchStack:
                 raw = self._linear(self.lin[l]["q"], h)
                 ctx.kvd_scaffold_query_finish(l, raw, raw.shape[1], pos_t, B, self.lw[l].get("gamma_q") if s.qk_norm else None, q)
             if policy == "kvdirect":
-                ctx.kvd_checkpoint_residual_step(l, list(range(B)), h, pos_t)  # STORE_RESIDUAL, the whole batch at once
                 n_old = max(0, wf - lo)
                 ranges = [(b, lo, n_old, self.k_old[b], self.v_old[b]) for b in range(B)] if n_old > 0 else []
-                # RECOMPUTE_KV for the evicted positions of every sequence + K_t, V_t of the new tokens: one launch
-                # (one row stride for all outputs of the call, so K_t, V_t land in a [batch, kdim] buffer)
-                ctx.kvd_recompute_kv_step(l, ranges, h, pos_t, B, self.k_new, self.v_new, kdim)
+                # STORE_RESIDUAL of the new rows, RECOMPUTE_KV for the evicted positions of every sequence and K_t, V_t
+                # of the new tokens written straight into the cache rows of the current position: ONE launch
+                ctx.kvd_decode_step_kv(l, ranges, kdim, h, pos_t, B, list(range(B)), kc[0, pos], vc[0, pos], mt * kdim)
                 self.recomputed_rows += B * n_old
                 first_live = max(wf, lo)
                 segs = [[(self.k_old[b], self.v_old[b], kdim, lo, n_old),
-                         (kc[b, first_live], vc[b, first_live], kdim, first_live, pos - first_live),
-                         (self.k_new[b], self.v_new[b], kdim, pos, 1)] for b in range(B)]
-                kv_new = True
+                         (kc[b, first_live], vc[b, first_live], kdim, first_live, pos + 1 - first_live)] for b in range(B)]
             else:
                 ctx.kvd_recompute_kv(l, h, pos_t, B, kc[0, pos], vc[0, pos], mt * kdim)
                 segs = [[(kc[b, lo], vc[b, lo], kdim, lo, pos + 1 - lo)] for b in range(B)]
-                kv_new = False
             ctx.kvd_decode_attention(l, B, q, qpos, segs, 0.0, out)
-            if kv_new:  # the new entries join the live window (a device copy, after attention as in Algorithm 1)
-                kc[:, pos].copy_(self.k_new)
-                vc[:, pos].copy_(self.v_new)
             if scaffold:
                 y = self._linear(self.lin[l]["o"], out.view(B, -1))
                 ctx.kvd_scaffold_add_rows(h, y, y.shape[1], B, s.d_hidden)

@@ -441,3 +441,71 @@ def test_bounded_wait_expires_and_is_reported_without_harming_the_device():
     assert torch.equal(K, K2) and torch.equal(V, V2)
     t = tr.cpu().numpy()
     assert t[0, 0, 5] > t[0, 0, 4] > 0 and t[0, 0, 7] > t[0, 0, 6] > 0  # MMA and epilogue intervals of tile 0
+
+
+@pytest.mark.parametrize("shape", [GEMMA3_4B_GLOBAL, SMOLLM2_135M], ids=lambda s: s.name)
+def test_decode_step_kv_equals_the_separate_calls_bit_for_bit(shape):
+    """kvd_decode_step_kv = STORE_RESIDUAL of the new rows + RECOMPUTE_KV of the evicted ranges + (K_t, V_t), one
+    launch: the store (rows, positions, statistics, counts), the recomputed K/V and the new tokens' K/V written
+    with a stride of their own must equal what kvd_checkpoint_residual_step + kvd_recompute_kv_step leave."""
+    batch, T, max_tokens = 5, 300, 512
+    kdim = shape.n_kv_heads * shape.d_head
+    desc_args = dict(max_tokens=max_tokens, max_batch=batch, max_seqs=batch, with_store=True)
+    ctx_a, w = open_layer(shape, **desc_args)
+    ctx_b, _ = open_layer(shape, **desc_args)
+    arena_a, arena_b = ctx_a._keep[-1], ctx_b._keep[-1]
+    arena_a.zero_()
+    arena_b.zero_()
+    X = dev(make_residuals(shape, T + batch, seed=31, outliers=True))
+    pos = torch.arange(T, dtype=torch.int32, device="cuda")
+    for b in range(batch):
+        rows = torch.roll(X[:T], shifts=-7 * b, dims=0).contiguous()
+        for c in (ctx_a, ctx_b):
+            c.kvd_checkpoint_residual(b, 0, rows, pos, T - b)   # ragged: sequence b holds T - b rows
+    x_new = X[T:T + batch].contiguous()
+    p_new = torch.tensor([T - b for b in range(batch)], dtype=torch.int32, device="cuda")
+    n_old = [T - b - 40 for b in range(batch)]
+    ko = [torch.zeros((T, kdim), dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    vo = [torch.zeros((T, kdim), dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    # (a) separate calls, contiguous K_t/V_t
+    ka, va = torch.zeros((batch, kdim), dtype=torch.bfloat16, device="cuda"), torch.zeros((batch, kdim), dtype=torch.bfloat16, device="cuda")
+    ctx_a.kvd_checkpoint_residual_step(0, list(range(batch)), x_new, p_new)
+    ctx_a.kvd_recompute_kv_step(0, [(b, 3, n_old[b], ko[0][3:], vo[0][3:]) for b in range(1)] +
+                                [(b, 0, 0, None, None) for b in range(1, batch)], x_new, p_new, batch, ka, va, kdim)
+    # (b) one launch; K_t/V_t scattered into a [batch][max_tokens][kdim] cache at each sequence's position 9
+    cache_k = torch.full((batch, max_tokens, kdim), 7.0, dtype=torch.bfloat16, device="cuda")
+    cache_v = torch.full_like(cache_k, 7.0)
+    n0 = ctx_b.kvd_launch_count()
+    ctx_b.kvd_decode_step_kv(0, [(0, 3, n_old[0], ko[1][3:], vo[1][3:])], kdim, x_new, p_new, batch, list(range(batch)),
+                             cache_k[0, 9], cache_v[0, 9], max_tokens * kdim)
+    assert ctx_b.kvd_launch_count() - n0 == 1
+    assert ctx_a.kvd_poll_status() == kvd.KVD_OK and ctx_b.kvd_poll_status() == kvd.KVD_OK
+    assert torch.equal(arena_a, arena_b), "store contents differ"
+    for b in range(batch):
+        assert ctx_a.kvd_rows_stored(0, b) == ctx_b.kvd_rows_stored(0, b) == T - b + 1
+    assert torch.equal(ko[0], ko[1]) and torch.equal(vo[0], vo[1])
+    assert torch.equal(cache_k[:, 9], ka) and torch.equal(cache_v[:, 9], va)
+    untouched = torch.ones((max_tokens,), dtype=torch.bool, device="cuda")
+    untouched[9] = False
+    assert torch.all(cache_k[:, untouched] == 7.0) and torch.all(cache_v[:, untouched] == 7.0)
+    # the appended rows can be recomputed from the store like any other (same bits as from the caller's buffer)
+    k2, v2 = torch.zeros((1, kdim), dtype=torch.bfloat16, device="cuda"), torch.zeros((1, kdim), dtype=torch.bfloat16, device="cuda")
+    for b in (0, batch - 1):
+        ctx_b.kvd_recompute_kv(0, None, None, 1, k2, v2, kdim, seq=b, first_row=T - b)
+        assert torch.equal(k2[0], ka[b]) and torch.equal(v2[0], va[b])
+    # limits: more than 64 appended rows, a full sequence, a bad slot -- nothing stored
+    before = [ctx_b.kvd_rows_stored(0, b) for b in range(batch)]
+    big = torch.zeros((65, shape.d_hidden), dtype=torch.bfloat16, device="cuda")
+    pb = torch.zeros((65,), dtype=torch.int32, device="cuda")
+    kb, vb = torch.zeros((65, kdim), dtype=torch.bfloat16, device="cuda"), torch.zeros((65, kdim), dtype=torch.bfloat16, device="cuda")
+    for seqs, n, status in (([0] * 65, 65, 4), ([batch], 1, 1), ([0] * 64, 64, 4 if before[0] + 64 > max_tokens else 0)):
+        try:
+            ctx_b.kvd_decode_step_kv(0, [], kdim, big, pb, n, seqs, kb, vb, kdim)
+            got = 0
+        except kvd.KvdError as e:
+            got = e.status
+        assert got == status, (seqs[:2], n, got)
+    if before[0] + 64 > max_tokens:
+        assert [ctx_b.kvd_rows_stored(0, b) for b in range(batch)] == before
+    ctx_a.close()
+    ctx_b.close()
