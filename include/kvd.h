@@ -330,6 +330,16 @@ kvd_status kvd_recompute_kv_fp8_rows(kvd_ctx *ctx, int layer, const kvd_store_ra
 kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, const void *q, const int32_t *q_pos,
                                 const kvd_kv_segment *segs, int n_segs, float scale, void *out, void *stream);
 
+/* ATTENTION of Algorithm 1 for SEVERAL tokens of ONE sequence, each with its own causal limit (a prefill segment, or
+ * the replay of an evicted prefix when only one residual row per token is kept): row i of q (DEVICE [n_rows,
+ * n_q_heads, d_head]) is the query of the token at position q_pos[i] (HOST int32 [n_rows]) and attends the keys of
+ * `segs` (HOST [n_segs]: the one sequence's segments, shared by all rows) at positions <= q_pos[i], inside the
+ * layer's window.  out DEVICE [n_rows, n_q_heads, d_head].  Every row's result has the bits kvd_decode_attention
+ * gives for that query alone: the rows go through the same kernels, as many per launch as the workspace's
+ * partial slots hold (at most 64), so the call is a host loop over launches, not one launch. */
+kvd_status kvd_decode_attention_rows(kvd_ctx *ctx, int layer, int n_rows, const void *q, const int32_t *q_pos,
+                                     const kvd_kv_segment *segs, int n_segs, float scale, void *out, void *stream);
+
 /* RECOMPUTE_KV and ATTENTION of Algorithm 1 in one pass for the evicted tokens (Eq. 13-14 feeding
  * Eq. 6-7): the keys and values rebuilt from the residual rows of ranges[b] are consumed inside the
  * recompute kernel -- the rotated key of a row is multiplied with the queries of its KV head, the value

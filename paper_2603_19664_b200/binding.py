@@ -40,7 +40,7 @@ EXPORTED_SYMBOLS = (
     "kvd_store_bytes_fp8", "kvd_attach_store_fp8", "kvd_rows_stored_fp8", "kvd_reset_sequence_fp8", "kvd_checkpoint_residual_fp8", "kvd_recompute_kv_fp8",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_checkpoint_residual_step", "kvd_decode_step_kv", "kvd_recompute_kv",
     "kvd_recompute_kv_step",
-    "kvd_decode_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_build_has_checks", "kvd_selftest_bounds_check", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
+    "kvd_decode_attention", "kvd_decode_attention_rows", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_build_has_checks", "kvd_selftest_bounds_check", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
     "kvd_status_string", "kvd_version",
     # include/kvd_scaffold.h: the parts of a decoder layer around the hot path, for whole-stack tests and benchmarks
     "kvd_scaffold_linear_create", "kvd_scaffold_linear_destroy", "kvd_scaffold_linear_out_cols", "kvd_scaffold_linear",
@@ -147,6 +147,9 @@ def load() -> ctypes.CDLL:
     lib.kvd_decode_attention.restype = i32
     lib.kvd_fused_recompute_pays.argtypes = [ctypes.POINTER(kvd_model_desc), i64, i32]
     lib.kvd_fused_recompute_pays.restype = i32
+    lib.kvd_decode_attention_rows.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
+                                              ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
+    lib.kvd_decode_attention_rows.restype = i32
     lib.kvd_set_dtype.argtypes = [vp, i32]
     lib.kvd_set_dtype.restype = i32
     lib.kvd_store_bytes_fp8.argtypes = [ctypes.POINTER(kvd_model_desc), i32]
@@ -422,6 +425,15 @@ class Kvd:
                     e.k, e.v, e.row_stride, e.first_pos, e.len = None, None, 0, 0, 0
         self._check(self._lib.kvd_decode_attention(self._h, layer, batch, _ptr(q), pos_arr, seg_arr, n_segs,
                                                    float(scale), _ptr(out), _stream(stream)), "kvd_decode_attention")
+
+    def kvd_decode_attention_rows(self, layer: int, n_rows: int, q, q_pos: Sequence[int], segs: Sequence[Segment],
+                                  scale: float, out, stream=None) -> None:
+        """Several query rows of one sequence (segs: that sequence's segments), each with its own position."""
+        n_segs, _, seg_arr = _marshal_segments(1, [0], [list(segs)])
+        pos_arr = (ctypes.c_int32 * max(n_rows, 1))(*[int(p) for p in q_pos])
+        self._check(self._lib.kvd_decode_attention_rows(self._h, layer, n_rows, _ptr(q), pos_arr, seg_arr, n_segs,
+                                                        float(scale), _ptr(out), _stream(stream)),
+                    "kvd_decode_attention_rows")
 
     def kvd_decode_attention_recompute(self, layer: int, batch: int, q, q_pos: Sequence[int],
                                        ranges: Sequence[Tuple[int, int, int]], rows, positions, n_rows: int,

@@ -982,6 +982,54 @@ extern "C" int kvd_fused_recompute_pays(const kvd_model_desc *desc, int64_t tota
   return total_rows >= (fp8 ? 4096 : 16384) ? 1 : 0;
 }
 
+extern "C" kvd_status kvd_decode_attention_rows(kvd_ctx *ctx, int layer, int n_rows, const void *q, const int32_t *q_pos,
+                                                const kvd_kv_segment *segs, int n_segs, float scale, void *out,
+                                                void *stream_) {
+  if (!ctx || n_rows < 0 || n_segs < 0 || n_segs > KVD_MAX_SEGMENTS) return KVD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return KVD_ERR_INVALID_ARG;
+  const LayerState &ls = ctx->layers[layer];
+  if (!ls.set) return KVD_ERR_STATE;
+  if (!ctx->part_o) return KVD_ERR_STATE;
+  if (ctx->dtype == KVD_DTYPE_F32) return KVD_ERR_UNSUPPORTED;
+  if (n_rows == 0) return KVD_OK;
+  if (!q || !q_pos || !out || (n_segs > 0 && !segs)) return KVD_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out)) return KVD_ERR_ALIGNMENT;
+  const kvd_model_desc &d = ctx->desc;
+  const int group = d.n_q_heads / d.n_kv_heads;
+  // the one sequence's segments, validated once with a query position that every row's replaces below
+  int32_t zero = 0;
+  kvd_status st = check_segments(ctx, 1, &zero, segs, n_segs);
+  if (st != KVD_OK) return st;
+  for (int i = 0; i < n_rows; ++i)
+    if (q_pos[i] < 0) return KVD_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  static thread_local AttnLaunch L;  // large: keep it off the stack
+  // every row is a "sequence" of a decode-attention launch that shares the segments; a launch takes as many
+  // rows as the launch descriptor (AT_MAX_SEQS) and the workspace's partial slots (max_parts) hold
+  std::vector<kvd_kv_segment> rep(static_cast<size_t>(AT_MAX_SEQS) * (n_segs > 0 ? n_segs : 1));
+  for (int i = 0; i < AT_MAX_SEQS; ++i)
+    for (int sg = 0; sg < n_segs; ++sg) rep[static_cast<size_t>(i) * n_segs + sg] = segs[sg];
+  const size_t row_elems = static_cast<size_t>(d.n_q_heads) * d.d_head;
+  const int es = 2;  // bf16 or fp16 queries and outputs
+  int r0 = 0;
+  while (r0 < n_rows) {
+    int nb = n_rows - r0 < AT_MAX_SEQS ? n_rows - r0 : AT_MAX_SEQS;
+    const uint8_t *qb = static_cast<const uint8_t *>(q) + static_cast<size_t>(r0) * row_elems * es;
+    uint8_t *ob = static_cast<uint8_t *>(out) + static_cast<size_t>(r0) * row_elems * es;
+    // shrink the launch until its partials fit the workspace (one row always has to)
+    while (true) {
+      st = build_attn_launch(ctx, ls, 0, nb, qb, q_pos + r0, rep.data(), n_segs, scale, ob, nullptr, L);
+      if (st != KVD_ERR_CAPACITY || nb == 1) break;
+      nb = nb / 2;
+    }
+    if (st != KVD_OK) return st;
+    st = launch_attention(ctx, L, d.d_head, group, stream);
+    if (st != KVD_OK) return st;
+    r0 += nb;
+  }
+  return KVD_OK;
+}
+
 // Decode attention over [K/V recomputed from store ranges] + [live segments], the recomputed part
 // inside the recompute kernel (its K/V never reach memory); see kvd.h.
 extern "C" kvd_status kvd_decode_attention_recompute(kvd_ctx *ctx, int layer, int batch, const void *q,

@@ -214,9 +214,7 @@ class GpuStack:
             first_live = max(wf, lo_min) if self.policy == "kvdirect" else 0
             segs.append((kl[first_live:], vl[first_live:], self.kdim, first_live, p0 + U - first_live))
             out = torch.empty((U, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
-            for b0 in range(0, U, 64):
-                nb = min(64, U - b0)
-                ctx.kvd_decode_attention(l, nb, q[b0:], positions[b0:b0 + nb], [segs] * nb, 0.0, out[b0:])
+            ctx.kvd_decode_attention_rows(l, U, q, positions, segs, 0.0, out)
             h = self._after_attention(l, h, out)
             if self.policy == "kvdirect":
                 self.win_first[l] = max(self.win_first[l], p0 + U - self.budget)
@@ -290,18 +288,14 @@ class GpuStackChained(GpuStack):
             segs_new.append((kl[N:], vl[N:], self.kdim, N, p0 + U - N))
             q_new = self._queries(l, h_new, pos_new_t)
             out_new = torch.empty((U, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
-            for b0 in range(0, U, 64):
-                nb = min(64, U - b0)
-                ctx.kvd_decode_attention(l, nb, q_new[b0:], pos_new[b0:b0 + nb], [segs_new] * nb, 0.0, out_new[b0:])
+            ctx.kvd_decode_attention_rows(l, U, q_new, pos_new, segs_new, 0.0, out_new)
             if N > 0 and l + 1 < s.n_layers:
                 # the evicted tokens' own step through this layer: each attends to the evicted keys up
                 # to its own position (the position mask does the rest)
                 q_old = self._queries(l, h_old, pos_old_t)
                 out_old = torch.empty((N, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
                 segs_old = [(self.k_old, self.v_old, self.kdim, 0, N)]
-                for b0 in range(0, N, 64):
-                    nb = min(64, N - b0)
-                    ctx.kvd_decode_attention(l, nb, q_old[b0:], pos_old[b0:b0 + nb], [segs_old] * nb, 0.0, out_old[b0:])
+                ctx.kvd_decode_attention_rows(l, N, q_old, pos_old, segs_old, 0.0, out_old)
                 h_old = self._after_attention(l, h_old, out_old)
                 self.replayed_rows += N
             h_new = self._after_attention(l, h_new, out_new)

@@ -249,3 +249,35 @@ def test_argument_errors():
     assert e.value.status == 4
     ctx.kvd_decode_attention(0, 2, q, [7, 7], [ok, ok], 0.0, out)
     assert ctx.kvd_poll_status() == kvd.KVD_OK
+
+
+@pytest.mark.parametrize("shape", [GEMMA3_4B_LOCAL, QWEN3_4B], ids=lambda s: s.name)
+def test_rows_of_one_sequence_with_their_own_causal_limit(shape):
+    """kvd_decode_attention_rows: many query tokens of one sequence over shared segments, each seeing the keys up
+    to its own position (and inside the window): every row must have the bits of a kvd_decode_attention call for
+    that query alone, and follow the oracle called per row.  A small workspace forces several launches."""
+    T, n_rows = 1500, 150
+    ctx, _ = open_layer(shape, max_tokens=2048, max_batch=2)  # room for two sequences' partials: many launches
+    kdim = shape.n_kv_heads * shape.d_head
+    K, V = make_kv(shape, T, seed=5)
+    cut = 900
+    segs_bits = [(K[:cut], V[:cut], 0), (K[cut:], V[cut:], cut)]
+    rng = np.random.default_rng(8)
+    q_pos = sorted(rng.choice(np.arange(3, T + 40), n_rows, replace=False).tolist())  # some beyond the last key
+    q_bits = make_query(shape, n_rows, seed=6)
+    q = dev(q_bits)
+    k0, v0, k1, v1 = dev(K[:cut]), dev(V[:cut]), dev(K[cut:]), dev(V[cut:])
+    segs = [(k0, v0, kdim, 0, cut), (k1, v1, kdim, cut, T - cut)]
+    out = torch.full((n_rows, shape.n_q_heads, shape.d_head), 9.0, dtype=torch.bfloat16, device="cuda")
+    n0 = ctx.kvd_launch_count()
+    ctx.kvd_decode_attention_rows(0, n_rows, q, q_pos, segs, 0.0, out)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    assert ctx.kvd_launch_count() - n0 > 2 * (n_rows // 64 + 1)  # the small workspace split the rows further
+    one = torch.empty((1, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda")
+    for i in (0, 1, 63, 64, 77, n_rows - 1):
+        ctx.kvd_decode_attention(0, 1, q[i:i + 1], [q_pos[i]], [segs], 0.0, one)
+        assert torch.equal(one[0], out[i]), i
+    sample = [0, 5, 64, 100, n_rows - 1]
+    ref = oracle_attention(shape, q_bits[sample], [q_pos[i] for i in sample], [segs_bits] * len(sample))
+    attn_check(host_f64(out[torch.tensor(sample).cuda()]), ref)
+    ctx.close()
