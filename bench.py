@@ -676,7 +676,8 @@ def run_gpu(args):
     long_attn = measure_long_attention(wl, peaks, timed_graph) if rank == 0 else None
     stack_decode = None
     if rank == 0 and world == 1 and not args.no_stack:
-        stack_decode = measure_stack_decode((1, 4, 16, 64) if args.stack_all else (1, 4))
+        stack_decode = measure_stack_decode((1, 4, 16, 64) if args.stack_all else (1, 4),
+                                            **({"session_turns": 3, "session_gen": 16, "seg": (256, 512)} if args.short_session else {}))
     sweep = run_sweep(wl, peaks) if args.sweep and rank == 0 else None
 
     if rank == 0:
@@ -761,16 +762,16 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
-def measure_stack_decode(batches, n_check_steps=4, session_turns=3, session_gen=16):
+def measure_stack_decode(batches, n_check_steps=4, session_turns=20, session_gen=128, seg=(256, 1024)):
     """Configs 3 and 5 on the whole 34-layer Gemma-3-4B-shaped stack, nothing multiplied: a decode step of
     `batch` sequences with 2048 tokens of context behind them and a 256-token window, KV-Direct arm against
     full-cache arm from one shared state (tests/stack_harness.py: BatchStack).  Every kernel on the path is
     the library's (hot path through include/kvd.h, the rest of the block through include/kvd_scaffold.h).
     The step is captured into a CUDA graph and replayed; the hot path is also timed alone (same launches
     without the scaffold) so that the scaffold's share is visible.  Tokens of the two arms over
-    `n_check_steps` greedy steps must be identical.  Then a shortened config-5 session (full-size stack,
-    `session_turns` turns of a 256-512-token user segment + `session_gen` greedy tokens) checks the token
-    match through prefill and decode."""
+    `n_check_steps` greedy steps must be identical.  Then the config-5 session (full-size stack, `session_turns`
+    turns of a user segment of seg[0]..seg[1] random tokens + `session_gen` greedy tokens, run once per cache
+    policy) checks the token match through prefill and decode and reports the memory held."""
     import torch
     sys.path.insert(0, os.path.join(ROOT, "tests"))
     from kvd_synth import GEMMA3_4B_STACK
@@ -822,7 +823,7 @@ def measure_stack_decode(batches, n_check_steps=4, session_turns=3, session_gen=
         del m
         torch.cuda.empty_cache()
         rows.append(rec)
-    seg = (256, 512)
+    t_session = time.perf_counter()
     recs, ok = run_session(stack, w, session_turns, session_gen, window, seg[0], seg[1],
                            session_turns * (seg[1] + session_gen) + 8)
     session = {"stack": stack.name, "turns": session_turns, "generated_per_turn": session_gen, "window": window,
@@ -830,7 +831,12 @@ def measure_stack_decode(batches, n_check_steps=4, session_turns=3, session_gen=
                "all_tokens_match": bool(ok), "peak_full_cache_kv_bytes": max(r["full_cache_kv_bytes"] for r in recs),
                "peak_kvdirect_live_kv_bytes": max(r["kvdirect_live_kv_bytes"] for r in recs),
                "rows_recomputed": recs[-1]["rows_recomputed_so_far"],
-               "note": "shortened form of the 20-turn session (python tests/session_config5.py runs all 20 turns)"}
+               "final_per_layer_checkpoint_bytes": recs[-1]["kvdirect_checkpoint_bytes_per_layer_rows"],
+               "eq28_bytes_single_checkpoint_accounting": recs[-1]["kvdirect_eq28_bytes_single_checkpoint_accounting"],
+               "last_turn_seconds_full_cache": recs[-1]["seconds_full_cache"],
+               "last_turn_seconds_kvdirect": recs[-1]["seconds_kvdirect"],
+               "wall_seconds_both_arms": time.perf_counter() - t_session,
+               "note": "config 5 of BASELINE.json on the full-size stack; python tests/session_config5.py prints it per turn"}
     return {"config3_gemma3_4b_stack_ctx2048_window256": rows, "config5_session": session,
             "note": "34 layers, every launch measured (CUDA graph of one whole decode step, 10 replays); "
                     "scaffold = the block's other products and small steps on the library's own kernels"}
@@ -1259,6 +1265,7 @@ def main():
     ap.add_argument("--profile-qwen", action="store_true",
                     help="eager launches of the Qwen3-4B-shaped layer's kernels (reduced long-context case) for a profiler")
     ap.add_argument("--no-stack", action="store_true", help="skip the whole-stack decode step (configs 3 and 5)")
+    ap.add_argument("--short-session", action="store_true", help="config 5 with 3 turns of 16 tokens instead of 20 of 128")
     ap.add_argument("--stack-all", action="store_true", help="whole-stack decode step at batch 1, 4, 16 and 64")
     ap.add_argument("--stack-configs", action="store_true",
                     help="time the hot path of the stack-shaped configurations instead of the contract line")

@@ -133,9 +133,9 @@ kvd_status kvd_create(const kvd_model_desc *desc, kvd_ctx **out);
 void kvd_destroy(kvd_ctx *ctx);
 
 /* Element type of residual rows, weights, K/V, queries and attention outputs.  bf16 is the default and the
- * only type the fused, FP8 and static entry points accept (KVD_ERR_UNSUPPORTED otherwise); fp16 exists for
- * kvd_checkpoint_residual / kvd_recompute_kv / kvd_recompute_kv_step / kvd_decode_attention, fp32 for the
- * first three (rows, weights and K/V outputs are fp32, strides count fp32 elements, the tensor cores read the
+ * only type the FP8 and static entry points accept (KVD_ERR_UNSUPPORTED otherwise); fp16 exists for
+ * kvd_checkpoint_residual / kvd_recompute_kv / kvd_recompute_kv_step / kvd_decode_step_kv / kvd_decode_attention /
+ * kvd_decode_attention_rows / kvd_decode_attention_recompute, fp32 for the checkpoint and recompute calls (rows, weights and K/V outputs are fp32, strides count fp32 elements, the tensor cores read the
  * operands as TF32 and accumulate in fp32) -- the reconstruction identities (Eq. 13-14) do not depend on the
  * element type, and the bitwise recompute-equals-first-pass check of the paper's Section 5.1 is run in all
  * three.  Call before kvd_set_layer, kvd_attach_store (when the element size changes) and any checkpoint

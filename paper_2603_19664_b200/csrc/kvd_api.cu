@@ -1043,7 +1043,7 @@ extern "C" kvd_status kvd_decode_attention_recompute(kvd_ctx *ctx, int layer, in
   const LayerState &ls = ctx->layers[layer];
   if (!ls.set) return KVD_ERR_STATE;
   if (!ctx->part_o || !ctx->store_rows) return KVD_ERR_STATE;
-  if (ctx->dtype != KVD_DTYPE_BF16) return KVD_ERR_UNSUPPORTED;
+  if (ctx->dtype == KVD_DTYPE_F32) return KVD_ERR_UNSUPPORTED;  // bf16 and fp16 contexts
   const kvd_model_desc &d = ctx->desc;
   const int group = d.n_q_heads / d.n_kv_heads, kdim = d.n_kv_heads * d.d_head;
   // shapes the fused kernel is built for (nothing is launched otherwise)

@@ -213,8 +213,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
   using Cfg = RcCfg<BLOCK_N, D_HEAD, FG, LOSM>;
   constexpr int STAGES = Cfg::STAGES;
   constexpr bool FUSED = FG > 0;
-  static_assert(DT == 0 || (FG == 0 && ((DT == 1 && EB == 2) || (DT == 2 && EB == 4))),
-                "fp16 and fp32 exist for the plain variant only");
+  static_assert(DT == 0 || (DT == 1 && EB == 2) || (DT == 2 && EB == 4 && FG == 0),
+                "fp16 exists for the plain and the fused variant on 16-bit rows, fp32 for the plain variant only");
   constexpr int EW = DT == 2 ? 2 : 1;  // 16-bit units per output element (output pointers count 16-bit units)
   constexpr int KB_ELEMS = RC_BLOCK_K * 2 / EB;  // channels per k block
   static_assert(BLOCK_N % D_HEAD == 0, "a tile must hold whole heads");
@@ -822,7 +822,7 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
                   const uint4 q0 = __ldg(qh + (g * D_HEAD + c * 16) / 8), q1 = __ldg(qh + (g * D_HEAD + c * 16) / 8 + 1);
                   const uint32_t qw[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
 #pragma unroll
-                  for (int w = 0; w < 8; ++w) sdot[g] = ffma2(bf16x2_to_f32x2(o[w]), bf16x2_to_f32x2(qw[w]), sdot[g]);
+                  for (int w = 0; w < 8; ++w) sdot[g] = ffma2(x2_to_f32x2<DT>(o[w]), x2_to_f32x2<DT>(qw[w]), sdot[g]);
                 }
               } else if (valid) {
                 store_row_piece<2 * EW>(dst + c * 16 * EW, o, wide);
@@ -869,8 +869,8 @@ kvd_recompute_kernel(const __grid_constant__ CUtensorMap tmap_store, const __gri
                   const uint32_t qb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
                   for (int w = 0; w < 8; ++w) {
-                    sdot[g] = ffma2(bf16x2_to_f32x2(oa[w]), bf16x2_to_f32x2(qa[w]), sdot[g]);
-                    sdot[g] = ffma2(bf16x2_to_f32x2(ob[w]), bf16x2_to_f32x2(qb[w]), sdot[g]);
+                    sdot[g] = ffma2(x2_to_f32x2<DT>(oa[w]), x2_to_f32x2<DT>(qa[w]), sdot[g]);
+                    sdot[g] = ffma2(x2_to_f32x2<DT>(ob[w]), x2_to_f32x2<DT>(qb[w]), sdot[g]);
                   }
                 }
               } else if (valid) {
@@ -988,6 +988,10 @@ static kvd_status launch_sel(kvd_ctx *ctx, const LayerState &ls, const CUtensorM
     // one tile per cluster at most: every key tile's epilogue is exposed -> the low table from shared memory
     if (p.num_m_blocks * p.num_n_blocks <= ctx->num_sms / 2)
       return launch_impl<BLOCK_N, D_HEAD, false, 0, 2, true>(ctx, ls, tmap_store, tmap_rows, p, fp, stream);
+  }
+  // the fused variant on fp16 rows, weights, queries and outputs (same tiles, MMA kind f16 with fp16 operands)
+  if constexpr (FG > 0) {
+    if (ctx->dtype == 1) return launch_impl<BLOCK_N, D_HEAD, false, FG, 2, true, 1>(ctx, ls, tmap_store, tmap_rows, p, fp, stream);
   }
   return launch_impl<BLOCK_N, D_HEAD, false, FG>(ctx, ls, tmap_store, tmap_rows, p, fp, stream);
 }

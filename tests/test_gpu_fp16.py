@@ -7,7 +7,8 @@ outputs:
   * K/V recomputed from checkpointed rows equal, bit for bit, the K/V of the first pass at every length
     16 ... 256 and for single rows (max |dK| = max |dV| = 0), as in bf16;
   * decode attention on fp16 q, K, V follows the oracle too, with bits independent of the segment layout;
-  * the bf16-only entry points (fused, FP8) refuse an fp16 context.
+  * the fused recompute + attention call on fp16 follows the oracle and the two-call fp16 path;
+  * the bf16-only entry points (FP8) refuse an fp16 context.
 """
 import numpy as np
 import pytest
@@ -158,13 +159,6 @@ def test_fp16_context_is_refused_by_the_bf16_only_entry_points_and_the_type_is_f
     with pytest.raises(kvd.KvdError) as e:        # a layer is set: too late to change the type
         ctx.kvd_set_dtype(0)
     assert e.value.status == 5
-    ws = torch.empty(kvd.kvd_workspace_bytes(ctx.desc), dtype=torch.uint8, device="cuda")
-    ctx.kvd_attach_workspace(ws)
-    kdim = shape.n_kv_heads * shape.d_head
-    q = torch.zeros((1, shape.n_q_heads, shape.d_head), dtype=torch.float16, device="cuda")
-    with pytest.raises(kvd.KvdError) as e:        # the fused path reads bf16 queries and writes bf16
-        ctx.kvd_decode_attention_recompute(0, 1, q, [3], [(0, 0, 0)], None, None, 0, None, None, kdim, [[]], 0.0, q)
-    assert e.value.status == 6
     x = torch.zeros((2, shape.d_hidden), dtype=torch.float16, device="cuda")
     p = torch.zeros((2,), dtype=torch.int32, device="cuda")
     arena = torch.zeros(kvd.kvd_store_bytes_fp8(ctx.desc, 1), dtype=torch.uint8, device="cuda")
@@ -224,4 +218,44 @@ def test_element_type_cannot_change_next_to_an_fp8_store():
             ctx.kvd_set_dtype(dt)
         assert e.value.status == 5
     ctx.kvd_set_dtype(0)
+    ctx.close()
+
+
+@pytest.mark.parametrize("shape,n_old,n_live", [(GEMMA3_4B_GLOBAL, 600, 40), (QWEN3_4B, 300, 0)], ids=lambda v: getattr(v, "name", v))
+def test_fp16_fused_recompute_attention_follows_the_oracle_and_the_two_call_path(shape, n_old, n_live):
+    import math
+    ctx, w16 = open_f16(shape, 1024)
+    ws = torch.empty(kvd.kvd_workspace_bytes(ctx.desc), dtype=torch.uint8, device="cuda")
+    ctx.kvd_attach_workspace(ws)
+    kdim = shape.n_kv_heads * shape.d_head
+    T = n_old + n_live + 1
+    X16 = as_f16(make_residuals(shape, T, seed=61, outliers=True))
+    pos = np.arange(T)
+    x, p = dev16(X16), torch.from_numpy(pos.astype(np.int32)).cuda()
+    ctx.kvd_checkpoint_residual(0, 0, x[:n_old], p[:n_old], n_old)
+    kl = torch.zeros((max(n_live, 1) + 1, kdim), dtype=torch.float16, device="cuda")
+    vl = torch.zeros_like(kl)
+    if n_live:
+        ctx.kvd_recompute_kv(0, x[n_old:n_old + n_live], p[n_old:n_old + n_live], n_live, kl, vl, kdim)
+    rng = np.random.Generator(np.random.PCG64(4))
+    q16 = rng.standard_normal((1, shape.n_q_heads, shape.d_head)).astype(np.float16)
+    q = dev16(q16)
+    live = [(kl, vl, kdim, n_old, n_live), (kl[n_live:], vl[n_live:], kdim, T - 1, 1)]
+    out_f = torch.zeros((1, shape.n_q_heads, shape.d_head), dtype=torch.float16, device="cuda")
+    ctx.kvd_decode_attention_recompute(0, 1, q, [T - 1], [(0, 0, n_old)], x[T - 1:], p[T - 1:], 1, kl[n_live:], vl[n_live:],
+                                       kdim, [live], 0.0, out_f)
+    # the two-call fp16 path on the same inputs
+    ko = torch.zeros((n_old, kdim), dtype=torch.float16, device="cuda")
+    vo = torch.zeros_like(ko)
+    ctx.kvd_recompute_kv(0, None, None, n_old, ko, vo, kdim, seq=0, first_row=0)
+    out_t = torch.zeros_like(out_f)
+    ctx.kvd_decode_attention(0, 1, q, [T - 1], [[(ko, vo, kdim, 0, n_old)] + live], 0.0, out_t)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    Kr, Vr = oracle_f16(shape, w16, X16, pos)
+    ref = oracle.decode_attention(q16[0].astype(np.float64), T - 1, [(Kr, Vr, 0)], 1.0 / math.sqrt(shape.d_head),
+                                  shape.sliding_window)
+    for name, got in (("fused", out_f), ("two-call", out_t)):
+        d = got[0].cpu().numpy().astype(np.float64) - ref
+        assert np.linalg.norm(d) / np.linalg.norm(ref) <= 1e-2, name
+        assert np.max(np.abs(d)) <= 1e-2 * np.max(np.abs(ref)), name
     ctx.close()
