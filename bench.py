@@ -282,6 +282,10 @@ class Workload:
         # the FP8 checkpoint variant's store (a second arena), filled once per set below
         self.arena8 = torch.empty(kvd.kvd_store_bytes_fp8(self.desc, 1), dtype=torch.uint8, device="cuda")
         self.ctx.kvd_attach_store_fp8(self.arena8, 1)
+        # the FP4 checkpoint variant's store (a third arena) and the scratch its recompute expands rows into
+        self.arena4 = torch.empty(kvd.kvd_store_bytes_fp4(self.desc, 1), dtype=torch.uint8, device="cuda")
+        self.ctx.kvd_attach_store_fp4(self.arena4, 1)
+        self.scratch4 = torch.empty(kvd.kvd_fp4_scratch_bytes(self.desc, T), dtype=torch.uint8, device="cuda")
         x_bits = make_residuals(shape, T + 1, seed=2, outliers=True)
         self.x_host_bits = x_bits
         x0 = dev(x_bits)
@@ -357,6 +361,16 @@ class Workload:
         # RECOMPUTE_KV from E4M3 checkpoints (rows and weights as FP8 codes, tensor-core kind f8f6f4)
         s = i % self.n_sets
         self.ctx.kvd_recompute_kv_fp8(0, [(s, 0, self.T, self.K[s], self.V[s])], self.kdim)
+
+    def k_checkpoint_fp4(self, i):
+        s = i % self.n_sets
+        self.ctx.kvd_reset_sequence_fp4(s)
+        self.ctx.kvd_checkpoint_residual_fp4(s, 0, self.X[s], self.pos, self.T)
+
+    def k_recompute_fp4(self, i):
+        # RECOMPUTE_KV from FP4 checkpoints: rows expanded to bf16 (exactly) into a scratch, then the bf16 projection
+        s = i % self.n_sets
+        self.ctx.kvd_recompute_kv_fp4(0, [(s, 0, self.T, self.K[s], self.V[s])], self.kdim, self.scratch4)
 
     def k_two_call(self, i):
         # recompute (T stored rows + the current token) followed by attention: the step's two K/V launches
@@ -568,6 +582,8 @@ def run_gpu(args):
               "recompute_from_caller_rows": timed_graph(wl.k_recompute_rows, 10),
               "current_token_kv_alone": timed_graph(wl.k_current, 10), "attention": timed_graph(wl.k_attention, 10),
               "checkpoint_fp8": timed_graph(wl.k_checkpoint_fp8, 10),
+              "checkpoint_fp4": timed_graph(wl.k_checkpoint_fp4, 10),
+              "recompute_from_fp4_checkpoints": timed_graph(wl.k_recompute_fp4, 10),
               "recompute_from_fp8_checkpoints": timed_graph(wl.k_recompute_fp8, 10),
               "recompute_then_attention_two_calls": timed_graph(wl.k_two_call, 10),
               "recompute_fused_into_attention": timed_graph(wl.k_fused, 10)}
@@ -731,6 +747,13 @@ def run_gpu(args):
                              "peak_source": peaks["source"] + " bf16 burst x 2 (nominal fp8 ratio)",
                              "avg_launch_us": iso_ms["recompute_from_fp8_checkpoints"] * 1e3,
                              "checkpoint_bytes_per_token": shape.d_hidden + 12, "traffic": None},
+            "fp4_checkpoints": {"checkpoint_bytes_per_token": shape.d_hidden // 2 + shape.d_hidden // 16 + 12,
+                                "bf16_checkpoint_bytes_per_token": 2 * shape.d_hidden + 8,
+                                "kv_bytes_per_token_replaced": 4 * shape.n_kv_heads * shape.d_head,
+                                "checkpoint_us": iso_ms["checkpoint_fp4"] * 1e3,
+                                "recompute_us": iso_ms["recompute_from_fp4_checkpoints"] * 1e3,
+                                "note": "E2M1 codes, E4M3 block scales per 16 channels, power-of-two row scale; rows are "
+                                        "expanded to bf16 exactly and projected by the bf16 kernel (two launches)"},
             "roofline_attention": {"kernel": "kvd_attn_split_kernel<256,2> + merge", "bound": "hbm",
                                    "achieved": attn_bytes / (attn_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                                    "unit": "GB/s", "frac": attn_bytes / (attn_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],

@@ -315,6 +315,36 @@ kvd_status kvd_quantize_rows_fp8(kvd_ctx *ctx, const void *rows, int n, void *co
 kvd_status kvd_recompute_kv_fp8_rows(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
                                      const kvd_fp8_rows *rows, int64_t out_row_stride, void *stream);
 
+/* ---- FP4 checkpoints (the same future-work item; again the format is this library's definition) ----
+ * A residual row x (bf16) is stored in 4 bits per channel with two levels of scales (the layout known as NVFP4,
+ * the outer scale taken per row and restricted to a power of two):
+ *     s_row = 2^(floor(log2 max|x|) - 10)                      (1 for an all-zero row; max|x| / s_row in [1024, 2048))
+ *     b     = e4m3((max|x_block| / 6) / s_row)                 per block of 16 consecutive channels, fp32, nearest even
+ *     c_k   = e2m1(x_k / (b * s_row))                          nearest of {0, .5, 1, 1.5, 2, 3, 4, 6}, ties to the even
+ *                                                              code, saturating; all codes 0 when b rounds to 0
+ * together with its position and the sum of squares of the ORIGINAL row.  A value decodes as c_k * b * s_row, which
+ * is exact in bf16.  RECOMPUTE_KV from such rows is Eq. 13-14 on the decoded rows with 1/rms of the original row:
+ * kvd_recompute_kv_fp4 expands the rows of its ranges into a caller-provided scratch (bf16 rows, positions,
+ * statistics; kvd_fp4_scratch_bytes for the total row count of a call) and runs the ordinary bf16 projection on
+ * them -- storage is 4-bit, the arithmetic is the bf16 path's; two launches.  Per token and layer the store holds
+ * d_hidden/2 + d_hidden/16 + 12 bytes (1,452 for d_hidden = 2560; bf16 rows 5,128; the K/V they replace 4,096).
+ * Accuracy is that of the format, reported by the tests, not claimed; exactness (Prop. 3.2) does not carry over,
+ * determinism does.  The FP4 store is a third, independent arena: codes uint8 [layers][max_seqs][max_tokens]
+ * [d_hidden/2] (channel 2j in the low nibble of byte j), block scales uint8 [...][d_hidden/16], positions int32,
+ * sums of squares fp32, row scales fp32, each region starting at a 256-byte multiple.  d_hidden % 64 == 0 and
+ * d_hidden <= 2560; bf16 contexts only. */
+size_t kvd_store_bytes_fp4(const kvd_model_desc *desc, int layers_stored);
+kvd_status kvd_attach_store_fp4(kvd_ctx *ctx, void *arena, size_t bytes, int layers_stored);
+int kvd_rows_stored_fp4(const kvd_ctx *ctx, int layer, int seq);
+kvd_status kvd_reset_sequence_fp4(kvd_ctx *ctx, int seq);
+kvd_status kvd_checkpoint_residual_fp4(kvd_ctx *ctx, int seq, int layer, const void *rows, const int32_t *positions,
+                                       int n, void *stream);
+size_t kvd_fp4_scratch_bytes(const kvd_model_desc *desc, int max_rows);
+/* ranges: rows first_row .. first_row+n-1 of the FP4 store of (layer, ranges[i].seq), K and V (bf16) to k_out / v_out
+ * with row stride out_row_stride.  scratch: DEVICE, 256-byte aligned, >= kvd_fp4_scratch_bytes(desc, sum of n). */
+kvd_status kvd_recompute_kv_fp4(kvd_ctx *ctx, int layer, const kvd_store_range *ranges, int n_ranges,
+                                int64_t out_row_stride, void *scratch, size_t scratch_bytes, void *stream);
+
 /* ATTENTION(Q, K_all, V_all) of Algorithm 1 for one new token per sequence (Eq. 6-7).
  *   q      DEVICE bf16 [batch, n_q_heads, d_head], already normalised and rotated to q_pos.
  *   q_pos  HOST int32 [batch]: position of each sequence's query token.

@@ -38,6 +38,8 @@ EXPORTED_SYMBOLS = (
     "kvd_decode_attention_recompute", "kvd_fused_recompute_pays", "kvd_decode_attention_recompute_fp8", "kvd_set_dtype", "kvd_store_bytes_dtype",
     "kvd_quantize_rows_fp8", "kvd_recompute_kv_fp8_rows", "kvd_decode_attention_recompute_fp8_rows",
     "kvd_store_bytes_fp8", "kvd_attach_store_fp8", "kvd_rows_stored_fp8", "kvd_reset_sequence_fp8", "kvd_checkpoint_residual_fp8", "kvd_recompute_kv_fp8",
+    "kvd_store_bytes_fp4", "kvd_attach_store_fp4", "kvd_rows_stored_fp4", "kvd_reset_sequence_fp4",
+    "kvd_checkpoint_residual_fp4", "kvd_fp4_scratch_bytes", "kvd_recompute_kv_fp4",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_checkpoint_residual_step", "kvd_decode_step_kv", "kvd_recompute_kv",
     "kvd_recompute_kv_step",
     "kvd_decode_attention", "kvd_decode_attention_rows", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_build_has_checks", "kvd_selftest_bounds_check", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
@@ -147,6 +149,20 @@ def load() -> ctypes.CDLL:
     lib.kvd_decode_attention.restype = i32
     lib.kvd_fused_recompute_pays.argtypes = [ctypes.POINTER(kvd_model_desc), i64, i32]
     lib.kvd_fused_recompute_pays.restype = i32
+    lib.kvd_store_bytes_fp4.argtypes = [ctypes.POINTER(kvd_model_desc), i32]
+    lib.kvd_store_bytes_fp4.restype = sz
+    lib.kvd_fp4_scratch_bytes.argtypes = [ctypes.POINTER(kvd_model_desc), i32]
+    lib.kvd_fp4_scratch_bytes.restype = sz
+    lib.kvd_attach_store_fp4.argtypes = [vp, vp, sz, i32]
+    lib.kvd_attach_store_fp4.restype = i32
+    lib.kvd_rows_stored_fp4.argtypes = [vp, i32, i32]
+    lib.kvd_rows_stored_fp4.restype = i32
+    lib.kvd_reset_sequence_fp4.argtypes = [vp, i32]
+    lib.kvd_reset_sequence_fp4.restype = i32
+    lib.kvd_checkpoint_residual_fp4.argtypes = [vp, i32, i32, vp, vp, i32, vp]
+    lib.kvd_checkpoint_residual_fp4.restype = i32
+    lib.kvd_recompute_kv_fp4.argtypes = [vp, i32, ctypes.POINTER(kvd_store_range), i32, i64, vp, sz, vp]
+    lib.kvd_recompute_kv_fp4.restype = i32
     lib.kvd_decode_attention_rows.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
                                               ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
     lib.kvd_decode_attention_rows.restype = i32
@@ -257,6 +273,14 @@ def kvd_store_bytes_dtype(desc: kvd_model_desc, layers_stored: int, dtype: int) 
 
 def kvd_store_bytes_fp8(desc: kvd_model_desc, layers_stored: int) -> int:
     return int(load().kvd_store_bytes_fp8(ctypes.byref(desc), layers_stored))
+
+
+def kvd_store_bytes_fp4(desc: kvd_model_desc, layers_stored: int) -> int:
+    return int(load().kvd_store_bytes_fp4(ctypes.byref(desc), layers_stored))
+
+
+def kvd_fp4_scratch_bytes(desc: kvd_model_desc, max_rows: int) -> int:
+    return int(load().kvd_fp4_scratch_bytes(ctypes.byref(desc), max_rows))
 
 
 def kvd_workspace_bytes(desc: kvd_model_desc) -> int:
@@ -544,6 +568,32 @@ class Kvd:
             arr[i].k_out, arr[i].v_out = _ptr(k_out), _ptr(v_out)
         self._check(self._lib.kvd_recompute_kv_fp8(self._h, layer, arr, len(ranges), out_row_stride, _stream(stream)),
                     "kvd_recompute_kv_fp8")
+
+    def kvd_attach_store_fp4(self, arena, layers_stored: int) -> None:
+        self._keep.append(arena)
+        self._check(self._lib.kvd_attach_store_fp4(self._h, _ptr(arena), arena.numel() * arena.element_size(),
+                                                   layers_stored), "kvd_attach_store_fp4")
+
+    def kvd_reset_sequence_fp4(self, seq: int) -> None:
+        self._check(self._lib.kvd_reset_sequence_fp4(self._h, seq), "kvd_reset_sequence_fp4")
+
+    def kvd_rows_stored_fp4(self, layer: int, seq: int) -> int:
+        return int(self._lib.kvd_rows_stored_fp4(self._h, layer, seq))
+
+    def kvd_checkpoint_residual_fp4(self, seq: int, layer: int, rows, positions, n: int, stream=None) -> None:
+        self._check(self._lib.kvd_checkpoint_residual_fp4(self._h, seq, layer, _ptr(rows), _ptr(positions), n,
+                                                          _stream(stream)), "kvd_checkpoint_residual_fp4")
+
+    def kvd_recompute_kv_fp4(self, layer: int, ranges: Sequence[Tuple[int, int, int, object, object]],
+                             out_row_stride: int, scratch, stream=None) -> None:
+        """ranges: (seq, first_row, n, k_out, v_out) over the FP4 store; scratch: a uint8 device tensor."""
+        arr = (kvd_store_range * max(len(ranges), 1))()
+        for i, (seq, first_row, n, k_out, v_out) in enumerate(ranges):
+            arr[i].seq, arr[i].first_row, arr[i].n, arr[i].reserved = int(seq), int(first_row), int(n), 0
+            arr[i].k_out, arr[i].v_out = _ptr(k_out), _ptr(v_out)
+        self._check(self._lib.kvd_recompute_kv_fp4(self._h, layer, arr, len(ranges), out_row_stride, _ptr(scratch),
+                                                   scratch.numel() * scratch.element_size(), _stream(stream)),
+                    "kvd_recompute_kv_fp4")
 
     def kvd_memory_stats(self) -> dict:
         ms = kvd_mem_stats()

@@ -271,7 +271,7 @@ extern "C" kvd_status kvd_set_dtype(kvd_ctx *ctx, int dtype) {
   for (int c : ctx->rows_stored)
     if (c != 0) return KVD_ERR_STATE;
   // the FP8 variant reads bf16 rows and bf16-folded weights: no other element type next to an FP8 store
-  if (dtype != KVD_DTYPE_BF16 && ctx->store8_codes) return KVD_ERR_STATE;
+  if (dtype != KVD_DTYPE_BF16 && (ctx->store8_codes || ctx->store4_codes)) return KVD_ERR_STATE;
   for (int c : ctx->rows_stored8)
     if (c != 0) return KVD_ERR_STATE;
   ctx->dtype = dtype;
@@ -1168,6 +1168,16 @@ extern "C" kvd_status kvd_memory_stats(const kvd_ctx *ctx, kvd_mem_stats *out) {
   }
   out->checkpoint_bytes_used += rows8 * (static_cast<uint64_t>(d.d_hidden) + 12);
   out->checkpoint_bytes_capacity += ctx->layers_stored8 > 0 ? kvd_store_bytes_fp8(&d, ctx->layers_stored8) : 0;
+  // ... and the FP4 store: codes, block scales, position, sum of squares, row scale
+  uint64_t rows4 = 0;
+  for (int l = 0; l < ctx->layers_stored4; ++l) {
+    uint64_t layer_rows = 0;
+    for (int s = 0; s < d.max_seqs; ++s) layer_rows += ctx->rows_stored4[static_cast<size_t>(l) * d.max_seqs + s];
+    rows4 += layer_rows;
+    if (layer_rows > tokens) tokens = layer_rows;
+  }
+  out->checkpoint_bytes_used += rows4 * (static_cast<uint64_t>(d.d_hidden) / 2 + d.d_hidden / 16 + 12);
+  out->checkpoint_bytes_capacity += ctx->layers_stored4 > 0 ? kvd_store_bytes_fp4(&d, ctx->layers_stored4) : 0;
   out->workspace_bytes = ctx->workspace_bytes;
   out->prepared_weight_bytes = ctx->prepared_bytes;
   out->tokens_stored = tokens;

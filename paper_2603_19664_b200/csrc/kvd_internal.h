@@ -251,6 +251,14 @@ struct kvd_ctx {
   int layers_stored8 = 0;
   std::vector<int> rows_stored8;
   std::vector<CUtensorMap> store8_maps;
+  // FP4 residual store (a third arena): E2M1 codes, E4M3 block scales, positions, sums of squares, row scales
+  uint8_t *store4_codes = nullptr;
+  uint8_t *store4_block = nullptr;
+  int32_t *store4_pos = nullptr;
+  float *store4_sumsq = nullptr;
+  float *store4_scale = nullptr;
+  int layers_stored4 = 0;
+  std::vector<int> rows_stored4;
   unsigned *amax_scratch = nullptr;  // one word, used while weights are prepared
   // attention scratch
   float *part_o = nullptr;
