@@ -370,6 +370,18 @@ kvd_status kvd_decode_attention(kvd_ctx *ctx, int layer, int batch, const void *
 kvd_status kvd_decode_attention_rows(kvd_ctx *ctx, int layer, int n_rows, const void *q, const int32_t *q_pos,
                                      const kvd_kv_segment *segs, int n_segs, float scale, void *out, void *stream);
 
+/* ATTENTION of Algorithm 1 (Eq. 6-7) for many tokens of one sequence in ONE launch, tiled over query rows on the
+ * tensor cores: the prefill-shaped call.  Arguments as kvd_decode_attention_rows, except that q_pos is a DEVICE
+ * int32 [n_rows] (nothing on the host depends on the positions).  Keys are taken in blocks of 64 aligned to absolute
+ * position; the softmax weights are rounded to the element type before the second product (fp32 accumulation).
+ * A row's result depends on that row, its position and the keys alone -- not on n_rows, on the row's index or on the
+ * other rows of the call -- so a token attended alone and the same token inside a long call give the same bits.
+ * They are NOT the bits of kvd_decode_attention / kvd_decode_attention_rows (another split of the keys): same
+ * tolerance against the definition; use one of the two families throughout where outputs must be bit-identical.
+ * bf16 and fp16 contexts; needs no workspace. */
+kvd_status kvd_prefill_attention(kvd_ctx *ctx, int layer, int n_rows, const void *q, const int32_t *q_pos,
+                                 const kvd_kv_segment *segs, int n_segs, float scale, void *out, void *stream);
+
 /* RECOMPUTE_KV and ATTENTION of Algorithm 1 in one pass for the evicted tokens (Eq. 13-14 feeding
  * Eq. 6-7): the keys and values rebuilt from the residual rows of ranges[b] are consumed inside the
  * recompute kernel -- the rotated key of a row is multiplied with the queries of its KV head, the value

@@ -42,7 +42,7 @@ EXPORTED_SYMBOLS = (
     "kvd_checkpoint_residual_fp4", "kvd_fp4_scratch_bytes", "kvd_recompute_kv_fp4",
     "kvd_rows_stored", "kvd_workspace_bytes", "kvd_attention_split", "kvd_attach_workspace", "kvd_checkpoint_residual", "kvd_checkpoint_residual_step", "kvd_decode_step_kv", "kvd_recompute_kv",
     "kvd_recompute_kv_step",
-    "kvd_decode_attention", "kvd_decode_attention_rows", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_build_has_checks", "kvd_selftest_bounds_check", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
+    "kvd_decode_attention", "kvd_decode_attention_rows", "kvd_prefill_attention", "kvd_decode_attention_static", "kvd_memory_stats", "kvd_poll_status", "kvd_selftest_wait_timeout", "kvd_build_has_checks", "kvd_selftest_bounds_check", "kvd_set_trace", "kvd_launch_count", "kvd_last_cuda_error",
     "kvd_status_string", "kvd_version",
     # include/kvd_scaffold.h: the parts of a decoder layer around the hot path, for whole-stack tests and benchmarks
     "kvd_scaffold_linear_create", "kvd_scaffold_linear_destroy", "kvd_scaffold_linear_out_cols", "kvd_scaffold_linear",
@@ -166,6 +166,8 @@ def load() -> ctypes.CDLL:
     lib.kvd_decode_attention_rows.argtypes = [vp, i32, i32, vp, ctypes.POINTER(ctypes.c_int32),
                                               ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
     lib.kvd_decode_attention_rows.restype = i32
+    lib.kvd_prefill_attention.argtypes = [vp, i32, i32, vp, vp, ctypes.POINTER(kvd_kv_segment), i32, ctypes.c_float, vp, vp]
+    lib.kvd_prefill_attention.restype = i32
     lib.kvd_set_dtype.argtypes = [vp, i32]
     lib.kvd_set_dtype.restype = i32
     lib.kvd_store_bytes_fp8.argtypes = [ctypes.POINTER(kvd_model_desc), i32]
@@ -458,6 +460,13 @@ class Kvd:
         self._check(self._lib.kvd_decode_attention_rows(self._h, layer, n_rows, _ptr(q), pos_arr, seg_arr, n_segs,
                                                         float(scale), _ptr(out), _stream(stream)),
                     "kvd_decode_attention_rows")
+
+    def kvd_prefill_attention(self, layer: int, n_rows: int, q, q_pos_dev, segs: Sequence[Segment], scale: float, out,
+                              stream=None) -> None:
+        """Many query rows of one sequence in one launch; q_pos_dev: int32 device tensor [n_rows]."""
+        n_segs, _, seg_arr = _marshal_segments(1, [0], [list(segs)])
+        self._check(self._lib.kvd_prefill_attention(self._h, layer, n_rows, _ptr(q), _ptr(q_pos_dev), seg_arr, n_segs,
+                                                    float(scale), _ptr(out), _stream(stream)), "kvd_prefill_attention")
 
     def kvd_decode_attention_recompute(self, layer: int, batch: int, q, q_pos: Sequence[int],
                                        ranges: Sequence[Tuple[int, int, int]], rows, positions, n_rows: int,

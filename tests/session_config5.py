@@ -30,16 +30,16 @@ from stack_harness import GpuStack, GpuStackChained, torch_stack_weights  # noqa
 
 
 def run_session(stack, weights, turns, gen, window, seg_lo, seg_hi, max_tokens, device_weights=True, log=None,
-                chained=False):
+                chained=False, tiled=False):
     """Returns (per-turn records, all-match flag)."""
     rng = np.random.Generator(np.random.PCG64(SEED_TOKENS + 77))
     segments = [rng.integers(0, stack.vocab, size=int(rng.integers(seg_lo, seg_hi + 1))).tolist() for _ in range(turns)]
     if chained:
-        full = GpuStack(stack, weights, "full", 0, max_tokens, device_weights)
-        kvdir = GpuStackChained(stack, weights, window, max_tokens, device_weights)
+        full = GpuStack(stack, weights, "full", 0, max_tokens, device_weights, tiled_attention=tiled)
+        kvdir = GpuStackChained(stack, weights, window, max_tokens, device_weights, tiled_attention=tiled)
     else:
-        full = GpuStack(stack, weights, "full", 0, max_tokens, device_weights)
-        kvdir = GpuStack(stack, weights, "kvdirect", window, max_tokens, device_weights)
+        full = GpuStack(stack, weights, "full", 0, max_tokens, device_weights, tiled_attention=tiled)
+        kvdir = GpuStack(stack, weights, "kvdirect", window, max_tokens, device_weights, tiled_attention=tiled)
     records, all_match = [], True
     for t in range(turns):
         outs = []
@@ -78,13 +78,14 @@ def main():
     ap.add_argument("--small", action="store_true", help="small 6-layer stack instead of the 34-layer one")
     ap.add_argument("--chained", action="store_true", help="one checkpointed row per token, chained recompute")
     ap.add_argument("--seg", type=int, nargs=2, default=None, help="user segment length range")
+    ap.add_argument("--tiled", action="store_true", help="all attention through kvd_prefill_attention (row-tiled kernel)")
     a = ap.parse_args()
     stack = S_GEMMA if a.small else GEMMA3_4B_STACK
     seg = tuple(a.seg) if a.seg else ((24, 64) if a.small else (256, 1024))
     max_tokens = a.turns * (seg[1] + a.gen) + 8
     w = torch_stack_weights(stack)
     recs, ok = run_session(stack, w, a.turns, a.gen, a.window, seg[0], seg[1], max_tokens,
-                           log=lambda s: print(s, flush=True), chained=a.chained)
+                           log=lambda s: print(s, flush=True), chained=a.chained, tiled=a.tiled)
     print(json.dumps({"summary": True, "stack": stack.name, "turns": a.turns, "all_tokens_match": ok,
                       "peak_full_cache_kv_bytes": max(r["full_cache_kv_bytes"] for r in recs),
                       "peak_kvdirect_live_kv_bytes": max(r["kvdirect_live_kv_bytes"] for r in recs),

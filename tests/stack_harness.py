@@ -60,8 +60,12 @@ def torch_stack_weights(stack, seed=0):
 
 class GpuStack:
     def __init__(self, stack, weights, policy="full", budget=0, max_tokens=512, device_weights=False,
-                 layers_stored=None):
+                 layers_stored=None, tiled_attention=False):
+        """tiled_attention: every attention call (prefill, decode step, replay) goes through kvd_prefill_attention,
+        the tensor-core kernel tiled over query rows, instead of the decode kernels.  Its rows do not depend on the
+        batch either, so the bit-identity experiments hold as long as BOTH arms use it."""
         assert policy in ("full", "kvdirect")
+        self.tiled = bool(tiled_attention)
         self.s, self.policy, self.budget, self.max_tokens = stack, policy, int(budget), max_tokens
         s = stack
         self.kdim = s.n_kv_heads * s.d_head
@@ -139,6 +143,14 @@ class GpuStack:
         ctx.kvd_scaffold_add_rows(h, y, y.shape[1], U, s.d_hidden)
         return h
 
+    def _attend(self, l, n, q, positions, positions_dev, segs, out):
+        """ATTENTION for n query tokens of the sequence over `segs`: the decode kernels (host loop over launches of at
+        most 64 rows) or, with tiled_attention, one launch of the row-tiled tensor-core kernel."""
+        if self.tiled:
+            self.ctx.kvd_prefill_attention(l, n, q, positions_dev, segs, 0.0, out)
+        else:
+            self.ctx.kvd_decode_attention_rows(l, n, q, positions, segs, 0.0, out)
+
     def _logits(self, h_last):
         """Final norm and vocabulary projection of one row; keeps the bf16 logits for greedy_token()."""
         self.logits_bf16 = self._linear(self.lin_head, h_last)
@@ -179,7 +191,7 @@ class GpuStack:
             first_live = max(wf, lo) if self.policy == "kvdirect" else 0
             segs.append((kl[first_live:], vl[first_live:], self.kdim, first_live, pos + 1 - first_live))
             out = torch.empty((1, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
-            ctx.kvd_decode_attention(l, 1, q, [pos], [segs], 0.0, out)
+            self._attend(l, 1, q, [pos], pos_t, segs, out)
             # scaffold: W_o, MLP
             h = self._after_attention(l, h, out)
             if self.policy == "kvdirect":
@@ -214,7 +226,7 @@ class GpuStack:
             first_live = max(wf, lo_min) if self.policy == "kvdirect" else 0
             segs.append((kl[first_live:], vl[first_live:], self.kdim, first_live, p0 + U - first_live))
             out = torch.empty((U, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
-            ctx.kvd_decode_attention_rows(l, U, q, positions, segs, 0.0, out)
+            self._attend(l, U, q, positions, pos_t, segs, out)
             h = self._after_attention(l, h, out)
             if self.policy == "kvdirect":
                 self.win_first[l] = max(self.win_first[l], p0 + U - self.budget)
@@ -253,9 +265,9 @@ class GpuStackChained(GpuStack):
     their current rows (the same kvd_recompute_kv as ever), serve the new tokens' attention and the
     evicted tokens' own causal attention, and are dropped when the rows move on to layer l + 1."""
 
-    def __init__(self, stack, weights, budget=0, max_tokens=512, device_weights=False):
+    def __init__(self, stack, weights, budget=0, max_tokens=512, device_weights=False, tiled_attention=False):
         super().__init__(stack, weights, policy="kvdirect", budget=budget, max_tokens=max_tokens,
-                         device_weights=device_weights, layers_stored=1)
+                         device_weights=device_weights, layers_stored=1, tiled_attention=tiled_attention)
         # the layer-0 rows as the library stores them (documented arena layout)
         self.rows0 = self.arena[:max_tokens * stack.d_hidden * 2].view(torch.bfloat16).view(max_tokens, stack.d_hidden)
         self.replayed_rows = 0
@@ -288,14 +300,14 @@ class GpuStackChained(GpuStack):
             segs_new.append((kl[N:], vl[N:], self.kdim, N, p0 + U - N))
             q_new = self._queries(l, h_new, pos_new_t)
             out_new = torch.empty((U, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
-            ctx.kvd_decode_attention_rows(l, U, q_new, pos_new, segs_new, 0.0, out_new)
+            self._attend(l, U, q_new, pos_new, pos_new_t, segs_new, out_new)
             if N > 0 and l + 1 < s.n_layers:
                 # the evicted tokens' own step through this layer: each attends to the evicted keys up
                 # to its own position (the position mask does the rest)
                 q_old = self._queries(l, h_old, pos_old_t)
                 out_old = torch.empty((N, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
                 segs_old = [(self.k_old, self.v_old, self.kdim, 0, N)]
-                ctx.kvd_decode_attention_rows(l, N, q_old, pos_old, segs_old, 0.0, out_old)
+                self._attend(l, N, q_old, pos_old, pos_old_t, segs_old, out_old)
                 h_old = self._after_attention(l, h_old, out_old)
                 self.replayed_rows += N
             h_new = self._after_attention(l, h_new, out_new)

@@ -281,3 +281,29 @@ def test_rows_of_one_sequence_with_their_own_causal_limit(shape):
     ref = oracle_attention(shape, q_bits[sample], [q_pos[i] for i in sample], [segs_bits] * len(sample))
     attn_check(host_f64(out[torch.tensor(sample).cuda()]), ref)
     ctx.close()
+
+
+def test_a_sequences_bits_do_not_depend_on_the_rest_of_the_batch_or_the_kernel_variant():
+    """One sequence of 4097 keys attended alone (260 CTAs: the streaming variant that issues the loads of both
+    iterations at once) and as one of a batch of six (1,500 CTAs: the four-CTAs-per-SM variant): the same bits.  The
+    split of a sequence is a function of its own visible range, and the two variants compute in the same order."""
+    shape = GEMMA3_4B_GLOBAL
+    lens = [4097, 1000, 4097, 2500, 65, 3333]
+    ctx, _ = open_layer(shape, max_tokens=4200, max_batch=len(lens))
+    kdim = shape.n_kv_heads * shape.d_head
+    q_bits = make_query(shape, len(lens), seed=12)
+    q = dev(q_bits)
+    kv = [make_kv(shape, n, seed=30 + i) for i, n in enumerate(lens)]
+    kd = [(dev(k), dev(v)) for k, v in kv]
+    segs = [[(kd[i][0], kd[i][1], kdim, 0, n)] for i, n in enumerate(lens)]
+    q_pos = [n - 1 for n in lens]
+    out_b = torch.zeros((len(lens), shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda")
+    ctx.kvd_decode_attention(0, len(lens), q, q_pos, segs, 0.0, out_b)
+    one = torch.zeros((1, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda")
+    for i in range(len(lens)):
+        ctx.kvd_decode_attention(0, 1, q[i:i + 1], [q_pos[i]], [segs[i]], 0.0, one)
+        assert torch.equal(one[0], out_b[i]), i
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    ref = oracle_attention(shape, q_bits[:2], q_pos[:2], [[(kv[i][0], kv[i][1], 0)] for i in range(2)])
+    attn_check(host_f64(out_b[:2]), ref)
+    ctx.close()

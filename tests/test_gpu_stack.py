@@ -195,3 +195,40 @@ def _step_from_layer(m, token, first_layer, h_in):
         h = m._after_attention(l, h, out)
     assert ctx.kvd_poll_status() == 0
     return entering, m._logits(h)
+
+
+@pytest.mark.parametrize("stack,ctx_len", [(S_GEMMA, 72), (S_QWEN, 48)], ids=lambda x: getattr(x, "name", x))
+def test_policies_stay_bit_identical_on_the_row_tiled_attention_kernel(stack, ctx_len):
+    """The same three policies with every attention call on kvd_prefill_attention (one launch per layer and call,
+    however many tokens): its rows do not depend on the batch either, so the bounded window with recomputation and
+    the single-checkpoint chained variant still reproduce the full-cache logits bit for bit."""
+    w = make_stack_weights(stack)
+    prompt = make_token_ids(ctx_len, stack.vocab, seed=4).tolist()
+    cut = ctx_len // 3
+
+    def run(m):
+        m.prefill(prompt[:cut])
+        logits = m.prefill(prompt[cut:])
+        toks, lgs = [], []
+        for i in range(12):
+            nxt = m.greedy_token()
+            toks.append(nxt)
+            lgs.append(logits.clone())
+            if i + 1 < 12:
+                logits = m.step(nxt)
+        assert m.ctx.kvd_poll_status() == 0
+        return toks, lgs
+
+    ref_tokens, ref_logits = run(GpuStack(stack, w, "full", tiled_attention=True))
+    assert len(set(ref_tokens)) > 2
+    for m in (GpuStack(stack, w, "kvdirect", 8, tiled_attention=True), GpuStackChained(stack, w, budget=8, tiled_attention=True),
+              GpuStackChained(stack, w, budget=0, tiled_attention=True)):
+        toks, logits = run(m)
+        assert toks == ref_tokens
+        for a, b in zip(logits, ref_logits):
+            assert torch.equal(a, b)
+    # and the tiled kernel agrees with the decode kernels to attention tolerance (other split of the keys)
+    plain_tokens, plain_logits = run(GpuStack(stack, w, "full"))
+    err = max(float((a - b).abs().max()) for a, b in zip(plain_logits, ref_logits))
+    scale = max(float(b.abs().max()) for b in ref_logits)
+    assert err <= 0.02 * scale, (err, scale)
