@@ -865,6 +865,27 @@ def measure_stack_decode(batches, n_check_steps=4, session_turns=20, session_gen
                     "scaffold = the block's other products and small steps on the library's own kernels"}
 
 
+def run_profile_stack(args):
+    """Eager launches of two whole-stack decode steps per cache policy (34 layers, batch 4, context 2048, window 256)
+    for a run under a profiler: every kernel of the measured config-3 step, hot path and scaffold."""
+    import torch
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from kvd_synth import GEMMA3_4B_STACK
+    from stack_harness import BatchStack, torch_stack_weights
+    from paper_2603_19664_b200.build import build
+    build()
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    w = torch_stack_weights(GEMMA3_4B_STACK, seed=3)
+    m = BatchStack(GEMMA3_4B_STACK, w, 4, 2048, 256, max_steps=8)
+    tok = torch.tensor([5, 6, 7, 8], dtype=torch.int32, device="cuda")
+    for policy in ("full", "kvdirect"):
+        for i in range(2):
+            m.step(tok, 2048 + i, policy)
+    torch.cuda.synchronize()
+    assert m.ctx.kvd_poll_status() == 0
+    print(json.dumps({"profile_run": "stack", "launches": m.ctx.kvd_launch_count()}))
+
+
 def measure_long_attention(wl, peaks, timed_graph, T=32768):
     """Decode attention over T + 1 keys of the same layer shape (134 MB per call): the size at which
     the HBM roofline, not launch latency, is the bound."""
@@ -1287,6 +1308,8 @@ def main():
                     help="with --profile: also run decode attention over 32769 keys a few times")
     ap.add_argument("--profile-qwen", action="store_true",
                     help="eager launches of the Qwen3-4B-shaped layer's kernels (reduced long-context case) for a profiler")
+    ap.add_argument("--profile-stack", action="store_true",
+                    help="eager launches of whole-stack decode steps (batch 4) for a run under a profiler")
     ap.add_argument("--no-stack", action="store_true", help="skip the whole-stack decode step (configs 3 and 5)")
     ap.add_argument("--short-session", action="store_true", help="config 5 with 3 turns of 16 tokens instead of 20 of 128")
     ap.add_argument("--stack-all", action="store_true", help="whole-stack decode step at batch 1, 4, 16 and 64")
@@ -1297,6 +1320,8 @@ def main():
         run_reference(args)
     elif args.profile_qwen:
         run_profile_qwen(args)
+    elif args.profile_stack:
+        run_profile_stack(args)
     elif args.stack_configs:
         run_stack_configs(args)
     else:

@@ -81,7 +81,9 @@ kvd_status kvd_scaffold_embed(kvd_ctx *ctx, const void *table, const int32_t *to
                               void *out, void *stream);
 
 /* tokens_out[r] = argmax_c logits[r * row_stride + c] over c < n, the lowest index among equal maxima
- * (NaNs never win).  logits DEVICE bf16; tokens_out DEVICE int32 [m]. */
+ * (NaNs never win; a row of NaNs yields 0).  logits DEVICE bf16; tokens_out DEVICE int32 [m].  Two small launches
+ * and a memset of a per-row slot owned by the context (allocated on first use: make the first call outside stream
+ * capture). */
 kvd_status kvd_scaffold_argmax(kvd_ctx *ctx, const void *logits, int64_t row_stride, int m, int n,
                                int32_t *tokens_out, void *stream);
 

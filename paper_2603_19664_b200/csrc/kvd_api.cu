@@ -170,6 +170,7 @@ extern "C" void kvd_destroy(kvd_ctx *ctx) {
   if (ctx->d_status) cudaFree(ctx->d_status);
   if (ctx->ext_sumsq) cudaFree(ctx->ext_sumsq);
   if (ctx->zero_pos) cudaFree(ctx->zero_pos);
+  if (ctx->argmax_keys) cudaFree(ctx->argmax_keys);
   if (ctx->amax_scratch) cudaFree(ctx->amax_scratch);
   cudaGetLastError();
   delete ctx;

@@ -239,6 +239,8 @@ struct kvd_ctx {
   float *store_sumsq = nullptr;
   float *ext_sumsq = nullptr;     // statistics of caller rows taken ahead of the recompute kernel
   size_t ext_sumsq_rows = 0;
+  unsigned long long *argmax_keys = nullptr;  // scaffold greedy pick: one slot per row
+  size_t argmax_rows = 0;
   int32_t *zero_pos = nullptr;    // ext_sumsq_rows zeros: the positions of rows that are not rotated (scaffold products)
   int layers_stored = 0;
   std::vector<int> rows_stored;  // [layers_stored * max_seqs]

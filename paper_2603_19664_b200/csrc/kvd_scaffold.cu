@@ -127,37 +127,44 @@ __global__ void __launch_bounds__(256) kvd_embed_kernel(const uint4 *__restrict_
   }
 }
 
-// One CTA per row.  Every thread scans a strided share of the row keeping its first maximum, then the
-// CTA reduces (value descending, index ascending): the lowest index among equal maxima wins.
-__global__ void __launch_bounds__(256) kvd_argmax_kernel(const __nv_bfloat16 *__restrict__ logits, long long stride, int n,
-                                                         int32_t *__restrict__ out) {
-  __shared__ float s_v[256];
-  __shared__ int s_i[256];
-  const __nv_bfloat16 *row = logits + static_cast<size_t>(blockIdx.x) * stride;
-  float best = -CUDART_INF_F;
-  int bi = 0x7fffffff;
-  for (int c = threadIdx.x; c < n; c += blockDim.x) {
+// Greedy pick in two small kernels.  (1) grid (column slices, rows): every CTA reduces its slice of a row to a
+// 64-bit key -- the logit's bits mapped so that unsigned order is numeric order, above the complement of the column
+// index -- and folds it into the row's slot with atomicMax: the largest value wins, among equal values the lowest
+// index; the result does not depend on the order in which the CTAs arrive.  (2) one thread per row decodes the index.
+constexpr int ARGMAX_SLICE = 4096;
+__device__ __forceinline__ unsigned long long argmax_key(float v, int c) {
+  uint32_t u = __float_as_uint(v);
+  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // monotone map of finite floats to unsigned
+  return (static_cast<unsigned long long>(u) << 32) | static_cast<uint32_t>(0x7fffffff - c);
+}
+__global__ void __launch_bounds__(256) kvd_argmax_slices_kernel(const __nv_bfloat16 *__restrict__ logits, long long stride, int n,
+                                                                unsigned long long *__restrict__ keys) {
+  __shared__ unsigned long long s_k[8];
+  const __nv_bfloat16 *row = logits + static_cast<size_t>(blockIdx.y) * stride;
+  const int c0 = blockIdx.x * ARGMAX_SLICE, c1 = min(n, c0 + ARGMAX_SLICE);
+  unsigned long long best = 0ull;
+  for (int c = c0 + threadIdx.x; c < c1; c += 256) {
     const float v = __bfloat162float(row[c]);
-    if (v > best || (v == best && c < bi)) {  // a NaN compares false: never taken
-      best = v;
-      bi = c;
+    if (v == v) {  // a NaN never wins
+      const unsigned long long k = argmax_key(v, c);
+      best = k > best ? k : best;
     }
   }
-  s_v[threadIdx.x] = best;
-  s_i[threadIdx.x] = bi;
+#pragma unroll
+  for (int msk = 16; msk >= 1; msk >>= 1) {
+    const unsigned long long o = __shfl_xor_sync(0xffffffffu, best, msk);
+    best = o > best ? o : best;
+  }
+  if ((threadIdx.x & 31) == 0) s_k[threadIdx.x >> 5] = best;
   __syncthreads();
-  for (int off = 128; off >= 1; off >>= 1) {
-    if (threadIdx.x < off) {
-      const float v = s_v[threadIdx.x + off];
-      const int j = s_i[threadIdx.x + off];
-      if (v > s_v[threadIdx.x] || (v == s_v[threadIdx.x] && j < s_i[threadIdx.x])) {
-        s_v[threadIdx.x] = v;
-        s_i[threadIdx.x] = j;
-      }
-    }
-    __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w) best = s_k[w] > best ? s_k[w] : best;
+    if (best != 0ull) atomicMax(keys + blockIdx.y, best);
   }
-  if (threadIdx.x == 0) out[blockIdx.x] = s_i[0] == 0x7fffffff ? 0 : s_i[0];
+}
+__global__ void kvd_argmax_finish_kernel(const unsigned long long *__restrict__ keys, int m, int32_t *__restrict__ out) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r < m) out[r] = keys[r] == 0ull ? 0 : 0x7fffffff - static_cast<int>(keys[r] & 0xffffffffull);
 }
 
 static unsigned grid_for(long long items, int per_block, int num_sms) {
@@ -365,7 +372,24 @@ extern "C" kvd_status kvd_scaffold_argmax(kvd_ctx *ctx, const void *logits, int6
   if (!ctx || m < 0 || n <= 0) return KVD_ERR_INVALID_ARG;
   if (m == 0) return KVD_OK;
   if (!logits || !tokens_out || row_stride < n) return KVD_ERR_INVALID_ARG;
-  kvd_argmax_kernel<<<static_cast<unsigned>(m), 256, 0, static_cast<cudaStream_t>(stream_)>>>(
-      static_cast<const __nv_bfloat16 *>(logits), row_stride, n, tokens_out);
-  return sc_launched(ctx, "launch argmax");
+  if (m > 65535) return KVD_ERR_CAPACITY;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  // one 64-bit slot per row, owned by the context (grown on demand; calls on a context are stream-ordered)
+  if (static_cast<size_t>(m) > ctx->argmax_rows) {
+    if (ctx->argmax_keys) cudaFree(ctx->argmax_keys);
+    ctx->argmax_keys = nullptr;
+    ctx->argmax_rows = 0;
+    const size_t rows = m < 64 ? 64 : static_cast<size_t>(m);
+    cudaError_t e = cudaMalloc(&ctx->argmax_keys, rows * sizeof(unsigned long long));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "scaffold argmax: scratch");
+    ctx->argmax_rows = rows;
+  }
+  cudaError_t e = cudaMemsetAsync(ctx->argmax_keys, 0, static_cast<size_t>(m) * sizeof(unsigned long long), stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "scaffold argmax: clear");
+  dim3 grid((n + ARGMAX_SLICE - 1) / ARGMAX_SLICE, m, 1);
+  kvd_argmax_slices_kernel<<<grid, 256, 0, stream>>>(static_cast<const __nv_bfloat16 *>(logits), row_stride, n, ctx->argmax_keys);
+  kvd_status st = sc_launched(ctx, "launch argmax (slices)");
+  if (st != KVD_OK) return st;
+  kvd_argmax_finish_kernel<<<(m + 127) / 128, 128, 0, stream>>>(ctx->argmax_keys, m, tokens_out);
+  return sc_launched(ctx, "launch argmax (finish)");
 }
