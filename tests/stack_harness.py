@@ -169,25 +169,22 @@ class GpuStack:
         pos_t = torch.tensor([pos], dtype=torch.int32, device="cuda")
         for l in range(s.n_layers):
             lw, ls = self.lw[l], s.layer_shape(l)
-            ctx.kvd_checkpoint_residual(0, l, h, pos_t, 1)  # STORE_RESIDUAL: the row entering layer l
             # scaffold: query
             q = self._queries(l, h, pos_t)
-            # hot path: K_t, V_t of the current token, written at its position in the live storage
+            # hot path, ONE launch: STORE_RESIDUAL of the row entering layer l, K_t, V_t of the current token written at
+            # its position in the live storage and, under the bounded policy, RECOMPUTE_KV(C, l) for the evicted tokens
+            # this layer still attends to
             kl, vl = self.k_live[l], self.v_live[l]
             lo = 0 if ls.sliding_window == 0 else max(0, pos - ls.sliding_window + 1)
             wf = self.win_first[l] if self.policy == "kvdirect" else 0
             wf = min(wf, pos)
-            segs = []
+            segs, ranges = [], []
             if self.policy == "kvdirect" and lo < wf:
-                # evicted tokens this layer still attends to: RECOMPUTE_KV(C, l), in the same launch
-                # as K_t, V_t of the current token
                 n = wf - lo
-                ctx.kvd_recompute_kv_step(l, [(0, lo, n, self.k_old, self.v_old)], h, pos_t, 1, kl[pos:], vl[pos:],
-                                          self.kdim)
+                ranges = [(0, lo, n, self.k_old, self.v_old)]
                 self.recomputed_rows += n
                 segs.append((self.k_old, self.v_old, self.kdim, lo, n))
-            else:
-                ctx.kvd_recompute_kv(l, h, pos_t, 1, kl[pos:], vl[pos:], self.kdim)
+            ctx.kvd_decode_step_kv(l, ranges, self.kdim, h, pos_t, 1, [0], kl[pos:], vl[pos:], self.kdim)
             first_live = max(wf, lo) if self.policy == "kvdirect" else 0
             segs.append((kl[first_live:], vl[first_live:], self.kdim, first_live, pos + 1 - first_live))
             out = torch.empty((1, s.n_q_heads, s.d_head), dtype=torch.bfloat16, device="cuda")
