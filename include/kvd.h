@@ -115,8 +115,8 @@ typedef struct {
 /* Byte counts reported by kvd_memory_stats.  The eq* fields are the paper's closed forms for the
  * numbers of tokens currently stored; the others are what this context actually occupies. */
 typedef struct {
-  uint64_t checkpoint_bytes_used;     /* rows + positions + statistics currently held (both stores)      */
-  uint64_t checkpoint_bytes_capacity; /* size the attached arenas must have (both stores)                 */
+  uint64_t checkpoint_bytes_used;     /* rows + positions + statistics currently held (all stores)       */
+  uint64_t checkpoint_bytes_capacity; /* size the attached arenas must have (all stores)                  */
   uint64_t workspace_bytes;           /* attention scratch (split partials)                               */
   uint64_t prepared_weight_bytes;     /* gamma-folded K-major copies of W_kv, rotation tables, key scales */
   uint64_t tokens_stored;             /* max over layers of the rows stored, summed over sequences        */
