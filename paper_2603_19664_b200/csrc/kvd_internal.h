@@ -314,6 +314,24 @@ kvd_status launch_checkpoint(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int3
 kvd_status launch_selftest_bounds(kvd_ctx *ctx, cudaStream_t stream);
 kvd_status launch_checkpoint_scatter(kvd_ctx *ctx, const __nv_bfloat16 *rows, const int32_t *pos, const CkptSlots &slots,
                                      int n, int d_hidden, cudaStream_t stream);
+// kvd_prefill_attention: many query tokens of one sequence, tiled over query rows (Eq. 6-7 per row)
+struct PrefillParams {
+  const __nv_bfloat16 *q;    // [n_rows][n_q][d_head]
+  __nv_bfloat16 *out;        // [n_rows][n_q][d_head]
+  const int32_t *q_pos;      // DEVICE [n_rows]
+  int n_rows, n_q, n_kv, window;
+  float scale_log2e;
+  int seg_lo, seg_hi;        // first and last position any segment holds
+  const __nv_bfloat16 *k[KVD_MAX_SEGMENTS];
+  const __nv_bfloat16 *v[KVD_MAX_SEGMENTS];
+  long long stride[KVD_MAX_SEGMENTS];
+  int first[KVD_MAX_SEGMENTS];
+  int len[KVD_MAX_SEGMENTS];
+  int *status;                    // device status word
+  unsigned long long timeout_ns;  // limit of every in-kernel wait
+};
+// the tcgen05 form of the call (128 MMA rows per CTA, scores and outputs in tensor memory)
+kvd_status launch_prefill_tc(kvd_ctx *ctx, const PrefillParams &P, int d_head, int group, cudaStream_t stream);
 kvd_status launch_selftest_timeout(kvd_ctx *ctx, unsigned long long timeout_ns, cudaStream_t stream);
 kvd_status cuda_fail(kvd_ctx *ctx, cudaError_t e, const char *where);
 // host helpers shared by the entry points (kvd_api.cu)

@@ -15,6 +15,7 @@
 // of kvd_decode_attention (another split, P rounded before the second product): same tolerance against the
 // definition, and callers that need bit-identical outputs across cache policies use one of the two calls throughout.
 #include <math_constants.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "kvd_internal.h"
@@ -25,25 +26,7 @@ namespace kvd {
 constexpr int PF_BLOCK_KEYS = 64;
 constexpr int PF_ROWS = 64;  // MMA rows per CTA
 
-struct PrefillParams {
-  const __nv_bfloat16 *q;    // [n_rows][n_q][d_head]
-  __nv_bfloat16 *out;        // [n_rows][n_q][d_head]
-  const int32_t *q_pos;      // DEVICE [n_rows]
-  int n_rows, n_q, n_kv, window;
-  float scale_log2e;
-  int seg_lo, seg_hi;        // first and last position any segment holds
-  const __nv_bfloat16 *k[KVD_MAX_SEGMENTS];
-  const __nv_bfloat16 *v[KVD_MAX_SEGMENTS];
-  long long stride[KVD_MAX_SEGMENTS];
-  int first[KVD_MAX_SEGMENTS];
-  int len[KVD_MAX_SEGMENTS];
-};
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid) {
-  const int sz = valid ? 16 : 0;  // 0 bytes read: the 16 destination bytes are zero-filled
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
@@ -342,8 +325,13 @@ extern "C" kvd_status kvd_prefill_attention(kvd_ctx *ctx, int layer, int n_rows,
   P.n_kv = d.n_kv_heads;
   P.window = ls.window;
   P.scale_log2e = (scale > 0.f ? scale : 1.0f / sqrtf(static_cast<float>(d.d_head))) * 1.4426950408889634f;
+  P.status = ctx->d_status;
+  P.timeout_ns = ctx->timeout_ns;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   const int group = d.n_q_heads / d.n_kv_heads;
+  // the tcgen05 form unless the environment asks for the mma.sync one (comparisons)
+  static const bool legacy = getenv("KVD_PREFILL_MMA_SYNC") != nullptr;
+  if (!legacy) return launch_prefill_tc(ctx, P, d.d_head, group, stream);
   switch (d.d_head) {
     case 64: return prefill_group<64>(ctx, P, group, stream);
     case 128: return prefill_group<128>(ctx, P, group, stream);

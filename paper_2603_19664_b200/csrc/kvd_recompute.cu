@@ -101,16 +101,6 @@ __device__ __forceinline__ void trace_put(long long *trace, int tile_iter, int f
   if (TRACE) trace_put<TRACE>(trace, tile_iter, field, clock64());
 }
 
-// One lane waits on the barrier, the result is broadcast: the other 31 lanes do not poll shared
-// memory.  The shuffle also orders the lanes' later reads after lane 0's acquire.
-__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag,
-                                          unsigned long long timeout_ns, int lane) {
-  int ok = 1;
-  if (lane == 0) ok = mbar_wait(bar, parity, abort_flag, timeout_ns) ? 1 : 0;
-  ok = __shfl_sync(0xffffffffu, ok, 0);
-  return ok != 0;
-}
-
 // The same wait with a cluster-scope acquire, for barriers whose arrivals publish data that threads of
 // the partner CTA wrote.
 __device__ __forceinline__ bool warp_wait_cluster(uint32_t bar, uint32_t parity, const volatile int *abort_flag,
@@ -128,11 +118,6 @@ __device__ __forceinline__ bool warp_wait_cluster(uint32_t bar, uint32_t parity,
   }
   ok = __shfl_sync(0xffffffffu, ok, 0);
   return ok != 0;
-}
-
-__device__ __forceinline__ void raise(int *status, int bit, volatile int *abort_flag) {
-  atomicOr(status, bit);
-  *abort_flag = 1;
 }
 
 // One k block (64 channels = four K=16 steps) of the pair MMA followed by the commit that frees the
