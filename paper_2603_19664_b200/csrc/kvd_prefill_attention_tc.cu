@@ -6,16 +6,19 @@
 //           tile can see to the last one.
 //   TMEM  = [ O : d_head columns | S_0, S_1 : 64 columns each | Q : d_head / 2 columns ].  The query tile is written
 //           there once (two elements per 32-bit column) and is the A operand of S_j = Q K_j^T; the softmax threads
-//           read S_j (one row per thread, no shuffles), write the weights P_j over it in the element type, and P_j is
-//           the A operand of O += P_j V_j.  Both products are tcgen05.mma with A from tensor memory; shared memory
-//           holds nothing but a ring of K and V blocks.
-//   warps = 0-3 softmax and epilogue (TMEM lane quarter = warp), 4 issues the MMAs, 5-8 gather K/V blocks from the
-//           segments with 16-byte cp.async into the 128-byte-swizzled layouts the two products expect (K block:
-//           K-major B operand, rows = keys; V block: the same bytes read as an MN-major B operand, rows = the
-//           contraction index).  Positions no segment holds are zero-filled and masked.
-//   order = S_0 | S_1 PV_0 | S_2 PV_1 | ... : S_{j+1} runs on the tensor cores while the softmax of block j runs on
-//           the ALUs; the two S buffers alternate.  The running maximum of a row changes rarely after its first blocks;
-//           O is rescaled in tensor memory only when a row of the warp needs it (the others multiply by exactly 1).
+//           read S_j (one row per thread, no shuffles) and hand its columns back at once; the weights P_j go to
+//           shared memory in the element type as the A operand of O += P_j V_j (tensor memory has no room for them
+//           beside two score buffers at d_head = 256, and scores that are free early let S run two blocks ahead).
+//   warps = 0-7 softmax and epilogue (two groups of four, TMEM lane quarter = warp % 4, alternating blocks), 8 issues
+//           the S products, 9 the PV products, 10-13 gather
+//           K/V blocks from the segments with 16-byte cp.async into the 128-byte-swizzled layouts the two products
+//           expect (K block: K-major B operand, rows = keys; V block: the same bytes read as an MN-major B operand,
+//           rows = the contraction index), a ring of K blocks and a ring of V blocks.  Positions no segment holds are
+//           zero-filled and masked.
+//   order = S_j is issued as soon as its K block has landed and the softmax threads have read S_{j-2} out of its
+//           columns, so the scores run up to two blocks ahead of the softmax; PV_j follows the softmax of block j.  The running
+//           maximum of a row changes rarely after its first blocks; O is rescaled in tensor memory only when a row of
+//           the warp needs it (the others multiply by exactly 1).
 //
 // A row's result depends on that row alone: the rows of an MMA are computed independently, every row walks the key
 // blocks of its tile in ascending order, a block without a visible key for the row changes nothing for it (weights 0,
@@ -24,6 +27,7 @@
 // rounded before the second product).  Every wait is bounded: on a timeout the CTA raises the status word, all roles
 // leave their loops, and tensor memory is freed.
 #include <math_constants.h>
+#include <stdio.h>
 
 #include "kvd_internal.h"
 #include "kvd_ptx.cuh"
@@ -32,65 +36,92 @@ namespace kvd {
 
 constexpr int PT_ROWS = 128;     // MMA rows per CTA
 constexpr int PT_KEYS = 64;      // keys per block
-constexpr int PT_THREADS = 288;  // nine warps
-constexpr int PT_LOADERS = 128;  // threads of warps 5-8
+constexpr int PT_THREADS = 448;  // fourteen warps
+constexpr int PT_LOADERS = 128;  // threads of warps 10-13
+constexpr float PT_TAU = 8.0f;   // log2 of the largest weight a row may reach before its reference maximum moves
 constexpr int PT_LAG = 3;        // blocks a loader thread keeps in flight behind the one it is issuing
 
 template <int D_HEAD>
 struct PtCfg {
   static constexpr int TILE_BYTES = PT_KEYS * D_HEAD * 2;       // one K or V block
   static constexpr int SLAB_BYTES = PT_KEYS * 128;              // 64 channels of every key of a block
-  static constexpr int SLOTS = D_HEAD == 256 ? 6 : 8;           // ring of blocks
+  static constexpr int SLOTS_K = D_HEAD == 256 ? 3 : 4;         // blocks in the K ring (the scores run ahead)
+  static constexpr int SLOTS_V = D_HEAD == 256 ? 2 : 4;         // blocks in the V ring
+  static constexpr int SLOTS = SLOTS_K + SLOTS_V;
   static constexpr int COL_O = 0, COL_S = D_HEAD, COL_Q = D_HEAD + 2 * PT_KEYS;
   static constexpr int COLS_USED = COL_Q + D_HEAD / 2;
   static constexpr int COLS = COLS_USED <= 256 ? 256 : 512;     // allocation: a power of two
-  static constexpr int N_BARS = 2 * SLOTS + 8;
-  static constexpr int SMEM_BYTES = 1024 + SLOTS * TILE_BYTES + N_BARS * 8;
+  static constexpr int P_BYTES = PT_ROWS * PT_KEYS * 2;        // one block of weights (K-major A operand of PV)
+  static constexpr int N_BARS = 2 * SLOTS + 22;
+  static constexpr int SMEM_BYTES = 1024 + SLOTS * TILE_BYTES + 2 * P_BYTES + N_BARS * 8;
 };
+
+#ifdef PT_EXP_TRACE
+__device__ long long pt_cta[8192][4];
+__device__ long long pt_trace[64][16];
+#define PT_STAMP(j, f) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (j) >= 32 && (j) < 96) pt_trace[(j) - 32][f] = clock64(); } while (0)
+#else
+#define PT_STAMP(j, f) do { } while (0)
+#endif
 
 template <int D_HEAD, int G, int DT>
 __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(const __grid_constant__ PrefillParams P) {
   using Cfg = PtCfg<D_HEAD>;
   constexpr int GP = G == 3 ? 4 : G;   // heads of the group, padded to a power of two
   constexpr int TOK = PT_ROWS / GP;    // query tokens per CTA
-  constexpr int SLOTS = Cfg::SLOTS;
+  constexpr int SLOTS = Cfg::SLOTS, SLOTS_K = Cfg::SLOTS_K, SLOTS_V = Cfg::SLOTS_V;
   extern __shared__ uint8_t pt_smem_raw[];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort_i, s_lo, s_hi;
+  __shared__ float s_mx[2][PT_ROWS], s_lx[2][PT_ROWS];  // per group: the row maximum after its last block, its part of the row sum
   volatile int *s_abort = &s_abort_i;
   // the ring starts on a 1024-byte boundary (the swizzle is a function of the address), the barriers follow it
   const uint32_t ring = (smem_u32(pt_smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_base = ring + SLOTS * Cfg::TILE_BYTES;
-  auto bar_full = [&](int s) { return bar_base + 8u * s; };
-  auto bar_empty = [&](int s) { return bar_base + 8u * (SLOTS + s); };
+  const uint32_t ring_v = ring + SLOTS_K * Cfg::TILE_BYTES;  // K blocks first, V blocks behind them
+  const uint32_t p_smem = ring + SLOTS * Cfg::TILE_BYTES;    // two blocks of weights
+  const uint32_t bar_base = p_smem + 2 * Cfg::P_BYTES;
+  auto bar_full = [&](int v, int s) { return bar_base + 8u * (v * SLOTS_K + s); };
+  auto bar_empty = [&](int v, int s) { return bar_base + 8u * (SLOTS + v * SLOTS_K + s); };
   auto bar_s_full = [&](int b) { return bar_base + 8u * (2 * SLOTS + b); };
   auto bar_p_ready = [&](int b) { return bar_base + 8u * (2 * SLOTS + 2 + b); };
   auto bar_pv_done = [&](int b) { return bar_base + 8u * (2 * SLOTS + 4 + b); };
   const uint32_t bar_o_full = bar_base + 8u * (2 * SLOTS + 6), bar_q_ready = bar_base + 8u * (2 * SLOTS + 7);
+  auto bar_s_free = [&](int b) { return bar_base + 8u * (2 * SLOTS + 8 + b); };
+  auto bar_m = [&](int grp, int q) { return bar_base + 8u * (2 * SLOTS + 10 + grp * 4 + q); };  // a row maximum was handed over
+  auto bar_l = [&](int q) { return bar_base + 8u * (2 * SLOTS + 18 + q); };                     // both parts of the row sums
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef PT_EXP_TRACE
+  if (tid == 0 && blockIdx.y * gridDim.x + blockIdx.x < 8192) pt_cta[blockIdx.y * gridDim.x + blockIdx.x][0] = globaltimer_ns();
+#endif
   // long tiles (late tokens of a causal call) first
   const int tok0 = (static_cast<int>(gridDim.x) - 1 - static_cast<int>(blockIdx.x)) * TOK, kvh = blockIdx.y;
   const unsigned long long tmo = P.timeout_ns;
 
   if (tid == 0) {
     for (int s = 0; s < SLOTS; ++s) {
-      mbar_init(bar_full(s), PT_LOADERS);  // one arrival per loader thread
-      mbar_init(bar_empty(s), 1);          // the MMA commit
+      mbar_init(bar_full(0, s), 4);   // one arrival per loader warp
+      mbar_init(bar_empty(0, s), 1);  // the MMA commit
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(bar_s_full(b), 1);         // the MMA commit
-      mbar_init(bar_p_ready(b), PT_ROWS);  // one arrival per softmax thread
+      mbar_init(bar_s_full(b), 1);    // the MMA commit
+      mbar_init(bar_p_ready(b), 4);   // one arrival per softmax warp of the group
       mbar_init(bar_pv_done(b), 1);
+      mbar_init(bar_s_free(b), 4);    // one arrival per softmax warp
+    }
+    for (int q = 0; q < 4; ++q) {
+      mbar_init(bar_m(0, q), 1);  // the warp of the group that owns these 32 rows
+      mbar_init(bar_m(1, q), 1);
+      mbar_init(bar_l(q), 2);     // that warp of either group
     }
     mbar_init(bar_o_full, 1);
-    mbar_init(bar_q_ready, PT_ROWS);
+    mbar_init(bar_q_ready, 8);
     fence_mbar_init();
     s_abort_i = 0;
     s_lo = INT_MAX;
     s_hi = -1;
   }
-  if (warp == 4) {
+  if (warp == 8) {
     tmem_alloc(smem_u32(&s_tmem), Cfg::COLS);
     tmem_relinquish();
   }
@@ -113,20 +144,24 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
   const int blk0 = s_hi >= 0 ? s_lo / PT_KEYS : 0;
   const int n_blk = s_hi >= 0 ? s_hi / PT_KEYS - blk0 + 1 : 0;
 
-  if (warp < 4) {
+  if (warp < 8) {
     // ------------------------------------------------------------------ softmax and epilogue: thread = MMA row
-    const int row = tid;
+    // two warpgroups share the 128 rows: group 0 takes the even blocks, group 1 the odd ones, each with its own score
+    // and weight buffer.  What a row carries from block to block is its running maximum, handed from group to group
+    // through shared memory; every group keeps its own part of the row sum.
+    const int wg = warp >> 2, q4 = warp & 3;
+    const int row = q4 * 32 + lane;
     const int tok = tok0 + row / GP, g = row % GP;
     const bool valid = tok < P.n_rows && g < G;
     const int qp = valid ? P.q_pos[tok] : -1;
     const int lo = P.window > 0 ? qp - P.window + 1 : 0;
-    const uint32_t lane_field = static_cast<uint32_t>(warp * 32) << 16;
+    const uint32_t lane_field = static_cast<uint32_t>(q4 * 32) << 16;
     const size_t row_off = (static_cast<size_t>(valid ? tok : 0) * P.n_q + kvh * G + (valid ? g : 0)) * D_HEAD;
     if (n_blk > 0) {
       // the query row into tensor memory: element pairs (2c, 2c + 1) -> column c (zeros for padding rows)
       const uint4 *qsrc = reinterpret_cast<const uint4 *>(P.q + row_off);
 #pragma unroll 1
-      for (int c = 0; c < D_HEAD / 64; ++c) {
+      for (int c = wg; c < D_HEAD / 64; c += 2) {
         uint32_t r[32];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -140,18 +175,23 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       }
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(bar_q_ready);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_q_ready);
     }
-    float m_run = -CUDART_INF_F, l_run = 0.f;
+    float m_own = -CUDART_INF_F;    // the maximum this group's part of the row sum refers to
+    uint64_t l2[2] = {0ull, 0ull};  // that part, in four chains (two packed pairs)
     bool ok = true;
-    for (int j = 0; j < n_blk; ++j) {
-      const int buf = j & 1;
-      if (!warp_wait(bar_s_full(buf), (j >> 1) & 1, s_abort, tmo, lane)) {
+    const uint64_t c2 = pack2(P.scale_log2e, P.scale_log2e), one2 = pack2(1.0f, 1.0f);
+    const int buf = wg;
+    for (int j = wg; j < n_blk; j += 2) {
+      const uint32_t ph = (j >> 1) & 1;
+      if (!warp_wait(bar_s_full(buf), ph, s_abort, tmo, lane)) {
         raise(P.status, STATUS_TIMEOUT, s_abort);
         ok = false;
         break;
       }
       tc_fence_after();
+      if ((tid & 127) == 0) PT_STAMP(j, 0);
       const uint32_t s_col = tmem_base + lane_field + Cfg::COL_S + buf * PT_KEYS;
       uint32_t s0[32], s1[32];
       tmem_ld_x32(s_col, s0);
@@ -173,6 +213,11 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
         vis &= b > a ? (b - a == 64 ? ~0ull : ((1ull << (b - a)) - 1ull) << a) : 0ull;
       }
       tmem_wait_ld();
+      // the scores are in registers: their columns may take this group's next block
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_s_free(buf));
+      if ((tid & 127) == 0) PT_STAMP(j, 1);
       if (!__all_sync(0xffffffffu, vis == ~0ull)) {
         const uint32_t v0 = static_cast<uint32_t>(vis), v1 = static_cast<uint32_t>(vis >> 32);
 #pragma unroll
@@ -181,45 +226,87 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
           if (!((v1 >> k) & 1u)) s1[k] = 0xff800000u;
         }
       }
-      // the block's maximum in four chains
+      // the block's maximum in four chains of three-input maxima
       float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-      for (int k = 0; k < 32; ++k) {
-        mx[k & 3] = fmaxf(mx[k & 3], __uint_as_float(s0[k]));
-        mx[k & 3] = fmaxf(mx[k & 3], __uint_as_float(s1[k]));
+      for (int k = 0; k < 32; k += 8) {
+        mx[0] = fmax3(mx[0], __uint_as_float(s0[k]), __uint_as_float(s0[k + 1]));
+        mx[1] = fmax3(mx[1], __uint_as_float(s0[k + 2]), __uint_as_float(s0[k + 3]));
+        mx[2] = fmax3(mx[2], __uint_as_float(s0[k + 4]), __uint_as_float(s0[k + 5]));
+        mx[3] = fmax3(mx[3], __uint_as_float(s0[k + 6]), __uint_as_float(s0[k + 7]));
+        mx[0] = fmax3(mx[0], __uint_as_float(s1[k]), __uint_as_float(s1[k + 1]));
+        mx[1] = fmax3(mx[1], __uint_as_float(s1[k + 2]), __uint_as_float(s1[k + 3]));
+        mx[2] = fmax3(mx[2], __uint_as_float(s1[k + 4]), __uint_as_float(s1[k + 5]));
+        mx[3] = fmax3(mx[3], __uint_as_float(s1[k + 6]), __uint_as_float(s1[k + 7]));
       }
       const float bm = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * P.scale_log2e;  // log2 units (scale > 0)
-      const float m_new = fmaxf(m_run, bm);
+      // the row's maximum after block j - 1 comes from the other group; the one after block j goes back to it
+      float m_prev = -CUDART_INF_F;
+      if (j > 0) {
+        if (!warp_wait(bar_m(wg ^ 1, q4), ((j - 1) >> 1) & 1, s_abort, tmo, lane)) {
+          raise(P.status, STATUS_TIMEOUT, s_abort);
+          ok = false;
+          break;
+        }
+        m_prev = s_mx[wg ^ 1][row];
+      }
+      // The reference m the weights 2^(s - m) are taken against follows the row's maximum lazily: it moves (and O and
+      // the row sums are rescaled) only when a block's maximum exceeds it by more than 2^PT_TAU; until then the
+      // weights may reach 2^PT_TAU, which fp32 sums and 16-bit weights hold as well as values below 1.  A function of
+      // the row's own scores and of the block order alone, like the maximum itself.
+      const float m_new = m_prev == -CUDART_INF_F ? bm : (bm > m_prev + PT_TAU ? bm : m_prev);
+      s_mx[wg][row] = m_new;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_m(wg, q4));
+      if ((tid & 127) == 0) PT_STAMP(j, 4);
       const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;
       // rescale of what the row has so far: exactly 1 when its maximum stays; while nothing has been seen O and l are 0
-      const float alpha = m_run == -CUDART_INF_F ? 1.0f : ex2_approx(m_run - m_use);
-      m_run = m_new;
-      // weights, rounded to the element type (the rounded weights are also what the row sum adds up)
+      const float alpha = m_prev == -CUDART_INF_F ? 1.0f : ex2_approx(m_prev - m_use);
+      const float alpha_own = m_own == -CUDART_INF_F ? 1.0f : ex2_approx(m_own - m_use);
+      m_own = m_new;
+      // weights 2^(s * scale - m): two per fused multiply-add; the row sum adds them up in fp32, the product takes
+      // them rounded to the element type
       uint32_t w[32];
-      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+      const uint64_t nm2 = pack2(-m_use, -m_use), al2 = pack2(alpha_own, alpha_own);
+      l2[0] = fmul2(l2[0], al2);
+      l2[1] = fmul2(l2[1], al2);
 #pragma unroll
       for (int k = 0; k < 32; k += 2) {
-        const float p0 = ex2_approx(fmaf(__uint_as_float(s0[k]), P.scale_log2e, -m_use));
-        const float p1 = ex2_approx(fmaf(__uint_as_float(s0[k + 1]), P.scale_log2e, -m_use));
+        float e0, e1;
+        unpack2(ffma2(pack2(__uint_as_float(s0[k]), __uint_as_float(s0[k + 1])), c2, nm2), e0, e1);
+        const float p0 = ex2_approx(e0), p1 = ex2_approx(e1);
         w[k >> 1] = pack_out<DT>(p0, p1);
-        float r0, r1;
-        unpack2(x2_to_f32x2<DT>(w[k >> 1]), r0, r1);
-        ls[(k >> 1) & 3] += r0 + r1;
+        l2[(k >> 1) & 1] = ffma2(pack2(p0, p1), one2, l2[(k >> 1) & 1]);
       }
 #pragma unroll
       for (int k = 0; k < 32; k += 2) {
-        const float p0 = ex2_approx(fmaf(__uint_as_float(s1[k]), P.scale_log2e, -m_use));
-        const float p1 = ex2_approx(fmaf(__uint_as_float(s1[k + 1]), P.scale_log2e, -m_use));
+        float e0, e1;
+        unpack2(ffma2(pack2(__uint_as_float(s1[k]), __uint_as_float(s1[k + 1])), c2, nm2), e0, e1);
+        const float p0 = ex2_approx(e0), p1 = ex2_approx(e1);
         w[16 + (k >> 1)] = pack_out<DT>(p0, p1);
-        float r0, r1;
-        unpack2(x2_to_f32x2<DT>(w[16 + (k >> 1)]), r0, r1);
-        ls[(k >> 1) & 3] += r0 + r1;
+        l2[(k >> 1) & 1] = ffma2(pack2(p0, p1), one2, l2[(k >> 1) & 1]);
       }
-      l_run = fmaf(l_run, alpha, (ls[0] + ls[1]) + (ls[2] + ls[3]));
-      tmem_st_x32(s_col, w);  // P_j over the first half of S_j
+      if ((tid & 127) == 0) PT_STAMP(j, 2);
+      // P_j into shared memory as a K-major A operand (row = MMA row, 128 bytes = 64 keys, 128-byte swizzle); the
+      // product that read this buffer two blocks ago has long finished
+      if (j >= 2 && !warp_wait(bar_pv_done(buf), ((j - 2) >> 1) & 1, s_abort, tmo, lane)) {
+        raise(P.status, STATUS_TIMEOUT, s_abort);
+        ok = false;
+        break;
+      }
+      {
+        const uint32_t prow = p_smem + buf * Cfg::P_BYTES + row * 128;
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(prow + ((i ^ (row & 7)) << 4)), "r"(w[4 * i]), "r"(w[4 * i + 1]),
+                       "r"(w[4 * i + 2]), "r"(w[4 * i + 3])
+                       : "memory");
+        fence_proxy_async_smem();
+      }
+      if ((tid & 127) == 0) PT_STAMP(j, 8);
       if (__any_sync(0xffffffffu, alpha != 1.0f)) {
         // O holds the blocks before j; the last of those products must have finished (j >= 1 here: a maximum exists)
-        if (!warp_wait(bar_pv_done((j - 1) & 1), ((j - 1) >> 1) & 1, s_abort, tmo, lane)) {
+        if (!warp_wait(bar_pv_done(buf ^ 1), ((j - 1) >> 1) & 1, s_abort, tmo, lane)) {
           raise(P.status, STATUS_TIMEOUT, s_abort);
           ok = false;
           break;
@@ -234,12 +321,42 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
           for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
           tmem_st_x32(tmem_base + lane_field + Cfg::COL_O + c * 32, r);
         }
+        tmem_wait_st();
+        tc_fence_before();
       }
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(bar_p_ready(buf));
+      __syncwarp();
+      if ((tid & 127) == 0) PT_STAMP(j, 3);
+      if (lane == 0) mbar_arrive(bar_p_ready(buf));
     }
-    // ---- normalise and store (a token without a visible key yields zeros)
+    // ---- the row sum: both parts referred to the final maximum, added in group order
+    float l_run = 0.f;
+    if (ok && n_blk > 0) {
+      const int last = n_blk - 1;
+      float m_fin = m_own;
+      if ((last & 1) != wg) {
+        if (!warp_wait(bar_m(wg ^ 1, q4), (last >> 1) & 1, s_abort, tmo, lane)) {
+          raise(P.status, STATUS_TIMEOUT, s_abort);
+          ok = false;
+        }
+        m_fin = s_mx[wg ^ 1][row];
+      }
+      if (ok) {
+        const float m_use = m_fin == -CUDART_INF_F ? 0.f : m_fin;
+        float a0, a1, a2, a3;
+        unpack2(l2[0], a0, a1);
+        unpack2(l2[1], a2, a3);
+        const float mine = ((a0 + a1) + (a2 + a3)) * (m_own == -CUDART_INF_F ? 1.0f : ex2_approx(m_own - m_use));
+        s_lx[wg][row] = mine;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_l(q4));
+        if (!warp_wait(bar_l(q4), 0, s_abort, tmo, lane)) {
+          raise(P.status, STATUS_TIMEOUT, s_abort);
+          ok = false;
+        }
+        l_run = s_lx[0][row] + s_lx[1][row];
+      }
+    }
+    // ---- normalise and store, each group its half of the channels (a token without a visible key yields zeros)
     if (ok && n_blk > 0 && !warp_wait(bar_o_full, 0, s_abort, tmo, lane)) {
       raise(P.status, STATUS_TIMEOUT, s_abort);
       ok = false;
@@ -249,7 +366,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       const float inv = l_run > 0.f ? 1.0f / l_run : 0.f;
       uint4 *dst = reinterpret_cast<uint4 *>(P.out + row_off);
 #pragma unroll 1
-      for (int c = 0; c < D_HEAD / 32; ++c) {
+      for (int c = wg * (D_HEAD / 64); c < (wg + 1) * (D_HEAD / 64); ++c) {
         uint32_t r[32];
         if (n_blk > 0) {
           tmem_ld_x32(tmem_base + lane_field + Cfg::COL_O + c * 32, r);
@@ -267,108 +384,157 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
         }
       }
     }
-  } else if (warp == 4) {
-    // ------------------------------------------------------------------ MMA issue (one thread)
-    if (lane == 0 && n_blk > 0) {
-      constexpr uint32_t IDESC_BASE = DT == 0 ? umma_idesc_bf16_f32(PT_ROWS, 8) & ~(1u << 17) : umma_idesc_f16_f32(PT_ROWS, 8) & ~(1u << 17);
-      constexpr uint32_t IDESC_S = IDESC_BASE | (static_cast<uint32_t>(PT_KEYS >> 3) << 17);                 // N = 64 keys, B K-major
-      constexpr uint32_t IDESC_O = IDESC_BASE | (static_cast<uint32_t>(D_HEAD >> 3) << 17) | (1u << 16);     // N = d_head, B MN-major
-      int t = 0;  // blocks taken from the ring so far
+  } else if (warp == 8 || warp == 9) {
+    // ------------------------------------------------------------------ MMA issue (one thread per product)
+    constexpr uint32_t IDESC_BASE = DT == 0 ? umma_idesc_bf16_f32(PT_ROWS, 8) & ~(1u << 17) : umma_idesc_f16_f32(PT_ROWS, 8) & ~(1u << 17);
+    constexpr uint32_t IDESC_S = IDESC_BASE | (static_cast<uint32_t>(PT_KEYS >> 3) << 17);              // N = 64 keys, B K-major
+    constexpr uint32_t IDESC_O = IDESC_BASE | (static_cast<uint32_t>(D_HEAD >> 3) << 17) | (1u << 16);  // N = d_head, B MN-major
+    if (lane == 0 && n_blk > 0 && warp == 8) {
+      // S_j = Q K_j^T into score buffer j & 1, as far ahead of the softmax as the two buffers allow
       bool ok = mbar_wait(bar_q_ready, 0, s_abort, tmo);
-      if (!ok) raise(P.status, STATUS_TIMEOUT, s_abort);
       tc_fence_after();
-      // S_j = Q K_j^T into score buffer j & 1
-      auto issue_s = [&](int j) -> bool {
-        const int slot = t % SLOTS;
-        if (!mbar_wait(bar_full(slot), (t / SLOTS) & 1, s_abort, tmo)) return false;
+      for (int j = 0; ok && j < n_blk; ++j) {
+        const int slot = j % SLOTS_K;
+        PT_STAMP(j, 9);
+        // the K block has landed; the softmax threads have read the scores of block j - 2 out of these columns
+        if (!mbar_wait(bar_full(0, slot), (j / SLOTS_K) & 1, s_abort, tmo) ||
+            (j >= 2 && !mbar_wait(bar_s_free(j & 1), ((j - 2) >> 1) & 1, s_abort, tmo))) {
+          ok = false;
+          break;
+        }
         tc_fence_after();
+        PT_STAMP(j, 10);
         const uint32_t kb = ring + slot * Cfg::TILE_BYTES;
         const uint32_t d = tmem_base + Cfg::COL_S + (j & 1) * PT_KEYS;
+        const uint64_t desc0 = umma_smem_desc_sw128(kb);
 #pragma unroll
         for (int ks = 0; ks < D_HEAD / 16; ++ks)
-          umma_f16_ts(d, tmem_base + Cfg::COL_Q + ks * 8, umma_smem_desc_sw128(kb + (ks >> 2) * Cfg::SLAB_BYTES + (ks & 3) * 32),
-                      IDESC_S, ks > 0 ? 1u : 0u);
-        umma_commit(bar_empty(slot));
+          umma_f16_ts(d, tmem_base + Cfg::COL_Q + ks * 8, desc0 + (((ks >> 2) * Cfg::SLAB_BYTES + (ks & 3) * 32) >> 4), IDESC_S,
+                      ks > 0 ? 1u : 0u);
+        umma_commit(bar_empty(0, slot));
         umma_commit(bar_s_full(j & 1));
-        ++t;
-        return true;
-      };
-      if (ok) ok = issue_s(0);
-      for (int j = 0; ok && j < n_blk; ++j) {
-        if (j + 1 < n_blk && !issue_s(j + 1)) {
-          ok = false;
-          break;
-        }
-        // O += P_j V_j once the weights are in place (and O has been rescaled where a maximum moved)
-        const int slot = t % SLOTS;
-        if (!mbar_wait(bar_p_ready(j & 1), (j >> 1) & 1, s_abort, tmo) || !mbar_wait(bar_full(slot), (t / SLOTS) & 1, s_abort, tmo)) {
+        PT_STAMP(j, 5);
+      }
+      if (!ok) raise(P.status, STATUS_TIMEOUT, s_abort);
+    } else if (lane == 0 && n_blk > 0) {
+      // O += P_j V_j once the weights are in place (and O has been rescaled where a maximum moved)
+      bool ok = true;
+      for (int j = 0; j < n_blk; ++j) {
+        const int slot = j % SLOTS_V;
+        if (!mbar_wait(bar_p_ready(j & 1), (j >> 1) & 1, s_abort, tmo) || !mbar_wait(bar_full(1, slot), (j / SLOTS_V) & 1, s_abort, tmo)) {
           ok = false;
           break;
         }
         tc_fence_after();
-        const uint32_t vb = ring + slot * Cfg::TILE_BYTES;
+        PT_STAMP(j, 6);
+        const uint64_t desc0 = umma_smem_desc_sw128_mn(ring_v + slot * Cfg::TILE_BYTES, Cfg::SLAB_BYTES);
+        const uint64_t pdesc0 = umma_smem_desc_sw128(p_smem + (j & 1) * Cfg::P_BYTES);
 #pragma unroll
         for (int ks = 0; ks < PT_KEYS / 16; ++ks)
-          umma_f16_ts(tmem_base + Cfg::COL_O, tmem_base + Cfg::COL_S + (j & 1) * PT_KEYS + ks * 8,
-                      umma_smem_desc_sw128_mn(vb + ks * 16 * 128, Cfg::SLAB_BYTES), IDESC_O, (j > 0 || ks > 0) ? 1u : 0u);
-        umma_commit(bar_empty(slot));
+          umma_bf16(tmem_base + Cfg::COL_O, pdesc0 + ((ks * 32) >> 4), desc0 + ((ks * 16 * 128) >> 4), IDESC_O,
+                    (j > 0 || ks > 0) ? 1u : 0u);
+        umma_commit(bar_empty(1, slot));
         umma_commit(bar_pv_done(j & 1));
-        ++t;
+        PT_STAMP(j, 7);
       }
       if (ok) umma_commit(bar_o_full);
       else raise(P.status, STATUS_TIMEOUT, s_abort);
     }
   } else {
-    // ------------------------------------------------------------------ K/V blocks into the ring
-    // ring order = the order the MMA thread consumes them: K_0 | K_1 V_0 | K_2 V_1 | ...
+    // ------------------------------------------------------------------ K/V blocks into the rings
+    // issue order = the order the products want them, the keys two blocks ahead: K_0 K_1 | K_2 V_0 | K_3 V_1 | ...
     constexpr int CPR = D_HEAD / 8;           // 16-byte pieces per key
     constexpr int RSTEP = PT_LOADERS / CPR;   // keys one pass of the 128 threads covers
-    const int ptid = tid - 5 * 32;
+    const int ptid = tid - 10 * 32;
     const int c = ptid % CPR, r0 = ptid / CPR;
     const uint32_t dst_c = static_cast<uint32_t>(c >> 3) * Cfg::SLAB_BYTES;
-    int t = 0;
+    // blocks issued and not yet published to the MMA threads, oldest first.  A block is published once PT_LAG younger
+    // ones have been issued -- or at once, all of them, when the next block would have to wait for a free slot (the
+    // slot is freed by a product that may itself be waiting for one of these blocks).
+    uint32_t pend[PT_LAG + 1] = {};
+    int n_pend = 0;
     bool ok = true;
-    auto emit = [&](bool is_v, int j) -> bool {
-      const int slot = t % SLOTS;
-      if (t >= SLOTS && !warp_wait(bar_empty(slot), ((t / SLOTS) - 1) & 1, s_abort, tmo, lane)) return false;
-      const int pos0 = (blk0 + j) * PT_KEYS;
-      const uint32_t base = ring + slot * Cfg::TILE_BYTES + dst_c;
+    auto publish_all = [&]() {
+      cp_async_wait_all();
+      fence_proxy_async_smem();
+      __syncwarp();
 #pragma unroll
-      for (int pass = 0; pass < PT_KEYS / RSTEP; ++pass) {
-        const int r = r0 + pass * RSTEP, pos = pos0 + r;
-        const __nv_bfloat16 *src = P.q;
-        bool have = false;
-#pragma unroll
-        for (int sg = 0; sg < KVD_MAX_SEGMENTS; ++sg) {
-          const int rr = pos - P.first[sg];
-          if (rr >= 0 && rr < P.len[sg]) {
-            src = (is_v ? P.v[sg] : P.k[sg]) + static_cast<size_t>(rr) * P.stride[sg] + static_cast<size_t>(kvh) * D_HEAD + c * 8;
-            have = true;
-          }
+      for (int i = 0; i <= PT_LAG; ++i)
+        if (i < n_pend && lane == 0) mbar_arrive(pend[i]);
+      n_pend = 0;
+    };
+    auto emit = [&](int is_v, int j) -> bool {
+      const int n_slots = is_v ? SLOTS_V : SLOTS_K, slot = j % n_slots;
+      if (j >= n_slots) {
+        const uint32_t par = ((j / n_slots) - 1) & 1;
+        int free_now = lane == 0 ? (mbar_try_wait(bar_empty(is_v, slot), par) ? 1 : 0) : 0;
+        free_now = __shfl_sync(0xffffffffu, free_now, 0);
+        if (!free_now) {
+          publish_all();
+          if (!warp_wait(bar_empty(is_v, slot), par, s_abort, tmo, lane)) return false;
         }
-        cp_async16(base + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, have);
+      }
+      const int pos0 = (blk0 + j) * PT_KEYS;
+      const uint32_t base = (is_v ? ring_v : ring) + slot * Cfg::TILE_BYTES + dst_c;
+      // the usual case: one segment holds the whole block -> one base pointer, one stride
+      int whole = -1;
+#pragma unroll
+      for (int sg = 0; sg < KVD_MAX_SEGMENTS; ++sg)
+        if (P.first[sg] <= pos0 && pos0 + PT_KEYS <= P.first[sg] + P.len[sg]) whole = sg;
+      if (whole >= 0) {
+        const long long stride = P.stride[whole];
+        const __nv_bfloat16 *src = (is_v ? P.v[whole] : P.k[whole]) + static_cast<size_t>(pos0 - P.first[whole] + r0) * stride +
+                                   static_cast<size_t>(kvh) * D_HEAD + c * 8;
+#pragma unroll
+        for (int pass = 0; pass < PT_KEYS / RSTEP; ++pass) {
+          const int r = r0 + pass * RSTEP;
+          cp_async16(base + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, true);
+          src += RSTEP * stride;
+        }
+      } else {
+#pragma unroll 1
+        for (int pass = 0; pass < PT_KEYS / RSTEP; ++pass) {
+          const int r = r0 + pass * RSTEP, pos = pos0 + r;
+          const __nv_bfloat16 *src = P.q;
+          bool have = false;
+#pragma unroll
+          for (int sg = 0; sg < KVD_MAX_SEGMENTS; ++sg) {
+            const int rr = pos - P.first[sg];
+            if (rr >= 0 && rr < P.len[sg]) {
+              src = (is_v ? P.v[sg] : P.k[sg]) + static_cast<size_t>(rr) * P.stride[sg] + static_cast<size_t>(kvh) * D_HEAD + c * 8;
+              have = true;
+            }
+          }
+          cp_async16(base + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, have);
+        }
       }
       cp_async_commit();
-      if (t >= PT_LAG) {
-        // the block issued PT_LAG blocks ago has landed: publish it to the tensor cores' view of shared memory
+#pragma unroll
+      for (int i = 0; i <= PT_LAG; ++i)
+        if (i == n_pend) pend[i] = bar_full(is_v, slot);
+      ++n_pend;
+      if (n_pend > PT_LAG) {
+        // the oldest block has PT_LAG younger ones behind it: it has landed by now, or nearly
         cp_async_wait_group<PT_LAG>();
         fence_proxy_async_smem();
-        mbar_arrive(bar_full((t - PT_LAG) % SLOTS));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pend[0]);
+#pragma unroll
+        for (int i = 0; i < PT_LAG; ++i) pend[i] = pend[i + 1];
+        --n_pend;
       }
-      ++t;
       return true;
     };
     if (n_blk > 0) {
-      ok = emit(false, 0);
+      ok = emit(0, 0);
+      if (ok && n_blk > 1) ok = emit(0, 1);
       for (int j = 0; ok && j < n_blk; ++j) {
-        if (j + 1 < n_blk) ok = emit(false, j + 1);
-        if (ok) ok = emit(true, j);
+        if (j + 2 < n_blk) ok = emit(0, j + 2);
+        if (ok) ok = emit(1, j);
       }
-      cp_async_wait_all();
-      if (ok) {
-        fence_proxy_async_smem();
-        for (int u = t > PT_LAG ? t - PT_LAG : 0; u < t; ++u) mbar_arrive(bar_full(u % SLOTS));
-      } else {
+      if (ok) publish_all();
+      else {
+        cp_async_wait_all();
         raise(P.status, STATUS_TIMEOUT, s_abort);
       }
     }
@@ -377,7 +543,19 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
   // ---- teardown: every role is done with tensor memory
   tc_fence_before();
   __syncthreads();
-  if (warp == 4) {
+#ifdef PT_EXP_TRACE
+  if (tid == 0) {
+    const int id = blockIdx.y * gridDim.x + blockIdx.x;
+    if (id < 8192) {
+      unsigned smid;
+      asm("mov.u32 %0, %%smid;" : "=r"(smid));
+      pt_cta[id][1] = globaltimer_ns();
+      pt_cta[id][2] = n_blk;
+      pt_cta[id][3] = smid;
+    }
+  }
+#endif
+  if (warp == 8) {
     tc_fence_after();
     tmem_dealloc(tmem_base, Cfg::COLS);
   }
@@ -402,6 +580,42 @@ static kvd_status prefill_tc_launch(kvd_ctx *ctx, const PrefillParams &P, cudaSt
   else k0<<<grid, PT_THREADS, Cfg::SMEM_BYTES, stream>>>(P);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(ctx, e, "launch prefill attention");
+#ifdef PT_EXP_TRACE
+  {
+    static int printed = 0;
+    if (!printed && grid.x > 200) {
+      printed = 1;
+      cudaDeviceSynchronize();
+      static long long h[64][16];
+      cudaMemcpyFromSymbol(h, pt_trace, sizeof(h));
+      {
+        static long long c[8192][4];
+        cudaMemcpyFromSymbol(c, pt_cta, sizeof(c));
+        const int n = grid.x * grid.y < 8192 ? grid.x * grid.y : 8192;
+        long long t0 = c[0][0], t1 = 0, busy[256] = {}, blocks[256] = {}, ctas[256] = {};
+        for (int i = 0; i < n; ++i) { if (c[i][0] < t0) t0 = c[i][0]; if (c[i][1] > t1) t1 = c[i][1]; }
+        double per_blk_sum = 0; int per_blk_n = 0;
+        for (int i = 0; i < n; ++i) {
+          const int sm = (int)c[i][3] & 255;
+          busy[sm] += c[i][1] - c[i][0]; blocks[sm] += c[i][2]; ctas[sm] += 1;
+          if (c[i][2] >= 64) { per_blk_sum += double(c[i][1] - c[i][0]) / c[i][2]; ++per_blk_n; }
+        }
+        fprintf(stderr, "kernel span %lld ns; ns per block over CTAs with >= 64 blocks: %.1f\n", t1 - t0, per_blk_sum / per_blk_n);
+        for (int sm = 0; sm < 148; sm += 21) fprintf(stderr, "  sm %3d: ctas %lld blocks %lld busy %lld ns\n", sm, ctas[sm], blocks[sm], busy[sm]);
+        long long bmin = 1ll << 60, bmax = 0, kmin = 1ll << 60, kmax = 0;
+        for (int sm = 0; sm < 148; ++sm) { if (busy[sm] < bmin) bmin = busy[sm]; if (busy[sm] > bmax) bmax = busy[sm]; if (blocks[sm] < kmin) kmin = blocks[sm]; if (blocks[sm] > kmax) kmax = blocks[sm]; }
+        fprintf(stderr, "  busy ns min %lld max %lld; blocks min %lld max %lld\n", bmin, bmax, kmin, kmax);
+        for (int i = 0; i < n; i += n / 16) fprintf(stderr, "  cta %4d: start %8lld dur %8lld blk %3lld sm %3lld  ns/blk %.1f\n", i, c[i][0] - t0, c[i][1] - c[i][0], c[i][2], c[i][3], c[i][2] ? double(c[i][1] - c[i][0]) / c[i][2] : 0.0);
+      }
+      for (int j = 0; j < 4; ++j) {
+        fprintf(stderr, "blk %3d:", j + 32);
+        for (int f = 0; f < 15; ++f) fprintf(stderr, " %7lld", h[j][f] ? h[j][f] - h[0][0] : -1);
+        fprintf(stderr, " %llx", h[j][15]);
+        fprintf(stderr, "\n");
+      }
+    }
+  }
+#endif
   ctx->launches += 1;
   return KVD_OK;
 }

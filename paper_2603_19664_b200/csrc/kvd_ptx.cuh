@@ -73,8 +73,11 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag,
                                           unsigned long long timeout_ns) {
-  if (mbar_try_wait(bar, parity)) return true;
-  if (mbar_try_wait(bar, parity)) return true;
+  // a short inline spin first: a hand-over between two warps completes within a few attempts, and entering the
+  // out-of-line path (a call, a timer read) would add its cost to every one of them
+#pragma unroll 1
+  for (int i = 0; i < 16; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, abort_flag, timeout_ns);
 }
 
@@ -95,6 +98,12 @@ __device__ __forceinline__ void raise(int *status, int bit, volatile int *abort_
   *abort_flag = 1;
 }
 
+// max(a, b, c) in one instruction
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 // 2^x on the special-function unit (subnormal results flush to zero; 2^-inf = 0)
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
