@@ -453,6 +453,12 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
     // slot is freed by a product that may itself be waiting for one of these blocks).
     uint32_t pend[PT_LAG + 1] = {};
     int n_pend = 0;
+#ifdef PT_EXP_TRACE
+    int ptag[PT_LAG + 1] = {};
+#define PT_PUB(i) do { if (ptid == 0) PT_STAMP(ptag[i] % 1000, ptag[i] >= 1000 ? 15 : 13); } while (0)
+#else
+#define PT_PUB(i) do { } while (0)
+#endif
     bool ok = true;
     auto publish_all = [&]() {
       cp_async_wait_all();
@@ -460,7 +466,10 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       __syncwarp();
 #pragma unroll
       for (int i = 0; i <= PT_LAG; ++i)
-        if (i < n_pend && lane == 0) mbar_arrive(pend[i]);
+        if (i < n_pend && lane == 0) {
+          mbar_arrive(pend[i]);
+          PT_PUB(i);
+        }
       n_pend = 0;
     };
     auto emit = [&](int is_v, int j) -> bool {
@@ -474,6 +483,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
           if (!warp_wait(bar_empty(is_v, slot), par, s_abort, tmo, lane)) return false;
         }
       }
+      if (ptid == 0) PT_STAMP(j, is_v ? 14 : 12);
       const int pos0 = (blk0 + j) * PT_KEYS;
       const uint32_t base = (is_v ? ring_v : ring) + slot * Cfg::TILE_BYTES + dst_c;
       // the usual case: one segment holds the whole block -> one base pointer, one stride
@@ -511,7 +521,12 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       cp_async_commit();
 #pragma unroll
       for (int i = 0; i <= PT_LAG; ++i)
-        if (i == n_pend) pend[i] = bar_full(is_v, slot);
+        if (i == n_pend) {
+          pend[i] = bar_full(is_v, slot);
+#ifdef PT_EXP_TRACE
+          ptag[i] = is_v * 1000 + j;
+#endif
+        }
       ++n_pend;
       if (n_pend > PT_LAG) {
         // the oldest block has PT_LAG younger ones behind it: it has landed by now, or nearly
@@ -519,8 +534,14 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(pend[0]);
+        PT_PUB(0);
 #pragma unroll
-        for (int i = 0; i < PT_LAG; ++i) pend[i] = pend[i + 1];
+        for (int i = 0; i < PT_LAG; ++i) {
+          pend[i] = pend[i + 1];
+#ifdef PT_EXP_TRACE
+          ptag[i] = ptag[i + 1];
+#endif
+        }
         --n_pend;
       }
       return true;
@@ -607,10 +628,9 @@ static kvd_status prefill_tc_launch(kvd_ctx *ctx, const PrefillParams &P, cudaSt
         fprintf(stderr, "  busy ns min %lld max %lld; blocks min %lld max %lld\n", bmin, bmax, kmin, kmax);
         for (int i = 0; i < n; i += n / 16) fprintf(stderr, "  cta %4d: start %8lld dur %8lld blk %3lld sm %3lld  ns/blk %.1f\n", i, c[i][0] - t0, c[i][1] - c[i][0], c[i][2], c[i][3], c[i][2] ? double(c[i][1] - c[i][0]) / c[i][2] : 0.0);
       }
-      for (int j = 0; j < 4; ++j) {
+      for (int j = 0; j < 8; ++j) {
         fprintf(stderr, "blk %3d:", j + 32);
-        for (int f = 0; f < 15; ++f) fprintf(stderr, " %7lld", h[j][f] ? h[j][f] - h[0][0] : -1);
-        fprintf(stderr, " %llx", h[j][15]);
+        for (int f = 0; f < 16; ++f) fprintf(stderr, " %7lld", h[j][f] ? h[j][f] - h[0][0] : -1);
         fprintf(stderr, "\n");
       }
     }

@@ -4,7 +4,9 @@
     layer's window), at the attention tolerance: relative Frobenius <= 1e-2, max abs <= 1e-2 * max |oracle|;
   * a row's bits depend on the row, its position and the keys only: the same token attended alone, in a short call
     and in a long one, first or last of its tile, gives identical bits;
-  * segments, gaps between segments, rows beyond the last key, rows without a visible key (zeros), group sizes 1-8.
+  * segments, gaps between segments, rows beyond the last key, rows without a visible key (zeros), group sizes 1-8;
+  * keys whose magnitude grows or shrinks from block to block (the lazily followed maximum and the rescale of the
+    accumulated output), odd tile counts, calls far longer than the sliding window, shuffled query rows, fp16.
 """
 import math
 
@@ -15,7 +17,7 @@ import torch
 import oracle
 import paper_2603_19664_b200 as kvd
 from kvd_synth import (LayerShape, GEMMA3_4B_GLOBAL, GEMMA3_4B_LOCAL, QWEN3_4B, SMOLLM2_135M, TINY_GQA, TINY_MHA, bf16_to_f64,
-                       make_kv, make_query)
+                       f32_to_bf16_bits, make_kv, make_layer_weights, make_query)
 from gpu_util import dev, host_f64, open_layer
 
 pytestmark = pytest.mark.gpu
@@ -103,4 +105,82 @@ def test_group_sizes(group):
     assert ctx.kvd_poll_status() == kvd.KVD_OK
     sample = [0, 1, 15, 16, 63, 64, 65, 199]
     attn_check(host_f64(out[torch.tensor(sample).cuda()]), oracle_rows(shape, q_bits, q_pos, [(K, V, 0)], sample))
+    ctx.close()
+
+
+@pytest.mark.parametrize("ramp", ["up", "down"])
+def test_scores_whose_maximum_jumps_by_large_factors(ramp):
+    """The kernel follows a row's maximum lazily (its reference moves only when a block exceeds it by 2^8) and
+    rescales what it has accumulated when it does: keys whose magnitude grows from block to block force that path in
+    every block, keys that shrink never take it again after the first; both must follow Eq. 6-7."""
+    shape = QWEN3_4B
+    ctx, _ = open_layer(shape, max_tokens=2048)
+    kdim = shape.n_kv_heads * shape.d_head
+    T = 700
+    K, V = make_kv(shape, T, seed=31)
+    kf = bf16_to_f64(K)
+    growth = 1.6 ** (np.arange(T) // 64)                       # x 1.6 per 64-key block: 11 blocks span a factor of 110
+    kf = kf * (growth if ramp == "up" else growth[::-1])[:, None, None]
+    K = f32_to_bf16_bits(kf.astype(np.float32))
+    q_pos = np.arange(T)
+    q_bits = make_query(shape, T, seed=32)
+    out = torch.zeros((T, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda")
+    ctx.kvd_prefill_attention(0, T, dev(q_bits), torch.from_numpy(q_pos.astype(np.int32)).cuda(), [(dev(K), dev(V), kdim, 0, T)], 0.0, out)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    sample = [0, 63, 64, 130, 257, 448, 449, 640, T - 1]
+    attn_check(host_f64(out[torch.tensor(sample).cuda()]), oracle_rows(shape, q_bits, q_pos, [(K, V, 0)], sample))
+    ctx.close()
+
+
+@pytest.mark.parametrize("shape,T", [(GEMMA3_4B_GLOBAL, 64 * 5 + 7), (GEMMA3_4B_LOCAL, 2500), (QWEN3_4B, 32 * 7), (SMOLLM2_135M, 32 * 3 + 1)],
+                         ids=lambda v: getattr(v, "name", str(v)))
+def test_odd_numbers_of_tiles_long_rows_and_unsorted_positions(shape, T):
+    """Tile counts that are odd, a call much longer than the sliding window (tiles that start far from position 0),
+    and query rows given in a shuffled order: every sampled row follows the oracle, and the shuffled call returns the
+    bits of the ordered one row for row."""
+    ctx, _ = open_layer(shape, max_tokens=4096)
+    kdim = shape.n_kv_heads * shape.d_head
+    K, V = make_kv(shape, T, seed=41)
+    k, v = dev(K), dev(V)
+    q_bits = make_query(shape, T, seed=42)
+    q_pos = np.arange(T)
+    out = torch.zeros((T, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda")
+    ctx.kvd_prefill_attention(0, T, dev(q_bits), torch.from_numpy(q_pos.astype(np.int32)).cuda(), [(k, v, kdim, 0, T)], 0.0, out)
+    rng = np.random.default_rng(43)
+    sample = sorted(set([0, 1, T // 2, T - 2, T - 1] + rng.choice(T, 10, replace=False).tolist()))
+    attn_check(host_f64(out[torch.tensor(sample).cuda()]), oracle_rows(shape, q_bits, q_pos, [(K, V, 0)], sample))
+    perm = rng.permutation(T)
+    out2 = torch.zeros_like(out)
+    ctx.kvd_prefill_attention(0, T, dev(q_bits[perm]), torch.from_numpy(q_pos[perm].astype(np.int32)).cuda(), [(k, v, kdim, 0, T)], 0.0, out2)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    assert torch.equal(out2, out[torch.from_numpy(perm).cuda()])
+    ctx.close()
+
+
+@pytest.mark.parametrize("shape", [GEMMA3_4B_GLOBAL, QWEN3_4B, SMOLLM2_135M], ids=lambda s: s.name)
+def test_fp16_prefill_attention_follows_the_oracle(shape):
+    w = make_layer_weights(shape)
+    desc = kvd.make_desc(1, shape.d_hidden, shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.rms_eps,
+                         shape.qk_norm, shape.rms_eps, shape.rope_style, 1, 2048, 1)
+    ctx = kvd.Kvd(desc)
+    ctx.kvd_set_dtype(1)
+    to16 = lambda bits: torch.from_numpy(bf16_to_f64(bits).astype(np.float16)).cuda()
+    ctx.kvd_set_layer(0, to16(w.w_kv), to16(w.gamma_in), to16(w.gamma_k) if w.gamma_k is not None else None, shape.rope_theta,
+                      shape.sliding_window)
+    kdim = shape.n_kv_heads * shape.d_head
+    T = 333
+    rng = np.random.default_rng(7)
+    q16 = rng.standard_normal((T, shape.n_q_heads, shape.d_head)).astype(np.float16)
+    k16 = rng.standard_normal((T, kdim)).astype(np.float16)
+    v16 = rng.standard_normal((T, kdim)).astype(np.float16)
+    q_pos = np.arange(T) + 9
+    out = torch.zeros((T, shape.n_q_heads, shape.d_head), dtype=torch.float16, device="cuda")
+    ctx.kvd_prefill_attention(0, T, torch.from_numpy(q16).cuda(), torch.from_numpy(q_pos.astype(np.int32)).cuda(),
+                              [(torch.from_numpy(k16).cuda(), torch.from_numpy(v16).cuda(), kdim, 9, T)], 0.0, out)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    sample = [0, 1, 63, 64, 65, 200, T - 1]
+    kv = (k16.astype(np.float64).reshape(T, shape.n_kv_heads, shape.d_head), v16.astype(np.float64).reshape(T, shape.n_kv_heads, shape.d_head), 9)
+    ref = np.stack([oracle.decode_attention(q16[i].astype(np.float64), int(q_pos[i]), [kv], 1.0 / math.sqrt(shape.d_head),
+                                            shape.sliding_window) for i in sample])
+    attn_check(out[torch.tensor(sample).cuda()].double().cpu().numpy(), ref)
     ctx.close()
