@@ -2,32 +2,40 @@
 //
 //   CTA   = (tile of query tokens, KV head): 128 MMA rows = 128 / Gp tokens x Gp query heads of the head's group
 //           (Gp = group size rounded up to a power of two; padding heads are zero rows that are never stored).
+//   pair  = for d_head >= 128 two CTAs with neighbouring tiles of the same KV head form a cluster and run the products
+//           as tcgen05.mma.cta_group::2 (M = 256, 128 rows per CTA): a K or V block is shared by the pair, each CTA
+//           loads and holds half of it (K: half the keys, V: half the channels -- the halves the instruction reads from
+//           either shared memory).  Half the bytes per CTA through L2 and shared memory, twice the blocks in flight.
 //   keys  = blocks of 64, aligned to ABSOLUTE position, walked in ascending order from the first block any row of the
-//           tile can see to the last one.
+//           pair can see to the last one.
 //   TMEM  = [ O : d_head columns | S_0, S_1 : 64 columns each | Q : d_head / 2 columns ].  The query tile is written
 //           there once (two elements per 32-bit column) and is the A operand of S_j = Q K_j^T; the softmax threads
 //           read S_j (one row per thread, no shuffles) and hand its columns back at once; the weights P_j go to
 //           shared memory in the element type as the A operand of O += P_j V_j (tensor memory has no room for them
 //           beside two score buffers at d_head = 256, and scores that are free early let S run two blocks ahead).
 //   warps = 0-7 softmax and epilogue (two groups of four, TMEM lane quarter = warp % 4, alternating blocks), 8 issues
-//           the S products, 9 the PV products, 10-13 gather
-//           K/V blocks from the segments with 16-byte cp.async into the 128-byte-swizzled layouts the two products
-//           expect (K block: K-major B operand, rows = keys; V block: the same bytes read as an MN-major B operand,
-//           rows = the contraction index), a ring of K blocks and a ring of V blocks.  Positions no segment holds are
+//           the S products, 9 the PV products (in the pair's leading CTA only), 10-13 gather K/V blocks from the
+//           segments with 16-byte cp.async into the 128-byte-swizzled layouts the two products expect (K block:
+//           K-major B operand, rows = keys; V block: the same bytes read as an MN-major B operand, rows = the
+//           contraction index), a ring of K blocks and a ring of V blocks.  Positions no segment holds are
 //           zero-filled and masked.
 //   order = S_j is issued as soon as its K block has landed and the softmax threads have read S_{j-2} out of its
-//           columns, so the scores run up to two blocks ahead of the softmax; PV_j follows the softmax of block j.  The running
-//           maximum of a row changes rarely after its first blocks; O is rescaled in tensor memory only when a row of
-//           the warp needs it (the others multiply by exactly 1).
+//           columns, so the scores run up to two blocks ahead of the softmax; PV_j follows the softmax of block j.  O is
+//           rescaled in tensor memory only when a row of the warp moves its reference maximum (the others multiply by
+//           exactly 1), and a row moves it only when a block's maximum exceeds it by a factor of 256: with exact maxima
+//           some row of a 128-row tile moves in nearly every block, and rescale -> PV_j -> rescale is a serial chain.
 //
 // A row's result depends on that row alone: the rows of an MMA are computed independently, every row walks the key
-// blocks of its tile in ascending order, a block without a visible key for the row changes nothing for it (weights 0,
-// rescale by exactly 1, O += 0), and the block boundaries are absolute.  So a token attended alone and the same token
-// inside any tile give the same bits.  They are not the bits of kvd_decode_attention (another split of the keys, P
-// rounded before the second product).  Every wait is bounded: on a timeout the CTA raises the status word, all roles
-// leave their loops, and tensor memory is freed.
+// blocks in ascending order, a block without a visible key for the row changes nothing for it (weights 0, rescale by
+// exactly 1, O += 0), and the block boundaries are absolute.  So a token attended alone and the same token inside any
+// tile give the same bits.  They are not the bits of kvd_decode_attention (another split of the keys, P rounded before
+// the second product).  Every wait is bounded: on a timeout the CTA raises the status word, all roles leave their
+// loops, and tensor memory is freed.
 #include <math_constants.h>
-#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <type_traits>
 
 #include "kvd_internal.h"
 #include "kvd_ptx.cuh"
@@ -41,73 +49,98 @@ constexpr int PT_LOADERS = 128;  // threads of warps 10-13
 constexpr float PT_TAU = 8.0f;   // log2 of the largest weight a row may reach before its reference maximum moves
 constexpr int PT_LAG = 3;        // blocks a loader thread keeps in flight behind the one it is issuing
 
-template <int D_HEAD>
+template <int D_HEAD, bool PAIR>
 struct PtCfg {
-  static constexpr int TILE_BYTES = PT_KEYS * D_HEAD * 2;       // one K or V block
-  static constexpr int SLAB_BYTES = PT_KEYS * 128;              // 64 channels of every key of a block
-  static constexpr int SLOTS_K = D_HEAD == 256 ? 3 : 4;         // blocks in the K ring (the scores run ahead)
-  static constexpr int SLOTS_V = D_HEAD == 256 ? 2 : 4;         // blocks in the V ring
+  static constexpr int NCTA = PAIR ? 2 : 1;
+  static constexpr int K_ROWS = PT_KEYS / NCTA;                   // keys of a block this CTA holds
+  static constexpr int V_COLS = D_HEAD / NCTA;                    // channels of a block this CTA holds
+  static constexpr int TILE_BYTES = PT_KEYS * D_HEAD * 2 / NCTA;  // this CTA's share of one K or V block
+  static constexpr int SLAB_K = K_ROWS * 128;                     // 64 channels of this CTA's keys
+  static constexpr int SLAB_V = PT_KEYS * 128;                    // 64 of this CTA's channels of every key
+  static constexpr int SLOTS_K = D_HEAD == 256 ? (PAIR ? 6 : 3) : (PAIR ? 6 : 4);  // blocks in the K ring (the scores run ahead)
+  static constexpr int SLOTS_V = D_HEAD == 256 ? (PAIR ? 4 : 2) : (PAIR ? 6 : 4);  // blocks in the V ring
   static constexpr int SLOTS = SLOTS_K + SLOTS_V;
   static constexpr int COL_O = 0, COL_S = D_HEAD, COL_Q = D_HEAD + 2 * PT_KEYS;
   static constexpr int COLS_USED = COL_Q + D_HEAD / 2;
-  static constexpr int COLS = COLS_USED <= 256 ? 256 : 512;     // allocation: a power of two
-  static constexpr int P_BYTES = PT_ROWS * PT_KEYS * 2;        // one block of weights (K-major A operand of PV)
+  static constexpr int COLS = COLS_USED <= 256 ? 256 : 512;       // allocation: a power of two
+  static constexpr int P_BYTES = PT_ROWS * PT_KEYS * 2;           // one block of weights (K-major A operand of PV)
   static constexpr int N_BARS = 2 * SLOTS + 22;
   static constexpr int SMEM_BYTES = 1024 + SLOTS * TILE_BYTES + 2 * P_BYTES + N_BARS * 8;
 };
 
-#ifdef PT_EXP_TRACE
-__device__ long long pt_cta[8192][4];
-__device__ long long pt_trace[64][16];
-#define PT_STAMP(j, f) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (j) >= 32 && (j) < 96) pt_trace[(j) - 32][f] = clock64(); } while (0)
-#else
-#define PT_STAMP(j, f) do { } while (0)
-#endif
+// A wait of the MMA threads: in a pair the arrivals may come from the partner CTA and publish what its threads wrote
+// to its own shared memory, so the acquire is at cluster scope.
+template <bool PAIR>
+__device__ __forceinline__ bool lead_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag, unsigned long long timeout_ns) {
+  if constexpr (!PAIR) {
+    return mbar_wait(bar, parity, abort_flag, timeout_ns);
+  } else {
+#pragma unroll 1
+    for (int i = 0; i < 16; ++i)
+      if (mbar_try_wait_cluster(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    uint32_t it = 0;
+    while (!mbar_try_wait_cluster(bar, parity)) {
+      if (((++it) & 31u) == 0u && (*abort_flag != 0 || globaltimer_ns() - t0 > timeout_ns)) return false;
+    }
+    return true;
+  }
+}
 
-template <int D_HEAD, int G, int DT>
+template <int D_HEAD, int G, int DT, bool PAIR>
 __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(const __grid_constant__ PrefillParams P) {
-  using Cfg = PtCfg<D_HEAD>;
+  using Cfg = PtCfg<D_HEAD, PAIR>;
   constexpr int GP = G == 3 ? 4 : G;   // heads of the group, padded to a power of two
   constexpr int TOK = PT_ROWS / GP;    // query tokens per CTA
+  constexpr int NCTA = Cfg::NCTA;
   constexpr int SLOTS = Cfg::SLOTS, SLOTS_K = Cfg::SLOTS_K, SLOTS_V = Cfg::SLOTS_V;
   extern __shared__ uint8_t pt_smem_raw[];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort_i, s_lo, s_hi;
   __shared__ float s_mx[2][PT_ROWS], s_lx[2][PT_ROWS];  // per group: the row maximum after its last block, its part of the row sum
   volatile int *s_abort = &s_abort_i;
-  // the ring starts on a 1024-byte boundary (the swizzle is a function of the address), the barriers follow it
+  // the rings start on a 1024-byte boundary (the swizzle is a function of the address), the barriers follow them
   const uint32_t ring = (smem_u32(pt_smem_raw) + 1023u) & ~1023u;
   const uint32_t ring_v = ring + SLOTS_K * Cfg::TILE_BYTES;  // K blocks first, V blocks behind them
   const uint32_t p_smem = ring + SLOTS * Cfg::TILE_BYTES;    // two blocks of weights
   const uint32_t bar_base = p_smem + 2 * Cfg::P_BYTES;
-  auto bar_full = [&](int v, int s) { return bar_base + 8u * (v * SLOTS_K + s); };
-  auto bar_empty = [&](int v, int s) { return bar_base + 8u * (SLOTS + v * SLOTS_K + s); };
-  auto bar_s_full = [&](int b) { return bar_base + 8u * (2 * SLOTS + b); };
-  auto bar_p_ready = [&](int b) { return bar_base + 8u * (2 * SLOTS + 2 + b); };
-  auto bar_pv_done = [&](int b) { return bar_base + 8u * (2 * SLOTS + 4 + b); };
+  // barriers the MMA threads wait on are used in the leading CTA only; the others (MMA commits) in both
+  auto bar_full = [&](int v, int s) { return bar_base + 8u * (v * SLOTS_K + s); };           // leader: a block has landed
+  auto bar_empty = [&](int v, int s) { return bar_base + 8u * (SLOTS + v * SLOTS_K + s); };  // both: its product is done
+  auto bar_s_full = [&](int b) { return bar_base + 8u * (2 * SLOTS + b); };                  // both: scores of a block
+  auto bar_p_ready = [&](int b) { return bar_base + 8u * (2 * SLOTS + 2 + b); };             // leader: weights in place
+  auto bar_pv_done = [&](int b) { return bar_base + 8u * (2 * SLOTS + 4 + b); };             // both: O += P V finished
   const uint32_t bar_o_full = bar_base + 8u * (2 * SLOTS + 6), bar_q_ready = bar_base + 8u * (2 * SLOTS + 7);
-  auto bar_s_free = [&](int b) { return bar_base + 8u * (2 * SLOTS + 8 + b); };
-  auto bar_m = [&](int grp, int q) { return bar_base + 8u * (2 * SLOTS + 10 + grp * 4 + q); };  // a row maximum was handed over
-  auto bar_l = [&](int q) { return bar_base + 8u * (2 * SLOTS + 18 + q); };                     // both parts of the row sums
+  auto bar_s_free = [&](int b) { return bar_base + 8u * (2 * SLOTS + 8 + b); };              // leader: scores were read
+  auto bar_m = [&](int grp, int q) { return bar_base + 8u * (2 * SLOTS + 10 + grp * 4 + q); };  // own: a row maximum was handed over
+  auto bar_l = [&](int q) { return bar_base + 8u * (2 * SLOTS + 18 + q); };                     // own: both parts of the row sums
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-#ifdef PT_EXP_TRACE
-  if (tid == 0 && blockIdx.y * gridDim.x + blockIdx.x < 8192) pt_cta[blockIdx.y * gridDim.x + blockIdx.x][0] = globaltimer_ns();
-#endif
-  // long tiles (late tokens of a causal call) first
-  const int tok0 = (static_cast<int>(gridDim.x) - 1 - static_cast<int>(blockIdx.x)) * TOK, kvh = blockIdx.y;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+  // long tiles (late tokens of a causal call) first; the CTAs of a pair have neighbouring tiles
+  const int tile = static_cast<int>(gridDim.x) - 1 - static_cast<int>(blockIdx.x);
+  const int tok0 = tile * TOK, kvh = blockIdx.y;
+  const int pair_tok0 = PAIR ? (tile & ~1) * TOK : tok0;  // the grid is even: tiles 2c and 2c + 1 share a cluster
   const unsigned long long tmo = P.timeout_ns;
+  // An arrival of one warp on a barrier of the leading CTA.  Across the pair it is a relaxed arrive: what it announces
+  // (scores read out of tensor memory; weights or K/V pieces written to this CTA's own shared memory) has been
+  // completed and fenced for the tensor cores' proxy by the announcing threads before they get here, and a
+  // cluster-scope release would make the warp wait for every outstanding memory operation of a busy SM.
+  auto arrive_lead = [&](uint32_t bar) {
+    if (!PAIR || rank == 0) mbar_arrive(bar);
+    else mbar_arrive_cluster(map_to_cta(bar, 0));
+  };
 
   if (tid == 0) {
     for (int s = 0; s < SLOTS; ++s) {
-      mbar_init(bar_full(0, s), 4);   // one arrival per loader warp
-      mbar_init(bar_empty(0, s), 1);  // the MMA commit
+      mbar_init(bar_full(0, s), 4 * NCTA);  // one arrival per loader warp of the pair
+      mbar_init(bar_empty(0, s), 1);        // the MMA commit
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(bar_s_full(b), 1);    // the MMA commit
-      mbar_init(bar_p_ready(b), 4);   // one arrival per softmax warp of the group
+      mbar_init(bar_s_full(b), 1);          // the MMA commit
+      mbar_init(bar_p_ready(b), 4 * NCTA);  // one arrival per softmax warp of the group, in both CTAs
       mbar_init(bar_pv_done(b), 1);
-      mbar_init(bar_s_free(b), 4);    // one arrival per softmax warp
+      mbar_init(bar_s_free(b), 4 * NCTA);   // the same
     }
     for (int q = 0; q < 4; ++q) {
       mbar_init(bar_m(0, q), 1);  // the warp of the group that owns these 32 rows
@@ -115,20 +148,25 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       mbar_init(bar_l(q), 2);     // that warp of either group
     }
     mbar_init(bar_o_full, 1);
-    mbar_init(bar_q_ready, 8);
+    mbar_init(bar_q_ready, 8 * NCTA);
     fence_mbar_init();
     s_abort_i = 0;
     s_lo = INT_MAX;
     s_hi = -1;
   }
   if (warp == 8) {
-    tmem_alloc(smem_u32(&s_tmem), Cfg::COLS);
-    tmem_relinquish();
+    if constexpr (PAIR) {
+      tmem_alloc_pair(smem_u32(&s_tmem), Cfg::COLS);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(smem_u32(&s_tmem), Cfg::COLS);
+      tmem_relinquish();
+    }
   }
   __syncthreads();
-  // ---- key positions the tile needs: from the smallest first-visible to the largest last-visible of its tokens
-  if (tid < TOK && tok0 + tid < P.n_rows) {
-    const int qp = P.q_pos[tok0 + tid];
+  // ---- key positions the pair needs: from the smallest first-visible to the largest last-visible of its tokens
+  if (tid < NCTA * TOK && pair_tok0 + tid < P.n_rows) {
+    const int qp = P.q_pos[pair_tok0 + tid];
     int lo = P.window > 0 ? qp - P.window + 1 : 0;
     lo = lo < P.seg_lo ? P.seg_lo : lo;
     const int hi = qp < P.seg_hi ? qp : P.seg_hi;
@@ -138,7 +176,8 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
     }
   }
   tc_fence_before();
-  __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();  // barriers of both CTAs are initialised before anyone signals across the pair
+  else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = s_tmem;
   const int blk0 = s_hi >= 0 ? s_lo / PT_KEYS : 0;
@@ -176,7 +215,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_q_ready);
+      if (lane == 0) arrive_lead(bar_q_ready);
     }
     float m_own = -CUDART_INF_F;    // the maximum this group's part of the row sum refers to
     uint64_t l2[2] = {0ull, 0ull};  // that part, in four chains (two packed pairs)
@@ -191,7 +230,6 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
         break;
       }
       tc_fence_after();
-      if ((tid & 127) == 0) PT_STAMP(j, 0);
       const uint32_t s_col = tmem_base + lane_field + Cfg::COL_S + buf * PT_KEYS;
       uint32_t s0[32], s1[32];
       tmem_ld_x32(s_col, s0);
@@ -216,8 +254,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       // the scores are in registers: their columns may take this group's next block
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_s_free(buf));
-      if ((tid & 127) == 0) PT_STAMP(j, 1);
+      if (lane == 0) arrive_lead(bar_s_free(buf));
       if (!__all_sync(0xffffffffu, vis == ~0ull)) {
         const uint32_t v0 = static_cast<uint32_t>(vis), v1 = static_cast<uint32_t>(vis >> 32);
 #pragma unroll
@@ -258,7 +295,6 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       s_mx[wg][row] = m_new;
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_m(wg, q4));
-      if ((tid & 127) == 0) PT_STAMP(j, 4);
       const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;
       // rescale of what the row has so far: exactly 1 when its maximum stays; while nothing has been seen O and l are 0
       const float alpha = m_prev == -CUDART_INF_F ? 1.0f : ex2_approx(m_prev - m_use);
@@ -286,7 +322,6 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
         w[16 + (k >> 1)] = pack_out<DT>(p0, p1);
         l2[(k >> 1) & 1] = ffma2(pack2(p0, p1), one2, l2[(k >> 1) & 1]);
       }
-      if ((tid & 127) == 0) PT_STAMP(j, 2);
       // P_j into shared memory as a K-major A operand (row = MMA row, 128 bytes = 64 keys, 128-byte swizzle); the
       // product that read this buffer two blocks ago has long finished
       if (j >= 2 && !warp_wait(bar_pv_done(buf), ((j - 2) >> 1) & 1, s_abort, tmo, lane)) {
@@ -303,7 +338,6 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
                        : "memory");
         fence_proxy_async_smem();
       }
-      if ((tid & 127) == 0) PT_STAMP(j, 8);
       if (__any_sync(0xffffffffu, alpha != 1.0f)) {
         // O holds the blocks before j; the last of those products must have finished (j >= 1 here: a maximum exists)
         if (!warp_wait(bar_pv_done(buf ^ 1), ((j - 1) >> 1) & 1, s_abort, tmo, lane)) {
@@ -325,8 +359,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
         tc_fence_before();
       }
       __syncwarp();
-      if ((tid & 127) == 0) PT_STAMP(j, 3);
-      if (lane == 0) mbar_arrive(bar_p_ready(buf));
+      if (lane == 0) arrive_lead(bar_p_ready(buf));
     }
     // ---- the row sum: both parts referred to the final maximum, added in group order
     float l_run = 0.f;
@@ -385,80 +418,75 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       }
     }
   } else if (warp == 8 || warp == 9) {
-    // ------------------------------------------------------------------ MMA issue (one thread per product)
-    constexpr uint32_t IDESC_BASE = DT == 0 ? umma_idesc_bf16_f32(PT_ROWS, 8) & ~(1u << 17) : umma_idesc_f16_f32(PT_ROWS, 8) & ~(1u << 17);
+    // ------------------------------------------------------------------ MMA issue (one thread per product, leading CTA)
+    constexpr uint32_t IDESC_BASE = (DT == 0 ? umma_idesc_bf16_f32(PT_ROWS * NCTA, 8) : umma_idesc_f16_f32(PT_ROWS * NCTA, 8)) & ~(1u << 17);
     constexpr uint32_t IDESC_S = IDESC_BASE | (static_cast<uint32_t>(PT_KEYS >> 3) << 17);              // N = 64 keys, B K-major
     constexpr uint32_t IDESC_O = IDESC_BASE | (static_cast<uint32_t>(D_HEAD >> 3) << 17) | (1u << 16);  // N = d_head, B MN-major
-    if (lane == 0 && n_blk > 0 && warp == 8) {
+    auto commit = [&](uint32_t bar) {
+      if constexpr (PAIR) umma_commit_pair(bar, 3);  // the barrier at this offset in both CTAs
+      else umma_commit(bar);
+    };
+    if (lane == 0 && n_blk > 0 && rank == 0 && warp == 8) {
       // S_j = Q K_j^T into score buffer j & 1, as far ahead of the softmax as the two buffers allow
-      bool ok = mbar_wait(bar_q_ready, 0, s_abort, tmo);
+      bool ok = lead_wait<PAIR>(bar_q_ready, 0, s_abort, tmo);
       tc_fence_after();
       for (int j = 0; ok && j < n_blk; ++j) {
         const int slot = j % SLOTS_K;
-        PT_STAMP(j, 9);
         // the K block has landed; the softmax threads have read the scores of block j - 2 out of these columns
-        if (!mbar_wait(bar_full(0, slot), (j / SLOTS_K) & 1, s_abort, tmo) ||
-            (j >= 2 && !mbar_wait(bar_s_free(j & 1), ((j - 2) >> 1) & 1, s_abort, tmo))) {
+        if (!lead_wait<PAIR>(bar_full(0, slot), (j / SLOTS_K) & 1, s_abort, tmo) ||
+            (j >= 2 && !lead_wait<PAIR>(bar_s_free(j & 1), ((j - 2) >> 1) & 1, s_abort, tmo))) {
           ok = false;
           break;
         }
         tc_fence_after();
-        PT_STAMP(j, 10);
-        const uint32_t kb = ring + slot * Cfg::TILE_BYTES;
         const uint32_t d = tmem_base + Cfg::COL_S + (j & 1) * PT_KEYS;
-        const uint64_t desc0 = umma_smem_desc_sw128(kb);
+        const uint64_t desc0 = umma_smem_desc_sw128(ring + slot * Cfg::TILE_BYTES);
 #pragma unroll
-        for (int ks = 0; ks < D_HEAD / 16; ++ks)
-          umma_f16_ts(d, tmem_base + Cfg::COL_Q + ks * 8, desc0 + (((ks >> 2) * Cfg::SLAB_BYTES + (ks & 3) * 32) >> 4), IDESC_S,
-                      ks > 0 ? 1u : 0u);
-        umma_commit(bar_empty(0, slot));
-        umma_commit(bar_s_full(j & 1));
-        PT_STAMP(j, 5);
+        for (int ks = 0; ks < D_HEAD / 16; ++ks) {
+          const uint64_t bdesc = desc0 + (((ks >> 2) * Cfg::SLAB_K + (ks & 3) * 32) >> 4);
+          if constexpr (PAIR) umma_f16_ts_pair(d, tmem_base + Cfg::COL_Q + ks * 8, bdesc, IDESC_S, ks > 0 ? 1u : 0u);
+          else umma_f16_ts(d, tmem_base + Cfg::COL_Q + ks * 8, bdesc, IDESC_S, ks > 0 ? 1u : 0u);
+        }
+        commit(bar_empty(0, slot));
+        commit(bar_s_full(j & 1));
       }
       if (!ok) raise(P.status, STATUS_TIMEOUT, s_abort);
-    } else if (lane == 0 && n_blk > 0) {
-      // O += P_j V_j once the weights are in place (and O has been rescaled where a maximum moved)
+    } else if (lane == 0 && n_blk > 0 && rank == 0) {
+      // O += P_j V_j once the weights are in place (and O has been rescaled where a reference maximum moved)
       bool ok = true;
       for (int j = 0; j < n_blk; ++j) {
         const int slot = j % SLOTS_V;
-        if (!mbar_wait(bar_p_ready(j & 1), (j >> 1) & 1, s_abort, tmo) || !mbar_wait(bar_full(1, slot), (j / SLOTS_V) & 1, s_abort, tmo)) {
+        if (!lead_wait<PAIR>(bar_p_ready(j & 1), (j >> 1) & 1, s_abort, tmo) ||
+            !lead_wait<PAIR>(bar_full(1, slot), (j / SLOTS_V) & 1, s_abort, tmo)) {
           ok = false;
           break;
         }
         tc_fence_after();
-        PT_STAMP(j, 6);
-        const uint64_t desc0 = umma_smem_desc_sw128_mn(ring_v + slot * Cfg::TILE_BYTES, Cfg::SLAB_BYTES);
+        const uint64_t desc0 = umma_smem_desc_sw128_mn(ring_v + slot * Cfg::TILE_BYTES, Cfg::SLAB_V);
         const uint64_t pdesc0 = umma_smem_desc_sw128(p_smem + (j & 1) * Cfg::P_BYTES);
 #pragma unroll
-        for (int ks = 0; ks < PT_KEYS / 16; ++ks)
-          umma_bf16(tmem_base + Cfg::COL_O, pdesc0 + ((ks * 32) >> 4), desc0 + ((ks * 16 * 128) >> 4), IDESC_O,
-                    (j > 0 || ks > 0) ? 1u : 0u);
-        umma_commit(bar_empty(1, slot));
-        umma_commit(bar_pv_done(j & 1));
-        PT_STAMP(j, 7);
+        for (int ks = 0; ks < PT_KEYS / 16; ++ks) {
+          if constexpr (PAIR) umma_bf16_pair(tmem_base + Cfg::COL_O, pdesc0 + ((ks * 32) >> 4), desc0 + ((ks * 16 * 128) >> 4), IDESC_O,
+                                             (j > 0 || ks > 0) ? 1u : 0u);
+          else umma_bf16(tmem_base + Cfg::COL_O, pdesc0 + ((ks * 32) >> 4), desc0 + ((ks * 16 * 128) >> 4), IDESC_O,
+                         (j > 0 || ks > 0) ? 1u : 0u);
+        }
+        commit(bar_empty(1, slot));
+        commit(bar_pv_done(j & 1));
       }
-      if (ok) umma_commit(bar_o_full);
+      if (ok) commit(bar_o_full);
       else raise(P.status, STATUS_TIMEOUT, s_abort);
     }
   } else {
     // ------------------------------------------------------------------ K/V blocks into the rings
     // issue order = the order the products want them, the keys two blocks ahead: K_0 K_1 | K_2 V_0 | K_3 V_1 | ...
-    constexpr int CPR = D_HEAD / 8;           // 16-byte pieces per key
-    constexpr int RSTEP = PT_LOADERS / CPR;   // keys one pass of the 128 threads covers
+    // This CTA's share of a block: K_ROWS keys of all channels (K), all 64 keys of V_COLS channels (V).
     const int ptid = tid - 10 * 32;
-    const int c = ptid % CPR, r0 = ptid / CPR;
-    const uint32_t dst_c = static_cast<uint32_t>(c >> 3) * Cfg::SLAB_BYTES;
     // blocks issued and not yet published to the MMA threads, oldest first.  A block is published once PT_LAG younger
     // ones have been issued -- or at once, all of them, when the next block would have to wait for a free slot (the
     // slot is freed by a product that may itself be waiting for one of these blocks).
     uint32_t pend[PT_LAG + 1] = {};
     int n_pend = 0;
-#ifdef PT_EXP_TRACE
-    int ptag[PT_LAG + 1] = {};
-#define PT_PUB(i) do { if (ptid == 0) PT_STAMP(ptag[i] % 1000, ptag[i] >= 1000 ? 15 : 13); } while (0)
-#else
-#define PT_PUB(i) do { } while (0)
-#endif
     bool ok = true;
     auto publish_all = [&]() {
       cp_async_wait_all();
@@ -466,11 +494,47 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       __syncwarp();
 #pragma unroll
       for (int i = 0; i <= PT_LAG; ++i)
-        if (i < n_pend && lane == 0) {
-          mbar_arrive(pend[i]);
-          PT_PUB(i);
-        }
+        if (i < n_pend && lane == 0) arrive_lead(pend[i]);
       n_pend = 0;
+    };
+    // rows [row_first, row_first + ROWS) of the block, CPR 16-byte pieces of each starting at element col_first
+    auto gather = [&](auto rows_c, auto cpr_c, uint32_t base, int slab_bytes, int pos_first, int col_first, bool is_v) {
+      constexpr int ROWS = decltype(rows_c)::value, CPR = decltype(cpr_c)::value;
+      constexpr int RSTEP = PT_LOADERS / CPR;  // rows one pass of the 128 threads covers
+      const int c = ptid % CPR, r0 = ptid / CPR;
+      const uint32_t dst = base + static_cast<uint32_t>(c >> 3) * slab_bytes;
+      // the usual case: one segment holds all the rows -> one base pointer, one stride
+      int whole = -1;
+#pragma unroll
+      for (int sg = 0; sg < KVD_MAX_SEGMENTS; ++sg)
+        if (P.first[sg] <= pos_first && pos_first + ROWS <= P.first[sg] + P.len[sg]) whole = sg;
+      if (whole >= 0) {
+        const long long stride = P.stride[whole];
+        const __nv_bfloat16 *src = (is_v ? P.v[whole] : P.k[whole]) + static_cast<size_t>(pos_first - P.first[whole] + r0) * stride +
+                                   static_cast<size_t>(kvh) * D_HEAD + col_first + c * 8;
+#pragma unroll
+        for (int pass = 0; pass < ROWS / RSTEP; ++pass) {
+          const int r = r0 + pass * RSTEP;
+          cp_async16(dst + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, true);
+          src += RSTEP * stride;
+        }
+      } else {
+#pragma unroll 1
+        for (int pass = 0; pass < ROWS / RSTEP; ++pass) {
+          const int r = r0 + pass * RSTEP, pos = pos_first + r;
+          const __nv_bfloat16 *src = P.q;
+          bool have = false;
+#pragma unroll
+          for (int sg = 0; sg < KVD_MAX_SEGMENTS; ++sg) {
+            const int rr = pos - P.first[sg];
+            if (rr >= 0 && rr < P.len[sg]) {
+              src = (is_v ? P.v[sg] : P.k[sg]) + static_cast<size_t>(rr) * P.stride[sg] + static_cast<size_t>(kvh) * D_HEAD + col_first + c * 8;
+              have = true;
+            }
+          }
+          cp_async16(dst + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, have);
+        }
+      }
     };
     auto emit = [&](int is_v, int j) -> bool {
       const int n_slots = is_v ? SLOTS_V : SLOTS_K, slot = j % n_slots;
@@ -483,65 +547,26 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
           if (!warp_wait(bar_empty(is_v, slot), par, s_abort, tmo, lane)) return false;
         }
       }
-      if (ptid == 0) PT_STAMP(j, is_v ? 14 : 12);
       const int pos0 = (blk0 + j) * PT_KEYS;
-      const uint32_t base = (is_v ? ring_v : ring) + slot * Cfg::TILE_BYTES + dst_c;
-      // the usual case: one segment holds the whole block -> one base pointer, one stride
-      int whole = -1;
-#pragma unroll
-      for (int sg = 0; sg < KVD_MAX_SEGMENTS; ++sg)
-        if (P.first[sg] <= pos0 && pos0 + PT_KEYS <= P.first[sg] + P.len[sg]) whole = sg;
-      if (whole >= 0) {
-        const long long stride = P.stride[whole];
-        const __nv_bfloat16 *src = (is_v ? P.v[whole] : P.k[whole]) + static_cast<size_t>(pos0 - P.first[whole] + r0) * stride +
-                                   static_cast<size_t>(kvh) * D_HEAD + c * 8;
-#pragma unroll
-        for (int pass = 0; pass < PT_KEYS / RSTEP; ++pass) {
-          const int r = r0 + pass * RSTEP;
-          cp_async16(base + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, true);
-          src += RSTEP * stride;
-        }
-      } else {
-#pragma unroll 1
-        for (int pass = 0; pass < PT_KEYS / RSTEP; ++pass) {
-          const int r = r0 + pass * RSTEP, pos = pos0 + r;
-          const __nv_bfloat16 *src = P.q;
-          bool have = false;
-#pragma unroll
-          for (int sg = 0; sg < KVD_MAX_SEGMENTS; ++sg) {
-            const int rr = pos - P.first[sg];
-            if (rr >= 0 && rr < P.len[sg]) {
-              src = (is_v ? P.v[sg] : P.k[sg]) + static_cast<size_t>(rr) * P.stride[sg] + static_cast<size_t>(kvh) * D_HEAD + c * 8;
-              have = true;
-            }
-          }
-          cp_async16(base + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, have);
-        }
-      }
+      if (is_v)
+        gather(std::integral_constant<int, PT_KEYS>(), std::integral_constant<int, Cfg::V_COLS / 8>(), ring_v + slot * Cfg::TILE_BYTES,
+               Cfg::SLAB_V, pos0, static_cast<int>(rank) * Cfg::V_COLS, true);
+      else
+        gather(std::integral_constant<int, Cfg::K_ROWS>(), std::integral_constant<int, D_HEAD / 8>(), ring + slot * Cfg::TILE_BYTES,
+               Cfg::SLAB_K, pos0 + static_cast<int>(rank) * Cfg::K_ROWS, 0, false);
       cp_async_commit();
 #pragma unroll
       for (int i = 0; i <= PT_LAG; ++i)
-        if (i == n_pend) {
-          pend[i] = bar_full(is_v, slot);
-#ifdef PT_EXP_TRACE
-          ptag[i] = is_v * 1000 + j;
-#endif
-        }
+        if (i == n_pend) pend[i] = bar_full(is_v, slot);
       ++n_pend;
       if (n_pend > PT_LAG) {
         // the oldest block has PT_LAG younger ones behind it: it has landed by now, or nearly
         cp_async_wait_group<PT_LAG>();
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(pend[0]);
-        PT_PUB(0);
+        if (lane == 0) arrive_lead(pend[0]);
 #pragma unroll
-        for (int i = 0; i < PT_LAG; ++i) {
-          pend[i] = pend[i + 1];
-#ifdef PT_EXP_TRACE
-          ptag[i] = ptag[i + 1];
-#endif
-        }
+        for (int i = 0; i < PT_LAG; ++i) pend[i] = pend[i + 1];
         --n_pend;
       }
       return true;
@@ -561,33 +586,24 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
     }
   }
 
-  // ---- teardown: every role is done with tensor memory
+  // ---- teardown: every role is done with tensor memory; in a pair nobody leaves while the partner can still signal
+  // into this CTA's shared memory
   tc_fence_before();
-  __syncthreads();
-#ifdef PT_EXP_TRACE
-  if (tid == 0) {
-    const int id = blockIdx.y * gridDim.x + blockIdx.x;
-    if (id < 8192) {
-      unsigned smid;
-      asm("mov.u32 %0, %%smid;" : "=r"(smid));
-      pt_cta[id][1] = globaltimer_ns();
-      pt_cta[id][2] = n_blk;
-      pt_cta[id][3] = smid;
-    }
-  }
-#endif
+  if constexpr (PAIR) cluster_sync_all();
+  else __syncthreads();
   if (warp == 8) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, Cfg::COLS);
+    if constexpr (PAIR) tmem_dealloc_pair(tmem_base, Cfg::COLS);
+    else tmem_dealloc(tmem_base, Cfg::COLS);
   }
 }
 
-template <int D_HEAD, int G>
+template <int D_HEAD, int G, bool PAIR>
 static kvd_status prefill_tc_launch(kvd_ctx *ctx, const PrefillParams &P, cudaStream_t stream) {
-  using Cfg = PtCfg<D_HEAD>;
+  using Cfg = PtCfg<D_HEAD, PAIR>;
   constexpr int GP = G == 3 ? 4 : G;
-  auto k0 = kvd_prefill_attn_tc_kernel<D_HEAD, G, 0>;
-  auto k1 = kvd_prefill_attn_tc_kernel<D_HEAD, G, 1>;
+  auto k0 = kvd_prefill_attn_tc_kernel<D_HEAD, G, 0, PAIR>;
+  auto k1 = kvd_prefill_attn_tc_kernel<D_HEAD, G, 1, PAIR>;
   static bool configured[64] = {};
   if (!configured[ctx->device & 63]) {
     cudaError_t e = cudaFuncSetAttribute(k0, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
@@ -596,58 +612,51 @@ static kvd_status prefill_tc_launch(kvd_ctx *ctx, const PrefillParams &P, cudaSt
     configured[ctx->device & 63] = true;
   }
   const int tok = PT_ROWS / GP;
-  dim3 grid((P.n_rows + tok - 1) / tok, P.n_kv, 1);
-  if (ctx->dtype == 1) k1<<<grid, PT_THREADS, Cfg::SMEM_BYTES, stream>>>(P);
-  else k0<<<grid, PT_THREADS, Cfg::SMEM_BYTES, stream>>>(P);
-  cudaError_t e = cudaGetLastError();
+  int tiles = (P.n_rows + tok - 1) / tok;
+  if (PAIR) tiles = (tiles + 1) & ~1;  // whole pairs: a CTA whose tile lies past the last row has no rows to store
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(tiles, P.n_kv, 1);
+  cfg.blockDim = dim3(PT_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = ctx->dtype == 1 ? cudaLaunchKernelEx(&cfg, k1, P) : cudaLaunchKernelEx(&cfg, k0, P);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "launch prefill attention");
-#ifdef PT_EXP_TRACE
-  {
-    static int printed = 0;
-    if (!printed && grid.x > 200) {
-      printed = 1;
-      cudaDeviceSynchronize();
-      static long long h[64][16];
-      cudaMemcpyFromSymbol(h, pt_trace, sizeof(h));
-      {
-        static long long c[8192][4];
-        cudaMemcpyFromSymbol(c, pt_cta, sizeof(c));
-        const int n = grid.x * grid.y < 8192 ? grid.x * grid.y : 8192;
-        long long t0 = c[0][0], t1 = 0, busy[256] = {}, blocks[256] = {}, ctas[256] = {};
-        for (int i = 0; i < n; ++i) { if (c[i][0] < t0) t0 = c[i][0]; if (c[i][1] > t1) t1 = c[i][1]; }
-        double per_blk_sum = 0; int per_blk_n = 0;
-        for (int i = 0; i < n; ++i) {
-          const int sm = (int)c[i][3] & 255;
-          busy[sm] += c[i][1] - c[i][0]; blocks[sm] += c[i][2]; ctas[sm] += 1;
-          if (c[i][2] >= 64) { per_blk_sum += double(c[i][1] - c[i][0]) / c[i][2]; ++per_blk_n; }
-        }
-        fprintf(stderr, "kernel span %lld ns; ns per block over CTAs with >= 64 blocks: %.1f\n", t1 - t0, per_blk_sum / per_blk_n);
-        for (int sm = 0; sm < 148; sm += 21) fprintf(stderr, "  sm %3d: ctas %lld blocks %lld busy %lld ns\n", sm, ctas[sm], blocks[sm], busy[sm]);
-        long long bmin = 1ll << 60, bmax = 0, kmin = 1ll << 60, kmax = 0;
-        for (int sm = 0; sm < 148; ++sm) { if (busy[sm] < bmin) bmin = busy[sm]; if (busy[sm] > bmax) bmax = busy[sm]; if (blocks[sm] < kmin) kmin = blocks[sm]; if (blocks[sm] > kmax) kmax = blocks[sm]; }
-        fprintf(stderr, "  busy ns min %lld max %lld; blocks min %lld max %lld\n", bmin, bmax, kmin, kmax);
-        for (int i = 0; i < n; i += n / 16) fprintf(stderr, "  cta %4d: start %8lld dur %8lld blk %3lld sm %3lld  ns/blk %.1f\n", i, c[i][0] - t0, c[i][1] - c[i][0], c[i][2], c[i][3], c[i][2] ? double(c[i][1] - c[i][0]) / c[i][2] : 0.0);
-      }
-      for (int j = 0; j < 8; ++j) {
-        fprintf(stderr, "blk %3d:", j + 32);
-        for (int f = 0; f < 16; ++f) fprintf(stderr, " %7lld", h[j][f] ? h[j][f] - h[0][0] : -1);
-        fprintf(stderr, "\n");
-      }
-    }
-  }
-#endif
   ctx->launches += 1;
   return KVD_OK;
 }
 
 template <int D_HEAD>
 static kvd_status prefill_tc_group(kvd_ctx *ctx, const PrefillParams &P, int group, cudaStream_t stream) {
+  // pairs where the K/V bytes per block bound the kernel (d_head = 256); at 128 the softmax does, and the hand-overs
+  // across the pair cost more than the halved traffic returns (measured).  KVD_PREFILL_PAIR=0/1 overrides, for comparisons.
+  static const char *env = getenv("KVD_PREFILL_PAIR");
+  const bool pair = D_HEAD >= 128 && (env ? env[0] == '1' : D_HEAD == 256);
+  if constexpr (D_HEAD >= 128) {
+    if (pair) {
+      switch (group) {
+        case 1: return prefill_tc_launch<D_HEAD, 1, true>(ctx, P, stream);
+        case 2: return prefill_tc_launch<D_HEAD, 2, true>(ctx, P, stream);
+        case 3: return prefill_tc_launch<D_HEAD, 3, true>(ctx, P, stream);
+        case 4: return prefill_tc_launch<D_HEAD, 4, true>(ctx, P, stream);
+        case 8: return prefill_tc_launch<D_HEAD, 8, true>(ctx, P, stream);
+        default: return KVD_ERR_SHAPE;
+      }
+    }
+  }
   switch (group) {
-    case 1: return prefill_tc_launch<D_HEAD, 1>(ctx, P, stream);
-    case 2: return prefill_tc_launch<D_HEAD, 2>(ctx, P, stream);
-    case 3: return prefill_tc_launch<D_HEAD, 3>(ctx, P, stream);
-    case 4: return prefill_tc_launch<D_HEAD, 4>(ctx, P, stream);
-    case 8: return prefill_tc_launch<D_HEAD, 8>(ctx, P, stream);
+    case 1: return prefill_tc_launch<D_HEAD, 1, false>(ctx, P, stream);
+    case 2: return prefill_tc_launch<D_HEAD, 2, false>(ctx, P, stream);
+    case 3: return prefill_tc_launch<D_HEAD, 3, false>(ctx, P, stream);
+    case 4: return prefill_tc_launch<D_HEAD, 4, false>(ctx, P, stream);
+    case 8: return prefill_tc_launch<D_HEAD, 8, false>(ctx, P, stream);
     default: return KVD_ERR_SHAPE;
   }
 }
