@@ -483,6 +483,9 @@ def run_gpu(args):
                 torch.cuda.synchronize()
                 return 1.0  # not a measurement
             measure_long_attention(wl, peaks, eager)
+        if args.profile_prefill_attn:
+            # a few causal prefill-attention calls over 4096 tokens of the layer
+            measure_prefill_attention(wl, peaks, lengths=(4096,))
         if rank == 0:
             print(json.dumps({"profile_run": True, "steps": steps, "launches": wl.ctx.kvd_launch_count()}))
         return
@@ -690,6 +693,7 @@ def run_gpu(args):
     d2h = out_pin.numel() * 2
 
     long_attn = measure_long_attention(wl, peaks, timed_graph) if rank == 0 else None
+    prefill_attn = measure_prefill_attention(wl, peaks) if rank == 0 else None
     stack_decode = None
     if rank == 0 and world == 1 and not args.no_stack:
         stack_decode = measure_stack_decode((1, 4, 16, 64) if args.stack_all else (1, 4),
@@ -762,6 +766,7 @@ def run_gpu(args):
                                    "avg_us": attn_ms * 1e3, "in_step_us": float(np.mean(t_attn)) * 1e3,
                                    "note": "16.8 MB per call: launch-latency bound; see attention_long"},
             "attention_long": long_attn,
+            "prefill_attention": prefill_attn,
             "decode_step_us": {"total": ms_per_step * 1e3,
                                "isolated": {k: v * 1e3 for k, v in iso_ms.items()},
                                "in_step_with_event_nodes": {"checkpoint": float(np.mean(t_ckpt)) * 1e3,
@@ -915,6 +920,46 @@ def measure_long_attention(wl, peaks, timed_graph, T=32768):
             "bound": "hbm", "kernel": "kvd_attn_split_kernel<256,2,4>",
             "frac_of_datasheet": byts / (ms * 1e-3) / 1e9 / DATASHEET_HBM_GBS,
             **({"traffic": tr["bytes"], "traffic_source": tr["source"]} if T == 32768 else {"traffic": None})}
+
+
+def measure_prefill_attention(wl, peaks, lengths=(4096, 16384)):
+    """kvd_prefill_attention: causal attention of T tokens of one sequence to themselves (a prefill, or the replay of
+    an evicted prefix when one residual row per token is kept), one launch of the tcgen05 kernel.  Flops are the causal
+    ones, 4 * n_q * d_head per (query, visible key) pair; the peak is the measured bf16 burst figure."""
+    import torch
+    import paper_2603_19664_b200 as kvd
+    shape, kdim = wl.shape, wl.kdim
+    out = {"kernel": "kvd_prefill_attn_tc_kernel<256,2> (CTA pairs, tcgen05.mma.cta_group::2, scores and output in tensor memory)",
+           "bound": "tensor", "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "cases": []}
+    for T in lengths:
+        desc = kvd.make_desc(1, shape.d_hidden, shape.n_q_heads, shape.n_kv_heads, shape.d_head, shape.rms_eps,
+                             shape.qk_norm, shape.rms_eps, shape.rope_style, 1, T + 8, 1)
+        ctx = kvd.Kvd(desc)
+        ctx.kvd_set_layer(0, wl.w_kv, wl.g_in, wl.g_k, shape.rope_theta, 0)
+        gen = torch.Generator(device="cuda").manual_seed(7)
+        K = torch.randn((T, kdim), device="cuda", generator=gen).to(torch.bfloat16)
+        V = torch.randn((T, kdim), device="cuda", generator=gen).to(torch.bfloat16)
+        q = torch.randn((T, shape.n_q_heads, shape.d_head), device="cuda", generator=gen).to(torch.bfloat16)
+        o = torch.empty_like(q)
+        qp = torch.arange(T, dtype=torch.int32, device="cuda")
+        for _ in range(3):
+            ctx.kvd_prefill_attention(0, T, q, qp, [(K, V, kdim, 0, T)], 0.0, o)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 20
+        a.record()
+        for _ in range(reps):
+            ctx.kvd_prefill_attention(0, T, q, qp, [(K, V, kdim, 0, T)], 0.0, o)
+        b.record()
+        torch.cuda.synchronize()
+        if ctx.kvd_poll_status() != kvd.KVD_OK:
+            raise RuntimeError("device status after prefill attention")
+        us = a.elapsed_time(b) * 1e3 / reps
+        flops = 4.0 * (T * (T + 1) / 2) * shape.n_q_heads * shape.d_head
+        out["cases"].append({"tokens": T, "avg_us": us, "achieved": flops / us * 1e-6,
+                             "frac": flops / us * 1e-6 / peaks["bf16_tflops"], "causal_gflop": flops * 1e-9})
+        ctx.close()
+    return out
 
 
 def run_sweep(wl, peaks):
@@ -1304,6 +1349,8 @@ def main():
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--sets", type=int, default=N_SETS, help="rotating buffer sets (each ~59 MB)")
     ap.add_argument("--profile", action="store_true", help="eager launches only, for a run under a profiler")
+    ap.add_argument("--profile-prefill-attn", action="store_true",
+                    help="with --profile: also launch kvd_prefill_attention over 4096 tokens a few times")
     ap.add_argument("--profile-long-attn", action="store_true",
                     help="with --profile: also run decode attention over 32769 keys a few times")
     ap.add_argument("--profile-qwen", action="store_true",

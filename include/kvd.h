@@ -373,7 +373,10 @@ kvd_status kvd_decode_attention_rows(kvd_ctx *ctx, int layer, int n_rows, const 
 /* ATTENTION of Algorithm 1 (Eq. 6-7) for many tokens of one sequence in ONE launch, tiled over query rows on the
  * tensor cores: the prefill-shaped call.  Arguments as kvd_decode_attention_rows, except that q_pos is a DEVICE
  * int32 [n_rows] (nothing on the host depends on the positions).  Keys are taken in blocks of 64 aligned to absolute
- * position; the softmax weights are rounded to the element type before the second product (fp32 accumulation).
+ * position; the softmax weights are rounded to the element type before the second product (fp32 accumulation); a
+ * row's weights are taken against a reference that follows its maximum in steps (it moves when a block exceeds it by
+ * 2^8), which changes rounding, not the softmax.  Both products run as tcgen05.mma with scores and output in tensor
+ * memory (CTA pairs at d_head 256); KVD_ERR_TIMEOUT from kvd_poll_status if an in-kernel wait ran out.
  * A row's result depends on that row, its position and the keys alone -- not on n_rows, on the row's index or on the
  * other rows of the call -- so a token attended alone and the same token inside a long call give the same bits.
  * They are NOT the bits of kvd_decode_attention / kvd_decode_attention_rows (another split of the keys): same
