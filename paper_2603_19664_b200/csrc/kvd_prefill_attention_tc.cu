@@ -10,9 +10,10 @@
 //           pair can see to the last one.
 //   TMEM  = [ O : d_head columns | S_0, S_1 : 64 columns each | Q : d_head / 2 columns ].  The query tile is written
 //           there once (two elements per 32-bit column) and is the A operand of S_j = Q K_j^T; the softmax threads
-//           read S_j (one row per thread, no shuffles) and hand its columns back at once; the weights P_j go to
-//           shared memory in the element type as the A operand of O += P_j V_j (tensor memory has no room for them
-//           beside two score buffers at d_head = 256, and scores that are free early let S run two blocks ahead).
+//           read S_j (one row per thread, no shuffles) and hand its columns back at once (scores that are free early
+//           let S run two blocks ahead); the weights P_j, in the element type, are the A operand of O += P_j V_j --
+//           from 2 x 32 more columns of tensor memory for d_head <= 128, from shared memory at 256, where tensor
+//           memory is full.
 //   warps = 0-7 softmax and epilogue (two groups of four, TMEM lane quarter = warp % 4, alternating blocks), 8 issues
 //           the S products, 9 the PV products (in the pair's leading CTA only), 10-13 gather K/V blocks from the
 //           segments with 16-byte cp.async into the 128-byte-swizzled layouts the two products expect (K block:
@@ -61,9 +62,11 @@ struct PtCfg {
   static constexpr int SLOTS_V = D_HEAD == 256 ? (PAIR ? 4 : 2) : (PAIR ? 6 : 4);  // blocks in the V ring
   static constexpr int SLOTS = SLOTS_K + SLOTS_V;
   static constexpr int COL_O = 0, COL_S = D_HEAD, COL_Q = D_HEAD + 2 * PT_KEYS;
-  static constexpr int COLS_USED = COL_Q + D_HEAD / 2;
+  static constexpr bool P_TMEM = D_HEAD <= 128;                   // room for the weights in tensor memory as well
+  static constexpr int COL_P = COL_Q + D_HEAD / 2;                // two blocks of weights, 32 columns each (P_TMEM)
+  static constexpr int COLS_USED = COL_P + (P_TMEM ? PT_KEYS : 0);
   static constexpr int COLS = COLS_USED <= 256 ? 256 : 512;       // allocation: a power of two
-  static constexpr int P_BYTES = PT_ROWS * PT_KEYS * 2;           // one block of weights (K-major A operand of PV)
+  static constexpr int P_BYTES = P_TMEM ? 0 : PT_ROWS * PT_KEYS * 2;  // one block of weights in shared memory otherwise
   static constexpr int N_BARS = 2 * SLOTS + 22;
   static constexpr int SMEM_BYTES = 1024 + SLOTS * TILE_BYTES + 2 * P_BYTES + N_BARS * 8;
 };
@@ -329,7 +332,9 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
         ok = false;
         break;
       }
-      {
+      if constexpr (Cfg::P_TMEM) {
+        tmem_st_x32(tmem_base + lane_field + Cfg::COL_P + buf * (PT_KEYS / 2), w);
+      } else {
         const uint32_t prow = p_smem + buf * Cfg::P_BYTES + row * 128;
 #pragma unroll
         for (int i = 0; i < 8; ++i)
@@ -355,6 +360,9 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
           for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
           tmem_st_x32(tmem_base + lane_field + Cfg::COL_O + c * 32, r);
         }
+        tmem_wait_st();
+        tc_fence_before();
+      } else if constexpr (Cfg::P_TMEM) {
         tmem_wait_st();
         tc_fence_before();
       }
@@ -464,12 +472,18 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
         tc_fence_after();
         const uint64_t desc0 = umma_smem_desc_sw128_mn(ring_v + slot * Cfg::TILE_BYTES, Cfg::SLAB_V);
         const uint64_t pdesc0 = umma_smem_desc_sw128(p_smem + (j & 1) * Cfg::P_BYTES);
+        const uint32_t ptmem = tmem_base + Cfg::COL_P + (j & 1) * (PT_KEYS / 2);
 #pragma unroll
         for (int ks = 0; ks < PT_KEYS / 16; ++ks) {
-          if constexpr (PAIR) umma_bf16_pair(tmem_base + Cfg::COL_O, pdesc0 + ((ks * 32) >> 4), desc0 + ((ks * 16 * 128) >> 4), IDESC_O,
-                                             (j > 0 || ks > 0) ? 1u : 0u);
-          else umma_bf16(tmem_base + Cfg::COL_O, pdesc0 + ((ks * 32) >> 4), desc0 + ((ks * 16 * 128) >> 4), IDESC_O,
-                         (j > 0 || ks > 0) ? 1u : 0u);
+          const uint64_t vdesc = desc0 + ((ks * 16 * 128) >> 4);
+          const uint32_t acc = (j > 0 || ks > 0) ? 1u : 0u;
+          if constexpr (Cfg::P_TMEM) {
+            if constexpr (PAIR) umma_f16_ts_pair(tmem_base + Cfg::COL_O, ptmem + ks * 8, vdesc, IDESC_O, acc);
+            else umma_f16_ts(tmem_base + Cfg::COL_O, ptmem + ks * 8, vdesc, IDESC_O, acc);
+          } else {
+            if constexpr (PAIR) umma_bf16_pair(tmem_base + Cfg::COL_O, pdesc0 + ((ks * 32) >> 4), vdesc, IDESC_O, acc);
+            else umma_bf16(tmem_base + Cfg::COL_O, pdesc0 + ((ks * 32) >> 4), vdesc, IDESC_O, acc);
+          }
         }
         commit(bar_empty(1, slot));
         commit(bar_pv_done(j & 1));
