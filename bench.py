@@ -851,6 +851,28 @@ def measure_stack_decode(batches, n_check_steps=4, session_turns=20, session_gen
         del m
         torch.cuda.empty_cache()
         rows.append(rec)
+    # ---- prefill of a whole segment through the stack: STORE_RESIDUAL and K/V of every layer, attention of all tokens
+    # to themselves in one tcgen05 launch per layer (kvd_prefill_attention), the block's products at M = segment length
+    from stack_harness import GpuStack
+    from kvd_synth import make_token_ids
+    prefill = []
+    for U in (2048, 8192):
+        g = GpuStack(stack, w, policy="full", max_tokens=U + 8, device_weights=True, tiled_attention=True)
+        toks = make_token_ids(U, stack.vocab, seed=11).tolist()
+        g.prefill(toks)  # warm-up at full size: first launches of every kernel, the allocator's blocks
+        g.ctx.kvd_reset_sequence(0)
+        g.t = 0
+        torch.cuda.synchronize()
+        l0, t0 = g.ctx.kvd_launch_count(), time.perf_counter()
+        g.prefill(toks)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        assert g.ctx.kvd_poll_status() == 0
+        prefill.append({"tokens": U, "ms": dt * 1e3, "tokens_per_s": U / dt, "kernel_launches": int(g.ctx.kvd_launch_count() - l0),
+                        "timing": "host clock around the eager launches and a synchronize"})
+        g.ctx.close()
+        del g
+        torch.cuda.empty_cache()
     t_session = time.perf_counter()
     recs, ok = run_session(stack, w, session_turns, session_gen, window, seg[0], seg[1],
                            session_turns * (seg[1] + session_gen) + 8)
@@ -865,7 +887,7 @@ def measure_stack_decode(batches, n_check_steps=4, session_turns=20, session_gen
                "last_turn_seconds_kvdirect": recs[-1]["seconds_kvdirect"],
                "wall_seconds_both_arms": time.perf_counter() - t_session,
                "note": "config 5 of BASELINE.json on the full-size stack; python tests/session_config5.py prints it per turn"}
-    return {"config3_gemma3_4b_stack_ctx2048_window256": rows, "config5_session": session,
+    return {"config3_gemma3_4b_stack_ctx2048_window256": rows, "stack_prefill": prefill, "config5_session": session,
             "note": "34 layers, every launch measured (CUDA graph of one whole decode step, 10 replays); "
                     "scaffold = the block's other products and small steps on the library's own kernels"}
 
