@@ -184,3 +184,23 @@ def test_fp16_prefill_attention_follows_the_oracle(shape):
                                             shape.sliding_window) for i in sample])
     attn_check(out[torch.tensor(sample).cuda()].double().cpu().numpy(), ref)
     ctx.close()
+
+
+def test_full_size_call_of_the_benchmark_on_sampled_rows():
+    """The launch `bench.py` times (key prefill_attention): 16384 tokens of the Gemma-shaped global layer attending to
+    themselves, 256 tiles in 128 CTA pairs per KV head.  Rows sampled across the call -- first and last rows of tiles,
+    of pairs, of the call -- against the fp64 oracle called for each row alone."""
+    shape = GEMMA3_4B_GLOBAL
+    T = 16384
+    ctx, _ = open_layer(shape, max_tokens=T + 8)
+    kdim = shape.n_kv_heads * shape.d_head
+    K, V = make_kv(shape, T, seed=61)
+    q_bits = make_query(shape, T, seed=62)
+    q_pos = np.arange(T)
+    out = torch.zeros((T, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda")
+    ctx.kvd_prefill_attention(0, T, dev(q_bits), torch.from_numpy(q_pos.astype(np.int32)).cuda(), [(dev(K), dev(V), kdim, 0, T)], 0.0, out)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    rng = np.random.default_rng(63)
+    sample = sorted(set([0, 63, 64, 127, 128, 8191, 8192, T - 129, T - 128, T - 65, T - 64, T - 1] + rng.choice(T, 12, replace=False).tolist()))
+    attn_check(host_f64(out[torch.tensor(sample).cuda()]), oracle_rows(shape, q_bits, q_pos, [(K, V, 0)], sample))
+    ctx.close()
