@@ -493,7 +493,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
     }
   } else {
     // ------------------------------------------------------------------ K/V blocks into the rings
-    // issue order = the order the products want them, the keys two blocks ahead: K_0 K_1 | K_2 V_0 | K_3 V_1 | ...
+    // issue order = the order the products want them, the keys three blocks ahead: K_0 K_1 K_2 | K_3 V_0 | K_4 V_1 | ...
     // This CTA's share of a block: K_ROWS keys of all channels (K), all 64 keys of V_COLS channels (V).
     const int ptid = tid - 10 * 32;
     // blocks issued and not yet published to the MMA threads, oldest first.  A block is published once PT_LAG younger
@@ -588,8 +588,9 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
     if (n_blk > 0) {
       ok = emit(0, 0);
       if (ok && n_blk > 1) ok = emit(0, 1);
+      if (ok && n_blk > 2) ok = emit(0, 2);
       for (int j = 0; ok && j < n_blk; ++j) {
-        if (j + 2 < n_blk) ok = emit(0, j + 2);
+        if (j + 3 < n_blk) ok = emit(0, j + 3);
         if (ok) ok = emit(1, j);
       }
       if (ok) publish_all();
