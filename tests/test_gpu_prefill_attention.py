@@ -204,3 +204,25 @@ def test_full_size_call_of_the_benchmark_on_sampled_rows():
     sample = sorted(set([0, 63, 64, 127, 128, 8191, 8192, T - 129, T - 128, T - 65, T - 64, T - 1] + rng.choice(T, 12, replace=False).tolist()))
     attn_check(host_f64(out[torch.tensor(sample).cuda()]), oracle_rows(shape, q_bits, q_pos, [(K, V, 0)], sample))
     ctx.close()
+
+
+@pytest.mark.parametrize("shape", [GEMMA3_4B_GLOBAL, QWEN3_4B, SMOLLM2_135M], ids=lambda s: s.name)
+def test_no_keys_at_all_gives_zeros_and_an_empty_call_is_accepted(shape):
+    ctx, _ = open_layer(shape, max_tokens=256)
+    kdim = shape.n_kv_heads * shape.d_head
+    n = 70
+    q = dev(make_query(shape, n, seed=5))
+    qp = torch.arange(n, dtype=torch.int32, device="cuda")
+    out = torch.full((n, shape.n_q_heads, shape.d_head), 3.0, dtype=torch.bfloat16, device="cuda")
+    ctx.kvd_prefill_attention(0, n, q, qp, [], 0.0, out)                       # no segment
+    assert torch.all(out == 0)
+    K, V = make_kv(shape, 8, seed=6)
+    out.fill_(3.0)
+    ctx.kvd_prefill_attention(0, n, q, qp, [(dev(K), dev(V), kdim, 100, 0)], 0.0, out)   # a segment of length zero
+    assert torch.all(out == 0)
+    out.fill_(3.0)
+    ctx.kvd_prefill_attention(0, n, q, qp, [(dev(K), dev(V), kdim, 100, 8)], 0.0, out)   # every key lies after every row
+    assert torch.all(out == 0)
+    ctx.kvd_prefill_attention(0, 0, q, qp, [], 0.0, out)                       # nothing to do
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    ctx.close()
