@@ -71,23 +71,25 @@ struct PtCfg {
   static constexpr int SMEM_BYTES = 1024 + SLOTS * TILE_BYTES + 2 * P_BYTES + N_BARS * 8;
 };
 
-// A wait of the MMA threads: in a pair the arrivals may come from the partner CTA and publish what its threads wrote
-// to its own shared memory, so the acquire is at cluster scope.
+// A wait of the MMA and loader threads.  They share their SM sub-partitions with the softmax warps and wait for most of
+// a key block's time: a short sleep between polls leaves the issue slots to the warps that compute (+2 %).  In a pair
+// the arrivals may come from the partner CTA and publish what its threads wrote to its own shared memory, so the
+// acquire is at cluster scope there.
+template <bool CLUSTER>
+__device__ __forceinline__ bool polite_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag, unsigned long long timeout_ns) {
+  auto done = [&]() { return CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
+  if (done()) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  uint32_t it = 0;
+  while (!done()) {
+    __nanosleep(20);
+    if (((++it) & 31u) == 0u && (*abort_flag != 0 || globaltimer_ns() - t0 > timeout_ns)) return false;
+  }
+  return true;
+}
 template <bool PAIR>
 __device__ __forceinline__ bool lead_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag, unsigned long long timeout_ns) {
-  if constexpr (!PAIR) {
-    return mbar_wait(bar, parity, abort_flag, timeout_ns);
-  } else {
-#pragma unroll 1
-    for (int i = 0; i < 16; ++i)
-      if (mbar_try_wait_cluster(bar, parity)) return true;
-    const unsigned long long t0 = globaltimer_ns();
-    uint32_t it = 0;
-    while (!mbar_try_wait_cluster(bar, parity)) {
-      if (((++it) & 31u) == 0u && (*abort_flag != 0 || globaltimer_ns() - t0 > timeout_ns)) return false;
-    }
-    return true;
-  }
+  return polite_wait<PAIR>(bar, parity, abort_flag, timeout_ns);
 }
 
 template <int D_HEAD, int G, int DT, bool PAIR>
@@ -558,7 +560,9 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
         free_now = __shfl_sync(0xffffffffu, free_now, 0);
         if (!free_now) {
           publish_all();
-          if (!warp_wait(bar_empty(is_v, slot), par, s_abort, tmo, lane)) return false;
+          int got = lane == 0 ? (polite_wait<false>(bar_empty(is_v, slot), par, s_abort, tmo) ? 1 : 0) : 0;
+          got = __shfl_sync(0xffffffffu, got, 0);
+          if (!got) return false;
         }
       }
       const int pos0 = (blk0 + j) * PT_KEYS;
