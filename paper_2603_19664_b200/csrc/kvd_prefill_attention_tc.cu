@@ -71,8 +71,9 @@ struct PtCfg {
   static constexpr int SMEM_BYTES = 1024 + SLOTS * TILE_BYTES + 2 * P_BYTES + N_BARS * 8;
 };
 
-// A wait of the MMA and loader threads.  They share their SM sub-partitions with the softmax warps and wait for most of
-// a key block's time: a short sleep between polls leaves the issue slots to the warps that compute (+2 %).  In a pair
+// A wait of this kernel.  Every SM sub-partition hosts a warp of either softmax group, a loader warp and possibly an MMA
+// thread, and at any time some of them wait: a short sleep between polls leaves the issue slots to the warps that
+// compute (+2 to 7 %).  In a pair
 // the arrivals may come from the partner CTA and publish what its threads wrote to its own shared memory, so the
 // acquire is at cluster scope there.
 template <bool CLUSTER>
@@ -86,6 +87,13 @@ __device__ __forceinline__ bool polite_wait(uint32_t bar, uint32_t parity, const
     if (((++it) & 31u) == 0u && (*abort_flag != 0 || globaltimer_ns() - t0 > timeout_ns)) return false;
   }
   return true;
+}
+// The same for a whole warp: lane 0 waits, the result is broadcast.
+__device__ __forceinline__ bool polite_warp_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag, unsigned long long timeout_ns, int lane) {
+  int ok = 1;
+  if (lane == 0) ok = polite_wait<false>(bar, parity, abort_flag, timeout_ns) ? 1 : 0;
+  ok = __shfl_sync(0xffffffffu, ok, 0);
+  return ok != 0;
 }
 template <bool PAIR>
 __device__ __forceinline__ bool lead_wait(uint32_t bar, uint32_t parity, const volatile int *abort_flag, unsigned long long timeout_ns) {
@@ -229,7 +237,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
     const int buf = wg;
     for (int j = wg; j < n_blk; j += 2) {
       const uint32_t ph = (j >> 1) & 1;
-      if (!warp_wait(bar_s_full(buf), ph, s_abort, tmo, lane)) {
+      if (!polite_warp_wait(bar_s_full(buf), ph, s_abort, tmo, lane)) {
         raise(P.status, STATUS_TIMEOUT, s_abort);
         ok = false;
         break;
@@ -285,7 +293,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       // the row's maximum after block j - 1 comes from the other group; the one after block j goes back to it
       float m_prev = -CUDART_INF_F;
       if (j > 0) {
-        if (!warp_wait(bar_m(wg ^ 1, q4), ((j - 1) >> 1) & 1, s_abort, tmo, lane)) {
+        if (!polite_warp_wait(bar_m(wg ^ 1, q4), ((j - 1) >> 1) & 1, s_abort, tmo, lane)) {
           raise(P.status, STATUS_TIMEOUT, s_abort);
           ok = false;
           break;
@@ -329,7 +337,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       }
       // P_j into shared memory as a K-major A operand (row = MMA row, 128 bytes = 64 keys, 128-byte swizzle); the
       // product that read this buffer two blocks ago has long finished
-      if (j >= 2 && !warp_wait(bar_pv_done(buf), ((j - 2) >> 1) & 1, s_abort, tmo, lane)) {
+      if (j >= 2 && !polite_warp_wait(bar_pv_done(buf), ((j - 2) >> 1) & 1, s_abort, tmo, lane)) {
         raise(P.status, STATUS_TIMEOUT, s_abort);
         ok = false;
         break;
@@ -347,7 +355,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       }
       if (__any_sync(0xffffffffu, alpha != 1.0f)) {
         // O holds the blocks before j; the last of those products must have finished (j >= 1 here: a maximum exists)
-        if (!warp_wait(bar_pv_done(buf ^ 1), ((j - 1) >> 1) & 1, s_abort, tmo, lane)) {
+        if (!polite_warp_wait(bar_pv_done(buf ^ 1), ((j - 1) >> 1) & 1, s_abort, tmo, lane)) {
           raise(P.status, STATUS_TIMEOUT, s_abort);
           ok = false;
           break;
@@ -377,7 +385,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       const int last = n_blk - 1;
       float m_fin = m_own;
       if ((last & 1) != wg) {
-        if (!warp_wait(bar_m(wg ^ 1, q4), (last >> 1) & 1, s_abort, tmo, lane)) {
+        if (!polite_warp_wait(bar_m(wg ^ 1, q4), (last >> 1) & 1, s_abort, tmo, lane)) {
           raise(P.status, STATUS_TIMEOUT, s_abort);
           ok = false;
         }
@@ -392,7 +400,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
         s_lx[wg][row] = mine;
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_l(q4));
-        if (!warp_wait(bar_l(q4), 0, s_abort, tmo, lane)) {
+        if (!polite_warp_wait(bar_l(q4), 0, s_abort, tmo, lane)) {
           raise(P.status, STATUS_TIMEOUT, s_abort);
           ok = false;
         }
@@ -400,7 +408,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
       }
     }
     // ---- normalise and store, each group its half of the channels (a token without a visible key yields zeros)
-    if (ok && n_blk > 0 && !warp_wait(bar_o_full, 0, s_abort, tmo, lane)) {
+    if (ok && n_blk > 0 && !polite_warp_wait(bar_o_full, 0, s_abort, tmo, lane)) {
       raise(P.status, STATUS_TIMEOUT, s_abort);
       ok = false;
     }
