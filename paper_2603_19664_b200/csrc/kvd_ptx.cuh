@@ -65,6 +65,7 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
   uint32_t it = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
+    __nanosleep(20);  // the warps that share this SM sub-partition and compute get the issue slots
     if (((++it) & 31u) == 0u) {
       if (*abort_flag != 0) return false;
       if (globaltimer_ns() - t0 > timeout_ns) return false;
