@@ -130,10 +130,15 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
-  // long tiles (late tokens of a causal call) first; the CTAs of a pair have neighbouring tiles
-  const int tile = static_cast<int>(gridDim.x) - 1 - static_cast<int>(blockIdx.x);
-  const int tok0 = tile * TOK, kvh = blockIdx.y;
-  const int pair_tok0 = PAIR ? (tile & ~1) * TOK : tok0;  // the grid is even: tiles 2c and 2c + 1 share a cluster
+  // One-dimensional grid in the order the CTAs should start: long tiles (late tokens of a causal call) first, and for
+  // every tile (pair of neighbouring tiles) all KV heads before the next shorter one -- with the heads as a second grid
+  // dimension the longest tiles of the last head would start last and set the launch's length.
+  const int n_tiles = static_cast<int>(gridDim.x) / P.n_kv;        // even for pairs
+  const int slot = static_cast<int>(blockIdx.x) / NCTA;            // cluster (or CTA) in start order
+  const int kvh = slot % P.n_kv;
+  const int tile = n_tiles - 1 - ((slot / P.n_kv) * NCTA + static_cast<int>(blockIdx.x) % NCTA);
+  const int tok0 = tile * TOK;
+  const int pair_tok0 = PAIR ? (tile & ~1) * TOK : tok0;           // tiles 2c and 2c + 1 share a cluster
   const unsigned long long tmo = P.timeout_ns;
   // An arrival of one warp on a barrier of the leading CTA.  Across the pair it is a relaxed arrive: what it announces
   // (scores read out of tensor memory; weights or K/V pieces written to this CTA's own shared memory) has been
@@ -643,7 +648,7 @@ static kvd_status prefill_tc_launch(kvd_ctx *ctx, const PrefillParams &P, cudaSt
   if (PAIR) tiles = (tiles + 1) & ~1;  // whole pairs: a CTA whose tile lies past the last row has no rows to store
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3(tiles, P.n_kv, 1);
+  cfg.gridDim = dim3(tiles * P.n_kv, 1, 1);
   cfg.blockDim = dim3(PT_THREADS, 1, 1);
   cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
   cfg.stream = stream;
