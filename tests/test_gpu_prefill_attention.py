@@ -226,3 +226,25 @@ def test_no_keys_at_all_gives_zeros_and_an_empty_call_is_accepted(shape):
     ctx.kvd_prefill_attention(0, 0, q, qp, [], 0.0, out)                       # nothing to do
     assert ctx.kvd_poll_status() == kvd.KVD_OK
     ctx.close()
+
+
+@pytest.mark.parametrize("shape", [GEMMA3_4B_GLOBAL, QWEN3_4B], ids=lambda s: s.name)
+def test_repeated_launches_give_the_same_bits(shape):
+    """Nothing in the kernel depends on timing: which softmax group is ahead, when a block lands, in which order the
+    CTAs start.  Thirty launches of a 3000-token call (pairs and single CTAs, several waves) return identical bits."""
+    T = 3000
+    ctx, _ = open_layer(shape, max_tokens=T + 8)
+    kdim = shape.n_kv_heads * shape.d_head
+    K, V = make_kv(shape, T, seed=71)
+    k, v = dev(K), dev(V)
+    q = dev(make_query(shape, T, seed=72))
+    qp = torch.arange(T, dtype=torch.int32, device="cuda")
+    first = torch.zeros((T, shape.n_q_heads, shape.d_head), dtype=torch.bfloat16, device="cuda")
+    ctx.kvd_prefill_attention(0, T, q, qp, [(k, v, kdim, 0, T)], 0.0, first)
+    out = torch.zeros_like(first)
+    for _ in range(30):
+        out.fill_(1.0)
+        ctx.kvd_prefill_attention(0, T, q, qp, [(k, v, kdim, 0, T)], 0.0, out)
+        assert torch.equal(out, first)
+    assert ctx.kvd_poll_status() == kvd.KVD_OK
+    ctx.close()
