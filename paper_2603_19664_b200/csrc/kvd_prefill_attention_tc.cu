@@ -1,7 +1,7 @@
 // ATTENTION of Algorithm 1 (Eq. 6-7) for many query tokens of one sequence on the fifth-generation tensor cores.
 //
-//   CTA   = (tile of query tokens, KV head): 128 MMA rows = 128 / Gp tokens x Gp query heads of the head's group
-//           (Gp = group size rounded up to a power of two; padding heads are zero rows that are never stored).
+//   CTA   = (tile of query tokens, KV head): 128 MMA rows = 128 / G tokens x the G query heads of the head's group (for
+//           G = 3, 42 tokens and two empty rows; empty rows are zeros that are never stored).
 //   pair  = for d_head >= 128 two CTAs with neighbouring tiles of the same KV head form a cluster and run the products
 //           as tcgen05.mma.cta_group::2 (M = 256, 128 rows per CTA): a K or V block is shared by the pair, each CTA
 //           loads and holds half of it (K: half the keys, V: half the channels -- the halves the instruction reads from
@@ -103,8 +103,7 @@ __device__ __forceinline__ bool lead_wait(uint32_t bar, uint32_t parity, const v
 template <int D_HEAD, int G, int DT, bool PAIR>
 __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(const __grid_constant__ PrefillParams P) {
   using Cfg = PtCfg<D_HEAD, PAIR>;
-  constexpr int GP = G == 3 ? 4 : G;   // heads of the group, padded to a power of two
-  constexpr int TOK = PT_ROWS / GP;    // query tokens per CTA
+  constexpr int TOK = PT_ROWS / G;     // query tokens per CTA (G = 3: 42 tokens, the last two MMA rows stay empty)
   constexpr int NCTA = Cfg::NCTA;
   constexpr int SLOTS = Cfg::SLOTS, SLOTS_K = Cfg::SLOTS_K, SLOTS_V = Cfg::SLOTS_V;
   extern __shared__ uint8_t pt_smem_raw[];
@@ -208,8 +207,8 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
     // through shared memory; every group keeps its own part of the row sum.
     const int wg = warp >> 2, q4 = warp & 3;
     const int row = q4 * 32 + lane;
-    const int tok = tok0 + row / GP, g = row % GP;
-    const bool valid = tok < P.n_rows && g < G;
+    const int tok = tok0 + row / G, g = row % G;
+    const bool valid = row / G < TOK && tok < P.n_rows;
     const int qp = valid ? P.q_pos[tok] : -1;
     const int lo = P.window > 0 ? qp - P.window + 1 : 0;
     const uint32_t lane_field = static_cast<uint32_t>(q4 * 32) << 16;
@@ -633,7 +632,6 @@ __global__ void __launch_bounds__(PT_THREADS, 1) kvd_prefill_attn_tc_kernel(cons
 template <int D_HEAD, int G, bool PAIR>
 static kvd_status prefill_tc_launch(kvd_ctx *ctx, const PrefillParams &P, cudaStream_t stream) {
   using Cfg = PtCfg<D_HEAD, PAIR>;
-  constexpr int GP = G == 3 ? 4 : G;
   auto k0 = kvd_prefill_attn_tc_kernel<D_HEAD, G, 0, PAIR>;
   auto k1 = kvd_prefill_attn_tc_kernel<D_HEAD, G, 1, PAIR>;
   static bool configured[64] = {};
@@ -643,7 +641,7 @@ static kvd_status prefill_tc_launch(kvd_ctx *ctx, const PrefillParams &P, cudaSt
     if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaFuncSetAttribute(prefill attention)");
     configured[ctx->device & 63] = true;
   }
-  const int tok = PT_ROWS / GP;
+  const int tok = PT_ROWS / G;
   int tiles = (P.n_rows + tok - 1) / tok;
   if (PAIR) tiles = (tiles + 1) & ~1;  // whole pairs: a CTA whose tile lies past the last row has no rows to store
   cudaLaunchConfig_t cfg;
